@@ -1,0 +1,236 @@
+"""SelectInfer oracle: TEST INFRASTRUCTURE ONLY, never a product path.
+
+Plain CPU statements of every step of the selective-computation hot path, written
+from the paper's description and independent of the CUDA library (no shared code,
+neither imports the other).  Only tests, the smoke check and the benchmark's
+cpu_baseline / reference legs may import this module.
+
+* ``ffn`` / ``ffn_tokens`` / ``ffn_dense_masked`` -- float64 selective SwiGLU FFN on the
+  full weights with global neuron ids (C loops in ``si_oracle.c``; Section 3 for the
+  neuron <-> weight-slice correspondence, Section 5 for "compute only the selected
+  loaded neurons").
+* ``select_topk`` -- Section 5: sort activations in descending order, keep the top
+  alpha, record their indices.  Tie-break (paper silent): lower index wins; +0 == -0;
+  NaN ranks below everything.  Output ascending by index.
+* ``select_threshold`` -- extension with no counterpart in the paper (brute-force
+  pinned only).
+* ``union`` -- sorted set union of per-token lists plus per-token membership bitmasks.
+* ``loadset`` -- Section 4: base = top delta of the task ranking, then the model
+  ranking in order, skipping ids already chosen, until gamma neurons are loaded.
+* ``memory_saving`` -- Eq. 2.
+* ``layer_range`` -- Table 1 "first layer 5 / last layer -2".
+
+Pins live in tests/test_oracle_pins.py.  Parity unpinned: the paper's task-accuracy
+results (they need its datasets and trained weights); nothing here computes them.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "si_oracle.c")
+_LIB = os.path.join(_HERE, "libsi_oracle.so")
+
+F64, F16, BF16 = 0, 1, 2
+_DTYPES = {"f64": F64, "f16": F16, "bf16": BF16}
+
+
+def build(force: bool = False) -> str:
+    """Compile si_oracle.c with gcc -O2 -fopenmp (no BLAS, no intrinsics)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, ip = ctypes.c_void_p, ctypes.c_int
+        lib.so_ffn.argtypes = [vp, vp, vp, ip, ip, ip, vp, vp, ip, vp, vp, ip]
+        lib.so_ffn.restype = ip
+        lib.so_ffn_dense_masked.argtypes = [vp, vp, vp, ip, ip, ip, vp, vp, vp]
+        lib.so_ffn_dense_masked.restype = ip
+        lib.so_ffn_tokens.argtypes = [vp, vp, vp, ip, ip, ip, vp, ip, vp, vp, vp, ip]
+        lib.so_ffn_tokens.restype = ip
+        _lib = lib
+    return _lib
+
+
+def _prep(a, dtype_code):
+    want = np.float64 if dtype_code == F64 else np.uint16
+    a = np.ascontiguousarray(a)
+    if a.dtype != want:
+        raise TypeError(f"expected {want} storage for dtype code {dtype_code}, got {a.dtype}")
+    return a
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def host_threads() -> int:
+    return len(os.sched_getaffinity(0))
+
+
+def ffn(Wg, Wu, Wd, x, A, dtype: str = "f64", threads: int = 1, return_h: bool = False):
+    """y[d_model] float64 = selective FFN over global neuron ids A (Sections 3, 5).
+
+    Wg, Wu: [d_ff, d_model]; Wd: [d_model, d_ff]; x: [d_model].  For dtype "f16"/"bf16"
+    the arrays hold raw uint16 bit patterns; for "f64" float64 values.
+    """
+    code = _DTYPES[dtype]
+    Wg, Wu, Wd, x = (_prep(a, code) for a in (Wg, Wu, Wd, x))
+    d_ff, d_model = Wg.shape
+    assert Wu.shape == (d_ff, d_model) and Wd.shape == (d_model, d_ff) and x.shape == (d_model,)
+    A = np.ascontiguousarray(A, dtype=np.int32)
+    y = np.empty(d_model, dtype=np.float64)
+    h = np.empty(max(len(A), 1), dtype=np.float64)
+    rc = _load().so_ffn(_ptr(Wg), _ptr(Wu), _ptr(Wd), code, d_ff, d_model, _ptr(x), _ptr(A),
+                        len(A), _ptr(y), _ptr(h), threads)
+    if rc:
+        raise ValueError("neuron ids must be distinct and in [0, d_ff)")
+    return (y, h[: len(A)]) if return_h else y
+
+
+def ffn_dense_masked(Wg, Wu, Wd, x, keep, dtype: str = "f64"):
+    """Dense FFN over all neurons with h_i zeroed where keep[i] == 0 (brute force)."""
+    code = _DTYPES[dtype]
+    Wg, Wu, Wd, x = (_prep(a, code) for a in (Wg, Wu, Wd, x))
+    d_ff, d_model = Wg.shape
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    assert keep.shape == (d_ff,)
+    y = np.empty(d_model, dtype=np.float64)
+    _load().so_ffn_dense_masked(_ptr(Wg), _ptr(Wu), _ptr(Wd), code, d_ff, d_model, _ptr(x),
+                                _ptr(keep), _ptr(y))
+    return y
+
+
+def ffn_tokens(Wg, Wu, Wd, X, lists, dtype: str = "f64", threads: int = 1):
+    """Y[T, d_model]: token t uses exactly lists[t] (masked-union semantics)."""
+    code = _DTYPES[dtype]
+    Wg, Wu, Wd, X = (_prep(a, code) for a in (Wg, Wu, Wd, X))
+    d_ff, d_model = Wg.shape
+    T = X.shape[0]
+    assert X.shape == (T, d_model) and len(lists) == T
+    offsets = np.zeros(T + 1, dtype=np.int32)
+    offsets[1:] = np.cumsum([len(l) for l in lists])
+    flat = (np.concatenate([np.asarray(l, dtype=np.int32) for l in lists])
+            if offsets[-1] else np.zeros(1, dtype=np.int32))
+    flat = np.ascontiguousarray(flat, dtype=np.int32)
+    Y = np.empty((T, d_model), dtype=np.float64)
+    rc = _load().so_ffn_tokens(_ptr(Wg), _ptr(Wu), _ptr(Wd), code, d_ff, d_model, _ptr(X), T,
+                               _ptr(flat), _ptr(offsets), _ptr(Y), threads)
+    if rc:
+        raise ValueError("neuron ids must be distinct and in [0, d_ff)")
+    return Y
+
+
+# --------------------------------------------------------------------------- selection
+
+def _rank_order(scores: np.ndarray, use_abs: bool):
+    """Indices ordered by (score descending, index ascending); NaN last; +0 == -0."""
+    s = np.asarray(scores, dtype=np.float32)
+    if use_abs:
+        s = np.abs(s)
+    order = []
+    for i, v in enumerate(s.tolist()):       # python floats: exact images of the float32s
+        is_nan = v != v
+        order.append((1 if is_nan else 0, 0.0 if is_nan else -v, i))
+    order.sort()                             # -0.0 == 0.0 compares equal, index breaks the tie
+    return [i for _, _, i in order]
+
+
+def select_topk(scores, k: int, use_abs: bool = False) -> np.ndarray:
+    """Section 5: top-k indices of the scores, returned ascending by index."""
+    n = len(scores)
+    if not 0 <= k <= n:
+        raise ValueError("k out of range")
+    chosen = _rank_order(scores, use_abs)[:k]
+    return np.array(sorted(chosen), dtype=np.int32)
+
+
+def select_threshold(scores, tau: float, use_abs: bool = False) -> np.ndarray:
+    """Extension (not in the paper): indices with score > tau, NaN excluded, ascending."""
+    s = np.asarray(scores, dtype=np.float32)
+    if use_abs:
+        s = np.abs(s)
+    tau32 = np.float32(tau)
+    return np.array([i for i, v in enumerate(s) if v > tau32], dtype=np.int32)
+
+
+def union(lists, n_loaded: int):
+    """Sorted union U of the lists, per-token bitmasks over positions in U, overlap ratios.
+
+    mask[t, p >> 5] bit (p & 31) is set iff U[p] is in lists[t].
+    overlap = 1 - |U| / sum_t |A_t|; coverage = |U| / n_loaded.
+    """
+    seen = set()
+    for l in lists:
+        seen.update(int(v) for v in l)
+    U = np.array(sorted(seen), dtype=np.int32)
+    pos = {int(v): p for p, v in enumerate(U)}
+    words = (len(U) + 31) // 32
+    mask = np.zeros((len(lists), max(words, 1)), dtype=np.uint32)
+    total = 0
+    for t, l in enumerate(lists):
+        for v in l:
+            p = pos[int(v)]
+            mask[t, p >> 5] |= np.uint32(1 << (p & 31))
+            total += 1
+    overlap = 1.0 - len(U) / total if total else 0.0
+    return U, mask[:, :words], overlap, len(U) / n_loaded
+
+
+def loadset(task_rank, model_rank, n_base: int, n_loaded: int) -> np.ndarray:
+    """Section 4: base neurons first (top n_base of the task ranking), then secondary
+    neurons from the model ranking, skipping those already chosen, until n_loaded."""
+    out = [int(v) for v in task_rank[:n_base]]
+    chosen = set(out)
+    for v in model_rank:
+        if len(out) >= n_loaded:
+            break
+        v = int(v)
+        if v not in chosen:
+            chosen.add(v)
+            out.append(v)
+    if len(out) != n_loaded:
+        raise ValueError("rankings too short for n_loaded")
+    return np.array(out, dtype=np.int32)
+
+
+def memory_saving(n_ffn_params: float, r_load: float, r_layer: float, bytes_per_param: float):
+    """Eq. 2: bytes saved = N_ffn * (1 - r_load) * r_layer * s."""
+    return n_ffn_params * (1.0 - r_load) * r_layer * bytes_per_param
+
+
+def layer_range(n_layers: int, first: int = 5, last: int = -2):
+    """Table 1: selective layers = first ... n_layers + last - 1 (0-based)."""
+    return list(range(first, n_layers + last))
+
+
+def count_from_pct(pct: int, n: int) -> int:
+    """Fractions -> counts: floor(pct * n / 100) in integers."""
+    return (pct * n) // 100
+
+
+def error_metrics(y, y_ref):
+    """(max|err| / max|y_ref|, mean|err| / mean|y_ref|) for one token."""
+    y = np.asarray(y, dtype=np.float64)
+    y_ref = np.asarray(y_ref, dtype=np.float64)
+    err = np.abs(y - y_ref)
+    mx = np.max(np.abs(y_ref))
+    mn = np.mean(np.abs(y_ref))
+    return (float(np.max(err) / mx) if mx > 0 else float(np.max(err)),
+            float(np.mean(err) / mn) if mn > 0 else float(np.mean(err)))

@@ -1,0 +1,278 @@
+"""Pins for the CPU oracle: it is checked against things other than itself before
+anything is compared with it -- library float64 routines, closed forms with printed
+constants, algebraic invariants, brute force on tiny inputs, and values the paper prints."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import selectinfer_oracle as so
+from paper_2607_18081_b200 import workloads as wl
+from tests.helpers import paper_values
+
+
+def _rand_problem(seed, d_ff=24, d_model=16, scale=0.5):
+    g = np.random.default_rng(seed)
+    Wg = g.normal(0, scale, (d_ff, d_model))
+    Wu = g.normal(0, scale, (d_ff, d_model))
+    Wd = g.normal(0, scale, (d_model, d_ff))
+    x = g.normal(0, 1, d_model)
+    return Wg, Wu, Wd, x
+
+
+# ------------------------------------------------------------------ O-FFN
+
+def test_all_neurons_equals_library_dense_swiglu():
+    """A = every neuron must be the textbook SwiGLU FFN, evaluated by a float64 library."""
+    Wg, Wu, Wd, x = _rand_problem(1, d_ff=96, d_model=64)
+    y = so.ffn(Wg, Wu, Wd, x, np.arange(96))
+    tWg, tWu, tWd, tx = (torch.from_numpy(a) for a in (Wg, Wu, Wd, x))
+    F = torch.nn.functional
+    ref = F.linear(F.silu(F.linear(tx, tWg)) * F.linear(tx, tWu), tWd).numpy()
+    np.testing.assert_allclose(y, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_subset_equals_library_masked_dense():
+    """Selective FFN == dense FFN with the unselected activations zeroed (library route)."""
+    Wg, Wu, Wd, x = _rand_problem(2, d_ff=96, d_model=64)
+    A = np.array([3, 95, 17, 0, 44, 45, 46, 80])
+    y = so.ffn(Wg, Wu, Wd, x, A)
+    tWg, tWu, tWd, tx = (torch.from_numpy(a) for a in (Wg, Wu, Wd, x))
+    F = torch.nn.functional
+    h = F.silu(F.linear(tx, tWg)) * F.linear(tx, tWu)
+    keep = torch.zeros(96, dtype=torch.float64)
+    keep[torch.from_numpy(A)] = 1
+    ref = F.linear(h * keep, tWd).numpy()
+    np.testing.assert_allclose(y, ref, rtol=1e-12, atol=1e-13)
+    # a transposed W_down or swapped gate/up must fail: check they really differ
+    wrong = F.linear(F.silu(F.linear(tx, tWu)) * F.linear(tx, tWg) * keep, tWd).numpy()
+    assert np.max(np.abs(wrong - ref)) > 1e-3
+
+
+@pytest.mark.parametrize("seed", [3, 4, 5])
+def test_mask_dense_identity_is_exact(seed):
+    """Brute force over all neurons with unselected h forced to 0: bit-for-bit equal."""
+    Wg, Wu, Wd, x = _rand_problem(seed, d_ff=40, d_model=24)
+    g = np.random.default_rng(seed + 100)
+    A = g.permutation(40)[: 13]
+    keep = np.zeros(40, dtype=np.uint8)
+    keep[A] = 1
+    y = so.ffn(Wg, Wu, Wd, x, A)
+    yb = so.ffn_dense_masked(Wg, Wu, Wd, x, keep)
+    assert np.array_equal(y, yb)
+    # all neurons selected == dense brute force, exactly
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, x, np.arange(40)),
+                          so.ffn_dense_masked(Wg, Wu, Wd, x, np.ones(40, np.uint8)))
+
+
+def test_closed_form_one_hot_neurons():
+    """Wg[i]=e_a, Wu[i]=e_b, Wd[:,i]=e_c  =>  y_c = SiLU(x_a) * x_b, with printed SiLU values."""
+    silu = {1.0: 0.7310585786300049, -1.0: -0.2689414213699951, 2.0: 1.7615941559557646}
+    d_ff, d_model = 6, 5
+    for xa, expect in silu.items():
+        Wg = np.zeros((d_ff, d_model)); Wu = np.zeros((d_ff, d_model)); Wd = np.zeros((d_model, d_ff))
+        a, b, c, i = 1, 3, 4, 2
+        Wg[i, a] = 1; Wu[i, b] = 1; Wd[c, i] = 1
+        x = np.array([9.0, xa, 7.0, 3.0, -5.0])
+        y = so.ffn(Wg, Wu, Wd, x, [i])
+        want = np.zeros(d_model); want[c] = expect * 3.0
+        np.testing.assert_allclose(y, want, rtol=1e-15, atol=0)
+        # the neuron not being selected gives exactly zero
+        assert np.array_equal(so.ffn(Wg, Wu, Wd, x, [0, 1, 3]), np.zeros(d_model))
+    # independent evaluation of SiLU via math.exp for an odd value
+    Wg = np.zeros((2, 2)); Wu = np.zeros((2, 2)); Wd = np.zeros((2, 2))
+    Wg[1, 0] = 0.5; Wu[1, 1] = -2.0; Wd[0, 1] = 4.0
+    x = np.array([3.0, 0.25])
+    g, u = 1.5, -0.5
+    want0 = g / (1 + math.exp(-g)) * u * 4.0
+    y = so.ffn(Wg, Wu, Wd, x, [1])
+    assert y[0] == pytest.approx(want0, rel=1e-15) and y[1] == 0.0
+
+
+def test_zero_input_and_empty_list():
+    Wg, Wu, Wd, x = _rand_problem(6)
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, np.zeros_like(x), np.arange(24)), np.zeros(16))
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, x, []), np.zeros(16))
+
+
+def test_additivity_and_order_invariance():
+    Wg, Wu, Wd, x = _rand_problem(7, d_ff=60, d_model=32)
+    g = np.random.default_rng(70)
+    p = g.permutation(60)
+    A, B = p[:20], p[20:45]
+    yA, yB = so.ffn(Wg, Wu, Wd, x, A), so.ffn(Wg, Wu, Wd, x, B)
+    yAB = so.ffn(Wg, Wu, Wd, x, np.concatenate([A, B]))
+    np.testing.assert_allclose(yA + yB, yAB, rtol=1e-12, atol=1e-14)
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, x, A), so.ffn(Wg, Wu, Wd, x, A[::-1].copy()))
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, x, A), so.ffn(Wg, Wu, Wd, x, np.sort(A)))
+
+
+def test_activation_matches_library_per_neuron():
+    """h_i returned by the oracle is SiLU(g_i) * u_i of a float64 library evaluation."""
+    Wg, Wu, Wd, x = _rand_problem(8, d_ff=50, d_model=20)
+    A = np.array([49, 1, 7, 30])
+    _, h = so.ffn(Wg, Wu, Wd, x, A, return_h=True)
+    gg = torch.from_numpy(Wg) @ torch.from_numpy(x)
+    uu = torch.from_numpy(Wu) @ torch.from_numpy(x)
+    ref = (torch.nn.functional.silu(gg) * uu).numpy()[np.sort(A)]
+    np.testing.assert_allclose(h, ref, rtol=1e-12)
+
+
+def test_bad_lists_rejected():
+    Wg, Wu, Wd, x = _rand_problem(9)
+    with pytest.raises(ValueError):
+        so.ffn(Wg, Wu, Wd, x, [1, 1])
+    with pytest.raises(ValueError):
+        so.ffn(Wg, Wu, Wd, x, [24])
+    with pytest.raises(ValueError):
+        so.ffn(Wg, Wu, Wd, x, [-1])
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_16bit_widening_is_exact(dtype):
+    """Bit patterns go through the oracle's own widening; numpy/torch widen them independently."""
+    g = np.random.default_rng(10)
+    d_ff, d_model = 32, 24
+    mk = lambda shape, s: wl.float_to_bits(g.normal(0, s, shape).astype(np.float32), dtype)
+    Wg, Wu, Wd, x = mk((d_ff, d_model), 0.3), mk((d_ff, d_model), 0.3), mk((d_model, d_ff), 0.3), mk((d_model,), 1)
+    # include subnormal / tiny / large values in the fp16 case
+    if dtype == "f16":
+        Wg[0, :4] = np.array([0x0001, 0x03FF, 0x8001, 0x7BFF], dtype=np.uint16)
+        x[:4] = np.array([0x3C00, 0x3C00, 0x3C00, 0x0400], dtype=np.uint16)
+    A = np.arange(0, d_ff, 3)
+    y = so.ffn(Wg, Wu, Wd, x, A, dtype=dtype)
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    widen = lambda a: torch.from_numpy(a.view(np.int16)).view(tdt).to(torch.float64).numpy()
+    y64 = so.ffn(widen(Wg), widen(Wu), widen(Wd), widen(x), A, dtype="f64")
+    assert np.array_equal(y, y64)
+    np.testing.assert_array_equal(widen(Wg), wl.bits_to_float64(Wg, dtype))
+
+
+def test_threads_do_not_change_bits():
+    Wg, Wu, Wd, x = _rand_problem(11, d_ff=200, d_model=48)
+    A = np.arange(0, 200, 2)
+    assert np.array_equal(so.ffn(Wg, Wu, Wd, x, A, threads=1), so.ffn(Wg, Wu, Wd, x, A, threads=4))
+
+
+def test_tokens_are_independent_masked_union():
+    Wg, Wu, Wd, _ = _rand_problem(12, d_ff=30, d_model=12)
+    X = np.random.default_rng(13).normal(0, 1, (3, 12))
+    lists = [[0, 5, 9], [], [29, 5, 1, 2]]
+    Y = so.ffn_tokens(Wg, Wu, Wd, X, lists)
+    for t in range(3):
+        assert np.array_equal(Y[t], so.ffn(Wg, Wu, Wd, X[t], lists[t]))
+
+
+# ------------------------------------------------------------------ O-SELECT
+
+def _brute_topk(scores, k):
+    """All k-subsets on tiny n: the unique subset consistent with (score desc, index asc)."""
+    s = [0.0 if (v == 0) else v for v in np.asarray(scores, np.float32).tolist()]
+    n = len(s)
+    def better(i, j):
+        ni, nj = math.isnan(s[i]), math.isnan(s[j])
+        if ni or nj:                       # NaN ranks below every number; NaN vs NaN: index
+            return (not ni) or (nj and i < j)
+        return s[i] > s[j] or (s[i] == s[j] and i < j)
+    good = []
+    for sub in itertools.combinations(range(n), k):
+        inside = set(sub)
+        if all(better(i, j) for i in sub for j in range(n) if j not in inside):
+            good.append(sub)
+    assert len(good) == 1
+    return np.array(good[0], dtype=np.int32)
+
+
+@pytest.mark.parametrize("scores", [
+    [0.5, -1.0, 3.0, 3.0, 0.0, -0.0, 2.0],
+    [1.0] * 7,
+    [float("nan"), 1.0, float("-inf"), float("inf"), float("nan"), 0.0, -0.0],
+    [-3.0, -2.0, -2.0, -2.0, -1.0, -2.0, -5.0],
+    [0.0, -0.0, 0.0, -0.0, 0.0, -0.0, 1e-45],
+])
+def test_topk_against_subset_brute_force(scores):
+    for k in range(len(scores) + 1):
+        got = so.select_topk(scores, k)
+        assert np.array_equal(got, _brute_topk(scores, k)), (scores, k)
+        assert got.dtype == np.int32
+
+
+def test_topk_invariants_random_with_ties():
+    g = np.random.default_rng(21)
+    for n, k in [(50, 0), (50, 50), (257, 31), (1000, 400)]:
+        s = np.round(g.normal(0, 1, n), 1).astype(np.float32)   # many exact ties
+        sel = so.select_topk(s, k)
+        assert len(sel) == k and np.all(np.diff(sel) > 0)
+        inside = np.zeros(n, bool); inside[sel] = True
+        if 0 < k < n:
+            lo, hi = s[inside].min(), s[~inside].max()
+            assert lo >= hi
+            if lo == hi:
+                assert sel[s[sel] == lo].max() < np.nonzero(~inside & (s == lo))[0].min()
+        # library cross-check: stable descending sort
+        ref = np.sort(np.argsort(-s.astype(np.float64), kind="stable")[:k])
+        assert np.array_equal(sel, ref)
+
+
+def test_topk_abs_and_threshold():
+    s = np.array([-4.0, 1.0, 3.0, -3.0, 0.5], np.float32)
+    assert so.select_topk(s, 2, use_abs=True).tolist() == [0, 2]      # |-3| ties |3|: lower index
+    assert so.select_topk(s, 3, use_abs=True).tolist() == [0, 2, 3]
+    assert so.select_threshold(s, 0.5).tolist() == [1, 2]
+    assert so.select_threshold(s, 0.5, use_abs=True).tolist() == [0, 1, 2, 3]
+    assert so.select_threshold([float("nan"), 1.0], -10).tolist() == [1]
+
+
+# ------------------------------------------------------------------ O-UNION / O-LOADSET
+
+def test_union_brute_force():
+    g = np.random.default_rng(31)
+    lists = [np.sort(g.permutation(100)[:30]).astype(np.int32) for _ in range(5)]
+    U, mask, overlap, cover = so.union(lists, 100)
+    assert U.tolist() == sorted(set(np.concatenate(lists).tolist()))
+    assert sum(bin(int(w)).count("1") for w in mask.ravel()) == 150
+    for t, l in enumerate(lists):
+        members = [int(U[p]) for p in range(len(U)) if (int(mask[t, p >> 5]) >> (p & 31)) & 1]
+        assert members == l.tolist()
+    assert overlap == pytest.approx(1 - len(U) / 150) and cover == pytest.approx(len(U) / 100)
+
+
+def test_loadset_tiny_and_table1_arithmetic():
+    pv = paper_values()
+    # Table 1: base 30 % + secondary 40 % = loaded 70 %; static 30 % + dynamic 10 % = computed 40 %
+    assert pv["table1_base_pct"] + pv["table1_secondary_pct"] == pv["table1_loaded_pct"]
+    assert pv["table1_base_pct"] + pv["table1_dynamic_pct"] == pv["table1_computed_pct"]
+    task = [4, 2, 9, 0, 1, 3, 5, 6, 7, 8]
+    model = [2, 7, 4, 5, 0, 9, 1, 3, 6, 8]
+    got = so.loadset(task, model, n_base=3, n_loaded=7)
+    assert got.tolist() == [4, 2, 9, 7, 5, 0, 1]       # 2, 4, 9 skipped in the model ranking
+    F = 11008
+    nb, nl = so.count_from_pct(30, F), so.count_from_pct(70, F)
+    g = np.random.default_rng(41)
+    ids = so.loadset(g.permutation(F), g.permutation(F), nb, nl)
+    assert len(ids) == nl == 7705 and len(set(ids.tolist())) == nl and nb == 3302
+
+
+def test_eq2_worked_example_and_layer_range():
+    pv = paper_values()
+    saving = so.memory_saving(pv["eq2_n_ffn"], pv["eq2_r_load"], pv["eq2_r_layer"], pv["eq2_bytes_per_param"])
+    assert saving / 1e9 == pytest.approx(pv["eq2_saving_gb"], rel=1e-12)
+    orig, sel = pv["table5_llama32_3b_original_gb"], pv["table5_llama32_3b_selectinfer_gb"]
+    assert round(100 * (orig - sel) / orig, 1) == pv["table5_saving_pct"]
+    assert abs((orig - sel) - pv["eq2_saving_gb"]) < 0.05          # "aligning with the value observed"
+    first, last = int(pv["table1_first_layer"]), int(pv["table1_last_layer"])
+    assert len(so.layer_range(int(pv["llama32_1b_layers"]), first, last)) == pv["llama32_1b_selective_layers"]
+    n3b = int(pv["llama32_3b_layers"])
+    assert len(so.layer_range(n3b, first, last)) / n3b == pv["eq2_r_layer"]
+    # Llama3.2-3B FFN parameter count ~ 2.1 B (3 matrices, d_model 3072, d_ff 8192, 28 layers)
+    assert round(3 * 3072 * 8192 * 28 / 1e9, 1) == pv["eq2_n_ffn"] / 1e9
+
+
+def test_count_rounding_of_configs():
+    assert wl.CONFIGS["c1"].n_loaded == 688 and wl.CONFIGS["c1"].k_active == 172
+    assert wl.CONFIGS["c2"].n_loaded == 7705 and wl.CONFIGS["c2"].k_active == 1541
+    assert wl.CONFIGS["c4"].k_active == 3082
+    got = [[so.count_from_pct(a, so.count_from_pct(l, 14336)) for a in wl.C5_ACTIVE] for l in wl.C5_LOADED]
+    assert got == [[215, 430, 860, 2150], [358, 716, 1433, 3584], [501, 1003, 2007, 5017], [716, 1433, 2867, 7168]]
