@@ -1,0 +1,194 @@
+/*
+ * selectinfer.h -- C ABI of the B200 (sm_100a) selective-FFN library.
+ *
+ * The library implements the selective-computation hot path of SelectInfer: a
+ * compacted store holding only the loaded FFN neurons (Section 4, "Selective
+ * Loading"), the per-token SwiGLU FFN over only the selected loaded neurons
+ * (Section 5, "Selective Computation"), and the per-token top-alpha index selection
+ * used to pick them (Section 5, dynamic neuron selection).
+ *
+ * Neuron i of an FFN layer (Section 3): row i of gate_proj.weight and up_proj.weight
+ * ([d_ff, d_model], PyTorch [out, in] storage) and column i of down_proj.weight
+ * ([d_model, d_ff]).  Its activation is h_i = SiLU(w_gate_i . x) * (w_up_i . x) and
+ * its contribution to the layer output is h_i * W_down[:, i].
+ *
+ * Conventions
+ *   - Every function returns an int status: SI_OK (0) or a negative SI_ERR_* code.
+ *     Nothing throws, aborts or prints.
+ *   - "device" pointers are CUDA device pointers owned by the caller; "host" pointers
+ *     are ordinary host memory.  The library allocates no device memory: the caller
+ *     supplies the store bytes and the workspace (sizes via si_store_bytes /
+ *     si_workspace_bytes).  The only thing the library owns is the small host-side
+ *     si_store_t handle.
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it and no
+ *     call synchronises except si_store_free and si_load_neurons (which waits for the
+ *     upload of its id list).  Calls sharing one workspace must be ordered on one stream.
+ *   - Errors that can be seen on the host (null or misaligned pointers, sizes out of
+ *     range, bad enum, layer out of range, buffers too small) are reported before
+ *     anything is launched.  Errors only the device can see (an index out of range or
+ *     a duplicate under SI_FLAG_CHECK, an expired bounded wait) are written to
+ *     *status_dev (caller-owned int32 in device memory, may be NULL) as an SI_ERR_*
+ *     code; the kernel then leaves y unspecified but never reads or writes out of
+ *     bounds and never hangs.  A status word is only ever overwritten with an error,
+ *     so the caller clears it.
+ *   - All device pointers must be 16-byte aligned; d_model must be a multiple of 64.
+ *   - Active lists hold SLOT indices (positions in the layer's store), distinct.
+ *     The list order does not change the result: contributions are accumulated in a
+ *     fixed order chosen by the library, so repeated calls are bit-identical.
+ *
+ * There is no CPU fallback: every entry point that computes runs CUDA kernels.
+ */
+#ifndef SELECTINFER_H
+#define SELECTINFER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct si_store si_store_t; /* opaque host-side handle: one per model (all layers) */
+
+typedef enum { SI_F16 = 1, SI_BF16 = 2, SI_F32 = 3 /* outputs only */ } si_dtype_t;
+
+enum {
+    SI_OK = 0,
+    SI_ERR_INVALID_ARG = -1,
+    SI_ERR_OUT_OF_RANGE = -2,
+    SI_ERR_DUPLICATE = -3,
+    SI_ERR_ALIGNMENT = -4,
+    SI_ERR_NOMEM = -5,        /* caller-supplied buffer too small */
+    SI_ERR_CUDA = -6,
+    SI_ERR_TIMEOUT = -7,      /* a bounded device-side wait expired */
+    SI_ERR_UNSUPPORTED = -8
+};
+
+/* flags */
+enum {
+    SI_FLAG_CHECK = 1u,          /* validate lists on the device (range, duplicates) first */
+    SI_FLAG_RESIDUAL = 2u,       /* y = x + FFN(x) instead of FFN(x) */
+    SI_FLAG_UNION_UNMASKED = 4u, /* T > 1 only: every token uses the whole union (extension) */
+    SI_FLAG_SCORE_ABS = 8u,      /* si_select: rank |score| instead of score */
+    SI_FLAG_SIMPLE_KERNELS = 256u /* decode: one plain-load kernel pair per step instead of the
+                                     persistent bulk-copy kernel (kept for cross-checking) */
+};
+
+/* selection modes for si_select */
+enum { SI_SELECT_TOPK = 0, SI_SELECT_THRESHOLD = 1 };
+
+const char *si_strerror(int status);
+
+/* ---------------------------------------------------------------- the neuron store
+
+ * Bytes of device memory a store of n_layers layers needs; n_loaded is a host array
+ * [n_layers] with the number of loaded neurons per layer.  Per layer the store holds
+ * n_loaded records of 3 * d_model 16-bit values -- [gate row | up row | down column as
+ * a row] -- i.e. exactly the loaded slices and nothing else (Section 4; the bytes not
+ * stored are Eq. 2's saving), plus the slot <-> global id maps. */
+int si_store_bytes(int n_layers, int d_model, int d_ff, const int *n_loaded, int dtype,
+                   size_t *bytes_out);
+
+/* Creates the handle over caller-owned device memory `store_mem` (256-byte aligned,
+ * at least si_store_bytes).  Nothing is launched.  The memory must stay valid until
+ * si_store_free. */
+int si_store_create(si_store_t **store_out, void *store_mem /*device*/, size_t store_mem_bytes,
+                    int n_layers, int d_model, int d_ff, const int *n_loaded /*host [L]*/,
+                    int dtype);
+
+/* Waits for the device to go idle and frees the handle (not the device memory). */
+int si_store_free(si_store_t *store);
+
+/* Selective loading of one layer (Section 4): gathers the slices of the listed neurons
+ * out of the full weights into the layer's records.
+ *   w_gate, w_up : device, [d_ff, d_model] row-major, store dtype
+ *   w_down       : device, [d_model, d_ff] row-major, store dtype
+ *   neuron_ids   : HOST int32 [n_loaded], global neuron ids, distinct, each in
+ *                  [0, d_ff): the n_base base (task-specific) neurons first, then the
+ *                  secondary (model-specific) ones; slot s holds neuron_ids[s].
+ *   n_loaded     : must equal the count given to si_store_create for this layer.
+ * Errors: SI_ERR_OUT_OF_RANGE / SI_ERR_DUPLICATE for bad ids (nothing is launched). */
+int si_load_neurons(si_store_t *store, int layer, const void *w_gate, const void *w_up,
+                    const void *w_down, const int32_t *neuron_ids, int n_loaded, int n_base,
+                    void *stream);
+
+/* Read-only views into the store (device pointers, valid while the store lives). */
+int si_store_slot_to_global(const si_store_t *store, int layer, const int32_t **dev_ptr_out,
+                            int *n_loaded_out, int *n_base_out);
+int si_store_global_to_slot(const si_store_t *store, int layer, const int32_t **dev_ptr_out);
+int si_store_records(const si_store_t *store, int layer, const void **dev_ptr_out,
+                     size_t *record_bytes_out);
+
+/* Workspace (device scratch) size for calls with at most T_max tokens per call, lists
+ * of at most k_max slots, and at most max_steps (token, layer) steps per stack call. */
+int si_workspace_bytes(const si_store_t *store, int T_max, int k_max, int max_steps,
+                       size_t *bytes_out);
+
+/* ---------------------------------------------------------------- selection
+
+ * Runtime selector (Section 5: sort the activations in descending order, keep the top
+ * alpha, record their indices).  scores: device float32 [n].
+ *   mode SI_SELECT_TOPK      : the k highest scores.  Ties: the lower index wins;
+ *                              +0 and -0 are equal; NaN ranks below every number.
+ *   mode SI_SELECT_THRESHOLD : all i with score[i] > tau, NaN excluded (extension; the
+ *                              paper has top-alpha only).
+ * idx_out: device int32 [cap], ascending by index; *n_out (device int32) = count
+ * written.  SI_ERR_NOMEM in *status-style return if cap < k (top-k); in threshold mode
+ * at most cap indices are written and *n_out holds the full count.
+ * workspace: device scratch of at least si_select_workspace_bytes(n). */
+int si_select_workspace_bytes(int n, size_t *bytes_out);
+int si_select(const float *scores, int n, int mode, int k, float tau, unsigned flags,
+              int32_t *idx_out, int cap, int32_t *n_out, void *workspace, size_t ws_bytes,
+              void *stream);
+
+/* ---------------------------------------------------------------- selective FFN
+
+ * y[t] = sum over i in list_t of h_i(x[t]) * down_i      (Section 5)
+ *   x   : device [T, d_model], store dtype
+ *   idx : device int32 slot indices.  If idx_offsets == NULL every token has k_fixed
+ *         entries: idx is [T, k_fixed].  Otherwise idx_offsets is device int32 [T + 1]
+ *         (CSR) and k_fixed is an upper bound on the longest list.
+ *   y   : device [T, d_model] of y_dtype (SI_F32, or the store dtype)
+ * T == 1 runs the memory-bound decode kernel; T > 1 forms the union of the lists and
+ * runs a gathered tensor-core contraction in which token t still uses exactly its own
+ * list (unless SI_FLAG_UNION_UNMASKED).  An empty list gives y = 0 (or x with
+ * SI_FLAG_RESIDUAL).  Accumulation is fp32; h is rounded to the store dtype before the
+ * down projection only on the T > 1 path. */
+int si_ffn_forward(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
+                   const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype, unsigned flags,
+                   void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* One layer = optional selection + selective FFN (+ residual) ("applied to each FFN
+ * layer", Section 4).  If scores != NULL (device float32 [T, n_loaded]) the k best
+ * slots per token are selected with si_select's top-k rule into the workspace and
+ * used as the lists; otherwise idx / idx_offsets / k are used as in si_ffn_forward. */
+int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, const float *scores,
+                     int k, const int32_t *idx, const int32_t *idx_offsets, void *y, int y_dtype,
+                     unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
+                     void *stream);
+
+/* Batch-1 decode over a stack: n_steps consecutive (token, layer) steps in one
+ * persistent launch, step s using layer layers[s] (HOST int32 [n_steps], or NULL for
+ * s mod n_layers).  x, y: device [n_steps, d_model]; idx: device [n_steps, k_fixed]
+ * (or CSR over n_steps lists).  Steps are executed strictly in order; the weight
+ * stream of later steps is prefetched while earlier steps finish.  Results equal
+ * n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of a list
+ * over SMs depends on the step's position in the call); each is run-to-run bit-stable. */
+int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
+                            const void *x, const int32_t *idx, const int32_t *idx_offsets,
+                            int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
+                            size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* Union of T lists (the first stage of the T > 1 path, exposed for inspection):
+ * union_out device int32 [n_loaded] ascending, *n_union_out device int32. */
+int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
+             const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
+             void *workspace, size_t ws_bytes, void *stream);
+
+/* Library build information: "sm_100a" etc.  Never NULL. */
+const char *si_build_info(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SELECTINFER_H */

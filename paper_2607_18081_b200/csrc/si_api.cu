@@ -1,0 +1,139 @@
+// Entry points that tie the steps together: workspace carving, si_ffn_forward,
+// si_layer_forward (selection + FFN), si_decode_stack_forward, si_union.
+#include "si_common.cuh"
+
+si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps) {
+    si_ws_layout w;
+    if (T_max < 1) T_max = 1;
+    if (k_max < 0) k_max = 0;
+    if (max_steps < 1) max_steps = 1;
+    int nl_max = 0;
+    for (int l = 0; l < s->n_layers; ++l) nl_max = nl_max > s->n_loaded[l] ? nl_max : s->n_loaded[l];
+    const size_t nl_pad = si_align_up((size_t)nl_max, 128);
+    const size_t t_pad = si_align_up((size_t)T_max, 16);
+    size_t off = 0;
+    auto take = [&](size_t &o, size_t &b, size_t bytes) { o = off; b = si_align_up(bytes, 256); off += b; };
+    take(w.ctrl_off, w.ctrl_bytes, 256);
+    size_t part = (size_t)2 * s->num_sms * s->d_model * 4;
+    size_t gpart = si_gemm_partial_bytes(s, T_max);
+    take(w.partial_off, w.partial_bytes, part > gpart ? part : gpart);
+    take(w.sel_off, w.sel_bytes, (size_t)T_max * (size_t)(k_max + 1) * 4);
+    take(w.union_off, w.union_bytes, nl_pad * 4 + 256 + nl_pad / 8 + 256);
+    take(w.mask_off, w.mask_bytes, T_max > 1 ? t_pad * (nl_pad / 32) * 4 : 0);
+    take(w.h_off, w.h_bytes, T_max > 1 ? t_pad * nl_pad * 2 : 0);
+    take(w.selws_off, w.selws_bytes, (size_t)T_max * si_select_ws_bytes_impl(nl_max));
+    take(w.steps_off, w.steps_bytes, (size_t)max_steps * 4);
+    w.total = off;
+    return w;
+}
+
+extern "C" int si_workspace_bytes(const si_store_t *store, int T_max, int k_max, int max_steps,
+                                  size_t *bytes_out) {
+    if (!si_store_ok(store) || !bytes_out || T_max < 1 || k_max < 0 || max_steps < 1) return SI_ERR_INVALID_ARG;
+    *bytes_out = si_ws_carve(store, T_max, k_max, max_steps).total;
+    return SI_OK;
+}
+
+static int check_common(const si_store *s, const void *x, const void *y, int y_dtype, const void *workspace,
+                        const int32_t *status_dev) {
+    if (!si_store_ok(s) || !x || !y || !workspace) return SI_ERR_INVALID_ARG;
+    if (y_dtype != SI_F32 && y_dtype != s->dtype) return SI_ERR_INVALID_ARG;
+    if (!si_aligned16(x) || !si_aligned16(y) || (((uintptr_t)workspace) & 255u)) return SI_ERR_ALIGNMENT;
+    if (status_dev && (((uintptr_t)status_dev) & 3u)) return SI_ERR_ALIGNMENT;
+    return SI_OK;
+}
+
+extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
+                              const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype, unsigned flags,
+                              void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream_) {
+    int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
+    if (rc) return rc;
+    if (layer < 0 || layer >= store->n_layers || T <= 0 || k_fixed < 0) return SI_ERR_INVALID_ARG;
+    if (!store->loaded[layer]) return SI_ERR_INVALID_ARG;
+    if (k_fixed > store->n_loaded[layer]) return SI_ERR_OUT_OF_RANGE;
+    if (k_fixed > 0 && !idx) return SI_ERR_INVALID_ARG;
+    if (idx && !si_aligned16(idx)) return SI_ERR_ALIGNMENT;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (ws_bytes < si_ws_carve(store, T, k_fixed, 1).total) return SI_ERR_NOMEM;
+    if (flags & SI_FLAG_CHECK) {
+        rc = si_check_lists_launch_impl(store, T, layer, nullptr, idx, idx_offsets, k_fixed, status_dev, stream);
+        if (rc) return rc;
+    }
+    if (T == 1) {
+        int32_t l = layer;
+        return si_decode_launch(store, 1, &l, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
+                                ws_bytes, status_dev, stream);
+    }
+    return si_multi_token_launch(store, layer, x, T, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
+                                 ws_bytes, status_dev, stream);
+}
+
+extern "C" int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, const float *scores,
+                                int k, const int32_t *idx, const int32_t *idx_offsets, void *y, int y_dtype,
+                                unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
+                                void *stream_) {
+    if (!scores)
+        return si_ffn_forward(store, layer, x, T, idx, idx_offsets, k, y, y_dtype, flags, workspace, ws_bytes,
+                              status_dev, stream_);
+    int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
+    if (rc) return rc;
+    if (layer < 0 || layer >= store->n_layers || T <= 0 || k < 0) return SI_ERR_INVALID_ARG;
+    const int n = store->n_loaded[layer];
+    if (k > n) return SI_ERR_OUT_OF_RANGE;
+    if (!si_aligned16(scores)) return SI_ERR_ALIGNMENT;
+    si_ws_layout ws = si_ws_carve(store, T, k, 1);
+    if (ws_bytes < ws.total) return SI_ERR_NOMEM;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    char *wsb = (char *)workspace;
+    int32_t *lists = (int32_t *)(wsb + ws.sel_off);
+    int32_t *counts = lists + (size_t)T * k;
+    rc = si_select_launch(scores, T, n, n, SI_SELECT_TOPK, k, 0.f, flags, lists, k, k, counts,
+                          wsb + ws.selws_off, ws.selws_bytes, stream);
+    if (rc) return rc;
+    return si_ffn_forward(store, layer, x, T, lists, nullptr, k, y, y_dtype, flags & ~SI_FLAG_CHECK, workspace,
+                          ws_bytes, status_dev, stream_);
+}
+
+extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
+                                       const void *x, const int32_t *idx, const int32_t *idx_offsets,
+                                       int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
+                                       size_t ws_bytes, int32_t *status_dev, void *stream_) {
+    int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
+    if (rc) return rc;
+    if (n_steps <= 0 || k_fixed < 0) return SI_ERR_INVALID_ARG;
+    if (k_fixed > 0 && !idx) return SI_ERR_INVALID_ARG;
+    if (idx && !si_aligned16(idx)) return SI_ERR_ALIGNMENT;
+    int min_loaded = store->d_ff;
+    for (int st = 0; st < n_steps; ++st) {
+        int l = layers ? layers[st] : st % store->n_layers;
+        if (l < 0 || l >= store->n_layers) return SI_ERR_INVALID_ARG;
+        min_loaded = min_loaded < store->n_loaded[l] ? min_loaded : store->n_loaded[l];
+    }
+    if (!idx_offsets && k_fixed > min_loaded) return SI_ERR_OUT_OF_RANGE;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    si_ws_layout ws = si_ws_carve(store, 1, k_fixed, n_steps);
+    if (ws_bytes < ws.total) return SI_ERR_NOMEM;
+    if (flags & SI_FLAG_CHECK) {
+        const int32_t *layers_dev = nullptr;
+        if (layers) {
+            int32_t *dst = (int32_t *)((char *)workspace + ws.steps_off);
+            SI_CUDA_TRY(cudaMemcpyAsync(dst, layers, (size_t)n_steps * 4, cudaMemcpyHostToDevice, stream));
+            layers_dev = dst;
+        }
+        rc = si_check_lists_launch_impl(store, n_steps, -1, layers_dev, idx, idx_offsets, k_fixed, status_dev, stream);
+        if (rc) return rc;
+    }
+    return si_decode_launch(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
+                            ws_bytes, status_dev, stream);
+}
+
+extern "C" int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
+                        const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
+                        void *workspace, size_t ws_bytes, void *stream) {
+    if (!si_store_ok(store) || layer < 0 || layer >= store->n_layers || T <= 0 || k_fixed < 0 || !union_out ||
+        !n_union_out || !workspace)
+        return SI_ERR_INVALID_ARG;
+    if (k_fixed > 0 && !idx) return SI_ERR_INVALID_ARG;
+    return si_union_launch(store, layer, T, idx, idx_offsets, k_fixed, union_out, n_union_out, workspace,
+                           ws_bytes, (cudaStream_t)stream);
+}

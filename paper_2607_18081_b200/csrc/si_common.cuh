@@ -1,0 +1,113 @@
+// Internal declarations shared by the translation units of libselectinfer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <vector>
+
+#include "selectinfer.h"
+
+#define SI_MAGIC 0x53494E46u /* "SINF" */
+#define SI_NUM_SMS_FALLBACK 148
+
+struct si_store {
+    uint32_t magic;
+    int device;
+    int n_layers, d_model, d_ff, dtype;
+    int num_sms;
+    char *mem;
+    size_t mem_bytes;
+    std::vector<int> n_loaded, n_base;
+    std::vector<char> loaded;              // layer packed at least once
+    std::vector<size_t> rec_off, s2g_off, g2s_off;
+    size_t record_bytes() const { return (size_t)3 * d_model * 2; }
+    const uint16_t *records(int l) const { return (const uint16_t *)(mem + rec_off[l]); }
+    int32_t *s2g(int l) const { return (int32_t *)(mem + s2g_off[l]); }
+    int32_t *g2s(int l) const { return (int32_t *)(mem + g2s_off[l]); }
+};
+
+static inline size_t si_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline bool si_aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+static inline bool si_store_ok(const si_store *s) { return s && s->magic == SI_MAGIC; }
+
+#define SI_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t e__ = (expr);                           \
+        if (e__ != cudaSuccess) return SI_ERR_CUDA;         \
+    } while (0)
+
+// ---- workspace carving (all sizes 256-byte aligned) -------------------------------
+// [0, 256)            : control words (barrier counters, tickets), zero on entry to every call
+// then                : fp32 partial outputs [max_ctas][T][d_model] (decode: T = 1)
+// then                : lists selected by si_layer_forward, union arrays, masks, H
+struct si_ws_layout {
+    size_t ctrl_off, ctrl_bytes;
+    size_t partial_off, partial_bytes;
+    size_t sel_off, sel_bytes;         // int32 [T_max][k_max] selected lists + [T_max] counts
+    size_t union_off, union_bytes;     // int32 [n_loaded_max] union + count + bitmap words
+    size_t mask_off, mask_bytes;       // uint32 [T_max][ceil(n_loaded_max / 32)]
+    size_t h_off, h_bytes;             // 16-bit H [T_pad][n_loaded_max padded]
+    size_t selws_off, selws_bytes;     // selector scratch
+    size_t steps_off, steps_bytes;     // per-step descriptors for stack calls
+    size_t total;
+};
+si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps);
+
+// implemented in si_decode.cu
+int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host, const void *x,
+                     const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y,
+                     int y_dtype, unsigned flags, void *workspace, size_t ws_bytes,
+                     int32_t *status_dev, cudaStream_t stream);
+
+// implemented in si_gemm.cu
+int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, const int32_t *idx,
+                          const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype,
+                          unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
+                          cudaStream_t stream);
+
+// implemented in si_select.cu
+size_t si_select_ws_bytes_impl(int n);
+int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int mode, int k,
+                     float tau, unsigned flags, int32_t *idx_out, int out_stride, int cap,
+                     int32_t *n_out, void *workspace, size_t ws_bytes, cudaStream_t stream);
+
+// implemented in si_check.cu: device-side list validation for SI_FLAG_CHECK
+int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed,
+                               const int32_t *step_layers_dev, const int32_t *idx,
+                               const int32_t *idx_offsets, int k_fixed, int32_t *status_dev,
+                               cudaStream_t stream);
+
+// implemented in si_gemm.cu
+size_t si_gemm_partial_bytes(const si_store *s, int T_max);
+int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
+                    int k_fixed, int32_t *union_out, int32_t *n_union_out, void *workspace,
+                    size_t ws_bytes, cudaStream_t stream);
+
+// ---- device helpers ---------------------------------------------------------------
+template <int DT> struct si_cvt;
+template <> struct si_cvt<SI_BF16> {
+    // two bf16 packed in a 32-bit word -> two floats (exact)
+    __device__ __forceinline__ static float lo(uint32_t w) { return __uint_as_float(w << 16); }
+    __device__ __forceinline__ static float hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+    __device__ __forceinline__ static uint16_t from_float(float f) {
+        return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+    }
+};
+template <> struct si_cvt<SI_F16> {
+    __device__ __forceinline__ static float lo(uint32_t w) {
+        return __half2float(__ushort_as_half((unsigned short)(w & 0xFFFFu)));
+    }
+    __device__ __forceinline__ static float hi(uint32_t w) {
+        return __half2float(__ushort_as_half((unsigned short)(w >> 16)));
+    }
+    __device__ __forceinline__ static uint16_t from_float(float f) {
+        return __half_as_ushort(__float2half_rn(f));
+    }
+};
+
+__device__ __forceinline__ float si_silu_mul(float g, float u) {
+    return (g / (1.0f + __expf(-g))) * u;
+}

@@ -1,0 +1,197 @@
+// Batch-1 selective decode (Section 5, "Selective Computation"):
+//     y = sum over selected slots i of SiLU(gate_i . x) * (up_i . x) * down_i
+// Purely HBM-bound: 6*d_model bytes and 6*d_model flops per selected neuron.
+//
+// Two implementations share the per-record arithmetic:
+//   * "simple": one launch per step, records read with 16-byte global loads, per-CTA fp32
+//     partial outputs reduced in CTA order by a second kernel;
+//   * "persistent" (si_decode_persistent.cuh): one launch for any number of steps, records
+//     streamed through a shared-memory ring by bulk async copies.
+// Both accumulate in a fixed order, so results are run-to-run bit-identical.
+#include "si_common.cuh"
+#include "si_decode_persistent.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+template <int DT>
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
+    f[0] = si_cvt<DT>::lo(v.x); f[1] = si_cvt<DT>::hi(v.x);
+    f[2] = si_cvt<DT>::lo(v.y); f[3] = si_cvt<DT>::hi(v.y);
+    f[4] = si_cvt<DT>::lo(v.z); f[5] = si_cvt<DT>::hi(v.z);
+    f[6] = si_cvt<DT>::lo(v.w); f[7] = si_cvt<DT>::hi(v.w);
+}
+
+template <int DT>
+__device__ __forceinline__ float dot8(const uint4 &v, const float (&x)[8]) {
+    float f[8];
+    unpack8<DT>(v, f);
+    float a = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a = fmaf(f[e], x[e], a);
+    return a;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// One CTA walks list positions blockIdx.x, blockIdx.x + G, ... two at a time.  Thread t
+// owns 16-byte chunks t, t + 256, ... of every row, i.e. 8*NCH output columns.
+template <int DT, int NCH>
+__global__ void __launch_bounds__(kThreads)
+si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks,
+                         const uint4 *__restrict__ x, const int32_t *__restrict__ idx,
+                         const int32_t *__restrict__ offsets, int list, int k_fixed,
+                         float *__restrict__ partial, int32_t *status) {
+    __shared__ float red[2][kThreads / 32][4];
+    const int base = offsets ? offsets[list] : list * k_fixed;
+    const int k = offsets ? offsets[list + 1] - base : k_fixed;
+    idx += base;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float xr[NCH][8], acc[NCH][8];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = tid + kThreads * i;
+        uint4 v = c < chunks ? __ldg(x + c) : make_uint4(0, 0, 0, 0);
+        unpack8<DT>(v, xr[i]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[i][e] = 0.f;
+    }
+    const int G = gridDim.x;
+    int it = 0;
+    for (int p = blockIdx.x; p < k; p += 2 * G, ++it) {
+        int s0 = idx[p];
+        int s1 = (p + G < k) ? idx[p + G] : -1;
+        bool ok0 = s0 >= 0 && s0 < n_loaded;
+        bool ok1 = s1 >= 0 && s1 < n_loaded;
+        if (tid == 0 && status && (!ok0 || (!ok1 && p + G < k))) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE);
+        const uint4 *r0 = rec + (size_t)(ok0 ? s0 : 0) * 3 * chunks;
+        const uint4 *r1 = rec + (size_t)(ok1 ? s1 : 0) * 3 * chunks;
+        float g0 = 0.f, u0 = 0.f, g1 = 0.f, u1 = 0.f;
+        uint4 dn0[NCH], dn1[NCH];
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            int c = tid + kThreads * i;
+            dn0[i] = dn1[i] = make_uint4(0, 0, 0, 0);
+            if (c < chunks) {
+                if (ok0) {
+                    uint4 a = __ldg(r0 + c), b = __ldg(r0 + chunks + c);
+                    dn0[i] = __ldg(r0 + 2 * chunks + c);
+                    g0 += dot8<DT>(a, xr[i]); u0 += dot8<DT>(b, xr[i]);
+                }
+                if (ok1) {
+                    uint4 a = __ldg(r1 + c), b = __ldg(r1 + chunks + c);
+                    dn1[i] = __ldg(r1 + 2 * chunks + c);
+                    g1 += dot8<DT>(a, xr[i]); u1 += dot8<DT>(b, xr[i]);
+                }
+            }
+        }
+        g0 = warp_sum(g0); u0 = warp_sum(u0); g1 = warp_sum(g1); u1 = warp_sum(u1);
+        float(*buf)[4] = red[it & 1];
+        if (lane == 0) { buf[warp][0] = g0; buf[warp][1] = u0; buf[warp][2] = g1; buf[warp][3] = u1; }
+        __syncthreads();
+        g0 = u0 = g1 = u1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) {
+            g0 += buf[w][0]; u0 += buf[w][1]; g1 += buf[w][2]; u1 += buf[w][3];
+        }
+        float h0 = ok0 ? si_silu_mul(g0, u0) : 0.f;
+        float h1 = ok1 ? si_silu_mul(g1, u1) : 0.f;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            float f0[8], f1[8];
+            unpack8<DT>(dn0[i], f0); unpack8<DT>(dn1[i], f1);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[i][e] = fmaf(h1, f1[e], fmaf(h0, f0[e], acc[i][e]));
+        }
+    }
+    float4 *out = reinterpret_cast<float4 *>(partial + (size_t)blockIdx.x * chunks * 8);
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        int c = tid + kThreads * i;
+        if (c < chunks) {
+            out[2 * c] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+            out[2 * c + 1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+        }
+    }
+}
+
+// y[j] = (x[j] +) sum over CTAs g = 0..G-1 of partial[g][j], in that order.
+template <int DT>
+__global__ void si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
+                                        const uint16_t *__restrict__ x, void *__restrict__ y,
+                                        int y_f32, int residual) {
+    int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d) return;
+    float a = 0.f;
+    for (int g = 0; g < G; ++g) a += partial[(size_t)g * d + j];
+    if (residual) {
+        uint32_t w = x[j];
+        a += (DT == SI_BF16) ? si_cvt<SI_BF16>::lo(w) : si_cvt<SI_F16>::lo(w);
+    }
+    if (y_f32) reinterpret_cast<float *>(y)[j] = a;
+    else reinterpret_cast<uint16_t *>(y)[j] = si_cvt<DT>::from_float(a);
+}
+
+template <int DT>
+int launch_simple_step(const si_store *s, int layer, const void *x, const int32_t *idx,
+                       const int32_t *offsets, int list, int k, void *y, int y_dtype, unsigned flags,
+                       float *partial, int32_t *status_dev, cudaStream_t stream) {
+    const int d = s->d_model, chunks = d / 8;
+    const int nch = (chunks + kThreads - 1) / kThreads;
+    int G = k < 2 * s->num_sms ? (k < 1 ? 1 : k) : 2 * s->num_sms;
+    const uint4 *rec = (const uint4 *)s->records(layer);
+    const int nl = s->n_loaded[layer];
+#define SI_LAUNCH_PARTIAL(N)                                                                        \
+    si_decode_partial_kernel<DT, N><<<G, kThreads, 0, stream>>>(rec, nl, chunks, (const uint4 *)x, \
+                                                                idx, offsets, list, k, partial, status_dev)
+    if (nch <= 1) SI_LAUNCH_PARTIAL(1);
+    else if (nch <= 2) SI_LAUNCH_PARTIAL(2);
+    else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
+    else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
+    else return SI_ERR_UNSUPPORTED;
+#undef SI_LAUNCH_PARTIAL
+    si_decode_reduce_kernel<DT><<<(d + 255) / 256, 256, 0, stream>>>(
+        partial, G, d, (const uint16_t *)x, y, y_dtype == SI_F32, (flags & SI_FLAG_RESIDUAL) != 0);
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}
+
+}  // namespace
+
+int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host, const void *x,
+                     const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y,
+                     int y_dtype, unsigned flags, void *workspace, size_t ws_bytes,
+                     int32_t *status_dev, cudaStream_t stream) {
+    si_ws_layout ws = si_ws_carve(s, 1, k_fixed, n_steps);
+    if (ws_bytes < ws.total) return SI_ERR_NOMEM;
+    if (n_steps <= 0) return SI_ERR_INVALID_ARG;
+    for (int st = 0; st < n_steps; ++st) {
+        int l = layers_host ? layers_host[st] : st % s->n_layers;
+        if (l < 0 || l >= s->n_layers) return SI_ERR_INVALID_ARG;
+        if (!s->loaded[l]) return SI_ERR_INVALID_ARG;
+    }
+    char *wsb = (char *)workspace;
+    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s);
+    if (!use_simple)
+        return si_decode_persistent_launch(s, n_steps, layers_host, x, idx, idx_offsets, k_fixed, y, y_dtype, flags,
+                                           wsb, ws, status_dev, stream);
+    // simple path: one partial + one reduce launch per step.  With CSR lists the true length
+    // is read on the device; k_fixed (an upper bound) only sizes the grid.
+    const size_t esz = 2, ysz = (y_dtype == SI_F32) ? 4 : 2;
+    float *partial = (float *)(wsb + ws.partial_off);
+    for (int st = 0; st < n_steps; ++st) {
+        int l = layers_host ? layers_host[st] : st % s->n_layers;
+        const void *xs = (const char *)x + (size_t)st * s->d_model * esz;
+        void *ys = (char *)y + (size_t)st * s->d_model * ysz;
+        int rc = (s->dtype == SI_BF16)
+                     ? launch_simple_step<SI_BF16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, status_dev, stream)
+                     : launch_simple_step<SI_F16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, status_dev, stream);
+        if (rc != SI_OK) return rc;
+    }
+    return SI_OK;
+}

@@ -1,0 +1,194 @@
+// Runtime selector (Section 5: "sort these activations in descending order and select the
+// top alpha neurons for that token and record the indices").
+//
+// No sort is needed to obtain the set: one CTA per score row finds the k-th largest value by
+// a 4-pass, 8-bit radix select over order-preserving 32-bit keys held in shared memory, then
+// one index-ordered prefix scan emits the selected indices ascending.  Ties at the k-th
+// value go to the lower indices; +0 == -0; NaN has the lowest key.  All integer decisions:
+// the result is exact and unique.
+#include "si_common.cuh"
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSmemKeys = 48 * 1024;   // rows up to this many scores keep their keys in shared memory
+
+__device__ __forceinline__ uint32_t score_key(float s, bool use_abs) {
+    if (s != s) return 0u;                     // NaN: below everything
+    if (use_abs) s = fabsf(s);
+    if (s == 0.f) s = 0.f;                     // -0 -> +0
+    uint32_t b = __float_as_uint(s);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Exclusive block scan of a pair of counters packed as (hi: a, lo: b) in 64 bits.
+__device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long long v,
+                                                                   unsigned long long *warp_tot,
+                                                                   unsigned long long *total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long w = lane < kSelThreads / 32 ? warp_tot[lane] : 0ull;
+        unsigned long long winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        warp_tot[lane] = winc - w;                   // exclusive prefix of warp totals
+        if (lane == 31) *total = winc;
+    }
+    __syncthreads();
+    return warp_tot[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mode, int k, float tau,
+                 int use_abs, int32_t *__restrict__ idx_out, int out_stride, int cap,
+                 int32_t *__restrict__ n_out, uint32_t *__restrict__ key_spill, int keys_in_smem) {
+    extern __shared__ uint32_t smem_keys[];
+    __shared__ unsigned int hist[256];
+    __shared__ unsigned long long warp_tot[32];
+    __shared__ unsigned long long total;
+    __shared__ uint32_t sh_prefix, sh_mask;
+    __shared__ int sh_need;
+
+    const int row = blockIdx.x, tid = threadIdx.x;
+    const float *s = scores + (size_t)row * row_stride;
+    int32_t *out = idx_out + (size_t)row * out_stride;
+    uint32_t *keys = keys_in_smem ? smem_keys : key_spill + (size_t)row * n;
+
+    uint32_t kstar = 0; int r = 0;          // threshold key and how many of its ties to take
+    if (mode == SI_SELECT_TOPK) {
+        for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
+        if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
+        __syncthreads();
+        if (k > 0 && k < n) {
+            for (int shift = 24; shift >= 0; shift -= 8) {
+                if (tid < 256) hist[tid] = 0;
+                __syncthreads();
+                const uint32_t prefix = sh_prefix, mask = sh_mask;
+                for (int i = tid; i < n; i += kSelThreads) {
+                    uint32_t key = keys[i];
+                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    int need = sh_need, bin = 255;
+                    for (; bin > 0; --bin) {              // walk from the largest digit down
+                        int c = (int)hist[bin];
+                        if (c >= need) break;
+                        need -= c;
+                    }
+                    sh_need = need;
+                    sh_prefix = prefix | ((uint32_t)bin << shift);
+                    sh_mask = mask | (255u << shift);
+                }
+                __syncthreads();
+            }
+            kstar = sh_prefix; r = sh_need;    // r of the keys equal to kstar are taken
+        } else if (k >= n) {
+            kstar = 0; r = n;                   // everything: all keys >= 0, ties = all
+        } else {
+            kstar = 0xFFFFFFFFu; r = 0;         // k == 0: nothing is > max key... guard below
+        }
+    }
+
+    // index-ordered emission: thread t owns the contiguous range [t*per, (t+1)*per)
+    const int per = (n + kSelThreads - 1) / kSelThreads;
+    const int lo = tid * per, hi = min(n, lo + per);
+    unsigned long long mine = 0;   // (hi 32: # strictly above threshold, lo 32: # ties)
+    for (int i = lo; i < hi; ++i) {
+        bool gt, eq;
+        if (mode == SI_SELECT_TOPK) {
+            uint32_t key = keys[i];
+            gt = (k > 0) && key > kstar; eq = (k > 0) && key == kstar;
+            if (k >= n) { gt = false; eq = true; }
+        } else {
+            float v = s[i];
+            if (use_abs) v = fabsf(v);
+            gt = v > tau; eq = false;
+        }
+        mine += ((unsigned long long)gt << 32) | (unsigned long long)eq;
+    }
+    unsigned long long before = block_exclusive_scan(mine, warp_tot, &total);
+    int gt_before = (int)(before >> 32), eq_before = (int)(before & 0xFFFFFFFFu);
+    for (int i = lo; i < hi; ++i) {
+        bool gt, eq;
+        if (mode == SI_SELECT_TOPK) {
+            uint32_t key = keys[i];
+            gt = (k > 0) && key > kstar; eq = (k > 0) && key == kstar;
+            if (k >= n) { gt = false; eq = true; }
+        } else {
+            float v = s[i];
+            if (use_abs) v = fabsf(v);
+            gt = v > tau; eq = false;
+        }
+        bool take = gt || (eq && eq_before < r);
+        if (take) {
+            int pos = gt_before + min(eq_before, r);
+            if (pos < cap) out[pos] = i;
+        }
+        gt_before += gt; eq_before += eq;
+    }
+    if (tid == 0 && n_out) {
+        int tot_gt = (int)(total >> 32), tot_eq = (int)(total & 0xFFFFFFFFu);
+        n_out[row] = tot_gt + min(tot_eq, r);
+    }
+}
+
+}  // namespace
+
+size_t si_select_ws_bytes_impl(int n) {
+    return n > kSmemKeys ? si_align_up((size_t)n * 4, 256) : 256;
+}
+
+int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int mode, int k,
+                     float tau, unsigned flags, int32_t *idx_out, int out_stride, int cap,
+                     int32_t *n_out, void *workspace, size_t ws_bytes, cudaStream_t stream) {
+    if (n_rows <= 0) return SI_OK;
+    const int in_smem = n <= kSmemKeys;
+    if (!in_smem && ws_bytes < (size_t)n_rows * n * 4) return SI_ERR_NOMEM;
+    size_t smem = in_smem ? (size_t)(n > 0 ? n : 1) * 4 : 0;
+    static bool attr_set = false;
+    if (!attr_set) {
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSmemKeys * 4));
+        attr_set = true;
+    }
+    si_select_kernel<<<n_rows, kSelThreads, smem, stream>>>(scores, n, row_stride, mode, k, tau,
+                                                            (flags & SI_FLAG_SCORE_ABS) != 0, idx_out,
+                                                            out_stride, cap, n_out, (uint32_t *)workspace, in_smem);
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}
+
+extern "C" int si_select_workspace_bytes(int n, size_t *bytes_out) {
+    if (n < 0 || !bytes_out) return SI_ERR_INVALID_ARG;
+    *bytes_out = si_select_ws_bytes_impl(n);
+    return SI_OK;
+}
+
+extern "C" int si_select(const float *scores, int n, int mode, int k, float tau, unsigned flags,
+                         int32_t *idx_out, int cap, int32_t *n_out, void *workspace, size_t ws_bytes,
+                         void *stream) {
+    if (!scores || !idx_out || n < 0 || cap < 0) return SI_ERR_INVALID_ARG;
+    if (mode != SI_SELECT_TOPK && mode != SI_SELECT_THRESHOLD) return SI_ERR_INVALID_ARG;
+    if (mode == SI_SELECT_TOPK && (k < 0 || k > n)) return SI_ERR_INVALID_ARG;
+    if (mode == SI_SELECT_TOPK && cap < k) return SI_ERR_NOMEM;
+    if (!si_aligned16(scores) || !si_aligned16(idx_out)) return SI_ERR_ALIGNMENT;
+    if (n > kSmemKeys && (!workspace || ws_bytes < (size_t)n * 4)) return SI_ERR_NOMEM;
+    if (n == 0) {
+        if (n_out) SI_CUDA_TRY(cudaMemsetAsync(n_out, 0, 4, (cudaStream_t)stream));
+        return SI_OK;
+    }
+    return si_select_launch(scores, 1, n, n, mode, k, tau, flags, idx_out, cap, cap, n_out, workspace,
+                            ws_bytes, (cudaStream_t)stream);
+}

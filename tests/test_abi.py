@@ -1,0 +1,62 @@
+"""CPU-only checks of the C-ABI boundary: the library builds for sm_100a, loads, and exports
+every function declared in include/selectinfer.h.  No compute call is made."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "selectinfer.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(si_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    from paper_2607_18081_b200 import build
+    path = build.build()
+    import torch  # noqa: F401  makes libcudart resolvable
+    lib = ctypes.CDLL(path)
+    names = _declared()
+    assert len(names) >= 14
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in selectinfer.h but not exported"
+    for required in ("si_load_neurons", "si_select", "si_ffn_forward", "si_layer_forward"):
+        assert required in names
+
+
+def test_binding_names_match_header_and_host_side_errors():
+    from paper_2607_18081_b200 import api
+    names = _declared()
+    for n in names:
+        assert n in api.EXPORTS or hasattr(api, n), n
+    for n in api.EXPORTS:
+        assert n in names, f"binding lists {n} which the header does not declare"
+    assert api.strerror(0) == "ok" and "range" in api.strerror(api.SI_ERR_OUT_OF_RANGE)
+    assert "sm_100a" in api.build_info()
+    # host-checkable argument errors need no GPU: bad shapes are refused before any CUDA call
+    out = ctypes.c_size_t(0)
+    n_loaded = (ctypes.c_int * 1)(10)
+    assert api.lib().si_store_bytes(1, 100, 64, n_loaded, api.SI_BF16, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG
+    assert api.lib().si_store_bytes(1, 128, 64, n_loaded, 7, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG
+    assert api.lib().si_store_bytes(1, 128, 64, n_loaded, api.SI_BF16, ctypes.byref(out)) == api.SI_OK
+    assert out.value >= 10 * 3 * 128 * 2 + 10 * 4 + 64 * 4
+    n_loaded[0] = 65
+    assert api.lib().si_store_bytes(1, 128, 64, n_loaded, api.SI_BF16, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG
+    assert api.lib().si_select(None, 4, 0, 1, 0.0, 0, None, 4, None, None, 0, None) == api.SI_ERR_INVALID_ARG
+
+
+def test_store_bytes_is_eq2_accounting():
+    """Bytes kept for the records = 3*d*e*n_loaded; bytes not stored = Eq. 2 with r_layer = 1."""
+    from paper_2607_18081_b200 import api
+    from oracle import selectinfer_oracle as so
+    L, d, F = 4, 4096, 11008
+    n_ld = so.count_from_pct(70, F)
+    total = api.si_store_bytes(L, d, F, [n_ld] * L, "bf16")
+    records = L * n_ld * 3 * d * 2
+    maps = total - records
+    assert 0 <= maps <= L * (n_ld * 4 + F * 4 + 3 * 256)
+    full = L * 3 * d * F * 2
+    saving = so.memory_saving(L * 3 * d * F, n_ld / F, 1.0, 2)
+    assert abs((full - records) - saving) < 1e-6 * full
