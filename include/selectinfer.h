@@ -79,6 +79,9 @@ enum { SI_SELECT_TOPK = 0, SI_SELECT_THRESHOLD = 1 };
 
 const char *si_strerror(int status);
 
+/* Text of the last CUDA runtime error behind an SI_ERR_CUDA return on this thread. */
+const char *si_last_cuda_error(void);
+
 /* ---------------------------------------------------------------- the neuron store
 
  * Bytes of device memory a store of n_layers layers needs; n_loaded is a host array
@@ -184,6 +187,17 @@ int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t 
 int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
              const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
              void *workspace, size_t ws_bytes, void *stream);
+
+/* Diagnostics: while dev_buf (device int64 [num_SMs][8]) is set, each persistent decode
+ * launch stores per-SM cycle counts of its phases there (wait for x, wait for records,
+ * record arithmetic, partial store, barrier arrive, wait for other SMs, reduction, unused).
+ * Pass NULL to switch it off.  Costs a few clock reads per record. */
+int si_debug_decode_profile(void *dev_buf);
+
+/* Diagnostics: while on != 0, persistent decode launches only stream the selected records
+ * through shared memory and skip the arithmetic (y is then meaningless).  Timing such a
+ * launch gives the practical ceiling of the record stream on the same lists. */
+int si_debug_decode_stream_only(int on);
 
 /* Library build information: "sm_100a" etc.  Never NULL. */
 const char *si_build_info(void);

@@ -26,17 +26,19 @@ SI_FLAG_SIMPLE_KERNELS = 256
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 
 EXPORTS = [
-    "si_strerror", "si_build_info", "si_store_bytes", "si_store_create", "si_store_free",
+    "si_strerror", "si_last_cuda_error", "si_build_info", "si_store_bytes", "si_store_create", "si_store_free",
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
-    "si_layer_forward", "si_decode_stack_forward", "si_union",
+    "si_layer_forward", "si_decode_stack_forward", "si_union", "si_debug_decode_profile",
+    "si_debug_decode_stream_only",
 ]
 
 
 class SelectInferError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {strerror(status)} ({status})")
+        detail = f": {_lib.si_last_cuda_error().decode()}" if status == SI_ERR_CUDA else ""
+        super().__init__(f"{where}: {strerror(status)} ({status}){detail}")
 
 
 def _load_library() -> ctypes.CDLL:
@@ -49,6 +51,7 @@ def _load_library() -> ctypes.CDLL:
     psz = ctypes.POINTER(ctypes.c_size_t)
     lib.si_strerror.argtypes = [ci]; lib.si_strerror.restype = ctypes.c_char_p
     lib.si_build_info.argtypes = []; lib.si_build_info.restype = ctypes.c_char_p
+    lib.si_last_cuda_error.argtypes = []; lib.si_last_cuda_error.restype = ctypes.c_char_p
     lib.si_store_bytes.argtypes = [ci, ci, ci, vp, ci, psz]
     lib.si_store_create.argtypes = [ctypes.POINTER(vp), vp, sz, ci, ci, ci, vp, ci]
     lib.si_store_free.argtypes = [vp]
@@ -63,9 +66,11 @@ def _load_library() -> ctypes.CDLL:
     lib.si_layer_forward.argtypes = [vp, ci, vp, ci, vp, ci, vp, vp, vp, ci, cu, vp, sz, vp, vp]
     lib.si_decode_stack_forward.argtypes = [vp, ci, vp, vp, vp, vp, ci, vp, ci, cu, vp, sz, vp, vp]
     lib.si_union.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
+    lib.si_debug_decode_profile.argtypes = [vp]
+    lib.si_debug_decode_stream_only.argtypes = [ci]
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("si_strerror", "si_build_info"):
+        if name not in ("si_strerror", "si_build_info", "si_last_cuda_error"):
             fn.restype = ci
     return lib
 
@@ -201,6 +206,14 @@ def si_union(handle, layer: int, T: int, idx, idx_offsets, k_fixed: int, union_o
     _check(_lib.si_union(handle, layer, T, _dp(idx), _dp(idx_offsets), k_fixed, _dp(union_out), _dp(n_union_out),
                          _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "si_union")
+
+
+def si_debug_decode_stream_only(on: bool) -> None:
+    _check(_lib.si_debug_decode_stream_only(1 if on else 0), "si_debug_decode_stream_only")
+
+
+def si_debug_decode_profile(buf) -> None:
+    _check(_lib.si_debug_decode_profile(_dp(buf)), "si_debug_decode_profile")
 
 
 # ------------------------------------------------------------------------- owner object

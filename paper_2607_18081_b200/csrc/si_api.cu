@@ -1,6 +1,7 @@
 // Entry points that tie the steps together: workspace carving, si_ffn_forward,
 // si_layer_forward (selection + FFN), si_decode_stack_forward, si_union.
 #include "si_common.cuh"
+#include "si_decode_persistent.cuh"
 
 si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps) {
     si_ws_layout w;
@@ -14,7 +15,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     size_t off = 0;
     auto take = [&](size_t &o, size_t &b, size_t bytes) { o = off; b = si_align_up(bytes, 256); off += b; };
     take(w.ctrl_off, w.ctrl_bytes, 256);
-    size_t part = (size_t)2 * s->num_sms * s->d_model * 4;
+    size_t part = si_persistent_partial_bytes(s);   // >= the per-step kernels' [2 * SMs][d_model]
     size_t gpart = si_gemm_partial_bytes(s, T_max);
     take(w.partial_off, w.partial_bytes, part > gpart ? part : gpart);
     take(w.sel_off, w.sel_bytes, (size_t)T_max * (size_t)(k_max + 1) * 4);
@@ -22,7 +23,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     take(w.mask_off, w.mask_bytes, T_max > 1 ? t_pad * (nl_pad / 32) * 4 : 0);
     take(w.h_off, w.h_bytes, T_max > 1 ? t_pad * nl_pad * 2 : 0);
     take(w.selws_off, w.selws_bytes, (size_t)T_max * si_select_ws_bytes_impl(nl_max));
-    take(w.steps_off, w.steps_bytes, (size_t)max_steps * 4);
+    take(w.steps_off, w.steps_bytes, si_align_up((size_t)max_steps * 4, 256) + (size_t)max_steps * 256);   // layer ids + 2 counter lines per step
     w.total = off;
     return w;
 }

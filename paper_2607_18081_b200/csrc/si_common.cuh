@@ -33,10 +33,17 @@ static inline size_t si_align_up(size_t v, size_t a) { return (v + a - 1) / a * 
 static inline bool si_aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
 static inline bool si_store_ok(const si_store *s) { return s && s->magic == SI_MAGIC; }
 
+// last CUDA runtime error seen by this library on the calling thread (si_last_cuda_error)
+int &si_last_cuda_error_code();
+
 #define SI_CUDA_TRY(expr)                                   \
     do {                                                    \
         cudaError_t e__ = (expr);                           \
-        if (e__ != cudaSuccess) return SI_ERR_CUDA;         \
+        if (e__ != cudaSuccess) {                           \
+            si_last_cuda_error_code() = (int)e__;           \
+            (void)cudaGetLastError();                       \
+            return SI_ERR_CUDA;                             \
+        }                                                   \
     } while (0)
 
 // ---- workspace carving (all sizes 256-byte aligned) -------------------------------

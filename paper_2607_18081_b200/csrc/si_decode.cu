@@ -11,6 +11,26 @@
 #include "si_common.cuh"
 #include "si_decode_persistent.cuh"
 
+long long *&si_decode_profile_buffer() {
+    static long long *buf = nullptr;
+    return buf;
+}
+
+int &si_decode_stream_only() {
+    static int v = 0;
+    return v;
+}
+
+extern "C" int si_debug_decode_stream_only(int on) {
+    si_decode_stream_only() = on;
+    return SI_OK;
+}
+
+extern "C" int si_debug_decode_profile(void *dev_buf) {
+    si_decode_profile_buffer() = (long long *)dev_buf;
+    return SI_OK;
+}
+
 namespace {
 
 constexpr int kThreads = 256;

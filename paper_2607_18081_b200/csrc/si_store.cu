@@ -106,6 +106,15 @@ extern "C" const char *si_strerror(int status) {
     }
 }
 
+int &si_last_cuda_error_code() {
+    static thread_local int code = 0;
+    return code;
+}
+
+extern "C" const char *si_last_cuda_error(void) {
+    return cudaGetErrorString((cudaError_t)si_last_cuda_error_code());
+}
+
 extern "C" const char *si_build_info(void) {
     return "libselectinfer sm_100a (persistent TMA decode, tcgen05 gathered GEMM, radix select)";
 }
