@@ -116,5 +116,5 @@ template <> struct si_cvt<SI_F16> {
 };
 
 __device__ __forceinline__ float si_silu_mul(float g, float u) {
-    return (g / (1.0f + __expf(-g))) * u;
+    return __fdividef(g, 1.0f + __expf(-g)) * u;   // fast division: ~2 ulp, far inside the tolerance
 }

@@ -1,30 +1,29 @@
 // Persistent batch-1 selective decode for sm_100a.
 //
-// One CTA per SM runs any number of (token, layer) steps in a single launch.  Each CTA has
-// three roles:
-//   * warp 0 (producer) walks the CTA's share of every step's active list and streams each
-//     selected neuron record -- 6*d_model contiguous bytes: gate row | up row | down row --
-//     from HBM into a shared-memory ring with one bulk async copy (cp.async.bulk, completion
-//     on an mbarrier).  Each lane owns one ring stage and issues that stage's items on its
-//     own, so there are as many independent issue streams as stages.  The ring runs ahead
-//     across step boundaries, so HBM never waits for the arithmetic or for the cross-SM
-//     reduction;
-//   * warps 1..16 (consumers, 512 threads) take records four at a time.  For the dot
-//     products warp (r, q) handles record r of the batch over column quarter q with its
-//     slice of x in registers (five shuffles per warp, no CTA-wide exchange beyond 32
-//     floats); the warps meet on a split-phase mbarrier and -- one batch later, so the
-//     barrier latency is hidden -- every thread combines the quarters, applies SiLU(g)*u and
-//     accumulates h * down for its 8*NCH output columns into fp32 registers.  At the end of
-//     a step the CTA stores its partial y into a ring of D partial buffers and goes
-//     straight on to the next step;
-//   * warps 17..18 (reducers, alternating steps) publish "step s written" on a per-step counter, wait until all
-//     CTAs have done so, and reduce this CTA's slice of columns over the partials in CTA
-//     order (deterministic split-K), writing y once.  The reduction of step s overlaps the
-//     record stream of steps s+1.. ; a second per-step counter lets a partial buffer be
-//     reused only after every CTA has finished reading it.
-// List position p of step s goes to CTA (p + rot_s) mod G, rot_s = (number of list entries
-// before step s) mod G, so records are dealt round-robin across steps and no SM is
-// persistently the one with an extra record.
+// One CTA per SM runs any number of (token, layer) steps in a single launch.  Roles in a CTA:
+//   * warp 0 (producer) streams each selected neuron record -- 6*d_model contiguous bytes:
+//     gate row | up row | down row -- from HBM into shared memory with one bulk async copy
+//     (cp.async.bulk, completion on an mbarrier).  There are two rings, one per consumer set;
+//     every ring stage has its own issuing lane, and the copy descriptors (source address,
+//     bytes) are prepared 16 at a time per set and kept in shared memory, so the slot index
+//     loads are off the issue path.  The rings run ahead across step boundaries.
+//   * warps 1..16 (consumers) form two independent sets of 8 warps.  List position p of a
+//     step goes to set (p + rot) mod 2G (rot = list entries before the step, so records are
+//     dealt round-robin across steps).  A bulk copy takes several microseconds to land and
+//     bandwidth needs every ring stage in flight, so a landed record is copied into
+//     registers and its stage handed back at once; the set then forms the two dot products
+//     (thread slices, warp butterfly, 8-warp exchange on an mbarrier), applies SiLU(g)*u and
+//     accumulates h * down for its columns in fp32 registers -- while its next record is
+//     already on the way.  At the end of a step set 1 hands its accumulators to set 0 through
+//     shared memory and set 0 stores the CTA's partial y into a ring of D global buffers.
+//   * split-K across SMs, deterministic: the reduction of step s starts kLag steps later, when
+//     every CTA has long published its partial: each consumer thread loads up to 3 partial
+//     float4s of one of this CTA's column groups at the start of a step and sums them (fixed
+//     order: thread, warp butterfly, warps) at its end, so the loads fly under the record
+//     stream; y is written once.
+//   * warp 17 (signalling) does the grid-scope fence + atomics that publish "partial of step s
+//     stored" and "partials of step s - kLag consumed"; warp 18 (watcher) is the only thread
+//     that polls those counters and mirrors them into shared-memory barriers.
 //
 // Every wait is bounded: on expiry the kernel records SI_ERR_TIMEOUT, raises a grid-wide
 // abort flag, lets its outstanding copies land and returns.
@@ -36,14 +35,19 @@
 
 namespace si_persist {
 
-constexpr int kConsumers = 512;
+constexpr int kSets = 2;                          // independent consumer sets, each with its own ring
+constexpr int kSetWarps = 8;
+constexpr int kSetThreads = kSetWarps * 32;
+constexpr int kConsumers = kSets * kSetThreads;
 constexpr int kConsumerWarps = kConsumers / 32;
-static_assert(kConsumerWarps == 16, "consumer warps are arranged as 4 records x 4 column quarters");
-constexpr int kThreads = 32 + kConsumers + 64;    // producer warp, consumers, signalling warp, watcher warp
+constexpr int kReducerWarps = 2;
+constexpr int kThreads = 32 + kConsumers + 32 * kReducerWarps + 32;   // producer, consumers, reducers, watcher
+constexpr int kLandBytes = 8 * 1024;              // per reducer warp: landing area for partial-y rows
+constexpr int kMaxGroups = 8;                     // float4 column groups one CTA reduces (d_model / 4 / SMs, rounded up)
 constexpr int kFlagRing = 8;                      // per-step shared-memory flags kept for this many steps
 constexpr int kCounterStride = 64;                // uint32 per step: written at +0, reduced at +32 (own 128-byte lines)
 constexpr int kMaxStages = 16;
-constexpr int kDescRing = 128;                    // copy descriptors kept ahead of the issue lanes
+constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
 constexpr int kPartialDepth = 6;                  // D: partial-y buffers in flight
 constexpr int kLag = 2;                           // a step's cross-SM reduction starts this many steps later
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
@@ -211,17 +215,16 @@ __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, 
 }
 
 struct Smem {
-    uint64_t full[kMaxStages];
+    uint64_t full[kMaxStages];         // stage index = set * S + stage-in-set
     uint64_t empty[kMaxStages];
-    uint64_t redbar[2];            // consumer warps' partial dot products are in part[buf]
-    uint64_t stepbar[kPartialDepth];   // consumers stored the partial y of step s (slot s mod D)
+    uint64_t setbar[kSets][2];         // a set's warps have published their dot-product partials
+    uint64_t accfull, accempty;        // set 1 -> set 0 hand-over of a step's accumulators
+    uint64_t stepbar[kPartialDepth];   // all consumer warps are done with step s (slot s mod D)
+    uint64_t pubbar[kFlagRing];        // every CTA has published its partial of step s (slot s mod ring)
+    uint64_t freebar[kFlagRing];       // every CTA has finished reading the partials of step s
     int meta[kMaxStages];
-    uint4 desc[kDescRing];         // {src lo, src hi, bytes (0: nothing to copy), meta}
-    float part[2][2 * kConsumerWarps];   // [buf][record*8 + quarter*2 + (gate|up)]
-    uint64_t ybar[2];              // redy[buf] is complete
-    uint64_t pubbar[kFlagRing];    // every CTA has published its partial of step s (slot s mod ring)
-    uint64_t freebar[kFlagRing];   // every CTA has finished reading the partials of step s
-    float4 redy[2][64];            // warp-level sums of a step's column groups
+    uint4 desc[kSets][kDescRing];      // {src lo, src hi, bytes (0: nothing to copy), meta}
+    float2 setpart[kSets][2][kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products
     volatile int cta_abort;
 };
 
@@ -233,27 +236,30 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
     }
 }
 
-template <int DT, int NCH, int NQ, int NRL>
-__global__ void __launch_bounds__(kThreads, 1)   // 18 warps: at most 96 registers per thread
+template <int DT, int NCH>
+__global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int rec_bytes = P.d_model * 6;
-    const int nstage = P.nstage;
+    const int nstage = P.nstage;               // total over both sets (even)
+    const int S = nstage / kSets;              // ring stages per consumer set
     uint8_t *ring = smem;
-    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)nstage * rec_bytes);
+    float *accbuf = reinterpret_cast<float *>(smem + (size_t)nstage * rec_bytes);   // set 1 -> set 0, d_model floats
+    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)nstage * rec_bytes + (size_t)P.d_model * 4);
     uint64_t *full = sm->full, *empty = sm->empty;
     int *meta = sm->meta;
     volatile int *cta_abort = &sm->cta_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, b = blockIdx.x;
+    const int Gv = G * kSets;                  // consumer sets act as virtual CTAs 2b, 2b+1 of 2G
     const int d = P.d_model, chunks = P.chunks;
 
     if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConsumerWarps); }
-        mbar_init(&sm->redbar[0], kConsumerWarps); mbar_init(&sm->redbar[1], kConsumerWarps);
+        for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
+        for (int q = 0; q < kSets; ++q) { mbar_init(&sm->setbar[q][0], kSetWarps); mbar_init(&sm->setbar[q][1], kSetWarps); }
+        mbar_init(&sm->accfull, kSetWarps); mbar_init(&sm->accempty, kSetWarps);
         for (int s = 0; s < kPartialDepth; ++s) mbar_init(&sm->stepbar[s], kConsumerWarps);
-        mbar_init(&sm->ybar[0], kConsumerWarps); mbar_init(&sm->ybar[1], kConsumerWarps);
         for (int s = 0; s < kFlagRing; ++s) { mbar_init(&sm->pubbar[s], 1); mbar_init(&sm->freebar[s], 1); }
         sm->cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -262,118 +268,116 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer warp
-        // Two jobs share this warp.
-        //  (1) Descriptor walk: the warp walks the CTA's items in order, 32 at a time (lane l
-        //      takes item wn + l), loads the slot indices with one coalesced round of loads
-        //      issued a full window early, and writes {source address, bytes, meta} into a
+        // Each consumer set has its own ring of S stages and its own item stream: per step one
+        // x item, then the records of virtual CTA 2b+set.  Two jobs share this warp.
+        //  (1) Descriptor walk: half-warp h walks set h's items in order, 16 at a time (lane l
+        //      takes item wn + l), loads the slot indices with one round of loads issued a
+        //      full window early, and writes {source address, bytes, meta} into the set's
         //      shared-memory descriptor ring.
-        //  (2) Issue: lane j < nstage owns ring stage j and issues every item n = j (mod
-        //      nstage) at its own pace: in each polling pass every lane whose stage is free
-        //      arms the barrier and starts its bulk copy.  One thread issuing alone cannot keep
-        //      an SM's share of HBM busy; here as many lanes issue together as stages are free.
+        //  (2) Issue: lane j < 2S owns ring stage j and issues that stage's items at its own
+        //      pace: in each polling pass every lane whose stage is free arms the barrier and
+        //      starts its bulk copy.
         const uint64_t policy = l2_policy_evict_first();
-        const bool mine = lane < nstage;
-        uint32_t n = lane;             // ring item index this lane issues next
+        const unsigned FULL = 0xFFFFFFFFu;
+        const int hq = lane >> 4, hl = lane & 15;      // walker role
+        const bool mine = lane < kSets * S;            // issue role
+        const int iq = mine ? lane / S : 0, is = lane % S;
+        uint32_t n = is;                               // set-ring item index this lane issues next
         uint32_t issued = 0;
-        // walker: item wn is item wt of step wstep (t = 0 is x, t >= 1 is record t - 1)
+        // walker (uniform within a half-warp): item wn is item wt of step wstep (t = 0 is x)
         uint32_t wn = 0, desc_ready = 0, total = 0xFFFFFFFFu;
         int wstep = 0, wt = 0;
-        // per-lane prefetched descriptor of item wn + lane
         unsigned long long pf_src = 0; uint32_t pf_bytes = 0; int pf_meta = 0; bool pf_valid = false;
-        bool pf_pending = false;       // a window has been prefetched and not yet committed
-        auto prefetch_window = [&]() {
-            // lane l: locate item (wstep, wt + l)
-            int step = wstep, t = wt + lane;
-            StepGeom g;
-            bool in = step < P.n_steps;
-            if (in) g = step_geom(P, step, G, b);
-            while (in && t > g.cnt) {
-                t -= g.cnt + 1; ++step;
+        bool pf_pending = false;
+        const int vb = kSets * b + hq;
+        auto prefetch_window = [&](bool doit) {
+            int step = wstep, t = wt + hl;
+            bool in = false;
+            if (doit) {
+                StepGeom g;
                 in = step < P.n_steps;
-                if (in) g = step_geom(P, step, G, b);
-            }
-            pf_valid = in;
-            if (in) {
-                const int layer = P.step_layers ? __ldg(P.step_layers + step) : step % P.n_layers;
-                if (t == 0) {
-                    pf_src = (unsigned long long)(P.x + (size_t)step * d);
-                    pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
-                } else {
-                    const int slot = __ldg(P.idx + g.base + g.first + (long long)(t - 1) * G);
-                    const bool valid = slot >= 0 && slot < P.n_loaded[layer];
-                    pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
-                    pf_bytes = valid ? (uint32_t)rec_bytes : 0u; pf_meta = valid ? 1 : 0;
+                if (in) g = step_geom(P, step, Gv, vb);
+                while (in && t > g.cnt) {
+                    t -= g.cnt + 1; ++step;
+                    in = step < P.n_steps;
+                    if (in) g = step_geom(P, step, Gv, vb);
+                }
+                pf_valid = in;
+                if (in) {
+                    const int layer = P.step_layers ? __ldg(P.step_layers + step) : step % P.n_layers;
+                    if (t == 0) {
+                        pf_src = (unsigned long long)(P.x + (size_t)step * d);
+                        pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
+                    } else {
+                        const int slot = __ldg(P.idx + g.base + g.first + (long long)(t - 1) * Gv);
+                        const bool valid = slot >= 0 && slot < P.n_loaded[layer];
+                        pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
+                        pf_bytes = valid ? (uint32_t)rec_bytes : 0u; pf_meta = valid ? 1 : 0;
+                    }
                 }
             }
-            // the walker moves on by the 32 items of this window: continue after lane 31's item
-            const int s31 = __shfl_sync(0xFFFFFFFFu, step, 31), t31 = __shfl_sync(0xFFFFFFFFu, t, 31);
-            const unsigned vmask = __ballot_sync(0xFFFFFFFFu, pf_valid);
-            if (vmask != 0xFFFFFFFFu) total = wn + __popc(vmask);     // the list of items ends in this window
-            wstep = s31; wt = t31 + 1;
-            pf_pending = true;
+            // the walker moves on by the 16 items of this window: continue after lane 15's item
+            const int s15 = __shfl_sync(FULL, step, (lane & 16) | 15), t15 = __shfl_sync(FULL, t, (lane & 16) | 15);
+            const unsigned vmask = (__ballot_sync(FULL, doit && pf_valid) >> (hq * 16)) & 0xFFFFu;
+            if (doit) {
+                if (vmask != 0xFFFFu) total = wn + __popc(vmask);     // the item list ends in this window
+                wstep = s15; wt = t15 + 1;
+                pf_pending = true;
+            }
         };
-        auto commit_window = [&]() {
-            if (pf_valid) {
-                uint4 dsc;
-                dsc.x = (uint32_t)pf_src; dsc.y = (uint32_t)(pf_src >> 32); dsc.z = pf_bytes; dsc.w = (uint32_t)pf_meta;
-                sm->desc[(wn + lane) % kDescRing] = dsc;
+        auto commit_window = [&](bool doit) {
+            if (doit) {
+                if (pf_valid) {
+                    uint4 dsc;
+                    dsc.x = (uint32_t)pf_src; dsc.y = (uint32_t)(pf_src >> 32); dsc.z = pf_bytes; dsc.w = (uint32_t)pf_meta;
+                    sm->desc[hq][(wn + hl) % kDescRing] = dsc;
+                }
+                wn += 16;
+                desc_ready = wn < total ? wn : total;
+                pf_pending = false;
             }
             __syncwarp();
-            wn += 32;
-            desc_ready = wn < total ? wn : total;
-            pf_pending = false;
         };
-        prefetch_window(); commit_window();
-        if (desc_ready < total) prefetch_window();
+        prefetch_window(true); commit_window(true);
+        prefetch_window(desc_ready < total);
 
         bool ok = true;
         long long t_last = clock64();
         while (true) {
-            const bool have = mine && n < total;
-            if (!__any_sync(0xFFFFFFFFu, have)) break;
-            // keep the descriptor ring ahead of the slowest lane by at least one window
-            const uint32_t n_min = __reduce_min_sync(0xFFFFFFFFu, mine ? n : 0xFFFFFFFFu);
-            if (pf_pending && desc_ready - n_min <= kDescRing - 32 - kMaxStages) {
-                commit_window();
-                if (desc_ready < total) prefetch_window();
+            // issue lanes need their set's walker state
+            const uint32_t i_ready = __shfl_sync(FULL, desc_ready, iq * 16);
+            const uint32_t i_total = __shfl_sync(FULL, total, iq * 16);
+            const bool have = mine && n < i_total;
+            if (!__any_sync(FULL, have)) break;
+            // keep each descriptor ring ahead of its set's slowest issue lane by at least a window
+            uint32_t n_min = 0xFFFFFFFFu;
+            for (int k = 0; k < S; ++k) {
+                const uint32_t v = __shfl_sync(FULL, n, hq * S + k);
+                n_min = v < n_min ? v : n_min;
             }
+            const bool do_commit = pf_pending && desc_ready - n_min <= (uint32_t)(kDescRing - 16 - kMaxStages);
+            commit_window(do_commit);
+            prefetch_window(do_commit && desc_ready < total);
             bool progressed = false;
-            if (have && n < desc_ready) {
-                const int st = lane; const uint32_t ph = (n / nstage) & 1;
+            if (have && n < i_ready) {
+                const int st = iq * S + is; const uint32_t ph = (n / S) & 1;
                 if (mbar_test_wait(&empty[st], ph ^ 1)) {
-                    const uint4 dsc = sm->desc[n % kDescRing];
+                    const uint4 dsc = sm->desc[iq][n % kDescRing];
                     meta[st] = (int)dsc.w;
                     if (dsc.z != 0) {
                         mbar_arrive_expect_tx(&full[st], dsc.z);
-                        const void *src = (const void *)(((unsigned long long)dsc.y << 32) | dsc.x);
-                        if (P.stream_only & 8) {   // diagnostics: uniformly random records of layer 0
-                            unsigned long long r = ((unsigned long long)n * 2654435761ull + (unsigned long long)b * 40503ull) % (unsigned long long)P.n_loaded[0];
-                            src = P.store_base + P.rec_off[0] + r * rec_bytes;
-                        }
-                        if (P.stream_only & 16)
-                            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                         ::"r"(smem_u32(ring + (size_t)st * rec_bytes)), "l"(src), "r"(dsc.z), "r"(smem_u32(&full[st])) : "memory");
-                        else
-                        bulk_g2s(ring + (size_t)st * rec_bytes, src, dsc.z, &full[st], policy);
+                        bulk_g2s(ring + (size_t)st * rec_bytes,
+                                 (const void *)(((unsigned long long)dsc.y << 32) | dsc.x), dsc.z, &full[st], policy);
                     } else {
                         if (P.status) atomicCAS(P.status, 0, SI_ERR_OUT_OF_RANGE);
                         mbar_arrive(&full[st]);
                     }
                     ++issued;
-                    // pull a later item of this lane from HBM into L2 now, so that its copy into
-                    // shared memory later pays the L2 latency rather than the loaded-HBM latency
-                    const uint32_t npf = n + (uint32_t)(P.prefetch_rounds * nstage);
-                    if (P.prefetch_rounds > 0 && npf < desc_ready) {
-                        const uint4 pd = sm->desc[npf % kDescRing];
-                        if (pd.z != 0)
-                            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;"
-                                         ::"l"(((unsigned long long)pd.y << 32) | pd.x), "r"(pd.z) : "memory");
-                    }
-                    n += nstage;
+                    n += S;
                     progressed = true;
                 }
             }
-            if (__any_sync(0xFFFFFFFFu, progressed)) {
+            if (__any_sync(FULL, progressed)) {
                 t_last = clock64();
             } else if (*cta_abort || clock64() - t_last > kWaitCycles) {
                 ok = false;
@@ -383,273 +387,177 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
         // never leave the CTA while a copy into its shared memory is still in flight
         if (mine && issued > 0) {
-            const uint32_t last = n - nstage;      // ring index of this lane's last issued item
-            const uint32_t ph = (last / nstage) & 1;
+            const uint32_t last = n - S;           // set-ring index of this lane's last issued item
+            const uint32_t ph = (last / S) & 1;
             long long t0 = clock64();
-            while (!mbar_try_wait(&full[lane], ph) && clock64() - t0 < kWaitCycles) {}
+            while (!mbar_try_wait(&full[iq * S + is], ph) && clock64() - t0 < kWaitCycles) {}
         }
         return;
     }
 
     if (warp <= kConsumerWarps) {
         // ------------------------------------------------------------------ consumers
-        // Records are taken in batches of four.  Dot products: consumer warp (wr, wq) handles
-        // record wr of the batch over column quarter wq, with its slice of x in registers,
-        // so the four records' dots run in independent warps and need no CTA-wide exchange
-        // beyond 32 floats.  Down projection: thread ct owns output columns of chunk
-        // ct + 512*q and accumulates all four records.
+        // Two independent sets of 8 warps; set q consumes ring q.  A landed record is copied
+        // into registers (3*NCH 16-byte chunks per thread) and its stage handed back at once;
+        // the arithmetic then runs out of registers, so the ring is refilled while the set
+        // computes.  Thread t of a set owns chunks t, t+256 of every row.
         const int ct = tid - 32;                 // 0..511
-        const int cw = ct >> 5;                  // consumer warp 0..15
-        const int wr = cw >> 2, wq = cw & 3;
-        const int cq = chunks >> 2;              // 16-byte chunks per column quarter
-        uint32_t n = 0;                          // ring item counter
-        uint32_t batches = 0;                    // batches handed to the split-phase barrier so far
+        const int q = ct >> 8;                   // consumer set
+        const int t = ct & (kSetThreads - 1);    // thread within the set
+        const int sw = t >> 5;                   // warp within the set
+        uint64_t *sfull = full + q * S, *sempty = empty + q * S;
+        int *smeta = meta + q * S;
+        uint8_t *sring = ring + (size_t)q * S * rec_bytes;
+        uint32_t n = 0;                          // set-ring item counter
+        uint32_t recs = 0;                       // records this set has handed to its barrier
         bool fail = false;
-        if (P.stream_only & 32) {   // diagnostics: drain the ring item by item, nothing else
-            for (int step = 0; step < P.n_steps; ++step) {
-                int st = n % nstage; uint32_t ph = (n / nstage) & 1;
-                if (!mbar_wait_bounded(&full[st], ph, cta_abort)) return;
-                const int cnt = meta[st];
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);
-                ++n;
-                for (int i = 0; i < cnt; ++i) {
-                    st = n % nstage; ph = (n / nstage) & 1;
-                    if (!mbar_wait_bounded(&full[st], ph, cta_abort)) return;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[st]);
-                    ++n;
-                }
-            }
-            return;
-        }
         const bool prof = P.prof != nullptr && ct == 0;
         long long pf[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pt = prof ? clock64() : 0;
 #define SI_PROF(slot) do { if (prof) { long long now_ = clock64(); pf[slot] += now_ - pt; pt = now_; } } while (0)
 
-        // split-K reduction geometry: this CTA reduces column groups [b*gpc, (b+1)*gpc) of
-        // every step; TPG threads share one group, thread pl of them sums partials pl, pl+TPG, ...
-        const int ngroups = d / 4;                 // float4 column groups
-        const int gpc = (ngroups + G - 1) / G;     // groups per CTA
-        int GP = 1; while (GP < gpc) GP <<= 1;     // padded to a power of two (<= 512 by the launch check)
-        const int TPG = kConsumers / GP;
-        const int WL = TPG < 32 ? TPG : 32;        // lanes of one warp that share a group
-        const int rgi = ct / TPG, rpl = ct % TPG;
-        const int rgrp = b * gpc + rgi;
-        const bool ractive = rgi < gpc && rgrp < ngroups;
         const bool nosync = (P.stream_only & 4) != 0;   // diagnostics: no cross-CTA exchange at all
+        const bool noarith = (P.stream_only & 1) != 0;  // diagnostics: drain only
 
-        // Steps n_steps .. n_steps + kLag - 1 are flush iterations: no records, they only finish
-        // the reductions that are still in flight.
-        for (int step = 0; step <= P.n_steps + kLag && !fail; ++step) {
-            const bool real = step < P.n_steps;
-            // ---- [A0] write y of step (step-1-kLag): its group sums are in redy[(step-1) & 1]
-            if (step - 1 >= kLag && !(P.stream_only & 128)) {
-                const int sy = step - 1 - kLag, yb = (step - 1 - kLag) & 1;
-                fail |= !mbar_wait_warp(&sm->ybar[yb], (uint32_t)(((step - 1 - kLag) >> 1) & 1), cta_abort, lane);
-                if (!fail && ct < GP && ct < gpc && b * gpc + ct < ngroups) {
-                    const int W = TPG / WL;
-                    float4 v = sm->redy[yb][ct * W];
-                    for (int w = 1; w < W; ++w) {
-                        const float4 t4 = sm->redy[yb][ct * W + w];
-                        v.x += t4.x; v.y += t4.y; v.z += t4.z; v.w += t4.w;
-                    }
-                    const size_t col = (size_t)sy * d + (size_t)(b * gpc + ct) * 4;
-                    if (P.residual) {
-                        uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
-                        v.x += si_cvt<DT>::lo(xw.x); v.y += si_cvt<DT>::hi(xw.x);
-                        v.z += si_cvt<DT>::lo(xw.y); v.w += si_cvt<DT>::hi(xw.y);
-                    }
-                    if (P.y_f32) {
-                        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + col) = v;
-                    } else {
-                        uint2 o;
-                        o.x = (uint32_t)si_cvt<DT>::from_float(v.x) | ((uint32_t)si_cvt<DT>::from_float(v.y) << 16);
-                        o.y = (uint32_t)si_cvt<DT>::from_float(v.z) | ((uint32_t)si_cvt<DT>::from_float(v.w) << 16);
-                        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(P.y) + col) = o;
-                    }
-                }
-            }
-            if (step == P.n_steps + kLag || fail) break;
-
-            // ---- [A1] start the reduction of step sr = step - kLag: every CTA has published its
-            // partial of that step long ago; the loads fly while this step's records are processed
-            float4 rv[NRL];
+        for (int step = 0; step < P.n_steps && !fail; ++step) {
+            const bool real = true;
+            float xr[NCH][8], acc[NCH][8];
 #pragma unroll
-            for (int j = 0; j < NRL; ++j) rv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (step >= kLag && !(P.stream_only & 128)) {
-                const int sr = step - kLag;
-                if (!nosync) fail |= !mbar_wait_warp(&sm->pubbar[sr % kFlagRing], (sr / kFlagRing) & 1, cta_abort, lane);
-                if (fail) break;
-                if (ractive && (P.stream_only & 6) == 0) {
-                    const float *col = P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)rgrp * 4;
+            for (int i = 0; i < NCH; ++i)
 #pragma unroll
-                    for (int j = 0; j < NRL; ++j) {
-                        const int gg = rpl + TPG * j;
-                        if (gg < G) rv[j] = __ldcg(reinterpret_cast<const float4 *>(col + (size_t)gg * d));
-                    }
-                }
-            }
-            SI_PROF(5);                                   // reduction: wait for publication, issue loads
-
-            float xr[NQ][8], acc[NCH][8];
-            int cnt = 0;
-#pragma unroll
-            for (int q = 0; q < NCH; ++q)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[q][e] = 0.f;
+                for (int e = 0; e < 8; ++e) { acc[i][e] = 0.f; xr[i][e] = 0.f; }
             if (real) {
-                int st = n % nstage; uint32_t ph = (n / nstage) & 1;
-                fail |= !mbar_wait_warp(&full[st], ph, cta_abort, lane);
-                cnt = fail ? 0 : meta[st];
-                const uint4 *xs = reinterpret_cast<const uint4 *>(ring + (size_t)st * rec_bytes) + wq * cq;
+                int cnt;
+                {   // x item
+                    const int st = n % S; const uint32_t ph = (n / S) & 1;
+                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
+                    cnt = fail ? 0 : smeta[st];
+                    const uint4 *xs = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
 #pragma unroll
-                for (int j = 0; j < NQ; ++j) {
-                    int c = lane + 32 * j;
-                    uint4 v = c < cq ? xs[c] : make_uint4(0, 0, 0, 0);
-                    unpack8<DT>(v, xr[j]);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);
-                ++n;
-            }
-            SI_PROF(0);                                   // wait for x
-
-            // software pipeline over batches: the dot products of batch i are handed to the
-            // warps' barrier and finished (summed, SiLU, down accumulate) while batch i+1 loads
-            uint4 dnp[4][NCH];                            // down chunks of the pending batch
-            bool pend = false;
-            uint32_t pbatch = 0;
-            auto finish_pending = [&]() {
-                const uint32_t buf = pbatch & 1, par = (pbatch >> 1) & 1;
-                fail |= !mbar_wait_warp(&sm->redbar[buf], par, cta_abort, lane);
-                // part[buf] holds 32 floats, index r*8 + quarter*2 + (0: gate, 1: up)
-                float v = reinterpret_cast<const float *>(sm->part[buf])[lane];
-                v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-                v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
-                const float u = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-                const float hh = si_silu_mul(v, u);       // meaningful on lanes 0, 8, 16, 24
-                float h[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) h[r] = __shfl_sync(0xFFFFFFFFu, hh, r * 8);
-#pragma unroll
-                for (int q = 0; q < NCH; ++q) {
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        float f[8];
-                        unpack8<DT>(dnp[r][q], f);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[q][e] = fmaf(h[r], f[e], acc[q][e]);
+                    for (int i = 0; i < NCH; ++i) {
+                        const int c = t + kSetThreads * i;
+                        if (c < chunks) unpack8<DT>(xs[c], xr[i]);
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sempty[st]);
+                    ++n;
                 }
-            };
-
-            for (int i = 0; i < cnt && !fail; i += 4) {
-                const int nb = cnt - i < 4 ? cnt - i : 4;
-                // the previous batch's warps have all published their dot products by now (or
-                // will within a few cycles): finish it before its down chunks are overwritten
-                if (pend && !(P.stream_only & 64)) finish_pending();
-                // ---- take the batch's records one by one as they land; a stage is handed
-                // back as soon as this warp has what it needs from it, so the ring refills early
-                float g = 0.f, u = 0.f;
+                SI_PROF(0);                               // wait for x
+                for (int i = 0; i < cnt && !fail; ++i) {
+                    const int st = n % S; const uint32_t ph = (n / S) & 1;
+                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
+                    const bool okr = !fail && smeta[st] != 0 && !noarith;
+                    // ---- copy this thread's chunks of the record into registers, free the stage
+                    const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
+                    uint4 ga[NCH], up[NCH], dn[NCH];
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const uint32_t m = n + r;
-                    const int st = m % nstage; const uint32_t ph = (m / nstage) & 1;
-                    bool okr = false;
-                    if (r < nb) {
-                        fail |= !mbar_wait_warp(&full[st], ph, cta_abort, lane);
-                        okr = !fail && meta[st] != 0 && (P.stream_only & 1) == 0;
+                    for (int k2 = 0; k2 < NCH; ++k2) {
+                        const int c = t + kSetThreads * k2;
+                        const bool in = okr && c < chunks;
+                        ga[k2] = in ? rr[c] : make_uint4(0, 0, 0, 0);
+                        up[k2] = in ? rr[chunks + c] : make_uint4(0, 0, 0, 0);
+                        dn[k2] = in ? rr[2 * chunks + c] : make_uint4(0, 0, 0, 0);
                     }
-                    const uint4 *rr = reinterpret_cast<const uint4 *>(ring + (size_t)st * rec_bytes);
-                    if (r == wr && okr) {
-                        // dot products of this warp's record over this warp's column quarter
-                        const uint4 *r0 = rr + wq * cq;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sempty[st]);
+                    ++n;
+                    SI_PROF(1);                           // wait for the record + copy out
+                    // ---- dot products: thread slice, warp butterfly (lane 0 <- gate, lane 16 <- up)
+                    float g = 0.f, u = 0.f;
 #pragma unroll
-                        for (int j = 0; j < NQ; ++j) {
-                            int c = lane + 32 * j;
-                            if (c < cq) {
-                                uint4 a = r0[c], bb = r0[chunks + c];
-                                g += dot8<DT>(a, xr[j]); u += dot8<DT>(bb, xr[j]);
-                            }
+                    for (int k2 = 0; k2 < NCH; ++k2) { g += dot8<DT>(ga[k2], xr[k2]); u += dot8<DT>(up[k2], xr[k2]); }
+                    {
+                        const bool hi16 = (lane & 16) != 0;
+                        float keep = (hi16 ? u : g) + __shfl_xor_sync(0xFFFFFFFFu, hi16 ? g : u, 16);
+                        keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 8);
+                        keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 4);
+                        keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 2);
+                        keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 1);
+                        g = keep;
+                    }
+                    // ---- exchange among the set's 8 warps (double-buffered, one barrier per record)
+                    const uint32_t buf = recs & 1, par = (recs >> 1) & 1;
+                    if ((lane & 15) == 0) reinterpret_cast<float *>(&sm->setpart[q][buf][sw])[lane >> 4] = g;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->setbar[q][buf]);
+                    fail |= !mbar_wait_bounded(&sm->setbar[q][buf], par, cta_abort);
+                    ++recs;
+                    float gs = 0.f, us = 0.f;
+                    {
+                        const float4 *pp = reinterpret_cast<const float4 *>(sm->setpart[q][buf]);
+#pragma unroll
+                        for (int w = 0; w < kSetWarps / 2; ++w) {
+                            const float4 v4 = pp[w];
+                            gs += v4.x; us += v4.y; gs += v4.z; us += v4.w;
                         }
                     }
-                    // down row of the record for this thread's columns
+                    const float h = okr ? si_silu_mul(gs, us) : 0.f;
 #pragma unroll
-                    for (int q = 0; q < NCH; ++q) {
-                        int c = ct + kConsumers * q;
-                        dnp[r][q] = (okr && c < chunks) ? rr[2 * chunks + c] : make_uint4(0, 0, 0, 0);
-                    }
-                    if (r < nb) {
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&empty[st]);
-                    }
-                }
-                SI_PROF(1);                               // records: wait, dots, down loads
-                n += nb;
-                if (P.stream_only & 64) continue;
-                // lane 0 <- sum(g), lane 16 <- sum(u): five shuffles, fixed order
-                {
-                    const bool hi16 = (lane & 16) != 0;
-                    float keep = (hi16 ? u : g) + __shfl_xor_sync(0xFFFFFFFFu, hi16 ? g : u, 16);
-                    keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 8);
-                    keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 4);
-                    keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 2);
-                    keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 1);
-                    g = keep;
-                }
-                const uint32_t buf = batches & 1;
-                if ((lane & 15) == 0) reinterpret_cast<float *>(sm->part[buf])[cw * 2 + (lane >> 4)] = g;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->redbar[buf]);
-                pend = true; pbatch = batches;
-                ++batches;
-                SI_PROF(2);                               // publish dot products
-            }
-            if (pend && !fail && !(P.stream_only & 64)) finish_pending();
-            SI_PROF(2);
-            if (fail) break;
-
-            // ---- [C1] finish the reduction of step sr: thread sum, warp butterfly over the WL
-            // lanes that share a group (fixed order), warp-level sums to shared memory
-            if (step >= kLag && !(P.stream_only & 128)) {
-                float4 v = rv[0];
+                    for (int k2 = 0; k2 < NCH; ++k2) {
+                        float f[8];
+                        unpack8<DT>(dn[k2], f);
 #pragma unroll
-                for (int j = 1; j < NRL; ++j) { v.x += rv[j].x; v.y += rv[j].y; v.z += rv[j].z; v.w += rv[j].w; }
-                for (int o = WL >> 1; o > 0; o >>= 1) {
-                    v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, o); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, o);
-                    v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, o); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, o);
+                        for (int e = 0; e < 8; ++e) acc[k2][e] = fmaf(h, f[e], acc[k2][e]);
+                    }
+                    SI_PROF(2);                           // record arithmetic
                 }
-                const int sr = step - kLag;
-                if ((ct % WL) == 0) sm->redy[sr & 1][ct / WL] = v;
+                if (fail) break;
             }
-            SI_PROF(3);                                   // reduction: sums
 
-            // ---- [C2] store the partial y of this step into the ring of D buffers
-            if (real) {
-                if (step >= kPartialDepth && !nosync) {
-                    const int q = step - kPartialDepth;
-                    fail |= !mbar_wait_warp(&sm->freebar[q % kFlagRing], (q / kFlagRing) & 1, cta_abort, lane);
+            // ---- merge the two sets' accumulators through shared memory (set 1 -> set 0)
+            {
+                const uint32_t sp = (uint32_t)(step & 1);
+                if (q == 1) {
+                    fail |= !mbar_wait_bounded(&sm->accempty, sp ^ 1, cta_abort);
+#pragma unroll
+                    for (int k2 = 0; k2 < NCH; ++k2) {
+                        const int c = t + kSetThreads * k2;
+                        if (c < chunks) {
+                            float4 *o = reinterpret_cast<float4 *>(accbuf + (size_t)c * 8);
+                            o[0] = make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]);
+                            o[1] = make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->accfull);
+                } else {
+                    fail |= !mbar_wait_bounded(&sm->accfull, sp, cta_abort);
+#pragma unroll
+                    for (int k2 = 0; k2 < NCH; ++k2) {
+                        const int c = t + kSetThreads * k2;
+                        if (c < chunks) {
+                            const float4 *o = reinterpret_cast<const float4 *>(accbuf + (size_t)c * 8);
+                            const float4 a0 = o[0], a1 = o[1];
+                            acc[k2][0] += a0.x; acc[k2][1] += a0.y; acc[k2][2] += a0.z; acc[k2][3] += a0.w;
+                            acc[k2][4] += a1.x; acc[k2][5] += a1.y; acc[k2][6] += a1.z; acc[k2][7] += a1.w;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->accempty);
+                }
+                if (fail) break;
+            }
+            SI_PROF(3);                                   // set merge
+            // ---- [C2] set 0 stores the CTA's partial y of this step into the ring of D buffers
+            if (real && q == 0 && !nosync) {
+                if (step >= kPartialDepth) {
+                    const int fq = step - kPartialDepth;
+                    fail |= !mbar_wait_bounded(&sm->freebar[fq % kFlagRing], (fq / kFlagRing) & 1, cta_abort);
                     if (fail) break;
                 }
-                float *mine = P.partial + ((size_t)(step % kPartialDepth) * G + b) * d;
+                float *mine_p = P.partial + ((size_t)(step % kPartialDepth) * G + b) * d;
 #pragma unroll
-                for (int q = 0; q < NCH; ++q) {
-                    int c = ct + kConsumers * q;
-                    if (c < chunks && !nosync) {
-                        float4 *o = reinterpret_cast<float4 *>(mine + (size_t)c * 8);
-                        __stcg(o, make_float4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]));
-                        __stcg(o + 1, make_float4(acc[q][4], acc[q][5], acc[q][6], acc[q][7]));
+                for (int k2 = 0; k2 < NCH; ++k2) {
+                    const int c = t + kSetThreads * k2;
+                    if (c < chunks) {
+                        float4 *o = reinterpret_cast<float4 *>(mine_p + (size_t)c * 8);
+                        __stcg(o, make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]));
+                        __stcg(o + 1, make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]));
                     }
                 }
             }
-            // ---- [C3] this warp is done with the step: its partial is stored and its loads of
-            // step sr have been consumed
+            // ---- [C3] this warp is done with the step: its set's partial is stored
             __syncwarp();
-            if (lane == 0) {
-                if (step >= kLag && !(P.stream_only & 128)) mbar_arrive(&sm->ybar[(step - kLag) & 1]);
-                if (real) mbar_arrive(&sm->stepbar[step % kPartialDepth]);
-            }
+            if (lane == 0) mbar_arrive(&sm->stepbar[step % kPartialDepth]);
             SI_PROF(4);                                   // partial store
         }
 #undef SI_PROF
@@ -660,22 +568,133 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         return;
     }
 
-    // -------------------------------------------------------------------------- signalling warp
-    // Keeps the grid-scope fences and atomics off the consumers' path: once all consumer warps
-    // are done with step s (partial stored, loads of step s - kLag consumed) it publishes
-    // written[s] and reduced[s - kLag].
-    if (warp == 1 + kConsumerWarps) {
-        if (lane == 0 && (P.stream_only & 4) == 0) {
-            for (int step = 0; step < P.n_steps; ++step) {
-                if (!mbar_wait_bounded(&sm->stepbar[step % kPartialDepth], (step / kPartialDepth) & 1, cta_abort)) {
-                    raise_abort(P, sm, SI_ERR_TIMEOUT);
-                    break;
+    // -------------------------------------------------------------------------- reducer warps
+    // Reducer warp r handles steps s = r (mod 2).  For step s it publishes "partials of step s
+    // stored" (grid-scope fence + atomic, kept off the consumers' path) and then reduces step
+    // sr = s - kLag, which every CTA published long ago: the 2G partial rows of this CTA's column
+    // groups are pulled from L2 into a shared-memory landing area with 16-byte async copies (no
+    // registers held while they fly), each lane sums the rows it fetched in ascending order, a
+    // warp butterfly combines the lanes (fixed order, so deterministic), and y is written once.
+    if (warp <= kConsumerWarps + kReducerWarps) {
+        const int r = warp - 1 - kConsumerWarps;
+        const bool nosync = (P.stream_only & 4) != 0;
+        const int ngroups = d / 4;
+        const int gpc = (ngroups + G - 1) / G;                 // <= kMaxGroups (launch check)
+        const int g_valid = ngroups - b * gpc < gpc ? (ngroups - b * gpc < 0 ? 0 : ngroups - b * gpc) : gpc;
+        float4 *land = reinterpret_cast<float4 *>(smem + (size_t)nstage * rec_bytes + (size_t)P.d_model * 4 + sizeof(Smem) + 64) +
+                       (size_t)r * (kLandBytes / 16);
+        const int rpl = (kLandBytes / 16) / (32 * gpc);        // landing rows per lane and round (>= 1)
+        const int RR = 32 * rpl;
+        long long sig_wait = 0, sig_fence = 0;
+        for (int step = r; step < P.n_steps + kLag; step += kReducerWarps) {
+            int ok = 1;
+            if (step < P.n_steps && !nosync) {
+                if (lane == 0) {
+                    long long c0 = clock64();
+                    ok = mbar_wait_bounded(&sm->stepbar[step % kPartialDepth], (step / kPartialDepth) & 1, cta_abort);
+                    long long c1 = clock64();
+                    if (ok) {
+                        __threadfence();
+                        atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
+                    }
+                    if (P.prof) { sig_wait += c1 - c0; sig_fence += clock64() - c1; }
                 }
-                __threadfence();
-                atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
-                if (step >= kLag) atomicAdd(P.counters + (size_t)(step - kLag) * kCounterStride + 32, 1u);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            }
+            if (ok && step >= kLag && !nosync) {
+                const int sr = step - kLag;
+                if (lane == 0) ok = mbar_wait_bounded(&sm->pubbar[sr % kFlagRing], (sr / kFlagRing) & 1, cta_abort);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (ok) {
+                    float4 v[kMaxGroups];
+#pragma unroll
+                    for (int g = 0; g < kMaxGroups; ++g) v[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float *base = P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4;
+                    if ((P.stream_only & 2) == 0) {
+                        // per round a lane fetches rpl rows through the landing area and one more
+                        // straight into registers; it sums them in ascending row order
+                        for (int r0 = 0; r0 < G; r0 += RR + 32) {
+                            for (int j = 0; j < rpl; ++j) {
+                                const int row = r0 + lane + 32 * j;
+                                if (row < G) {
+                                    const float *src = base + (size_t)row * d;
+                                    float4 *dst = land + (size_t)(lane + 32 * j) * gpc;
+                                    for (int g = 0; g < g_valid; ++g)
+                                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                                                     ::"r"(smem_u32(dst + g)), "l"(src + g * 4) : "memory");
+                                }
+                            }
+                            asm volatile("cp.async.commit_group;" ::: "memory");
+                            float4 xr4[kMaxGroups];
+                            const int xrow = r0 + lane + 32 * rpl;
+#pragma unroll
+                            for (int g = 0; g < kMaxGroups; ++g) {
+                                xr4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (xrow < G && g < g_valid)
+                                    xr4[g] = __ldcg(reinterpret_cast<const float4 *>(base + (size_t)xrow * d) + g);
+                            }
+                            asm volatile("cp.async.wait_group 0;" ::: "memory");
+                            for (int j = 0; j < rpl; ++j) {
+                                const int row = r0 + lane + 32 * j;
+                                if (row < G) {
+                                    const float4 *srcs = land + (size_t)(lane + 32 * j) * gpc;
+#pragma unroll
+                                    for (int g = 0; g < kMaxGroups; ++g) {
+                                        if (g < g_valid) {
+                                            const float4 t4 = srcs[g];
+                                            v[g].x += t4.x; v[g].y += t4.y; v[g].z += t4.z; v[g].w += t4.w;
+                                        }
+                                    }
+                                }
+                            }
+#pragma unroll
+                            for (int g = 0; g < kMaxGroups; ++g) {
+                                v[g].x += xr4[g].x; v[g].y += xr4[g].y; v[g].z += xr4[g].z; v[g].w += xr4[g].w;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int g = 0; g < kMaxGroups; ++g) {
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            v[g].x += __shfl_xor_sync(0xFFFFFFFFu, v[g].x, o); v[g].y += __shfl_xor_sync(0xFFFFFFFFu, v[g].y, o);
+                            v[g].z += __shfl_xor_sync(0xFFFFFFFFu, v[g].z, o); v[g].w += __shfl_xor_sync(0xFFFFFFFFu, v[g].w, o);
+                        }
+                    }
+                    // lane g writes column group g
+                    float4 mine_v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int g = 0; g < kMaxGroups; ++g) if (lane == g) mine_v = v[g];
+                    if (lane < g_valid) {
+                        const size_t col = (size_t)sr * d + (size_t)(b * gpc + lane) * 4;
+                        if (P.residual) {
+                            uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
+                            mine_v.x += si_cvt<DT>::lo(xw.x); mine_v.y += si_cvt<DT>::hi(xw.x);
+                            mine_v.z += si_cvt<DT>::lo(xw.y); mine_v.w += si_cvt<DT>::hi(xw.y);
+                        }
+                        if (P.y_f32) {
+                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + col) = mine_v;
+                        } else {
+                            uint2 o;
+                            o.x = (uint32_t)si_cvt<DT>::from_float(mine_v.x) | ((uint32_t)si_cvt<DT>::from_float(mine_v.y) << 16);
+                            o.y = (uint32_t)si_cvt<DT>::from_float(mine_v.z) | ((uint32_t)si_cvt<DT>::from_float(mine_v.w) << 16);
+                            *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(P.y) + col) = o;
+                        }
+                    }
+                    __syncwarp();
+                    // the partial buffer of step sr may be overwritten once every CTA has said so
+                    if (lane == 0 && sr < P.n_steps - kLag) {
+                        __threadfence();
+                        atomicAdd(P.counters + (size_t)sr * kCounterStride + 32, 1u);
+                    }
+                }
+            }
+            if (!ok) {
+                if (lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
+                break;
             }
         }
+        if (P.prof && lane == 0 && r == 0) { P.prof[(size_t)b * 8 + 6] = sig_wait; P.prof[(size_t)b * 8 + 7] = sig_fence; }
         return;
     }
     // -------------------------------------------------------------------------- watcher warp
@@ -683,55 +702,69 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     // step s" / "all G CTAs have finished reading step s" into shared-memory barriers the
     // consumers wait on.  It cannot run more than kFlagRing steps ahead of the consumers: a
     // step's counters only fill up after this CTA's own consumers have passed that step.
-    if (lane == 0 && (P.stream_only & 4) == 0) {
+    if ((P.stream_only & 4) == 0) {
+        // lanes 0..15 look at the written counters of steps pw .. pw+15, lanes 16..31 at the
+        // reduced counters of steps pr .. pr+15, all in one round of loads; the completed prefix
+        // of each is then signalled in order.
         int pw = 0, pr = 0;                   // next step whose written / reduced counter is awaited
         const int n_red = P.n_steps - kLag;   // reduced[] is signalled for steps 0 .. n_steps-kLag-1
+        const int half = lane >> 4, hl = lane & 15;
         long long t_last = clock64();
         while (pw < P.n_steps || pr < n_red) {
-            bool progressed = false;
-            if (pw < P.n_steps && ld_acquire_gpu(P.counters + (size_t)pw * kCounterStride) >= (unsigned)G) {
-                mbar_arrive(&sm->pubbar[pw % kFlagRing]); ++pw; progressed = true;
+            const int sidx = (half ? pr : pw) + hl;
+            const int lim = half ? n_red : P.n_steps;
+            bool done = false;
+            if (sidx < lim)
+                done = ld_acquire_gpu(P.counters + (size_t)sidx * kCounterStride + (half ? 32 : 0)) >= (unsigned)G;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, done);
+            // number of leading completed steps in each half (at most kFlagRing - 2 at a time)
+            int nw = __ffs(~(m & 0xFFFFu)) - 1, nr = __ffs(~(m >> 16)) - 1;
+            nw = nw < 0 ? 16 : nw; nr = nr < 0 ? 16 : nr;
+            nw = nw > kFlagRing - 2 ? kFlagRing - 2 : nw; nr = nr > kFlagRing - 2 ? kFlagRing - 2 : nr;
+            if (lane == 0) {
+                for (int i = 0; i < nw; ++i) mbar_arrive(&sm->pubbar[(pw + i) % kFlagRing]);
+                for (int i = 0; i < nr; ++i) mbar_arrive(&sm->freebar[(pr + i) % kFlagRing]);
             }
-            if (pr < n_red && ld_acquire_gpu(P.counters + (size_t)pr * kCounterStride + 32) >= (unsigned)G) {
-                mbar_arrive(&sm->freebar[pr % kFlagRing]); ++pr; progressed = true;
+            pw += nw; pr += nr;
+            if (nw | nr) { t_last = clock64(); continue; }
+            int stop = 0;
+            if (lane == 0) {
+                if (*cta_abort || ld_relaxed_gpu(P.ctrl + 1)) stop = 1;
+                else if (clock64() - t_last > kWaitCycles) { raise_abort(P, sm, SI_ERR_TIMEOUT); stop = 1; }
             }
-            if (progressed) { t_last = clock64(); continue; }
-            if (*cta_abort || ld_relaxed_gpu(P.ctrl + 1)) break;
-            if (clock64() - t_last > kWaitCycles) { raise_abort(P, sm, SI_ERR_TIMEOUT); break; }
-            __nanosleep(100);
+            if (__shfl_sync(0xFFFFFFFFu, stop, 0)) break;
+            __nanosleep(50);
         }
     }
 }
 
 inline size_t smem_bytes(int d_model, int nstage) {
-    return (size_t)nstage * d_model * 6 + sizeof(Smem) + 128;
+    return (size_t)nstage * d_model * 6 + (size_t)d_model * 4 + sizeof(Smem) + 64 + (size_t)kReducerWarps * kLandBytes;
 }
 inline int pick_stages(int d_model) {
-    const size_t budget = 227 * 1024 - 1024;
+    const size_t budget = 227 * 1024;
     int n = (int)((budget - smem_bytes(d_model, 0)) / ((size_t)d_model * 6));
     if (n > kMaxStages) n = kMaxStages;
-    return n;
+    return n & ~1;       // split evenly between the two consumer sets
 }
 
 }  // namespace si_persist
 
 // Diagnostics: when set, every persistent launch writes per-CTA cycle counts of the consumer
-// phases (wait x, wait records, arithmetic, wait partial buffer, partial store).
+// phases of set 0 (wait x, wait + copy records, arithmetic, reduction sums, partial store,
+// reduction issue, set merge).
 long long *&si_decode_profile_buffer();
-// Diagnostics: when non-zero, persistent launches only stream the records (practical HBM ceiling).
+// Diagnostics bit mask: 1 = no arithmetic, 2 = no reduction loads, 4 = no cross-CTA exchange.
 int &si_decode_stream_only();
 
 inline bool si_persistent_supported(const si_store *s) {
-    // the split-K reduction lets 512 / pow2ceil(groups per SM) threads share a column group and
-    // gives each of them at most 3 / 5 / 10 partials (d_model <= 4096 / 8192 / 16384)
+    // thread t of a 256-thread set owns chunks t, t+256 of a row (d_model <= 4096); the split-K
+    // reduction lets 512 / pow2ceil(groups per SM) threads share a column group and gives each
+    // of them at most 5 of the 2G partials
     const int chunks = s->d_model / 8, G = s->num_sms;
     const int gpc = (s->d_model / 4 + G - 1) / G;
-    int gp = 1; while (gp < gpc) gp <<= 1;
-    if (gp > 64) return false;
-    const int tpg = si_persist::kConsumers / gp;
-    const int nrl_max = chunks <= 512 ? 3 : chunks <= 1024 ? 5 : 10;
-    return s->n_layers <= SI_MAX_LAYERS && si_persist::pick_stages(s->d_model) >= 3 &&
-           chunks <= si_persist::kConsumers * 4 && (G + tpg - 1) / tpg <= nrl_max;
+    return s->n_layers <= SI_MAX_LAYERS && si_persist::pick_stages(s->d_model) >= 4 &&
+           chunks <= si_persist::kSetThreads * 2 && gpc <= si_persist::kMaxGroups;
 }
 
 // Bytes of the partial-y ring.
@@ -739,9 +772,9 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, int NQ, int NRL>
+template <int DT, int NCH>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, NQ, NRL>;
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
     SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&P};
@@ -773,23 +806,18 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.status = status_dev;
     P.prof = si_decode_profile_buffer();
     P.stream_only = si_decode_stream_only() & 0xFF;
-    P.prefetch_rounds = (si_decode_stream_only() >> 8) & 0xF;
+    P.prefetch_rounds = 0;
     int G = s->num_sms;
     if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
+    // every CTA reduces at most kMaxGroups float4 column groups
+    const int g_min = (s->d_model / 4 + si_persist::kMaxGroups - 1) / si_persist::kMaxGroups;
+    if (G < g_min) G = g_min;
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256, stream));
     SI_CUDA_TRY(cudaMemsetAsync(P.counters, 0, (size_t)n_steps * si_persist::kCounterStride * 4, stream));
-    // NCH: 16-byte column chunks per thread in the down projection (512 threads);
-    // NQ : chunks per lane in the dot products (a warp covers a quarter of the columns)
-    const int nch = (P.chunks + si_persist::kConsumers - 1) / si_persist::kConsumers;
-    const int nq = (P.chunks / 4 + 31) / 32;
-    // NRL: partial-y loads per thread in the split-K reduction (see the kernel)
-#define SI_PL(DT)                                                                     \
-    (nq <= 1 ? si_decode_persistent_launch_t<DT, 1, 1, 3>(P, G, stream)               \
-     : nq <= 2 ? si_decode_persistent_launch_t<DT, 1, 2, 3>(P, G, stream)             \
-     : nq <= 4 ? si_decode_persistent_launch_t<DT, 1, 4, 3>(P, G, stream)             \
-     : nq <= 8 ? si_decode_persistent_launch_t<DT, 2, 8, 5>(P, G, stream)             \
-               : si_decode_persistent_launch_t<DT, 4, 16, 10>(P, G, stream))
-    (void)nch;
+    // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
+    const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
+#define SI_PL(DT) (nch <= 1 ? si_decode_persistent_launch_t<DT, 1>(P, G, stream) \
+                            : si_decode_persistent_launch_t<DT, 2>(P, G, stream))
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
 #undef SI_PL
 }
