@@ -70,6 +70,7 @@ enum {
     SI_FLAG_RESIDUAL = 2u,       /* y = x + FFN(x) instead of FFN(x) */
     SI_FLAG_UNION_UNMASKED = 4u, /* T > 1 only: every token uses the whole union (extension) */
     SI_FLAG_SCORE_ABS = 8u,      /* si_select: rank |score| instead of score */
+    SI_FLAG_SHARED_LIST = 16u,   /* T > 1 only: idx is ONE list of k_fixed slots used by every token */
     SI_FLAG_SIMPLE_KERNELS = 256u /* decode: one plain-load kernel pair per step instead of the
                                      persistent bulk-copy kernel (kept for cross-checking) */
 };

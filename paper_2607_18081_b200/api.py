@@ -22,6 +22,7 @@ SI_OK = 0
 SI_ERR_INVALID_ARG, SI_ERR_OUT_OF_RANGE, SI_ERR_DUPLICATE, SI_ERR_ALIGNMENT = -1, -2, -3, -4
 SI_ERR_NOMEM, SI_ERR_CUDA, SI_ERR_TIMEOUT, SI_ERR_UNSUPPORTED = -5, -6, -7, -8
 SI_FLAG_CHECK, SI_FLAG_RESIDUAL, SI_FLAG_UNION_UNMASKED, SI_FLAG_SCORE_ABS = 1, 2, 4, 8
+SI_FLAG_SHARED_LIST = 16
 SI_FLAG_SIMPLE_KERNELS = 256
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 

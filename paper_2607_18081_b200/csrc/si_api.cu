@@ -11,7 +11,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     int nl_max = 0;
     for (int l = 0; l < s->n_layers; ++l) nl_max = nl_max > s->n_loaded[l] ? nl_max : s->n_loaded[l];
     const size_t nl_pad = si_align_up((size_t)nl_max, 128);
-    const size_t t_pad = si_align_up((size_t)T_max, 16);
+    const size_t t_pad = T_max <= 256 ? si_align_up((size_t)T_max, 16) : si_align_up((size_t)T_max, 256);
     size_t off = 0;
     auto take = [&](size_t &o, size_t &b, size_t bytes) { o = off; b = si_align_up(bytes, 256); off += b; };
     take(w.ctrl_off, w.ctrl_bytes, 256);
@@ -19,7 +19,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     size_t gpart = si_gemm_partial_bytes(s, T_max);
     take(w.partial_off, w.partial_bytes, part > gpart ? part : gpart);
     take(w.sel_off, w.sel_bytes, (size_t)T_max * (size_t)(k_max + 1) * 4);
-    take(w.union_off, w.union_bytes, nl_pad * 4 + 256 + nl_pad / 8 + 256);
+    take(w.union_off, w.union_bytes, T_max > 1 ? nl_pad * 4 + 256 + nl_pad * 4 : 0);   // union, count, slot -> position
     take(w.mask_off, w.mask_bytes, T_max > 1 ? t_pad * (nl_pad / 32) * 4 : 0);
     take(w.h_off, w.h_bytes, T_max > 1 ? t_pad * nl_pad * 2 : 0);
     take(w.selws_off, w.selws_bytes, (size_t)T_max * si_select_ws_bytes_impl(nl_max));
@@ -57,7 +57,8 @@ extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x,
     cudaStream_t stream = (cudaStream_t)stream_;
     if (ws_bytes < si_ws_carve(store, T, k_fixed, 1).total) return SI_ERR_NOMEM;
     if (flags & SI_FLAG_CHECK) {
-        rc = si_check_lists_launch_impl(store, T, layer, nullptr, idx, idx_offsets, k_fixed, status_dev, stream);
+        rc = si_check_lists_launch_impl(store, (flags & SI_FLAG_SHARED_LIST) ? 1 : T, layer, nullptr, idx, idx_offsets,
+                                        k_fixed, status_dev, stream);
         if (rc) return rc;
     }
     if (T == 1) {

@@ -1,0 +1,125 @@
+"""GPU parity: union builder (bit-exact) and the multi-token tensor-core path vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import selectinfer_oracle as so
+from paper_2607_18081_b200 import workloads as wl
+from tests.gpu_utils import LoadedModel, assert_close, from_dev, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2607_18081_b200 import api as _api
+    return _api
+
+
+@pytest.fixture(scope="module")
+def c1(api):
+    return LoadedModel(wl.CONFIGS["c1"])
+
+
+@pytest.fixture(scope="module")
+def m7b(api):
+    return LoadedModel(wl.CONFIGS["c2"], n_layers=1)
+
+
+def _status():
+    return torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+def _run(api, m, layer, x_bits, lists_flat, offsets, k_fixed, T, flags=0, y_dtype=torch.float32):
+    cfg = m.cfg
+    ws = m.store.workspace(T, max(k_fixed, 1), 1)
+    y = torch.full((T, cfg.d_model), 3.0, dtype=y_dtype, device="cuda")
+    st = _status()
+    idx = torch.from_numpy(np.ascontiguousarray(lists_flat, dtype=np.int32)).cuda()
+    off = None if offsets is None else torch.from_numpy(np.ascontiguousarray(offsets, dtype=np.int32)).cuda()
+    api.si_ffn_forward(m.store.handle, layer, to_dev(x_bits, cfg.dtype), T, idx, off, k_fixed, y, flags, ws, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0, api.strerror(int(st.item()))
+    return y
+
+
+def test_union_is_bit_exact(api, c1):
+    cfg = c1.cfg
+    T, k = 5, cfg.k_active
+    lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=c1.slot_of_rank[0])
+    ws = c1.store.workspace(T, k, 1)
+    uni = torch.full((cfg.n_loaded,), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(4, dtype=torch.int32, device="cuda")
+    api.si_union(c1.store.handle, 0, T, torch.from_numpy(lists).cuda(), None, k, uni, cnt, ws)
+    torch.cuda.synchronize()
+    U, mask, overlap, cover = so.union(lists, cfg.n_loaded)
+    n = int(cnt[0].item())
+    assert n == len(U) and np.array_equal(uni[:n].cpu().numpy(), U)
+    assert 0.0 < overlap < 1.0 and cover <= 1.0
+
+
+@pytest.mark.parametrize("T", [2, 4, 16])
+def test_c1_multitoken_matches_per_token_oracle(api, c1, T):
+    cfg = c1.cfg
+    lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=c1.slot_of_rank[0])
+    x = wl.x_tokens(cfg, 0, T)
+    y = _run(api, c1, 0, x, lists, None, cfg.k_active, T)
+    for t in range(T):
+        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], lists[t]), f"T={T} token {t}")
+
+
+def test_c1_ragged_empty_unmasked_residual(api, c1):
+    cfg = c1.cfg
+    n = cfg.n_loaded
+    g = np.random.default_rng(9)
+    lens = [40, 0, 200, n, 1]
+    T = len(lens)
+    lists = [np.sort(g.permutation(n)[:k]).astype(np.int32) for k in lens]
+    offsets = np.zeros(T + 1, np.int32); offsets[1:] = np.cumsum(lens)
+    x = wl.x_tokens(cfg, 0, T, first_token=50)
+    flat = np.concatenate(lists)
+    y = _run(api, c1, 0, x, flat, offsets, n, T, flags=api.SI_FLAG_RESIDUAL | api.SI_FLAG_CHECK)
+    for t in range(T):
+        ref = c1.oracle_y(0, x[t], lists[t]) + wl.bits_to_float64(x[t], cfg.dtype)
+        assert_close(from_dev(y[t]), ref, f"ragged token {t}")
+    # token 1 has an empty list: exactly x
+    assert np.array_equal(from_dev(y[1]), wl.bits_to_float64(x[1], cfg.dtype))
+    # unmasked extension: every token uses the whole union
+    lists3 = [lists[0], lists[2], lists[4]]
+    off3 = np.array([0, 40, 240, 241], np.int32)
+    U, _, _, _ = so.union(lists3, n)
+    y = _run(api, c1, 0, x[:3], np.concatenate(lists3), off3, n, 3, flags=api.SI_FLAG_UNION_UNMASKED)
+    for t in range(3):
+        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], U), f"unmasked token {t}")
+
+
+@pytest.mark.parametrize("T", [4, 32])
+def test_7b_batched_decode_union(api, m7b, T):
+    """Config-3 shape: T tokens with independent Zipf lists over a 7B-shaped layer."""
+    cfg = m7b.cfg
+    k = cfg.k_active
+    lists = wl.zipf_lists(cfg, 0, T)
+    x = wl.x_tokens(cfg, 0, T)
+    y = _run(api, m7b, 0, x, lists, None, k, T)
+    yb = _run(api, m7b, 0, x, lists, None, k, T, y_dtype=torch.bfloat16)
+    for t in sorted({0, 1, T // 2, T - 1}):
+        ref = m7b.oracle_y(0, x[t], lists[t])
+        assert_close(from_dev(y[t]), ref, f"T={T} token {t}")
+        assert_close(from_dev(yb[t]), ref, f"T={T} token {t} bf16 out")
+    # run-to-run bit stability
+    y2 = _run(api, m7b, 0, x, lists, None, k, T)
+    assert torch.equal(y, y2)
+
+
+def test_7b_prefill_shared_list(api, m7b):
+    """Config-4 shape: 512 tokens, one shared list = the first 40 % of the loaded slots."""
+    cfg = wl.CONFIGS["c4"]
+    T, k = 512, cfg.k_active
+    assert k == 3082
+    shared = np.arange(k, dtype=np.int32)
+    x = wl.x_tokens(cfg, 0, T)
+    y = _run(api, m7b, 0, x, shared, None, k, T, flags=api.SI_FLAG_SHARED_LIST)
+    for t in (0, 17, 255, 256, 300, 511):
+        # the model was loaded from the c2 recipe; the oracle uses that model's weights
+        ref = m7b.oracle_y(0, x[t], shared)
+        assert_close(from_dev(y[t]), ref, f"prefill token {t}")
