@@ -97,8 +97,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 __global__ void __launch_bounds__(1024)
 si_union_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int T,
                 int shared_list, int n_loaded, int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out,
-                int32_t *__restrict__ pos_of_slot, uint32_t *__restrict__ masks, int mask_words, int union_cap,
-                int unmasked, int32_t *status) {
+                int32_t *__restrict__ pos_of_slot, int union_cap, int32_t *status) {
     extern __shared__ uint32_t sh[];
     uint32_t *bitmap = sh;                         // [words]
     uint32_t *wprefix = sh + (n_loaded + 31) / 32; // [words] exclusive popcount prefix
@@ -106,7 +105,6 @@ si_union_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ off
     const int words = (n_loaded + 31) / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int w = tid; w < words; w += 1024) bitmap[w] = 0u;
-    for (int i = tid; i < T * mask_words; i += 1024) masks[i] = 0u;
     __syncthreads();
     const int n_lists = shared_list ? 1 : T;
     const int total = offsets ? offsets[n_lists] : n_lists * k_fixed;
@@ -156,27 +154,38 @@ si_union_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ off
         for (int w = 0; w < words; ++w) if (bitmap[w]) { first = w * 32 + __ffs(bitmap[w]) - 1; break; }
         for (int p = n_u + tid; p < union_cap; p += 1024) union_out[p] = first;
     }
-    __threadfence_block();
-    __syncthreads();
-    // membership masks
-    if (unmasked) {
-        for (int i = tid; i < T * mask_words; i += 1024) {
-            int w = i % mask_words;
-            int lo = w * 32;
-            uint32_t m = lo + 32 <= n_u ? 0xFFFFFFFFu : (lo < n_u ? ((1u << (n_u - lo)) - 1u) : 0u);
-            masks[i] = m;
+}
+
+// Membership masks over union positions, many CTAs: mask[t] bit p set iff U[p] is in list t.
+// The masks are zero on entry (memset by the host side of the call).
+__global__ void si_union_masks_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed,
+                                      int T, int shared_list, int n_loaded, const int32_t *__restrict__ n_union,
+                                      const int32_t *__restrict__ pos_of_slot, uint32_t *__restrict__ masks,
+                                      int mask_words, int unmasked) {
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x, gstride = (long long)gridDim.x * blockDim.x;
+    if (unmasked || shared_list) {
+        // every token uses the whole union (with one shared list the union is that list)
+        const int n_u = *n_union;
+        for (long long i = gid; i < (long long)T * mask_words; i += gstride) {
+            const int lo = (int)(i % mask_words) * 32;
+            masks[i] = lo + 32 <= n_u ? 0xFFFFFFFFu : (lo < n_u ? ((1u << (n_u - lo)) - 1u) : 0u);
         }
-    } else {
-        for (int t = 0; t < T; ++t) {
-            int base = shared_list ? 0 : (offsets ? offsets[t] : t * k_fixed);
-            int k = shared_list ? total : (offsets ? offsets[t + 1] - base : k_fixed);
-            for (int e = tid; e < k; e += 1024) {
-                int s = idx[base + e];
-                if (s < 0 || s >= n_loaded) continue;
-                int p = pos_of_slot[s];
-                atomicOr(&masks[(size_t)t * mask_words + (p >> 5)], 1u << (p & 31));
-            }
+        return;
+    }
+    const long long total = offsets ? offsets[T] : (long long)T * k_fixed;
+    for (long long e = gid; e < total; e += gstride) {
+        int t;
+        if (offsets) {            // largest t with offsets[t] <= e
+            int lo = 0, hi = T;
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
+            t = lo;
+        } else {
+            t = (int)(e / k_fixed);
         }
+        const int s = idx[e];
+        if (s < 0 || s >= n_loaded) continue;
+        const int p = pos_of_slot[s];
+        atomicOr(&masks[(size_t)t * mask_words + (p >> 5)], 1u << (p & 31));
     }
 }
 
@@ -340,9 +349,10 @@ template <int DT>
 __global__ void si_gemm_combine_kernel(const float *__restrict__ partial, int n_split, int nu_pad, int t_pad_total,
                                        int T, const int32_t *__restrict__ n_union, const uint32_t *__restrict__ masks,
                                        int mask_words, uint16_t *__restrict__ h) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;       // union position
-    const int t = blockIdx.y;
-    if (i >= nu_pad) return;
+    // threads run over tokens fastest (the partial tiles are [position][token]); H is [token][position]
+    const int t = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int i = blockIdx.y * 8 + (threadIdx.x >> 5);
+    if (i >= nu_pad || t >= t_pad_total) return;
     float out = 0.f;
     if (t < T && i < *n_union && ((masks[(size_t)t * mask_words + (i >> 5)] >> (i & 31)) & 1u)) {
         float g = 0.f, u = 0.f;
@@ -511,8 +521,11 @@ int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, con
     uint32_t *masks = (uint32_t *)(wsb + ws.mask_off);
     const int mask_words = (int)(si_align_up((size_t)n_loaded, 128) / 32);
     size_t smem = (size_t)(2 * words + 2) * 4;
+    SI_CUDA_TRY(cudaMemsetAsync(masks, 0, (size_t)T * mask_words * 4, stream));
     si_union_kernel<<<1, 1024, smem, stream>>>(idx, idx_offsets, k_fixed, T, 0, n_loaded, union_out, n_union_out, pos,
-                                               masks, mask_words, n_loaded, 0, nullptr);
+                                               n_loaded, nullptr);
+    si_union_masks_kernel<<<64, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, 0, n_loaded, n_union_out, pos, masks,
+                                                  mask_words, 0);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }
@@ -552,9 +565,12 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     {
         const int words = (n_loaded + 31) / 32;
         size_t smem = (size_t)(2 * words + 2) * 4;
+        SI_CUDA_TRY(cudaMemsetAsync(masks, 0, (size_t)T * mask_words * 4, stream));
         si_union_kernel<<<1, 1024, smem, stream>>>(idx, idx_offsets, k_fixed, T, shared ? 1 : 0, n_loaded, uni, n_union,
-                                                   pos, masks, mask_words, nu_pad,
-                                                   (flags & SI_FLAG_UNION_UNMASKED) != 0, status_dev);
+                                                   pos, nu_pad, status_dev);
+        si_union_masks_kernel<<<2 * s->num_sms, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, shared ? 1 : 0, n_loaded,
+                                                                   n_union, pos, masks, mask_words,
+                                                                   (flags & SI_FLAG_UNION_UNMASKED) != 0);
     }
     // ---- tiling
     const int t_pad_total = (int)si_align_up((size_t)T, 16);
@@ -590,7 +606,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         si_gemm_gateup_kernel<<<grid, kGemmThreads, smem, stream>>>(P);
     }
     {
-        dim3 grid((nu_pad + 255) / 256, t_pad_alloc);
+        dim3 grid((t_pad_alloc + 31) / 32, (nu_pad + 7) / 8);
         if (s->dtype == SI_BF16)
             si_gemm_combine_kernel<SI_BF16><<<grid, 256, 0, stream>>>(P.partial, s1, nu_pad, t_pad_alloc, T, n_union, masks, mask_words, (uint16_t *)(wsb + ws.h_off));
         else
