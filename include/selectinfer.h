@@ -61,7 +61,8 @@ enum {
     SI_ERR_NOMEM = -5,        /* caller-supplied buffer too small */
     SI_ERR_CUDA = -6,
     SI_ERR_TIMEOUT = -7,      /* a bounded device-side wait expired */
-    SI_ERR_UNSUPPORTED = -8
+    SI_ERR_UNSUPPORTED = -8,
+    SI_ERR_TOO_LARGE = -9     /* a size exceeds a fixed built-in limit (si_ffn_forward_noalloc) */
 };
 
 /* flags */
@@ -182,6 +183,28 @@ int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t 
                             const void *x, const int32_t *idx, const int32_t *idx_offsets,
                             int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
                             size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* Batch-1 selective FFN for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of si_ffn_forward with T = 1.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that owns and budgets all device memory, a callback running under someone else's
+ * allocator, a real-time loop that may not touch the allocator after start-up.  Such a caller can
+ * still hand over its inputs and outputs, but it has no way to provide the scratch the kernels
+ * need, so the scratch lives inside the library: a fixed device array of 304 x 8192 floats
+ * (about 9.5 MiB) that every GPU loading the library holds until the process exits.
+ *
+ *   x, idx (k distinct slots), y, y_dtype, status_dev, stream: as for si_ffn_forward with T = 1;
+ *   flags: SI_FLAG_RESIDUAL only (others are ignored).
+ * Limits: d_model <= 8192 and at most 152 SMs; beyond that the call returns SI_ERR_TOO_LARGE and
+ * launches nothing.  The call never allocates or frees memory, directly or through a library.
+ * The first call on each device looks up the array's device address (the device must be current);
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * it needs no clearing between calls (each call overwrites what it later reads), but two calls
+ * whose kernels overlap on the GPU -- different streams without ordering -- race on it.  Results
+ * are bit-identical to si_ffn_forward with SI_FLAG_SIMPLE_KERNELS on the same inputs. */
+int si_ffn_forward_noalloc(const si_store_t *store, int layer, const void *x, const int32_t *idx, int k,
+                           void *y, int y_dtype, unsigned flags, int32_t *status_dev, void *stream);
 
 /* Union of T lists (the first stage of the T > 1 path, exposed for inspection):
  * union_out device int32 [n_loaded] ascending, *n_union_out device int32. */

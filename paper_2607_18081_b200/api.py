@@ -21,6 +21,7 @@ SI_F16, SI_BF16, SI_F32 = 1, 2, 3
 SI_OK = 0
 SI_ERR_INVALID_ARG, SI_ERR_OUT_OF_RANGE, SI_ERR_DUPLICATE, SI_ERR_ALIGNMENT = -1, -2, -3, -4
 SI_ERR_NOMEM, SI_ERR_CUDA, SI_ERR_TIMEOUT, SI_ERR_UNSUPPORTED = -5, -6, -7, -8
+SI_ERR_TOO_LARGE = -9
 SI_FLAG_CHECK, SI_FLAG_RESIDUAL, SI_FLAG_UNION_UNMASKED, SI_FLAG_SCORE_ABS = 1, 2, 4, 8
 SI_FLAG_SHARED_LIST = 16
 SI_FLAG_SIMPLE_KERNELS = 256
@@ -30,7 +31,7 @@ EXPORTS = [
     "si_strerror", "si_last_cuda_error", "si_build_info", "si_store_bytes", "si_store_create", "si_store_free",
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
-    "si_layer_forward", "si_decode_stack_forward", "si_union", "si_debug_decode_profile",
+    "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
     "si_debug_decode_stream_only",
 ]
 
@@ -67,6 +68,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_layer_forward.argtypes = [vp, ci, vp, ci, vp, ci, vp, vp, vp, ci, cu, vp, sz, vp, vp]
     lib.si_decode_stack_forward.argtypes = [vp, ci, vp, vp, vp, vp, ci, vp, ci, cu, vp, sz, vp, vp]
     lib.si_union.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
+    lib.si_ffn_forward_noalloc.argtypes = [vp, ci, vp, vp, ci, vp, ci, cu, vp, vp]
     lib.si_debug_decode_profile.argtypes = [vp]
     lib.si_debug_decode_stream_only.argtypes = [ci]
     for name in EXPORTS:
@@ -200,6 +202,13 @@ def si_decode_stack_forward(handle, n_steps: int, layers, x, idx, idx_offsets, k
                                         dtype_code(y.dtype), flags, _dp(workspace),
                                         workspace.numel() * workspace.element_size(), _dp(status),
                                         _stream(stream)), "si_decode_stack_forward")
+
+
+def si_ffn_forward_noalloc(handle, layer: int, x, idx, k: int, y, flags: int, status=None, stream=None) -> None:
+    """Batch-1 selective FFN through the entry point that allocates nothing: its scratch is a
+    fixed array inside the library, so only inputs and outputs are passed."""
+    _check(_lib.si_ffn_forward_noalloc(handle, layer, _dp(x), _dp(idx), k, _dp(y), dtype_code(y.dtype), flags,
+                                       _dp(status), _stream(stream)), "si_ffn_forward_noalloc")
 
 
 def si_union(handle, layer: int, T: int, idx, idx_offsets, k_fixed: int, union_out, n_union_out, workspace,

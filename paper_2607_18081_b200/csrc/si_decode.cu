@@ -215,3 +215,68 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
     }
     return SI_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate device memory.
+//
+// The per-step kernels above need scratch for the per-CTA partial outputs.  Here that scratch is
+// a fixed array that is part of the library image: it is reserved on every GPU that loads the
+// library and stays reserved until the process exits.
+namespace {
+
+constexpr int kNoAllocMaxDModel = 8192;
+constexpr int kNoAllocMaxCtas = 304;          // 2 CTAs per SM on up to 152 SMs
+static __device__ __align__(256) float si_noalloc_scratch[(size_t)kNoAllocMaxCtas * kNoAllocMaxDModel];
+
+// In host code the array's name above is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+struct NoAllocDevices {
+    void *ptr[64];
+    bool ready[64];
+};
+NoAllocDevices &noalloc_devices() {
+    static NoAllocDevices d = {};
+    return d;
+}
+
+int noalloc_scratch_for_current_device(float **out) {
+    int dev = -1;
+    SI_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SI_ERR_UNSUPPORTED;
+    NoAllocDevices &d = noalloc_devices();
+    if (!d.ready[dev]) {
+        void *p = nullptr;
+        SI_CUDA_TRY(cudaGetSymbolAddress(&p, si_noalloc_scratch));
+        if (!p) return SI_ERR_CUDA;
+        d.ptr[dev] = p;
+        d.ready[dev] = true;
+    }
+    *out = (float *)d.ptr[dev];
+    return SI_OK;
+}
+
+}  // namespace
+
+extern "C" int si_ffn_forward_noalloc(const si_store_t *store, int layer, const void *x, const int32_t *idx,
+                                      int k, void *y, int y_dtype, unsigned flags, int32_t *status_dev,
+                                      void *stream_) {
+    if (!si_store_ok(store) || !x || !y) return SI_ERR_INVALID_ARG;
+    if (y_dtype != SI_F32 && y_dtype != store->dtype) return SI_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= store->n_layers || k < 0 || !store->loaded[layer]) return SI_ERR_INVALID_ARG;
+    if (k > store->n_loaded[layer]) return SI_ERR_OUT_OF_RANGE;
+    if (k > 0 && !idx) return SI_ERR_INVALID_ARG;
+    if (!si_aligned16(x) || !si_aligned16(y) || (idx && !si_aligned16(idx))) return SI_ERR_ALIGNMENT;
+    if (status_dev && (((uintptr_t)status_dev) & 3u)) return SI_ERR_ALIGNMENT;
+    // the fixed scratch holds one fp32 row of d_model values per CTA of the partial kernel
+    if (store->d_model > kNoAllocMaxDModel || 2 * store->num_sms > kNoAllocMaxCtas) return SI_ERR_TOO_LARGE;
+    float *scratch = nullptr;
+    int rc = noalloc_scratch_for_current_device(&scratch);
+    if (rc != SI_OK) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    // every CTA of the partial kernel writes its whole row before the reduce kernel reads it, so
+    // nothing left over from an earlier call is ever read and nothing needs clearing
+    const unsigned f = flags & SI_FLAG_RESIDUAL;
+    return store->dtype == SI_BF16
+               ? launch_simple_step<SI_BF16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, status_dev, stream)
+               : launch_simple_step<SI_F16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, status_dev, stream);
+}

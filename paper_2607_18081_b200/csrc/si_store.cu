@@ -102,6 +102,7 @@ extern "C" const char *si_strerror(int status) {
         case SI_ERR_CUDA: return "CUDA runtime error";
         case SI_ERR_TIMEOUT: return "bounded device-side wait expired";
         case SI_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SI_ERR_TOO_LARGE: return "size exceeds a fixed built-in limit";
         default: return "unknown status";
     }
 }
