@@ -28,7 +28,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2607_18081_b200 import workloads as wl  # noqa: E402
+from paper_2607_18081_b200 import replicas, workloads as wl  # noqa: E402
 
 METRIC = "selective_ffn_decode_tokens_per_s_batch1"
 UNIT = "tokens/s"
@@ -107,6 +107,8 @@ def cell_config(args):
         kw["loaded_pct"] = args.loaded_pct
     if args.active_pct:
         kw["active_pct"] = args.active_pct
+    if args.batch:
+        kw["batch"] = args.batch
     return cfg.with_(**kw) if kw else cfg
 
 
@@ -162,9 +164,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = replicas.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the selective-FFN library has no CPU path")
     torch.cuda.set_device(local_rank)
@@ -175,6 +175,8 @@ def run_ours(args):
     build.build()
 
     cfg = cell_config(args)
+    if cfg.name in ("c3", "c4"):
+        return run_multitoken(args, cfg, rank, world, local_rank)
     L, d, k, tokens = cfg.n_layers, cfg.d_model, cfg.k_active, cfg.tokens
     tdt = api.torch_dtype(cfg.dtype)
     host_threads = max(1, len(os.sched_getaffinity(0)) // world)
@@ -208,7 +210,7 @@ def run_ours(args):
     load_s = time.perf_counter() - t_load0
 
     # ---- synthetic decode inputs for this rank (pinned host memory)
-    first_token = rank * tokens
+    first_token, _ = replicas.token_range(rank, world, tokens)
     x_host = torch.empty(tokens, L, d, dtype=torch.int16).pin_memory()
     idx_host = torch.empty(tokens, L, k, dtype=torch.int32).pin_memory()
     for l in range(L):
@@ -235,9 +237,8 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier()
+        torch.cuda.synchronize()
 
     def timed(fn, steps, warmup, sampler=None):
         for _ in range(warmup):
@@ -253,10 +254,7 @@ def run_ours(args):
         t1 = time.time()
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
         total_ms = ev[0].elapsed_time(ev[steps])
-        if world > 1:
-            t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
+        total_ms = replicas.max_over_ranks(total_ms, device="cuda")
         return total_ms, per, (t0, t1)
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -271,8 +269,8 @@ def run_ours(args):
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        tok_s = world * tokens * args.steps / (total_ms * 1e-3)
-        e2e_tok_s = world * tokens * args.steps / (e2e_ms * 1e-3)
+        tok_s = replicas.aggregate_throughput(tokens * args.steps, world, total_ms)
+        e2e_tok_s = replicas.aggregate_throughput(tokens * args.steps, world, e2e_ms)
         alg_bytes = wl.selected_bytes_per_token(cfg) * tokens          # per launch (= per step), per GPU
         launch_ms = statistics.mean(per_step_ms)
         achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
@@ -282,8 +280,10 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": workload_name(cfg), "tokens_per_step": tokens, "layers": L,
                        "parallelism": f"replicas x{world} (no data-path collective)",
-                       "l2": "inputs exceed L2: %.0f MB of selected records per token" %
-                             (wl.selected_bytes_per_token(cfg) / 1e6),
+                       "l2": ("inputs exceed L2: %.0f MB of selected records per launch, no flush needed"
+                              if wl.selected_bytes_per_token(cfg) * tokens > 2 * 126e6 else
+                              "%.0f MB of selected records per launch: partly L2-resident, see traffic")
+                             % (wl.selected_bytes_per_token(cfg) * tokens / 1e6),
                        "kernel": "simple" if args.simple else "persistent"},
             "e2e": {"value": e2e_tok_s, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * 2 + idx_host.numel() * 4,
                     "d2h_bytes_per_step": y_host.numel() * y_host.element_size()},
@@ -313,6 +313,98 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_multitoken(args, cfg, rank, world, local_rank):
+    """Configs 3 (batched decode: the union of B lists per layer) and 4 (512-token prefill with one
+    shared list): per-layer si_ffn_forward calls with T > 1 on the tensor-core path.  Not the
+    headline line; reports tokens/s, union size / overlap and achieved GB/s or TFLOP/s."""
+    import torch
+    from paper_2607_18081_b200 import api
+    L, d = cfg.n_layers, cfg.d_model
+    tdt = api.torch_dtype(cfg.dtype)
+    prefill = cfg.shared_list
+    T = cfg.tokens if prefill else cfg.batch
+    k = cfg.k_active
+    n_groups = 1 if prefill else max(1, cfg.tokens // T if cfg.tokens >= T else 1)
+    store = api.NeuronStore(L, d, cfg.d_ff, [cfg.n_loaded] * L, cfg.dtype, device=f"cuda:{local_rank}")
+    for l in range(L):
+        wg, wu, wd = wl.layer_weights(cfg, l)
+        ids, _ = wl.loaded_ids(cfg, l)
+        to_dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(tdt)
+        store.load(l, to_dev(wg), to_dev(wu), to_dev(wd), ids, cfg.n_base)
+        del wg, wu, wd
+    first_token, _ = replicas.token_range(rank, world, n_groups * T)
+    x = torch.empty(n_groups, L, T, d, dtype=torch.int16)
+    for l in range(L):
+        xs = wl.x_tokens(cfg, l, n_groups * T, first_token)
+        x[:, l] = torch.from_numpy(xs.view(np.int16)).view(n_groups, T, d)
+    x = x.cuda().view(tdt)
+    union_sizes = []
+    if prefill:
+        idx = torch.arange(k, dtype=torch.int32, device="cuda")
+        flags = api.SI_FLAG_SHARED_LIST
+        union_sizes = [k]
+    else:
+        lists = np.empty((n_groups, L, T, k), dtype=np.int32)
+        for l in range(L):
+            ll = wl.zipf_lists(cfg, l, n_groups * T, first_token=first_token)
+            lists[:, l] = ll.reshape(n_groups, T, k)
+        union_sizes = [len(np.unique(lists[g, l])) for g in range(n_groups) for l in range(min(L, 4))]
+        idx = torch.from_numpy(lists).cuda()
+        flags = 0
+    y = torch.empty(n_groups, L, T, d, dtype=tdt, device="cuda")
+    ws = store.workspace(T, k, 1)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step():
+        for g in range(n_groups):
+            for l in range(L):
+                api.si_ffn_forward(store.handle, l, x[g, l], T, idx if prefill else idx[g, l], None, k, y[g, l],
+                                   flags, ws, status)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize(); replicas.barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize(); replicas.barrier(); torch.cuda.synchronize()
+    total_ms = replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {status.item()}: {api.strerror(int(status.item()))}")
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        tokens_per_step = n_groups * T
+        tok_s = replicas.aggregate_throughput(tokens_per_step * args.steps, world, total_ms)
+        u = float(np.mean(union_sizes))
+        layer_calls = args.steps * n_groups * L
+        us_per_layer = total_ms * 1e3 / layer_calls
+        union_bytes = u * cfg.record_bytes
+        flops = 6.0 * d * u * T
+        out = {
+            "metric": "selective_ffn_multitoken_tokens_per_s", "value": tok_s, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: {L} layers d_model={d} d_ff={cfg.d_ff} {cfg.dtype}, "
+                                   f"{cfg.n_loaded} loaded, T={T} tokens per call, "
+                                   + ("one shared list of %d slots (prefill)" % k if prefill else
+                                      "own %d-slot Zipf list per token (batched decode)" % k),
+                       "mean_union": u, "union_overlap": None if prefill else 1.0 - u / (T * k),
+                       "union_coverage_of_loaded": u / cfg.n_loaded, "us_per_layer_call": us_per_layer,
+                       "l2": "weights of one pass exceed L2"},
+            "gpu_launches": layer_calls * 6,
+            "roofline": ({"bound": "tensor", "achieved": flops / us_per_layer / 1e6, "peak": peaks["bf16_tflops_sustained"],
+                          "unit": "TFLOP/s", "frac": flops / us_per_layer / 1e6 / peaks["bf16_tflops_sustained"],
+                          "peak_kind": f"of {peak_kind} (sustained)", "traffic": None} if prefill else
+                         {"bound": "hbm", "achieved": union_bytes / us_per_layer / 1e3, "peak": peaks["hbm_gbs"],
+                          "unit": "GB/s", "frac": union_bytes / us_per_layer / 1e3 / peaks["hbm_gbs"],
+                          "peak_kind": f"of {peak_kind}", "traffic": None}),
+        }
+        print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -324,6 +416,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override the number of decode tokens per step")
     ap.add_argument("--loaded-pct", type=int, default=0)
     ap.add_argument("--active-pct", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="c3: tokens processed together per step")
     ap.add_argument("--cpu-tokens", type=int, default=8, help="tokens of the oracle cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simple", action="store_true", help="time the per-step plain-load kernels instead")

@@ -16,14 +16,15 @@
 //     accumulates h * down for its columns in fp32 registers -- while its next record is
 //     already on the way.  At the end of a step set 1 hands its accumulators to set 0 through
 //     shared memory and set 0 stores the CTA's partial y into a ring of D global buffers.
-//   * split-K across SMs, deterministic: the reduction of step s starts kLag steps later, when
-//     every CTA has long published its partial: each consumer thread loads up to 3 partial
-//     float4s of one of this CTA's column groups at the start of a step and sums them (fixed
-//     order: thread, warp butterfly, warps) at its end, so the loads fly under the record
-//     stream; y is written once.
-//   * warp 17 (signalling) does the grid-scope fence + atomics that publish "partial of step s
-//     stored" and "partials of step s - kLag consumed"; warp 18 (watcher) is the only thread
-//     that polls those counters and mirrors them into shared-memory barriers.
+//   * warps 17..18 (reducers, alternating steps): split-K across SMs, deterministic.  A reducer
+//     publishes "partial of step s stored" (grid-scope fence + atomic, kept off the consumers'
+//     path) and then reduces step s - kLag, which every CTA published long ago: the partial
+//     rows of this CTA's column groups are pulled from L2 with 16-byte async copies into a
+//     landing area (plus one row per lane in registers), each lane sums its rows in ascending
+//     order, a warp butterfly combines the lanes, and y is written once.  The reduction thus
+//     trails the record stream by kLag steps and never stalls it.
+//   * warp 19 (watcher) is the only thread group that polls the global per-step counters; it
+//     mirrors them into shared-memory barriers the reducers and consumers wait on.
 //
 // Every wait is bounded: on expiry the kernel records SI_ERR_TIMEOUT, raises a grid-wide
 // abort flag, lets its outstanding copies land and returns.
