@@ -33,6 +33,10 @@ from paper_2607_18081_b200 import replicas, workloads as wl  # noqa: E402
 METRIC = "selective_ffn_decode_tokens_per_s_batch1"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of si_decode_persistent_kernel per (token, layer) step
+# of the config-2 shape, from the capture summarised in
+# profiles/decode_persistent_c2_8layers_32tokens_full.md: (9.6985e9 + 0.2786e9) / 256 steps
+NCU_DRAM_BYTES_PER_C2_STEP = (9.6985e9 + 0.2786e9) / 256
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -294,7 +298,9 @@ def run_ours(args):
                          "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                          "kernel": "si_decode_persistent_kernel" if not args.simple else "si_decode_partial_kernel",
                          "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": launch_ms,
-                         "traffic": args.traffic_bytes},
+                         "traffic": (args.traffic_bytes if args.traffic_bytes is not None else
+                                     (NCU_DRAM_BYTES_PER_C2_STEP * n_steps
+                                      if (cfg.name == "c2" and not args.simple) else None))},
             "load_seconds": load_s,
         }
         if cpu_tokens:
@@ -421,7 +427,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simple", action="store_true", help="time the per-step plain-load kernels instead")
     ap.add_argument("--traffic-bytes", type=float, default=None,
-                    help="DRAM bytes per launch from an ncu capture (reported, not measured here)")
+                    help="DRAM bytes per launch from an ncu capture (default: the committed capture of the "
+                         "persistent kernel, scaled by the number of steps)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
