@@ -164,6 +164,20 @@ __device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src_gmem, u
         : "memory");
 }
 
+// Hardware barrier over the 256 threads of consumer set q (barrier id 1 + q) that also ORs a flag:
+// every thread of the set learns whether any of them has a failed wait, so the set always leaves
+// its loops together and nobody is left waiting at the barrier.
+__device__ __forceinline__ bool set_barrier_or(int q, bool v) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, f;\n\t"
+        "setp.ne.u32 f, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, f;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"((uint32_t)v), "r"(1 + q), "n"(kSetThreads) : "memory");
+    return r != 0;
+}
+
 template <int DT>
 __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
     f[0] = si_cvt<DT>::lo(v.x); f[1] = si_cvt<DT>::hi(v.x);
@@ -380,9 +394,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             }
             if (__any_sync(FULL, progressed)) {
                 t_last = clock64();
-            } else if (*cta_abort || clock64() - t_last > kWaitCycles) {
-                ok = false;
-                break;
+            } else {
+                if (*cta_abort || clock64() - t_last > kWaitCycles) { ok = false; break; }
+                __nanosleep(40);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -442,8 +456,11 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     if (lane == 0) mbar_arrive(&sempty[st]);
                     ++n;
                 }
+                // the record count steers the set's barriers: agree on it (and on failure) first
+                fail = set_barrier_or(q, fail);
+                if (fail) break;
                 SI_PROF(0);                               // wait for x
-                for (int i = 0; i < cnt && !fail; ++i) {
+                for (int i = 0; i < cnt; ++i) {
                     const int st = n % S; const uint32_t ph = (n / S) & 1;
                     fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
                     const bool okr = !fail && smeta[st] != 0 && !noarith;
@@ -475,13 +492,14 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 1);
                         g = keep;
                     }
+                    SI_PROF(5);                           // dots + butterfly
                     // ---- exchange among the set's 8 warps (double-buffered, one barrier per record)
-                    const uint32_t buf = recs & 1, par = (recs >> 1) & 1;
+                    const uint32_t buf = recs & 1;
                     if ((lane & 15) == 0) reinterpret_cast<float *>(&sm->setpart[q][buf][sw])[lane >> 4] = g;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->setbar[q][buf]);
-                    fail |= !mbar_wait_bounded(&sm->setbar[q][buf], par, cta_abort);
+                    fail = set_barrier_or(q, fail);       // also orders the partials for the whole set
+                    SI_PROF(6);                           // 8-warp exchange
                     ++recs;
+                    if (fail) break;
                     float gs = 0.f, us = 0.f;
                     {
                         const float4 *pp = reinterpret_cast<const float4 *>(sm->setpart[q][buf]);
@@ -563,7 +581,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         }
 #undef SI_PROF
         if (prof) {
-            for (int i = 0; i < 6; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
+            for (int i = 0; i < 7; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
         }
         if (fail && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
         return;
@@ -695,7 +713,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 break;
             }
         }
-        if (P.prof && lane == 0 && r == 0) { P.prof[(size_t)b * 8 + 6] = sig_wait; P.prof[(size_t)b * 8 + 7] = sig_fence; }
+        if (P.prof && lane == 0 && r == 0) { P.prof[(size_t)b * 8 + 7] = sig_wait; }
         return;
     }
     // -------------------------------------------------------------------------- watcher warp
@@ -734,7 +752,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 else if (clock64() - t_last > kWaitCycles) { raise_abort(P, sm, SI_ERR_TIMEOUT); stop = 1; }
             }
             if (__shfl_sync(0xFFFFFFFFu, stop, 0)) break;
-            __nanosleep(50);
+            __nanosleep(200);
         }
     }
 }
@@ -808,6 +826,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.prof = si_decode_profile_buffer();
     P.stream_only = si_decode_stream_only() & 0xFF;
     P.prefetch_rounds = 0;
+    if ((si_decode_stream_only() >> 8) & 0xF) P.nstage = 2 * ((si_decode_stream_only() >> 8) & 0xF);   // diagnostics: shallower rings
     int G = s->num_sms;
     if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
     // every CTA reduces at most kMaxGroups float4 column groups
