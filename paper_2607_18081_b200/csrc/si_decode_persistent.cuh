@@ -14,17 +14,14 @@
 //     registers and its stage handed back at once; the set then forms the two dot products
 //     (thread slices, warp butterfly, 8-warp exchange on an mbarrier), applies SiLU(g)*u and
 //     accumulates h * down for its columns in fp32 registers -- while its next record is
-//     already on the way.  At the end of a step set 1 hands its accumulators to set 0 through
-//     shared memory and set 0 stores the CTA's partial y into a ring of D global buffers.
-//   * warps 17..18 (reducers, alternating steps): split-K across SMs, deterministic.  A reducer
-//     publishes "partial of step s stored" (grid-scope fence + atomic, kept off the consumers'
-//     path) and then reduces step s - kLag, which every CTA published long ago: the partial
-//     rows of this CTA's column groups are pulled from L2 with 16-byte async copies into a
-//     landing area (plus one row per lane in registers), each lane sums its rows in ascending
-//     order, a warp butterfly combines the lanes, and y is written once.  The reduction thus
-//     trails the record stream by kLag steps and never stalls it.
-//   * warp 19 (watcher) is the only thread group that polls the global per-step counters; it
-//     mirrors them into shared-memory barriers the reducers and consumers wait on.
+//     already on the way.  At the end of a step each set leaves its accumulators in shared
+//     memory for the reducer warps and goes straight on to the next step.
+//   * warps 17..19 (reducers, step s goes to warp s mod 3) own everything that involves other
+//     SMs: they add the two sets' accumulators, store the CTA's partial y into a ring of D
+//     global buffers, publish it (grid-scope fence + atomic), and kLag steps later -- when every
+//     CTA has long published that step -- sum the partial rows of this CTA's column groups in a
+//     fixed order (lane rows ascending, warp butterfly: deterministic split-K) and write y
+//     once.  The reduction trails the record stream and never stalls it.
 //
 // Every wait is bounded: on expiry the kernel records SI_ERR_TIMEOUT, raises a grid-wide
 // abort flag, lets its outstanding copies land and returns.
@@ -41,11 +38,9 @@ constexpr int kSetWarps = 8;
 constexpr int kSetThreads = kSetWarps * 32;
 constexpr int kConsumers = kSets * kSetThreads;
 constexpr int kConsumerWarps = kConsumers / 32;
-constexpr int kReducerWarps = 2;
-constexpr int kThreads = 32 + kConsumers + 32 * kReducerWarps + 32;   // producer, consumers, reducers, watcher
-constexpr int kLandBytes = 8 * 1024;              // per reducer warp: landing area for partial-y rows
+constexpr int kReducerWarps = 3;
+constexpr int kThreads = 32 + kConsumers + 32 * kReducerWarps;        // producer, consumers, reducers
 constexpr int kMaxGroups = 8;                     // float4 column groups one CTA reduces (d_model / 4 / SMs, rounded up)
-constexpr int kFlagRing = 8;                      // per-step shared-memory flags kept for this many steps
 constexpr int kCounterStride = 64;                // uint32 per step: written at +0, reduced at +32 (own 128-byte lines)
 constexpr int kMaxStages = 16;
 constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
@@ -233,10 +228,9 @@ struct Smem {
     uint64_t full[kMaxStages];         // stage index = set * S + stage-in-set
     uint64_t empty[kMaxStages];
     uint64_t setbar[kSets][2];         // a set's warps have published their dot-product partials
-    uint64_t accfull, accempty;        // set 1 -> set 0 hand-over of a step's accumulators
-    uint64_t stepbar[kPartialDepth];   // all consumer warps are done with step s (slot s mod D)
-    uint64_t pubbar[kFlagRing];        // every CTA has published its partial of step s (slot s mod ring)
-    uint64_t freebar[kFlagRing];       // every CTA has finished reading the partials of step s
+    // consumer set -> reducers hand-over of a step's accumulators (one buffer per set); one barrier
+    // per reducer warp (slot s mod 3), so that each waiter follows the phases of its own barrier
+    uint64_t accfull[kSets][kReducerWarps], accempty[kSets][kReducerWarps];
     int meta[kMaxStages];
     uint4 desc[kSets][kDescRing];      // {src lo, src hi, bytes (0: nothing to copy), meta}
     float2 setpart[kSets][2][kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products
@@ -259,8 +253,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     const int nstage = P.nstage;               // total over both sets (even)
     const int S = nstage / kSets;              // ring stages per consumer set
     uint8_t *ring = smem;
-    float *accbuf = reinterpret_cast<float *>(smem + (size_t)nstage * rec_bytes);   // set 1 -> set 0, d_model floats
-    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)nstage * rec_bytes + (size_t)P.d_model * 4);
+    float *accbuf = reinterpret_cast<float *>(smem + (size_t)nstage * rec_bytes);   // [set][d_model] hand-over to the reducers
+    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)nstage * rec_bytes + (size_t)kSets * P.d_model * 4);
     uint64_t *full = sm->full, *empty = sm->empty;
     int *meta = sm->meta;
     volatile int *cta_abort = &sm->cta_abort;
@@ -273,9 +267,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
         for (int q = 0; q < kSets; ++q) { mbar_init(&sm->setbar[q][0], kSetWarps); mbar_init(&sm->setbar[q][1], kSetWarps); }
-        mbar_init(&sm->accfull, kSetWarps); mbar_init(&sm->accempty, kSetWarps);
-        for (int s = 0; s < kPartialDepth; ++s) mbar_init(&sm->stepbar[s], kConsumerWarps);
-        for (int s = 0; s < kFlagRing; ++s) { mbar_init(&sm->pubbar[s], 1); mbar_init(&sm->freebar[s], 1); }
+        for (int q = 0; q < kSets; ++q)
+            for (int w = 0; w < kReducerWarps; ++w) { mbar_init(&sm->accfull[q][w], kSetWarps); mbar_init(&sm->accempty[q][w], 1); }
         sm->cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -522,153 +515,131 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 if (fail) break;
             }
 
-            // ---- merge the two sets' accumulators through shared memory (set 1 -> set 0)
+            // ---- hand this set's accumulators of the step to the reducer warps (shared memory);
+            // the set is then free for the next step: it never touches global synchronisation
             {
-                const uint32_t sp = (uint32_t)(step & 1);
-                if (q == 1) {
-                    fail |= !mbar_wait_bounded(&sm->accempty, sp ^ 1, cta_abort);
-#pragma unroll
-                    for (int k2 = 0; k2 < NCH; ++k2) {
-                        const int c = t + kSetThreads * k2;
-                        if (c < chunks) {
-                            float4 *o = reinterpret_cast<float4 *>(accbuf + (size_t)c * 8);
-                            o[0] = make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]);
-                            o[1] = make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]);
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->accfull);
-                } else {
-                    fail |= !mbar_wait_bounded(&sm->accfull, sp, cta_abort);
-#pragma unroll
-                    for (int k2 = 0; k2 < NCH; ++k2) {
-                        const int c = t + kSetThreads * k2;
-                        if (c < chunks) {
-                            const float4 *o = reinterpret_cast<const float4 *>(accbuf + (size_t)c * 8);
-                            const float4 a0 = o[0], a1 = o[1];
-                            acc[k2][0] += a0.x; acc[k2][1] += a0.y; acc[k2][2] += a0.z; acc[k2][3] += a0.w;
-                            acc[k2][4] += a1.x; acc[k2][5] += a1.y; acc[k2][6] += a1.z; acc[k2][7] += a1.w;
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->accempty);
+                if (step > 0) {      // the buffer was last handed over at step - 1
+                    const int ps = step - 1;
+                    fail |= !mbar_wait_bounded(&sm->accempty[q][ps % kReducerWarps], (uint32_t)((ps / kReducerWarps) & 1), cta_abort);
                 }
                 if (fail) break;
-            }
-            SI_PROF(3);                                   // set merge
-            // ---- [C2] set 0 stores the CTA's partial y of this step into the ring of D buffers
-            if (real && q == 0 && !nosync) {
-                if (step >= kPartialDepth) {
-                    const int fq = step - kPartialDepth;
-                    fail |= !mbar_wait_bounded(&sm->freebar[fq % kFlagRing], (fq / kFlagRing) & 1, cta_abort);
-                    if (fail) break;
-                }
-                float *mine_p = P.partial + ((size_t)(step % kPartialDepth) * G + b) * d;
+                float *ab = accbuf + (size_t)q * d;
 #pragma unroll
                 for (int k2 = 0; k2 < NCH; ++k2) {
                     const int c = t + kSetThreads * k2;
                     if (c < chunks) {
-                        float4 *o = reinterpret_cast<float4 *>(mine_p + (size_t)c * 8);
-                        __stcg(o, make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]));
-                        __stcg(o + 1, make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]));
+                        float4 *o = reinterpret_cast<float4 *>(ab + (size_t)c * 8);
+                        o[0] = make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]);
+                        o[1] = make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]);
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->accfull[q][step % kReducerWarps]);
             }
-            // ---- [C3] this warp is done with the step: its set's partial is stored
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm->stepbar[step % kPartialDepth]);
-            SI_PROF(4);                                   // partial store
+            SI_PROF(3);                                   // accumulator hand-over
         }
 #undef SI_PROF
         if (prof) {
-            for (int i = 0; i < 7; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
+            for (int i = 0; i < 4; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
+            P.prof[(size_t)b * 8 + 5] = pf[5] + pf[6];
         }
         if (fail && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
         return;
     }
 
     // -------------------------------------------------------------------------- reducer warps
-    // Reducer warp r handles steps s = r (mod 2).  For step s it publishes "partials of step s
-    // stored" (grid-scope fence + atomic, kept off the consumers' path) and then reduces step
-    // sr = s - kLag, which every CTA published long ago: the 2G partial rows of this CTA's column
-    // groups are pulled from L2 into a shared-memory landing area with 16-byte async copies (no
-    // registers held while they fly), each lane sums the rows it fetched in ascending order, a
-    // warp butterfly combines the lanes (fixed order, so deterministic), and y is written once.
-    if (warp <= kConsumerWarps + kReducerWarps) {
-        const int r = warp - 1 - kConsumerWarps;
+    // Everything that needs other SMs lives here, off the consumers' path.  Reducer warp r handles
+    // steps s = r (mod 3), in two phases:
+    //  (A) when both consumer sets have handed over their accumulators of step s: add the two,
+    //      store the CTA's partial y into slot s mod D of the global ring (after every CTA has
+    //      finished reading the step that used the slot before), give the hand-over buffers back,
+    //      and publish "partial of step s stored" (grid-scope fence + atomic);
+    //  (B) reduce step sr = s - kLag, which every CTA published long ago: each lane loads rows
+    //      lane, lane+32, ... of this CTA's column groups and sums them in
+    //      ascending order; a warp butterfly combines the lanes (fixed order: deterministic
+    //      split-K); y is written once; "partials of step sr consumed" is published.
+    {
+        const int r = warp - 1 - kConsumerWarps;               // 0 .. kReducerWarps-1
         const bool nosync = (P.stream_only & 4) != 0;
         const int ngroups = d / 4;
         const int gpc = (ngroups + G - 1) / G;                 // <= kMaxGroups (launch check)
         const int g_valid = ngroups - b * gpc < gpc ? (ngroups - b * gpc < 0 ? 0 : ngroups - b * gpc) : gpc;
-        float4 *land = reinterpret_cast<float4 *>(smem + (size_t)nstage * rec_bytes + (size_t)P.d_model * 4 + sizeof(Smem) + 64) +
-                       (size_t)r * (kLandBytes / 16);
-        const int rpl = (kLandBytes / 16) / (32 * gpc);        // landing rows per lane and round (>= 1)
-        const int RR = 32 * rpl;
-        long long sig_wait = 0, sig_fence = 0;
+        const bool rprof = P.prof != nullptr && r == 0 && lane == 0;
+        long long rp_a = 0, rp_b = 0, rp_wait = 0;
         for (int step = r; step < P.n_steps + kLag; step += kReducerWarps) {
             int ok = 1;
-            if (step < P.n_steps && !nosync) {
+            long long c0 = rprof ? clock64() : 0;
+            if (step < P.n_steps) {
+                // ---- phase A
                 if (lane == 0) {
-                    long long c0 = clock64();
-                    ok = mbar_wait_bounded(&sm->stepbar[step % kPartialDepth], (step / kPartialDepth) & 1, cta_abort);
-                    long long c1 = clock64();
-                    if (ok) {
-                        __threadfence();
-                        atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
-                    }
-                    if (P.prof) { sig_wait += c1 - c0; sig_fence += clock64() - c1; }
+                    const uint32_t par = (uint32_t)((step / kReducerWarps) & 1);
+                    ok = mbar_wait_bounded(&sm->accfull[0][r], par, cta_abort) &&
+                         mbar_wait_bounded(&sm->accfull[1][r], par, cta_abort);
+                    if (ok && !nosync && step >= kPartialDepth)
+                        ok = counter_wait_bounded(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32,
+                                                  (unsigned)G, P.ctrl + 1, cta_abort);
                 }
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                long long c1 = rprof ? clock64() : 0;
+                if (rprof) rp_wait += c1 - c0;
+                if (ok) {
+                    const float4 *a0 = reinterpret_cast<const float4 *>(accbuf);
+                    const float4 *a1 = reinterpret_cast<const float4 *>(accbuf + d);
+                    float4 *dst = reinterpret_cast<float4 *>(P.partial + ((size_t)(step % kPartialDepth) * G + b) * d);
+                    // add the two sets' accumulators and store the CTA's partial y, 8 float4 per lane at a
+                    // time (loads first, so their latencies overlap)
+                    const int n4 = d / 4;
+                    for (int i0 = 0; i0 < n4; i0 += 32 * 8) {
+                        float4 u0[8], u1[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int i = i0 + lane + 32 * j;
+                            u0[j] = i < n4 ? a0[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+                            u1[j] = i < n4 ? a1[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int i = i0 + lane + 32 * j;
+                            if (i < n4 && !nosync)
+                                __stcg(dst + i, make_float4(u0[j].x + u1[j].x, u0[j].y + u1[j].y, u0[j].z + u1[j].z, u0[j].w + u1[j].w));
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&sm->accempty[0][r]); mbar_arrive(&sm->accempty[1][r]);
+                        if (!nosync) {
+                            __threadfence();
+                            atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
+                        }
+                    }
+                }
+                if (rprof) rp_a += clock64() - c1;
             }
             if (ok && step >= kLag && !nosync) {
+                // ---- phase B
+                long long c2 = rprof ? clock64() : 0;
                 const int sr = step - kLag;
-                if (lane == 0) ok = mbar_wait_bounded(&sm->pubbar[sr % kFlagRing], (sr / kFlagRing) & 1, cta_abort);
+                if (lane == 0)
+                    ok = counter_wait_bounded(P.counters + (size_t)sr * kCounterStride, (unsigned)G, P.ctrl + 1, cta_abort);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (ok) {
                     float4 v[kMaxGroups];
 #pragma unroll
                     for (int g = 0; g < kMaxGroups; ++g) v[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    const float *base = P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4;
+                    const float4 *base = reinterpret_cast<const float4 *>(
+                        P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4);
+                    const size_t row_stride = (size_t)d / 4;
                     if ((P.stream_only & 2) == 0) {
-                        // per round a lane fetches rpl rows through the landing area and one more
-                        // straight into registers; it sums them in ascending row order
-                        for (int r0 = 0; r0 < G; r0 += RR + 32) {
-                            for (int j = 0; j < rpl; ++j) {
-                                const int row = r0 + lane + 32 * j;
-                                if (row < G) {
-                                    const float *src = base + (size_t)row * d;
-                                    float4 *dst = land + (size_t)(lane + 32 * j) * gpc;
-                                    for (int g = 0; g < g_valid; ++g)
-                                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                                                     ::"r"(smem_u32(dst + g)), "l"(src + g * 4) : "memory");
-                                }
-                            }
-                            asm volatile("cp.async.commit_group;" ::: "memory");
-                            float4 xr4[kMaxGroups];
-                            const int xrow = r0 + lane + 32 * rpl;
+                        for (int r0 = lane; r0 < G; r0 += 32) {
+                            float4 t0[kMaxGroups];
 #pragma unroll
                             for (int g = 0; g < kMaxGroups; ++g) {
-                                xr4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (xrow < G && g < g_valid)
-                                    xr4[g] = __ldcg(reinterpret_cast<const float4 *>(base + (size_t)xrow * d) + g);
-                            }
-                            asm volatile("cp.async.wait_group 0;" ::: "memory");
-                            for (int j = 0; j < rpl; ++j) {
-                                const int row = r0 + lane + 32 * j;
-                                if (row < G) {
-                                    const float4 *srcs = land + (size_t)(lane + 32 * j) * gpc;
-#pragma unroll
-                                    for (int g = 0; g < kMaxGroups; ++g) {
-                                        if (g < g_valid) {
-                                            const float4 t4 = srcs[g];
-                                            v[g].x += t4.x; v[g].y += t4.y; v[g].z += t4.z; v[g].w += t4.w;
-                                        }
-                                    }
-                                }
+                                t0[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (g < g_valid) t0[g] = __ldcg(base + (size_t)r0 * row_stride + g);
                             }
 #pragma unroll
                             for (int g = 0; g < kMaxGroups; ++g) {
-                                v[g].x += xr4[g].x; v[g].y += xr4[g].y; v[g].z += xr4[g].z; v[g].w += xr4[g].w;
+                                v[g].x += t0[g].x; v[g].y += t0[g].y; v[g].z += t0[g].z; v[g].w += t0[g].w;
                             }
                         }
                     }
@@ -680,8 +651,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                             v[g].z += __shfl_xor_sync(0xFFFFFFFFu, v[g].z, o); v[g].w += __shfl_xor_sync(0xFFFFFFFFu, v[g].w, o);
                         }
                     }
-                    // lane g writes column group g
-                    float4 mine_v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float4 mine_v = make_float4(0.f, 0.f, 0.f, 0.f);      // lane g writes column group g
 #pragma unroll
                     for (int g = 0; g < kMaxGroups; ++g) if (lane == g) mine_v = v[g];
                     if (lane < g_valid) {
@@ -701,64 +671,25 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         }
                     }
                     __syncwarp();
-                    // the partial buffer of step sr may be overwritten once every CTA has said so
-                    if (lane == 0 && sr < P.n_steps - kLag) {
+                    // the ring slot of step sr may be overwritten once every CTA has said so
+                    if (lane == 0 && sr + kPartialDepth < P.n_steps) {
                         __threadfence();
                         atomicAdd(P.counters + (size_t)sr * kCounterStride + 32, 1u);
                     }
                 }
+                if (rprof) rp_b += clock64() - c2;
             }
             if (!ok) {
                 if (lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
                 break;
             }
         }
-        if (P.prof && lane == 0 && r == 0) { P.prof[(size_t)b * 8 + 7] = sig_wait; }
-        return;
-    }
-    // -------------------------------------------------------------------------- watcher warp
-    // The only thread of the CTA that polls global memory: it turns "all G CTAs have published
-    // step s" / "all G CTAs have finished reading step s" into shared-memory barriers the
-    // consumers wait on.  It cannot run more than kFlagRing steps ahead of the consumers: a
-    // step's counters only fill up after this CTA's own consumers have passed that step.
-    if ((P.stream_only & 4) == 0) {
-        // lanes 0..15 look at the written counters of steps pw .. pw+15, lanes 16..31 at the
-        // reduced counters of steps pr .. pr+15, all in one round of loads; the completed prefix
-        // of each is then signalled in order.
-        int pw = 0, pr = 0;                   // next step whose written / reduced counter is awaited
-        const int n_red = P.n_steps - kLag;   // reduced[] is signalled for steps 0 .. n_steps-kLag-1
-        const int half = lane >> 4, hl = lane & 15;
-        long long t_last = clock64();
-        while (pw < P.n_steps || pr < n_red) {
-            const int sidx = (half ? pr : pw) + hl;
-            const int lim = half ? n_red : P.n_steps;
-            bool done = false;
-            if (sidx < lim)
-                done = ld_acquire_gpu(P.counters + (size_t)sidx * kCounterStride + (half ? 32 : 0)) >= (unsigned)G;
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, done);
-            // number of leading completed steps in each half (at most kFlagRing - 2 at a time)
-            int nw = __ffs(~(m & 0xFFFFu)) - 1, nr = __ffs(~(m >> 16)) - 1;
-            nw = nw < 0 ? 16 : nw; nr = nr < 0 ? 16 : nr;
-            nw = nw > kFlagRing - 2 ? kFlagRing - 2 : nw; nr = nr > kFlagRing - 2 ? kFlagRing - 2 : nr;
-            if (lane == 0) {
-                for (int i = 0; i < nw; ++i) mbar_arrive(&sm->pubbar[(pw + i) % kFlagRing]);
-                for (int i = 0; i < nr; ++i) mbar_arrive(&sm->freebar[(pr + i) % kFlagRing]);
-            }
-            pw += nw; pr += nr;
-            if (nw | nr) { t_last = clock64(); continue; }
-            int stop = 0;
-            if (lane == 0) {
-                if (*cta_abort || ld_relaxed_gpu(P.ctrl + 1)) stop = 1;
-                else if (clock64() - t_last > kWaitCycles) { raise_abort(P, sm, SI_ERR_TIMEOUT); stop = 1; }
-            }
-            if (__shfl_sync(0xFFFFFFFFu, stop, 0)) break;
-            __nanosleep(200);
-        }
+        if (rprof) { P.prof[(size_t)b * 8 + 4] = rp_wait; P.prof[(size_t)b * 8 + 6] = rp_a; P.prof[(size_t)b * 8 + 7] = rp_b; }
     }
 }
 
 inline size_t smem_bytes(int d_model, int nstage) {
-    return (size_t)nstage * d_model * 6 + (size_t)d_model * 4 + sizeof(Smem) + 64 + (size_t)kReducerWarps * kLandBytes;
+    return (size_t)nstage * d_model * 6 + (size_t)kSets * d_model * 4 + sizeof(Smem) + 64;
 }
 inline int pick_stages(int d_model) {
     const size_t budget = 227 * 1024;
