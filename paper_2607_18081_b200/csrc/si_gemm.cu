@@ -56,6 +56,17 @@ __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// wait until at most n of this thread's committed copy groups are still in flight (n <= 5)
+__device__ __forceinline__ void cp_async_wait_dyn(int n) {
+    switch (n) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        default: cp_async_wait<5>(); break;
+    }
+}
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -249,20 +260,27 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
 
     if (warp < 4) {
         // ---------------------------------------------------------------- gather loads
-        const int r = tid;                                           // tile row = union position mt*128 + r
-        const int slot = P.union_slots[mt * 128 + r];
-        const char *grow = P.rec_base + (size_t)slot * P.rec_bytes;  // gate row; up row follows at d_model*2
-        const int sw = r & 7;
+        // Copy j of a thread covers 16-byte piece (tid & 7) of tile row 16*j + (tid >> 3): the 32 lanes
+        // of a warp instruction read four whole 128-byte row segments, so the gather is coalesced.
+        const int q8 = tid & 7;
+        const char *grow[8];                                         // gate rows; the up row follows at d_model*2
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            grow[j] = P.rec_base + (size_t)P.union_slots[mt * 128 + 16 * j + (tid >> 3)] * P.rec_bytes + q8 * 16;
+        const int r = tid;                                           // epilogue: this thread's tile row
         int pending = 0;                                             // committed groups not yet signalled
+        const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;         // chunks of copies kept in flight
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
             uint8_t *sg = tiles + (size_t)st * stage_bytes, *su = sg + 128 * 128, *sx = su + 128 * 128;
-            const char *gsrc = grow + (size_t)(c0 + c) * 128;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                cp_async16(sg + r * 128 + ((q ^ sw) << 4), gsrc + q * 16);
-                cp_async16(su + r * 128 + ((q ^ sw) << 4), gsrc + (size_t)P.d_model * 2 + q * 16);
+            for (int j = 0; j < 8; ++j) {
+                const int row = 16 * j + (tid >> 3);
+                const char *gsrc = grow[j] + (size_t)(c0 + c) * 128;
+                const int off = row * 128 + ((q8 ^ (row & 7)) << 4);
+                cp_async16(sg + off, gsrc);
+                cp_async16(su + off, gsrc + (size_t)P.d_model * 2);
             }
             for (int e = tid; e < N * 8; e += kLoaderThreads) {
                 const int n = e >> 3, q = e & 7;
@@ -275,18 +293,21 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
             }
             cp_async_commit();
             ++pending;
-            if (pending == 3) {          // keep two chunks of copies in flight per thread
-                cp_async_wait<2>();
+            if (pending == la + 1) {     // keep `la` chunks of copies in flight per thread
+                cp_async_wait_dyn(la);
                 fence_async_proxy();
-                mbar_arrive(&full[(c - 2) % P.nstage]);
+                mbar_arrive(&full[(c - la) % P.nstage]);
                 --pending;
             }
         }
         // drain
         if (!*failed) {
             const int done = n_chunks;
-            if (pending >= 2) { cp_async_wait<1>(); fence_async_proxy(); mbar_arrive(&full[(done - 2) % P.nstage]); }
-            if (pending >= 1) { cp_async_wait<0>(); fence_async_proxy(); mbar_arrive(&full[(done - 1) % P.nstage]); }
+            for (; pending > 0; --pending) {
+                cp_async_wait_dyn(pending - 1);
+                fence_async_proxy();
+                mbar_arrive(&full[(done - pending) % P.nstage]);
+            }
         } else {
             cp_async_wait<0>();
         }
@@ -406,20 +427,24 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     const uint32_t tmem = *tmem_slot;
 
     if (warp < 4) {
-        // thread -> (union entry kk of the chunk, half of the 128 columns)
-        const int kk = tid >> 1, half = tid & 1;
-        const int kg = kk >> 3, k8 = kk & 7;
+        // Copy j of a thread covers 16-byte piece (tid & 15) of the 256-byte down-row segment of union
+        // entry 8*j + (tid >> 4) of the chunk: a warp instruction reads two whole segments (coalesced).
+        const int c16 = tid & 15;
         int pending = 0;
+        const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
             uint8_t *sa = tiles + (size_t)st * stage_bytes, *sh = sa + 64 * 256;
-            const int slot = P.union_slots[(c0 + c) * kChunkK + kk];            // padded entries carry a valid slot
-            const char *src = P.rec_base + (size_t)slot * P.rec_bytes + (size_t)P.d_model * 4 +
-                              ((size_t)mt * 128 + half * 64) * 2;
-            uint8_t *dst = sa + kg * 2048 + half * 1024 + k8 * 128;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) cp_async16(dst + ((q ^ k8) << 4), src + q * 16);
+            for (int j = 0; j < 8; ++j) {
+                const int kk = 8 * j + (tid >> 4);                              // union entry of the chunk
+                const int slot = P.union_slots[(c0 + c) * kChunkK + kk];        // padded entries carry a valid slot
+                const char *src = P.rec_base + (size_t)slot * P.rec_bytes + (size_t)P.d_model * 4 +
+                                  (size_t)mt * 256 + c16 * 16;
+                const int half = c16 >> 3, q = c16 & 7, k8 = kk & 7;
+                cp_async16(sa + (kk >> 3) * 2048 + half * 1024 + k8 * 128 + ((q ^ k8) << 4), src);
+            }
             for (int e = tid; e < N * 8; e += kLoaderThreads) {
                 const int n = e >> 3, q = e & 7;
                 cp_async16(sh + n * 128 + ((q ^ (n & 7)) << 4),
@@ -427,17 +452,20 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
             }
             cp_async_commit();
             ++pending;
-            if (pending == 3) {
-                cp_async_wait<2>();
+            if (pending == la + 1) {
+                cp_async_wait_dyn(la);
                 fence_async_proxy();
-                mbar_arrive(&full[(c - 2) % P.nstage]);
+                mbar_arrive(&full[(c - la) % P.nstage]);
                 --pending;
             }
         }
         if (!*failed) {
             const int done = n_chunks;
-            if (pending >= 2) { cp_async_wait<1>(); fence_async_proxy(); mbar_arrive(&full[(done - 2) % P.nstage]); }
-            if (pending >= 1) { cp_async_wait<0>(); fence_async_proxy(); mbar_arrive(&full[(done - 1) % P.nstage]); }
+            for (; pending > 0; --pending) {
+                cp_async_wait_dyn(pending - 1);
+                fence_async_proxy();
+                mbar_arrive(&full[(done - pending) % P.nstage]);
+            }
         } else {
             cp_async_wait<0>();
         }
@@ -588,7 +616,9 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.fmt = s->dtype == SI_BF16 ? 1 : 0;
     P.status = status_dev;
     // gate/up: split K = d_model so that about one wave of CTAs is launched
-    int s1 = s->num_sms / (m_tiles * tok_tiles);
+    // the grid is sized for the largest possible union; with few tokens the real union is much
+    // smaller and the surplus CTAs exit at once, so aim at about two CTAs per SM there
+    int s1 = (t_pad_alloc <= 64 ? 2 * s->num_sms + m_tiles * tok_tiles - 1 : s->num_sms) / (m_tiles * tok_tiles);
     const int k_chunks = d / kChunkK;
     if (s1 < 1) s1 = 1;
     if (s1 > 8) s1 = 8;
