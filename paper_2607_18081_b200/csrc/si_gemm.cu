@@ -103,27 +103,29 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 // ------------------------------------------------------------------------------- union
-// One CTA: bitmap OR of all list entries, popcount prefix scan -> sorted union, position map,
-// per-token membership masks over union positions.
+// Step 1 (many CTAs): OR every list entry into a bitmap over the loaded slots (zero on entry).
+__global__ void si_union_bitmap_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed,
+                                       int n_lists, int n_loaded, uint32_t *__restrict__ bitmap, int32_t *status) {
+    const long long total = offsets ? offsets[n_lists] : (long long)n_lists * k_fixed;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        const int s = idx[e];
+        if (s < 0 || s >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
+        const uint32_t bit = 1u << (s & 31);
+        if (!(bitmap[s >> 5] & bit)) atomicOr(&bitmap[s >> 5], bit);     // hot slots are set by the first token
+    }
+}
+
+// Step 2 (one CTA): popcount prefix scan over the bitmap -> sorted union, slot -> position map.
 __global__ void __launch_bounds__(1024)
-si_union_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int T,
-                int shared_list, int n_loaded, int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out,
-                int32_t *__restrict__ pos_of_slot, int union_cap, int32_t *status) {
+si_union_kernel(const uint32_t *__restrict__ bitmap_g, int n_loaded, int32_t *__restrict__ union_out,
+                int32_t *__restrict__ n_union_out, int32_t *__restrict__ pos_of_slot, int union_cap) {
     extern __shared__ uint32_t sh[];
     uint32_t *bitmap = sh;                         // [words]
     uint32_t *wprefix = sh + (n_loaded + 31) / 32; // [words] exclusive popcount prefix
     __shared__ uint32_t warp_tot[32];
     const int words = (n_loaded + 31) / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int w = tid; w < words; w += 1024) bitmap[w] = 0u;
-    __syncthreads();
-    const int n_lists = shared_list ? 1 : T;
-    const int total = offsets ? offsets[n_lists] : n_lists * k_fixed;
-    for (int e = tid; e < total; e += 1024) {
-        int s = idx[e];
-        if (s < 0 || s >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
-        atomicOr(&bitmap[s >> 5], 1u << (s & 31));
-    }
+    for (int w = tid; w < words; w += 1024) bitmap[w] = bitmap_g[w];
     __syncthreads();
     // exclusive prefix of popcounts over the bitmap words (words <= 2048 for d_ff <= 65536)
     uint32_t carry = 0;
@@ -221,7 +223,7 @@ struct GemmParams {
 // Gate/up contraction.  grid = (union tiles of 128, K splits of d_model, token tiles).
 // D_gate[128 neurons x N tokens] (+)= Wg[U tile, k] . X[tokens, k]^T, same for up, accumulated in
 // tensor memory (columns [0,N) gate, [N,2N) up).
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, 2)
 si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
@@ -389,7 +391,7 @@ __global__ void si_gemm_combine_kernel(const float *__restrict__ partial, int n_
 // Down contraction.  grid = (d_model / 128 column tiles, K splits over the union, token tiles).
 // D[128 output columns x N tokens] (+)= Wd[U_k, columns]^T . H[tokens, U_k]^T: A is MN-major (a
 // down row is contiguous along the output columns), B is K-major.
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, 2)
 si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
@@ -432,14 +434,24 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
         const int c16 = tid & 15;
         int pending = 0;
         const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;
+        int slots_next[8];                                           // union slots of the next chunk (prefetched)
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            slots_next[j] = n_chunks > 0 ? P.union_slots[c0 * kChunkK + 8 * j + (tid >> 4)] : 0;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
+            int slots[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                slots[j] = slots_next[j];
+                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c0 + c + 1) * kChunkK + 8 * j + (tid >> 4)];
+            }
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
             uint8_t *sa = tiles + (size_t)st * stage_bytes, *sh = sa + 64 * 256;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int kk = 8 * j + (tid >> 4);                              // union entry of the chunk
-                const int slot = P.union_slots[(c0 + c) * kChunkK + kk];        // padded entries carry a valid slot
+                const int slot = slots[j];                                      // padded entries carry a valid slot
                 const char *src = P.rec_base + (size_t)slot * P.rec_bytes + (size_t)P.d_model * 4 +
                                   (size_t)mt * 256 + c16 * 16;
                 const int half = c16 >> 3, q = c16 & 7, k8 = kk & 7;
@@ -524,8 +536,9 @@ __global__ void si_gemm_reduce_kernel(const float *__restrict__ partial, int n_s
     else reinterpret_cast<uint16_t *>(y)[(size_t)t * d + j] = si_cvt<DT>::from_float(a);
 }
 
-int pick_stages_gemm(size_t stage_bytes) {
-    size_t budget = 200 * 1024;
+int pick_stages_gemm(size_t stage_bytes, int n_tok) {
+    // few tokens: the kernels are latency-bound gathers, two CTAs per SM hide more of it
+    size_t budget = n_tok <= 64 ? 112 * 1024 : 200 * 1024;
     int n = (int)(budget / stage_bytes);
     return n > kMaxStages ? kMaxStages : n;
 }
@@ -549,9 +562,10 @@ int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, con
     uint32_t *masks = (uint32_t *)(wsb + ws.mask_off);
     const int mask_words = (int)(si_align_up((size_t)n_loaded, 128) / 32);
     size_t smem = (size_t)(2 * words + 2) * 4;
-    SI_CUDA_TRY(cudaMemsetAsync(masks, 0, (size_t)T * mask_words * 4, stream));
-    si_union_kernel<<<1, 1024, smem, stream>>>(idx, idx_offsets, k_fixed, T, 0, n_loaded, union_out, n_union_out, pos,
-                                               n_loaded, nullptr);
+    uint32_t *bitmap = masks + (size_t)T * mask_words;
+    SI_CUDA_TRY(cudaMemsetAsync(masks, 0, ((size_t)T * mask_words + words) * 4, stream));
+    si_union_bitmap_kernel<<<64, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, n_loaded, bitmap, nullptr);
+    si_union_kernel<<<1, 1024, smem, stream>>>(bitmap, n_loaded, union_out, n_union_out, pos, n_loaded);
     si_union_masks_kernel<<<64, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, 0, n_loaded, n_union_out, pos, masks,
                                                   mask_words, 0);
     SI_CUDA_TRY(cudaGetLastError());
@@ -593,9 +607,11 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     {
         const int words = (n_loaded + 31) / 32;
         size_t smem = (size_t)(2 * words + 2) * 4;
-        SI_CUDA_TRY(cudaMemsetAsync(masks, 0, (size_t)T * mask_words * 4, stream));
-        si_union_kernel<<<1, 1024, smem, stream>>>(idx, idx_offsets, k_fixed, T, shared ? 1 : 0, n_loaded, uni, n_union,
-                                                   pos, nu_pad, status_dev);
+        uint32_t *bitmap = masks + (size_t)T * mask_words;
+        SI_CUDA_TRY(cudaMemsetAsync(masks, 0, ((size_t)T * mask_words + words) * 4, stream));
+        si_union_bitmap_kernel<<<s->num_sms, 256, 0, stream>>>(idx, idx_offsets, k_fixed, shared ? 1 : T, n_loaded, bitmap,
+                                                               status_dev);
+        si_union_kernel<<<1, 1024, smem, stream>>>(bitmap, n_loaded, uni, n_union, pos, nu_pad);
         si_union_masks_kernel<<<2 * s->num_sms, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, shared ? 1 : 0, n_loaded,
                                                                    n_union, pos, masks, mask_words,
                                                                    (flags & SI_FLAG_UNION_UNMASKED) != 0);
@@ -628,8 +644,8 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     if ((size_t)t_pad_alloc * nu_pad * 2 > ws.h_bytes) return SI_ERR_NOMEM;
     {
         const size_t stage = 2 * 128 * 128 + (size_t)n_tok * 128;
-        P.nstage = pick_stages_gemm(stage); P.n_split = s1;
-        if (P.nstage < 3) return SI_ERR_UNSUPPORTED;   // the loaders run two chunks ahead of their arrivals
+        P.nstage = pick_stages_gemm(stage, n_tok); P.n_split = s1;
+        if (P.nstage < 2) return SI_ERR_UNSUPPORTED;
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(m_tiles, s1, tok_tiles);
@@ -643,7 +659,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
             si_gemm_combine_kernel<SI_F16><<<grid, 256, 0, stream>>>(P.partial, s1, nu_pad, t_pad_alloc, T, n_union, masks, mask_words, (uint16_t *)(wsb + ws.h_off));
     }
     // down: split K = union
-    int s2 = s->num_sms / ((d / 128) * tok_tiles);
+    int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
     if (s2 < 1) s2 = 1;
     if (s2 > 8) s2 = 8;
     if (s2 > nu_pad / kChunkK) s2 = nu_pad / kChunkK;
@@ -651,7 +667,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     if ((size_t)s2 * t_pad_alloc * d * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
     {
         const size_t stage = 64 * 256 + (size_t)n_tok * 128;
-        P.nstage = pick_stages_gemm(stage); P.n_split = s2;
+        P.nstage = pick_stages_gemm(stage, n_tok); P.n_split = s2;
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(d / 128, s2, tok_tiles);
