@@ -523,6 +523,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     fail |= !mbar_wait_bounded(&sm->accempty[q][ps % kReducerWarps], (uint32_t)((ps / kReducerWarps) & 1), cta_abort);
                 }
                 if (fail) break;
+                SI_PROF(4);                               // wait for the hand-over buffer
                 float *ab = accbuf + (size_t)q * d;
 #pragma unroll
                 for (int k2 = 0; k2 < NCH; ++k2) {
@@ -540,7 +541,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         }
 #undef SI_PROF
         if (prof) {
-            for (int i = 0; i < 4; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
+            for (int i = 0; i < 5; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
             P.prof[(size_t)b * 8 + 5] = pf[5] + pf[6];
         }
         if (fail && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -684,7 +685,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 break;
             }
         }
-        if (rprof) { P.prof[(size_t)b * 8 + 4] = rp_wait; P.prof[(size_t)b * 8 + 6] = rp_a; P.prof[(size_t)b * 8 + 7] = rp_b; }
+        if (rprof) { P.prof[(size_t)b * 8 + 6] = rp_a; P.prof[(size_t)b * 8 + 7] = rp_b; }
+        (void)rp_wait;
     }
 }
 
