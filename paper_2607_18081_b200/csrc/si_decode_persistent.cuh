@@ -12,7 +12,7 @@
 //     dealt round-robin across steps).  A bulk copy takes several microseconds to land and
 //     bandwidth needs every ring stage in flight, so a landed record is copied into
 //     registers and its stage handed back at once; the set then forms the two dot products
-//     (thread slices, warp butterfly, 8-warp exchange on an mbarrier), applies SiLU(g)*u and
+//     (thread slices, warp butterfly, 8-warp exchange through a hardware named barrier), applies SiLU(g)*u and
 //     accumulates h * down for its columns in fp32 registers -- while its next record is
 //     already on the way.  At the end of a step each set leaves its accumulators in shared
 //     memory for the reducer warps and goes straight on to the next step.
