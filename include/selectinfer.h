@@ -212,9 +212,12 @@ int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
              const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
              void *workspace, size_t ws_bytes, void *stream);
 
-/* Diagnostics: while dev_buf (device int64 [num_SMs][8]) is set, each persistent decode
- * launch stores per-SM cycle counts of its phases there (wait for x, wait for records,
- * record arithmetic, partial store, barrier arrive, wait for other SMs, reduction, unused).
+/* Diagnostics: while dev_buf (device int64 [num_SMs][16]) is set, each persistent decode
+ * launch stores per-SM cycle counts of its phases there.  Slots 0..5: first consumer set (wait
+ * for x, wait for a record + copy to registers, record arithmetic, accumulator hand-over,
+ * wait for the hand-over buffer, dot products + exchange); 6..7: second set (wait for the
+ * hand-over buffer, wait for a record); 8..13: first reducer warp (idle, wait for a free
+ * partial-ring slot, copy accumulators out, publish, wait for all SMs, reduce + write y).
  * Pass NULL to switch it off.  Costs a few clock reads per record. */
 int si_debug_decode_profile(void *dev_buf);
 

@@ -45,6 +45,7 @@ constexpr int kCounterStride = 64;                // uint32 per step: written at
 constexpr int kMaxStages = 16;
 constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
 constexpr int kPartialDepth = 6;                  // D: partial-y buffers in flight
+constexpr int kProfSlots = 16;                    // int64 cycle counters per SM in the optional phase profile
 constexpr int kLag = 2;                           // a step's cross-SM reduction starts this many steps later
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
 
@@ -65,7 +66,7 @@ struct Params {
                                   // stored their partial of the step, +32 "reduced" = CTAs that finished
                                   // reading the step's partials
     int32_t *status;
-    long long *prof;              // optional phase profile: int64 [G][8] cycle counters, or nullptr
+    long long *prof;              // optional phase profile: int64 [G][kProfSlots] cycle counters, or nullptr
     int stream_only;              // diagnostics bit mask (see si_debug_decode_stream_only)
     int prefetch_rounds;          // L2 prefetch distance in ring rounds (0 = off)
 };
@@ -121,6 +122,16 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, v
     int ok = 1;
     if (lane == 0) ok = mbar_wait_bounded(bar, parity, cta_abort) ? 1 : 0;
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+// Strong (gpu-scope) vector store and vector add-reduction at L2; one thread issues both to the same
+// address in program order, so the add lands on the stored value.
+__device__ __forceinline__ void st_relaxed_gpu_f4(float4 *p, float4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void red_add_gpu_f4(float4 *p, float4 v) {
+    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
 }
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
@@ -403,13 +414,18 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         return;
     }
 
-    if (warp <= kConsumerWarps) {
+    // Warp w runs on scheduler partition w mod 4.  The service warps (producer 0, reducers 4, 8, 12)
+    // share partition 0 with one consumer warp, so that their rarely executed code does not compete
+    // with four consumer warps for the partition's instruction cache and issue slots.
+    const bool is_reducer = (warp & 3) == 0 && warp >= 4 && warp <= 4 * kReducerWarps;
+    if (!is_reducer) {
         // ------------------------------------------------------------------ consumers
         // Two independent sets of 8 warps; set q consumes ring q.  A landed record is copied
         // into registers (3*NCH 16-byte chunks per thread) and its stage handed back at once;
         // the arithmetic then runs out of registers, so the ring is refilled while the set
         // computes.  Thread t of a set owns chunks t, t+256 of every row.
-        const int ct = tid - 32;                 // 0..511
+        const int cw = warp < 16 ? warp - (warp / 4 + 1) : warp - 4;   // consumer warp index 0..15
+        const int ct = cw * 32 + lane;           // 0..511
         const int q = ct >> 8;                   // consumer set
         const int t = ct & (kSetThreads - 1);    // thread within the set
         const int sw = t >> 5;                   // warp within the set
@@ -419,7 +435,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         uint32_t n = 0;                          // set-ring item counter
         uint32_t recs = 0;                       // records this set has handed to its barrier
         bool fail = false;
-        const bool prof = P.prof != nullptr && ct == 0;
+        const bool prof = P.prof != nullptr && t == 0;
         long long pf[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pt = prof ? clock64() : 0;
 #define SI_PROF(slot) do { if (prof) { long long now_ = clock64(); pf[slot] += now_ - pt; pt = now_; } } while (0)
 
@@ -540,10 +556,11 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             SI_PROF(3);                                   // accumulator hand-over
         }
 #undef SI_PROF
-        if (prof) {
-            for (int i = 0; i < 5; ++i) P.prof[(size_t)b * 8 + i] = pf[i];
-            P.prof[(size_t)b * 8 + 5] = pf[5] + pf[6];
+        if (prof && q == 0) {
+            for (int i = 0; i < 5; ++i) P.prof[(size_t)b * kProfSlots + i] = pf[i];
+            P.prof[(size_t)b * kProfSlots + 5] = pf[5] + pf[6];
         }
+        if (prof && q == 1) { P.prof[(size_t)b * kProfSlots + 6] = pf[4]; P.prof[(size_t)b * kProfSlots + 7] = pf[1]; }
         if (fail && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
         return;
     }
@@ -560,133 +577,146 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     //      ascending order; a warp butterfly combines the lanes (fixed order: deterministic
     //      split-K); y is written once; "partials of step sr consumed" is published.
     {
-        const int r = warp - 1 - kConsumerWarps;               // 0 .. kReducerWarps-1
+        const int r = warp / 4 - 1;                            // 0 .. kReducerWarps-1
         const bool nosync = (P.stream_only & 4) != 0;
         const int ngroups = d / 4;
         const int gpc = (ngroups + G - 1) / G;                 // <= kMaxGroups (launch check)
         const int g_valid = ngroups - b * gpc < gpc ? (ngroups - b * gpc < 0 ? 0 : ngroups - b * gpc) : gpc;
         const bool rprof = P.prof != nullptr && r == 0 && lane == 0;
-        long long rp_a = 0, rp_b = 0, rp_wait = 0;
+        long long rp[6] = {0, 0, 0, 0, 0, 0}, rt = rprof ? clock64() : 0;
+#define SI_RPROF(slot) do { if (rprof) { long long now_ = clock64(); rp[slot] += now_ - rt; rt = now_; } } while (0)
+        const int bg = lane & (kMaxGroups - 1);                // phase B: this lane's column group ...
+        const int brc = lane / kMaxGroups;                     // ... and row class (rows brc, brc + 4, ...)
+        constexpr int kRowClasses = 32 / kMaxGroups;
+        constexpr int kRowBatch = 13;                          // partial rows in flight per lane
         for (int step = r; step < P.n_steps + kLag; step += kReducerWarps) {
             int ok = 1;
-            long long c0 = rprof ? clock64() : 0;
             if (step < P.n_steps) {
-                // ---- phase A
-                if (lane == 0) {
-                    const uint32_t par = (uint32_t)((step / kReducerWarps) & 1);
-                    ok = mbar_wait_bounded(&sm->accfull[0][r], par, cta_abort) &&
-                         mbar_wait_bounded(&sm->accfull[1][r], par, cta_abort);
-                    if (ok && !nosync && step >= kPartialDepth)
-                        ok = counter_wait_bounded(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32,
-                                                  (unsigned)G, P.ctrl + 1, cta_abort);
-                }
-                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                long long c1 = rprof ? clock64() : 0;
-                if (rprof) rp_wait += c1 - c0;
-                if (ok) {
-                    const float4 *a0 = reinterpret_cast<const float4 *>(accbuf);
-                    const float4 *a1 = reinterpret_cast<const float4 *>(accbuf + d);
-                    float4 *dst = reinterpret_cast<float4 *>(P.partial + ((size_t)(step % kPartialDepth) * G + b) * d);
-                    // add the two sets' accumulators and store the CTA's partial y, 8 float4 per lane at a
-                    // time (loads first, so their latencies overlap)
-                    const int n4 = d / 4;
+                // ---- phase A: take each set's accumulators as soon as that set hands them over.  The
+                // first set's row is stored, the second set's is added with vector reductions at L2
+                // (a + b is the same whichever arrives first, so y stays bit-reproducible).
+                const uint32_t par = (uint32_t)((step / kReducerWarps) & 1);
+                float4 *dst = reinterpret_cast<float4 *>(P.partial + ((size_t)(step % kPartialDepth) * G + b) * d);
+                const int n4 = d / 4;
+                int taken = 0;                            // bit q: set q's accumulators already consumed
+                // has every SM finished reading the step that used this ring slot before?  Asked
+                // now, while nothing is waiting for this warp; the answer is needed after the idle wait.
+                unsigned freed = (unsigned)G;
+                if (lane == 0 && !nosync && step >= kPartialDepth)
+                    freed = ld_acquire_gpu(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32);
+                for (int sub = 0; sub < kSets && ok; ++sub) {
+                    int q = 0;
+                    if (lane == 0) {
+                        q = -1;
+                        long long t0 = clock64();
+                        while (q < 0) {
+                            if (!(taken & 1) && mbar_test_wait(&sm->accfull[0][r], par)) q = 0;
+                            else if (!(taken & 2) && mbar_test_wait(&sm->accfull[1][r], par)) q = 1;
+                            else {
+                                if (*cta_abort || clock64() - t0 > kWaitCycles) break;
+                                __nanosleep(64);
+                            }
+                        }
+                        ok = q >= 0;
+                        SI_RPROF(0);                      // idle: waiting for a set's hand-over
+                        if (ok && sub == 0 && freed < (unsigned)G)
+                            ok = counter_wait_bounded(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32,
+                                                      (unsigned)G, P.ctrl + 1, cta_abort);
+                    }
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                    q = __shfl_sync(0xFFFFFFFFu, q, 0);
+                    SI_RPROF(1);                          // ring slot of the partial buffer free again
+                    if (!ok) break;
+                    const float4 *a = reinterpret_cast<const float4 *>(accbuf + (size_t)q * d);
                     for (int i0 = 0; i0 < n4; i0 += 32 * 8) {
-                        float4 u0[8], u1[8];
+                        float4 u0[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const int i = i0 + lane + 32 * j;
-                            u0[j] = i < n4 ? a0[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-                            u1[j] = i < n4 ? a1[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+                            u0[j] = i < n4 ? a[i] : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const int i = i0 + lane + 32 * j;
-                            if (i < n4 && !nosync)
-                                __stcg(dst + i, make_float4(u0[j].x + u1[j].x, u0[j].y + u1[j].y, u0[j].z + u1[j].z, u0[j].w + u1[j].w));
+                            if (i < n4 && !nosync) {
+                                if (sub == 0) st_relaxed_gpu_f4(dst + i, u0[j]);
+                                else red_add_gpu_f4(dst + i, u0[j]);
+                            }
                         }
                     }
                     __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(&sm->accempty[0][r]); mbar_arrive(&sm->accempty[1][r]);
-                        if (!nosync) {
-                            __threadfence();
-                            atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
-                        }
-                    }
+                    if (lane == 0) mbar_arrive(&sm->accempty[q][r]);
+                    taken |= 1 << q;
+                    SI_RPROF(2);                          // copy the accumulators out
                 }
-                if (rprof) rp_a += clock64() - c1;
             }
-            if (ok && step >= kLag && !nosync) {
-                // ---- phase B
-                long long c2 = rprof ? clock64() : 0;
-                const int sr = step - kLag;
+            const int sr = step - kLag;
+            if (ok && sr >= 0 && !nosync) {
+                // ---- phase B: lane (group bg, row class brc) sums rows brc, brc + 4, ... of its column
+                // group in ascending order, kRowBatch loads in flight; two butterfly steps combine the
+                // four row classes (fixed order: deterministic split-K)
                 if (lane == 0)
                     ok = counter_wait_bounded(P.counters + (size_t)sr * kCounterStride, (unsigned)G, P.ctrl + 1, cta_abort);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                SI_RPROF(4);                              // every SM has published the step
                 if (ok) {
-                    float4 v[kMaxGroups];
-#pragma unroll
-                    for (int g = 0; g < kMaxGroups; ++g) v[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                     const float4 *base = reinterpret_cast<const float4 *>(
-                        P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4);
+                        P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4) + bg;
                     const size_t row_stride = (size_t)d / 4;
-                    if ((P.stream_only & 2) == 0) {
-                        for (int r0 = lane; r0 < G; r0 += 32) {
-                            float4 t0[kMaxGroups];
+                    if (bg < g_valid && (P.stream_only & 2) == 0) {
+                        for (int r0 = brc; r0 < G; r0 += kRowClasses * kRowBatch) {
+                            float4 t0[kRowBatch];
 #pragma unroll
-                            for (int g = 0; g < kMaxGroups; ++g) {
-                                t0[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (g < g_valid) t0[g] = __ldcg(base + (size_t)r0 * row_stride + g);
+                            for (int j = 0; j < kRowBatch; ++j) {
+                                const int row = r0 + kRowClasses * j;
+                                t0[j] = row < G ? __ldcg(base + (size_t)row * row_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
                             }
 #pragma unroll
-                            for (int g = 0; g < kMaxGroups; ++g) {
-                                v[g].x += t0[g].x; v[g].y += t0[g].y; v[g].z += t0[g].z; v[g].w += t0[g].w;
-                            }
+                            for (int j = 0; j < kRowBatch; ++j) { v.x += t0[j].x; v.y += t0[j].y; v.z += t0[j].z; v.w += t0[j].w; }
                         }
                     }
 #pragma unroll
-                    for (int g = 0; g < kMaxGroups; ++g) {
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            v[g].x += __shfl_xor_sync(0xFFFFFFFFu, v[g].x, o); v[g].y += __shfl_xor_sync(0xFFFFFFFFu, v[g].y, o);
-                            v[g].z += __shfl_xor_sync(0xFFFFFFFFu, v[g].z, o); v[g].w += __shfl_xor_sync(0xFFFFFFFFu, v[g].w, o);
-                        }
+                    for (int o = kMaxGroups; o < 32; o <<= 1) {
+                        v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, o); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, o);
+                        v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, o); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, o);
                     }
-                    float4 mine_v = make_float4(0.f, 0.f, 0.f, 0.f);      // lane g writes column group g
-#pragma unroll
-                    for (int g = 0; g < kMaxGroups; ++g) if (lane == g) mine_v = v[g];
-                    if (lane < g_valid) {
-                        const size_t col = (size_t)sr * d + (size_t)(b * gpc + lane) * 4;
+                    if (brc == 0 && bg < g_valid) {
+                        const size_t col = (size_t)sr * d + (size_t)(b * gpc + bg) * 4;
                         if (P.residual) {
                             uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
-                            mine_v.x += si_cvt<DT>::lo(xw.x); mine_v.y += si_cvt<DT>::hi(xw.x);
-                            mine_v.z += si_cvt<DT>::lo(xw.y); mine_v.w += si_cvt<DT>::hi(xw.y);
+                            v.x += si_cvt<DT>::lo(xw.x); v.y += si_cvt<DT>::hi(xw.x);
+                            v.z += si_cvt<DT>::lo(xw.y); v.w += si_cvt<DT>::hi(xw.y);
                         }
                         if (P.y_f32) {
-                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + col) = mine_v;
+                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + col) = v;
                         } else {
                             uint2 o;
-                            o.x = (uint32_t)si_cvt<DT>::from_float(mine_v.x) | ((uint32_t)si_cvt<DT>::from_float(mine_v.y) << 16);
-                            o.y = (uint32_t)si_cvt<DT>::from_float(mine_v.z) | ((uint32_t)si_cvt<DT>::from_float(mine_v.w) << 16);
+                            o.x = (uint32_t)si_cvt<DT>::from_float(v.x) | ((uint32_t)si_cvt<DT>::from_float(v.y) << 16);
+                            o.y = (uint32_t)si_cvt<DT>::from_float(v.z) | ((uint32_t)si_cvt<DT>::from_float(v.w) << 16);
                             *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(P.y) + col) = o;
                         }
                     }
-                    __syncwarp();
-                    // the ring slot of step sr may be overwritten once every CTA has said so
-                    if (lane == 0 && sr + kPartialDepth < P.n_steps) {
-                        __threadfence();
-                        atomicAdd(P.counters + (size_t)sr * kCounterStride + 32, 1u);
-                    }
                 }
-                if (rprof) rp_b += clock64() - c2;
+                SI_RPROF(5);                              // load + sum the partial rows, write y
             }
             if (!ok) {
                 if (lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
                 break;
             }
+            // ---- publish with one fence: "partial of this step stored" and "partials of step sr
+            // consumed" (its ring slot may be overwritten once every SM has said so)
+            __syncwarp();
+            if (lane == 0 && !nosync) {
+                __threadfence();
+                if (step < P.n_steps) atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
+                if (sr >= 0 && sr + kPartialDepth < P.n_steps) atomicAdd(P.counters + (size_t)sr * kCounterStride + 32, 1u);
+            }
+            SI_RPROF(3);                                  // publish (fence + atomics)
         }
-        if (rprof) { P.prof[(size_t)b * 8 + 6] = rp_a; P.prof[(size_t)b * 8 + 7] = rp_b; }
-        (void)rp_wait;
+        if (rprof)
+            for (int i = 0; i < 6; ++i) P.prof[(size_t)b * kProfSlots + 8 + i] = rp[i];
+#undef SI_RPROF
     }
 }
 
