@@ -54,8 +54,8 @@ struct si_ws_layout {
     size_t ctrl_off, ctrl_bytes;
     size_t partial_off, partial_bytes;
     size_t sel_off, sel_bytes;         // int32 [T_max][k_max] selected lists + [T_max] counts
-    size_t union_off, union_bytes;     // int32 [n_loaded_max] union + count + bitmap words
-    size_t mask_off, mask_bytes;       // uint32 [T_max][ceil(n_loaded_max / 32)]
+    size_t union_off, union_bytes;     // int32 [n_loaded_max] union + count
+    size_t mask_off, mask_bytes;       // uint32 [T_max + 1][ceil(n_loaded_max / 32)] slot bitmaps, then counters
     size_t h_off, h_bytes;             // 16-bit H [T_pad][n_loaded_max padded]
     size_t selws_off, selws_bytes;     // selector scratch
     size_t steps_off, steps_bytes;     // per-step descriptors for stack calls
@@ -89,6 +89,7 @@ int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed,
 
 // implemented in si_gemm.cu
 size_t si_gemm_partial_bytes(const si_store *s, int T_max);
+size_t si_gemm_counter_bytes(const si_store *s, size_t nl_pad, size_t t_pad);
 int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
                     int k_fixed, int32_t *union_out, int32_t *n_union_out, void *workspace,
                     size_t ws_bytes, cudaStream_t stream);

@@ -439,7 +439,6 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         long long pf[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pt = prof ? clock64() : 0;
 #define SI_PROF(slot) do { if (prof) { long long now_ = clock64(); pf[slot] += now_ - pt; pt = now_; } } while (0)
 
-        const bool nosync = (P.stream_only & 4) != 0;   // diagnostics: no cross-CTA exchange at all
         const bool noarith = (P.stream_only & 1) != 0;  // diagnostics: drain only
 
         for (int step = 0; step < P.n_steps && !fail; ++step) {

@@ -21,8 +21,9 @@
 
 namespace {
 
-constexpr int kLoaderThreads = 128;              // warps 0..3: gather loads, later the epilogue
-constexpr int kGemmThreads = kLoaderThreads + 32; // warp 4: MMA issue + tensor-memory allocation
+constexpr int kLoaderThreads = 256;              // warps 0..7: gather loads, later the epilogue
+constexpr int kLoaderWarps = kLoaderThreads / 32;
+constexpr int kGemmThreads = kLoaderThreads + 32; // warp 8: MMA issue + tensor-memory allocation
 constexpr int kMaxStages = 6;
 constexpr int kChunkK = 64;                      // K elements per pipeline stage (128 bytes per row)
 constexpr long long kSpinLimit = 1ll << 24;      // bounded waits (mbarrier probes)
@@ -52,6 +53,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
 }
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+// 16-byte copy that reads src_bytes (0 or 16) bytes and zero-fills the rest
+__device__ __forceinline__ void cp_async16_zfill(void *dst_smem, const void *src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -103,31 +108,50 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 // ------------------------------------------------------------------------------- union
-// Step 1 (many CTAs): OR every list entry into a bitmap over the loaded slots (zero on entry).
-__global__ void si_union_bitmap_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed,
-                                       int n_lists, int n_loaded, uint32_t *__restrict__ bitmap, int32_t *status) {
+// Sorted union of the lists in one launch.  Every block ORs its share of the list entries into a
+// bitmap over the loaded slots and -- when each token has its own list -- into that token's own
+// slot bitmap (membership test of the combine step).  The block that finishes last turns the
+// bitmap into the ascending union by a popcount prefix scan.  bitmap, tokbits and ticket are zero
+// on entry.  blockDim.x = 1024; dynamic shared memory = (2 * words + 2) * 4 bytes.
+__global__ void __launch_bounds__(1024)
+si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int n_lists,
+                      int n_loaded, uint32_t *bitmap_g, uint32_t *tokbits, int mask_words, unsigned *ticket,
+                      int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out, int union_cap, int32_t *status) {
+    extern __shared__ uint32_t sh[];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long total = offsets ? offsets[n_lists] : (long long)n_lists * k_fixed;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    for (long long e = (long long)blockIdx.x * blockDim.x + tid; e < total; e += (long long)gridDim.x * blockDim.x) {
         const int s = idx[e];
         if (s < 0 || s >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
         const uint32_t bit = 1u << (s & 31);
-        if (!(bitmap[s >> 5] & bit)) atomicOr(&bitmap[s >> 5], bit);     // hot slots are set by the first token
+        if (!(bitmap_g[s >> 5] & bit)) atomicOr(&bitmap_g[s >> 5], bit);     // hot slots are set by the first token
+        if (tokbits) {
+            int t;
+            if (offsets) {            // largest t with offsets[t] <= e
+                int lo = 0, hi = n_lists;
+                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
+                t = lo;
+            } else {
+                t = (int)(e / k_fixed);
+            }
+            atomicOr(&tokbits[(size_t)t * mask_words + (s >> 5)], bit);
+        }
     }
-}
-
-// Step 2 (one CTA): popcount prefix scan over the bitmap -> sorted union, slot -> position map.
-__global__ void __launch_bounds__(1024)
-si_union_kernel(const uint32_t *__restrict__ bitmap_g, int n_loaded, int32_t *__restrict__ union_out,
-                int32_t *__restrict__ n_union_out, int32_t *__restrict__ pos_of_slot, int union_cap) {
-    extern __shared__ uint32_t sh[];
-    uint32_t *bitmap = sh;                         // [words]
-    uint32_t *wprefix = sh + (n_loaded + 31) / 32; // [words] exclusive popcount prefix
-    __shared__ uint32_t warp_tot[32];
-    const int words = (n_loaded + 31) / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int w = tid; w < words; w += 1024) bitmap[w] = bitmap_g[w];
+    __threadfence();
     __syncthreads();
-    // exclusive prefix of popcounts over the bitmap words (words <= 2048 for d_ff <= 65536)
+    if (tid == 0) is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // ---- last block: popcount prefix scan over the bitmap -> ascending union
+    const int words = (n_loaded + 31) / 32;
+    uint32_t *bitmap = sh;                         // [words]
+    uint32_t *wprefix = sh + words;                // [words] exclusive popcount prefix
+    for (int w = tid; w < words; w += 1024) bitmap[w] = __ldcg(bitmap_g + w);
+    __syncthreads();
     uint32_t carry = 0;
     for (int base = 0; base < words; base += 1024) {
         int w = base + tid;
@@ -140,7 +164,7 @@ si_union_kernel(const uint32_t *__restrict__ bitmap_g, int n_loaded, int32_t *__
             uint32_t v = warp_tot[lane], vi = v;
             for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, vi, o); if (lane >= o) vi += t; }
             warp_tot[lane] = vi - v;
-            if (lane == 31) warp_tot[31] = vi - v, sh[2 * words] = vi;   // total of this block of words
+            if (lane == 31) sh[2 * words] = vi;    // total of this block of words
         }
         __syncthreads();
         if (w < words) wprefix[w] = carry + warp_tot[warp] + inc - c;
@@ -149,56 +173,19 @@ si_union_kernel(const uint32_t *__restrict__ bitmap_g, int n_loaded, int32_t *__
     }
     const int n_u = (int)carry;
     if (tid == 0) *n_union_out = n_u;
-    // emit the union (ascending) and the slot -> position map
     for (int w = tid; w < words; w += 1024) {
         uint32_t bits = bitmap[w]; int p = (int)wprefix[w];
         while (bits) {
             int bpos = __ffs(bits) - 1; bits &= bits - 1;
-            int s = w * 32 + bpos;
-            if (p < union_cap) union_out[p] = s;
-            pos_of_slot[s] = p;
+            if (p < union_cap) union_out[p] = w * 32 + bpos;
             ++p;
         }
     }
-    // pad the union up to the capacity with its first entry (masked out everywhere)
-    __syncthreads();
+    // pad the union up to the capacity with its first entry (padded positions contribute nothing)
     {
         int first = 0;
         for (int w = 0; w < words; ++w) if (bitmap[w]) { first = w * 32 + __ffs(bitmap[w]) - 1; break; }
         for (int p = n_u + tid; p < union_cap; p += 1024) union_out[p] = first;
-    }
-}
-
-// Membership masks over union positions, many CTAs: mask[t] bit p set iff U[p] is in list t.
-// The masks are zero on entry (memset by the host side of the call).
-__global__ void si_union_masks_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed,
-                                      int T, int shared_list, int n_loaded, const int32_t *__restrict__ n_union,
-                                      const int32_t *__restrict__ pos_of_slot, uint32_t *__restrict__ masks,
-                                      int mask_words, int unmasked) {
-    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x, gstride = (long long)gridDim.x * blockDim.x;
-    if (unmasked || shared_list) {
-        // every token uses the whole union (with one shared list the union is that list)
-        const int n_u = *n_union;
-        for (long long i = gid; i < (long long)T * mask_words; i += gstride) {
-            const int lo = (int)(i % mask_words) * 32;
-            masks[i] = lo + 32 <= n_u ? 0xFFFFFFFFu : (lo < n_u ? ((1u << (n_u - lo)) - 1u) : 0u);
-        }
-        return;
-    }
-    const long long total = offsets ? offsets[T] : (long long)T * k_fixed;
-    for (long long e = gid; e < total; e += gstride) {
-        int t;
-        if (offsets) {            // largest t with offsets[t] <= e
-            int lo = 0, hi = T;
-            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
-            t = lo;
-        } else {
-            t = (int)(e / k_fixed);
-        }
-        const int s = idx[e];
-        if (s < 0 || s >= n_loaded) continue;
-        const int p = pos_of_slot[s];
-        atomicOr(&masks[(size_t)t * mask_words + (p >> 5)], 1u << (p & 31));
     }
 }
 
@@ -218,12 +205,20 @@ struct GemmParams {
     int fmt;                       // 0 f16, 1 bf16
     int nstage;
     int32_t *status;
+    // fused finishing passes: the CTA that completes a tile's last K split sums the splits
+    unsigned *tile_ctr;            // per (tile, token tile) arrival counters, zero on entry
+    const uint32_t *tokbits;       // [T][mask_words] slot bitmaps of the tokens' own lists, or nullptr: all tokens
+    int mask_words;                //   use the whole union
+    uint16_t *h_out;               // gate/up: H [t_pad_total][nu_pad]
+    void *y;                       // down: output [T][d_model]
+    int y_f32, residual;
 };
 
 // Gate/up contraction.  grid = (union tiles of 128, K splits of d_model, token tiles).
 // D_gate[128 neurons x N tokens] (+)= Wg[U tile, k] . X[tokens, k]^T, same for up, accumulated in
 // tensor memory (columns [0,N) gate, [N,2N) up).
-__global__ void __launch_bounds__(kGemmThreads, 2)
+__global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
+
 si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
@@ -251,7 +246,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == kLoaderWarps) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(ncols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -260,38 +255,39 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp < 4) {
+    if (warp < kLoaderWarps) {
         // ---------------------------------------------------------------- gather loads
-        // Copy j of a thread covers 16-byte piece (tid & 7) of tile row 16*j + (tid >> 3): the 32 lanes
+        // Copy j of a thread covers 16-byte piece (tid & 7) of tile row 32*j + (tid >> 3): the 32 lanes
         // of a warp instruction read four whole 128-byte row segments, so the gather is coalesced.
-        const int q8 = tid & 7;
-        const char *grow[8];                                         // gate rows; the up row follows at d_model*2
+        // All addresses advance by constants, so a chunk costs a handful of instructions per copy.
+        const int q8 = tid & 7, r32 = tid >> 3;
+        const char *grow[4];                                         // gate rows; the up row follows at d_model*2
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            grow[j] = P.rec_base + (size_t)P.union_slots[mt * 128 + 16 * j + (tid >> 3)] * P.rec_bytes + q8 * 16;
-        const int r = tid;                                           // epilogue: this thread's tile row
+        for (int j = 0; j < 4; ++j)
+            grow[j] = P.rec_base + (size_t)P.union_slots[mt * 128 + 32 * j + r32] * P.rec_bytes + q8 * 16 + (size_t)c0 * 128;
+        const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);      // rows 32*j + r32 share (row & 7)
+        const size_t up_off = (size_t)P.d_model * 2;
+        const char *xsrc = reinterpret_cast<const char *>(P.x) + ((size_t)(tok0 + r32) * P.d_model + (size_t)c0 * kChunkK) * 2 + q8 * 16;
+        const size_t xstride = (size_t)32 * P.d_model * 2;           // 32 token rows further
         int pending = 0;                                             // committed groups not yet signalled
         const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;         // chunks of copies kept in flight
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
-            uint8_t *sg = tiles + (size_t)st * stage_bytes, *su = sg + 128 * 128, *sx = su + 128 * 128;
+            uint8_t *sg = tiles + (size_t)st * stage_bytes + off0, *su = sg + 128 * 128, *sx = su + 128 * 128;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int row = 16 * j + (tid >> 3);
-                const char *gsrc = grow[j] + (size_t)(c0 + c) * 128;
-                const int off = row * 128 + ((q8 ^ (row & 7)) << 4);
-                cp_async16(sg + off, gsrc);
-                cp_async16(su + off, gsrc + (size_t)P.d_model * 2);
+            for (int j = 0; j < 4; ++j) {
+                cp_async16(sg + j * 4096, grow[j]);
+                cp_async16(su + j * 4096, grow[j] + up_off);
+                grow[j] += 128;
             }
-            for (int e = tid; e < N * 8; e += kLoaderThreads) {
-                const int n = e >> 3, q = e & 7;
-                const int tok = tok0 + n;
-                if (tok < P.T)
-                    cp_async16(sx + n * 128 + ((q ^ (n & 7)) << 4),
-                               reinterpret_cast<const char *>(P.x) + ((size_t)tok * P.d_model + (size_t)(c0 + c) * kChunkK) * 2 + q * 16);
-                else
-                    *reinterpret_cast<uint4 *>(sx + n * 128 + ((q ^ (n & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            {
+                const char *xs = xsrc;
+                for (int n = r32; n < N; n += 32, xs += xstride) {
+                    const bool in = tok0 + n < P.T;                  // padded token rows are zero-filled
+                    cp_async16_zfill(sx + (n - r32) * 128, in ? xs : reinterpret_cast<const char *>(P.x), in ? 16 : 0);
+                }
+                xsrc += 128;
             }
             cp_async_commit();
             ++pending;
@@ -316,25 +312,26 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         // ---------------------------------------------------------------- epilogue
         bool ok = !*failed && mbar_wait(accbar, 0);
         tc_fence_after();
+        // a warp reads tensor-memory lanes 32*(warp % 4) ..: warps w and w + 4 share the rows and take
+        // alternate 16-column blocks.  Thread row r = union row mt*128 + r: N gate values, N up values
+        const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
+        float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
+        float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
         if (ok && n_chunks > 0) {
-            // thread r holds union row mt*128 + r: N gate values then N up values
-            float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-            float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-            for (int n0 = 0; n0 < N; n0 += 16) {
+            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
                 uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)n0, v);
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     *reinterpret_cast<uint4 *>(pg + n0 + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(N + n0), v);
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(N + n0), v);
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     *reinterpret_cast<uint4 *>(pu + n0 + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
             }
         } else if (ok) {
-            float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-            float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-            for (int n = 0; n < N; ++n) { pg[n] = 0.f; pu[n] = 0.f; }
+            for (int n0 = 16 * cb; n0 < N; n0 += 32)
+                for (int n = n0; n < n0 + 16; ++n) { pg[n] = 0.f; pu[n] = 0.f; }
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else {
@@ -360,38 +357,82 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
             umma_commit(accbar);                  // accumulators complete (or nothing was issued)
         }
     }
+    __threadfence();                       // this CTA's partial tile is visible device-wide ...
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kLoaderWarps) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
     }
-}
-
-// H[t][i] = mask ? SiLU(sum_s G) * (sum_s U) : 0, rounded to the store dtype.  grid over (t, i).
-template <int DT>
-__global__ void si_gemm_combine_kernel(const float *__restrict__ partial, int n_split, int nu_pad, int t_pad_total,
-                                       int T, const int32_t *__restrict__ n_union, const uint32_t *__restrict__ masks,
-                                       int mask_words, uint16_t *__restrict__ h) {
-    // threads run over tokens fastest (the partial tiles are [position][token]); H is [token][position]
-    const int t = blockIdx.x * 32 + (threadIdx.x & 31);
-    const int i = blockIdx.y * 8 + (threadIdx.x >> 5);
-    if (i >= nu_pad || t >= t_pad_total) return;
-    float out = 0.f;
-    if (t < T && i < *n_union && ((masks[(size_t)t * mask_words + (i >> 5)] >> (i & 31)) & 1u)) {
-        float g = 0.f, u = 0.f;
-        for (int s = 0; s < n_split; ++s) {
-            g += partial[(((size_t)s * 2 + 0) * nu_pad + i) * t_pad_total + t];
-            u += partial[(((size_t)s * 2 + 1) * nu_pad + i) * t_pad_total + t];
+    // ---- combine: the CTA that delivers the tile's last K split forms H for the tile.  The splits are
+    // summed in split order whoever is last, so H does not depend on the arrival order.
+    int *last_flag = const_cast<int *>(failed) + 1;
+    if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
+    __syncthreads();
+    if (!*last_flag || *failed) return;
+    __threadfence();
+    {
+        // H[t][i] = member(t, U[i]) ? SiLU(sum_s G) * (sum_s U) : 0, rounded to the store dtype.  Reads
+        // run along tokens (the partial tiles are [position][token]), H is [token][position]: transpose
+        // through shared memory (the pipeline stages are free now)
+        constexpr int kRowPitch = 128 + 8;                           // uint16 per token row of the staging tile
+        uint16_t *hs = reinterpret_cast<uint16_t *>(smem);
+        const size_t plane = (size_t)P.nu_pad * P.t_pad_total;       // one gate or up plane of a split
+        // one item = (union row, four consecutive tokens); all of an item's loads are issued before any
+        // is used, four splits at a time
+        const int nq = N / 4;
+        for (int it = tid; it < 128 * nq; it += kGemmThreads) {
+            const int r = it / nq, n = (it - r * nq) * 4;
+            const int i = mt * 128 + r;
+            const float *prow = P.partial + (size_t)i * P.t_pad_total + tok0 + n;
+            float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+            for (int sp0 = 0; sp0 < P.n_split; sp0 += 4) {
+                float4 gv[4], uv[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const bool in = sp0 + k < P.n_split;
+                    gv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k)) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    uv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k) + 1) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    g.x += gv[k].x; g.y += gv[k].y; g.z += gv[k].z; g.w += gv[k].w;
+                    u.x += uv[k].x; u.y += uv[k].y; u.z += uv[k].z; u.w += uv[k].w;
+                }
+            }
+            const float gg[4] = {g.x, g.y, g.z, g.w}, uu[4] = {u.x, u.y, u.z, u.w};
+            uint32_t member = 0;
+            if (i < n_u) {
+                if (P.tokbits) {
+                    const int slot = P.union_slots[i];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (tok0 + n + k < P.T)
+                            member |= ((P.tokbits[(size_t)(tok0 + n + k) * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u) << k;
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) member |= (tok0 + n + k < P.T ? 1u : 0u) << k;
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float out = (member >> k) & 1u ? si_silu_mul(gg[k], uu[k]) : 0.f;
+                hs[(n + k) * kRowPitch + r] = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
+            }
         }
-        out = si_silu_mul(g, u);
+        __syncthreads();
+        for (int e = tid; e < N * 16; e += kGemmThreads) {
+            const int n = e >> 4, piece = e & 15;
+            *reinterpret_cast<uint4 *>(P.h_out + (size_t)(tok0 + n) * P.nu_pad + (size_t)mt * 128 + piece * 8) =
+                *reinterpret_cast<const uint4 *>(hs + n * kRowPitch + piece * 8);
+        }
     }
-    h[(size_t)t * nu_pad + i] = si_cvt<DT>::from_float(out);
 }
 
 // Down contraction.  grid = (d_model / 128 column tiles, K splits over the union, token tiles).
 // D[128 output columns x N tokens] (+)= Wd[U_k, columns]^T . H[tokens, U_k]^T: A is MN-major (a
 // down row is contiguous along the output columns), B is K-major.
-__global__ void __launch_bounds__(kGemmThreads, 2)
+__global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
+
 si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
@@ -419,7 +460,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
         *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == kLoaderWarps) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(ncols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -428,39 +469,42 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp < 4) {
+    if (warp < kLoaderWarps) {
         // Copy j of a thread covers 16-byte piece (tid & 15) of the 256-byte down-row segment of union
-        // entry 8*j + (tid >> 4) of the chunk: a warp instruction reads two whole segments (coalesced).
-        const int c16 = tid & 15;
+        // entry 16*j + (tid >> 4) of the chunk: a warp instruction reads two whole segments (coalesced).
+        const int c16 = tid & 15, e16 = tid >> 4;
         int pending = 0;
         const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;
-        int slots_next[8];                                           // union slots of the next chunk (prefetched)
+        int slots_next[4];                                           // union slots of the next chunk (prefetched)
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            slots_next[j] = n_chunks > 0 ? P.union_slots[c0 * kChunkK + 8 * j + (tid >> 4)] : 0;
+        for (int j = 0; j < 4; ++j)
+            slots_next[j] = n_chunks > 0 ? P.union_slots[c0 * kChunkK + 16 * j + e16] : 0;
+        // entry kk = 16*j + e16 lands at (kk >> 3) * 2048 + half * 1024 + (kk & 7) * 128 + swizzled piece
+        const int k8 = e16 & 7;
+        const int dst0 = (e16 >> 3) * 2048 + (c16 >> 3) * 1024 + k8 * 128 + (((c16 & 7) ^ k8) << 4);
+        const char *dsrc0 = P.rec_base + (size_t)P.d_model * 4 + (size_t)mt * 256 + c16 * 16;
+        // H tile: piece (tid & 7) of token rows (tid >> 3) + 32*i
+        const int q8 = tid & 7, r32 = tid >> 3;
+        const int hoff0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);
+        const char *hsrc = reinterpret_cast<const char *>(P.h) + ((size_t)(tok0 + r32) * P.nu_pad + (size_t)c0 * kChunkK) * 2 + q8 * 16;
+        const size_t hstride = (size_t)32 * P.nu_pad * 2;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
-            int slots[8];
+            int slots[4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < 4; ++j) {
                 slots[j] = slots_next[j];
-                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c0 + c + 1) * kChunkK + 8 * j + (tid >> 4)];
+                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c0 + c + 1) * kChunkK + 16 * j + e16];
             }
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
-            uint8_t *sa = tiles + (size_t)st * stage_bytes, *sh = sa + 64 * 256;
+            uint8_t *sa = tiles + (size_t)st * stage_bytes, *sh = sa + 64 * 256 + hoff0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int kk = 8 * j + (tid >> 4);                              // union entry of the chunk
-                const int slot = slots[j];                                      // padded entries carry a valid slot
-                const char *src = P.rec_base + (size_t)slot * P.rec_bytes + (size_t)P.d_model * 4 +
-                                  (size_t)mt * 256 + c16 * 16;
-                const int half = c16 >> 3, q = c16 & 7, k8 = kk & 7;
-                cp_async16(sa + (kk >> 3) * 2048 + half * 1024 + k8 * 128 + ((q ^ k8) << 4), src);
-            }
-            for (int e = tid; e < N * 8; e += kLoaderThreads) {
-                const int n = e >> 3, q = e & 7;
-                cp_async16(sh + n * 128 + ((q ^ (n & 7)) << 4),
-                           reinterpret_cast<const char *>(P.h) + ((size_t)(tok0 + n) * P.nu_pad + (size_t)(c0 + c) * kChunkK) * 2 + q * 16);
+            for (int j = 0; j < 4; ++j)                                      // padded entries carry a valid slot
+                cp_async16(sa + j * 4096 + dst0, dsrc0 + (size_t)slots[j] * P.rec_bytes);
+            {
+                const char *hs = hsrc;
+                for (int n = r32; n < N; n += 32, hs += hstride) cp_async16(sh + (n - r32) * 128, hs);
+                hsrc += 128;
             }
             cp_async_commit();
             ++pending;
@@ -483,17 +527,20 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
         }
         bool ok = !*failed && mbar_wait(accbar, 0);
         tc_fence_after();
-        // thread holds output column mt*128 + tid for N tokens
-        float *py = P.partial + ((size_t)ks * P.t_pad_total + tok0) * P.d_model + (size_t)mt * 128 + tid;
+        // thread holds output column mt*128 + r for the tokens; warps w and w + 4 share the rows and
+        // take alternate 16-token blocks
+        const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
+        float *py = P.partial + ((size_t)ks * P.t_pad_total + tok0) * P.d_model + (size_t)mt * 128 + r;
         if (ok && n_chunks > 0) {
-            for (int n0 = 0; n0 < N; n0 += 16) {
+            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
                 uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)n0, v);
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
 #pragma unroll
                 for (int q = 0; q < 16; ++q) py[(size_t)(n0 + q) * P.d_model] = __uint_as_float(v[q]);
             }
         } else if (ok) {
-            for (int n = 0; n < N; ++n) py[(size_t)n * P.d_model] = 0.f;
+            for (int n0 = 16 * cb; n0 < N; n0 += 32)
+                for (int n = n0; n < n0 + 16; ++n) py[(size_t)n * P.d_model] = 0.f;
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else {
@@ -516,10 +563,53 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
             umma_commit(accbar);
         }
     }
+    __threadfence();                       // this CTA's partial tile is visible device-wide ...
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kLoaderWarps) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
+    }
+    // ---- reduce: the CTA that delivers the column tile's last K split writes y for the tile:
+    // y[t][j] = (x[t][j] +) sum over the splits in split order (independent of the arrival order)
+    int *last_flag = const_cast<int *>(failed) + 1;
+    if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
+    __syncthreads();
+    if (!*last_flag || *failed) return;
+    __threadfence();
+    // one item = (token, four consecutive columns); an item's loads are issued before any is used
+    for (int it = tid; it < N * 32; it += kGemmThreads) {
+        const int n = it >> 5, col = mt * 128 + (it & 31) * 4, t = tok0 + n;
+        if (t >= P.T) continue;
+        const float *pp = P.partial + (size_t)t * P.d_model + col;
+        const size_t plane = (size_t)P.t_pad_total * P.d_model;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp0 = 0; sp0 < P.n_split; sp0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                v[k] = sp0 + k < P.n_split ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(sp0 + k) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { a.x += v[k].x; a.y += v[k].y; a.z += v[k].z; a.w += v[k].w; }
+        }
+        const size_t o = (size_t)t * P.d_model + col;
+        if (P.residual) {
+            const uint2 xw = *reinterpret_cast<const uint2 *>(P.x + o);
+            if (P.fmt) { a.x += si_cvt<SI_BF16>::lo(xw.x); a.y += si_cvt<SI_BF16>::hi(xw.x); a.z += si_cvt<SI_BF16>::lo(xw.y); a.w += si_cvt<SI_BF16>::hi(xw.y); }
+            else { a.x += si_cvt<SI_F16>::lo(xw.x); a.y += si_cvt<SI_F16>::hi(xw.x); a.z += si_cvt<SI_F16>::lo(xw.y); a.w += si_cvt<SI_F16>::hi(xw.y); }
+        }
+        if (P.y_f32) {
+            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + o) = a;
+        } else {
+            uint2 w;
+            if (P.fmt) {
+                w.x = (uint32_t)si_cvt<SI_BF16>::from_float(a.x) | ((uint32_t)si_cvt<SI_BF16>::from_float(a.y) << 16);
+                w.y = (uint32_t)si_cvt<SI_BF16>::from_float(a.z) | ((uint32_t)si_cvt<SI_BF16>::from_float(a.w) << 16);
+            } else {
+                w.x = (uint32_t)si_cvt<SI_F16>::from_float(a.x) | ((uint32_t)si_cvt<SI_F16>::from_float(a.y) << 16);
+                w.y = (uint32_t)si_cvt<SI_F16>::from_float(a.z) | ((uint32_t)si_cvt<SI_F16>::from_float(a.w) << 16);
+            }
+            *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(P.y) + o) = w;
+        }
     }
 }
 
@@ -543,6 +633,26 @@ int pick_stages_gemm(size_t stage_bytes, int n_tok) {
     return n > kMaxStages ? kMaxStages : n;
 }
 
+// Zero-on-entry scratch of a multi-token call, carved from the workspace's mask region:
+// [T][mask_words] token slot bitmaps | [mask_words] union bitmap | counters (ticket, tile counters)
+struct UnionScratch { uint32_t *tokbits, *bitmap; unsigned *ticket, *ctr; size_t zero_bytes; int mask_words; };
+UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws, int T, int n_loaded, int n_ctr) {
+    (void)s;
+    UnionScratch u;
+    u.mask_words = (int)(si_align_up((size_t)n_loaded, 128) / 32);
+    u.tokbits = (uint32_t *)(wsb + ws.mask_off);
+    u.bitmap = u.tokbits + (size_t)T * u.mask_words;
+    u.ticket = (unsigned *)(u.bitmap + u.mask_words);
+    u.ctr = u.ticket + 64;
+    u.zero_bytes = ((size_t)(T + 1) * u.mask_words + 64 + (size_t)n_ctr) * 4;
+    return u;
+}
+int union_blocks(const si_store *s, long long entries) {
+    long long b = (entries + 4095) / 4096;           // four entries per thread at least
+    if (b < 1) b = 1;
+    return (int)(b > s->num_sms ? s->num_sms : b);
+}
+
 }  // namespace
 
 size_t si_gemm_partial_bytes(const si_store *s, int T_max) {
@@ -550,24 +660,25 @@ size_t si_gemm_partial_bytes(const si_store *s, int T_max) {
     return T_max > 1 ? kPartialCap : 0;
 }
 
+// Counters a call may need beyond the bitmaps: one per (tile, token tile) of either contraction.
+size_t si_gemm_counter_bytes(const si_store *s, size_t nl_pad, size_t t_pad) {
+    const size_t tok_tiles = (t_pad + 255) / 256;
+    return (64 + (nl_pad / 128 + (size_t)s->d_model / 128 + 2) * tok_tiles) * 4;
+}
+
 int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
                     int k_fixed, int32_t *union_out, int32_t *n_union_out, void *workspace, size_t ws_bytes,
                     cudaStream_t stream) {
     si_ws_layout ws = si_ws_carve(s, T, k_fixed, 1);
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
-    char *wsb = (char *)workspace;
     const int n_loaded = s->n_loaded[layer];
     const int words = (n_loaded + 31) / 32;
-    int32_t *pos = (int32_t *)(wsb + ws.union_off) + si_align_up((size_t)n_loaded, 128) + 64;
-    uint32_t *masks = (uint32_t *)(wsb + ws.mask_off);
-    const int mask_words = (int)(si_align_up((size_t)n_loaded, 128) / 32);
-    size_t smem = (size_t)(2 * words + 2) * 4;
-    uint32_t *bitmap = masks + (size_t)T * mask_words;
-    SI_CUDA_TRY(cudaMemsetAsync(masks, 0, ((size_t)T * mask_words + words) * 4, stream));
-    si_union_bitmap_kernel<<<64, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, n_loaded, bitmap, nullptr);
-    si_union_kernel<<<1, 1024, smem, stream>>>(bitmap, n_loaded, union_out, n_union_out, pos, n_loaded);
-    si_union_masks_kernel<<<64, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, 0, n_loaded, n_union_out, pos, masks,
-                                                  mask_words, 0);
+    UnionScratch u = union_scratch(s, (char *)workspace, ws, T, n_loaded, 0);
+    SI_CUDA_TRY(cudaMemsetAsync(u.bitmap, 0, ((size_t)u.mask_words + 64) * 4, stream));
+    const long long entries = idx_offsets ? (long long)T * n_loaded : (long long)T * k_fixed;
+    si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+        idx, idx_offsets, k_fixed, T, n_loaded, u.bitmap, nullptr, u.mask_words, u.ticket, union_out, n_union_out,
+        n_loaded, nullptr);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }
@@ -597,32 +708,32 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     const size_t nl_pad = si_align_up((size_t)n_loaded, 128);
     int32_t *uni = (int32_t *)(wsb + ws.union_off);
     int32_t *n_union = uni + nl_pad;                       // one int32 (64 reserved)
-    int32_t *pos = uni + nl_pad + 64;
-    uint32_t *masks = (uint32_t *)(wsb + ws.mask_off);
-    const int mask_words = (int)(nl_pad / 32);
     // host-known upper bound of the union size sizes the grids
     long long cap = shared ? (long long)k_fixed : (idx_offsets ? (long long)n_loaded : (long long)T * k_fixed);
     if (cap > n_loaded) cap = n_loaded;
     const int nu_pad = (int)si_align_up((size_t)cap, 128);
-    {
-        const int words = (n_loaded + 31) / 32;
-        size_t smem = (size_t)(2 * words + 2) * 4;
-        uint32_t *bitmap = masks + (size_t)T * mask_words;
-        SI_CUDA_TRY(cudaMemsetAsync(masks, 0, ((size_t)T * mask_words + words) * 4, stream));
-        si_union_bitmap_kernel<<<s->num_sms, 256, 0, stream>>>(idx, idx_offsets, k_fixed, shared ? 1 : T, n_loaded, bitmap,
-                                                               status_dev);
-        si_union_kernel<<<1, 1024, smem, stream>>>(bitmap, n_loaded, uni, n_union, pos, nu_pad);
-        si_union_masks_kernel<<<2 * s->num_sms, 256, 0, stream>>>(idx, idx_offsets, k_fixed, T, shared ? 1 : 0, n_loaded,
-                                                                   n_union, pos, masks, mask_words,
-                                                                   (flags & SI_FLAG_UNION_UNMASKED) != 0);
-    }
-    // ---- tiling
     const int t_pad_total = (int)si_align_up((size_t)T, 16);
     const int tok_tiles = (t_pad_total + 255) / 256;
+    const int m_tiles = nu_pad / 128;
+    const bool own_lists = !shared && !(flags & SI_FLAG_UNION_UNMASKED);   // membership differs per token
+    const int n_ctr_gu = m_tiles * tok_tiles, n_ctr_dn = (d / 128) * tok_tiles;
+    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn);
+    if (us.zero_bytes > ws.mask_bytes) return SI_ERR_NOMEM;
+    {
+        const int words = (n_loaded + 31) / 32;
+        // token bitmaps are only read (and so only cleared) when the tokens have lists of their own
+        char *z0 = own_lists ? (char *)us.tokbits : (char *)us.bitmap;
+        SI_CUDA_TRY(cudaMemsetAsync(z0, 0, us.zero_bytes - (size_t)(z0 - (char *)us.tokbits), stream));
+        const int n_lists = shared ? 1 : T;
+        const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
+        si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+            idx, idx_offsets, k_fixed, n_lists, n_loaded, us.bitmap, own_lists ? us.tokbits : nullptr, us.mask_words,
+            us.ticket, uni, n_union, nu_pad, status_dev);
+    }
+    // ---- tiling
     const int n_tok = tok_tiles > 1 ? 256 : t_pad_total;
     // with several token tiles every tile must be full width: pad the token dimension
     const int t_pad_alloc = tok_tiles * n_tok;
-    const int m_tiles = nu_pad / 128;
     GemmParams P;
     P.rec_base = (const char *)s->records(layer); P.rec_bytes = (int)s->record_bytes(); P.d_model = d; P.chunks = d / 8;
     P.union_slots = uni; P.n_union = n_union; P.nu_pad = nu_pad;
@@ -631,6 +742,9 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.partial = (float *)(wsb + ws.partial_off);
     P.fmt = s->dtype == SI_BF16 ? 1 : 0;
     P.status = status_dev;
+    P.tokbits = own_lists ? us.tokbits : nullptr; P.mask_words = us.mask_words;
+    P.h_out = (uint16_t *)(wsb + ws.h_off);
+    P.y = y; P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
     // gate/up: split K = d_model so that about one wave of CTAs is launched
     // the grid is sized for the largest possible union; with few tokens the real union is much
     // smaller and the surplus CTAs exit at once, so aim at about two CTAs per SM there
@@ -649,14 +763,8 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(m_tiles, s1, tok_tiles);
+        P.tile_ctr = us.ctr;
         si_gemm_gateup_kernel<<<grid, kGemmThreads, smem, stream>>>(P);
-    }
-    {
-        dim3 grid((t_pad_alloc + 31) / 32, (nu_pad + 7) / 8);
-        if (s->dtype == SI_BF16)
-            si_gemm_combine_kernel<SI_BF16><<<grid, 256, 0, stream>>>(P.partial, s1, nu_pad, t_pad_alloc, T, n_union, masks, mask_words, (uint16_t *)(wsb + ws.h_off));
-        else
-            si_gemm_combine_kernel<SI_F16><<<grid, 256, 0, stream>>>(P.partial, s1, nu_pad, t_pad_alloc, T, n_union, masks, mask_words, (uint16_t *)(wsb + ws.h_off));
     }
     // down: split K = union
     int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
@@ -671,14 +779,8 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(d / 128, s2, tok_tiles);
+        P.tile_ctr = us.ctr + n_ctr_gu;
         si_gemm_down_kernel<<<grid, kGemmThreads, smem, stream>>>(P);
-    }
-    {
-        dim3 grid((d + 255) / 256, T);
-        if (s->dtype == SI_BF16)
-            si_gemm_reduce_kernel<SI_BF16><<<grid, 256, 0, stream>>>(P.partial, s2, t_pad_alloc, d, T, (const uint16_t *)x, y, y_dtype == SI_F32, (flags & SI_FLAG_RESIDUAL) != 0);
-        else
-            si_gemm_reduce_kernel<SI_F16><<<grid, 256, 0, stream>>>(P.partial, s2, t_pad_alloc, d, T, (const uint16_t *)x, y, y_dtype == SI_F32, (flags & SI_FLAG_RESIDUAL) != 0);
     }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
