@@ -237,7 +237,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     const int k_per = (P.d_model / kChunkK + P.n_split - 1) / P.n_split;   // chunks per split
     const int c0 = ks * k_per, c1 = min(P.d_model / kChunkK, c0 + k_per);
     const int n_chunks = c1 > c0 ? c1 - c0 : 0;
-    const int tok0 = tt * 256;
+    const int tok0 = tt * N;
 
     uint32_t ncols = 32; while (ncols < (uint32_t)(2 * N)) ncols <<= 1;
     if (tid == 0) {
@@ -317,7 +317,27 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
         float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
         float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-        if (ok && n_chunks > 0) {
+        if (ok && P.n_split == 1) {
+            // whole K in this CTA: form H straight from the accumulators (no partial tiles); the tile is
+            // staged in shared memory -- every MMA has finished reading the stages -- and written out below
+            constexpr int kRowPitch = 128 + 8;
+            uint16_t *hs = reinterpret_cast<uint16_t *>(smem);
+            const int i = mt * 128 + r;
+            const int slot = P.union_slots[i];
+            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
+                uint32_t g[16], u[16];
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, g);
+                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(N + n0), u);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const int t = tok0 + n0 + q;
+                    bool keep = n_chunks > 0 && t < P.T && i < n_u;
+                    if (keep && P.tokbits) keep = (P.tokbits[(size_t)t * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u;
+                    const float out = keep ? si_silu_mul(__uint_as_float(g[q]), __uint_as_float(u[q])) : 0.f;
+                    hs[(n0 + q) * kRowPitch + r] = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
+                }
+            }
+        } else if (ok && n_chunks > 0) {
             for (int n0 = 16 * cb; n0 < N; n0 += 32) {
                 uint32_t v[16];
                 tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
@@ -366,10 +386,14 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     // ---- combine: the CTA that delivers the tile's last K split forms H for the tile.  The splits are
     // summed in split order whoever is last, so H does not depend on the arrival order.
     int *last_flag = const_cast<int *>(failed) + 1;
-    if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
-    __syncthreads();
-    if (!*last_flag || *failed) return;
-    __threadfence();
+    if (P.n_split > 1) {
+        if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
+        __syncthreads();
+        if (!*last_flag || *failed) return;
+        __threadfence();
+    } else if (*failed) {
+        return;
+    }
     {
         // H[t][i] = member(t, U[i]) ? SiLU(sum_s G) * (sum_s U) : 0, rounded to the store dtype.  Reads
         // run along tokens (the partial tiles are [position][token]), H is [token][position]: transpose
@@ -380,7 +404,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         // one item = (union row, four consecutive tokens); all of an item's loads are issued before any
         // is used, four splits at a time
         const int nq = N / 4;
-        for (int it = tid; it < 128 * nq; it += kGemmThreads) {
+        for (int it = tid; it < (P.n_split > 1 ? 128 * nq : 0); it += kGemmThreads) {
             const int r = it / nq, n = (it - r * nq) * 4;
             const int i = mt * 128 + r;
             const float *prow = P.partial + (size_t)i * P.t_pad_total + tok0 + n;
@@ -451,7 +475,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
     const int c0 = ks * k_per, c1 = min(total_chunks, c0 + k_per);
     const int n_chunks = c1 > c0 ? c1 - c0 : 0;
-    const int tok0 = tt * 256;
+    const int tok0 = tt * N;
 
     uint32_t ncols = 32; while (ncols < (uint32_t)N) ncols <<= 1;
     if (tid == 0) {
@@ -531,7 +555,25 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
         // take alternate 16-token blocks
         const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
         float *py = P.partial + ((size_t)ks * P.t_pad_total + tok0) * P.d_model + (size_t)mt * 128 + r;
-        if (ok && n_chunks > 0) {
+        if (ok && P.n_split == 1) {
+            // whole K in this CTA: write y straight from the accumulators (a warp writes 32 consecutive
+            // columns of one token at a time)
+            const int col = mt * 128 + r;
+            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
+                uint32_t v[16];
+                if (n_chunks > 0) tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const int t = tok0 + n0 + q;
+                    if (t >= P.T) continue;
+                    const size_t o = (size_t)t * P.d_model + col;
+                    float a = n_chunks > 0 ? __uint_as_float(v[q]) : 0.f;
+                    if (P.residual) a += P.fmt ? si_cvt<SI_BF16>::lo((uint32_t)P.x[o]) : si_cvt<SI_F16>::lo((uint32_t)P.x[o]);
+                    if (P.y_f32) reinterpret_cast<float *>(P.y)[o] = a;
+                    else reinterpret_cast<uint16_t *>(P.y)[o] = P.fmt ? si_cvt<SI_BF16>::from_float(a) : si_cvt<SI_F16>::from_float(a);
+                }
+            }
+        } else if (ok && n_chunks > 0) {
             for (int n0 = 16 * cb; n0 < N; n0 += 32) {
                 uint32_t v[16];
                 tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
@@ -571,6 +613,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     }
     // ---- reduce: the CTA that delivers the column tile's last K split writes y for the tile:
     // y[t][j] = (x[t][j] +) sum over the splits in split order (independent of the arrival order)
+    if (P.n_split == 1) return;
     int *last_flag = const_cast<int *>(failed) + 1;
     if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
     __syncthreads();
@@ -662,7 +705,7 @@ size_t si_gemm_partial_bytes(const si_store *s, int T_max) {
 
 // Counters a call may need beyond the bitmaps: one per (tile, token tile) of either contraction.
 size_t si_gemm_counter_bytes(const si_store *s, size_t nl_pad, size_t t_pad) {
-    const size_t tok_tiles = (t_pad + 255) / 256;
+    const size_t tok_tiles = (t_pad + 127) / 128;
     return (64 + (nl_pad / 128 + (size_t)s->d_model / 128 + 2) * tok_tiles) * 4;
 }
 
@@ -713,8 +756,12 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     if (cap > n_loaded) cap = n_loaded;
     const int nu_pad = (int)si_align_up((size_t)cap, 128);
     const int t_pad_total = (int)si_align_up((size_t)T, 16);
-    const int tok_tiles = (t_pad_total + 255) / 256;
     const int m_tiles = nu_pad / 128;
+    // token tile width: 256 reads the weights least often, but with few weight tiles 128-wide token
+    // tiles put twice as many CTAs to work (and often make K splits unnecessary)
+    int tile_n = 256;
+    if (t_pad_total > 128 && m_tiles * ((t_pad_total + 255) / 256) * 10 < s->num_sms * 6) tile_n = 128;
+    const int tok_tiles = (t_pad_total + tile_n - 1) / tile_n;
     const bool own_lists = !shared && !(flags & SI_FLAG_UNION_UNMASKED);   // membership differs per token
     const int n_ctr_gu = m_tiles * tok_tiles, n_ctr_dn = (d / 128) * tok_tiles;
     UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn);
@@ -731,7 +778,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
             us.ticket, uni, n_union, nu_pad, status_dev);
     }
     // ---- tiling
-    const int n_tok = tok_tiles > 1 ? 256 : t_pad_total;
+    const int n_tok = tok_tiles > 1 ? tile_n : t_pad_total;
     // with several token tiles every tile must be full width: pad the token dimension
     const int t_pad_alloc = tok_tiles * n_tok;
     GemmParams P;
