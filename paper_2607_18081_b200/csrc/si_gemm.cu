@@ -72,6 +72,12 @@ __device__ __forceinline__ void cp_async_wait_dyn(int n) {
         default: cp_async_wait<5>(); break;
     }
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
+// while its predecessor in the stream still runs; pdl_wait() returns once the predecessor has
+// finished and its writes are visible, pdl_launch() lets the successor start being scheduled.  Both
+// are no-ops in launches without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -121,6 +127,7 @@ si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     __shared__ uint32_t warp_tot[32];
     __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch();
     const long long total = offsets ? offsets[n_lists] : (long long)n_lists * k_fixed;
     for (long long e = (long long)blockIdx.x * blockDim.x + tid; e < total; e += (long long)gridDim.x * blockDim.x) {
         const int s = idx[e];
@@ -206,6 +213,7 @@ struct GemmParams {
     int nstage;
     int32_t *status;
     // fused finishing passes: the CTA that completes a tile's last K split sums the splits
+    int tok_tiles, target_ctas;    // gate/up: token tiles; CTAs that can be resident at once
     unsigned *tile_ctr;            // per (tile, token tile) arrival counters, zero on entry
     const uint32_t *tokbits;       // [T][mask_words] slot bitmaps of the tokens' own lists, or nullptr: all tokens
     int mask_words;                //   use the whole union
@@ -214,7 +222,7 @@ struct GemmParams {
     int y_f32, residual;
 };
 
-// Gate/up contraction.  grid = (union tiles of 128, K splits of d_model, token tiles).
+// Gate/up contraction.  One CTA per (union tile of 128, K split of d_model, token tile), flat grid.
 // D_gate[128 neurons x N tokens] (+)= Wg[U tile, k] . X[tokens, k]^T, same for up, accumulated in
 // tensor memory (columns [0,N) gate, [N,2N) up).
 __global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
@@ -231,10 +239,18 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mt = blockIdx.x, ks = blockIdx.y, tt = blockIdx.z;
+    // Flat grid sized on the host for the largest possible union.  The real union is known here: its
+    // tiles are split along K just far enough to give every SM slot one unit (P.n_split is the most
+    // the partial buffer holds), and the surplus CTAs leave at once.
+    pdl_wait();                                 // the union kernel's results
+    pdl_launch();
     const int n_u = *P.n_union;
-    if (mt * 128 >= n_u && mt > 0) return;                          // nothing of the union in this tile
-    const int k_per = (P.d_model / kChunkK + P.n_split - 1) / P.n_split;   // chunks per split
+    const int n_real = n_u > 128 ? (n_u + 127) / 128 : 1;
+    int ns = P.target_ctas / (n_real * P.tok_tiles);
+    ns = ns < 1 ? 1 : (ns > P.n_split ? P.n_split : ns);
+    if ((int)blockIdx.x >= n_real * P.tok_tiles * ns) return;
+    const int ks = blockIdx.x % ns, mt = (blockIdx.x / ns) % n_real, tt = blockIdx.x / (ns * n_real);
+    const int k_per = (P.d_model / kChunkK + ns - 1) / ns;         // chunks per split
     const int c0 = ks * k_per, c1 = min(P.d_model / kChunkK, c0 + k_per);
     const int n_chunks = c1 > c0 ? c1 - c0 : 0;
     const int tok0 = tt * N;
@@ -317,7 +333,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
         float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
         float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-        if (ok && P.n_split == 1) {
+        if (ok && ns == 1) {
             // whole K in this CTA: form H straight from the accumulators (no partial tiles); the tile is
             // staged in shared memory -- every MMA has finished reading the stages -- and written out below
             constexpr int kRowPitch = 128 + 8;
@@ -386,8 +402,8 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     // ---- combine: the CTA that delivers the tile's last K split forms H for the tile.  The splits are
     // summed in split order whoever is last, so H does not depend on the arrival order.
     int *last_flag = const_cast<int *>(failed) + 1;
-    if (P.n_split > 1) {
-        if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
+    if (ns > 1) {
+        if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * P.tok_tiles + tt], 1u) == (unsigned)ns - 1;   // ... before it is counted
         __syncthreads();
         if (!*last_flag || *failed) return;
         __threadfence();
@@ -404,16 +420,16 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
         // one item = (union row, four consecutive tokens); all of an item's loads are issued before any
         // is used, four splits at a time
         const int nq = N / 4;
-        for (int it = tid; it < (P.n_split > 1 ? 128 * nq : 0); it += kGemmThreads) {
+        for (int it = tid; it < (ns > 1 ? 128 * nq : 0); it += kGemmThreads) {
             const int r = it / nq, n = (it - r * nq) * 4;
             const int i = mt * 128 + r;
             const float *prow = P.partial + (size_t)i * P.t_pad_total + tok0 + n;
             float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-            for (int sp0 = 0; sp0 < P.n_split; sp0 += 4) {
+            for (int sp0 = 0; sp0 < ns; sp0 += 4) {
                 float4 gv[4], uv[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const bool in = sp0 + k < P.n_split;
+                    const bool in = sp0 + k < ns;
                     gv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k)) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
                     uv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k) + 1) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
@@ -470,6 +486,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.x, ks = blockIdx.y, tt = blockIdx.z;
+    pdl_wait();                                 // H of the gate/up kernel
     const int n_u = *P.n_union;
     const int total_chunks = (n_u + kChunkK - 1) / kChunkK;        // 64 union entries per chunk
     const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
@@ -669,6 +686,18 @@ __global__ void si_gemm_reduce_kernel(const float *__restrict__ partial, int n_s
     else reinterpret_cast<uint16_t *>(y)[(size_t)t * d + j] = si_cvt<DT>::from_float(a);
 }
 
+// Launch a contraction kernel so that it may be scheduled while the previous kernel of the stream is
+// still finishing (the kernel itself waits for that kernel's results with pdl_wait()).
+cudaError_t launch_after_predecessor(void (*kern)(GemmParams), dim3 grid, size_t smem, cudaStream_t stream, const GemmParams &P) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, P);
+}
+
 int pick_stages_gemm(size_t stage_bytes, int n_tok) {
     // few tokens: the kernels are latency-bound gathers, two CTAs per SM hide more of it
     size_t budget = n_tok <= 64 ? 112 * 1024 : 200 * 1024;
@@ -691,9 +720,11 @@ UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws,
     return u;
 }
 int union_blocks(const si_store *s, long long entries) {
-    long long b = (entries + 4095) / 4096;           // four entries per thread at least
+    // one entry per thread while the blocks fit the machine at once: an entry is a chain of dependent
+    // global accesses (index, bitmap word, atomic), so the chains should all run side by side
+    long long b = (entries + 1023) / 1024;
     if (b < 1) b = 1;
-    return (int)(b > s->num_sms ? s->num_sms : b);
+    return (int)(b > 2 * s->num_sms ? 2 * s->num_sms : b);
 }
 
 }  // namespace
@@ -792,16 +823,15 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.tokbits = own_lists ? us.tokbits : nullptr; P.mask_words = us.mask_words;
     P.h_out = (uint16_t *)(wsb + ws.h_off);
     P.y = y; P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
-    // gate/up: split K = d_model so that about one wave of CTAs is launched
-    // the grid is sized for the largest possible union; with few tokens the real union is much
-    // smaller and the surplus CTAs exit at once, so aim at about two CTAs per SM there
-    int s1 = (t_pad_alloc <= 64 ? 2 * s->num_sms + m_tiles * tok_tiles - 1 : s->num_sms) / (m_tiles * tok_tiles);
+    // gate/up: K = d_model may be split up to s1 ways (what the partial buffer holds); the kernel
+    // picks the split from the real union size so that one wave of CTAs covers the SM slots (two CTAs
+    // per SM with few tokens: the gathers are latency-bound)
+    const int target = (t_pad_alloc <= 64 ? 2 : 1) * s->num_sms;
     const int k_chunks = d / kChunkK;
-    if (s1 < 1) s1 = 1;
-    if (s1 > 8) s1 = 8;
-    if (s1 > k_chunks) s1 = k_chunks;
-    while (s1 > 1 && (size_t)s1 * 2 * nu_pad * t_pad_alloc * 4 > kPartialCap) --s1;
-    if ((size_t)s1 * 2 * nu_pad * t_pad_alloc * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
+    int s1 = k_chunks < 8 ? k_chunks : 8;
+    const size_t part_cap = kPartialCap < ws.partial_bytes ? kPartialCap : ws.partial_bytes;
+    while (s1 > 1 && (size_t)s1 * 2 * nu_pad * t_pad_alloc * 4 > part_cap) --s1;
+    if ((size_t)2 * nu_pad * t_pad_alloc * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
     if ((size_t)t_pad_alloc * nu_pad * 2 > ws.h_bytes) return SI_ERR_NOMEM;
     {
         const size_t stage = 2 * 128 * 128 + (size_t)n_tok * 128;
@@ -809,9 +839,11 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         if (P.nstage < 2) return SI_ERR_UNSUPPORTED;
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        dim3 grid(m_tiles, s1, tok_tiles);
+        const int units = m_tiles * tok_tiles;
+        dim3 grid(units > target ? units : target);
+        P.tok_tiles = tok_tiles; P.target_ctas = target;
         P.tile_ctr = us.ctr;
-        si_gemm_gateup_kernel<<<grid, kGemmThreads, smem, stream>>>(P);
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P));
     }
     // down: split K = union
     int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
@@ -827,7 +859,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(d / 128, s2, tok_tiles);
         P.tile_ctr = us.ctr + n_ctr_gu;
-        si_gemm_down_kernel<<<grid, kGemmThreads, smem, stream>>>(P);
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_down_kernel, grid, smem, stream, P));
     }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
