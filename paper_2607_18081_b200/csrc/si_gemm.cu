@@ -239,22 +239,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // Flat grid sized on the host for the largest possible union.  The real union is known here: its
-    // tiles are split along K just far enough to give every SM slot one unit (P.n_split is the most
-    // the partial buffer holds), and the surplus CTAs leave at once.
-    pdl_wait();                                 // the union kernel's results
-    pdl_launch();
-    const int n_u = *P.n_union;
-    const int n_real = n_u > 128 ? (n_u + 127) / 128 : 1;
-    int ns = P.target_ctas / (n_real * P.tok_tiles);
-    ns = ns < 1 ? 1 : (ns > P.n_split ? P.n_split : ns);
-    if ((int)blockIdx.x >= n_real * P.tok_tiles * ns) return;
-    const int ks = blockIdx.x % ns, mt = (blockIdx.x / ns) % n_real, tt = blockIdx.x / (ns * n_real);
-    const int k_per = (P.d_model / kChunkK + ns - 1) / ns;         // chunks per split
-    const int c0 = ks * k_per, c1 = min(P.d_model / kChunkK, c0 + k_per);
-    const int n_chunks = c1 > c0 ? c1 - c0 : 0;
-    const int tok0 = tt * N;
-
+    // ---- set-up that needs nothing from the union kernel (runs while that kernel finishes)
     uint32_t ncols = 32; while (ncols < (uint32_t)(2 * N)) ncols <<= 1;
     if (tid == 0) {
         for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads); mbar_init(&empty[s], 1); }
@@ -270,6 +255,26 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+
+    // Flat grid sized on the host for the largest possible union.  The real union is known here: its
+    // tiles are split along K just far enough to give every SM slot one unit (P.n_split is the most
+    // the partial buffer holds), and the surplus CTAs leave at once.
+    pdl_wait();                                 // the union kernel's results
+    pdl_launch();
+    const int n_u = *P.n_union;
+    const int n_real = n_u > 128 ? (n_u + 127) / 128 : 1;
+    int ns = P.target_ctas / (n_real * P.tok_tiles);
+    ns = ns < 1 ? 1 : (ns > P.n_split ? P.n_split : ns);
+    if ((int)blockIdx.x >= n_real * P.tok_tiles * ns) {
+        if (warp == kLoaderWarps)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
+        return;
+    }
+    const int ks = blockIdx.x % ns, mt = (blockIdx.x / ns) % n_real, tt = blockIdx.x / (ns * n_real);
+    const int k_per = (P.d_model / kChunkK + ns - 1) / ns;         // chunks per split
+    const int c0 = ks * k_per, c1 = min(P.d_model / kChunkK, c0 + k_per);
+    const int n_chunks = c1 > c0 ? c1 - c0 : 0;
+    const int tok0 = tt * N;
 
     if (warp < kLoaderWarps) {
         // ---------------------------------------------------------------- gather loads
@@ -486,14 +491,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.x, ks = blockIdx.y, tt = blockIdx.z;
-    pdl_wait();                                 // H of the gate/up kernel
-    const int n_u = *P.n_union;
-    const int total_chunks = (n_u + kChunkK - 1) / kChunkK;        // 64 union entries per chunk
-    const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
-    const int c0 = ks * k_per, c1 = min(total_chunks, c0 + k_per);
-    const int n_chunks = c1 > c0 ? c1 - c0 : 0;
-    const int tok0 = tt * N;
-
+    // ---- set-up that needs nothing from the gate/up kernel (runs while that kernel finishes)
     uint32_t ncols = 32; while (ncols < (uint32_t)N) ncols <<= 1;
     if (tid == 0) {
         for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads); mbar_init(&empty[s], 1); }
@@ -509,6 +507,14 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+
+    pdl_wait();                                 // H of the gate/up kernel
+    const int n_u = *P.n_union;
+    const int total_chunks = (n_u + kChunkK - 1) / kChunkK;        // 64 union entries per chunk
+    const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
+    const int c0 = ks * k_per, c1 = min(total_chunks, c0 + k_per);
+    const int n_chunks = c1 > c0 ? c1 - c0 : 0;
+    const int tok0 = tt * N;
 
     if (warp < kLoaderWarps) {
         // Copy j of a thread covers 16-byte piece (tid & 15) of the 256-byte down-row segment of union
