@@ -11,7 +11,8 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     int nl_max = 0;
     for (int l = 0; l < s->n_layers; ++l) nl_max = nl_max > s->n_loaded[l] ? nl_max : s->n_loaded[l];
     const size_t nl_pad = si_align_up((size_t)nl_max, 128);
-    const size_t t_pad = T_max <= 256 ? si_align_up((size_t)T_max, 16) : si_align_up((size_t)T_max, 256);
+    // tokens are padded to 16; beyond 128 they run in token tiles of 128 or 256, padded to whole tiles
+    const size_t t_pad = T_max <= 128 ? si_align_up((size_t)T_max, 16) : si_align_up((size_t)T_max, 256);
     size_t off = 0;
     auto take = [&](size_t &o, size_t &b, size_t bytes) { o = off; b = si_align_up(bytes, 256); off += b; };
     take(w.ctrl_off, w.ctrl_bytes, 256);

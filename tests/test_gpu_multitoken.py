@@ -123,3 +123,37 @@ def test_7b_prefill_shared_list(api, m7b):
         # the model was loaded from the c2 recipe; the oracle uses that model's weights
         ref = m7b.oracle_y(0, x[t], shared)
         assert_close(from_dev(y[t]), ref, f"prefill token {t}")
+
+
+def test_7b_many_tokens_own_lists_residual(api, m7b):
+    """300 tokens with lists of their own: two 256-wide token tiles, the union covers nearly the whole
+    loaded set, the down contraction is split along K and finished by the last-arriving CTA."""
+    cfg = m7b.cfg
+    T, k = 300, cfg.k_active
+    lists = wl.zipf_lists(cfg, 0, T)
+    x = wl.x_tokens(cfg, 0, T)
+    y = _run(api, m7b, 0, x, lists, None, k, T, flags=api.SI_FLAG_RESIDUAL, y_dtype=torch.bfloat16)
+    for t in (0, 128, 255, 256, 299):
+        ref = m7b.oracle_y(0, x[t], lists[t]) + wl.bits_to_float64(x[t], cfg.dtype)
+        assert_close(from_dev(y[t]), ref, f"300-token batch, token {t}")
+
+
+@pytest.mark.parametrize("T", [130, 200])
+def test_c1_many_tokens_narrow_token_tiles(api, c1, T):
+    """More than 128 tokens over a small layer: 128-wide token tiles, ragged lists, padded last tile."""
+    cfg = c1.cfg
+    n = cfg.n_loaded
+    g = np.random.default_rng(100 + T)
+    lens = g.integers(0, n // 2, size=T)
+    lens[3] = 0
+    lists = [np.sort(g.permutation(n)[:k]).astype(np.int32) for k in lens]
+    offsets = np.zeros(T + 1, np.int32); offsets[1:] = np.cumsum(lens)
+    x = wl.x_tokens(cfg, 0, T, first_token=7)
+    y = _run(api, c1, 0, x, np.concatenate(lists), offsets, n, T)
+    for t in (0, 3, 64, 127, 128, T - 1):
+        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], lists[t]), f"T={T} token {t}")
+    # one shared list for all tokens
+    shared = np.sort(g.permutation(n)[: n // 3]).astype(np.int32)
+    y = _run(api, c1, 0, x, shared, None, len(shared), T, flags=api.SI_FLAG_SHARED_LIST, y_dtype=torch.float16)
+    for t in (0, 127, 128, T - 1):
+        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], shared), f"shared list, T={T} token {t}")
