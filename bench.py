@@ -400,7 +400,7 @@ def run_multitoken(args, cfg, rank, world, local_rank):
                        "mean_union": u, "union_overlap": None if prefill else 1.0 - u / (T * k),
                        "union_coverage_of_loaded": u / cfg.n_loaded, "us_per_layer_call": us_per_layer,
                        "l2": "weights of one pass exceed L2"},
-            "gpu_launches": layer_calls * 6,
+            "gpu_launches": layer_calls * 3,
             "roofline": ({"bound": "tensor", "achieved": flops / us_per_layer / 1e6, "peak": peaks["bf16_tflops_sustained"],
                           "unit": "TFLOP/s", "frac": flops / us_per_layer / 1e6 / peaks["bf16_tflops_sustained"],
                           "peak_kind": f"of {peak_kind} (sustained)", "traffic": None} if prefill else
