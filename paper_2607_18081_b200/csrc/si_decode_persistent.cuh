@@ -68,7 +68,6 @@ struct Params {
     int32_t *status;
     long long *prof;              // optional phase profile: int64 [G][kProfSlots] cycle counters, or nullptr
     int stream_only;              // diagnostics bit mask (see si_debug_decode_stream_only)
-    int prefetch_rounds;          // L2 prefetch distance in ring rounds (0 = off)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -114,14 +113,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
         if (*cta_abort) return false;
         if (clock64() - t0 > kWaitCycles) return false;
     }
-}
-// Warp-level wait: only lane 0 polls the barrier (32 lanes polling one barrier word cost 32
-// shared-memory barrier operations per probe), the warp then reconverges; the shuffle orders the
-// other lanes' subsequent reads after lane 0's acquire.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *cta_abort, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait_bounded(bar, parity, cta_abort) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 // Strong (gpu-scope) vector store and vector add-reduction at L2; one thread issues both to the same
 // address in program order, so the add lands on the stored value.
@@ -201,24 +192,7 @@ __device__ __forceinline__ float dot8(const uint4 &v, const float (&x)[8]) {
     return a;
 }
 
-// Warp reduction of four values with six shuffles: afterwards lane 0 holds sum(v0), lane 8
-// sum(v1), lane 16 sum(v2), lane 24 sum(v3).  Fixed order, hence deterministic.
-__device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane) {
-    const bool hi16 = (lane & 16) != 0;
-    float s0 = hi16 ? v0 : v2, s1 = hi16 ? v1 : v3;
-    float k0 = hi16 ? v2 : v0, k1 = hi16 ? v3 : v1;
-    k0 += __shfl_xor_sync(0xFFFFFFFFu, s0, 16);
-    k1 += __shfl_xor_sync(0xFFFFFFFFu, s1, 16);
-    const bool hi8 = (lane & 8) != 0;
-    float s = hi8 ? k0 : k1, k = hi8 ? k1 : k0;
-    k += __shfl_xor_sync(0xFFFFFFFFu, s, 8);
-    k += __shfl_xor_sync(0xFFFFFFFFu, k, 4);
-    k += __shfl_xor_sync(0xFFFFFFFFu, k, 2);
-    k += __shfl_xor_sync(0xFFFFFFFFu, k, 1);
-    return k;
-}
-
-// Per-step list geometry, identical in producer and consumers.
+// Per-step list geometry: which entries of the step's list belong to virtual CTA b of G.
 struct StepGeom { int base, k, first, cnt; };
 __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, int b) {
     StepGeom g;
@@ -238,7 +212,6 @@ __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, 
 struct Smem {
     uint64_t full[kMaxStages];         // stage index = set * S + stage-in-set
     uint64_t empty[kMaxStages];
-    uint64_t setbar[kSets][2];         // a set's warps have published their dot-product partials
     // consumer set -> reducers hand-over of a step's accumulators (one buffer per set); one barrier
     // per reducer warp (slot s mod 3), so that each waiter follows the phases of its own barrier
     uint64_t accfull[kSets][kReducerWarps], accempty[kSets][kReducerWarps];
@@ -277,7 +250,6 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
-        for (int q = 0; q < kSets; ++q) { mbar_init(&sm->setbar[q][0], kSetWarps); mbar_init(&sm->setbar[q][1], kSetWarps); }
         for (int q = 0; q < kSets; ++q)
             for (int w = 0; w < kReducerWarps; ++w) { mbar_init(&sm->accfull[q][w], kSetWarps); mbar_init(&sm->accempty[q][w], 1); }
         sm->cta_abort = 0;
@@ -442,13 +414,12 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const bool noarith = (P.stream_only & 1) != 0;  // diagnostics: drain only
 
         for (int step = 0; step < P.n_steps && !fail; ++step) {
-            const bool real = true;
             float xr[NCH][8], acc[NCH][8];
 #pragma unroll
             for (int i = 0; i < NCH; ++i)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { acc[i][e] = 0.f; xr[i][e] = 0.f; }
-            if (real) {
+            {
                 int cnt;
                 {   // x item
                     const int st = n % S; const uint32_t ph = (n / S) & 1;
@@ -787,7 +758,6 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.status = status_dev;
     P.prof = si_decode_profile_buffer();
     P.stream_only = si_decode_stream_only() & 0xFF;
-    P.prefetch_rounds = 0;
     if ((si_decode_stream_only() >> 8) & 0xF) P.nstage = 2 * ((si_decode_stream_only() >> 8) & 0xF);   // diagnostics: shallower rings
     int G = s->num_sms;
     if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
