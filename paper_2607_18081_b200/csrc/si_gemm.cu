@@ -4,19 +4,21 @@
 //
 //   union      U = sorted union of the T lists, mask[t] = which entries of U token t selected
 //   gate/up    G^T, Up^T [|U| x T] = W_gate[U, :] . X^T, W_up[U, :] . X^T     (K = d_model)
-//   combine    H[t, i] = mask[t, i] ? SiLU(G[i, t]) * Up[i, t] : 0, rounded to the store dtype
+//   combine    H[t, i] = mask[t, i] ? SiLU(G[i, t]) * Up[i, t] : 0, rounded to the store dtype (fused)
 //   down       Y^T [d_model x T] = W_down[:, U] . H^T                          (K = |U|)
 //
 // Token t therefore uses exactly its own list (Section 5 applied per token), whatever the
 // other tokens selected; with SI_FLAG_UNION_UNMASKED every token uses the whole union.
 //
 // Tiling.  Both contractions put the weight side on the MMA M dimension (128 rows of the
-// store per CTA tile) and the tokens on N (T padded to 16, at most 256 per tile), so the
-// weights -- the dominant bytes -- are read exactly once.  Weight rows are gathered straight
-// out of the neuron records with 16-byte cp.async copies into the 128-byte-swizzled shared
-// memory layouts the MMA descriptors expect (gate/up rows are K-major, down rows MN-major).
-// K is split across CTAs so that small unions still fill the machine; the fp32 partial tiles
-// are summed in split order by the combine / reduce kernels, so results are deterministic.
+// store per CTA tile) and the tokens on N (T padded to 16; tiles of 128 or 256 tokens beyond
+// that), so with one token tile the weights -- the dominant bytes -- are read exactly once.
+// Weight rows are gathered straight out of the neuron records with 16-byte cp.async copies into
+// the 128-byte-swizzled shared memory layouts the MMA descriptors expect (gate/up rows are
+// K-major, down rows MN-major).  K is split across CTAs so that small unions still fill the
+// machine.  The finishing passes (combine, split reduction) have no kernels of their own: an
+// unsplit tile is finished in the contraction's epilogue, a split tile by the CTA that delivers
+// its last fp32 partial, which sums the partials in split order -- so results are deterministic.
 #include "si_common.cuh"
 
 namespace {
@@ -679,7 +681,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     }
 }
 
-// y[t][j] = (x[t][j] +) sum over K splits, in split order.
+// y[t][j] = (x[t][j] +) sum over K splits, in split order (here only for calls that select nothing).
 template <int DT>
 __global__ void si_gemm_reduce_kernel(const float *__restrict__ partial, int n_split, int t_pad_total, int d, int T,
                                       const uint16_t *__restrict__ x, void *__restrict__ y, int y_f32, int residual) {
