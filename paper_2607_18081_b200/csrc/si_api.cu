@@ -24,7 +24,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     take(w.mask_off, w.mask_bytes, T_max > 1 ? (t_pad + 1) * (nl_pad / 32) * 4 + si_gemm_counter_bytes(s, nl_pad, t_pad) : 0);   // token slot bitmaps, union bitmap, counters
     take(w.h_off, w.h_bytes, T_max > 1 ? t_pad * nl_pad * 2 : 0);
     take(w.selws_off, w.selws_bytes, (size_t)T_max * si_select_ws_bytes_impl(nl_max));
-    take(w.steps_off, w.steps_bytes, si_align_up((size_t)max_steps * 4, 256) + (size_t)max_steps * 256);   // layer ids + 2 counter lines per step
+    take(w.steps_off, w.steps_bytes, si_align_up((size_t)max_steps * 4, 256) + 256 + (size_t)max_steps * 256);   // layer ids, control words, 2 counter lines per step
     w.total = off;
     return w;
 }

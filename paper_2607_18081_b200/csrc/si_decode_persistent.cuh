@@ -45,6 +45,7 @@ constexpr int kCounterStride = 64;                // uint32 per step: written at
 constexpr int kMaxStages = 16;
 constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
 constexpr int kPartialDepth = 8;                  // D: partial-y buffers in flight
+constexpr int kFewSteps = 16;                     // launches this short carry their layer ids as kernel arguments
 constexpr int kProfSlots = 16;                    // int64 cycle counters per SM in the optional phase profile
 constexpr int kLag = 3;                           // a step's cross-SM reduction starts this many steps later
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
@@ -54,7 +55,9 @@ struct Params {
     unsigned long long rec_off[SI_MAX_LAYERS];
     int n_loaded[SI_MAX_LAYERS];
     int n_layers, n_steps, k_fixed, d_model, chunks, nstage;
-    const int32_t *step_layers;   // device int32 [n_steps] or nullptr (step mod n_layers)
+    const int32_t *step_layers;   // device int32 [n_steps] or nullptr (then: few_layers, else step mod n_layers)
+    int n_few;                    // > 0: the launch has n_few <= kFewSteps steps, their layers are in few_layers
+    unsigned char few_layers[16];
     const uint16_t *x;            // [n_steps, d_model]
     const int32_t *idx;           // [n_steps, k_fixed] or CSR payload
     const int32_t *idx_offsets;   // CSR [n_steps + 1] or nullptr
@@ -295,7 +298,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 }
                 pf_valid = in;
                 if (in) {
-                    const int layer = P.step_layers ? __ldg(P.step_layers + step) : step % P.n_layers;
+                    const int layer = P.step_layers ? __ldg(P.step_layers + step) : (P.n_few ? (int)P.few_layers[step] : step % P.n_layers);
                     if (t == 0) {
                         pf_src = (unsigned long long)(P.x + (size_t)step * d);
                         pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
@@ -728,7 +731,13 @@ template <int DT, int NCH>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
     auto kern = si_persist::si_decode_persistent_kernel<DT, NCH>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
-    SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
+    int dev = 0;
+    SI_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 8 || smem_set[dev] < smem) {
+        SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        if (dev >= 0 && dev < 8) smem_set[dev] = smem;
+    }
     void *args[] = {(void *)&P};
     SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G), dim3(si_persist::kThreads), args, smem, stream));
     return SI_OK;
@@ -743,18 +752,21 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     for (int l = 0; l < s->n_layers; ++l) { P.rec_off[l] = s->rec_off[l]; P.n_loaded[l] = s->n_loaded[l]; }
     P.n_layers = s->n_layers; P.n_steps = n_steps; P.k_fixed = k_fixed; P.d_model = s->d_model;
     P.chunks = s->d_model / 8; P.nstage = si_persist::pick_stages(s->d_model);
-    P.step_layers = nullptr;
-    // steps region: [n_steps] layer ids | [n_steps][64] counters
+    P.step_layers = nullptr; P.n_few = 0;
+    // steps region: [n_steps] layer ids | control words (256 bytes) | [n_steps][64] counters
     int32_t *steps = (int32_t *)(wsb + ws.steps_off);
-    if (layers_host) {
+    if (layers_host && n_steps <= si_persist::kFewSteps) {
+        P.n_few = n_steps;                      // short launch: no copy, the ids travel with the arguments
+        for (int i = 0; i < n_steps; ++i) P.few_layers[i] = (unsigned char)layers_host[i];
+    } else if (layers_host) {
         SI_CUDA_TRY(cudaMemcpyAsync(steps, layers_host, (size_t)n_steps * 4, cudaMemcpyHostToDevice, stream));
         P.step_layers = steps;
     }
-    P.counters = (unsigned int *)(wsb + ws.steps_off + si_align_up((size_t)n_steps * 4, 256));
+    P.ctrl = (unsigned int *)(wsb + ws.steps_off + si_align_up((size_t)n_steps * 4, 256));
+    P.counters = P.ctrl + 64;
     P.x = (const uint16_t *)x; P.idx = idx; P.idx_offsets = idx_offsets; P.y = y;
     P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
     P.partial = (float *)(wsb + ws.partial_off);
-    P.ctrl = (unsigned int *)(wsb + ws.ctrl_off);
     P.status = status_dev;
     P.prof = si_decode_profile_buffer();
     P.stream_only = si_decode_stream_only() & 0xFF;
@@ -764,8 +776,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // every CTA reduces at most kMaxGroups float4 column groups
     const int g_min = (s->d_model / 4 + si_persist::kMaxGroups - 1) / si_persist::kMaxGroups;
     if (G < g_min) G = g_min;
-    SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256, stream));
-    SI_CUDA_TRY(cudaMemsetAsync(P.counters, 0, (size_t)n_steps * si_persist::kCounterStride * 4, stream));
+    SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
     const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
 #define SI_PL(DT) (nch <= 1 ? si_decode_persistent_launch_t<DT, 1>(P, G, stream) \

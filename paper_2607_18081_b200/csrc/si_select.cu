@@ -75,21 +75,45 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
                 if (tid < 256) hist[tid] = 0;
                 __syncthreads();
                 const uint32_t prefix = sh_prefix, mask = sh_mask;
-                for (int i = tid; i < n; i += kSelThreads) {
-                    uint32_t key = keys[i];
-                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+                const int need = sh_need;
+                // histogram of the current digit over the keys that still match the prefix.  Scores from
+                // one distribution crowd into a few bins of the high digits, so lanes with the same digit
+                // are merged first and one of them adds their count
+                for (int i0 = 0; i0 < n; i0 += kSelThreads) {
+                    const int i = i0 + tid;
+                    uint32_t digit = 0xFFFFFFFFu;                    // no key / key no longer in play
+                    if (i < n) {
+                        const uint32_t key = keys[i];
+                        if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+                    }
+                    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+                    if (digit != 0xFFFFFFFFu && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&hist[digit], (unsigned)__popc(peers));
                 }
                 __syncthreads();
-                if (tid == 0) {
-                    int need = sh_need, bin = 255;
-                    for (; bin > 0; --bin) {              // walk from the largest digit down
-                        int c = (int)hist[bin];
-                        if (c >= need) break;
-                        need -= c;
+                // find the digit where the count from the largest digit down reaches `need`: thread t
+                // owns bin 255 - t, so a prefix sum over threads is a suffix sum over bins
+                unsigned c = 0, inc = 0;
+                if (tid < 256) {
+                    c = hist[255 - tid];
+                    inc = c;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                        if ((tid & 31) >= o) inc += t;
                     }
-                    sh_need = need;
-                    sh_prefix = prefix | ((uint32_t)bin << shift);
-                    sh_mask = mask | (255u << shift);
+                    if ((tid & 31) == 31) warp_tot[tid >> 5] = inc;
+                }
+                __syncthreads();
+                if (tid < 256) {
+                    unsigned base = 0;
+                    for (int w = 0; w < (tid >> 5); ++w) base += (unsigned)warp_tot[w];
+                    const unsigned incl = base + inc, excl = incl - c;      // keys in bins >= / > this one
+                    // the keys in play are at least `need`, so exactly one bin satisfies this (bin 0 at the latest)
+                    if (excl < (unsigned)need && (unsigned)need <= incl) {
+                        sh_need = need - (int)excl;
+                        sh_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+                        sh_mask = mask | (255u << shift);
+                    }
                 }
                 __syncthreads();
             }
