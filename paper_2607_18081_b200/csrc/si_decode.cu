@@ -34,6 +34,7 @@ extern "C" int si_debug_decode_profile(void *dev_buf) {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kSimpleCtasPerSm = 2;
 
 template <int DT>
 __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
@@ -140,30 +141,56 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
     }
 }
 
-// y[j] = (x[j] +) sum over CTAs g = 0..G-1 of partial[g][j], in that order.
+// y[j] = (x[j] +) sum over CTAs g = 0..G-1 of partial[g][j].  One block per 32 output columns (eight
+// float4 groups); thread (group = tid & 7, row class = tid >> 3) sums rows class, class + 32, ... in
+// ascending order -- all its loads are independent -- and the 32 classes are then added in class
+// order, so the result does not depend on scheduling.
 template <int DT>
-__global__ void si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
-                                        const uint16_t *__restrict__ x, void *__restrict__ y,
-                                        int y_f32, int residual) {
-    int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= d) return;
-    float a = 0.f;
-    for (int g = 0; g < G; ++g) a += partial[(size_t)g * d + j];
-    if (residual) {
-        uint32_t w = x[j];
-        a += (DT == SI_BF16) ? si_cvt<SI_BF16>::lo(w) : si_cvt<SI_F16>::lo(w);
+__global__ void __launch_bounds__(256)
+si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
+                        const uint16_t *__restrict__ x, void *__restrict__ y,
+                        int y_f32, int residual) {
+    __shared__ float4 part[32][8];
+    const int g = threadIdx.x & 7, rc = threadIdx.x >> 3;
+    const int col = (blockIdx.x * 8 + g) * 4;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (col < d) {
+        for (int r0 = rc; r0 < G; r0 += 32 * 8) {
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = r0 + 32 * j;
+                v[j] = r < G ? __ldg(reinterpret_cast<const float4 *>(partial + (size_t)r * d + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w; }
+        }
     }
-    if (y_f32) reinterpret_cast<float *>(y)[j] = a;
-    else reinterpret_cast<uint16_t *>(y)[j] = si_cvt<DT>::from_float(a);
+    part[rc][g] = a;
+    __syncthreads();
+    if (rc != 0 || col >= d) return;
+    for (int c = 1; c < 32; ++c) { const float4 v = part[c][g]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+    if (residual) {
+        const uint2 xw = *reinterpret_cast<const uint2 *>(x + col);
+        a.x += si_cvt<DT>::lo(xw.x); a.y += si_cvt<DT>::hi(xw.x); a.z += si_cvt<DT>::lo(xw.y); a.w += si_cvt<DT>::hi(xw.y);
+    }
+    if (y_f32) {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(y) + col) = a;
+    } else {
+        uint2 w;
+        w.x = (uint32_t)si_cvt<DT>::from_float(a.x) | ((uint32_t)si_cvt<DT>::from_float(a.y) << 16);
+        w.y = (uint32_t)si_cvt<DT>::from_float(a.z) | ((uint32_t)si_cvt<DT>::from_float(a.w) << 16);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(y) + col) = w;
+    }
 }
 
 template <int DT>
 int launch_simple_step(const si_store *s, int layer, const void *x, const int32_t *idx,
                        const int32_t *offsets, int list, int k, void *y, int y_dtype, unsigned flags,
-                       float *partial, int32_t *status_dev, cudaStream_t stream) {
+                       float *partial, int max_ctas, int32_t *status_dev, cudaStream_t stream) {
     const int d = s->d_model, chunks = d / 8;
     const int nch = (chunks + kThreads - 1) / kThreads;
-    int G = k < 2 * s->num_sms ? (k < 1 ? 1 : k) : 2 * s->num_sms;
+    int G = k < max_ctas ? (k < 1 ? 1 : k) : max_ctas;          // one partial row per CTA
     const uint4 *rec = (const uint4 *)s->records(layer);
     const int nl = s->n_loaded[layer];
 #define SI_LAUNCH_PARTIAL(N)                                                                        \
@@ -175,7 +202,7 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
-    si_decode_reduce_kernel<DT><<<(d + 255) / 256, 256, 0, stream>>>(
+    si_decode_reduce_kernel<DT><<<(d + 31) / 32, 256, 0, stream>>>(
         partial, G, d, (const uint16_t *)x, y, y_dtype == SI_F32, (flags & SI_FLAG_RESIDUAL) != 0);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
@@ -196,7 +223,8 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
         if (!s->loaded[l]) return SI_ERR_INVALID_ARG;
     }
     char *wsb = (char *)workspace;
-    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s);
+    // a single step is served faster by two plain launches than by starting the persistent kernel
+    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps == 1;
     if (!use_simple)
         return si_decode_persistent_launch(s, n_steps, layers_host, x, idx, idx_offsets, k_fixed, y, y_dtype, flags,
                                            wsb, ws, status_dev, stream);
@@ -204,13 +232,17 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
     // is read on the device; k_fixed (an upper bound) only sizes the grid.
     const size_t esz = 2, ysz = (y_dtype == SI_F32) ? 4 : 2;
     float *partial = (float *)(wsb + ws.partial_off);
+    // CTAs of the partial kernel (one fp32 row of the partial buffer each): as many as can be resident
+    int max_ctas = kSimpleCtasPerSm * s->num_sms;
+    const size_t rows = ws.partial_bytes / ((size_t)s->d_model * 4);
+    if ((size_t)max_ctas > rows) max_ctas = (int)rows;
     for (int st = 0; st < n_steps; ++st) {
         int l = layers_host ? layers_host[st] : st % s->n_layers;
         const void *xs = (const char *)x + (size_t)st * s->d_model * esz;
         void *ys = (char *)y + (size_t)st * s->d_model * ysz;
         int rc = (s->dtype == SI_BF16)
-                     ? launch_simple_step<SI_BF16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, status_dev, stream)
-                     : launch_simple_step<SI_F16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, status_dev, stream);
+                     ? launch_simple_step<SI_BF16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream)
+                     : launch_simple_step<SI_F16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream);
         if (rc != SI_OK) return rc;
     }
     return SI_OK;
@@ -277,6 +309,6 @@ extern "C" int si_ffn_forward_noalloc(const si_store_t *store, int layer, const 
     // nothing left over from an earlier call is ever read and nothing needs clearing
     const unsigned f = flags & SI_FLAG_RESIDUAL;
     return store->dtype == SI_BF16
-               ? launch_simple_step<SI_BF16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, status_dev, stream)
-               : launch_simple_step<SI_F16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, status_dev, stream);
+               ? launch_simple_step<SI_BF16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, 2 * store->num_sms, status_dev, stream)
+               : launch_simple_step<SI_F16>(store, layer, x, idx, nullptr, 0, k, y, y_dtype, f, scratch, 2 * store->num_sms, status_dev, stream);
 }
