@@ -194,6 +194,7 @@ def run_ours(args):
     if cpu_tokens:
         from oracle import selectinfer_oracle as oracle  # cpu_baseline leg only
     cpu_time = 0.0
+    cpu_time_1t, cpu_layers_1t = 0.0, 0
     parity = []
     for l in range(L):
         wg, wu, wd = wl.layer_weights(cfg, l)
@@ -207,6 +208,11 @@ def run_ours(args):
             for t in range(cpu_tokens):
                 y_ref = oracle.ffn(wg, wu, wd, xs[t], ids[lists[t]], dtype=cfg.dtype, threads=host_threads)
             cpu_time += time.perf_counter() - t0
+            if l < 4:                                     # one token on four layers with a single thread
+                t0 = time.perf_counter()
+                oracle.ffn(wg, wu, wd, xs[0], ids[lists[0]], dtype=cfg.dtype, threads=1)
+                cpu_time_1t += time.perf_counter() - t0
+                cpu_layers_1t += 1
             if l in (0, L - 1):
                 cpu_samples.append((l, cpu_tokens - 1, y_ref))
         del wg, wu, wd
@@ -308,6 +314,19 @@ def run_ours(args):
         alg_bytes = wl.selected_bytes_per_token(cfg) * tokens          # per launch (= per step), per GPU
         launch_ms = statistics.mean(per_step_ms)
         achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
+        # practical ceiling beside it: one kernel that only reads the store once with plain loads
+        chk = torch.zeros(1, dtype=torch.int32, device="cuda")
+        rb_bytes = store.nbytes - store.nbytes % 16
+        for _ in range(2):
+            api.si_debug_read_bandwidth(store.mem_aligned, rb_bytes, chk)
+        torch.cuda.synchronize()
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(3):
+            api.si_debug_read_bandwidth(store.mem_aligned, rb_bytes, chk)
+        r1.record()
+        torch.cuda.synchronize()
+        read_ceiling = rb_bytes * 3 / (r0.elapsed_time(r1) * 1e-3) / 1e9
         out = {
             "metric": METRIC, "value": tok_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -330,6 +349,9 @@ def run_ours(args):
                          "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                          "kernel": "si_decode_persistent_kernel" if not args.simple else "si_decode_partial_kernel",
                          "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": launch_ms,
+                         "launch_ms_median": statistics.median(per_step_ms), "launch_ms_best": min(per_step_ms),
+                         "read_only_kernel_gbs": read_ceiling,
+                         "frac_of_read_only_kernel": achieved / read_ceiling,
                          "traffic": (args.traffic_bytes if args.traffic_bytes is not None else
                                      (NCU_DRAM_BYTES_PER_C2_STEP * n_steps
                                       if (cfg.name == "c2" and not args.simple) else None))},
@@ -345,7 +367,9 @@ def run_ours(args):
             out["cpu_baseline"] = {
                 "value": cpu_tokens / cpu_time, "unit": UNIT, "cores": host_threads, "kind": "oracle",
                 "sample": f"{cpu_tokens} tokens x all {L} layers, float64 oracle as it stands, "
-                          f"{host_threads} OpenMP threads"}
+                          f"{host_threads} OpenMP threads",
+                "single_thread": {"value": (cpu_layers_1t / L) / cpu_time_1t if cpu_time_1t > 0 else None, "unit": UNIT,
+                                  "sample": f"1 token x {cpu_layers_1t} layers with one thread, scaled to {L} layers"}}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

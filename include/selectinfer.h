@@ -226,6 +226,13 @@ int si_debug_decode_profile(void *dev_buf);
  * launch gives the practical ceiling of the record stream on the same lists. */
 int si_debug_decode_stream_only(int on);
 
+/* Diagnostics: one launch that reads `bytes` bytes (a multiple of 16) at the 16-byte-aligned device
+ * pointer `mem` once with plain 16-byte loads, all SMs busy, and stores a checksum of them in
+ * *checksum_dev (device uint32).  Timing it on the neuron store gives the read bandwidth a kernel
+ * with no other work reaches on this GPU, the practical ceiling quoted beside the decode kernel.  The
+ * paper has no counterpart. */
+int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream);
+
 /* Library build information: "sm_100a" etc.  Never NULL. */
 const char *si_build_info(void);
 

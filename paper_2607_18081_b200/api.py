@@ -32,7 +32,7 @@ EXPORTS = [
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only",
+    "si_debug_decode_stream_only", "si_debug_read_bandwidth",
 ]
 
 
@@ -71,6 +71,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_ffn_forward_noalloc.argtypes = [vp, ci, vp, vp, ci, vp, ci, cu, vp, vp]
     lib.si_debug_decode_profile.argtypes = [vp]
     lib.si_debug_decode_stream_only.argtypes = [ci]
+    lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("si_strerror", "si_build_info", "si_last_cuda_error"):
@@ -216,6 +217,10 @@ def si_union(handle, layer: int, T: int, idx, idx_offsets, k_fixed: int, union_o
     _check(_lib.si_union(handle, layer, T, _dp(idx), _dp(idx_offsets), k_fixed, _dp(union_out), _dp(n_union_out),
                          _dp(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "si_union")
+
+
+def si_debug_read_bandwidth(mem, nbytes: int, checksum, stream=None) -> None:
+    _check(_lib.si_debug_read_bandwidth(_dp(mem), nbytes, _dp(checksum), _stream(stream)), "si_debug_read_bandwidth")
 
 
 def si_debug_decode_stream_only(on: bool) -> None:

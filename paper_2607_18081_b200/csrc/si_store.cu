@@ -226,3 +226,37 @@ extern "C" int si_store_records(const si_store_t *store, int layer, const void *
     if (record_bytes_out) *record_bytes_out = store->record_bytes();
     return SI_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Diagnostics: read-only streaming kernel (bandwidth ceiling of plain loads).
+namespace {
+__global__ void __launch_bounds__(512)
+si_read_bandwidth_kernel(const uint4 *__restrict__ p, size_t n16, unsigned int *checksum) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned int acc = 0;
+    // eight independent 16-byte loads per thread and round
+    for (; i + 7 * stride < n16; i += 8 * stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = __ldcs(p + i + j * stride);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc ^= v[j].x ^ v[j].y ^ v[j].z ^ v[j].w;
+    }
+    for (; i < n16; i += stride) { const uint4 v = __ldcs(p + i); acc ^= v.x ^ v.y ^ v.z ^ v.w; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if ((threadIdx.x & 31) == 0 && acc != 0) atomicXor(checksum, acc);
+}
+}  // namespace
+
+extern "C" int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream) {
+    if (!mem || !checksum_dev || (bytes & 15) || (((uintptr_t)mem) & 15)) return SI_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    SI_CUDA_TRY(cudaGetDevice(&dev));
+    SI_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    SI_CUDA_TRY(cudaMemsetAsync(checksum_dev, 0, 4, (cudaStream_t)stream));
+    si_read_bandwidth_kernel<<<sms * 4, 512, 0, (cudaStream_t)stream>>>((const uint4 *)mem, bytes / 16, checksum_dev);
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}
