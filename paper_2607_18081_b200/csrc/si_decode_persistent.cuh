@@ -195,6 +195,38 @@ __device__ __forceinline__ float dot8(const uint4 &v, const float (&x)[8]) {
     return a;
 }
 
+// Packed pairs of fp32 values in 64-bit registers and the two-wide fp32 FMA of sm_100: half the
+// FMA instructions of the scalar form for the dot products and the down accumulate.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// the two 16-bit elements of a 32-bit word as a packed fp32 pair (element order kept)
+template <int DT>
+__device__ __forceinline__ unsigned long long pair_of(uint32_t w) {
+    return pack2(si_cvt<DT>::lo(w), si_cvt<DT>::hi(w));
+}
+template <int DT>
+__device__ __forceinline__ void unpack8p(const uint4 &v, unsigned long long (&f)[4]) {
+    f[0] = pair_of<DT>(v.x); f[1] = pair_of<DT>(v.y); f[2] = pair_of<DT>(v.z); f[3] = pair_of<DT>(v.w);
+}
+// a += (v[0..7] * x[0..7]) pairwise: even elements accumulate in the low half, odd ones in the high half
+template <int DT>
+__device__ __forceinline__ unsigned long long dot8p(const uint4 &v, const unsigned long long (&x)[4], unsigned long long a) {
+    a = fma2(pair_of<DT>(v.x), x[0], a); a = fma2(pair_of<DT>(v.y), x[1], a);
+    a = fma2(pair_of<DT>(v.z), x[2], a); a = fma2(pair_of<DT>(v.w), x[3], a);
+    return a;
+}
+
 // Per-step list geometry: which entries of the step's list belong to virtual CTA b of G.
 struct StepGeom { int base, k, first, cnt; };
 __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, int b) {
@@ -232,7 +264,7 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
     }
 }
 
-template <int DT, int NCH>
+template <int DT, int NCH, bool kFull>   // kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256)
 __global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -375,7 +407,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 t_last = clock64();
             } else {
                 if (*cta_abort || clock64() - t_last > kWaitCycles) { ok = false; break; }
-                __nanosleep(40);       // nothing to issue: do not burn issue slots and power
+                __nanosleep(100);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -417,11 +449,11 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const bool noarith = (P.stream_only & 1) != 0;  // diagnostics: drain only
 
         for (int step = 0; step < P.n_steps && !fail; ++step) {
-            float xr[NCH][8], acc[NCH][8];
+            unsigned long long xr[NCH][4], acc[NCH][4];   // packed fp32 pairs
 #pragma unroll
             for (int i = 0; i < NCH; ++i)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { acc[i][e] = 0.f; xr[i][e] = 0.f; }
+                for (int e = 0; e < 4; ++e) { acc[i][e] = 0ull; xr[i][e] = 0ull; }
             {
                 int cnt;
                 {   // x item
@@ -432,7 +464,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 #pragma unroll
                     for (int i = 0; i < NCH; ++i) {
                         const int c = t + kSetThreads * i;
-                        if (c < chunks) unpack8<DT>(xs[c], xr[i]);
+                        if (kFull || c < chunks) unpack8p<DT>(xs[c], xr[i]);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sempty[st]);
@@ -445,26 +477,36 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 for (int i = 0; i < cnt; ++i) {
                     const int st = n % S; const uint32_t ph = (n / S) & 1;
                     fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
-                    const bool okr = !fail && smeta[st] != 0 && !noarith;
+                    const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0 and no accumulate
                     // ---- copy this thread's chunks of the record into registers, free the stage
                     const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
                     uint4 ga[NCH], up[NCH], dn[NCH];
 #pragma unroll
                     for (int k2 = 0; k2 < NCH; ++k2) {
                         const int c = t + kSetThreads * k2;
-                        const bool in = okr && c < chunks;
-                        ga[k2] = in ? rr[c] : make_uint4(0, 0, 0, 0);
-                        up[k2] = in ? rr[chunks + c] : make_uint4(0, 0, 0, 0);
-                        dn[k2] = in ? rr[2 * chunks + c] : make_uint4(0, 0, 0, 0);
+                        if (kFull) {
+                            ga[k2] = rr[c]; up[k2] = rr[chunks + c]; dn[k2] = rr[2 * chunks + c];
+                        } else {
+                            const bool in = c < chunks;
+                            ga[k2] = in ? rr[c] : make_uint4(0, 0, 0, 0);
+                            up[k2] = in ? rr[chunks + c] : make_uint4(0, 0, 0, 0);
+                            dn[k2] = in ? rr[2 * chunks + c] : make_uint4(0, 0, 0, 0);
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sempty[st]);
                     ++n;
                     SI_PROF(1);                           // wait for the record + copy out
                     // ---- dot products: thread slice, warp butterfly (lane 0 <- gate, lane 16 <- up)
-                    float g = 0.f, u = 0.f;
+                    float g, u;
+                    {
+                        unsigned long long g2 = 0ull, u2 = 0ull;
 #pragma unroll
-                    for (int k2 = 0; k2 < NCH; ++k2) { g += dot8<DT>(ga[k2], xr[k2]); u += dot8<DT>(up[k2], xr[k2]); }
+                        for (int k2 = 0; k2 < NCH; ++k2) { g2 = dot8p<DT>(ga[k2], xr[k2], g2); u2 = dot8p<DT>(up[k2], xr[k2], u2); }
+                        float lo, hi;
+                        unpack2(g2, lo, hi); g = lo + hi;
+                        unpack2(u2, lo, hi); u = lo + hi;
+                    }
                     {
                         const bool hi16 = (lane & 16) != 0;
                         float keep = (hi16 ? u : g) + __shfl_xor_sync(0xFFFFFFFFu, hi16 ? g : u, 16);
@@ -491,13 +533,16 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                             gs += v4.x; us += v4.y; gs += v4.z; us += v4.w;
                         }
                     }
-                    const float h = okr ? si_silu_mul(gs, us) : 0.f;
+                    if (okr) {         // a record that was not copied (slot out of range) holds stale bytes
+                        const float h = si_silu_mul(gs, us);
+                        const unsigned long long hh = pack2(h, h);
 #pragma unroll
-                    for (int k2 = 0; k2 < NCH; ++k2) {
-                        float f[8];
-                        unpack8<DT>(dn[k2], f);
+                        for (int k2 = 0; k2 < NCH; ++k2) {
+                            unsigned long long f[4];
+                            unpack8p<DT>(dn[k2], f);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[k2][e] = fmaf(h, f[e], acc[k2][e]);
+                            for (int e = 0; e < 4; ++e) acc[k2][e] = fma2(hh, f[e], acc[k2][e]);
+                        }
                     }
                     SI_PROF(2);                           // record arithmetic
                 }
@@ -517,10 +562,10 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 #pragma unroll
                 for (int k2 = 0; k2 < NCH; ++k2) {
                     const int c = t + kSetThreads * k2;
-                    if (c < chunks) {
-                        float4 *o = reinterpret_cast<float4 *>(ab + (size_t)c * 8);
-                        o[0] = make_float4(acc[k2][0], acc[k2][1], acc[k2][2], acc[k2][3]);
-                        o[1] = make_float4(acc[k2][4], acc[k2][5], acc[k2][6], acc[k2][7]);
+                    if (kFull || c < chunks) {
+                        ulonglong2 *o = reinterpret_cast<ulonglong2 *>(ab + (size_t)c * 8);   // pairs are consecutive columns
+                        o[0] = make_ulonglong2(acc[k2][0], acc[k2][1]);
+                        o[1] = make_ulonglong2(acc[k2][2], acc[k2][3]);
                     }
                 }
                 __syncwarp();
@@ -587,7 +632,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                             else if (!(taken & 2) && mbar_test_wait(&sm->accfull[1][r], par)) q = 1;
                             else {
                                 if (*cta_abort || clock64() - t0 > kWaitCycles) break;
-                                __nanosleep(64);
+                                __nanosleep(200);
                             }
                         }
                         ok = q >= 0;
@@ -727,9 +772,9 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH>
+template <int DT, int NCH, bool FULL>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH>;
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
     static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
     int dev = 0;
@@ -779,8 +824,11 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
     const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
-#define SI_PL(DT) (nch <= 1 ? si_decode_persistent_launch_t<DT, 1>(P, G, stream) \
-                            : si_decode_persistent_launch_t<DT, 2>(P, G, stream))
+    const bool full = P.chunks == nch * si_persist::kSetThreads;
+#define SI_PL(DT) (nch <= 1 ? (full ? si_decode_persistent_launch_t<DT, 1, true>(P, G, stream)   \
+                                    : si_decode_persistent_launch_t<DT, 1, false>(P, G, stream)) \
+                            : (full ? si_decode_persistent_launch_t<DT, 2, true>(P, G, stream)   \
+                                    : si_decode_persistent_launch_t<DT, 2, false>(P, G, stream)))
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
 #undef SI_PL
 }
