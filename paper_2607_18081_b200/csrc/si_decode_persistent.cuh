@@ -309,6 +309,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const bool mine = lane < kSets * S;            // issue role
         const int iq = mine ? lane / S : 0, is = lane % S;
         uint32_t n = is;                               // set-ring item index this lane issues next
+        uint32_t iph = 0;                              // phase parity of that item's round through the ring
         uint32_t issued = 0;
         // walker (uniform within a half-warp): item wn is item wt of step wstep (t = 0 is x)
         uint32_t wn = 0, desc_ready = 0, total = 0xFFFFFFFFu;
@@ -386,8 +387,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             prefetch_window(do_commit && desc_ready < total);
             bool progressed = false;
             if (have && n < i_ready) {
-                const int st = iq * S + is; const uint32_t ph = (n / S) & 1;
-                if (mbar_test_wait(&empty[st], ph ^ 1)) {
+                const int st = iq * S + is;
+                if (mbar_test_wait(&empty[st], iph ^ 1)) {
                     const uint4 dsc = sm->desc[iq][n % kDescRing];
                     meta[st] = (int)dsc.w;
                     if (dsc.z != 0) {
@@ -399,7 +400,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         mbar_arrive(&full[st]);
                     }
                     ++issued;
-                    n += S;
+                    n += S; iph ^= 1;
                     progressed = true;
                 }
             }
@@ -439,7 +440,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         uint64_t *sfull = full + q * S, *sempty = empty + q * S;
         int *smeta = meta + q * S;
         uint8_t *sring = ring + (size_t)q * S * rec_bytes;
-        uint32_t n = 0;                          // set-ring item counter
+        int st = 0; uint32_t ph = 0;             // ring stage and phase parity of the set's next item
         uint32_t recs = 0;                       // records this set has handed to its barrier
         bool fail = false;
         const bool prof = P.prof != nullptr && t == 0;
@@ -457,7 +458,6 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             {
                 int cnt;
                 {   // x item
-                    const int st = n % S; const uint32_t ph = (n / S) & 1;
                     fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
                     cnt = fail ? 0 : smeta[st];
                     const uint4 *xs = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
@@ -468,14 +468,13 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sempty[st]);
-                    ++n;
+                    if (++st == S) { st = 0; ph ^= 1; }
                 }
                 // the record count steers the set's barriers: agree on it (and on failure) first
                 fail = set_barrier_or(q, fail);
                 if (fail) break;
                 SI_PROF(0);                               // wait for x
                 for (int i = 0; i < cnt; ++i) {
-                    const int st = n % S; const uint32_t ph = (n / S) & 1;
                     fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
                     const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0 and no accumulate
                     // ---- copy this thread's chunks of the record into registers, free the stage
@@ -495,7 +494,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sempty[st]);
-                    ++n;
+                    if (++st == S) { st = 0; ph ^= 1; }
                     SI_PROF(1);                           // wait for the record + copy out
                     // ---- dot products: thread slice, warp butterfly (lane 0 <- gate, lane 16 <- up)
                     float g, u;
