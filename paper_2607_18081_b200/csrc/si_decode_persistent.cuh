@@ -44,10 +44,10 @@ constexpr int kMaxGroups = 8;                     // float4 column groups one CT
 constexpr int kCounterStride = 64;                // uint32 per step: written at +0, reduced at +32 (own 128-byte lines)
 constexpr int kMaxStages = 16;
 constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
-constexpr int kPartialDepth = 8;                  // D: partial-y buffers in flight
+constexpr int kPartialDepth = 10;                 // D: partial-y buffers in flight
 constexpr int kFewSteps = 16;                     // launches this short carry their layer ids as kernel arguments
 constexpr int kProfSlots = 16;                    // int64 cycle counters per SM in the optional phase profile
-constexpr int kLag = 3;                           // a step's cross-SM reduction starts this many steps later
+constexpr int kLag = 4;                           // a step's cross-SM reduction starts this many steps later
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
 
 struct Params {
