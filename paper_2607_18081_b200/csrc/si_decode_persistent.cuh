@@ -264,7 +264,7 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
     }
 }
 
-template <int DT, int NCH, bool kFull>   // kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256)
+template <int DT, int NCH, bool kFull, bool kProf>   // kProf: phase profile compiled in; kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256)
 __global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -443,7 +443,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         int st = 0; uint32_t ph = 0;             // ring stage and phase parity of the set's next item
         uint32_t recs = 0;                       // records this set has handed to its barrier
         bool fail = false;
-        const bool prof = P.prof != nullptr && t == 0;
+        const bool prof = kProf && P.prof != nullptr && t == 0;
         long long pf[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pt = prof ? clock64() : 0;
 #define SI_PROF(slot) do { if (prof) { long long now_ = clock64(); pf[slot] += now_ - pt; pt = now_; } } while (0)
 
@@ -599,7 +599,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const int ngroups = d / 4;
         const int gpc = (ngroups + G - 1) / G;                 // <= kMaxGroups (launch check)
         const int g_valid = ngroups - b * gpc < gpc ? (ngroups - b * gpc < 0 ? 0 : ngroups - b * gpc) : gpc;
-        const bool rprof = P.prof != nullptr && r == 0 && lane == 0;
+        const bool rprof = kProf && P.prof != nullptr && r == 0 && lane == 0;
         long long rp[6] = {0, 0, 0, 0, 0, 0}, rt = rprof ? clock64() : 0;
 #define SI_RPROF(slot) do { if (rprof) { long long now_ = clock64(); rp[slot] += now_ - rt; rt = now_; } } while (0)
         const int bg = lane & (kMaxGroups - 1);                // phase B: this lane's column group ...
@@ -771,9 +771,9 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, bool FULL>
+template <int DT, int NCH, bool FULL, bool PROF>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL>;
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
     static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
     int dev = 0;
@@ -824,10 +824,12 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
     const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
     const bool full = P.chunks == nch * si_persist::kSetThreads;
-#define SI_PL(DT) (nch <= 1 ? (full ? si_decode_persistent_launch_t<DT, 1, true>(P, G, stream)   \
-                                    : si_decode_persistent_launch_t<DT, 1, false>(P, G, stream)) \
-                            : (full ? si_decode_persistent_launch_t<DT, 2, true>(P, G, stream)   \
-                                    : si_decode_persistent_launch_t<DT, 2, false>(P, G, stream)))
+    // the phase profile is a separate instantiation: the production kernel carries no clock reads
+#define SI_PL2(DT, N, F) (P.prof ? si_decode_persistent_launch_t<DT, N, F, true>(P, G, stream) \
+                                 : si_decode_persistent_launch_t<DT, N, F, false>(P, G, stream))
+#define SI_PL(DT) (nch <= 1 ? (full ? SI_PL2(DT, 1, true) : SI_PL2(DT, 1, false)) \
+                            : (full ? SI_PL2(DT, 2, true) : SI_PL2(DT, 2, false)))
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
+#undef SI_PL2
 #undef SI_PL
 }
