@@ -24,6 +24,7 @@ SI_ERR_NOMEM, SI_ERR_CUDA, SI_ERR_TIMEOUT, SI_ERR_UNSUPPORTED = -5, -6, -7, -8
 SI_ERR_TOO_LARGE = -9
 SI_FLAG_CHECK, SI_FLAG_RESIDUAL, SI_FLAG_UNION_UNMASKED, SI_FLAG_SCORE_ABS = 1, 2, 4, 8
 SI_FLAG_SHARED_LIST = 16
+SI_FLAG_UNION_PATH = 32
 SI_FLAG_SIMPLE_KERNELS = 256
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 

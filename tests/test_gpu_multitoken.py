@@ -60,12 +60,15 @@ def test_union_is_bit_exact(api, c1):
 
 @pytest.mark.parametrize("T", [2, 4, 16])
 def test_c1_multitoken_matches_per_token_oracle(api, c1, T):
+    """Both routes for a few tokens: the default (decode kernel token by token up to 4 tokens) and
+    the union path forced by its flag."""
     cfg = c1.cfg
     lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=c1.slot_of_rank[0])
     x = wl.x_tokens(cfg, 0, T)
-    y = _run(api, c1, 0, x, lists, None, cfg.k_active, T)
-    for t in range(T):
-        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], lists[t]), f"T={T} token {t}")
+    for flags in (0, api.SI_FLAG_UNION_PATH):
+        y = _run(api, c1, 0, x, lists, None, cfg.k_active, T, flags=flags)
+        for t in range(T):
+            assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], lists[t]), f"T={T} token {t} flags={flags}")
 
 
 def test_c1_ragged_empty_unmasked_residual(api, c1):
@@ -100,14 +103,14 @@ def test_7b_batched_decode_union(api, m7b, T):
     k = cfg.k_active
     lists = wl.zipf_lists(cfg, 0, T)
     x = wl.x_tokens(cfg, 0, T)
-    y = _run(api, m7b, 0, x, lists, None, k, T)
+    y = _run(api, m7b, 0, x, lists, None, k, T, flags=api.SI_FLAG_UNION_PATH)
     yb = _run(api, m7b, 0, x, lists, None, k, T, y_dtype=torch.bfloat16)
     for t in sorted({0, 1, T // 2, T - 1}):
         ref = m7b.oracle_y(0, x[t], lists[t])
         assert_close(from_dev(y[t]), ref, f"T={T} token {t}")
         assert_close(from_dev(yb[t]), ref, f"T={T} token {t} bf16 out")
     # run-to-run bit stability
-    y2 = _run(api, m7b, 0, x, lists, None, k, T)
+    y2 = _run(api, m7b, 0, x, lists, None, k, T, flags=api.SI_FLAG_UNION_PATH)
     assert torch.equal(y, y2)
 
 
