@@ -412,7 +412,7 @@ def run_multitoken(args, cfg, rank, world, local_rank):
             lists[:, l] = ll.reshape(n_groups, T, k)
         union_sizes = [len(np.unique(lists[g, l])) for g in range(n_groups) for l in range(min(L, 4))]
         idx = torch.from_numpy(lists).cuda()
-        flags = 0
+        flags = api.SI_FLAG_UNION_PATH     # config 3 is about the union path (few tokens would otherwise take the decode route)
     y = torch.empty(n_groups, L, T, d, dtype=tdt, device="cuda")
     ws = store.workspace(T, k, 1)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
