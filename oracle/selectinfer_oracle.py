@@ -14,6 +14,8 @@ cpu_baseline / reference legs may import this module.
   NaN ranks below everything.  Output ascending by index.
 * ``select_threshold`` -- extension with no counterpart in the paper (brute-force
   pinned only).
+* ``prefill_vote`` -- Section 5: per-token top alpha, frequency count over the prompt's tokens,
+  top beta by frequency, merge with the static prefix up to phi.
 * ``union`` -- sorted set union of per-token lists plus per-token membership bitmasks.
 * ``loadset`` -- Section 4: base = top delta of the task ranking, then the model
   ranking in order, skipping ids already chosen, until gamma neurons are loaded.
@@ -168,6 +170,41 @@ def select_threshold(scores, tau: float, use_abs: bool = False) -> np.ndarray:
         s = np.abs(s)
     tau32 = np.float32(tau)
     return np.array([i for i, v in enumerate(s) if v > tau32], dtype=np.int32)
+
+
+def prefill_vote(acts, alpha: int, beta: int, n_static: int, phi_count: int, use_abs: bool = True):
+    """Section 5, selection of the dynamic neurons during prefill, in the paper's order:
+
+    1. for every prompt token, rank the activations of all loaded neurons in descending order and
+       record the indices of the top alpha (``select_topk``: ties to the lower index);
+    2. count how often each neuron occurs in these lists;
+    3. the beta neurons with the highest frequency are the dynamic candidates (ties: lower slot;
+       a neuron that occurs in no list is never a candidate -- reading, the paper is silent);
+    4. the static neurons (slots 0 .. n_static-1: the base neurons come first in the store) are
+       combined with the candidates, walked in order of frequency, candidates that are already
+       static skipped, until phi_count neurons are chosen.
+
+    acts: [T, n] activations h_i(x_t) of the n loaded neurons.  use_abs ranks |a| (the paper's
+    profiling and overlap studies define "most active" by the absolute value; its run-time text
+    says only "descending order").  Returns (chosen slots ascending, int64 counts [n]).
+    """
+    a = np.asarray(acts, dtype=np.float32)
+    T, n = a.shape
+    if not (0 <= alpha <= n and 0 <= beta <= n and 0 <= n_static <= n and 0 <= phi_count <= n):
+        raise ValueError("count out of range")
+    counts = np.zeros(n, dtype=np.int64)
+    for t in range(T):
+        for i in select_topk(a[t], alpha, use_abs=use_abs):
+            counts[i] += 1
+    by_frequency = sorted(range(n), key=lambda i: (-int(counts[i]), i))
+    candidates = [i for i in by_frequency[:beta] if counts[i] > 0]
+    chosen = list(range(min(n_static, phi_count)))
+    for i in candidates:
+        if len(chosen) >= phi_count:
+            break
+        if i >= n_static:
+            chosen.append(i)
+    return np.array(sorted(chosen), dtype=np.int32), counts
 
 
 def union(lists, n_loaded: int):

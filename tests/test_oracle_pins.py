@@ -276,3 +276,57 @@ def test_count_rounding_of_configs():
     assert wl.CONFIGS["c4"].k_active == 3082
     got = [[so.count_from_pct(a, so.count_from_pct(l, 14336)) for a in wl.C5_ACTIVE] for l in wl.C5_LOADED]
     assert got == [[215, 430, 860, 2150], [358, 716, 1433, 3584], [501, 1003, 2007, 5017], [716, 1433, 2867, 7168]]
+
+
+# --------------------------------------------------------------------------- prefill vote (Section 5)
+
+def test_prefill_vote_worked_example():
+    """Hand-worked case.  4 tokens, 6 loaded neurons, alpha = 2: the per-token top-2 lists by |a| are
+    {1,4}, {4,5}, {1,4}, {0,5}, hence the counts [1, 2, 0, 0, 3, 2]."""
+    acts = np.array([[0.1, -9.0, 0.2, 0.0, 8.0, 0.3],      # |a|: top 2 = {1, 4}
+                     [0.1, 0.2, 0.3, 0.0, -7.0, 6.0],      # {4, 5}
+                     [0.0, 5.0, 0.1, 0.2, 5.5, 0.3],       # {1, 4}
+                     [-4.0, 0.1, 0.2, 0.3, 0.0, 3.0]],     # {0, 5}
+                    dtype=np.float32)
+    chosen, counts = so.prefill_vote(acts, alpha=2, beta=3, n_static=1, phi_count=3)
+    assert counts.tolist() == [1, 2, 0, 0, 3, 2]
+    # frequency order: 4 (3), 1 (2), 5 (2), 0 (1) ... ; beta = 3 candidates {4, 1, 5}; static = {0};
+    # phi = 3 -> static 0 plus the two most frequent candidates 4 and 1
+    assert chosen.tolist() == [0, 1, 4]
+    # with n_static = 2 slot 1 is static already: the walk skips it and takes 4, then 5
+    chosen, _ = so.prefill_vote(acts, alpha=2, beta=3, n_static=2, phi_count=4)
+    assert chosen.tolist() == [0, 1, 4, 5]
+    # signed ranking: token 0's top 2 become {4, 5}, token 1's {2, 5}, token 3's {3, 5}
+    chosen, counts = so.prefill_vote(acts, alpha=2, beta=2, n_static=0, phi_count=2, use_abs=False)
+    assert counts.tolist() == [0, 1, 1, 1, 2, 3] and chosen.tolist() == [4, 5]
+
+
+def test_prefill_vote_special_cases_and_invariants():
+    g = np.random.default_rng(77)
+    T, n = 9, 40
+    acts = g.standard_normal((T, n)).astype(np.float32)
+    # beta = 0: nothing dynamic; phi below the static count truncates the static prefix
+    assert so.prefill_vote(acts, 5, 0, 7, 20)[0].tolist() == list(range(7))
+    assert so.prefill_vote(acts, 5, 10, 7, 4)[0].tolist() == list(range(4))
+    # alpha = n: every neuron is in every list, all counts equal T, candidates are the lowest slots
+    chosen, counts = so.prefill_vote(acts, n, 12, 3, 10)
+    assert set(counts.tolist()) == {T} and chosen.tolist() == list(range(10))
+    # one token: the dynamic part is that token's top alpha by |a|, lowest frequency-tied slots first
+    one = acts[:1]
+    chosen, counts = so.prefill_vote(one, 6, n, 0, 6)
+    assert chosen.tolist() == so.select_topk(one[0], 6, use_abs=True).tolist()
+    # invariants on random cases: size, static prefix, counts sum, dominance of the chosen candidates
+    for trial in range(20):
+        alpha, beta = int(g.integers(0, n + 1)), int(g.integers(0, n + 1))
+        n_static, phi = int(g.integers(0, n + 1)), int(g.integers(0, n + 1))
+        chosen, counts = so.prefill_vote(acts, alpha, beta, n_static, phi)
+        assert counts.sum() == T * alpha and len(set(chosen.tolist())) == len(chosen) <= phi
+        assert chosen.tolist() == sorted(chosen.tolist())
+        assert all(s in chosen for s in range(min(n_static, phi)))
+        dyn = [i for i in chosen if i >= n_static]
+        assert all(counts[i] > 0 for i in dyn)
+        if dyn and len(chosen) == phi:      # a chosen candidate is never less frequent than a left-out neuron
+            worst = min((counts[i], -i) for i in dyn)
+            top_beta = sorted(range(n), key=lambda i: (-int(counts[i]), i))[:beta]
+            left_out = [i for i in top_beta if i >= n_static and i not in dyn and counts[i] > 0]
+            assert all((counts[i], -i) < worst for i in left_out)
