@@ -217,6 +217,31 @@ int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
              const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
              void *workspace, size_t ws_bytes, void *stream);
 
+/* ---------------------------------------------------------------- prefill: dynamic neurons
+ *
+ * Section 5: during prefill the activations of all loaded neurons are computed for every prompt
+ * token; each token's top alpha neurons are recorded, the occurrences are counted over the
+ * tokens, the beta most frequent neurons are the dynamic candidates, and the static neurons
+ * (slots 0 .. n_static-1: the base neurons come first in the store) are combined with the
+ * candidates, in order of frequency, until phi_count neurons are chosen.  Ties (per-token
+ * activations, frequencies) go to the lower slot; a neuron that occurs in no list is never
+ * dynamic; candidates that are static already are skipped.  If phi_count <= n_static the
+ * result is the first phi_count static slots.
+ *
+ * si_prefill_vote works on given activations:
+ *   acts       device float32 [T, row_stride >= n]: activation of loaded slot i for token t
+ *   flags      SI_FLAG_SCORE_ABS ranks |activation| (what the paper's "most active" means in its
+ *              profiling; without the flag the signed value is ranked)
+ *   idx_out    device int32, capacity cap >= phi_count: chosen slots, ascending; *n_out (device
+ *              int32) their number (<= phi_count)
+ *   counts_out optional device int32 [n]: the frequency of every slot
+ *   workspace  device, 256-byte aligned, si_prefill_vote_workspace_bytes(T, n, alpha) bytes
+ * Asynchronous on stream; integer decisions only, so the result is exact and unique. */
+int si_prefill_vote_workspace_bytes(int T, int n, int alpha, size_t *bytes_out);
+int si_prefill_vote(const float *acts, int T, int n, int row_stride, int alpha, int beta, int n_static,
+                    int phi_count, unsigned flags, int32_t *idx_out, int cap, int32_t *n_out,
+                    int32_t *counts_out, void *workspace, size_t ws_bytes, void *stream);
+
 /* Diagnostics: while dev_buf (device int64 [num_SMs][16]) is set, each persistent decode
  * launch stores per-SM cycle counts of its phases there.  Slots 0..5: first consumer set (wait
  * for x, wait for a record + copy to registers, record arithmetic, accumulator hand-over,

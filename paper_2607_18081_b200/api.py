@@ -33,7 +33,7 @@ EXPORTS = [
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only", "si_debug_read_bandwidth",
+    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote",
 ]
 
 
@@ -73,6 +73,8 @@ def _load_library() -> ctypes.CDLL:
     lib.si_debug_decode_profile.argtypes = [vp]
     lib.si_debug_decode_stream_only.argtypes = [ci]
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
+    lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
+    lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("si_strerror", "si_build_info", "si_last_cuda_error"):
@@ -179,6 +181,20 @@ def si_select(scores, mode: int, k: int, tau: float, flags: int, idx_out, n_out,
                           _dp(n_out), _dp(workspace),
                           0 if workspace is None else workspace.numel() * workspace.element_size(),
                           _stream(stream)), "si_select")
+
+
+def si_prefill_vote_workspace_bytes(T: int, n: int, alpha: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.si_prefill_vote_workspace_bytes(T, n, alpha, ctypes.byref(out)), "si_prefill_vote_workspace_bytes")
+    return out.value
+
+
+def si_prefill_vote(acts, alpha: int, beta: int, n_static: int, phi_count: int, flags: int, idx_out, n_out,
+                    counts_out, workspace, stream=None) -> None:
+    T, n = acts.shape
+    _check(_lib.si_prefill_vote(_dp(acts), T, n, acts.stride(0), alpha, beta, n_static, phi_count, flags, _dp(idx_out),
+                                idx_out.numel(), _dp(n_out), _dp(counts_out), _dp(workspace),
+                                workspace.numel() * workspace.element_size(), _stream(stream)), "si_prefill_vote")
 
 
 def si_ffn_forward(handle, layer: int, x, T: int, idx, idx_offsets, k_fixed: int, y, flags: int, workspace,

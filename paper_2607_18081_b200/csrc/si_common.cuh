@@ -81,6 +81,12 @@ int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int
                      float tau, unsigned flags, int32_t *idx_out, int out_stride, int cap,
                      int32_t *n_out, void *workspace, size_t ws_bytes, cudaStream_t stream);
 
+// implemented in si_vote.cu
+size_t si_prefill_vote_ws_bytes_impl(int T, int n, int alpha);
+int si_prefill_vote_launch(const float *acts, int T, int n, int row_stride, int alpha, int beta, int n_static,
+                           int phi_count, unsigned flags, int32_t *idx_out, int cap, int32_t *n_out,
+                           int32_t *counts_out, void *workspace, size_t ws_bytes, cudaStream_t stream);
+
 // implemented in si_check.cu: device-side list validation for SI_FLAG_CHECK
 int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed,
                                const int32_t *step_layers_dev, const int32_t *idx,
