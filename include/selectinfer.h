@@ -242,6 +242,22 @@ int si_prefill_vote(const float *acts, int T, int n, int row_stride, int alpha, 
                     int phi_count, unsigned flags, int32_t *idx_out, int cap, int32_t *n_out,
                     int32_t *counts_out, void *workspace, size_t ws_bytes, void *stream);
 
+/* si_prefill_forward: prefill of one layer for the prompt's T tokens as the paper describes it --
+ * y[t] = FFN over ALL loaded neurons of the layer (tensor-core path, one shared list of every slot) --
+ * followed by si_prefill_vote on the activations h = SiLU(g) * u that this computation itself
+ * produced (rounded to the store dtype, as they enter the down projection).
+ *   x, y       device [T, d_model] (y of y_dtype: SI_F32 or the store dtype); flags: SI_FLAG_RESIDUAL,
+ *              SI_FLAG_SCORE_ABS
+ *   idx_out, cap, n_out, alpha, beta, n_static, phi_count: as for si_prefill_vote
+ *   acts_out   optional device float32 [T, n_loaded]: receives the activations that were ranked
+ *   workspace  si_workspace_bytes(store, T, n_loaded, 1) bytes; vote_workspace
+ *              si_prefill_vote_workspace_bytes(T, n_loaded, alpha) bytes, both 256-byte aligned
+ * Asynchronous on stream. */
+int si_prefill_forward(const si_store_t *store, int layer, const void *x, int T, void *y, int y_dtype,
+                       int alpha, int beta, int n_static, int phi_count, unsigned flags, int32_t *idx_out,
+                       int cap, int32_t *n_out, float *acts_out, void *workspace, size_t ws_bytes,
+                       void *vote_workspace, size_t vote_ws_bytes, int32_t *status_dev, void *stream);
+
 /* Diagnostics: while dev_buf (device int64 [num_SMs][16]) is set, each persistent decode
  * launch stores per-SM cycle counts of its phases there.  Slots 0..5: first consumer set (wait
  * for x, wait for a record + copy to registers, record arithmetic, accumulator hand-over,

@@ -33,7 +33,7 @@ EXPORTS = [
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote",
+    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward",
 ]
 
 
@@ -75,6 +75,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
     lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
     lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
+    lib.si_prefill_forward.argtypes = [vp, ci, vp, ci, vp, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("si_strerror", "si_build_info", "si_last_cuda_error"):
@@ -195,6 +196,15 @@ def si_prefill_vote(acts, alpha: int, beta: int, n_static: int, phi_count: int, 
     _check(_lib.si_prefill_vote(_dp(acts), T, n, acts.stride(0), alpha, beta, n_static, phi_count, flags, _dp(idx_out),
                                 idx_out.numel(), _dp(n_out), _dp(counts_out), _dp(workspace),
                                 workspace.numel() * workspace.element_size(), _stream(stream)), "si_prefill_vote")
+
+
+def si_prefill_forward(handle, layer: int, x, T: int, y, alpha: int, beta: int, n_static: int, phi_count: int,
+                       flags: int, idx_out, n_out, acts_out, workspace, vote_workspace, status=None, stream=None) -> None:
+    _check(_lib.si_prefill_forward(handle, layer, _dp(x), T, _dp(y), dtype_code(y.dtype), alpha, beta, n_static,
+                                   phi_count, flags, _dp(idx_out), idx_out.numel(), _dp(n_out), _dp(acts_out),
+                                   _dp(workspace), workspace.numel() * workspace.element_size(), _dp(vote_workspace),
+                                   vote_workspace.numel() * vote_workspace.element_size(), _dp(status),
+                                   _stream(stream)), "si_prefill_forward")
 
 
 def si_ffn_forward(handle, layer: int, x, T: int, idx, idx_offsets, k_fixed: int, y, flags: int, workspace,

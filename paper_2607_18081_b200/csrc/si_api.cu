@@ -157,3 +157,61 @@ extern "C" int si_union(const si_store_t *store, int layer, int T, const int32_t
     return si_union_launch(store, layer, T, idx, idx_offsets, k_fixed, union_out, n_union_out, workspace,
                            ws_bytes, (cudaStream_t)stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Prefill of one layer with the selection of the dynamic neurons (Section 5): the FFN over ALL loaded
+// neurons for the prompt's T tokens, then the vote on the activations h = SiLU(g) * u that this very
+// computation produced (H of the gathered contraction, in the store dtype).
+namespace {
+__global__ void si_iota_kernel(int32_t *out, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = i;
+}
+template <int DT>
+__global__ void si_widen_h_kernel(const uint16_t *__restrict__ h, int h_stride, int T, int n, float *__restrict__ acts) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x, t = blockIdx.y;
+    if (i < n && t < T) acts[(size_t)t * n + i] = si_cvt<DT>::lo((uint32_t)h[(size_t)t * h_stride + i]);
+}
+}  // namespace
+
+extern "C" int si_prefill_forward(const si_store_t *store, int layer, const void *x, int T, void *y, int y_dtype,
+                                  int alpha, int beta, int n_static, int phi_count, unsigned flags,
+                                  int32_t *idx_out, int cap, int32_t *n_out, float *acts_out, void *workspace,
+                                  size_t ws_bytes, void *vote_workspace, size_t vote_ws_bytes, int32_t *status_dev,
+                                  void *stream_) {
+    int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
+    if (rc) return rc;
+    if (layer < 0 || layer >= store->n_layers || T <= 0 || !store->loaded[layer]) return SI_ERR_INVALID_ARG;
+    const int n = store->n_loaded[layer];
+    if (n <= 0 || !idx_out || !vote_workspace) return SI_ERR_INVALID_ARG;
+    if (alpha < 0 || alpha > n || beta < 0 || beta > n || n_static < 0 || n_static > n || phi_count < 0 || phi_count > n)
+        return SI_ERR_INVALID_ARG;
+    if (cap < phi_count) return SI_ERR_NOMEM;
+    if (!si_aligned16(idx_out) || (((uintptr_t)vote_workspace) & 255u) || (acts_out && !si_aligned16(acts_out)))
+        return SI_ERR_ALIGNMENT;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const si_ws_layout ws = si_ws_carve(store, T, n, 1);
+    if (ws_bytes < ws.total) return SI_ERR_NOMEM;
+    char *wsb = (char *)workspace;
+    // one shared list: every loaded slot, so the union is the store in slot order (position p = slot p)
+    int32_t *all = (int32_t *)(wsb + ws.sel_off);
+    si_iota_kernel<<<(n + 255) / 256, 256, 0, stream>>>(all, n);
+    rc = si_multi_token_launch(store, layer, x, T, all, nullptr, n, y, y_dtype,
+                               (flags & SI_FLAG_RESIDUAL) | SI_FLAG_SHARED_LIST, workspace, ws_bytes, status_dev, stream);
+    if (rc) return rc;
+    // the activations the contraction used, widened exactly to fp32 (the partial-tile area is free again)
+    float *acts = acts_out;
+    if (!acts) {
+        if ((size_t)T * n * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
+        acts = (float *)(wsb + ws.partial_off);
+    }
+    const int h_stride = (int)si_align_up((size_t)n, 128);
+    dim3 grid((n + 255) / 256, T);
+    if (store->dtype == SI_BF16)
+        si_widen_h_kernel<SI_BF16><<<grid, 256, 0, stream>>>((const uint16_t *)(wsb + ws.h_off), h_stride, T, n, acts);
+    else
+        si_widen_h_kernel<SI_F16><<<grid, 256, 0, stream>>>((const uint16_t *)(wsb + ws.h_off), h_stride, T, n, acts);
+    SI_CUDA_TRY(cudaGetLastError());
+    return si_prefill_vote_launch(acts, T, n, n, alpha, beta, n_static, phi_count, flags, idx_out, cap, n_out, nullptr,
+                                  vote_workspace, vote_ws_bytes, stream);
+}

@@ -1,5 +1,5 @@
-// Runtime selector (Section 5: "sort these activations in descending order and select the
-// top alpha neurons for that token and record the indices").
+// Runtime selector (Section 5: rank a token's activations from the largest down and record the
+// indices of the top alpha).
 //
 // No sort is needed to obtain the set: one CTA per score row finds the k-th largest value by
 // a 4-pass, 8-bit radix select over order-preserving 32-bit keys held in shared memory, then

@@ -1,7 +1,7 @@
-// Prefill selection of the dynamic neurons (Section 5): "For each token, we compute activation
-// values for all loaded neurons", keep each token's top alpha, count how often every neuron
-// occurs over the prompt's tokens, take the beta most frequent as the dynamic candidates and
-// combine them with the static neurons until phi neurons are chosen.
+// Prefill selection of the dynamic neurons (Section 5): with the activations of all loaded
+// neurons at hand for every prompt token, keep each token's top alpha, count how often every
+// neuron occurs over the prompt's tokens, take the beta most frequent as the dynamic candidates
+// and combine them with the static neurons until phi neurons are chosen.
 //
 // Everything is built from the radix selector (one CTA per score row, ties to the lower index):
 //   1. T rows of activations          -> T lists of alpha indices

@@ -68,3 +68,58 @@ def test_vote_prefill_shape_7b(api):
     n_static = (30 * cfg.d_ff) // 100
     phi = (40 * cfg.d_ff) // 100
     _check(api, acts, (20 * n) // 100, 2 * (phi - n_static), n_static, phi)
+
+
+def _aligned(nbytes):
+    t = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    return t[(-t.data_ptr()) % 256:]
+
+
+@pytest.mark.parametrize("cfg_name,T", [("c1", 24), ("c2", 40)])
+def test_prefill_forward_outputs_activations_and_vote(api, cfg_name, T):
+    """si_prefill_forward: y over all loaded neurons and the activations against the float64 oracle; the
+    chosen slots against si_prefill_vote on the exported activations (same library, same decision
+    precision) and, as a sanity check, against the oracle's vote on its own float64 activations."""
+    from tests.gpu_utils import LoadedModel, assert_close, from_dev, to_dev
+    cfg = wl.CONFIGS[cfg_name]
+    m = LoadedModel(cfg, n_layers=1)
+    n, d = cfg.n_loaded, cfg.d_model
+    x = wl.x_tokens(cfg, 0, T)
+    n_static, phi, alpha = (30 * n) // 100, (45 * n) // 100, (15 * n) // 100
+    beta = 2 * (phi - n_static)
+    tdt = torch.float16 if cfg.dtype == "f16" else torch.bfloat16
+    y = torch.empty(T, d, dtype=tdt, device="cuda")
+    acts = torch.empty(T, n, dtype=torch.float32, device="cuda")
+    idx = torch.full((phi,), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(4, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = m.store.workspace(T, n, 1)
+    vws = _aligned(api.si_prefill_vote_workspace_bytes(T, n, alpha))
+    api.si_prefill_forward(m.store.handle, 0, to_dev(x, cfg.dtype), T, y, alpha, beta, n_static, phi,
+                           api.SI_FLAG_SCORE_ABS, idx, cnt, acts, ws, vws, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    wg, wu, wd = m.host[0]
+    gids = m.ids[0]                                  # global neuron id of every slot
+    slot_of_sorted = np.argsort(gids, kind="stable")  # the oracle reports h for the ids in ascending order
+    h_ref = np.empty((T, n))
+    for t in range(T):
+        y_ref, h = so.ffn(wg, wu, wd, x[t], gids, dtype=cfg.dtype, threads=so.host_threads(), return_h=True)
+        h_ref[t, slot_of_sorted] = h
+        assert_close(from_dev(y[t]), y_ref, f"{cfg_name} prefill token {t}")
+    # activations: fp32-accumulated tensor-core dot products rounded to the store dtype
+    a = acts.cpu().numpy().astype(np.float64)
+    rel = np.abs(a - h_ref).max() / np.abs(h_ref).max()
+    assert rel <= (2e-3 if cfg.dtype == "f16" else 1e-2), rel
+    # the decision: identical to the standalone vote on the exported activations
+    idx2 = torch.full((phi,), -1, dtype=torch.int32, device="cuda")
+    cnt2 = torch.zeros(4, dtype=torch.int32, device="cuda")
+    api.si_prefill_vote(acts, alpha, beta, n_static, phi, api.SI_FLAG_SCORE_ABS, idx2, cnt2, None, vws)
+    torch.cuda.synchronize()
+    k = int(cnt[0].item())
+    assert k == int(cnt2[0].item()) and torch.equal(idx[:k], idx2[:k])
+    # and close to the oracle's own end-to-end answer (rounding can only flip near-ties)
+    ref, _ = so.prefill_vote(h_ref.astype(np.float32), alpha, beta, n_static, phi, use_abs=True)
+    got = set(idx[:k].cpu().numpy().tolist())
+    inter = len(got & set(ref.tolist()))
+    assert k == len(ref) and inter >= 0.97 * len(ref), (k, len(ref), inter)
