@@ -75,6 +75,9 @@ enum {
     SI_FLAG_UNION_PATH = 32u,    /* T > 1 only: always form the union and run the tensor-core contractions
                                     (by default up to 4 tokens with lists of their own go through the
                                     batch-1 decode kernel one after the other, which is faster there) */
+    SI_FLAG_LIST_PER_LAYER = 64u, /* si_decode_stack_forward, fixed-length lists only: idx holds ONE list per layer
+                                    ([n_layers, k_fixed]) and every step uses the list of its layer -- the paper's
+                                    decode, where the set chosen during prefill stays fixed for the prompt */
     SI_FLAG_SIMPLE_KERNELS = 256u /* decode: one plain-load kernel pair per step instead of the
                                      persistent bulk-copy kernel (kept for cross-checking) */
 };
@@ -183,7 +186,9 @@ int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, c
  * (or CSR over n_steps lists).  Steps are executed strictly in order; the weight
  * stream of later steps is prefetched while earlier steps finish.  Results equal
  * n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of a list
- * over SMs depends on the step's position in the call); each is run-to-run bit-stable. */
+ * over SMs depends on the step's position in the call); each is run-to-run bit-stable.
+ * With SI_FLAG_LIST_PER_LAYER (fixed-length lists only) idx is [n_layers, k_fixed] and a step
+ * uses the list of its layer: the set chosen during prefill serves every token of the prompt. */
 int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
                             const void *x, const int32_t *idx, const int32_t *idx_offsets,
                             int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
@@ -278,6 +283,13 @@ int si_debug_decode_stream_only(int on);
  * with no other work reaches on this GPU, the practical ceiling quoted beside the decode kernel.  The
  * paper has no counterpart. */
 int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream);
+
+/* Layer policy of Table 1 ("first layer" f, "last layer" l, l <= 0 counted from the end): the layers
+ * that run selectively are first_out .. last_out - 1 = f .. n_layers + l - 1 (0-based); the others
+ * keep their whole FFN.  With f = 5, l = -2 this gives 9 of 16 and 21 of 28 layers, the counts the
+ * paper's evaluation states.  Host function; returns SI_ERR_INVALID_ARG if the range is empty or
+ * outside the model. */
+int si_layer_range(int n_layers, int first, int last, int *first_out, int *last_out);
 
 /* Library build information: "sm_100a" etc.  Never NULL. */
 const char *si_build_info(void);

@@ -25,6 +25,7 @@ SI_ERR_TOO_LARGE = -9
 SI_FLAG_CHECK, SI_FLAG_RESIDUAL, SI_FLAG_UNION_UNMASKED, SI_FLAG_SCORE_ABS = 1, 2, 4, 8
 SI_FLAG_SHARED_LIST = 16
 SI_FLAG_UNION_PATH = 32
+SI_FLAG_LIST_PER_LAYER = 64
 SI_FLAG_SIMPLE_KERNELS = 256
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 
@@ -33,7 +34,7 @@ EXPORTS = [
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward",
+    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range",
 ]
 
 
@@ -75,6 +76,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
     lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
     lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
+    lib.si_layer_range.argtypes = [ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.si_prefill_forward.argtypes = [vp, ci, vp, ci, vp, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -182,6 +184,13 @@ def si_select(scores, mode: int, k: int, tau: float, flags: int, idx_out, n_out,
                           _dp(n_out), _dp(workspace),
                           0 if workspace is None else workspace.numel() * workspace.element_size(),
                           _stream(stream)), "si_select")
+
+
+def si_layer_range(n_layers: int, first: int = 5, last: int = -2):
+    """Selective layers of Table 1's policy as a half-open range (first, end)."""
+    lo, hi = ctypes.c_int(0), ctypes.c_int(0)
+    _check(_lib.si_layer_range(n_layers, first, last, ctypes.byref(lo), ctypes.byref(hi)), "si_layer_range")
+    return lo.value, hi.value
 
 
 def si_prefill_vote_workspace_bytes(T: int, n: int, alpha: int) -> int:

@@ -130,6 +130,7 @@ extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, con
         min_loaded = min_loaded < store->n_loaded[l] ? min_loaded : store->n_loaded[l];
     }
     if (!idx_offsets && k_fixed > min_loaded) return SI_ERR_OUT_OF_RANGE;
+    if ((flags & SI_FLAG_LIST_PER_LAYER) && idx_offsets) return SI_ERR_INVALID_ARG;   // per-layer lists have one fixed length
     cudaStream_t stream = (cudaStream_t)stream_;
     si_ws_layout ws = si_ws_carve(store, 1, k_fixed, n_steps);
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
@@ -140,8 +141,15 @@ extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, con
             SI_CUDA_TRY(cudaMemcpyAsync(dst, layers, (size_t)n_steps * 4, cudaMemcpyHostToDevice, stream));
             layers_dev = dst;
         }
-        rc = si_check_lists_launch_impl(store, n_steps, -1, layers_dev, idx, idx_offsets, k_fixed, status_dev, stream);
-        if (rc) return rc;
+        if ((flags & SI_FLAG_LIST_PER_LAYER) && !idx_offsets) {     // one list per layer: check list l against layer l
+            for (int l = 0; l < store->n_layers; ++l) {
+                rc = si_check_lists_launch_impl(store, 1, l, nullptr, idx + (size_t)l * k_fixed, nullptr, k_fixed, status_dev, stream);
+                if (rc) return rc;
+            }
+        } else {
+            rc = si_check_lists_launch_impl(store, n_steps, -1, layers_dev, idx, idx_offsets, k_fixed, status_dev, stream);
+            if (rc) return rc;
+        }
     }
     return si_decode_launch(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
                             ws_bytes, status_dev, stream);

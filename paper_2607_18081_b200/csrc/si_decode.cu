@@ -238,11 +238,12 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
     if ((size_t)max_ctas > rows) max_ctas = (int)rows;
     for (int st = 0; st < n_steps; ++st) {
         int l = layers_host ? layers_host[st] : st % s->n_layers;
+        const int list = ((flags & SI_FLAG_LIST_PER_LAYER) && !idx_offsets) ? l : st;   // which list the step uses
         const void *xs = (const char *)x + (size_t)st * s->d_model * esz;
         void *ys = (char *)y + (size_t)st * s->d_model * ysz;
         int rc = (s->dtype == SI_BF16)
-                     ? launch_simple_step<SI_BF16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream)
-                     : launch_simple_step<SI_F16>(s, l, xs, idx, idx_offsets, st, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream);
+                     ? launch_simple_step<SI_BF16>(s, l, xs, idx, idx_offsets, list, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream)
+                     : launch_simple_step<SI_F16>(s, l, xs, idx, idx_offsets, list, k_fixed, ys, y_dtype, flags, partial, max_ctas, status_dev, stream);
         if (rc != SI_OK) return rc;
     }
     return SI_OK;

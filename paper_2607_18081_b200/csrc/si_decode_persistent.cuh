@@ -63,6 +63,7 @@ struct Params {
     const int32_t *idx_offsets;   // CSR [n_steps + 1] or nullptr
     void *y;
     int y_f32, residual;
+    int per_layer_lists;          // fixed-length lists only: idx is [n_layers][k_fixed], a step uses the list of its layer
     float *partial;               // [D][G][d_model]
     unsigned int *ctrl;           // [1] abort flag (zero at launch)
     unsigned int *counters;       // [n_steps][kCounterStride], zero at launch: +0 "written" = CTAs that
@@ -336,7 +337,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         pf_src = (unsigned long long)(P.x + (size_t)step * d);
                         pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
                     } else {
-                        const int slot = __ldg(P.idx + g.base + g.first + (long long)(t - 1) * Gv);
+                        const int lbase = P.per_layer_lists ? layer * P.k_fixed : g.base;
+                        const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - 1) * Gv);
                         const bool valid = slot >= 0 && slot < P.n_loaded[layer];
                         pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
                         pf_bytes = valid ? (uint32_t)rec_bytes : 0u; pf_meta = valid ? 1 : 0;
@@ -810,6 +812,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.counters = P.ctrl + 64;
     P.x = (const uint16_t *)x; P.idx = idx; P.idx_offsets = idx_offsets; P.y = y;
     P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
+    P.per_layer_lists = (flags & SI_FLAG_LIST_PER_LAYER) != 0 && !idx_offsets;
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
     P.prof = si_decode_profile_buffer();

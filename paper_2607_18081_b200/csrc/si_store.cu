@@ -227,6 +227,15 @@ extern "C" int si_store_records(const si_store_t *store, int layer, const void *
     return SI_OK;
 }
 
+extern "C" int si_layer_range(int n_layers, int first, int last, int *first_out, int *last_out) {
+    if (!first_out || !last_out || n_layers <= 0 || first < 0 || last > 0) return SI_ERR_INVALID_ARG;
+    const int end = n_layers + last;          // one past the last selective layer
+    if (first >= end || end > n_layers) return SI_ERR_INVALID_ARG;
+    *first_out = first;
+    *last_out = end;
+    return SI_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Diagnostics: read-only streaming kernel (bandwidth ceiling of plain loads).
 namespace {

@@ -60,3 +60,20 @@ def test_store_bytes_is_eq2_accounting():
     full = L * 3 * d * F * 2
     saving = so.memory_saving(L * 3 * d * F, n_ld / F, 1.0, 2)
     assert abs((full - records) - saving) < 1e-6 * full
+
+
+def test_layer_range_matches_the_papers_layer_counts():
+    """Host-only entry point: Table 1's layer policy gives the layer counts of the paper's evaluation."""
+    from oracle import selectinfer_oracle as so
+    from paper_2607_18081_b200 import api
+    from tests.helpers import paper_values
+    pv = paper_values()
+    first, last = int(pv["table1_first_layer"]), int(pv["table1_last_layer"])
+    for n_layers in (int(pv["llama32_1b_layers"]), int(pv["llama32_3b_layers"]), 32):
+        lo, hi = api.si_layer_range(n_layers, first, last)
+        assert list(range(lo, hi)) == so.layer_range(n_layers, first, last)
+    lo, hi = api.si_layer_range(int(pv["llama32_1b_layers"]), first, last)
+    assert hi - lo == pv["llama32_1b_selective_layers"]
+    import pytest
+    with pytest.raises(api.SelectInferError):
+        api.si_layer_range(6, 5, -2)

@@ -162,6 +162,44 @@ def test_ragged_csr_lists_over_a_stack(api, flags_name):
             assert_close(from_dev(y[s]), ref, f"step {s}")
 
 
+@pytest.mark.parametrize("flags_name", ["persistent", "simple"])
+def test_stack_with_one_list_per_layer(api, flags_name):
+    """The paper's decode: the set chosen for a layer stays fixed for the prompt, so the stack call takes
+    one list per layer.  Results equal the same call with the list repeated for every step, bit for bit."""
+    cfg = _tiny_cfg("bf16", d_model=256, d_ff=400, loaded_pct=60)
+    m = LoadedModel(cfg)
+    base = api.SI_FLAG_SIMPLE_KERNELS if flags_name == "simple" else 0
+    L, tokens, n = m.L, 5, cfg.n_loaded
+    k = n // 3
+    g = np.random.default_rng(12)
+    lists = np.stack([np.sort(g.permutation(n)[:k]).astype(np.int32) for _ in range(L)])     # [L, k]
+    n_steps = tokens * L
+    x = np.stack([wl.x_tokens(cfg, s % L, 1, first_token=s // L)[0] for s in range(n_steps)])
+    xd = to_dev(x, cfg.dtype)
+    ws = m.store.workspace(1, k, n_steps)
+    y1 = torch.empty(n_steps, cfg.d_model, dtype=torch.float32, device="cuda")
+    y2 = torch.empty_like(y1)
+    st = _status()
+    api.si_decode_stack_forward(m.store.handle, n_steps, None, xd, torch.from_numpy(lists).cuda(), None, k, y1,
+                                base | api.SI_FLAG_LIST_PER_LAYER | api.SI_FLAG_CHECK, ws, st)
+    per_step = np.stack([lists[s % L] for s in range(n_steps)])
+    api.si_decode_stack_forward(m.store.handle, n_steps, None, xd, torch.from_numpy(per_step).cuda(), None, k, y2,
+                                base, ws, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert torch.equal(y1, y2)
+    for s in (0, 1, L, n_steps - 1):
+        assert_close(from_dev(y1[s]), m.oracle_y(s % L, x[s], lists[s % L]), f"step {s}")
+    # custom layer order
+    order = [1, 0, 1, 1, 0]
+    y3 = torch.empty(len(order), cfg.d_model, dtype=torch.float32, device="cuda")
+    api.si_decode_stack_forward(m.store.handle, len(order), order, xd[: len(order)], torch.from_numpy(lists).cuda(),
+                                None, k, y3, base | api.SI_FLAG_LIST_PER_LAYER, ws, st)
+    torch.cuda.synchronize()
+    for s, l in enumerate(order):
+        assert_close(from_dev(y3[s]), m.oracle_y(l, x[s], lists[l]), f"ordered step {s}")
+
+
 def test_7b_shaped_two_layers_stack_and_determinism(api):
     """Llama-2-7B FFN shape (d_model 4096, d_ff 11008, bf16), 2 layers x 3 tokens: spans many
     SMs, several ring passes and a ragged tail of records per SM."""
