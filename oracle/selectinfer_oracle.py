@@ -17,6 +17,8 @@ cpu_baseline / reference legs may import this module.
 * ``prefill_vote`` -- Section 5: per-token top alpha, frequency count over the prompt's tokens,
   top beta by frequency, merge with the static prefix up to phi.
 * ``union`` -- sorted set union of per-token lists plus per-token membership bitmasks.
+* ``profile_scores`` / ``merge_scores`` / ``ranking`` -- Section 3, Eq. 1: per-neuron sums of absolute
+  activations, merged over score files after normalising by token count, ranked by importance.
 * ``loadset`` -- Section 4: base = top delta of the task ranking, then the model
   ranking in order, skipping ids already chosen, until gamma neurons are loaded.
 * ``memory_saving`` -- Eq. 2.
@@ -245,6 +247,36 @@ def loadset(task_rank, model_rank, n_base: int, n_loaded: int) -> np.ndarray:
     if len(out) != n_loaded:
         raise ValueError("rankings too short for n_loaded")
     return np.array(out, dtype=np.int32)
+
+
+def profile_scores(acts, scores=None) -> np.ndarray:
+    """Eq. 1: s_n = sum over the processed tokens t of |a_n(t)|.  acts: [T, n] float32 activations;
+    scores: running float64 totals of earlier prompts (added to, tokens in order) or None."""
+    a = np.asarray(acts, dtype=np.float32)
+    out = np.zeros(a.shape[1], dtype=np.float64) if scores is None else np.array(scores, dtype=np.float64)
+    for t in range(a.shape[0]):                  # token by token, in order
+        out += np.abs(a[t]).astype(np.float64)
+    return out
+
+
+def merge_scores(files) -> np.ndarray:
+    """Section 3: score files are merged by normalising each file's scores by its token count and
+    summing the normalised values.  files: sequence of (scores float64 [n], tokens), added in order."""
+    merged = None
+    for scores, tokens in files:
+        if tokens <= 0:
+            raise ValueError("token count must be positive")
+        part = np.asarray(scores, dtype=np.float64) / float(tokens)
+        merged = part if merged is None else merged + part
+    return merged
+
+
+def ranking(scores) -> np.ndarray:
+    """Section 3: neuron indices in decreasing order of importance (ties: lower index first; NaN last)."""
+    s = np.asarray(scores, dtype=np.float64)
+    key = [(1 if v != v else 0, 0.0 if v != v else -v, i) for i, v in enumerate(s.tolist())]
+    key.sort()
+    return np.array([i for _, _, i in key], dtype=np.int32)
 
 
 def memory_saving(n_ffn_params: float, r_load: float, r_layer: float, bytes_per_param: float):

@@ -330,3 +330,33 @@ def test_prefill_vote_special_cases_and_invariants():
             top_beta = sorted(range(n), key=lambda i: (-int(counts[i]), i))[:beta]
             left_out = [i for i in top_beta if i >= n_static and i not in dyn and counts[i] > 0]
             assert all((counts[i], -i) < worst for i in left_out)
+
+
+# --------------------------------------------------------------------------- profiler (Section 3, Eq. 1)
+
+def test_profiler_scores_merge_and_ranking():
+    """Eq. 1 on a hand-worked case, additivity over prompts, the merge rule and the ranking's tie-break."""
+    a = np.array([[1.0, -2.0, 0.5, 0.0], [-3.0, 2.0, 0.5, -0.0], [0.25, 0.0, -0.5, 0.0]], dtype=np.float32)
+    s = so.profile_scores(a)
+    assert s.tolist() == [4.25, 4.0, 1.5, 0.0]                       # column sums of |a|
+    # scoring a prompt in two pieces gives the same totals as scoring it at once (same order of additions)
+    assert np.array_equal(so.profile_scores(a[2:], so.profile_scores(a[:2])), s)
+    # Eq. 1 against a library evaluation on random data
+    g = np.random.default_rng(3)
+    b = g.standard_normal((57, 33)).astype(np.float32)
+    assert np.allclose(so.profile_scores(b), np.abs(b.astype(np.float64)).sum(axis=0), rtol=1e-14, atol=0)
+    # merge: normalise by token count, then sum -- a file with twice the tokens and twice the scores counts the same
+    f1, f2 = (np.array([4.0, 2.0, 0.0]), 2), (np.array([8.0, 4.0, 0.0]), 4)
+    assert so.merge_scores([f1]).tolist() == [2.0, 1.0, 0.0]
+    assert so.merge_scores([f1, f2]).tolist() == [4.0, 2.0, 0.0]
+    with pytest.raises(ValueError):
+        so.merge_scores([(np.ones(3), 0)])
+    # ranking: decreasing score, ties to the lower index, NaN last
+    assert so.ranking(np.array([1.0, 3.0, 3.0, np.nan, 0.0, 7.0])).tolist() == [5, 1, 2, 0, 4, 3]
+    r = so.ranking(so.merge_scores([(so.profile_scores(b), 57)]))
+    m = so.profile_scores(b)
+    assert sorted(r.tolist()) == list(range(33)) and all(m[r[i]] >= m[r[i + 1]] for i in range(32))
+    # ranking feeds the load set of Section 4: base neurons from the task ranking come first
+    task, model = so.ranking(so.profile_scores(b[:20])), r
+    ids = so.loadset(task, model, 5, 12)
+    assert ids[:5].tolist() == task[:5].tolist() and len(set(ids.tolist())) == 12
