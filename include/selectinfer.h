@@ -284,6 +284,33 @@ int si_debug_decode_stream_only(int on);
  * paper has no counterpart. */
 int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream);
 
+/* ---------------------------------------------------------------- offline: profiler and load set
+ *
+ * Section 3 (Eq. 1): the score of a neuron is the sum, over the tokens processed during profiling, of
+ * the absolute value of its activation (the input of the down projection).  Scores and token counts
+ * go to score files; files are merged by dividing each file's scores by its token count and summing;
+ * the outcome is the list of neuron indices in decreasing order of importance.  Section 4: the
+ * neurons to load are the top n_base of a task ranking (base neurons), then the model ranking in
+ * order, neurons already chosen skipped, until n_loaded neurons (secondary neurons).
+ *
+ *   si_profile_accumulate  scores[i] += sum_t |acts[t, i]| (device float64 [n], caller zeroes it for a
+ *                          new file; tokens are added in order, so totals are bit-reproducible).  The
+ *                          activations of all d_ff neurons of a layer come from si_prefill_forward's
+ *                          acts_out on a store that holds every neuron.
+ *   si_profile_merge       merged[i] += scores[i] / tokens   (device float64 [n]; files in call order)
+ *   si_profile_rank        ranking (device int32 [n]) = indices by decreasing score, ties to the lower
+ *                          index, NaN last
+ *   si_loadset             ids_out (device int32 [n_loaded]) from two rankings over n neurons;
+ *                          workspace: ceil(n / 32) * 4 bytes; *status_dev (optional) receives
+ *                          SI_ERR_OUT_OF_RANGE / SI_ERR_DUPLICATE for a malformed ranking and
+ *                          SI_ERR_INVALID_ARG if the rankings do not yield n_loaded distinct neurons
+ * All asynchronous on stream; all decisions and sums are exact and ordered, hence unique. */
+int si_profile_accumulate(const float *acts, int T, int n, int row_stride, double *scores, void *stream);
+int si_profile_merge(double *merged, const double *scores, long long tokens, int n, void *stream);
+int si_profile_rank(const double *scores, int n, int32_t *ranking, void *stream);
+int si_loadset(const int32_t *task_rank, const int32_t *model_rank, int n, int n_base, int n_loaded,
+               int32_t *ids_out, void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream);
+
 /* Layer policy of Table 1 ("first layer" f, "last layer" l, l <= 0 counted from the end): the layers
  * that run selectively are first_out .. last_out - 1 = f .. n_layers + l - 1 (0-based); the others
  * keep their whole FFN.  With f = 5, l = -2 this gives 9 of 16 and 21 of 28 layers, the counts the

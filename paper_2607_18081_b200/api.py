@@ -34,7 +34,8 @@ EXPORTS = [
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range",
+    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
+    "si_loadset",
 ]
 
 
@@ -76,6 +77,10 @@ def _load_library() -> ctypes.CDLL:
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
     lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
     lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
+    lib.si_profile_accumulate.argtypes = [vp, ci, ci, ci, vp, vp]
+    lib.si_profile_merge.argtypes = [vp, vp, ctypes.c_longlong, ci, vp]
+    lib.si_profile_rank.argtypes = [vp, ci, vp, vp]
+    lib.si_loadset.argtypes = [vp, vp, ci, ci, ci, vp, vp, sz, vp, vp]
     lib.si_layer_range.argtypes = [ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.si_prefill_forward.argtypes = [vp, ci, vp, ci, vp, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in EXPORTS:
@@ -184,6 +189,25 @@ def si_select(scores, mode: int, k: int, tau: float, flags: int, idx_out, n_out,
                           _dp(n_out), _dp(workspace),
                           0 if workspace is None else workspace.numel() * workspace.element_size(),
                           _stream(stream)), "si_select")
+
+
+def si_profile_accumulate(acts, scores, stream=None) -> None:
+    T, n = acts.shape
+    _check(_lib.si_profile_accumulate(_dp(acts), T, n, acts.stride(0), _dp(scores), _stream(stream)), "si_profile_accumulate")
+
+
+def si_profile_merge(merged, scores, tokens: int, stream=None) -> None:
+    _check(_lib.si_profile_merge(_dp(merged), _dp(scores), tokens, scores.numel(), _stream(stream)), "si_profile_merge")
+
+
+def si_profile_rank(scores, ranking, stream=None) -> None:
+    _check(_lib.si_profile_rank(_dp(scores), scores.numel(), _dp(ranking), _stream(stream)), "si_profile_rank")
+
+
+def si_loadset(task_rank, model_rank, n_base: int, ids_out, workspace, status=None, stream=None) -> None:
+    _check(_lib.si_loadset(_dp(task_rank), _dp(model_rank), task_rank.numel(), n_base, ids_out.numel(), _dp(ids_out),
+                           _dp(workspace), workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)),
+           "si_loadset")
 
 
 def si_layer_range(n_layers: int, first: int = 5, last: int = -2):
