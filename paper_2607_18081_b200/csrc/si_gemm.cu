@@ -19,6 +19,8 @@
 // machine.  The finishing passes (combine, split reduction) have no kernels of their own: an
 // unsplit tile is finished in the contraction's epilogue, a split tile by the CTA that delivers
 // its last fp32 partial, which sums the partials in split order -- so results are deterministic.
+#include <cuda.h>       // CUtensorMap and the encode function's signature only; the function is looked up at run time
+
 #include "si_common.cuh"
 
 namespace {
@@ -56,10 +58,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
 }
-// 16-byte copy that reads src_bytes (0 or 16) bytes and zero-fills the rest
-__device__ __forceinline__ void cp_async16_zfill(void *dst_smem, const void *src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst_smem)), "l"(src), "r"(src_bytes) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -80,6 +78,16 @@ __device__ __forceinline__ void cp_async_wait_dyn(int n) {
 // are no-ops in launches without the attribute.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// TMA: one 2-D tile of a dense 16-bit matrix (box = 64 columns x box rows, 128-byte swizzle) into shared
+// memory; x = first column (a multiple of 64, i.e. of 128 bytes), y = first row; rows past the matrix
+// read as zero.  Completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void tma_load_tile(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst_smem)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -229,7 +237,7 @@ struct GemmParams {
 // tensor memory (columns [0,N) gate, [N,2N) up).
 __global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
 
-si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
+si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
     const int stage_bytes = 2 * 128 * 128 + N * 128;              // gate tile, up tile, x tile
@@ -244,7 +252,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
     // ---- set-up that needs nothing from the union kernel (runs while that kernel finishes)
     uint32_t ncols = 32; while (ncols < (uint32_t)(2 * N)) ncols <<= 1;
     if (tid == 0) {
-        for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads + 1); mbar_init(&empty[s], 1); }
         mbar_init(accbar, 1);
         *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -290,27 +298,21 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
             grow[j] = P.rec_base + (size_t)P.union_slots[mt * 128 + 32 * j + r32] * P.rec_bytes + q8 * 16 + (size_t)c0 * 128;
         const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);      // rows 32*j + r32 share (row & 7)
         const size_t up_off = (size_t)P.d_model * 2;
-        const char *xsrc = reinterpret_cast<const char *>(P.x) + ((size_t)(tok0 + r32) * P.d_model + (size_t)c0 * kChunkK) * 2 + q8 * 16;
-        const size_t xstride = (size_t)32 * P.d_model * 2;           // 32 token rows further
         int pending = 0;                                             // committed groups not yet signalled
         const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;         // chunks of copies kept in flight
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
-            uint8_t *sg = tiles + (size_t)st * stage_bytes + off0, *su = sg + 128 * 128, *sx = su + 128 * 128;
+            uint8_t *sg = tiles + (size_t)st * stage_bytes + off0, *su = sg + 128 * 128;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 cp_async16(sg + j * 4096, grow[j]);
                 cp_async16(su + j * 4096, grow[j] + up_off);
                 grow[j] += 128;
             }
-            {
-                const char *xs = xsrc;
-                for (int n = r32; n < N; n += 32, xs += xstride) {
-                    const bool in = tok0 + n < P.T;                  // padded token rows are zero-filled
-                    cp_async16_zfill(sx + (n - r32) * 128, in ? xs : reinterpret_cast<const char *>(P.x), in ? 16 : 0);
-                }
-                xsrc += 128;
+            if (tid == 0) {      // the dense X tile comes as one TMA copy (token rows past T read as zero)
+                mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
+                tma_load_tile(tiles + (size_t)st * stage_bytes + 2 * 128 * 128, &x_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
             cp_async_commit();
             ++pending;
@@ -480,7 +482,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P) {
 // down row is contiguous along the output columns), B is K-major.
 __global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
 
-si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
+si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap h_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
     const int stage_bytes = 64 * 256 + N * 128;                   // 64 down-row segments of 128 columns, H tile
@@ -496,7 +498,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
     // ---- set-up that needs nothing from the gate/up kernel (runs while that kernel finishes)
     uint32_t ncols = 32; while (ncols < (uint32_t)N) ncols <<= 1;
     if (tid == 0) {
-        for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < P.nstage; ++s) { mbar_init(&full[s], kLoaderThreads + 1); mbar_init(&empty[s], 1); }
         mbar_init(accbar, 1);
         *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -532,11 +534,6 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
         const int k8 = e16 & 7;
         const int dst0 = (e16 >> 3) * 2048 + (c16 >> 3) * 1024 + k8 * 128 + (((c16 & 7) ^ k8) << 4);
         const char *dsrc0 = P.rec_base + (size_t)P.d_model * 4 + (size_t)mt * 256 + c16 * 16;
-        // H tile: piece (tid & 7) of token rows (tid >> 3) + 32*i
-        const int q8 = tid & 7, r32 = tid >> 3;
-        const int hoff0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);
-        const char *hsrc = reinterpret_cast<const char *>(P.h) + ((size_t)(tok0 + r32) * P.nu_pad + (size_t)c0 * kChunkK) * 2 + q8 * 16;
-        const size_t hstride = (size_t)32 * P.nu_pad * 2;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             int slots[4];
@@ -546,14 +543,13 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P) {
                 if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c0 + c + 1) * kChunkK + 16 * j + e16];
             }
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
-            uint8_t *sa = tiles + (size_t)st * stage_bytes, *sh = sa + 64 * 256 + hoff0;
+            uint8_t *sa = tiles + (size_t)st * stage_bytes;
 #pragma unroll
             for (int j = 0; j < 4; ++j)                                      // padded entries carry a valid slot
                 cp_async16(sa + j * 4096 + dst0, dsrc0 + (size_t)slots[j] * P.rec_bytes);
-            {
-                const char *hs = hsrc;
-                for (int n = r32; n < N; n += 32, hs += hstride) cp_async16(sh + (n - r32) * 128, hs);
-                hsrc += 128;
+            if (tid == 0) {      // the dense H tile comes as one TMA copy
+                mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
+                tma_load_tile(sa + 64 * 256, &h_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
             cp_async_commit();
             ++pending;
@@ -696,14 +692,39 @@ __global__ void si_gemm_reduce_kernel(const float *__restrict__ partial, int n_s
 
 // Launch a contraction kernel so that it may be scheduled while the previous kernel of the stream is
 // still finishing (the kernel itself waits for that kernel's results with pdl_wait()).
-cudaError_t launch_after_predecessor(void (*kern)(GemmParams), dim3 grid, size_t smem, cudaStream_t stream, const GemmParams &P) {
+cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap), dim3 grid, size_t smem, cudaStream_t stream,
+                                     const GemmParams &P, const CUtensorMap &map) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, P);
+    return cudaLaunchKernelEx(&cfg, kern, P, map);
+}
+
+// Tensor map of a dense row-major 16-bit matrix [rows][cols] for tiles of box_rows x 64 columns with the
+// 128-byte swizzle the MMA descriptors expect.  base must be 16-byte aligned, row_bytes a multiple of 16.
+int make_tile_map(CUtensorMap *map, const void *base, size_t cols, size_t rows, size_t row_bytes, int box_rows) {
+    typedef CUresult (*encode_fn_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn_t encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        SI_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (!fn || q != cudaDriverEntryPointSuccess) return SI_ERR_CUDA;
+        encode = (encode_fn_t)fn;
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)kChunkK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SI_OK : SI_ERR_CUDA;
 }
 
 int pick_stages_gemm(size_t stage_bytes, int n_tok) {
@@ -851,7 +872,10 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         dim3 grid(units > target ? units : target);
         P.tok_tiles = tok_tiles; P.target_ctas = target;
         P.tile_ctr = us.ctr;
-        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P));
+        CUtensorMap x_map;
+        int rc = make_tile_map(&x_map, x, (size_t)d, (size_t)T, (size_t)d * 2, n_tok);
+        if (rc) return rc;
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P, x_map));
     }
     // down: split K = union
     int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
@@ -867,7 +891,10 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         dim3 grid(d / 128, s2, tok_tiles);
         P.tile_ctr = us.ctr + n_ctr_gu;
-        SI_CUDA_TRY(launch_after_predecessor(si_gemm_down_kernel, grid, smem, stream, P));
+        CUtensorMap h_map;
+        int rc = make_tile_map(&h_map, wsb + ws.h_off, (size_t)nu_pad, (size_t)t_pad_alloc, (size_t)nu_pad * 2, n_tok);
+        if (rc) return rc;
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_down_kernel, grid, smem, stream, P, h_map));
     }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
