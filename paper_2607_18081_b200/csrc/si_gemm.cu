@@ -237,7 +237,8 @@ struct GemmParams {
 // tensor memory (columns [0,N) gate, [N,2N) up).
 __global__ void __launch_bounds__(320, 2)   // kGemmThreads = 288 threads are launched; 320 caps the registers at 96
 
-si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map) {
+si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map,
+                      const __grid_constant__ CUtensorMap rec_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int N = P.n_tok;
     const int stage_bytes = 2 * 128 * 128 + N * 128;              // gate tile, up tile, x tile
@@ -298,21 +299,32 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
             grow[j] = P.rec_base + (size_t)P.union_slots[mt * 128 + 32 * j + r32] * P.rec_bytes + q8 * 16 + (size_t)c0 * 128;
         const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);      // rows 32*j + r32 share (row & 7)
         const size_t up_off = (size_t)P.d_model * 2;
+        // A tile whose 128 union entries are consecutive slots (a static prefix, a whole layer) needs no
+        // gather: its gate and up tiles are two TMA copies out of the record matrix
+        const int slot_first = P.union_slots[mt * 128];
+        const bool run = P.union_slots[mt * 128 + 127] - slot_first == 127;
         int pending = 0;                                             // committed groups not yet signalled
         const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;         // chunks of copies kept in flight
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
             uint8_t *sg = tiles + (size_t)st * stage_bytes + off0, *su = sg + 128 * 128;
+            if (!run) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                cp_async16(sg + j * 4096, grow[j]);
-                cp_async16(su + j * 4096, grow[j] + up_off);
-                grow[j] += 128;
+                for (int j = 0; j < 4; ++j) {
+                    cp_async16(sg + j * 4096, grow[j]);
+                    cp_async16(su + j * 4096, grow[j] + up_off);
+                    grow[j] += 128;
+                }
             }
             if (tid == 0) {      // the dense X tile comes as one TMA copy (token rows past T read as zero)
-                mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
-                tma_load_tile(tiles + (size_t)st * stage_bytes + 2 * 128 * 128, &x_map, (c0 + c) * kChunkK, tok0, &full[st]);
+                uint8_t *stage = tiles + (size_t)st * stage_bytes;
+                mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u + (run ? 2u * 128u * 128u : 0u));
+                if (run) {
+                    tma_load_tile(stage, &rec_map, (c0 + c) * kChunkK, slot_first, &full[st]);
+                    tma_load_tile(stage + 128 * 128, &rec_map, P.d_model + (c0 + c) * kChunkK, slot_first, &full[st]);
+                }
+                tma_load_tile(stage + 2 * 128 * 128, &x_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
             cp_async_commit();
             ++pending;
@@ -703,6 +715,17 @@ cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap), dim3
     return cudaLaunchKernelEx(&cfg, kern, P, map);
 }
 
+cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap, CUtensorMap), dim3 grid, size_t smem,
+                                     cudaStream_t stream, const GemmParams &P, const CUtensorMap &m0, const CUtensorMap &m1) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, P, m0, m1);
+}
+
 // Tensor map of a dense row-major 16-bit matrix [rows][cols] for tiles of box_rows x 64 columns with the
 // 128-byte swizzle the MMA descriptors expect.  base must be 16-byte aligned, row_bytes a multiple of 16.
 int make_tile_map(CUtensorMap *map, const void *base, size_t cols, size_t rows, size_t row_bytes, int box_rows) {
@@ -872,10 +895,13 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         dim3 grid(units > target ? units : target);
         P.tok_tiles = tok_tiles; P.target_ctas = target;
         P.tile_ctr = us.ctr;
-        CUtensorMap x_map;
+        CUtensorMap x_map, rec_map;
         int rc = make_tile_map(&x_map, x, (size_t)d, (size_t)T, (size_t)d * 2, n_tok);
         if (rc) return rc;
-        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P, x_map));
+        // the layer's records as a matrix [n_loaded][3 * d_model]: 128 consecutive slots x 64 columns per tile
+        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 128);
+        if (rc) return rc;
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P, x_map, rec_map));
     }
     // down: split K = union
     int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
