@@ -37,9 +37,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -58,20 +55,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// wait until at most n of this thread's committed copy groups are still in flight (n <= 5)
-__device__ __forceinline__ void cp_async_wait_dyn(int n) {
-    switch (n) {
-        case 0: cp_async_wait<0>(); break;
-        case 1: cp_async_wait<1>(); break;
-        case 2: cp_async_wait<2>(); break;
-        case 3: cp_async_wait<3>(); break;
-        case 4: cp_async_wait<4>(); break;
-        default: cp_async_wait<5>(); break;
-    }
+// Arrival that fires by itself once all cp.async copies this thread has issued so far have landed: the
+// loader never blocks on its own copies, so every stage can be in flight and the producer side is
+// decoupled from the consumer (counts as one of the barrier's expected arrivals).
+__device__ __forceinline__ void cp_async_arrive_when_landed(uint64_t *bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
 // while its predecessor in the stream still runs; pdl_wait() returns once the predecessor has
 // finished and its writes are visible, pdl_launch() lets the successor start being scheduled.  Both
@@ -303,8 +293,6 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         // gather: its gate and up tiles are two TMA copies out of the record matrix
         const int slot_first = P.union_slots[mt * 128];
         const bool run = P.union_slots[mt * 128 + 127] - slot_first == 127;
-        int pending = 0;                                             // committed groups not yet signalled
-        const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;         // chunks of copies kept in flight
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
@@ -326,26 +314,9 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 }
                 tma_load_tile(stage + 2 * 128 * 128, &x_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
-            cp_async_commit();
-            ++pending;
-            if (pending == la + 1) {     // keep `la` chunks of copies in flight per thread
-                cp_async_wait_dyn(la);
-                fence_async_proxy();
-                mbar_arrive(&full[(c - la) % P.nstage]);
-                --pending;
-            }
+            cp_async_arrive_when_landed(&full[st]);
         }
-        // drain
-        if (!*failed) {
-            const int done = n_chunks;
-            for (; pending > 0; --pending) {
-                cp_async_wait_dyn(pending - 1);
-                fence_async_proxy();
-                mbar_arrive(&full[(done - pending) % P.nstage]);
-            }
-        } else {
-            cp_async_wait<0>();
-        }
+        cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
         // ---------------------------------------------------------------- epilogue
         bool ok = !*failed && mbar_wait(accbar, 0);
         tc_fence_after();
@@ -400,6 +371,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
                 ok = mbar_wait(&full[st], ph) && !*failed;
                 if (!ok) break;
+                fence_async_proxy();               // the gathered rows were written by cp.async (generic proxy)
                 tc_fence_after();
                 const uint32_t sg = smem_u32(tiles + (size_t)st * stage_bytes), su = sg + 128 * 128, sx = su + 128 * 128;
 #pragma unroll
@@ -536,8 +508,6 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         // Copy j of a thread covers 16-byte piece (tid & 15) of the 256-byte down-row segment of union
         // entry 16*j + (tid >> 4) of the chunk: a warp instruction reads two whole segments (coalesced).
         const int c16 = tid & 15, e16 = tid >> 4;
-        int pending = 0;
-        const int la = P.nstage - 1 < 5 ? P.nstage - 1 : 5;
         int slots_next[4];                                           // union slots of the next chunk (prefetched)
 #pragma unroll
         for (int j = 0; j < 4; ++j)
@@ -563,25 +533,9 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
                 tma_load_tile(sa + 64 * 256, &h_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
-            cp_async_commit();
-            ++pending;
-            if (pending == la + 1) {
-                cp_async_wait_dyn(la);
-                fence_async_proxy();
-                mbar_arrive(&full[(c - la) % P.nstage]);
-                --pending;
-            }
+            cp_async_arrive_when_landed(&full[st]);
         }
-        if (!*failed) {
-            const int done = n_chunks;
-            for (; pending > 0; --pending) {
-                cp_async_wait_dyn(pending - 1);
-                fence_async_proxy();
-                mbar_arrive(&full[(done - pending) % P.nstage]);
-            }
-        } else {
-            cp_async_wait<0>();
-        }
+        cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
         bool ok = !*failed && mbar_wait(accbar, 0);
         tc_fence_after();
         // thread holds output column mt*128 + r for the tokens; warps w and w + 4 share the rows and
@@ -626,6 +580,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
                 ok = mbar_wait(&full[st], ph) && !*failed;
                 if (!ok) break;
+                fence_async_proxy();               // the gathered rows were written by cp.async (generic proxy)
                 tc_fence_after();
                 const uint32_t sa = smem_u32(tiles + (size_t)st * stage_bytes), sh = sa + 64 * 256;
 #pragma unroll
