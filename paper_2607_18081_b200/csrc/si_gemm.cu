@@ -707,7 +707,7 @@ int make_tile_map(CUtensorMap *map, const void *base, size_t cols, size_t rows, 
 
 int pick_stages_gemm(size_t stage_bytes, int n_tok) {
     // few tokens: the kernels are latency-bound gathers, two CTAs per SM hide more of it
-    size_t budget = n_tok <= 64 ? 112 * 1024 : 200 * 1024;
+    size_t budget = n_tok <= 16 ? 112 * 1024 : 200 * 1024;
     int n = (int)(budget / stage_bytes);
     return n > kMaxStages ? kMaxStages : n;
 }
@@ -833,7 +833,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     // gate/up: K = d_model may be split up to s1 ways (what the partial buffer holds); the kernel
     // picks the split from the real union size so that one wave of CTAs covers the SM slots (two CTAs
     // per SM with few tokens: the gathers are latency-bound)
-    const int target = (t_pad_alloc <= 64 ? 2 : 1) * s->num_sms;
+    const int target = (t_pad_alloc <= 16 ? 2 : 1) * s->num_sms;
     const int k_chunks = d / kChunkK;
     int s1 = k_chunks < 8 ? k_chunks : 8;
     const size_t part_cap = kPartialCap < ws.partial_bytes ? kPartialCap : ws.partial_bytes;
@@ -859,7 +859,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P, x_map, rec_map));
     }
     // down: split K = union
-    int s2 = (t_pad_alloc <= 64 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
+    int s2 = (t_pad_alloc <= 16 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
     if (s2 < 1) s2 = 1;
     if (s2 > 8) s2 = 8;
     if (s2 > nu_pad / kChunkK) s2 = nu_pad / kChunkK;
