@@ -255,7 +255,7 @@ int si_prefill_vote(const float *acts, int T, int n, int row_stride, int alpha, 
  *              SI_FLAG_SCORE_ABS
  *   idx_out, cap, n_out, alpha, beta, n_static, phi_count: as for si_prefill_vote
  *   acts_out   optional device float32 [T, n_loaded]: receives the activations that were ranked
- *   workspace  si_workspace_bytes(store, T, n_loaded, 1) bytes; vote_workspace
+ *   workspace  si_workspace_bytes(store, max(T, 2), n_loaded, 1) bytes; vote_workspace
  *              si_prefill_vote_workspace_bytes(T, n_loaded, alpha) bytes, both 256-byte aligned
  * Asynchronous on stream. */
 int si_prefill_forward(const si_store_t *store, int layer, const void *x, int T, void *y, int y_dtype,

@@ -198,7 +198,7 @@ extern "C" int si_prefill_forward(const si_store_t *store, int layer, const void
     if (!si_aligned16(idx_out) || (((uintptr_t)vote_workspace) & 255u) || (acts_out && !si_aligned16(acts_out)))
         return SI_ERR_ALIGNMENT;
     cudaStream_t stream = (cudaStream_t)stream_;
-    const si_ws_layout ws = si_ws_carve(store, T, n, 1);
+    const si_ws_layout ws = si_ws_carve(store, T < 2 ? 2 : T, n, 1);      // the multi-token regions exist from T_max = 2 on
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
     char *wsb = (char *)workspace;
     // one shared list: every loaded slot, so the union is the store in slot order (position p = slot p)

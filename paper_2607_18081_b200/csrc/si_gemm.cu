@@ -769,7 +769,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
                           void *workspace, size_t ws_bytes, int32_t *status_dev, cudaStream_t stream) {
     const int d = s->d_model;
     if (d % 128 != 0) return SI_ERR_UNSUPPORTED;
-    si_ws_layout ws = si_ws_carve(s, T, k_fixed, 1);
+    si_ws_layout ws = si_ws_carve(s, T < 2 ? 2 : T, k_fixed, 1);       // the multi-token regions exist from T_max = 2 on
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
     char *wsb = (char *)workspace;
     const int n_loaded = s->n_loaded[layer];

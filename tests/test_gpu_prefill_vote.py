@@ -123,3 +123,33 @@ def test_prefill_forward_outputs_activations_and_vote(api, cfg_name, T):
     got = set(idx[:k].cpu().numpy().tolist())
     inter = len(got & set(ref.tolist()))
     assert k == len(ref) and inter >= 0.97 * len(ref), (k, len(ref), inter)
+
+
+@pytest.mark.parametrize("T", [1, 3, 129])
+def test_prefill_forward_short_and_odd_prompts(api, T):
+    """A one-token prompt, an odd handful, and one token past a 128-wide token tile."""
+    from tests.gpu_utils import LoadedModel, assert_close, from_dev, to_dev
+    cfg = wl.CONFIGS["c1"]
+    m = LoadedModel(cfg, n_layers=1)
+    n, d = cfg.n_loaded, cfg.d_model
+    x = wl.x_tokens(cfg, 0, T)
+    y = torch.empty(T, d, dtype=torch.float16, device="cuda")
+    idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(4, dtype=torch.int32, device="cuda")
+    acts = torch.empty(T, n, dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = m.store.workspace(max(T, 2), n, 1)
+    vws = _aligned(api.si_prefill_vote_workspace_bytes(T, n, 50))
+    api.si_prefill_forward(m.store.handle, 0, to_dev(x, cfg.dtype), T, y, 50, 200, 100, 250, api.SI_FLAG_SCORE_ABS,
+                           idx, cnt, acts, ws, vws, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    for t in sorted({0, T - 1}):
+        assert_close(from_dev(y[t]), m.oracle_y(0, x[t], np.arange(n)), f"T={T} token {t}")
+    k = int(cnt[0].item())
+    got = idx[:k].cpu().numpy()
+    assert 100 <= k <= 250 and np.array_equal(got[:100], np.arange(100)) and np.all(np.diff(got) > 0)
+    # with one token every candidate occurs exactly once: the dynamic part is a subset of that token's top alpha
+    if T == 1:
+        top = so.select_topk(acts[0].cpu().numpy(), 50, use_abs=True)
+        assert set(got[100:].tolist()) <= set(top.tolist())
