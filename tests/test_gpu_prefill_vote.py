@@ -151,5 +151,6 @@ def test_prefill_forward_short_and_odd_prompts(api, T):
     assert 100 <= k <= 250 and np.array_equal(got[:100], np.arange(100)) and np.all(np.diff(got) > 0)
     # with one token every candidate occurs exactly once: the dynamic part is a subset of that token's top alpha
     if T == 1:
-        top = so.select_topk(acts[0].cpu().numpy(), 50, use_abs=True)
+        a = np.abs(acts[0].cpu().numpy())
+        top = np.argsort(-a, kind="stable")[:50]          # the exported activations, ranked by a library sort
         assert set(got[100:].tolist()) <= set(top.tolist())
