@@ -69,6 +69,7 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
                          const int32_t *__restrict__ offsets, int list, int k_fixed,
                          float *__restrict__ partial, int32_t *status) {
     __shared__ float red[2][kThreads / 32][4];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the reduce kernel may be scheduled already
     const int base = offsets ? offsets[list] : list * k_fixed;
     const int k = offsets ? offsets[list + 1] - base : k_fixed;
     idx += base;
@@ -151,6 +152,7 @@ si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
                         const uint16_t *__restrict__ x, void *__restrict__ y,
                         int y_f32, int residual) {
     __shared__ float4 part[32][8];
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // the partial rows of the preceding kernel
     const int g = threadIdx.x & 7, rc = threadIdx.x >> 3;
     const int col = (blockIdx.x * 8 + g) * 4;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -202,8 +204,18 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
-    si_decode_reduce_kernel<DT><<<(d + 31) / 32, 256, 0, stream>>>(
-        partial, G, d, (const uint16_t *)x, y, y_dtype == SI_F32, (flags & SI_FLAG_RESIDUAL) != 0);
+    {
+        // programmatic dependent launch: the reduce kernel is scheduled while the partial kernel finishes
+        // and waits for its rows with griddepcontrol.wait
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((d + 31) / 32); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_reduce_kernel<DT>, (const float *)partial, G, d, (const uint16_t *)x, y,
+                                       (int)(y_dtype == SI_F32), (int)((flags & SI_FLAG_RESIDUAL) != 0)));
+    }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }
