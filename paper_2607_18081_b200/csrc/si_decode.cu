@@ -142,6 +142,103 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
     }
 }
 
+// The same walk for rows of at most 512 chunks (d_model <= 4096), one record at a time with the loads of
+// the next P records already in flight: the records a CTA owns are independent, so nothing but registers
+// limits how far ahead their loads may run.  The list entry of the record after those is fetched one
+// record early, so that no address waits for it.  Sums are taken in the order of the kernel above.
+template <int DT, int NCH, int P>
+__global__ void __launch_bounds__(kThreads, kSimpleCtasPerSm)
+si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks,
+                               const uint4 *__restrict__ x, const int32_t *__restrict__ idx,
+                               const int32_t *__restrict__ offsets, int list, int k_fixed,
+                               float *__restrict__ partial, int32_t *status) {
+    __shared__ float red[2][kThreads / 32][2];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int base = offsets ? offsets[list] : list * k_fixed;
+    const int k = offsets ? offsets[list + 1] - base : k_fixed;
+    idx += base;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = gridDim.x;
+    const int n_mine = k > (int)blockIdx.x ? (k - (int)blockIdx.x + G - 1) / G : 0;   // records of this CTA
+    const int32_t *my = idx + blockIdx.x;
+    int first[P];
+#pragma unroll
+    for (int st = 0; st < P; ++st) first[st] = st < n_mine ? my[(size_t)st * G] : 0;
+    int ahead = P < n_mine ? my[(size_t)P * G] : 0;              // list entry of record j + P
+    uint4 xp[NCH];
+    float acc[NCH][8];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int c = tid + kThreads * i;
+        xp[i] = c < chunks ? __ldg(x + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[i][e] = 0.f;
+    }
+    uint4 buf[P][3 * NCH];
+    bool ok[P];
+    auto fetch = [&](uint4 (&b)[3 * NCH], bool &good, int slot) {
+        good = slot >= 0 && slot < n_loaded;
+        if (!good && tid == 0 && status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE);
+        const uint4 *r = rec + (size_t)(good ? slot : 0) * 3 * chunks;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int c = tid + kThreads * i;
+            if (c < chunks) {
+                b[3 * i] = __ldg(r + c); b[3 * i + 1] = __ldg(r + chunks + c); b[3 * i + 2] = __ldg(r + 2 * chunks + c);
+            } else {
+                b[3 * i] = b[3 * i + 1] = b[3 * i + 2] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+#pragma unroll
+    for (int st = 0; st < P; ++st) {
+        ok[st] = false;
+        if (st < n_mine) fetch(buf[st], ok[st], first[st]);
+    }
+    for (int j0 = 0; j0 < n_mine; j0 += P) {
+#pragma unroll
+        for (int st = 0; st < P; ++st) {
+            const int j = j0 + st;
+            if (j < n_mine) {                                      // uniform over the CTA
+                float g = 0.f, u = 0.f;
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    float xr[8];
+                    unpack8<DT>(xp[i], xr);
+                    g += dot8<DT>(buf[st][3 * i], xr); u += dot8<DT>(buf[st][3 * i + 1], xr);
+                }
+                g = warp_sum(g); u = warp_sum(u);
+                float(*rb)[2] = red[j & 1];
+                if (lane == 0) { rb[warp][0] = g; rb[warp][1] = u; }
+                __syncthreads();
+                g = u = 0.f;
+#pragma unroll
+                for (int w = 0; w < kThreads / 32; ++w) { g += rb[w][0]; u += rb[w][1]; }
+                const float h = ok[st] ? si_silu_mul(g, u) : 0.f;
+#pragma unroll
+                for (int i = 0; i < NCH; ++i) {
+                    float f[8];
+                    unpack8<DT>(buf[st][3 * i + 2], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[i][e] = fmaf(h, f[e], acc[i][e]);
+                }
+                const int jn = j + P;
+                if (jn < n_mine) fetch(buf[st], ok[st], ahead);
+                ahead = jn + 1 < n_mine ? my[(size_t)(jn + 1) * G] : 0;
+            }
+        }
+    }
+    float4 *out = reinterpret_cast<float4 *>(partial + (size_t)blockIdx.x * chunks * 8);
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const int c = tid + kThreads * i;
+        if (c < chunks) {
+            out[2 * c] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+            out[2 * c + 1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+        }
+    }
+}
+
 // y[j] = (x[j] +) sum over CTAs g = 0..G-1 of partial[g][j].  One block per 32 output columns (eight
 // float4 groups); thread (group = tid & 7, row class = tid >> 3) sums rows class, class + 32, ... in
 // ascending order -- all its loads are independent -- and the 32 classes are then added in class
@@ -198,12 +295,16 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 #define SI_LAUNCH_PARTIAL(N)                                                                        \
     si_decode_partial_kernel<DT, N><<<G, kThreads, 0, stream>>>(rec, nl, chunks, (const uint4 *)x, \
                                                                 idx, offsets, list, k, partial, status_dev)
-    if (nch <= 1) SI_LAUNCH_PARTIAL(1);
-    else if (nch <= 2) SI_LAUNCH_PARTIAL(2);
+#define SI_LAUNCH_AHEAD(N, P)                                                                             \
+    si_decode_partial_ahead_kernel<DT, N, P><<<G, kThreads, 0, stream>>>(rec, nl, chunks, (const uint4 *)x, \
+                                                                         idx, offsets, list, k, partial, status_dev)
+    if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
+    else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3);
     else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
+#undef SI_LAUNCH_AHEAD
     {
         // programmatic dependent launch: the reduce kernel is scheduled while the partial kernel finishes
         // and waits for its rows with griddepcontrol.wait

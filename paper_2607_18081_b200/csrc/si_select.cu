@@ -2,8 +2,8 @@
 // indices of the top alpha).
 //
 // No sort is needed to obtain the set: one CTA per score row finds the k-th largest value by
-// a 4-pass, 8-bit radix select over order-preserving 32-bit keys held in shared memory, then
-// one index-ordered prefix scan emits the selected indices ascending.  Ties at the k-th
+// a 3-pass radix select (digits of 11, 11 and 10 bits) over order-preserving 32-bit keys held in
+// shared memory, then one index-ordered prefix scan emits the selected indices ascending.  Ties at the k-th
 // value go to the lower indices; +0 == -0; NaN has the lowest key.  All integer decisions:
 // the result is exact and unique.
 #include "si_common.cuh"
@@ -12,6 +12,7 @@ namespace {
 
 constexpr int kSelThreads = 1024;
 constexpr int kSmemKeys = 48 * 1024;   // rows up to this many scores keep their keys in shared memory
+constexpr int kBins = 2048;            // histogram bins: digits of 11, 11 and 10 bits
 
 __device__ __forceinline__ uint32_t score_key(float s, bool use_abs) {
     if (s != s) return 0u;                     // NaN: below everything
@@ -53,8 +54,8 @@ __global__ void __launch_bounds__(kSelThreads)
 si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mode, int k, float tau,
                  int use_abs, int32_t *__restrict__ idx_out, int out_stride, int cap,
                  int32_t *__restrict__ n_out, uint32_t *__restrict__ key_spill, int keys_in_smem) {
-    extern __shared__ uint32_t smem_keys[];
-    __shared__ unsigned int hist[256];
+    extern __shared__ __align__(16) uint32_t smem_keys[];
+    __shared__ __align__(8) unsigned int hist[kBins];
     __shared__ unsigned long long warp_tot[32];
     __shared__ unsigned long long total;
     __shared__ uint32_t sh_prefix, sh_mask;
@@ -67,53 +68,82 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
 
     uint32_t kstar = 0; int r = 0;          // threshold key and how many of its ties to take
     if (mode == SI_SELECT_TOPK) {
-        for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
+        if (((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(keys)) & 15u) == 0) {
+            // all of a thread's 16-byte loads are issued before the first key is formed
+            const float4 *s4 = reinterpret_cast<const float4 *>(s);
+            const int n4 = n >> 2;
+            for (int q0 = 0; q0 < n4; q0 += 4 * kSelThreads) {
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int q = q0 + j * kSelThreads + tid;
+                    v[j] = q < n4 ? __ldg(s4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int q = q0 + j * kSelThreads + tid;
+                    if (q < n4) {
+                        uint4 kk;
+                        kk.x = score_key(v[j].x, use_abs != 0); kk.y = score_key(v[j].y, use_abs != 0);
+                        kk.z = score_key(v[j].z, use_abs != 0); kk.w = score_key(v[j].w, use_abs != 0);
+                        *reinterpret_cast<uint4 *>(keys + 4 * q) = kk;
+                    }
+                }
+            }
+            for (int i = 4 * n4 + tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
+        } else {
+            for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
+        }
         if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
         __syncthreads();
         if (k > 0 && k < n) {
-            for (int shift = 24; shift >= 0; shift -= 8) {
-                if (tid < 256) hist[tid] = 0;
+#pragma unroll 1
+            for (int pass = 0; pass < 3; ++pass) {
+                const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+                const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+                hist[tid] = 0; hist[tid + kSelThreads] = 0;
                 __syncthreads();
                 const uint32_t prefix = sh_prefix, mask = sh_mask;
                 const int need = sh_need;
-                // histogram of the current digit over the keys that still match the prefix.  Scores from
-                // one distribution crowd into a few bins of the high digits, so lanes with the same digit
-                // are merged first and one of them adds their count
-                for (int i0 = 0; i0 < n; i0 += kSelThreads) {
-                    const int i = i0 + tid;
-                    uint32_t digit = 0xFFFFFFFFu;                    // no key / key no longer in play
-                    if (i < n) {
-                        const uint32_t key = keys[i];
-                        if ((key & mask) == prefix) digit = (key >> shift) & 255u;
-                    }
-                    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
-                    if (digit != 0xFFFFFFFFu && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+                // histogram of the current digit over the keys that still match the prefix
+                for (int i = tid; i < n; i += kSelThreads) {
+                    const uint32_t key = keys[i];
+                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
                 }
                 __syncthreads();
-                // find the digit where the count from the largest digit down reaches `need`: thread t
-                // owns bin 255 - t, so a prefix sum over threads is a suffix sum over bins
-                unsigned c = 0, inc = 0;
-                if (tid < 256) {
-                    c = hist[255 - tid];
-                    inc = c;
+                // find the digit where the count from the largest digit down reaches `need`: thread t owns
+                // bins 2047 - 2t and 2046 - 2t, so a prefix sum over threads is a suffix sum over bins
+                const uint2 c2 = reinterpret_cast<const uint2 *>(hist)[kSelThreads - 1 - tid];
+                const unsigned c_hi = c2.y, c_lo = c2.x, pair = c_hi + c_lo;
+                unsigned inc = pair;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if ((tid & 31) >= o) inc += t;
+                }
+                if ((tid & 31) == 31) warp_tot[tid >> 5] = inc;
+                __syncthreads();
+                if (tid < 32) {
+                    const unsigned w = (unsigned)warp_tot[tid];
+                    unsigned winc = w;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
-                        const unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                        if ((tid & 31) >= o) inc += t;
+                        const unsigned t = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+                        if (tid >= o) winc += t;
                     }
-                    if ((tid & 31) == 31) warp_tot[tid >> 5] = inc;
+                    warp_tot[tid] = winc - w;
                 }
                 __syncthreads();
-                if (tid < 256) {
-                    unsigned base = 0;
-                    for (int w = 0; w < (tid >> 5); ++w) base += (unsigned)warp_tot[w];
-                    const unsigned incl = base + inc, excl = incl - c;      // keys in bins >= / > this one
-                    // the keys in play are at least `need`, so exactly one bin satisfies this (bin 0 at the latest)
-                    if (excl < (unsigned)need && (unsigned)need <= incl) {
-                        sh_need = need - (int)excl;
-                        sh_prefix = prefix | ((uint32_t)(255 - tid) << shift);
-                        sh_mask = mask | (255u << shift);
-                    }
+                const unsigned excl = (unsigned)warp_tot[tid >> 5] + inc - pair;    // keys in bins above this pair
+                // the keys in play are at least `need`, so exactly one bin satisfies this (bin 0 at the latest)
+                if (excl < (unsigned)need && (unsigned)need <= excl + c_hi) {
+                    sh_need = need - (int)excl;
+                    sh_prefix = prefix | ((uint32_t)(kBins - 1 - 2 * tid) << shift);
+                    sh_mask = mask | (dmask << shift);
+                } else if (excl + c_hi < (unsigned)need && (unsigned)need <= excl + pair) {
+                    sh_need = need - (int)(excl + c_hi);
+                    sh_prefix = prefix | ((uint32_t)(kBins - 2 - 2 * tid) << shift);
+                    sh_mask = mask | (dmask << shift);
                 }
                 __syncthreads();
             }
@@ -121,18 +151,16 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
         } else if (k >= n) {
             kstar = 0; r = n;                   // everything: all keys >= 0, ties = all
         } else {
-            kstar = 0xFFFFFFFFu; r = 0;         // k == 0: nothing is > max key... guard below
+            kstar = 0xFFFFFFFFu; r = 0;         // k == 0: nothing is taken (guards below)
         }
     }
 
     // index-ordered emission: thread t owns the contiguous range [t*per, (t+1)*per)
     const int per = (n + kSelThreads - 1) / kSelThreads;
-    const int lo = tid * per, hi = min(n, lo + per);
-    unsigned long long mine = 0;   // (hi 32: # strictly above threshold, lo 32: # ties)
-    for (int i = lo; i < hi; ++i) {
-        bool gt, eq;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    auto classify = [&](int i, bool &gt, bool &eq) {
         if (mode == SI_SELECT_TOPK) {
-            uint32_t key = keys[i];
+            const uint32_t key = keys[i];
             gt = (k > 0) && key > kstar; eq = (k > 0) && key == kstar;
             if (k >= n) { gt = false; eq = true; }
         } else {
@@ -140,27 +168,47 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
             if (use_abs) v = fabsf(v);
             gt = v > tau; eq = false;
         }
-        mine += ((unsigned long long)gt << 32) | (unsigned long long)eq;
-    }
-    unsigned long long before = block_exclusive_scan(mine, warp_tot, &total);
-    int gt_before = (int)(before >> 32), eq_before = (int)(before & 0xFFFFFFFFu);
-    for (int i = lo; i < hi; ++i) {
-        bool gt, eq;
-        if (mode == SI_SELECT_TOPK) {
-            uint32_t key = keys[i];
-            gt = (k > 0) && key > kstar; eq = (k > 0) && key == kstar;
-            if (k >= n) { gt = false; eq = true; }
-        } else {
-            float v = s[i];
-            if (use_abs) v = fabsf(v);
-            gt = v > tau; eq = false;
+    };
+    if (per <= 32) {
+        // the range's verdicts fit two 32-bit masks: classify once, then walk the set bits
+        uint32_t gm = 0, em = 0;
+        for (int i = lo; i < hi; ++i) {
+            bool gt, eq;
+            classify(i, gt, eq);
+            gm |= (uint32_t)gt << (i - lo); em |= (uint32_t)eq << (i - lo);
         }
-        bool take = gt || (eq && eq_before < r);
-        if (take) {
-            int pos = gt_before + min(eq_before, r);
-            if (pos < cap) out[pos] = i;
+        const unsigned long long mine = ((unsigned long long)__popc(gm) << 32) | (unsigned long long)__popc(em);
+        const unsigned long long before = block_exclusive_scan(mine, warp_tot, &total);
+        const int gt_before = (int)(before >> 32), eq_before = (int)(before & 0xFFFFFFFFu);
+        int eq_take = r - eq_before;                           // ties of this range that are still taken: its first ones
+        eq_take = eq_take < 0 ? 0 : eq_take;
+        uint32_t e = em, take = gm;
+        for (int c = 0; c < eq_take && e; ++c) { take |= e & (0u - e); e &= e - 1; }
+        int pos = gt_before + min(eq_before, r);
+        while (take) {
+            const int b = __ffs(take) - 1;
+            take &= take - 1;
+            if (pos < cap) out[pos] = lo + b;
+            ++pos;
         }
-        gt_before += gt; eq_before += eq;
+    } else {
+        unsigned long long mine = 0;   // (hi 32: # strictly above threshold, lo 32: # ties)
+        for (int i = lo; i < hi; ++i) {
+            bool gt, eq;
+            classify(i, gt, eq);
+            mine += ((unsigned long long)gt << 32) | (unsigned long long)eq;
+        }
+        const unsigned long long before = block_exclusive_scan(mine, warp_tot, &total);
+        int gt_before = (int)(before >> 32), eq_before = (int)(before & 0xFFFFFFFFu);
+        for (int i = lo; i < hi; ++i) {
+            bool gt, eq;
+            classify(i, gt, eq);
+            if (gt || (eq && eq_before < r)) {
+                const int pos = gt_before + min(eq_before, r);
+                if (pos < cap) out[pos] = i;
+            }
+            gt_before += gt; eq_before += eq;
+        }
     }
     if (tid == 0 && n_out) {
         int tot_gt = (int)(total >> 32), tot_eq = (int)(total & 0xFFFFFFFFu);
