@@ -496,7 +496,8 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    pdl_wait();                                 // H of the gate/up kernel
+    // The gate/up kernel lets this kernel start only after the union kernel has completed, so the union
+    // and the down rows it names can be read at once; only H has to wait for the gate/up kernel.
     const int n_u = *P.n_union;
     const int total_chunks = (n_u + kChunkK - 1) / kChunkK;        // 64 union entries per chunk
     const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
@@ -516,6 +517,9 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         const int k8 = e16 & 7;
         const int dst0 = (e16 >> 3) * 2048 + (c16 >> 3) * 1024 + k8 * 128 + (((c16 & 7) ^ k8) << 4);
         const char *dsrc0 = P.rec_base + (size_t)P.d_model * 4 + (size_t)mt * 256 + c16 * 16;
+        // the down rows of the first chunks (one per stage: the ring is empty) are fetched while the
+        // gate/up kernel finishes
+        const int pre = n_chunks < P.nstage ? n_chunks : P.nstage;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             int slots[4];
@@ -524,16 +528,32 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 slots[j] = slots_next[j];
                 if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c0 + c + 1) * kChunkK + 16 * j + e16];
             }
-            if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
+            if (c == pre) {      // (n_chunks > nstage) the ring is primed: now H is needed
+                pdl_wait();
+                if (tid == 0)
+                    for (int q = 0; q < pre; ++q) {
+                        mbar_arrive_expect_tx(&full[q], (uint32_t)N * 128u);
+                        tma_load_tile(tiles + (size_t)q * stage_bytes + 64 * 256, &h_map, (c0 + q) * kChunkK, tok0, &full[q]);
+                    }
+            }
+            if (c >= pre && !mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
             uint8_t *sa = tiles + (size_t)st * stage_bytes;
 #pragma unroll
             for (int j = 0; j < 4; ++j)                                      // padded entries carry a valid slot
                 cp_async16(sa + j * 4096 + dst0, dsrc0 + (size_t)slots[j] * P.rec_bytes);
-            if (tid == 0) {      // the dense H tile comes as one TMA copy
+            if (c >= pre && tid == 0) {      // the dense H tile comes as one TMA copy
                 mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
                 tma_load_tile(sa + 64 * 256, &h_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
             cp_async_arrive_when_landed(&full[st]);
+        }
+        if (n_chunks <= pre) {   // short K range: everything was primed above
+            pdl_wait();
+            if (tid == 0)
+                for (int q = 0; q < pre; ++q) {
+                    mbar_arrive_expect_tx(&full[q], (uint32_t)N * 128u);
+                    tma_load_tile(tiles + (size_t)q * stage_bytes + 64 * 256, &h_map, (c0 + q) * kChunkK, tok0, &full[q]);
+                }
         }
         cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
         bool ok = !*failed && mbar_wait(accbar, 0);
@@ -573,6 +593,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else {
+        pdl_wait();
         if (lane == 0) {
             const uint32_t idesc = make_idesc(P.fmt, 1, 0, 128, N);
             bool ok = true;

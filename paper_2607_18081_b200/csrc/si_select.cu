@@ -50,6 +50,130 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
     return warp_tot[warp] + inc - v;
 }
 
+// keys[i] = score_key(s[i]) for the whole row, by all threads of the CTA
+__device__ __forceinline__ void load_keys(const float *__restrict__ s, uint32_t *keys, int n, bool use_abs) {
+    const int tid = threadIdx.x;
+    if (((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(keys)) & 15u) == 0) {
+        // all of a thread's 16-byte loads are issued before the first key is formed
+        const float4 *s4 = reinterpret_cast<const float4 *>(s);
+        const int n4 = n >> 2;
+        for (int q0 = 0; q0 < n4; q0 += 4 * kSelThreads) {
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int q = q0 + j * kSelThreads + tid;
+                v[j] = q < n4 ? __ldg(s4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int q = q0 + j * kSelThreads + tid;
+                if (q < n4) {
+                    uint4 kk;
+                    kk.x = score_key(v[j].x, use_abs); kk.y = score_key(v[j].y, use_abs);
+                    kk.z = score_key(v[j].z, use_abs); kk.w = score_key(v[j].w, use_abs);
+                    *reinterpret_cast<uint4 *>(keys + 4 * q) = kk;
+                }
+            }
+        }
+        for (int i = 4 * n4 + tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs);
+    } else {
+        for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs);
+    }
+}
+
+// Top-k of rows of at most PER * 1024 scores (0 < k < n): thread t keeps the keys of its index range
+// [t*per, (t+1)*per) in registers, so the three radix passes and the emission read no memory but the
+// histogram.  Each thread clears the two bins it reads, which readies the histogram for the next pass.
+template <int PER>
+__global__ void __launch_bounds__(kSelThreads)
+si_select_topk_reg_kernel(const float *__restrict__ scores, int n, int row_stride, int k, int use_abs,
+                          int32_t *__restrict__ idx_out, int out_stride, int cap, int32_t *__restrict__ n_out) {
+    extern __shared__ __align__(16) uint32_t smem_keys[];
+    __shared__ __align__(8) unsigned int hist[kBins];
+    __shared__ unsigned int warp_cnt[32];
+    __shared__ unsigned long long warp_tot[32];
+    __shared__ unsigned long long total;
+    __shared__ uint32_t sh_prefix, sh_mask;
+    __shared__ int sh_need;
+
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float *s = scores + (size_t)row * row_stride;
+    int32_t *out = idx_out + (size_t)row * out_stride;
+    hist[tid] = 0; hist[tid + kSelThreads] = 0;
+    load_keys(s, smem_keys, n, use_abs != 0);
+    if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
+    __syncthreads();
+    const int per = (n + kSelThreads - 1) / kSelThreads;
+    const int lo = min(n, tid * per), cnt = min(n, lo + per) - lo;
+    uint32_t kr[PER];
+#pragma unroll
+    for (int j = 0; j < PER; ++j) kr[j] = j < cnt ? smem_keys[lo + j] : 0u;
+
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+        const uint32_t prefix = sh_prefix, mask = sh_mask;
+        const int need = sh_need;
+#pragma unroll
+        for (int j = 0; j < PER; ++j)
+            if (j < cnt && (kr[j] & mask) == prefix) atomicAdd(&hist[(kr[j] >> shift) & dmask], 1u);
+        __syncthreads();
+        // thread t owns bins 2047 - 2t and 2046 - 2t: a prefix sum over threads is a suffix sum over bins
+        uint2 *hp = reinterpret_cast<uint2 *>(hist) + (kSelThreads - 1 - tid);
+        const uint2 c2 = *hp;
+        *hp = make_uint2(0u, 0u);
+        const unsigned c_hi = c2.y, c_lo = c2.x, pair = c_hi + c_lo;
+        unsigned inc = pair;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) warp_cnt[warp] = inc;
+        __syncthreads();
+        const unsigned wt = warp_cnt[lane];
+        const unsigned excl = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? wt : 0u) + inc - pair;   // keys in bins above this pair
+        // the keys in play are at least `need`, so exactly one bin satisfies this (bin 0 at the latest)
+        if (excl < (unsigned)need && (unsigned)need <= excl + c_hi) {
+            sh_need = need - (int)excl;
+            sh_prefix = prefix | ((uint32_t)(kBins - 1 - 2 * tid) << shift);
+            sh_mask = mask | (dmask << shift);
+        } else if (excl + c_hi < (unsigned)need && (unsigned)need <= excl + pair) {
+            sh_need = need - (int)(excl + c_hi);
+            sh_prefix = prefix | ((uint32_t)(kBins - 2 - 2 * tid) << shift);
+            sh_mask = mask | (dmask << shift);
+        }
+        __syncthreads();
+    }
+    const uint32_t kstar = sh_prefix;
+    const int r = sh_need;                 // r of the keys equal to kstar are taken, the lowest indices first
+
+    uint32_t gm = 0, em = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        if (j < cnt) { gm |= (uint32_t)(kr[j] > kstar) << j; em |= (uint32_t)(kr[j] == kstar) << j; }
+    }
+    const unsigned long long mine = ((unsigned long long)__popc(gm) << 32) | (unsigned long long)__popc(em);
+    const unsigned long long before = block_exclusive_scan(mine, warp_tot, &total);
+    const int gt_before = (int)(before >> 32), eq_before = (int)(before & 0xFFFFFFFFu);
+    int eq_take = r - eq_before;
+    eq_take = eq_take < 0 ? 0 : eq_take;
+    uint32_t e = em, take = gm;
+    for (int c = 0; c < eq_take && e; ++c) { take |= e & (0u - e); e &= e - 1; }
+    int pos = gt_before + min(eq_before, r);
+    while (take) {
+        const int b = __ffs(take) - 1;
+        take &= take - 1;
+        if (pos < cap) out[pos] = lo + b;
+        ++pos;
+    }
+    if (tid == 0 && n_out) {
+        const int tot_gt = (int)(total >> 32), tot_eq = (int)(total & 0xFFFFFFFFu);
+        n_out[row] = tot_gt + min(tot_eq, r);
+    }
+}
+
 __global__ void __launch_bounds__(kSelThreads)
 si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mode, int k, float tau,
                  int use_abs, int32_t *__restrict__ idx_out, int out_stride, int cap,
@@ -68,32 +192,7 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
 
     uint32_t kstar = 0; int r = 0;          // threshold key and how many of its ties to take
     if (mode == SI_SELECT_TOPK) {
-        if (((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(keys)) & 15u) == 0) {
-            // all of a thread's 16-byte loads are issued before the first key is formed
-            const float4 *s4 = reinterpret_cast<const float4 *>(s);
-            const int n4 = n >> 2;
-            for (int q0 = 0; q0 < n4; q0 += 4 * kSelThreads) {
-                float4 v[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int q = q0 + j * kSelThreads + tid;
-                    v[j] = q < n4 ? __ldg(s4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int q = q0 + j * kSelThreads + tid;
-                    if (q < n4) {
-                        uint4 kk;
-                        kk.x = score_key(v[j].x, use_abs != 0); kk.y = score_key(v[j].y, use_abs != 0);
-                        kk.z = score_key(v[j].z, use_abs != 0); kk.w = score_key(v[j].w, use_abs != 0);
-                        *reinterpret_cast<uint4 *>(keys + 4 * q) = kk;
-                    }
-                }
-            }
-            for (int i = 4 * n4 + tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
-        } else {
-            for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i], use_abs != 0);
-        }
+        load_keys(s, keys, n, use_abs != 0);
         if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
         __syncthreads();
         if (k > 0 && k < n) {
@@ -231,12 +330,29 @@ int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int
     size_t smem = in_smem ? (size_t)(n > 0 ? n : 1) * 4 : 0;
     static bool attr_set = false;
     if (!attr_set) {
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemKeys * 4));
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemKeys * 4));
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kSelThreads * 4));
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kSelThreads * 4));
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * kSelThreads * 4));
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * kSelThreads * 4));
         attr_set = true;
     }
-    si_select_kernel<<<n_rows, kSelThreads, smem, stream>>>(scores, n, row_stride, mode, k, tau,
-                                                            (flags & SI_FLAG_SCORE_ABS) != 0, idx_out,
+    const int use_abs = (flags & SI_FLAG_SCORE_ABS) != 0;
+    if (mode == SI_SELECT_TOPK && k > 0 && k < n && n <= 32 * kSelThreads) {
+        // the common case: a proper subset of a row whose keys fit the threads' registers
+        const int per = (n + kSelThreads - 1) / kSelThreads;
+#define SI_SELECT_REG(P)                                                                                              \
+    si_select_topk_reg_kernel<P><<<n_rows, kSelThreads, (size_t)n * 4, stream>>>(scores, n, row_stride, k, use_abs, \
+                                                                                 idx_out, out_stride, cap, n_out)
+        if (per <= 4) SI_SELECT_REG(4);
+        else if (per <= 8) SI_SELECT_REG(8);
+        else if (per <= 16) SI_SELECT_REG(16);
+        else SI_SELECT_REG(32);
+#undef SI_SELECT_REG
+        SI_CUDA_TRY(cudaGetLastError());
+        return SI_OK;
+    }
+    si_select_kernel<<<n_rows, kSelThreads, smem, stream>>>(scores, n, row_stride, mode, k, tau, use_abs, idx_out,
                                                             out_stride, cap, n_out, (uint32_t *)workspace, in_smem);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
