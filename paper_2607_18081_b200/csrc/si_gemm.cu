@@ -114,51 +114,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 // ------------------------------------------------------------------------------- union
-// Sorted union of the lists in one launch.  Every block ORs its share of the list entries into a
-// bitmap over the loaded slots and -- when each token has its own list -- into that token's own
-// slot bitmap (membership test of the combine step).  The block that finishes last turns the
-// bitmap into the ascending union by a popcount prefix scan.  bitmap, tokbits and ticket are zero
-// on entry.  blockDim.x = 1024; dynamic shared memory = (2 * words + 2) * 4 bytes.
-__global__ void __launch_bounds__(1024)
-si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int n_lists,
-                      int n_loaded, uint32_t *bitmap_g, uint32_t *tokbits, int mask_words, unsigned *ticket,
-                      int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out, int union_cap, int32_t *status) {
-    extern __shared__ uint32_t sh[];
-    __shared__ uint32_t warp_tot[32];
-    __shared__ int is_last;
+// sh[0 .. words) holds the bitmap; sh[words .. 2*words + 2) is scratch.  Writes the ascending union, its
+// size, and pads the list up to union_cap with its first entry (padded positions contribute nothing).
+__device__ __forceinline__ void union_scan_emit(uint32_t *sh, uint32_t *warp_tot, int words, int32_t *__restrict__ union_out,
+                                                int32_t *__restrict__ n_union_out, int union_cap) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    pdl_launch();
-    const long long total = offsets ? offsets[n_lists] : (long long)n_lists * k_fixed;
-    for (long long e = (long long)blockIdx.x * blockDim.x + tid; e < total; e += (long long)gridDim.x * blockDim.x) {
-        const int s = idx[e];
-        if (s < 0 || s >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
-        const uint32_t bit = 1u << (s & 31);
-        if (!(bitmap_g[s >> 5] & bit)) atomicOr(&bitmap_g[s >> 5], bit);     // hot slots are set by the first token
-        if (tokbits) {
-            int t;
-            if (offsets) {            // largest t with offsets[t] <= e
-                int lo = 0, hi = n_lists;
-                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
-                t = lo;
-            } else {
-                t = (int)(e / k_fixed);
-            }
-            atomicOr(&tokbits[(size_t)t * mask_words + (s >> 5)], bit);
-        }
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-
-    // ---- last block: popcount prefix scan over the bitmap -> ascending union
-    const int words = (n_loaded + 31) / 32;
     uint32_t *bitmap = sh;                         // [words]
     uint32_t *wprefix = sh + words;                // [words] exclusive popcount prefix
-    for (int w = tid; w < words; w += 1024) bitmap[w] = __ldcg(bitmap_g + w);
-    __syncthreads();
     uint32_t carry = 0;
     for (int base = 0; base < words; base += 1024) {
         int w = base + tid;
@@ -188,12 +150,101 @@ si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
             ++p;
         }
     }
-    // pad the union up to the capacity with its first entry (padded positions contribute nothing)
     {
         int first = 0;
         for (int w = 0; w < words; ++w) if (bitmap[w]) { first = w * 32 + __ffs(bitmap[w]) - 1; break; }
         for (int p = n_u + tid; p < union_cap; p += 1024) union_out[p] = first;
     }
+}
+
+// Sorted union of the lists in one launch.  Every block ORs its share of the list entries into a
+// bitmap over the loaded slots and -- when each token has its own list -- into that token's own
+// slot bitmap (membership test of the combine step).  The block that finishes last turns the
+// bitmap into the ascending union by a popcount prefix scan.  bitmap, tokbits and ticket are zero
+// on entry.  blockDim.x = 1024; dynamic shared memory = (2 * words + 2) * 4 bytes.
+__global__ void __launch_bounds__(1024)
+si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int n_lists,
+                      int n_loaded, uint32_t *bitmap_g, uint32_t *tokbits, int mask_words, unsigned *ticket,
+                      int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out, int union_cap, int32_t *status) {
+    extern __shared__ uint32_t sh[];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
+    pdl_launch();
+    const long long total = offsets ? offsets[n_lists] : (long long)n_lists * k_fixed;
+    for (long long e = (long long)blockIdx.x * blockDim.x + tid; e < total; e += (long long)gridDim.x * blockDim.x) {
+        const int s = idx[e];
+        if (s < 0 || s >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
+        const uint32_t bit = 1u << (s & 31);
+        if (!(bitmap_g[s >> 5] & bit)) atomicOr(&bitmap_g[s >> 5], bit);     // hot slots are set by the first token
+        if (tokbits) {
+            int t;
+            if (offsets) {            // largest t with offsets[t] <= e
+                int lo = 0, hi = n_lists;
+                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
+                t = lo;
+            } else {
+                t = (int)(e / k_fixed);
+            }
+            atomicOr(&tokbits[(size_t)t * mask_words + (s >> 5)], bit);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // ---- last block: popcount prefix scan over the bitmap -> ascending union
+    const int words = (n_loaded + 31) / 32;
+    for (int w = tid; w < words; w += 1024) sh[w] = __ldcg(bitmap_g + w);
+    __syncthreads();
+    union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
+}
+
+// The same result from one block, for calls with few list entries: the bitmap lives in shared memory,
+// the block clears the words the later kernels expect to be zero itself (no memset node), and nothing
+// has to cross blocks.  zero_g[0 .. zero_words) covers the token bitmaps and the arrival counters.
+__global__ void __launch_bounds__(1024)
+si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int n_lists,
+                      int n_loaded, uint32_t *zero_g, int zero_words, uint32_t *tokbits, int mask_words,
+                      int32_t *__restrict__ union_out, int32_t *__restrict__ n_union_out, int union_cap, int32_t *status) {
+    extern __shared__ uint32_t sh[];
+    __shared__ uint32_t warp_tot[32];
+    const int tid = threadIdx.x;
+    pdl_launch();
+    const int words = (n_loaded + 31) / 32;
+    for (int w = tid; w < zero_words; w += 1024) zero_g[w] = 0u;
+    for (int w = tid; w < words; w += 1024) sh[w] = 0u;
+    __syncthreads();
+    const int total = offsets ? offsets[n_lists] : n_lists * k_fixed;
+    for (int e0 = 0; e0 < total; e0 += 4 * 1024) {
+        int sl[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { const int e = e0 + j * 1024 + tid; sl[j] = e < total ? idx[e] : -2; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int e = e0 + j * 1024 + tid, sv = sl[j];
+            if (sv == -2 && e >= total) continue;
+            if (sv < 0 || sv >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
+            const uint32_t bit = 1u << (sv & 31);
+            atomicOr(&sh[sv >> 5], bit);
+            if (tokbits) {
+                int t;
+                if (offsets) {            // largest t with offsets[t] <= e
+                    int lo = 0, hi = n_lists;
+                    while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
+                    t = lo;
+                } else {
+                    t = e / k_fixed;
+                }
+                atomicOr(&tokbits[(size_t)t * mask_words + (sv >> 5)], bit);
+            }
+        }
+    }
+    __syncthreads();
+    union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
 }
 
 // ------------------------------------------------------------------------------- contractions
@@ -747,6 +798,8 @@ UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws,
     u.zero_bytes = ((size_t)(T + 1) * u.mask_words + 64 + (size_t)n_ctr) * 4;
     return u;
 }
+constexpr long long kUnionSmallEntries = 8 * 1024;      // up to here one block builds the union faster than several
+constexpr size_t kUnionSmallZeroBytes = 256 * 1024;
 int union_blocks(const si_store *s, long long entries) {
     // one entry per thread while the blocks fit the machine at once: an entry is a chain of dependent
     // global accesses (index, bitmap word, atomic), so the chains should all run side by side
@@ -776,11 +829,16 @@ int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, con
     const int n_loaded = s->n_loaded[layer];
     const int words = (n_loaded + 31) / 32;
     UnionScratch u = union_scratch(s, (char *)workspace, ws, T, n_loaded, 0);
-    SI_CUDA_TRY(cudaMemsetAsync(u.bitmap, 0, ((size_t)u.mask_words + 64) * 4, stream));
     const long long entries = idx_offsets ? (long long)T * n_loaded : (long long)T * k_fixed;
-    si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
-        idx, idx_offsets, k_fixed, T, n_loaded, u.bitmap, nullptr, u.mask_words, u.ticket, union_out, n_union_out,
-        n_loaded, nullptr);
+    if (entries <= kUnionSmallEntries) {
+        si_union_small_kernel<<<1, 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+            idx, idx_offsets, k_fixed, T, n_loaded, nullptr, 0, nullptr, u.mask_words, union_out, n_union_out, n_loaded, nullptr);
+    } else {
+        SI_CUDA_TRY(cudaMemsetAsync(u.bitmap, 0, ((size_t)u.mask_words + 64) * 4, stream));
+        si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+            idx, idx_offsets, k_fixed, T, n_loaded, u.bitmap, nullptr, u.mask_words, u.ticket, union_out, n_union_out,
+            n_loaded, nullptr);
+    }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }
@@ -829,12 +887,20 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         const int words = (n_loaded + 31) / 32;
         // token bitmaps are only read (and so only cleared) when the tokens have lists of their own
         char *z0 = own_lists ? (char *)us.tokbits : (char *)us.bitmap;
-        SI_CUDA_TRY(cudaMemsetAsync(z0, 0, us.zero_bytes - (size_t)(z0 - (char *)us.tokbits), stream));
+        const size_t zero_bytes = us.zero_bytes - (size_t)(z0 - (char *)us.tokbits);
         const int n_lists = shared ? 1 : T;
         const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
-        si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
-            idx, idx_offsets, k_fixed, n_lists, n_loaded, us.bitmap, own_lists ? us.tokbits : nullptr, us.mask_words,
-            us.ticket, uni, n_union, nu_pad, status_dev);
+        if (entries <= kUnionSmallEntries && zero_bytes <= kUnionSmallZeroBytes) {
+            // few entries: one block does everything, the clearing included
+            si_union_small_kernel<<<1, 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+                idx, idx_offsets, k_fixed, n_lists, n_loaded, (uint32_t *)z0, (int)(zero_bytes / 4),
+                own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
+        } else {
+            SI_CUDA_TRY(cudaMemsetAsync(z0, 0, zero_bytes, stream));
+            si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+                idx, idx_offsets, k_fixed, n_lists, n_loaded, us.bitmap, own_lists ? us.tokbits : nullptr, us.mask_words,
+                us.ticket, uni, n_union, nu_pad, status_dev);
+        }
     }
     // ---- tiling
     const int n_tok = tok_tiles > 1 ? tile_n : t_pad_total;
