@@ -70,6 +70,7 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
                          float *__restrict__ partial, int32_t *status) {
     __shared__ float red[2][kThreads / 32][4];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the reduce kernel may be scheduled already
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // x and the list may come from the kernel before
     const int base = offsets ? offsets[list] : list * k_fixed;
     const int k = offsets ? offsets[list + 1] - base : k_fixed;
     idx += base;
@@ -154,6 +155,7 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
                                float *__restrict__ partial, int32_t *status) {
     __shared__ float red[2][kThreads / 32][2];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // x and the list may come from the kernel before
     const int base = offsets ? offsets[list] : list * k_fixed;
     const int k = offsets ? offsets[list + 1] - base : k_fixed;
     idx += base;
@@ -249,6 +251,7 @@ si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
                         const uint16_t *__restrict__ x, void *__restrict__ y,
                         int y_f32, int residual) {
     __shared__ float4 part[32][8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a following kernel may be scheduled (it waits for y itself)
     asm volatile("griddepcontrol.wait;" ::: "memory");                // the partial rows of the preceding kernel
     const int g = threadIdx.x & 7, rc = threadIdx.x >> 3;
     const int col = (blockIdx.x * 8 + g) * 4;
@@ -292,12 +295,22 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
     int G = k < max_ctas ? (k < 1 ? 1 : k) : max_ctas;          // one partial row per CTA
     const uint4 *rec = (const uint4 *)s->records(layer);
     const int nl = s->n_loaded[layer];
-#define SI_LAUNCH_PARTIAL(N)                                                                        \
-    si_decode_partial_kernel<DT, N><<<G, kThreads, 0, stream>>>(rec, nl, chunks, (const uint4 *)x, \
-                                                                idx, offsets, list, k, partial, status_dev)
-#define SI_LAUNCH_AHEAD(N, P)                                                                             \
-    si_decode_partial_ahead_kernel<DT, N, P><<<G, kThreads, 0, stream>>>(rec, nl, chunks, (const uint4 *)x, \
-                                                                         idx, offsets, list, k, partial, status_dev)
+    // Both kernels are launched as programmatic dependents: each may be scheduled while its predecessor in
+    // the stream finishes and waits for that kernel's results with griddepcontrol.wait before it reads
+    // anything.  After a predecessor that never triggers early this is an ordinary launch.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(G); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const uint4 *x4 = (const uint4 *)x;
+#define SI_LAUNCH_PARTIAL(N)                                                                                       \
+    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_kernel<DT, N>, rec, nl, chunks, x4, idx, offsets, list, k, \
+                                   partial, status_dev))
+#define SI_LAUNCH_AHEAD(N, P)                                                                                           \
+    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P>, rec, nl, chunks, x4, idx, offsets, list, \
+                                   k, partial, status_dev))
     if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
     else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3);
     else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
@@ -305,18 +318,9 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
 #undef SI_LAUNCH_AHEAD
-    {
-        // programmatic dependent launch: the reduce kernel is scheduled while the partial kernel finishes
-        // and waits for its rows with griddepcontrol.wait
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((d + 31) / 32); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_reduce_kernel<DT>, (const float *)partial, G, d, (const uint16_t *)x, y,
-                                       (int)(y_dtype == SI_F32), (int)((flags & SI_FLAG_RESIDUAL) != 0)));
-    }
+    cfg.gridDim = dim3((d + 31) / 32); cfg.blockDim = dim3(256);
+    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_reduce_kernel<DT>, (const float *)partial, G, d, (const uint16_t *)x, y,
+                                   (int)(y_dtype == SI_F32), (int)((flags & SI_FLAG_RESIDUAL) != 0)));
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }

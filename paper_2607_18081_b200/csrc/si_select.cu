@@ -99,6 +99,7 @@ si_select_topk_reg_kernel(const float *__restrict__ scores, int n, int row_strid
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float *s = scores + (size_t)row * row_stride;
     int32_t *out = idx_out + (size_t)row * out_stride;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent kernel waits for the lists itself
     hist[tid] = 0; hist[tid + kSelThreads] = 0;
     load_keys(s, smem_keys, n, use_abs != 0);
     if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
