@@ -49,7 +49,8 @@ def test_topk_adversarial_ties_bit_exact(api, scores):
 
 
 @pytest.mark.parametrize("n,k", [(1, 1), (33, 7), (1000, 400), (4300, 215), (7705, 1541), (14336, 7168),
-                                 (14336, 0), (14336, 14336), (50000, 12345), (70000, 3000)])
+                                 (14336, 0), (14336, 14336), (16385, 1), (20000, 19999), (28672, 5734),
+                                 (40000, 777), (50000, 12345), (70000, 3000)])
 def test_topk_random_and_tied_scores(api, n, k):
     g = np.random.default_rng(n + k)
     for tied in (False, True):
