@@ -21,6 +21,9 @@ cpu_baseline / reference legs may import this module.
   activations, merged over score files after normalising by token count, ranked by importance.
 * ``loadset`` -- Section 4: base = top delta of the task ranking, then the model
   ranking in order, skipping ids already chosen, until gamma neurons are loaded.
+* ``shard_slots`` / ``shard_lists`` -- the loaded slots dealt round-robin to P devices and a slot list
+  rewritten for one of them.  Section 5 defines the layer output as a sum over the selected neurons, so
+  the partial outputs of disjoint neuron subsets add up to it; the paper itself runs on one device.
 * ``memory_saving`` -- Eq. 2.
 * ``layer_range`` -- Table 1 "first layer 5 / last layer -2".
 
@@ -277,6 +280,21 @@ def ranking(scores) -> np.ndarray:
     key = [(1 if v != v else 0, 0.0 if v != v else -v, i) for i, v in enumerate(s.tolist())]
     key.sort()
     return np.array([i for _, _, i in key], dtype=np.int32)
+
+
+def shard_slots(n_loaded: int, rank: int, world: int) -> np.ndarray:
+    """Global slots owned by device `rank` of `world`: rank, rank + world, ...  (local slot j = global
+    slot rank + j * world, so every device keeps the importance order and a share of the hot slots)."""
+    return np.arange(rank, n_loaded, world, dtype=np.int32)
+
+
+def shard_lists(lists, rank: int, world: int):
+    """Each list restricted to the slots device `rank` owns, as local slot numbers, order kept."""
+    out = []
+    for l in lists:
+        l = np.asarray(l, dtype=np.int64)
+        out.append((l[l % world == rank] // world).astype(np.int32))
+    return out
 
 
 def memory_saving(n_ffn_params: float, r_load: float, r_layer: float, bytes_per_param: float):

@@ -360,3 +360,41 @@ def test_profiler_scores_merge_and_ranking():
     task, model = so.ranking(so.profile_scores(b[:20])), r
     ids = so.loadset(task, model, 5, 12)
     assert ids[:5].tolist() == task[:5].tolist() and len(set(ids.tolist())) == 12
+
+
+# ---------------------------------------------------------------------------------------------
+# Neuron-sharded evaluation: Section 5 writes the layer output as a sum over the selected neurons, so
+# partial outputs over disjoint neuron subsets must add up to it.
+@pytest.mark.parametrize("world", [1, 2, 3, 5])
+def test_shard_partition_and_partial_sums(world):
+    Wg, Wu, Wd, x = _rand_problem(21 + world, d_ff=90, d_model=24)
+    g = np.random.default_rng(world)
+    loaded = g.permutation(90)[:61].astype(np.int32)              # slot -> global neuron id
+    lists = [np.sort(g.permutation(61)[:k]).astype(np.int32) for k in (0, 1, 17, 61)]
+    # every slot is owned exactly once, local order = global order
+    owned = [so.shard_slots(61, r, world) for r in range(world)]
+    assert sorted(np.concatenate(owned).tolist()) == list(range(61))
+    for r in range(world):
+        assert np.all(np.diff(owned[r]) > 0)
+    for l in lists:
+        parts = [so.shard_lists([l], r, world)[0] for r in range(world)]
+        # mapping back local -> global recovers the list, split without loss or duplication
+        back = np.sort(np.concatenate([owned[r][parts[r]] for r in range(world)]))
+        assert np.array_equal(back, l)
+        for r in range(world):
+            assert np.all(np.diff(parts[r]) > 0)                   # order kept
+        y_full = so.ffn(Wg, Wu, Wd, x, loaded[l])
+        y_sum = np.zeros_like(y_full)
+        for r in range(world):
+            ids_r = loaded[owned[r]]                               # the ids device r loads, in local slot order
+            y_sum += so.ffn(Wg, Wu, Wd, x, ids_r[parts[r]])
+        np.testing.assert_allclose(y_sum, y_full, rtol=1e-12, atol=1e-14)
+
+
+def test_shard_lists_hand_example():
+    # slots 0..9 on 3 devices: device 0 owns 0,3,6,9; device 1 owns 1,4,7; device 2 owns 2,5,8
+    l = np.array([1, 3, 4, 8, 9], dtype=np.int32)
+    assert so.shard_lists([l], 0, 3)[0].tolist() == [1, 3]         # slots 3, 9 -> local 1, 3
+    assert so.shard_lists([l], 1, 3)[0].tolist() == [0, 1]         # slots 1, 4 -> local 0, 1
+    assert so.shard_lists([l], 2, 3)[0].tolist() == [2]            # slot 8 -> local 2
+    assert so.shard_slots(10, 1, 3).tolist() == [1, 4, 7]
