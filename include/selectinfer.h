@@ -318,6 +318,42 @@ int si_loadset(const int32_t *task_rank, const int32_t *model_rank, int n, int n
  * outside the model. */
 int si_layer_range(int n_layers, int first, int last, int *first_out, int *last_out);
 
+/* ---------------------------------------------------------------- neuron shards over several GPUs
+ *
+ * Section 5 gives the layer output as a sum over the selected neurons, so P devices that each hold a
+ * disjoint share of the loaded neurons can each compute the partial output of their share; the
+ * partial outputs (fp32) are then added.  The paper runs on one device; this split is for layers
+ * whose loaded set does not fit one GPU or for many tokens per call.  Shares are dealt round-robin:
+ * device r of P holds global slots r, r + P, r + 2P, ... as its local slots 0, 1, 2, ... (load it with
+ * neuron_ids[r + j*P] and n_base_local = ceil((n_base - r) / P)), so every device keeps the importance
+ * order, the static-prefix property and an equal share of the frequently active slots.
+ *
+ *   si_shard_count    host function: *count_out = number of global slots < n that device `rank` holds.
+ *   si_shard_lists    rewrites slot lists for one device: of every list it keeps the entries s with
+ *                     s mod world == rank, as s div world, order kept, and packs the lists back to
+ *                     back: list t is idx_out[offsets_out[t] .. offsets_out[t+1]).  Input lists as
+ *                     in si_ffn_forward (idx_offsets[n_lists+1], or NULL and k_fixed entries each).
+ *                     idx_out: device int32, room for every input entry; offsets_out: device int32
+ *                     [n_lists + 1]; workspace: (n_lists + 64) * 4 bytes, 16-byte aligned.  Entries
+ *                     below 0 are dropped and reported through *status_dev (SI_ERR_OUT_OF_RANGE).
+ *                     Feed the result to si_ffn_forward with idx_offsets = offsets_out and k_fixed =
+ *                     an upper bound of the local list lengths.  Lists are fixed per prompt
+ *                     (Section 5), so this runs once per prompt and layer, not per token.
+ *   si_shard_reduce   y[t][j] = (x[t][j] +) parts[0][t][j] + parts[1][t][j] + ... in rank order (a fixed
+ *                     order: the result is the same on every device).  parts_dev: DEVICE array of
+ *                     `world` device pointers to fp32 [T][d_model] partial outputs -- peer pointers
+ *                     for a one-shot all-reduce by plain peer loads, or a single pointer to a buffer an
+ *                     all-reduce has already summed (world = 1: residual and conversion only).  The
+ *                     caller orders this call after the partial outputs are complete on every device.
+ *                     x, y: as in si_ffn_forward (x may be NULL without SI_FLAG_RESIDUAL).
+ * All device work is asynchronous on stream.  No counterpart in the paper. */
+int si_shard_count(int n, int rank, int world, int *count_out);
+int si_shard_lists(const int32_t *idx, const int32_t *idx_offsets, int k_fixed, int n_lists, int rank, int world,
+                   int32_t *idx_out, int32_t *offsets_out, void *workspace, size_t ws_bytes, int32_t *status_dev,
+                   void *stream);
+int si_shard_reduce(const float *const *parts_dev, int world, const void *x, int x_dtype, int T, int d_model,
+                    void *y, int y_dtype, unsigned flags, void *stream);
+
 /* Library build information: "sm_100a" etc.  Never NULL. */
 const char *si_build_info(void);
 

@@ -35,7 +35,7 @@ EXPORTS = [
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
     "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
     "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
-    "si_loadset",
+    "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce",
 ]
 
 
@@ -82,6 +82,9 @@ def _load_library() -> ctypes.CDLL:
     lib.si_profile_rank.argtypes = [vp, ci, vp, vp]
     lib.si_loadset.argtypes = [vp, vp, ci, ci, ci, vp, vp, sz, vp, vp]
     lib.si_layer_range.argtypes = [ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.si_shard_count.argtypes = [ci, ci, ci, ctypes.POINTER(ci)]
+    lib.si_shard_lists.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, sz, vp, vp]
+    lib.si_shard_reduce.argtypes = [vp, ci, vp, ci, ci, ci, vp, ci, cu, vp]
     lib.si_prefill_forward.argtypes = [vp, ci, vp, ci, vp, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -263,6 +266,26 @@ def si_decode_stack_forward(handle, n_steps: int, layers, x, idx, idx_offsets, k
                                         dtype_code(y.dtype), flags, _dp(workspace),
                                         workspace.numel() * workspace.element_size(), _dp(status),
                                         _stream(stream)), "si_decode_stack_forward")
+
+
+def si_shard_count(n: int, rank: int, world: int) -> int:
+    out = ctypes.c_int(0)
+    _check(_lib.si_shard_count(n, rank, world, ctypes.byref(out)), "si_shard_count")
+    return out.value
+
+
+def si_shard_lists(idx, idx_offsets, k_fixed: int, n_lists: int, rank: int, world: int, idx_out, offsets_out,
+                   workspace, status=None, stream=None) -> None:
+    _check(_lib.si_shard_lists(_dp(idx), _dp(idx_offsets), k_fixed, n_lists, rank, world, _dp(idx_out), _dp(offsets_out),
+                               _dp(workspace), workspace.numel() * workspace.element_size(), _dp(status),
+                               _stream(stream)), "si_shard_lists")
+
+
+def si_shard_reduce(parts_dev, world: int, x, T: int, d_model: int, y, flags: int, x_dtype=None, stream=None) -> None:
+    """parts_dev: int64 CUDA tensor holding `world` device addresses of fp32 [T, d_model] buffers."""
+    xd = dtype_code(x.dtype) if x is not None else dtype_code(torch.bfloat16 if x_dtype is None else x_dtype)
+    _check(_lib.si_shard_reduce(_dp(parts_dev), world, _dp(x), xd, T, d_model, _dp(y), dtype_code(y.dtype), flags,
+                                _stream(stream)), "si_shard_reduce")
 
 
 def si_ffn_forward_noalloc(handle, layer: int, x, idx, k: int, y, flags: int, status=None, stream=None) -> None:
