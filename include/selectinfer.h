@@ -272,9 +272,13 @@ int si_prefill_forward(const si_store_t *store, int layer, const void *x, int T,
  * Pass NULL to switch it off.  Costs a few clock reads per record. */
 int si_debug_decode_profile(void *dev_buf);
 
-/* Diagnostics: while on != 0, persistent decode launches only stream the selected records
- * through shared memory and skip the arithmetic (y is then meaningless).  Timing such a
- * launch gives the practical ceiling of the record stream on the same lists. */
+/* Diagnostics, a bit field (0 = normal operation).  Bits 0..2: persistent decode launches leave out
+ * part of the work (1: the arithmetic, 2: the loads of the cross-SM reduction, 4: the cross-SM
+ * exchange altogether; y is then meaningless) -- timing such a launch gives the practical ceiling of
+ * the record stream on the same lists.  Bits 8..11: ring stages per consumer set (0 = as many as
+ * fit).  Bits 12..15: number of step groups the SMs are split into (0 = the library's choice, 4 on
+ * 148 SMs; used by the tests to cover 1, 2 and 4 groups).  Results stay correct for every value of
+ * bits 8..15. */
 int si_debug_decode_stream_only(int on);
 
 /* Diagnostics: one launch that reads `bytes` bytes (a multiple of 16) at the 16-byte-aligned device

@@ -40,7 +40,7 @@ constexpr int kConsumers = kSets * kSetThreads;
 constexpr int kConsumerWarps = kConsumers / 32;
 constexpr int kReducerWarps = 3;
 constexpr int kThreads = 32 + kConsumers + 32 * kReducerWarps;        // producer, consumers, reducers
-constexpr int kMaxGroups = 8;                     // float4 column groups one CTA reduces (d_model / 4 / SMs, rounded up)
+constexpr int kMaxGroups = 32;                    // most float4 column groups one CTA reduces (d_model / 4 / CTAs per step group, rounded up)
 constexpr int kCounterStride = 64;                // uint32 per step: written at +0, reduced at +32 (own 128-byte lines)
 constexpr int kMaxStages = 16;
 constexpr int kDescRing = 64;                     // copy descriptors per set kept ahead of the issue lanes
@@ -64,7 +64,9 @@ struct Params {
     void *y;
     int y_f32, residual;
     int per_layer_lists;          // fixed-length lists only: idx is [n_layers][k_fixed], a step uses the list of its layer
-    float *partial;               // [D][G][d_model]
+    int n_groups;                 // step groups: CTA c belongs to group c mod n_groups and, with the other CTAs of its
+                                  // group, runs the steps s = group (mod n_groups); 1 = every CTA works on every step
+    float *partial;               // [n_groups][D][G][d_model], G = CTAs per group
     unsigned int *ctrl;           // [1] abort flag (zero at launch)
     unsigned int *counters;       // [n_steps][kCounterStride], zero at launch: +0 "written" = CTAs that
                                   // stored their partial of the step, +32 "reduced" = CTAs that finished
@@ -265,7 +267,9 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
     }
 }
 
-template <int DT, int NCH, bool kFull, bool kProf>   // kProf: phase profile compiled in; kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256)
+// kProf: phase profile compiled in; kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256);
+// GRP: float4 column groups a reducer warp covers at once (its 32 lanes = GRP groups x 32/GRP row classes)
+template <int DT, int NCH, bool kFull, bool kProf, int GRP>
 __global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -280,7 +284,12 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     volatile int *cta_abort = &sm->cta_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = gridDim.x, b = blockIdx.x;
+    // Step groups: the CTAs of group `grp` run the steps grp, grp + NG, ... among themselves (their v-th
+    // step is step v * NG + grp of the launch).  With short lists this divides the per-step fixed work --
+    // the x copy, the hand-over, the partial rows and their reduction -- by NG for the same records.
+    const int NG = P.n_groups, grp = blockIdx.x % NG;
+    const int G = gridDim.x / NG, b = blockIdx.x / NG;      // CTAs of this group, index within it
+    const int nv = P.n_steps > grp ? (P.n_steps - grp + NG - 1) / NG : 0;   // steps of this group
     const int Gv = G * kSets;                  // consumer sets act as virtual CTAs 2b, 2b+1 of 2G
     const int d = P.d_model, chunks = P.chunks;
 
@@ -323,18 +332,19 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             bool in = false;
             if (doit) {
                 StepGeom g;
-                in = step < P.n_steps;
-                if (in) g = step_geom(P, step, Gv, vb);
+                in = step < nv;
+                if (in) g = step_geom(P, step * NG + grp, Gv, vb);
                 while (in && t > g.cnt) {
                     t -= g.cnt + 1; ++step;
-                    in = step < P.n_steps;
-                    if (in) g = step_geom(P, step, Gv, vb);
+                    in = step < nv;
+                    if (in) g = step_geom(P, step * NG + grp, Gv, vb);
                 }
                 pf_valid = in;
                 if (in) {
-                    const int layer = P.step_layers ? __ldg(P.step_layers + step) : (P.n_few ? (int)P.few_layers[step] : step % P.n_layers);
+                    const int rs = step * NG + grp;               // step of the launch
+                    const int layer = P.step_layers ? __ldg(P.step_layers + rs) : (P.n_few ? (int)P.few_layers[rs] : rs % P.n_layers);
                     if (t == 0) {
-                        pf_src = (unsigned long long)(P.x + (size_t)step * d);
+                        pf_src = (unsigned long long)(P.x + (size_t)rs * d);
                         pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
                     } else {
                         const int lbase = P.per_layer_lists ? layer * P.k_fixed : g.base;
@@ -451,7 +461,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 
         const bool noarith = (P.stream_only & 1) != 0;  // diagnostics: drain only
 
-        for (int step = 0; step < P.n_steps && !fail; ++step) {
+        for (int step = 0; step < nv && !fail; ++step) {         // the group's steps, in its own numbering
             unsigned long long xr[NCH][4], acc[NCH][4];   // packed fp32 pairs
 #pragma unroll
             for (int i = 0; i < NCH; ++i)
@@ -576,10 +586,10 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         }
 #undef SI_PROF
         if (prof && q == 0) {
-            for (int i = 0; i < 5; ++i) P.prof[(size_t)b * kProfSlots + i] = pf[i];
-            P.prof[(size_t)b * kProfSlots + 5] = pf[5] + pf[6];
+            for (int i = 0; i < 5; ++i) P.prof[(size_t)blockIdx.x * kProfSlots + i] = pf[i];
+            P.prof[(size_t)blockIdx.x * kProfSlots + 5] = pf[5] + pf[6];
         }
-        if (prof && q == 1) { P.prof[(size_t)b * kProfSlots + 6] = pf[4]; P.prof[(size_t)b * kProfSlots + 7] = pf[1]; }
+        if (prof && q == 1) { P.prof[(size_t)blockIdx.x * kProfSlots + 6] = pf[4]; P.prof[(size_t)blockIdx.x * kProfSlots + 7] = pf[1]; }
         if (fail && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
         return;
     }
@@ -599,30 +609,32 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const int r = warp / 4 - 1;                            // 0 .. kReducerWarps-1
         const bool nosync = (P.stream_only & 4) != 0;
         const int ngroups = d / 4;
-        const int gpc = (ngroups + G - 1) / G;                 // <= kMaxGroups (launch check)
+        const int gpc = (ngroups + G - 1) / G;                 // <= GRP (launch check)
         const int g_valid = ngroups - b * gpc < gpc ? (ngroups - b * gpc < 0 ? 0 : ngroups - b * gpc) : gpc;
         const bool rprof = kProf && P.prof != nullptr && r == 0 && lane == 0;
         long long rp[6] = {0, 0, 0, 0, 0, 0}, rt = rprof ? clock64() : 0;
 #define SI_RPROF(slot) do { if (rprof) { long long now_ = clock64(); rp[slot] += now_ - rt; rt = now_; } } while (0)
-        const int bg = lane & (kMaxGroups - 1);                // phase B: this lane's column group ...
-        const int brc = lane / kMaxGroups;                     // ... and row class (rows brc, brc + 4, ...)
-        constexpr int kRowClasses = 32 / kMaxGroups;
+        const int bg = lane & (GRP - 1);                       // phase B: this lane's column group ...
+        const int brc = lane / GRP;                            // ... and row class (rows brc, brc + kRowClasses, ...)
+        constexpr int kRowClasses = 32 / GRP;
+        float *const gpartial = P.partial + (size_t)grp * kPartialDepth * G * d;   // this group's ring of partial rows
+        auto ctr_of = [&](int v) { return P.counters + ((size_t)v * NG + grp) * kCounterStride; };   // counters of the group's step v
         constexpr int kRowBatch = 13;                          // partial rows in flight per lane
-        for (int step = r; step < P.n_steps + kLag; step += kReducerWarps) {
+        for (int step = r; step < nv + kLag; step += kReducerWarps) {
             int ok = 1;
-            if (step < P.n_steps) {
+            if (step < nv) {
                 // ---- phase A: take each set's accumulators as soon as that set hands them over.  The
                 // first set's row is stored, the second set's is added with vector reductions at L2
                 // (a + b is the same whichever arrives first, so y stays bit-reproducible).
                 const uint32_t par = (uint32_t)((step / kReducerWarps) & 1);
-                float4 *dst = reinterpret_cast<float4 *>(P.partial + ((size_t)(step % kPartialDepth) * G + b) * d);
+                float4 *dst = reinterpret_cast<float4 *>(gpartial + ((size_t)(step % kPartialDepth) * G + b) * d);
                 const int n4 = d / 4;
                 int taken = 0;                            // bit q: set q's accumulators already consumed
                 // has every SM finished reading the step that used this ring slot before?  Asked
                 // now, while nothing is waiting for this warp; the answer is needed after the idle wait.
                 unsigned freed = (unsigned)G;
                 if (lane == 0 && !nosync && step >= kPartialDepth)
-                    freed = ld_acquire_gpu(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32);
+                    freed = ld_acquire_gpu(ctr_of(step - kPartialDepth) + 32);
                 for (int sub = 0; sub < kSets && ok; ++sub) {
                     int q = 0;
                     if (lane == 0) {
@@ -639,8 +651,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         ok = q >= 0;
                         SI_RPROF(0);                      // idle: waiting for a set's hand-over
                         if (ok && sub == 0 && freed < (unsigned)G)
-                            ok = counter_wait_bounded(P.counters + (size_t)(step - kPartialDepth) * kCounterStride + 32,
-                                                      (unsigned)G, P.ctrl + 1, cta_abort);
+                            ok = counter_wait_bounded(ctr_of(step - kPartialDepth) + 32, (unsigned)G, P.ctrl + 1, cta_abort);
                     }
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     q = __shfl_sync(0xFFFFFFFFu, q, 0);
@@ -675,13 +686,13 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 // group in ascending order, kRowBatch loads in flight; two butterfly steps combine the
                 // four row classes (fixed order: deterministic split-K)
                 if (lane == 0)
-                    ok = counter_wait_bounded(P.counters + (size_t)sr * kCounterStride, (unsigned)G, P.ctrl + 1, cta_abort);
+                    ok = counter_wait_bounded(ctr_of(sr), (unsigned)G, P.ctrl + 1, cta_abort);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 SI_RPROF(4);                              // every SM has published the step
                 if (ok) {
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                     const float4 *base = reinterpret_cast<const float4 *>(
-                        P.partial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4) + bg;
+                        gpartial + (size_t)(sr % kPartialDepth) * G * d + (size_t)b * gpc * 4) + bg;
                     const size_t row_stride = (size_t)d / 4;
                     if (bg < g_valid && (P.stream_only & 2) == 0) {
                         for (int r0 = brc; r0 < G; r0 += kRowClasses * kRowBatch) {
@@ -696,12 +707,12 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         }
                     }
 #pragma unroll
-                    for (int o = kMaxGroups; o < 32; o <<= 1) {
+                    for (int o = GRP; o < 32; o <<= 1) {
                         v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, o); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, o);
                         v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, o); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, o);
                     }
                     if (brc == 0 && bg < g_valid) {
-                        const size_t col = (size_t)sr * d + (size_t)(b * gpc + bg) * 4;
+                        const size_t col = ((size_t)sr * NG + grp) * d + (size_t)(b * gpc + bg) * 4;
                         if (P.residual) {
                             uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
                             v.x += si_cvt<DT>::lo(xw.x); v.y += si_cvt<DT>::hi(xw.x);
@@ -728,16 +739,22 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             __syncwarp();
             if (lane == 0 && !nosync) {
                 __threadfence();
-                if (step < P.n_steps) atomicAdd(P.counters + (size_t)step * kCounterStride, 1u);
-                if (sr >= 0 && sr + kPartialDepth < P.n_steps) atomicAdd(P.counters + (size_t)sr * kCounterStride + 32, 1u);
+                if (step < nv) atomicAdd(ctr_of(step), 1u);
+                if (sr >= 0 && sr + kPartialDepth < nv) atomicAdd(ctr_of(sr) + 32, 1u);
             }
             SI_RPROF(3);                                  // publish (fence + atomics)
         }
         if (rprof)
-            for (int i = 0; i < 6; ++i) P.prof[(size_t)b * kProfSlots + 8 + i] = rp[i];
+            for (int i = 0; i < 6; ++i) P.prof[(size_t)blockIdx.x * kProfSlots + 8 + i] = rp[i];
 #undef SI_RPROF
     }
 }
+
+// Step groups on n_sms SMs (1 = none).  Four groups were the fastest or within noise of it for every list
+// length measured (215 .. 7168 entries at d_model 4096): a step's fixed work -- the x copy, two hand-overs,
+// a partial row per CTA and its share of the reduction -- is paid by a quarter of the SMs for the same
+// records.  More groups would give a CTA more column groups to reduce than a warp has lanes.
+inline int pick_groups(int n_sms) { return n_sms % 4 == 0 ? 4 : (n_sms % 2 == 0 ? 2 : 1); }
 
 inline size_t smem_bytes(int d_model, int nstage) {
     return (size_t)nstage * d_model * 6 + (size_t)kSets * d_model * 4 + sizeof(Smem) + 64;
@@ -765,7 +782,7 @@ inline bool si_persistent_supported(const si_store *s) {
     const int chunks = s->d_model / 8, G = s->num_sms;
     const int gpc = (s->d_model / 4 + G - 1) / G;
     return s->n_layers <= SI_MAX_LAYERS && si_persist::pick_stages(s->d_model) >= 4 &&
-           chunks <= si_persist::kSetThreads * 2 && gpc <= si_persist::kMaxGroups;
+           chunks <= si_persist::kSetThreads * 2 && gpc <= 8;
 }
 
 // Bytes of the partial-y ring.
@@ -773,9 +790,9 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, bool FULL, bool PROF>
+template <int DT, int NCH, bool FULL, bool PROF, int GRP>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF>;
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
     static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
     int dev = 0;
@@ -823,16 +840,31 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // every CTA reduces at most kMaxGroups float4 column groups
     const int g_min = (s->d_model / 4 + si_persist::kMaxGroups - 1) / si_persist::kMaxGroups;
     if (G < g_min) G = g_min;
+    // Step groups: the SMs are split into groups that each take every n-th step on their own (launches of
+    // at least two steps per group; a launch that uses fewer CTAs than SMs keeps one group).
+    int ng = 1;
+    if (G == s->num_sms) {
+        const int forced = (si_decode_stream_only() >> 12) & 0xF;   // diagnostics: force a group count
+        ng = forced ? forced : si_persist::pick_groups(s->num_sms);
+        while (ng > 1 && (s->num_sms % ng != 0 || n_steps < 2 * ng ||
+                          (s->d_model / 4 + s->num_sms / ng - 1) / (s->num_sms / ng) > si_persist::kMaxGroups))
+            ng >>= 1;
+    }
+    P.n_groups = ng;
+    const int gpc = (s->d_model / 4 + G / ng - 1) / (G / ng);       // column groups per CTA -> lanes of a reducer warp
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
     const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
     const bool full = P.chunks == nch * si_persist::kSetThreads;
     // the phase profile is a separate instantiation: the production kernel carries no clock reads
-#define SI_PL2(DT, N, F) (P.prof ? si_decode_persistent_launch_t<DT, N, F, true>(P, G, stream) \
-                                 : si_decode_persistent_launch_t<DT, N, F, false>(P, G, stream))
+#define SI_PL3(DT, N, F, PR) (gpc <= 8 ? si_decode_persistent_launch_t<DT, N, F, PR, 8>(P, G, stream)    \
+                              : gpc <= 16 ? si_decode_persistent_launch_t<DT, N, F, PR, 16>(P, G, stream) \
+                                          : si_decode_persistent_launch_t<DT, N, F, PR, 32>(P, G, stream))
+#define SI_PL2(DT, N, F) (P.prof ? SI_PL3(DT, N, F, true) : SI_PL3(DT, N, F, false))
 #define SI_PL(DT) (nch <= 1 ? (full ? SI_PL2(DT, 1, true) : SI_PL2(DT, 1, false)) \
                             : (full ? SI_PL2(DT, 2, true) : SI_PL2(DT, 2, false)))
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
 #undef SI_PL2
+#undef SI_PL3
 #undef SI_PL
 }

@@ -232,6 +232,57 @@ def test_7b_shaped_two_layers_stack_and_determinism(api):
     assert_close(from_dev(yb[3]), m.oracle_y(1, x[1, 1], lists[1, 1]), "bf16 out")
 
 
+def test_7b_shaped_step_groups(api):
+    """The persistent kernel with its SMs split into 1, 2 and 4 step groups (4 is the default for
+    launches of 8 steps or more): 13 steps, so the groups get 4, 3, 3 and 3 steps; lists of equal
+    length, ragged lists with offsets (an empty one among them) and one list per layer; residual."""
+    cfg = wl.CONFIGS["c2"]
+    m = LoadedModel(cfg, n_layers=2)
+    steps, L, k, n = 13, 2, cfg.k_active, cfg.n_loaded
+    g = np.random.default_rng(77)
+    x = np.stack([wl.x_tokens(cfg, s % L, 1, first_token=s)[0] for s in range(steps)])
+    xd = to_dev(x, cfg.dtype)
+    fixed = np.stack([wl.zipf_lists(cfg, s % L, 1, first_token=s)[0] for s in range(steps)])
+    lens = [int(v) for v in g.integers(1, 2 * k, size=steps)]
+    lens[4] = 0
+    ragged = [np.sort(g.permutation(n)[:c]).astype(np.int32) for c in lens]
+    off = np.zeros(steps + 1, dtype=np.int32)
+    off[1:] = np.cumsum(lens)
+    per_layer = np.stack([wl.zipf_lists(cfg, l, 1)[0] for l in range(L)])
+    ws = m.store.workspace(1, max(max(lens), k), steps)
+    cases = [
+        ("fixed", torch.from_numpy(fixed).cuda(), None, k, 0, lambda s: fixed[s]),
+        ("offsets", torch.from_numpy(np.concatenate(ragged + [np.zeros(4, np.int32)])).cuda(), torch.from_numpy(off).cuda(),
+         max(lens), api.SI_FLAG_RESIDUAL, lambda s: ragged[s]),
+        ("per layer", torch.from_numpy(per_layer).cuda(), None, k, api.SI_FLAG_LIST_PER_LAYER, lambda s: per_layer[s % L]),
+    ]
+    try:
+        for name, idx, offsets, kk, flags, list_of in cases:
+            refs = None
+            for ng in (1, 2, 4):
+                api.lib().si_debug_decode_stream_only(ng << 12)
+                runs = []
+                for _ in range(2):
+                    y = torch.full((steps, cfg.d_model), 9.0, dtype=torch.float32, device="cuda")
+                    st = _status()
+                    api.si_decode_stack_forward(m.store.handle, steps, None, xd, idx, offsets, kk, y, flags, ws, st)
+                    torch.cuda.synchronize()
+                    assert st.item() == 0, (name, ng, api.strerror(int(st.item())))
+                    runs.append(y.cpu())
+                assert torch.equal(runs[0], runs[1]), f"{name}: {ng} groups not run-to-run bit-stable"
+                if refs is None:
+                    refs = []
+                    for s in range(steps):
+                        ref = m.oracle_y(s % L, x[s], list_of(s))
+                        if flags & api.SI_FLAG_RESIDUAL:
+                            ref = ref + wl.bits_to_float64(x[s], cfg.dtype)
+                        refs.append(ref)
+                for s in range(steps):
+                    assert_close(runs[0][s].double().numpy(), refs[s], f"{name}, {ng} groups, step {s}")
+    finally:
+        api.lib().si_debug_decode_stream_only(0)
+
+
 def test_check_flag_reports_bad_lists_without_faulting(api):
     cfg = _tiny_cfg()
     m = LoadedModel(cfg)
