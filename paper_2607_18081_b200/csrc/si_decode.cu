@@ -340,8 +340,11 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
         if (!s->loaded[l]) return SI_ERR_INVALID_ARG;
     }
     char *wsb = (char *)workspace;
-    // a single step is served faster by two plain launches than by starting the persistent kernel
-    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps == 1;
+    // one or two steps are served faster by two plain launches each than by starting the persistent
+    // kernel: a launch of it costs about 33 us beyond its steps, a plain step 12 us against 5.4 us
+    // (replayed from a CUDA graph; launched one by one from the host three steps already favour the
+    // persistent kernel, whose single launch costs the host less than six)
+    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps <= 2;
     if (!use_simple)
         return si_decode_persistent_launch(s, n_steps, layers_host, x, idx, idx_offsets, k_fixed, y, y_dtype, flags,
                                            wsb, ws, status_dev, stream);
