@@ -242,7 +242,7 @@ def run_ours(args):
     # End to end: the step's x and lists start in pinned host memory and y ends there.  The tokens go
     # through in chunks so that the copies of one chunk run beside the decode launch of another
     # (copy-in stream -> launch stream -> copy-out stream, two device input buffers).
-    n_chunk = 4 if tokens % 4 == 0 and tokens >= 8 else 1
+    n_chunk = args.e2e_chunks if args.e2e_chunks > 0 and tokens % args.e2e_chunks == 0 and tokens >= 2 * args.e2e_chunks else 1
     ct = tokens // n_chunk                                   # tokens per chunk
     cs = ct * L                                              # (token, layer) steps per chunk
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
@@ -481,6 +481,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="c3: tokens processed together per step")
     ap.add_argument("--cpu-tokens", type=int, default=8, help="tokens of the oracle cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-chunks", type=int, default=4, help="chunks the end-to-end step is pipelined in (measured: 4 beats 8 and 16)")
     ap.add_argument("--simple", action="store_true", help="time the per-step plain-load kernels instead")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch from an ncu capture (default: the committed capture of the "
