@@ -144,25 +144,29 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
 }
 
 // The same walk for rows of at most 512 chunks (d_model <= 4096), one record at a time with the loads of
-// the next P records already in flight: the records a CTA owns are independent, so nothing but registers
+// the next P records already in flight: the records of a walker are independent, so nothing but registers
 // limits how far ahead their loads may run.  The list entry of the record after those is fetched one
-// record early, so that no address waits for it.  Sums are taken in the order of the kernel above.
-template <int DT, int NCH, int P>
-__global__ void __launch_bounds__(kThreads, kSimpleCtasPerSm)
+// record early, so that no address waits for it.  A CTA holds SETS independent walkers of 256 threads
+// (walker v of all takes list positions v, v + walkers, ...), each with its own named barrier; with two,
+// the second leaves its sums in shared memory and the first adds them to its own, so the CTA writes one
+// partial row: half as many rows for the reduce kernel as with one walker per CTA.
+template <int DT, int NCH, int P, int SETS>
+__global__ void __launch_bounds__(kThreads * SETS, kSimpleCtasPerSm / SETS)
 si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks,
                                const uint4 *__restrict__ x, const int32_t *__restrict__ idx,
                                const int32_t *__restrict__ offsets, int list, int k_fixed,
                                float *__restrict__ partial, int32_t *status) {
-    __shared__ float red[2][kThreads / 32][2];
+    __shared__ float red[SETS][2][kThreads / 32][2];
+    __shared__ float4 merge[SETS > 1 ? 2 * NCH * kThreads : 1];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");                // x and the list may come from the kernel before
     const int base = offsets ? offsets[list] : list * k_fixed;
     const int k = offsets ? offsets[list + 1] - base : k_fixed;
     idx += base;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int G = gridDim.x;
-    const int n_mine = k > (int)blockIdx.x ? (k - (int)blockIdx.x + G - 1) / G : 0;   // records of this CTA
-    const int32_t *my = idx + blockIdx.x;
+    const int q = threadIdx.x / kThreads, tid = threadIdx.x % kThreads, lane = tid & 31, warp = tid >> 5;
+    const int G = gridDim.x * SETS, vb = blockIdx.x * SETS + q;      // walkers, this one's index
+    const int n_mine = k > vb ? (k - vb + G - 1) / G : 0;             // records of this walker
+    const int32_t *my = idx + vb;
     int first[P];
 #pragma unroll
     for (int st = 0; st < P; ++st) first[st] = st < n_mine ? my[(size_t)st * G] : 0;
@@ -201,7 +205,7 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
 #pragma unroll
         for (int st = 0; st < P; ++st) {
             const int j = j0 + st;
-            if (j < n_mine) {                                      // uniform over the CTA
+            if (j < n_mine) {                                      // uniform over the walker
                 float g = 0.f, u = 0.f;
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
@@ -210,9 +214,10 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
                     g += dot8<DT>(buf[st][3 * i], xr); u += dot8<DT>(buf[st][3 * i + 1], xr);
                 }
                 g = warp_sum(g); u = warp_sum(u);
-                float(*rb)[2] = red[j & 1];
+                float(*rb)[2] = red[q][j & 1];
                 if (lane == 0) { rb[warp][0] = g; rb[warp][1] = u; }
-                __syncthreads();
+                if (SETS == 1) __syncthreads();
+                else asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "n"(kThreads) : "memory");   // this walker's 256 threads
                 g = u = 0.f;
 #pragma unroll
                 for (int w = 0; w < kThreads / 32; ++w) { g += rb[w][0]; u += rb[w][1]; }
@@ -228,6 +233,23 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
                 if (jn < n_mine) fetch(buf[st], ok[st], ahead);
                 ahead = jn + 1 < n_mine ? my[(size_t)(jn + 1) * G] : 0;
             }
+        }
+    }
+    if (SETS > 1) {
+        if (q == 1) {
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+                merge[(2 * i) * kThreads + tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                merge[(2 * i + 1) * kThreads + tid] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+            }
+        }
+        __syncthreads();
+        if (q != 0) return;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const float4 lo = merge[(2 * i) * kThreads + tid], hi = merge[(2 * i + 1) * kThreads + tid];
+            acc[i][0] += lo.x; acc[i][1] += lo.y; acc[i][2] += lo.z; acc[i][3] += lo.w;
+            acc[i][4] += hi.x; acc[i][5] += hi.y; acc[i][6] += hi.z; acc[i][7] += hi.w;
         }
     }
     float4 *out = reinterpret_cast<float4 *>(partial + (size_t)blockIdx.x * chunks * 8);
@@ -308,11 +330,16 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 #define SI_LAUNCH_PARTIAL(N)                                                                                       \
     SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_kernel<DT, N>, rec, nl, chunks, x4, idx, offsets, list, k, \
                                    partial, status_dev))
-#define SI_LAUNCH_AHEAD(N, P)                                                                                           \
-    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P>, rec, nl, chunks, x4, idx, offsets, list, \
+#define SI_LAUNCH_AHEAD(N, P)                                                                                              \
+    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P, 2>, rec, nl, chunks, x4, idx, offsets, list, \
                                    k, partial, status_dev))
-    if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
-    else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3);
+    if (nch <= 2) {
+        // two walkers of 256 threads per CTA, one CTA per SM slot pair: one partial row per CTA
+        G = (G + 1) / 2;
+        cfg.gridDim = dim3(G); cfg.blockDim = dim3(2 * kThreads);
+        if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
+        else SI_LAUNCH_AHEAD(2, 3);
+    }
     else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
     else return SI_ERR_UNSUPPORTED;
