@@ -207,19 +207,26 @@ extern "C" int si_prefill_forward(const si_store_t *store, int layer, const void
     rc = si_multi_token_launch(store, layer, x, T, all, nullptr, n, y, y_dtype,
                                (flags & SI_FLAG_RESIDUAL) | SI_FLAG_SHARED_LIST, workspace, ws_bytes, status_dev, stream);
     if (rc) return rc;
-    // the activations the contraction used, widened exactly to fp32 (the partial-tile area is free again)
-    float *acts = acts_out;
-    if (!acts) {
-        if ((size_t)T * n * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
-        acts = (float *)(wsb + ws.partial_off);
-    }
     const int h_stride = (int)si_align_up((size_t)n, 128);
-    dim3 grid((n + 255) / 256, T);
-    if (store->dtype == SI_BF16)
-        si_widen_h_kernel<SI_BF16><<<grid, 256, 0, stream>>>((const uint16_t *)(wsb + ws.h_off), h_stride, T, n, acts);
-    else
-        si_widen_h_kernel<SI_F16><<<grid, 256, 0, stream>>>((const uint16_t *)(wsb + ws.h_off), h_stride, T, n, acts);
-    SI_CUDA_TRY(cudaGetLastError());
-    return si_prefill_vote_launch(acts, T, n, n, alpha, beta, n_static, phi_count, flags, idx_out, cap, n_out, nullptr,
+    const uint16_t *h = (const uint16_t *)(wsb + ws.h_off);
+    // The vote ranks the activations the contraction itself produced: H, in the store dtype.  Where the
+    // register selector applies it reads H as it is (widening is exact, so the order is that of the fp32
+    // values); fp32 copies are made only for a caller who asks for them, or for the general selector.
+    const bool fused = si_prefill_vote_fused_ok(n, alpha);
+    float *acts = acts_out;
+    if (acts || !fused) {
+        if (!acts) {
+            if ((size_t)T * n * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
+            acts = (float *)(wsb + ws.partial_off);       // the partial-tile area is free again
+        }
+        dim3 grid((n + 255) / 256, T);
+        if (store->dtype == SI_BF16) si_widen_h_kernel<SI_BF16><<<grid, 256, 0, stream>>>(h, h_stride, T, n, acts);
+        else si_widen_h_kernel<SI_F16><<<grid, 256, 0, stream>>>(h, h_stride, T, n, acts);
+        SI_CUDA_TRY(cudaGetLastError());
+    }
+    if (fused)
+        return si_prefill_vote_launch(h, store->dtype, T, n, h_stride, alpha, beta, n_static, phi_count, flags, idx_out, cap,
+                                      n_out, nullptr, vote_workspace, vote_ws_bytes, stream);
+    return si_prefill_vote_launch(acts, SI_F32, T, n, n, alpha, beta, n_static, phi_count, flags, idx_out, cap, n_out, nullptr,
                                   vote_workspace, vote_ws_bytes, stream);
 }

@@ -80,10 +80,17 @@ size_t si_select_ws_bytes_impl(int n);
 int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int mode, int k,
                      float tau, unsigned flags, int32_t *idx_out, int out_stride, int cap,
                      int32_t *n_out, void *workspace, size_t ws_bytes, cudaStream_t stream);
+// top-k of every row counted straight into counts[n]; scores of src_dtype (SI_F32 / SI_F16 / SI_BF16), row_stride
+// in elements; SI_ERR_UNSUPPORTED when the rows do not fit the register kernel
+int si_select_vote_launch(const void *scores, int src_dtype, int n_rows, int n, int row_stride, int k, unsigned flags,
+                          int *counts, cudaStream_t stream);
 
 // implemented in si_vote.cu
 size_t si_prefill_vote_ws_bytes_impl(int T, int n, int alpha);
-int si_prefill_vote_launch(const float *acts, int T, int n, int row_stride, int alpha, int beta, int n_static,
+// acts: [T] rows of acts_dtype (SI_F32, or a 16-bit type where the register selector applies: see
+// si_prefill_vote_fused_ok), row_stride in elements
+bool si_prefill_vote_fused_ok(int n, int alpha);
+int si_prefill_vote_launch(const void *acts, int acts_dtype, int T, int n, int row_stride, int alpha, int beta, int n_static,
                            int phi_count, unsigned flags, int32_t *idx_out, int cap, int32_t *n_out,
                            int32_t *counts_out, void *workspace, size_t ws_bytes, cudaStream_t stream);
 

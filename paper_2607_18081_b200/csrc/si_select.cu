@@ -81,13 +81,51 @@ __device__ __forceinline__ void load_keys(const float *__restrict__ s, uint32_t 
     }
 }
 
+// The same for a row of 16-bit scores (DT: SI_F16 / SI_BF16; widening to fp32 is exact, so the keys are
+// those of the widened row)
+template <int DT>
+__device__ __forceinline__ void load_keys16(const uint16_t *__restrict__ s, uint32_t *keys, int n, bool use_abs) {
+    const int tid = threadIdx.x;
+    if (((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(keys)) & 15u) == 0) {
+        const uint4 *s8 = reinterpret_cast<const uint4 *>(s);
+        const int n8 = n >> 3;
+        for (int q0 = 0; q0 < n8; q0 += 2 * kSelThreads) {
+            uint4 v[2];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int q = q0 + j * kSelThreads + tid;
+                v[j] = q < n8 ? __ldg(s8 + q) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int q = q0 + j * kSelThreads + tid;
+                if (q < n8) {
+                    uint4 lo, hi;
+                    lo.x = score_key(si_cvt<DT>::lo(v[j].x), use_abs); lo.y = score_key(si_cvt<DT>::hi(v[j].x), use_abs);
+                    lo.z = score_key(si_cvt<DT>::lo(v[j].y), use_abs); lo.w = score_key(si_cvt<DT>::hi(v[j].y), use_abs);
+                    hi.x = score_key(si_cvt<DT>::lo(v[j].z), use_abs); hi.y = score_key(si_cvt<DT>::hi(v[j].z), use_abs);
+                    hi.z = score_key(si_cvt<DT>::lo(v[j].w), use_abs); hi.w = score_key(si_cvt<DT>::hi(v[j].w), use_abs);
+                    *reinterpret_cast<uint4 *>(keys + 8 * q) = lo;
+                    *reinterpret_cast<uint4 *>(keys + 8 * q + 4) = hi;
+                }
+            }
+        }
+        for (int i = 8 * n8 + tid; i < n; i += kSelThreads) keys[i] = score_key(si_cvt<DT>::lo((uint32_t)s[i]), use_abs);
+    } else {
+        for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(si_cvt<DT>::lo((uint32_t)s[i]), use_abs);
+    }
+}
+
 // Top-k of rows of at most PER * 1024 scores (0 < k < n): thread t keeps the keys of its index range
 // [t*per, (t+1)*per) in registers, so the three radix passes and the emission read no memory but the
 // histogram.  Each thread clears the two bins it reads, which readies the histogram for the next pass.
-template <int PER>
+// SRC: type of the scores (SI_F32, or a 16-bit type).  With vote_counts set, every selected index adds one
+// to its entry there (the frequency count of the prefill vote) and idx_out may be NULL.
+template <int PER, int SRC>
 __global__ void __launch_bounds__(kSelThreads)
-si_select_topk_reg_kernel(const float *__restrict__ scores, int n, int row_stride, int k, int use_abs,
-                          int32_t *__restrict__ idx_out, int out_stride, int cap, int32_t *__restrict__ n_out) {
+si_select_topk_reg_kernel(const void *__restrict__ scores, int n, int row_stride, int k, int use_abs,
+                          int32_t *__restrict__ idx_out, int out_stride, int cap, int32_t *__restrict__ n_out,
+                          int *__restrict__ vote_counts) {
     extern __shared__ __align__(16) uint32_t smem_keys[];
     __shared__ __align__(8) unsigned int hist[kBins];
     __shared__ unsigned int warp_cnt[32];
@@ -97,11 +135,11 @@ si_select_topk_reg_kernel(const float *__restrict__ scores, int n, int row_strid
     __shared__ int sh_need;
 
     const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float *s = scores + (size_t)row * row_stride;
-    int32_t *out = idx_out + (size_t)row * out_stride;
+    int32_t *out = idx_out ? idx_out + (size_t)row * out_stride : nullptr;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent kernel waits for the lists itself
     hist[tid] = 0; hist[tid + kSelThreads] = 0;
-    load_keys(s, smem_keys, n, use_abs != 0);
+    if (SRC == SI_F32) load_keys(reinterpret_cast<const float *>(scores) + (size_t)row * row_stride, smem_keys, n, use_abs != 0);
+    else load_keys16<SRC == SI_F32 ? SI_BF16 : SRC>(reinterpret_cast<const uint16_t *>(scores) + (size_t)row * row_stride, smem_keys, n, use_abs != 0);
     if (tid == 0) { sh_prefix = 0; sh_mask = 0; sh_need = k; }
     __syncthreads();
     const int per = (n + kSelThreads - 1) / kSelThreads;
@@ -166,7 +204,8 @@ si_select_topk_reg_kernel(const float *__restrict__ scores, int n, int row_strid
     while (take) {
         const int b = __ffs(take) - 1;
         take &= take - 1;
-        if (pos < cap) out[pos] = lo + b;
+        if (out && pos < cap) out[pos] = lo + b;
+        if (vote_counts) atomicAdd(&vote_counts[lo + b], 1);
         ++pos;
     }
     if (tid == 0 && n_out) {
@@ -316,6 +355,43 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
     }
 }
 
+int select_set_attrs() {
+    static bool attr_set = false;
+    if (!attr_set) {
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemKeys * 4));
+#define SI_SEL_ATTR(P, S) SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<P, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, P * kSelThreads * 4))
+#define SI_SEL_ATTRS(S) SI_SEL_ATTR(4, S); SI_SEL_ATTR(8, S); SI_SEL_ATTR(16, S); SI_SEL_ATTR(32, S)
+        SI_SEL_ATTRS(SI_F32); SI_SEL_ATTRS(SI_F16); SI_SEL_ATTRS(SI_BF16);
+#undef SI_SEL_ATTRS
+#undef SI_SEL_ATTR
+        attr_set = true;
+    }
+    return SI_OK;
+}
+
+// the common case: a proper subset of a row whose keys fit the threads' registers
+int select_reg_launch(const void *scores, int src, int n_rows, int n, int row_stride, int k, int use_abs, int32_t *idx_out,
+                      int out_stride, int cap, int32_t *n_out, int *vote_counts, cudaStream_t stream) {
+    const int per = (n + kSelThreads - 1) / kSelThreads;
+#define SI_SELECT_REG2(P, S)                                                                                             \
+    si_select_topk_reg_kernel<P, S><<<n_rows, kSelThreads, (size_t)n * 4, stream>>>(scores, n, row_stride, k, use_abs, \
+                                                                                    idx_out, out_stride, cap, n_out, vote_counts)
+#define SI_SELECT_REG(P)                                                   \
+    do {                                                                   \
+        if (src == SI_F32) SI_SELECT_REG2(P, SI_F32);                      \
+        else if (src == SI_F16) SI_SELECT_REG2(P, SI_F16);                 \
+        else SI_SELECT_REG2(P, SI_BF16);                                   \
+    } while (0)
+    if (per <= 4) SI_SELECT_REG(4);
+    else if (per <= 8) SI_SELECT_REG(8);
+    else if (per <= 16) SI_SELECT_REG(16);
+    else SI_SELECT_REG(32);
+#undef SI_SELECT_REG
+#undef SI_SELECT_REG2
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}
+
 }  // namespace
 
 size_t si_select_ws_bytes_impl(int n) {
@@ -329,34 +405,28 @@ int si_select_launch(const float *scores, int n_rows, int n, int row_stride, int
     const int in_smem = n <= kSmemKeys;
     if (!in_smem && ws_bytes < (size_t)n_rows * n * 4) return SI_ERR_NOMEM;
     size_t smem = in_smem ? (size_t)(n > 0 ? n : 1) * 4 : 0;
-    static bool attr_set = false;
-    if (!attr_set) {
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemKeys * 4));
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kSelThreads * 4));
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * kSelThreads * 4));
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * kSelThreads * 4));
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_select_topk_reg_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * kSelThreads * 4));
-        attr_set = true;
-    }
+    int arc = select_set_attrs();
+    if (arc) return arc;
     const int use_abs = (flags & SI_FLAG_SCORE_ABS) != 0;
-    if (mode == SI_SELECT_TOPK && k > 0 && k < n && n <= 32 * kSelThreads) {
-        // the common case: a proper subset of a row whose keys fit the threads' registers
-        const int per = (n + kSelThreads - 1) / kSelThreads;
-#define SI_SELECT_REG(P)                                                                                              \
-    si_select_topk_reg_kernel<P><<<n_rows, kSelThreads, (size_t)n * 4, stream>>>(scores, n, row_stride, k, use_abs, \
-                                                                                 idx_out, out_stride, cap, n_out)
-        if (per <= 4) SI_SELECT_REG(4);
-        else if (per <= 8) SI_SELECT_REG(8);
-        else if (per <= 16) SI_SELECT_REG(16);
-        else SI_SELECT_REG(32);
-#undef SI_SELECT_REG
-        SI_CUDA_TRY(cudaGetLastError());
-        return SI_OK;
-    }
+    if (mode == SI_SELECT_TOPK && k > 0 && k < n && n <= 32 * kSelThreads)
+        return select_reg_launch(scores, SI_F32, n_rows, n, row_stride, k, use_abs, idx_out, out_stride, cap, n_out, nullptr, stream);
     si_select_kernel<<<n_rows, kSelThreads, smem, stream>>>(scores, n, row_stride, mode, k, tau, use_abs, idx_out,
                                                             out_stride, cap, n_out, (uint32_t *)workspace, in_smem);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
+}
+
+// Per-token top-k of T rows (fp32 or 16-bit scores) counted straight into counts[n] (zero on entry): the
+// first two steps of the prefill vote in one launch.  SI_ERR_UNSUPPORTED when the rows do not fit the
+// register kernel (the caller then selects into lists and counts them).
+int si_select_vote_launch(const void *scores, int src_dtype, int n_rows, int n, int row_stride, int k, unsigned flags,
+                          int *counts, cudaStream_t stream) {
+    if (!(k > 0 && k < n && n <= 32 * kSelThreads)) return SI_ERR_UNSUPPORTED;
+    if (n_rows <= 0) return SI_OK;
+    int rc = select_set_attrs();
+    if (rc) return rc;
+    return select_reg_launch(scores, src_dtype, n_rows, n, row_stride, k, (flags & SI_FLAG_SCORE_ABS) != 0, nullptr, 0, 0,
+                             nullptr, counts, stream);
 }
 
 extern "C" int si_select_workspace_bytes(int n, size_t *bytes_out) {

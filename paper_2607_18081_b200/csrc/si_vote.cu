@@ -97,7 +97,10 @@ vote_assemble_kernel(const int32_t *__restrict__ cand, int n_cand, const float *
 
 size_t si_prefill_vote_ws_bytes_impl(int T, int n, int alpha) { return vote_layout(T, n, alpha).total; }
 
-int si_prefill_vote_launch(const float *acts, int T, int n, int row_stride, int alpha, int beta, int n_static,
+// the register selector takes the rows as they are (any score type) and counts while it selects
+bool si_prefill_vote_fused_ok(int n, int alpha) { return alpha > 0 && alpha < n && n <= 32 * 1024; }
+
+int si_prefill_vote_launch(const void *acts, int acts_dtype, int T, int n, int row_stride, int alpha, int beta, int n_static,
                            int phi_count, unsigned flags, int32_t *idx_out, int cap, int32_t *n_out,
                            int32_t *counts_out, void *workspace, size_t ws_bytes, cudaStream_t stream) {
     const VoteLayout L = vote_layout(T, n, alpha);
@@ -112,12 +115,20 @@ int si_prefill_vote_launch(const float *acts, int T, int n, int row_stride, int 
 
     SI_CUDA_TRY(cudaMemsetAsync(counts, 0, (size_t)n * 4, stream));
     if (alpha > 0 && T > 0) {
-        int rc = si_select_launch(acts, T, n, row_stride, SI_SELECT_TOPK, alpha, 0.f, flags & SI_FLAG_SCORE_ABS, lists,
-                                  alpha, alpha, nullptr, w + L.selws, (size_t)T * si_select_ws_bytes_impl(n), stream);
-        if (rc) return rc;
-        const long long entries = (long long)T * alpha;
-        const int blocks = (int)((entries + 255) / 256 < 1184 ? (entries + 255) / 256 : 1184);
-        vote_histogram_kernel<<<blocks, 256, 0, stream>>>(lists, entries, n, counts);
+        // steps 1 and 2 in one launch where the rows fit the register selector: every selected slot adds
+        // one to its count; otherwise lists first, then their histogram (fp32 rows only)
+        int rc = si_select_vote_launch(acts, acts_dtype, T, n, row_stride, alpha, flags & SI_FLAG_SCORE_ABS, counts, stream);
+        if (rc == SI_ERR_UNSUPPORTED) {
+            if (acts_dtype != SI_F32) return SI_ERR_UNSUPPORTED;
+            rc = si_select_launch((const float *)acts, T, n, row_stride, SI_SELECT_TOPK, alpha, 0.f, flags & SI_FLAG_SCORE_ABS,
+                                  lists, alpha, alpha, nullptr, w + L.selws, (size_t)T * si_select_ws_bytes_impl(n), stream);
+            if (rc) return rc;
+            const long long entries = (long long)T * alpha;
+            const int blocks = (int)((entries + 255) / 256 < 1184 ? (entries + 255) / 256 : 1184);
+            vote_histogram_kernel<<<blocks, 256, 0, stream>>>(lists, entries, n, counts);
+        } else if (rc) {
+            return rc;
+        }
     }
     if (counts_out) SI_CUDA_TRY(cudaMemcpyAsync(counts_out, counts, (size_t)n * 4, cudaMemcpyDeviceToDevice, stream));
     vote_scores_kernel<<<(n + 255) / 256, 256, 0, stream>>>(counts, n, score_a, score_b);
@@ -151,6 +162,6 @@ extern "C" int si_prefill_vote(const float *acts, int T, int n, int row_stride, 
         return SI_ERR_INVALID_ARG;
     if (cap < phi_count) return SI_ERR_NOMEM;
     if (!si_aligned16(acts) || !si_aligned16(idx_out) || (((uintptr_t)workspace) & 255u)) return SI_ERR_ALIGNMENT;
-    return si_prefill_vote_launch(acts, T, n, row_stride, alpha, beta, n_static, phi_count, flags, idx_out, cap, n_out,
-                                  counts_out, workspace, ws_bytes, (cudaStream_t)stream);
+    return si_prefill_vote_launch(acts, SI_F32, T, n, row_stride, alpha, beta, n_static, phi_count, flags, idx_out, cap,
+                                  n_out, counts_out, workspace, ws_bytes, (cudaStream_t)stream);
 }
