@@ -263,37 +263,45 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
     }
 }
 
-// y[j] = (x[j] +) sum over CTAs g = 0..G-1 of partial[g][j].  One block per 32 output columns (eight
-// float4 groups); thread (group = tid & 7, row class = tid >> 3) sums rows class, class + 32, ... in
-// ascending order -- all its loads are independent -- and the 32 classes are then added in class
-// order, so the result does not depend on scheduling.
+// y[j] = (x[j] +) sum over the partial rows g = 0..G-1 of partial[g][j].  One block per 32 output columns
+// (eight float4 groups); thread (group = tid & 7, row class = tid >> 3) sums rows class, class + 32, ... in
+// ascending order, five loads in flight (one round for up to 160 rows).  The 32 classes are then added in
+// a fixed tree -- the four classes of a warp by two shuffle steps, the eight warps in warp order -- so the
+// result does not depend on scheduling.
 template <int DT>
 __global__ void __launch_bounds__(256)
 si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
-                        const uint16_t *__restrict__ x, void *__restrict__ y,
-                        int y_f32, int residual) {
-    __shared__ float4 part[32][8];
+                             const uint16_t *__restrict__ x, void *__restrict__ y,
+                             int y_f32, int residual) {
+    __shared__ float4 part[8][8];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a following kernel may be scheduled (it waits for y itself)
     asm volatile("griddepcontrol.wait;" ::: "memory");                // the partial rows of the preceding kernel
-    const int g = threadIdx.x & 7, rc = threadIdx.x >> 3;
+    const int g = threadIdx.x & 7, rc = threadIdx.x >> 3, warp = threadIdx.x >> 5;
     const int col = (blockIdx.x * 8 + g) * 4;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     if (col < d) {
-        for (int r0 = rc; r0 < G; r0 += 32 * 8) {
-            float4 v[8];
+        for (int r0 = rc; r0 < G; r0 += 32 * 5) {
+            float4 v[5];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < 5; ++j) {
                 const int r = r0 + 32 * j;
                 v[j] = r < G ? __ldg(reinterpret_cast<const float4 *>(partial + (size_t)r * d + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w; }
+            for (int j = 0; j < 5; ++j) { a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w; }
         }
     }
-    part[rc][g] = a;
+#pragma unroll
+    for (int o = 8; o <= 16; o <<= 1) {
+        a.x += __shfl_xor_sync(0xFFFFFFFFu, a.x, o); a.y += __shfl_xor_sync(0xFFFFFFFFu, a.y, o);
+        a.z += __shfl_xor_sync(0xFFFFFFFFu, a.z, o); a.w += __shfl_xor_sync(0xFFFFFFFFu, a.w, o);
+    }
+    if ((threadIdx.x & 31) < 8) part[warp][g] = a;
     __syncthreads();
-    if (rc != 0 || col >= d) return;
-    for (int c = 1; c < 32; ++c) { const float4 v = part[c][g]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+    if (threadIdx.x >= 8 || col >= d) return;
+    a = part[0][g];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) { const float4 v = part[w][g]; a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
     if (residual) {
         const uint2 xw = *reinterpret_cast<const uint2 *>(x + col);
         a.x += si_cvt<DT>::lo(xw.x); a.y += si_cvt<DT>::hi(xw.x); a.z += si_cvt<DT>::lo(xw.y); a.w += si_cvt<DT>::hi(xw.y);
