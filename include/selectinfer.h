@@ -183,10 +183,12 @@ int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, c
 /* Batch-1 decode over a stack: n_steps consecutive (token, layer) steps in one
  * persistent launch, step s using layer layers[s] (HOST int32 [n_steps], or NULL for
  * s mod n_layers).  x, y: device [n_steps, d_model]; idx: device [n_steps, k_fixed]
- * (or CSR over n_steps lists).  Steps are executed strictly in order; the weight
- * stream of later steps is prefetched while earlier steps finish.  Results equal
- * n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of a list
- * over SMs depends on the step's position in the call); each is run-to-run bit-stable.
+ * (or CSR over n_steps lists).  The steps are independent -- every step's x is an input of
+ * the call -- and several are in flight at once: the SMs work in up to four groups that each
+ * take every fourth step, and within a group the weight stream of later steps is prefetched
+ * while earlier steps finish.  All of y is complete when the call's work on the stream is.
+ * Results equal n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of
+ * a list over SMs depends on the step's position in the call); each is run-to-run bit-stable.
  * With SI_FLAG_LIST_PER_LAYER (fixed-length lists only) idx is [n_layers, k_fixed] and a step
  * uses the list of its layer: the set chosen during prefill serves every token of the prompt. */
 int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
