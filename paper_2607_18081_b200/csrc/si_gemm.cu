@@ -142,12 +142,13 @@ __device__ __forceinline__ void union_scan_emit(uint32_t *sh, uint32_t *warp_tot
     }
     const int n_u = (int)carry;
     if (tid == 0) *n_union_out = n_u;
-    for (int w = tid; w < words; w += 1024) {
-        uint32_t bits = bitmap[w]; int p = (int)wprefix[w];
-        while (bits) {
-            int bpos = __ffs(bits) - 1; bits &= bits - 1;
-            if (p < union_cap) union_out[p] = w * 32 + bpos;
-            ++p;
+    // one slot per thread and round: a set bit's position in the union is its word's prefix plus the set
+    // bits below it in the word -- no chain from one entry to the next
+    for (int i = tid; i < words * 32; i += 1024) {
+        const uint32_t bits = bitmap[i >> 5], below = (1u << (i & 31)) - 1u;
+        if ((bits >> (i & 31)) & 1u) {
+            const int p = (int)wprefix[i >> 5] + __popc(bits & below);
+            if (p < union_cap) union_out[p] = i;
         }
     }
     {
@@ -203,9 +204,13 @@ si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
 }
 
-// The same result from one block, for calls with few list entries: the bitmap lives in shared memory,
-// the block clears the words the later kernels expect to be zero itself (no memset node), and nothing
-// has to cross blocks.  zero_g[0 .. zero_words) covers the token bitmaps and the arrival counters.
+// The same result from one block, for calls with few list entries and few lists: the union's bitmap and
+// the tokens' bitmaps are built in shared memory (no global atomics, nothing to clear beforehand: every
+// word of the token bitmaps is written once, with plain stores), all list entries of a thread are loaded
+// before the first is used and merged per bitmap word in registers, the block clears the arrival counters the later kernels expect to be zero
+// (no memset node), and nothing has to cross blocks.  Dynamic shared memory: (2 * words + 2 + n_lists *
+// mask_words) * 4 bytes (the last term only with tokbits).
+constexpr int kUnionSmallBatch = 16;           // list entries per thread in flight
 __global__ void __launch_bounds__(1024)
 si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict__ offsets, int k_fixed, int n_lists,
                       int n_loaded, uint32_t *zero_g, int zero_words, uint32_t *tokbits, int mask_words,
@@ -215,35 +220,54 @@ si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     const int tid = threadIdx.x;
     pdl_launch();
     const int words = (n_loaded + 31) / 32;
+    uint32_t *tok_s = sh + 2 * words + 2;                          // [n_lists][mask_words]
+    const int tok_words = tokbits ? n_lists * mask_words : 0;
+    const int total = offsets ? offsets[n_lists] : n_lists * k_fixed;
+    // thread t takes the consecutive entries [t * per, (t + 1) * per): a list is ascending, so its entries
+    // fall into the same bitmap word several in a row, and the thread collects their bits in a register
+    // and updates shared memory once per (list, word) run
+    const int per = (total + 1023) / 1024;                         // <= kUnionSmallBatch (launch condition)
+    const int e_lo = tid * per;
+    int sl[kUnionSmallBatch];
+#pragma unroll
+    for (int j = 0; j < kUnionSmallBatch; ++j) { const int e = e_lo + j; sl[j] = (j < per && e < total) ? idx[e] : -1; }
     for (int w = tid; w < zero_words; w += 1024) zero_g[w] = 0u;
     for (int w = tid; w < words; w += 1024) sh[w] = 0u;
+    for (int w = tid; w < tok_words; w += 1024) tok_s[w] = 0u;
     __syncthreads();
-    const int total = offsets ? offsets[n_lists] : n_lists * k_fixed;
-    for (int e0 = 0; e0 < total; e0 += 4 * 1024) {
-        int sl[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { const int e = e0 + j * 1024 + tid; sl[j] = e < total ? idx[e] : -2; }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int e = e0 + j * 1024 + tid, sv = sl[j];
-            if (sv == -2 && e >= total) continue;
-            if (sv < 0 || sv >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
-            const uint32_t bit = 1u << (sv & 31);
-            atomicOr(&sh[sv >> 5], bit);
-            if (tokbits) {
-                int t;
-                if (offsets) {            // largest t with offsets[t] <= e
-                    int lo = 0, hi = n_lists;
-                    while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e) lo = mid; else hi = mid; }
-                    t = lo;
-                } else {
-                    t = e / k_fixed;
-                }
-                atomicOr(&tokbits[(size_t)t * mask_words + (sv >> 5)], bit);
+    {
+        int t = 0, t_end = 0;                                      // list of the current entry, first entry past it
+        if (e_lo < total) {
+            if (offsets) {            // largest t with offsets[t] <= e_lo
+                int lo = 0, hi = n_lists;
+                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (offsets[mid] <= e_lo) lo = mid; else hi = mid; }
+                t = lo; t_end = offsets[t + 1];
+            } else {
+                t = e_lo / k_fixed; t_end = (t + 1) * k_fixed;
             }
         }
+        int cur_w = -1, cur_t = 0;
+        uint32_t cur_bits = 0;
+        auto flush = [&]() {
+            if (cur_w >= 0) {
+                if ((sh[cur_w] & cur_bits) != cur_bits) atomicOr(&sh[cur_w], cur_bits);     // hot slots are set by the first token
+                if (tokbits) atomicOr(&tok_s[cur_t * mask_words + cur_w], cur_bits);
+            }
+        };
+#pragma unroll
+        for (int j = 0; j < kUnionSmallBatch; ++j) {
+            const int e = e_lo + j, sv = sl[j];
+            if (j >= per || e >= total) continue;
+            while (e >= t_end) { ++t; t_end = offsets ? offsets[t + 1] : t_end + k_fixed; }   // next list (empty ones skipped)
+            if (sv < 0 || sv >= n_loaded) { if (status) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
+            const int w = sv >> 5;
+            if (w != cur_w || t != cur_t) { flush(); cur_w = w; cur_t = t; cur_bits = 0; }
+            cur_bits |= 1u << (sv & 31);
+        }
+        flush();
     }
     __syncthreads();
+    for (int w = tid; w < tok_words; w += 1024) tokbits[w] = tok_s[w];
     union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
 }
 
@@ -798,8 +822,8 @@ UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws,
     u.zero_bytes = ((size_t)(T + 1) * u.mask_words + 64 + (size_t)n_ctr) * 4;
     return u;
 }
-constexpr long long kUnionSmallEntries = 8 * 1024;      // up to here one block builds the union faster than several
-constexpr size_t kUnionSmallZeroBytes = 256 * 1024;
+constexpr long long kUnionSmallEntries = 16 * 1024;     // up to here one block builds the union faster than several
+constexpr size_t kUnionSmallSmem = 160 * 1024;          // shared memory the one-block union may use
 int union_blocks(const si_store *s, long long entries) {
     // one entry per thread while the blocks fit the machine at once: an entry is a chain of dependent
     // global accesses (index, bitmap word, atomic), so the chains should all run side by side
@@ -890,10 +914,19 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         const size_t zero_bytes = us.zero_bytes - (size_t)(z0 - (char *)us.tokbits);
         const int n_lists = shared ? 1 : T;
         const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
-        if (entries <= kUnionSmallEntries && zero_bytes <= kUnionSmallZeroBytes) {
-            // few entries: one block does everything, the clearing included
-            si_union_small_kernel<<<1, 1024, (size_t)(2 * words + 2) * 4, stream>>>(
-                idx, idx_offsets, k_fixed, n_lists, n_loaded, (uint32_t *)z0, (int)(zero_bytes / 4),
+        const size_t small_smem = ((size_t)2 * words + 2 + (own_lists ? (size_t)n_lists * us.mask_words : 0)) * 4;
+        if (entries <= kUnionSmallEntries && small_smem <= kUnionSmallSmem) {
+            // few entries, few lists: one block does everything in shared memory, the clearing of the
+            // counters included
+            static bool attr_set = false;
+            if (!attr_set) {
+                SI_CUDA_TRY(cudaFuncSetAttribute(si_union_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUnionSmallSmem));
+                attr_set = true;
+            }
+            uint32_t *zc = (uint32_t *)us.ticket;                          // ticket words and the arrival counters
+            const size_t zc_bytes = us.zero_bytes - (size_t)((char *)us.ticket - (char *)us.tokbits);
+            si_union_small_kernel<<<1, 1024, small_smem, stream>>>(
+                idx, idx_offsets, k_fixed, n_lists, n_loaded, zc, (int)(zc_bytes / 4),
                 own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
         } else {
             SI_CUDA_TRY(cudaMemsetAsync(z0, 0, zero_bytes, stream));
