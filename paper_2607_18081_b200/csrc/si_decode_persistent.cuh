@@ -776,13 +776,13 @@ long long *&si_decode_profile_buffer();
 int &si_decode_stream_only();
 
 inline bool si_persistent_supported(const si_store *s) {
-    // thread t of a 256-thread set owns chunks t, t+256 of a row (d_model <= 4096); the split-K
-    // reduction lets 512 / pow2ceil(groups per SM) threads share a column group and gives each
-    // of them at most 5 of the 2G partials
+    // thread t of a 256-thread set owns chunks t, t + 256 (, t + 512) of a row (d_model <= 6144); the
+    // rings need at least two stages per consumer set beside the two hand-over buffers; a reducer warp's
+    // lanes cover the float4 column groups of a CTA
     const int chunks = s->d_model / 8, G = s->num_sms;
     const int gpc = (s->d_model / 4 + G - 1) / G;
     return s->n_layers <= SI_MAX_LAYERS && si_persist::pick_stages(s->d_model) >= 4 &&
-           chunks <= si_persist::kSetThreads * 2 && gpc <= 8;
+           chunks <= si_persist::kSetThreads * 3 && gpc <= si_persist::kMaxGroups;
 }
 
 // Bytes of the partial-y ring.
@@ -861,10 +861,15 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
                               : gpc <= 16 ? si_decode_persistent_launch_t<DT, N, F, PR, 16>(P, G, stream) \
                                           : si_decode_persistent_launch_t<DT, N, F, PR, 32>(P, G, stream))
 #define SI_PL2(DT, N, F) (P.prof ? SI_PL3(DT, N, F, true) : SI_PL3(DT, N, F, false))
-#define SI_PL(DT) (nch <= 1 ? (full ? SI_PL2(DT, 1, true) : SI_PL2(DT, 1, false)) \
-                            : (full ? SI_PL2(DT, 2, true) : SI_PL2(DT, 2, false)))
+    // three chunks per thread (d_model 4104 .. 6144): no phase profile, 16 or 32 column groups per warp
+#define SI_PL_W(DT, F) (gpc <= 16 ? si_decode_persistent_launch_t<DT, 3, F, false, 16>(P, G, stream) \
+                                  : si_decode_persistent_launch_t<DT, 3, F, false, 32>(P, G, stream))
+#define SI_PL(DT) (nch <= 1 ? (full ? SI_PL2(DT, 1, true) : SI_PL2(DT, 1, false))     \
+                   : nch <= 2 ? (full ? SI_PL2(DT, 2, true) : SI_PL2(DT, 2, false)) \
+                              : (full ? SI_PL_W(DT, true) : SI_PL_W(DT, false)))
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
 #undef SI_PL2
 #undef SI_PL3
+#undef SI_PL_W
 #undef SI_PL
 }

@@ -16,7 +16,8 @@ SHAPES = [
     (2048, 1000, "bf16"),
     (3200, 900, "bf16"),      # 400 16-byte chunks per row: a ragged last round of the 256-thread walk
     (4096, 1024, "f16"),
-    (5120, 1024, "bf16"),
+    (5120, 1024, "bf16"),     # three chunks per thread in the persistent kernel, ragged
+    (6144, 800, "f16"),       # three full chunks per thread, two ring stages per consumer set
     (8192, 640, "bf16"),
 ]
 
