@@ -143,7 +143,7 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
     }
 }
 
-// The same walk for rows of at most 512 chunks (d_model <= 4096), one record at a time with the loads of
+// The same walk for rows of at most 768 chunks (d_model <= 6144), one record at a time with the loads of
 // the next P records already in flight: the records of a walker are independent, so nothing but registers
 // limits how far ahead their loads may run.  The list entry of the record after those is fetched one
 // record early, so that no address waits for it.  A CTA holds SETS independent walkers of 256 threads
@@ -341,12 +341,13 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 #define SI_LAUNCH_AHEAD(N, P)                                                                                              \
     SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P, 2>, rec, nl, chunks, x4, idx, offsets, list, \
                                    k, partial, status_dev))
-    if (nch <= 2) {
+    if (nch <= 3) {
         // two walkers of 256 threads per CTA, one CTA per SM slot pair: one partial row per CTA
         G = (G + 1) / 2;
         cfg.gridDim = dim3(G); cfg.blockDim = dim3(2 * kThreads);
         if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
-        else SI_LAUNCH_AHEAD(2, 3);
+        else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3);
+        else SI_LAUNCH_AHEAD(3, 2);
     }
     else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
