@@ -147,23 +147,24 @@ si_decode_partial_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks
 // the next P records already in flight: the records of a walker are independent, so nothing but registers
 // limits how far ahead their loads may run.  The list entry of the record after those is fetched one
 // record early, so that no address waits for it.  A CTA holds SETS independent walkers of 256 threads
-// (walker v of all takes list positions v, v + walkers, ...), each with its own named barrier; with two,
+// (W = 256; rows of more than 768 chunks get one walker of W = 512 threads; walker v of all takes list
+// positions v, v + walkers, ...), each with its own named barrier; with two,
 // the second leaves its sums in shared memory and the first adds them to its own, so the CTA writes one
 // partial row: half as many rows for the reduce kernel as with one walker per CTA.
-template <int DT, int NCH, int P, int SETS>
-__global__ void __launch_bounds__(kThreads * SETS, kSimpleCtasPerSm / SETS)
+template <int DT, int NCH, int P, int SETS, int W>
+__global__ void __launch_bounds__(W * SETS, 512 / (W * SETS))
 si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int chunks,
                                const uint4 *__restrict__ x, const int32_t *__restrict__ idx,
                                const int32_t *__restrict__ offsets, int list, int k_fixed,
                                float *__restrict__ partial, int32_t *status) {
-    __shared__ float red[SETS][2][kThreads / 32][2];
-    __shared__ float4 merge[SETS > 1 ? 2 * NCH * kThreads : 1];
+    __shared__ float red[SETS][2][W / 32][2];
+    __shared__ float4 merge[SETS > 1 ? 2 * NCH * W : 1];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");                // x and the list may come from the kernel before
     const int base = offsets ? offsets[list] : list * k_fixed;
     const int k = offsets ? offsets[list + 1] - base : k_fixed;
     idx += base;
-    const int q = threadIdx.x / kThreads, tid = threadIdx.x % kThreads, lane = tid & 31, warp = tid >> 5;
+    const int q = threadIdx.x / W, tid = threadIdx.x % W, lane = tid & 31, warp = tid >> 5;
     const int G = gridDim.x * SETS, vb = blockIdx.x * SETS + q;      // walkers, this one's index
     const int n_mine = k > vb ? (k - vb + G - 1) / G : 0;             // records of this walker
     const int32_t *my = idx + vb;
@@ -175,7 +176,7 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
     float acc[NCH][8];
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
-        const int c = tid + kThreads * i;
+        const int c = tid + W * i;
         xp[i] = c < chunks ? __ldg(x + c) : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[i][e] = 0.f;
@@ -188,7 +189,7 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
         const uint4 *r = rec + (size_t)(good ? slot : 0) * 3 * chunks;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            const int c = tid + kThreads * i;
+            const int c = tid + W * i;
             if (c < chunks) {
                 b[3 * i] = __ldg(r + c); b[3 * i + 1] = __ldg(r + chunks + c); b[3 * i + 2] = __ldg(r + 2 * chunks + c);
             } else {
@@ -217,10 +218,10 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
                 float(*rb)[2] = red[q][j & 1];
                 if (lane == 0) { rb[warp][0] = g; rb[warp][1] = u; }
                 if (SETS == 1) __syncthreads();
-                else asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "n"(kThreads) : "memory");   // this walker's 256 threads
+                else asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "n"(W) : "memory");   // this walker's 256 threads
                 g = u = 0.f;
 #pragma unroll
-                for (int w = 0; w < kThreads / 32; ++w) { g += rb[w][0]; u += rb[w][1]; }
+                for (int w = 0; w < W / 32; ++w) { g += rb[w][0]; u += rb[w][1]; }
                 const float h = ok[st] ? si_silu_mul(g, u) : 0.f;
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
@@ -239,15 +240,15 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
         if (q == 1) {
 #pragma unroll
             for (int i = 0; i < NCH; ++i) {
-                merge[(2 * i) * kThreads + tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                merge[(2 * i + 1) * kThreads + tid] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+                merge[(2 * i) * W + tid] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                merge[(2 * i + 1) * W + tid] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
             }
         }
         __syncthreads();
         if (q != 0) return;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            const float4 lo = merge[(2 * i) * kThreads + tid], hi = merge[(2 * i + 1) * kThreads + tid];
+            const float4 lo = merge[(2 * i) * W + tid], hi = merge[(2 * i + 1) * W + tid];
             acc[i][0] += lo.x; acc[i][1] += lo.y; acc[i][2] += lo.z; acc[i][3] += lo.w;
             acc[i][4] += hi.x; acc[i][5] += hi.y; acc[i][6] += hi.z; acc[i][7] += hi.w;
         }
@@ -255,7 +256,7 @@ si_decode_partial_ahead_kernel(const uint4 *__restrict__ rec, int n_loaded, int 
     float4 *out = reinterpret_cast<float4 *>(partial + (size_t)blockIdx.x * chunks * 8);
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
-        const int c = tid + kThreads * i;
+        const int c = tid + W * i;
         if (c < chunks) {
             out[2 * c] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
             out[2 * c + 1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
@@ -338,18 +339,22 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 #define SI_LAUNCH_PARTIAL(N)                                                                                       \
     SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_kernel<DT, N>, rec, nl, chunks, x4, idx, offsets, list, k, \
                                    partial, status_dev))
-#define SI_LAUNCH_AHEAD(N, P)                                                                                              \
-    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P, 2>, rec, nl, chunks, x4, idx, offsets, list, \
-                                   k, partial, status_dev))
+#define SI_LAUNCH_AHEAD(N, P, SETS, W)                                                                                        \
+    SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_partial_ahead_kernel<DT, N, P, SETS, W>, rec, nl, chunks, x4, idx, offsets, \
+                                   list, k, partial, status_dev))
     if (nch <= 3) {
         // two walkers of 256 threads per CTA, one CTA per SM slot pair: one partial row per CTA
         G = (G + 1) / 2;
         cfg.gridDim = dim3(G); cfg.blockDim = dim3(2 * kThreads);
-        if (nch <= 1) SI_LAUNCH_AHEAD(1, 4);
-        else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3);
-        else SI_LAUNCH_AHEAD(3, 2);
+        if (nch <= 1) SI_LAUNCH_AHEAD(1, 4, 2, 256);
+        else if (nch <= 2) SI_LAUNCH_AHEAD(2, 3, 2, 256);
+        else SI_LAUNCH_AHEAD(3, 2, 2, 256);
+    } else if (nch <= 4) {
+        // rows of up to 1024 chunks (d_model <= 8192): one walker of 512 threads per CTA and SM
+        G = (G + 1) / 2;
+        cfg.gridDim = dim3(G); cfg.blockDim = dim3(512);
+        SI_LAUNCH_AHEAD(2, 3, 1, 512);
     }
-    else if (nch <= 4) SI_LAUNCH_PARTIAL(4);
     else if (nch <= 8) SI_LAUNCH_PARTIAL(8);
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
