@@ -33,7 +33,7 @@
 
 namespace si_persist {
 
-constexpr int kSets = 2;                          // independent consumer sets, each with its own ring
+constexpr int kSets = 2;                          // independent consumer sets, each with its own ring (one set of 16 warps for wide rows)
 constexpr int kSetWarps = 8;
 constexpr int kSetThreads = kSetWarps * 32;
 constexpr int kConsumers = kSets * kSetThreads;
@@ -170,6 +170,7 @@ __device__ __forceinline__ void bulk_g2s(void *dst_smem, const void *src_gmem, u
 // Hardware barrier over the 256 threads of consumer set q (barrier id 1 + q) that also ORs a flag:
 // every thread of the set learns whether any of them has a failed wait, so the set always leaves
 // its loops together and nobody is left waiting at the barrier.
+template <int kSetThreadsT>
 __device__ __forceinline__ bool set_barrier_or(int q, bool v) {
     uint32_t r;
     asm volatile(
@@ -177,7 +178,7 @@ __device__ __forceinline__ bool set_barrier_or(int q, bool v) {
         "setp.ne.u32 f, %1, 0;\n\t"
         "bar.red.or.pred p, %2, %3, f;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"((uint32_t)v), "r"(1 + q), "n"(kSetThreads) : "memory");
+        : "=r"(r) : "r"((uint32_t)v), "r"(1 + q), "n"(kSetThreadsT) : "memory");
     return r != 0;
 }
 
@@ -255,7 +256,7 @@ struct Smem {
     uint64_t accfull[kSets][kReducerWarps], accempty[kSets][kReducerWarps];
     int meta[kMaxStages];
     uint4 desc[kSets][kDescRing];      // {src lo, src hi, bytes (0: nothing to copy), meta}
-    float2 setpart[kSets][2][kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products
+    float2 setpart[kSets][2][2 * kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products (16 warps in the one wide set)
     volatile int cta_abort;
 };
 
@@ -268,11 +269,14 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
 }
 
 // kProf: phase profile compiled in; kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256);
-// GRP: float4 column groups a reducer warp covers at once (its 32 lanes = GRP groups x 32/GRP row classes)
-template <int DT, int NCH, bool kFull, bool kProf, int GRP>
+// GRP: float4 column groups a reducer warp covers at once (its 32 lanes = GRP groups x 32/GRP row classes);
+// SETW: warps per consumer set -- 8: two sets of 256 threads; 16: one set of 512 threads (rows too long for
+// two rings and two hand-over buffers: thread t then owns chunks t, t + 512)
+template <int DT, int NCH, bool kFull, bool kProf, int GRP, int SETW = 8>
 __global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
+    constexpr int kSets = 16 / SETW, kSetWarps = SETW, kSetThreads = SETW * 32;   // shadow the two-set defaults
     const int rec_bytes = P.d_model * 6;
     const int nstage = P.nstage;               // total over both sets (even)
     const int S = nstage / kSets;              // ring stages per consumer set
@@ -317,7 +321,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         const unsigned FULL = 0xFFFFFFFFu;
         const int hq = lane >> 4, hl = lane & 15;      // walker role
         const bool mine = lane < kSets * S;            // issue role
-        const int iq = mine ? lane / S : 0, is = lane % S;
+        const int iq = mine ? lane / S : 0, is = lane % S;   // (iq < kSets)
         uint32_t n = is;                               // set-ring item index this lane issues next
         uint32_t iph = 0;                              // phase parity of that item's round through the ring
         uint32_t issued = 0;
@@ -327,16 +331,17 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         unsigned long long pf_src = 0; uint32_t pf_bytes = 0; int pf_meta = 0; bool pf_valid = false;
         bool pf_pending = false;
         const int vb = kSets * b + hq;
+        const int nvw = hq < kSets ? nv : 0;           // a half-warp without a set has nothing to walk
         auto prefetch_window = [&](bool doit) {
             int step = wstep, t = wt + hl;
             bool in = false;
             if (doit) {
                 StepGeom g;
-                in = step < nv;
+                in = step < nvw;
                 if (in) g = step_geom(P, step * NG + grp, Gv, vb);
                 while (in && t > g.cnt) {
                     t -= g.cnt + 1; ++step;
-                    in = step < nv;
+                    in = step < nvw;
                     if (in) g = step_geom(P, step * NG + grp, Gv, vb);
                 }
                 pf_valid = in;
@@ -391,7 +396,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             // keep each descriptor ring ahead of its set's slowest issue lane by at least a window
             uint32_t n_min = 0xFFFFFFFFu;
             for (int k = 0; k < S; ++k) {
-                const uint32_t v = __shfl_sync(FULL, n, hq * S + k);
+                const uint32_t v = __shfl_sync(FULL, n, (hq < kSets ? hq : 0) * S + k);
                 n_min = v < n_min ? v : n_min;
             }
             const bool do_commit = pf_pending && desc_ready - n_min <= (uint32_t)(kDescRing - 16 - kMaxStages);
@@ -446,7 +451,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         // computes.  Thread t of a set owns chunks t, t+256 of every row.
         const int cw = warp < 16 ? warp - (warp / 4 + 1) : warp - 4;   // consumer warp index 0..15
         const int ct = cw * 32 + lane;           // 0..511
-        const int q = ct >> 8;                   // consumer set
+        const int q = ct / kSetThreads;          // consumer set
         const int t = ct & (kSetThreads - 1);    // thread within the set
         const int sw = t >> 5;                   // warp within the set
         uint64_t *sfull = full + q * S, *sempty = empty + q * S;
@@ -483,7 +488,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     if (++st == S) { st = 0; ph ^= 1; }
                 }
                 // the record count steers the set's barriers: agree on it (and on failure) first
-                fail = set_barrier_or(q, fail);
+                fail = set_barrier_or<kSetThreads>(q, fail);
                 if (fail) break;
                 SI_PROF(0);                               // wait for x
                 for (int i = 0; i < cnt; ++i) {
@@ -531,7 +536,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     // ---- exchange among the set's 8 warps (double-buffered, one barrier per record)
                     const uint32_t buf = recs & 1;
                     if ((lane & 15) == 0) reinterpret_cast<float *>(&sm->setpart[q][buf][sw])[lane >> 4] = g;
-                    fail = set_barrier_or(q, fail);       // also orders the partials for the whole set
+                    fail = set_barrier_or<kSetThreads>(q, fail);       // also orders the partials for the whole set
                     SI_PROF(6);                           // 8-warp exchange
                     ++recs;
                     if (fail) break;
@@ -642,7 +647,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         long long t0 = clock64();
                         while (q < 0) {
                             if (!(taken & 1) && mbar_test_wait(&sm->accfull[0][r], par)) q = 0;
-                            else if (!(taken & 2) && mbar_test_wait(&sm->accfull[1][r], par)) q = 1;
+                            else if (kSets > 1 && !(taken & 2) && mbar_test_wait(&sm->accfull[kSets - 1][r], par)) q = 1;
                             else {
                                 if (*cta_abort || clock64() - t0 > kWaitCycles) break;
                                 __nanosleep(200);
@@ -756,14 +761,20 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
 // records.  More groups would give a CTA more column groups to reduce than a warp has lanes.
 inline int pick_groups(int n_sms) { return n_sms % 4 == 0 ? 4 : (n_sms % 2 == 0 ? 2 : 1); }
 
-inline size_t smem_bytes(int d_model, int nstage) {
-    return (size_t)nstage * d_model * 6 + (size_t)kSets * d_model * 4 + sizeof(Smem) + 64;
+inline size_t smem_bytes(int d_model, int nstage, int sets = kSets) {
+    return (size_t)nstage * d_model * 6 + (size_t)sets * d_model * 4 + sizeof(Smem) + 64;
 }
-inline int pick_stages(int d_model) {
+inline int pick_stages(int d_model, int sets = kSets) {
     const size_t budget = 227 * 1024;
-    int n = (int)((budget - smem_bytes(d_model, 0)) / ((size_t)d_model * 6));
+    if (smem_bytes(d_model, 0, sets) >= budget) return 0;
+    int n = (int)((budget - smem_bytes(d_model, 0, sets)) / ((size_t)d_model * 6));
     if (n > kMaxStages) n = kMaxStages;
-    return n & ~1;       // split evenly between the two consumer sets
+    return sets == 2 ? n & ~1 : n;       // split evenly between the consumer sets
+}
+// Rows too long for two sets (more than three chunks per thread of a 256-thread set, or no room for two
+// stages per ring): one consumer set of 512 threads, thread t owning chunks t and t + 512.
+inline bool wide_rows(int d_model) {
+    return d_model / 8 > kSetThreads * 3 || pick_stages(d_model) < 4;
 }
 
 }  // namespace si_persist
@@ -781,8 +792,10 @@ inline bool si_persistent_supported(const si_store *s) {
     // lanes cover the float4 column groups of a CTA
     const int chunks = s->d_model / 8, G = s->num_sms;
     const int gpc = (s->d_model / 4 + G - 1) / G;
-    return s->n_layers <= SI_MAX_LAYERS && si_persist::pick_stages(s->d_model) >= 4 &&
-           chunks <= si_persist::kSetThreads * 3 && gpc <= si_persist::kMaxGroups;
+    if (s->n_layers > SI_MAX_LAYERS || gpc > si_persist::kMaxGroups) return false;
+    if (si_persist::wide_rows(s->d_model))      // one set of 512 threads, two chunks per thread, at least three ring stages
+        return chunks <= si_persist::kSetThreads * 4 && si_persist::pick_stages(s->d_model, 1) >= 3;
+    return si_persist::pick_stages(s->d_model) >= 4 && chunks <= si_persist::kSetThreads * 3;
 }
 
 // Bytes of the partial-y ring.
@@ -790,10 +803,10 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, bool FULL, bool PROF, int GRP>
+template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP>;
-    size_t smem = si_persist::smem_bytes(P.d_model, P.nstage);
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP, SETW>;
+    size_t smem = si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW);
     static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
     int dev = 0;
     SI_CUDA_TRY(cudaGetDevice(&dev));
@@ -814,7 +827,8 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.store_base = s->mem;
     for (int l = 0; l < s->n_layers; ++l) { P.rec_off[l] = s->rec_off[l]; P.n_loaded[l] = s->n_loaded[l]; }
     P.n_layers = s->n_layers; P.n_steps = n_steps; P.k_fixed = k_fixed; P.d_model = s->d_model;
-    P.chunks = s->d_model / 8; P.nstage = si_persist::pick_stages(s->d_model);
+    const bool wide = si_persist::wide_rows(s->d_model);
+    P.chunks = s->d_model / 8; P.nstage = si_persist::pick_stages(s->d_model, wide ? 1 : 2);
     P.step_layers = nullptr; P.n_few = 0;
     // steps region: [n_steps] layer ids | control words (256 bytes) | [n_steps][64] counters
     int32_t *steps = (int32_t *)(wsb + ws.steps_off);
@@ -834,7 +848,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.status = status_dev;
     P.prof = si_decode_profile_buffer();
     P.stream_only = si_decode_stream_only() & 0xFF;
-    if ((si_decode_stream_only() >> 8) & 0xF) P.nstage = 2 * ((si_decode_stream_only() >> 8) & 0xF);   // diagnostics: shallower rings
+    if (((si_decode_stream_only() >> 8) & 0xF) && !wide) P.nstage = 2 * ((si_decode_stream_only() >> 8) & 0xF);   // diagnostics: shallower rings
     int G = s->num_sms;
     if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
     // every CTA reduces at most kMaxGroups float4 column groups
@@ -854,8 +868,9 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     const int gpc = (s->d_model / 4 + G / ng - 1) / (G / ng);       // column groups per CTA -> lanes of a reducer warp
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
-    const int nch = (P.chunks + si_persist::kSetThreads - 1) / si_persist::kSetThreads;
-    const bool full = P.chunks == nch * si_persist::kSetThreads;
+    const int set_threads = wide ? 2 * si_persist::kSetThreads : si_persist::kSetThreads;
+    const int nch = (P.chunks + set_threads - 1) / set_threads;
+    const bool full = P.chunks == nch * set_threads;
     // the phase profile is a separate instantiation: the production kernel carries no clock reads
 #define SI_PL3(DT, N, F, PR) (gpc <= 8 ? si_decode_persistent_launch_t<DT, N, F, PR, 8>(P, G, stream)    \
                               : gpc <= 16 ? si_decode_persistent_launch_t<DT, N, F, PR, 16>(P, G, stream) \
@@ -867,6 +882,12 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
 #define SI_PL(DT) (nch <= 1 ? (full ? SI_PL2(DT, 1, true) : SI_PL2(DT, 1, false))     \
                    : nch <= 2 ? (full ? SI_PL2(DT, 2, true) : SI_PL2(DT, 2, false)) \
                               : (full ? SI_PL_W(DT, true) : SI_PL_W(DT, false)))
+    // wide rows: one set of 16 warps, two chunks per thread, no phase profile
+#define SI_PL_X(DT, F) (gpc <= 16 ? si_decode_persistent_launch_t<DT, 2, F, false, 16, 16>(P, G, stream) \
+                                  : si_decode_persistent_launch_t<DT, 2, F, false, 32, 16>(P, G, stream))
+    if (wide) return s->dtype == SI_BF16 ? (full ? SI_PL_X(SI_BF16, true) : SI_PL_X(SI_BF16, false))
+                                         : (full ? SI_PL_X(SI_F16, true) : SI_PL_X(SI_F16, false));
+#undef SI_PL_X
     return s->dtype == SI_BF16 ? SI_PL(SI_BF16) : SI_PL(SI_F16);
 #undef SI_PL2
 #undef SI_PL3

@@ -18,7 +18,8 @@ SHAPES = [
     (4096, 1024, "f16"),
     (5120, 1024, "bf16"),     # three chunks per thread in the persistent kernel, ragged
     (6144, 800, "f16"),       # three full chunks per thread, two ring stages per consumer set
-    (8192, 640, "bf16"),
+    (7168, 700, "bf16"),      # one consumer set of 512 threads in the persistent kernel, ragged
+    (8192, 640, "bf16"),      # the same with full rows
 ]
 
 
