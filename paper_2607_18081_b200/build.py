@@ -34,6 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     srcs = [os.path.join(CSRC, f) for f in SOURCES if os.path.exists(os.path.join(CSRC, f))]
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "--threads", "0",                       # the sources compile side by side
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "shared", "-I", os.path.join(ROOT, "include"),
            "-I", CSRC, "-o", tmp] + srcs
     if verbose:
