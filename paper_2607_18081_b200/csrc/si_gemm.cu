@@ -347,8 +347,8 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         return;
     }
     const int ks = blockIdx.x % ns, mt = (blockIdx.x / ns) % n_real, tt = blockIdx.x / (ns * n_real);
-    const int k_per = (P.d_model / kChunkK + ns - 1) / ns;         // chunks per split
-    const int c0 = ks * k_per, c1 = min(P.d_model / kChunkK, c0 + k_per);
+    const int total_k = P.d_model / kChunkK;                       // chunks; split ks takes an even share of them
+    const int c0 = (int)((long long)ks * total_k / ns), c1 = (int)((long long)(ks + 1) * total_k / ns);
     const int n_chunks = c1 > c0 ? c1 - c0 : 0;
     const int tok0 = tt * N;
 
