@@ -77,3 +77,27 @@ def test_layer_range_matches_the_papers_layer_counts():
     import pytest
     with pytest.raises(api.SelectInferError):
         api.si_layer_range(6, 5, -2)
+
+
+def test_shard_entry_points_host_side():
+    """Neuron shards: the share sizes and the argument checks need no GPU."""
+    from paper_2607_18081_b200 import api
+    for n, world in ((10, 3), (7705, 8), (5, 8), (0, 2), (1, 1)):
+        counts = [api.si_shard_count(n, r, world) for r in range(world)]
+        assert sum(counts) == n and max(counts) - min(counts) <= 1
+        assert counts == [len(range(r, n, world)) for r in range(world)]
+    lib, null = api.lib(), ctypes.c_void_p(0)
+    out = ctypes.c_int(0)
+    assert lib.si_shard_count(10, 3, 3, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG       # rank outside the world
+    assert lib.si_shard_count(10, 0, 0, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG
+    assert lib.si_shard_count(-1, 0, 2, ctypes.byref(out)) == api.SI_ERR_INVALID_ARG
+    # null outputs, a rank outside the world, a workspace that is too small: refused before any launch
+    buf = ctypes.c_void_p(0x1000)
+    assert lib.si_shard_lists(buf, null, 4, 2, 0, 2, null, buf, buf, 4096, null, null) == api.SI_ERR_INVALID_ARG
+    assert lib.si_shard_lists(buf, null, 4, 2, 2, 2, buf, buf, buf, 4096, null, null) == api.SI_ERR_INVALID_ARG
+    assert lib.si_shard_lists(buf, null, 4, 2, 0, 2, buf, buf, buf, 16, null, null) == api.SI_ERR_NOMEM
+    assert lib.si_shard_reduce(null, 2, null, api.SI_BF16, 1, 64, buf, api.SI_F32, 0, null) == api.SI_ERR_INVALID_ARG
+    assert lib.si_shard_reduce(buf, 0, null, api.SI_BF16, 1, 64, buf, api.SI_F32, 0, null) == api.SI_ERR_INVALID_ARG
+    assert lib.si_shard_reduce(buf, 2, null, api.SI_BF16, 1, 64, buf, api.SI_F32, api.SI_FLAG_RESIDUAL, null) == \
+        api.SI_ERR_INVALID_ARG                                                              # residual without x
+    assert lib.si_shard_reduce(buf, 2, null, api.SI_F32, 1, 64, buf, api.SI_F32, 0, null) == api.SI_ERR_INVALID_ARG
