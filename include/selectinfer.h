@@ -78,6 +78,10 @@ enum {
     SI_FLAG_LIST_PER_LAYER = 64u, /* si_decode_stack_forward, fixed-length lists only: idx holds ONE list per layer
                                     ([n_layers, k_fixed]) and every step uses the list of its layer -- the paper's
                                     decode, where the set chosen during prefill stays fixed for the prompt */
+    SI_FLAG_STEPS_ANY_ORDER = 128u, /* si_decode_stack_forward: the caller states that the steps do not depend on one
+                                    another and may be computed in any order and several at a time: the SMs then
+                                    work in up to four groups that each take every fourth step.  Without the flag
+                                    every SM works through the steps in their order. */
     SI_FLAG_SIMPLE_KERNELS = 256u /* decode: one plain-load kernel pair per step instead of the
                                      persistent bulk-copy kernel (kept for cross-checking) */
 };
@@ -183,10 +187,12 @@ int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, c
 /* Batch-1 decode over a stack: n_steps consecutive (token, layer) steps in one
  * persistent launch, step s using layer layers[s] (HOST int32 [n_steps], or NULL for
  * s mod n_layers).  x, y: device [n_steps, d_model]; idx: device [n_steps, k_fixed]
- * (or CSR over n_steps lists).  The steps are independent -- every step's x is an input of
- * the call -- and several are in flight at once: the SMs work in up to four groups that each
- * take every fourth step, and within a group the weight stream of later steps is prefetched
- * while earlier steps finish.  All of y is complete when the call's work on the stream is.
+ * (or CSR over n_steps lists).  Every SM works through the steps in their order; the weight
+ * stream of later steps is prefetched while earlier steps finish, and a step's sum over the
+ * SMs completes a few steps behind the stream.  With SI_FLAG_STEPS_ANY_ORDER -- every step's x
+ * is an input of the call, so nothing in the call depends on the order -- the SMs work in up to
+ * four groups that each take every fourth step on their own, which divides the fixed work of a
+ * step by the number of groups.  All of y is complete when the call's work on the stream is.
  * Results equal n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of
  * a list over SMs depends on the step's position in the call); each is run-to-run bit-stable.
  * With SI_FLAG_LIST_PER_LAYER (fixed-length lists only) idx is [n_layers, k_fixed] and a step
@@ -278,8 +284,9 @@ int si_debug_decode_profile(void *dev_buf);
  * part of the work (1: the arithmetic, 2: the loads of the cross-SM reduction, 4: the cross-SM
  * exchange altogether; y is then meaningless) -- timing such a launch gives the practical ceiling of
  * the record stream on the same lists.  Bits 8..11: ring stages per consumer set (0 = as many as
- * fit).  Bits 12..15: number of step groups the SMs are split into (0 = the library's choice, 4 on
- * 148 SMs; used by the tests to cover 1, 2 and 4 groups).  Results stay correct for every value of
+ * fit).  Bits 12..15: number of step groups the SMs are split into, whatever the call's flags say
+ * (0 = the library's choice: one, or up to four with SI_FLAG_STEPS_ANY_ORDER; used by the tests to
+ * cover 1, 2 and 4 groups).  Results stay correct for every value of
  * bits 8..15. */
 int si_debug_decode_stream_only(int on);
 

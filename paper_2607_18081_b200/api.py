@@ -26,6 +26,7 @@ SI_FLAG_CHECK, SI_FLAG_RESIDUAL, SI_FLAG_UNION_UNMASKED, SI_FLAG_SCORE_ABS = 1, 
 SI_FLAG_SHARED_LIST = 16
 SI_FLAG_UNION_PATH = 32
 SI_FLAG_LIST_PER_LAYER = 64
+SI_FLAG_STEPS_ANY_ORDER = 128
 SI_FLAG_SIMPLE_KERNELS = 256
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 

@@ -80,8 +80,9 @@ extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x,
         if (!(ip >= w0 && ip < w0 + decode_total)) {
             int32_t ls[kDecodeRouteMaxT];
             for (int t = 0; t < T; ++t) ls[t] = layer;
-            return si_decode_launch(store, T, ls, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
-                                    ws_bytes, status_dev, stream);
+            // the tokens of a call are independent of one another by definition
+            return si_decode_launch(store, T, ls, x, idx, idx_offsets, k_fixed, y, y_dtype, flags | SI_FLAG_STEPS_ANY_ORDER,
+                                    workspace, ws_bytes, status_dev, stream);
         }
     }
     return si_multi_token_launch(store, layer, x, T, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,

@@ -854,12 +854,13 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // every CTA reduces at most kMaxGroups float4 column groups
     const int g_min = (s->d_model / 4 + si_persist::kMaxGroups - 1) / si_persist::kMaxGroups;
     if (G < g_min) G = g_min;
-    // Step groups: the SMs are split into groups that each take every n-th step on their own (launches of
-    // at least two steps per group; a launch that uses fewer CTAs than SMs keeps one group).
+    // Step groups, for callers who state that the order of the steps does not matter: the SMs are split
+    // into groups that each take every n-th step on their own (launches of at least two steps per group;
+    // a launch that uses fewer CTAs than SMs keeps one group).
     int ng = 1;
     if (G == s->num_sms) {
         const int forced = (si_decode_stream_only() >> 12) & 0xF;   // diagnostics: force a group count
-        ng = forced ? forced : si_persist::pick_groups(s->num_sms);
+        ng = forced ? forced : ((flags & SI_FLAG_STEPS_ANY_ORDER) ? si_persist::pick_groups(s->num_sms) : 1);
         while (ng > 1 && (s->num_sms % ng != 0 || n_steps < 2 * ng ||
                           (s->d_model / 4 + s->num_sms / ng - 1) / (s->num_sms / ng) > si_persist::kMaxGroups))
             ng >>= 1;

@@ -233,8 +233,8 @@ def test_7b_shaped_two_layers_stack_and_determinism(api):
 
 
 def test_7b_shaped_step_groups(api):
-    """The persistent kernel with its SMs split into 1, 2 and 4 step groups (4 is the default for
-    launches of 8 steps or more): 13 steps, so the groups get 4, 3, 3 and 3 steps; lists of equal
+    """The persistent kernel with its SMs split into 1, 2 and 4 step groups (one by default, up to
+    four with SI_FLAG_STEPS_ANY_ORDER for launches of 8 steps or more): 13 steps, so the groups get 4, 3, 3 and 3 steps; lists of equal
     length, ragged lists with offsets (an empty one among them) and one list per layer; residual."""
     cfg = wl.CONFIGS["c2"]
     m = LoadedModel(cfg, n_layers=2)
@@ -259,13 +259,15 @@ def test_7b_shaped_step_groups(api):
     try:
         for name, idx, offsets, kk, flags, list_of in cases:
             refs = None
-            for ng in (1, 2, 4):
+            for ng in (1, 2, 4, 0):       # 0: the library's own choice under SI_FLAG_STEPS_ANY_ORDER
                 api.lib().si_debug_decode_stream_only(ng << 12)
                 runs = []
                 for _ in range(2):
                     y = torch.full((steps, cfg.d_model), 9.0, dtype=torch.float32, device="cuda")
                     st = _status()
-                    api.si_decode_stack_forward(m.store.handle, steps, None, xd, idx, offsets, kk, y, flags, ws, st)
+                    # (the debug knob fixes the group count; the flag is what a caller would pass for more than one)
+                    api.si_decode_stack_forward(m.store.handle, steps, None, xd, idx, offsets, kk, y,
+                                                flags | (api.SI_FLAG_STEPS_ANY_ORDER if ng != 1 else 0), ws, st)
                     torch.cuda.synchronize()
                     assert st.item() == 0, (name, ng, api.strerror(int(st.item())))
                     runs.append(y.cpu())
