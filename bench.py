@@ -36,7 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of si_decode_persistent_kernel per (token, layer) step
 # of the config-2 shape, from the capture summarised in
 # profiles/decode_persistent_c2_8layers_32tokens_full.md: (9.6461e9 + 0.2290e9) / 256 steps
-NCU_DRAM_BYTES_PER_C2_STEP = (9.3476e9 + 0.0749e9) / 256
+NCU_DRAM_BYTES_PER_C2_STEP = (9.6454e9 + 0.2272e9) / 256
 FALLBACK_HBM_GBS = 6650.0
 
 
