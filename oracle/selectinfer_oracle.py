@@ -9,6 +9,10 @@ cpu_baseline / reference legs may import this module.
   full weights with global neuron ids (C loops in ``si_oracle.c``; Section 3 for the
   neuron <-> weight-slice correspondence, Section 5 for "compute only the selected
   loaded neurons").
+* ``ffn_chain`` -- the FFN applied layer after layer (Section 4: the same for every FFN layer), each
+  step reading the output of the step before it, rounded to the model's 16-bit type; ``rmsnorm`` is
+  the gain-free RMS normalisation in front of the FFN of the paper's pre-norm models and ``round_bits``
+  the rounding (both library-pinned).
 * ``select_topk`` -- Section 5: sort activations in descending order, keep the top
   alpha, record their indices.  Tie-break (paper silent): lower index wins; +0 == -0;
   NaN ranks below everything.  Output ascending by index.
@@ -142,6 +146,59 @@ def ffn_tokens(Wg, Wu, Wd, X, lists, dtype: str = "f64", threads: int = 1):
     if rc:
         raise ValueError("neuron ids must be distinct and in [0, d_ff)")
     return Y
+
+
+# --------------------------------------------------------------------------- chained layers
+
+def round_bits(v, dtype: str) -> np.ndarray:
+    """float64 values -> fp16 / bf16 bit patterns, round to nearest even (through float32, as a model
+    that keeps its hidden state in a 16-bit type does)."""
+    f = np.asarray(v, dtype=np.float64).astype(np.float32)
+    if dtype == "f16":
+        return f.astype(np.float16).view(np.uint16)
+    u = f.view(np.uint32).astype(np.uint64)
+    nan = np.isnan(f)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+    r[nan] = 0x7FC0
+    return r
+
+
+def widen_bits(bits, dtype: str) -> np.ndarray:
+    """fp16 / bf16 bit patterns -> float64 (exact)."""
+    b = np.asarray(bits, dtype=np.uint16)
+    if dtype == "f16":
+        return b.view(np.float16).astype(np.float64)
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def rmsnorm(x, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) in float64: the normalisation a pre-norm transformer block applies in
+    front of its FFN, without the learned gain."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt(np.mean(x * x) + float(eps))
+
+
+def ffn_chain(layer_weights, layers, ids, lists, x0_bits, dtype: str, residual: bool = False, prenorm: bool = False,
+              eps: float = 0.0, threads: int = 1):
+    """One chain: step s runs the selective FFN of layer layers[s] (weights layer_weights[layers[s]],
+    global ids ids[layers[s]][lists[s]]) on the output of step s - 1; step 0 reads x0.  Per step:
+        in   = x0 or the rounded output of the step before          (16-bit)
+        xn   = round(rmsnorm(in))  if prenorm  else  in             (16-bit: what the dot products see)
+        out  = round((in if residual else 0) + FFN(xn))             (16-bit: what the next step reads)
+    Returns (out bits [steps, d], xn bits [steps, d], float64 outputs before rounding [steps, d])."""
+    cur = np.asarray(x0_bits, dtype=np.uint16)
+    outs, xns, raws = [], [], []
+    for s, layer in enumerate(layers):
+        xin = widen_bits(cur, dtype)
+        xn_bits = round_bits(rmsnorm(xin, eps), dtype) if prenorm else cur
+        wg, wu, wd = layer_weights[layer]
+        gids = np.asarray(ids[layer])[np.asarray(lists[s], dtype=np.int64)] if len(lists[s]) else np.zeros(0, np.int32)
+        y = ffn(wg, wu, wd, xn_bits, gids, dtype=dtype, threads=threads)
+        if residual:
+            y = y + xin
+        cur = round_bits(y, dtype)
+        outs.append(cur); xns.append(xn_bits); raws.append(y)
+    return np.stack(outs), np.stack(xns), np.stack(raws)
 
 
 # --------------------------------------------------------------------------- selection

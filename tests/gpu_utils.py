@@ -7,6 +7,11 @@ from paper_2607_18081_b200 import workloads as wl
 
 MAX_ERR = 2e-2      # max|err| <= 2e-2 * max|y_ref|   (per token)
 MEAN_REL = 5e-3     # mean|err| / mean|y_ref| <= 5e-3 (per token)
+# fp32 outputs of the decode kernels: 16-bit inputs are widened exactly and every product and sum is
+# fp32, so the error against float64 is a few fp32 roundings of a sum of up to ~10^4 terms of mixed sign
+# (observed ~1e-6 of max|y_ref|).  A dropped column group, record or split shows up at 1e-2 and more.
+F32_MAX_ERR = 5e-5
+F32_MEAN_REL = 2e-5
 
 
 def to_dev(bits: np.ndarray, dtype: str) -> torch.Tensor:
@@ -53,4 +58,12 @@ def assert_close(y, y_ref, what=""):
     from oracle import selectinfer_oracle as so
     e_max, e_mean = so.error_metrics(y, y_ref)
     assert e_max <= MAX_ERR and e_mean <= MEAN_REL, f"{what}: max-rel {e_max:.3e}, mean-rel {e_mean:.3e}"
+    return e_max, e_mean
+
+
+def assert_close_f32(y, y_ref, what=""):
+    """Tight bound for fp32 outputs of the decode kernels (no 16-bit rounding anywhere on the way)."""
+    from oracle import selectinfer_oracle as so
+    e_max, e_mean = so.error_metrics(y, y_ref)
+    assert e_max <= F32_MAX_ERR and e_mean <= F32_MEAN_REL, f"{what}: max-rel {e_max:.3e}, mean-rel {e_mean:.3e} (fp32 bound)"
     return e_max, e_mean

@@ -398,3 +398,143 @@ def test_shard_lists_hand_example():
     assert so.shard_lists([l], 1, 3)[0].tolist() == [0, 1]         # slots 1, 4 -> local 0, 1
     assert so.shard_lists([l], 2, 3)[0].tolist() == [2]            # slot 8 -> local 2
     assert so.shard_slots(10, 1, 3).tolist() == [1, 4, 7]
+
+
+# ------------------------------------------------------------------ the error measure of the parity tests
+
+def test_error_metrics_hand_worked_values():
+    """error_metrics carries every FFN parity assertion, so it is pinned on vectors worked by hand:
+    y_ref = (4, -2, 0, 1), y = (4.5, -2, -0.25, 1)  =>  |err| = (0.5, 0, 0.25, 0);
+    max|err| / max|y_ref| = 0.5 / 4 = 0.125;  mean|err| / mean|y_ref| = 0.1875 / 1.75 = 3/28.
+    The two ratios differ, each differs from the figure a swapped max/mean would give (0.5 / 1.75,
+    0.1875 / 4), and normalising by y instead of y_ref would give 0.5 / 4.5."""
+    y_ref = np.array([4.0, -2.0, 0.0, 1.0])
+    y = np.array([4.5, -2.0, -0.25, 1.0])
+    e_max, e_mean = so.error_metrics(y, y_ref)
+    assert e_max == 0.125
+    assert e_mean == pytest.approx(3.0 / 28.0, rel=1e-15)
+    # a negative error counts by its size; the sign of the reference does not matter
+    assert so.error_metrics(-y, -y_ref) == (e_max, e_mean)
+    assert so.error_metrics(2 * y_ref - y, y_ref) == (e_max, e_mean)
+    # the reference normalises, not the value under test
+    e2 = so.error_metrics(y_ref, y)
+    assert e2[0] == pytest.approx(0.5 / 4.5, rel=1e-15) and e2[1] == pytest.approx(0.1875 / 1.9375, rel=1e-15)
+    # exact agreement is exactly zero; one wrong element of many moves the max ratio, barely the mean ratio
+    assert so.error_metrics(y_ref, y_ref) == (0.0, 0.0)
+    big_ref = np.ones(1000)
+    big = big_ref.copy()
+    big[123] = 1.5
+    e_max, e_mean = so.error_metrics(big, big_ref)
+    assert e_max == 0.5 and e_mean == pytest.approx(0.5 / 1000, rel=1e-12)
+    # a reference of zeros: the raw errors come back (nothing to divide by)
+    assert so.error_metrics(np.array([0.25, -0.5]), np.zeros(2)) == (0.5, 0.375)
+    # 16-bit and fp32 inputs are widened, not truncated
+    assert so.error_metrics(np.array([1.5], dtype=np.float32), np.array([1.0], dtype=np.float16)) == (0.5, 0.5)
+
+
+def test_parity_tolerances_are_the_stated_ones():
+    """The GPU parity helper uses the stated bounds -- max|err| <= 2e-2 max|y_ref| and
+    mean|err| / mean|y_ref| <= 5e-3 per token -- and fails just outside either."""
+    from tests import gpu_utils
+    assert gpu_utils.MAX_ERR == 2e-2 and gpu_utils.MEAN_REL == 5e-3
+    ref = np.ones(100)
+    ok = ref.copy(); ok[0] = 1.0 + 1.9e-2                     # max ratio 1.9e-2, mean ratio 1.9e-4
+    gpu_utils.assert_close(ok, ref)
+    bad_max = ref.copy(); bad_max[0] = 1.0 + 2.1e-2
+    with pytest.raises(AssertionError):
+        gpu_utils.assert_close(bad_max, ref)
+    bad_mean = ref + 5.1e-3                                    # max ratio 5.1e-3 passes, mean ratio 5.1e-3 does not
+    with pytest.raises(AssertionError):
+        gpu_utils.assert_close(bad_mean, ref)
+    gpu_utils.assert_close(ref + 4.9e-3, ref)
+    # the tight bound used for fp32 outputs of the decode kernels
+    assert gpu_utils.F32_MAX_ERR <= 1e-4
+    with pytest.raises(AssertionError):
+        gpu_utils.assert_close_f32(ref + 2e-4, ref)
+    gpu_utils.assert_close_f32(ref + 1e-6, ref)
+
+
+# ------------------------------------------------------------------ chained layers: rounding, normalisation, chain
+
+@pytest.mark.parametrize("dtype,tdt", [("bf16", torch.bfloat16), ("f16", torch.float16)])
+def test_round_bits_matches_library_rounding(dtype, tdt):
+    """Round-to-nearest-even to the 16-bit types against torch's conversion, ties and specials included."""
+    g = np.random.default_rng(11)
+    v = np.concatenate([g.normal(0, 1, 4000), g.normal(0, 1e-3, 1000), g.normal(0, 300, 1000),
+                        [0.0, -0.0, 1.0, -1.0, np.inf, -np.inf, 65504.0, 1e-8]])
+    if dtype == "bf16":
+        # exact ties: 1 + 2^-8 lies halfway between two bf16 values (-> even: 1.0); 1 + 3 * 2^-8 -> 1 + 2^-6
+        v = np.concatenate([v, [1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8)]])
+    else:
+        v = np.concatenate([v, [1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 6e-8, 2.0 ** -24, 2.0 ** -25]])
+    bits = so.round_bits(v, dtype)
+    ref = torch.from_numpy(v.astype(np.float32)).to(tdt).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(bits, ref)
+    # widening is the exact inverse on representable values
+    back = so.widen_bits(bits, dtype)
+    assert np.array_equal(so.round_bits(back, dtype), bits)
+    assert np.array_equal(back, torch.from_numpy(ref.view(np.int16)).view(tdt).to(torch.float64).numpy())
+    if dtype == "bf16":
+        assert so.widen_bits(so.round_bits([1.0 + 2.0 ** -8], dtype), dtype)[0] == 1.0
+        assert so.widen_bits(so.round_bits([1.0 + 3 * 2.0 ** -8], dtype), dtype)[0] == 1.0 + 2.0 ** -6
+
+
+def test_rmsnorm_closed_forms_and_library():
+    """x = (3, 4): mean square 12.5, so the result is (3, 4) / sqrt(12.5); unit RMS after normalising with
+    eps = 0; scale invariance; eps in the right place; torch's rms_norm in float64."""
+    y = so.rmsnorm([3.0, 4.0], 0.0)
+    np.testing.assert_allclose(y, np.array([3.0, 4.0]) / math.sqrt(12.5), rtol=1e-15)
+    np.testing.assert_allclose(so.rmsnorm([3.0, 4.0], 3.5), np.array([3.0, 4.0]) / 4.0, rtol=1e-15)   # 12.5 + 3.5 = 16
+    g = np.random.default_rng(5)
+    x = g.normal(0, 3, 257)
+    y = so.rmsnorm(x, 0.0)
+    assert abs(np.sqrt(np.mean(y * y)) - 1.0) < 1e-14
+    np.testing.assert_allclose(so.rmsnorm(7.5 * x, 0.0), y, rtol=1e-13)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (257,), eps=1e-5).numpy()
+    np.testing.assert_allclose(so.rmsnorm(x, 1e-5), ref, rtol=1e-13)
+    # a sum in place of the mean, or eps outside the root, must fail: they differ visibly
+    assert np.max(np.abs(x / np.sqrt(np.sum(x * x) + 1e-5) - ref)) > 1e-2
+    assert np.max(np.abs(x / (np.sqrt(np.mean(x * x)) + 0.5) - so.rmsnorm(x, 0.5))) > 1e-3
+
+
+def test_ffn_chain_is_the_ffn_applied_step_after_step():
+    """The chain against its definition written out with the pinned pieces, on a tiny two-layer model:
+    rounding between steps, the residual taken from the step's own input, the normalised row fed to
+    the FFN, lists and layers indexed per step."""
+    g = np.random.default_rng(21)
+    d_ff, d = 20, 16
+    mk = lambda *shape: so.round_bits(g.normal(0, 0.4, shape), "bf16")
+    weights = [(mk(d_ff, d), mk(d_ff, d), mk(d, d_ff)) for _ in range(2)]
+    ids = [g.permutation(d_ff)[:12].astype(np.int32) for _ in range(2)]
+    lists = [np.sort(g.permutation(12)[:k]).astype(np.int32) for k in (5, 7, 0, 12)]
+    layers = [0, 1, 1, 0]
+    x0 = so.round_bits(g.normal(0, 1, d), "bf16")
+    for residual in (False, True):
+        for prenorm in (False, True):
+            out, xn, raw = so.ffn_chain(weights, layers, ids, lists, x0, "bf16", residual=residual, prenorm=prenorm, eps=1e-5)
+            cur = x0
+            for s in range(4):
+                xin = so.widen_bits(cur, "bf16")
+                xs = so.round_bits(so.rmsnorm(xin, 1e-5), "bf16") if prenorm else cur
+                assert np.array_equal(xn[s], xs)
+                wg, wu, wd = weights[layers[s]]
+                y = so.ffn(wg, wu, wd, xs, ids[layers[s]][lists[s]], dtype="bf16")
+                if residual:
+                    y = y + xin
+                assert np.array_equal(raw[s], y)
+                cur = so.round_bits(y, "bf16")
+                assert np.array_equal(out[s], cur)
+            # the empty list of step 2: the FFN adds nothing
+            assert np.array_equal(raw[2], so.widen_bits(out[1], "bf16") if residual else np.zeros(d))
+    # float64 library evaluation of a two-step chain without rounding effects: weights and x chosen so
+    # that every intermediate is exactly representable is not possible in general, so compare loosely
+    out, _, raw = so.ffn_chain(weights, [0, 1], ids, [np.arange(12), np.arange(12)], x0, "bf16")
+    F = torch.nn.functional
+    W = [[torch.from_numpy(so.widen_bits(w, "bf16")) for w in ws] for ws in weights]
+    def dense(l, v):
+        sel = torch.from_numpy(ids[l].astype(np.int64))
+        return F.linear(F.silu(F.linear(v, W[l][0][sel])) * F.linear(v, W[l][1][sel]), W[l][2][:, sel])
+    y0 = dense(0, torch.from_numpy(so.widen_bits(x0, "bf16")))
+    np.testing.assert_allclose(raw[0], y0.numpy(), rtol=1e-12, atol=1e-14)
+    y1 = dense(1, torch.from_numpy(so.widen_bits(so.round_bits(y0.numpy(), "bf16"), "bf16")))
+    np.testing.assert_allclose(raw[1], y1.numpy(), rtol=1e-12, atol=1e-14)
