@@ -28,10 +28,14 @@
  *     anything is launched.  Errors only the device can see (an index out of range or
  *     a duplicate under SI_FLAG_CHECK, an expired bounded wait) are written to
  *     *status_dev (caller-owned int32 in device memory, may be NULL) as an SI_ERR_*
- *     code; the kernel then leaves y unspecified but never reads or writes out of
- *     bounds and never hangs.  A status word is only ever overwritten with an error,
+ *     code; the kernel then leaves y unspecified but never hangs, and slot indices never
+ *     lead to an access outside the store.  CSR offsets (idx_offsets) are trusted unless
+ *     SI_FLAG_CHECK is given, which verifies that they start at or above 0, never decrease
+ *     and describe lists of at most k_fixed entries (SI_ERR_OUT_OF_RANGE otherwise).  A status word is only ever overwritten with an error,
  *     so the caller clears it.
  *   - All device pointers must be 16-byte aligned; d_model must be a multiple of 64.
+ *   - A store belongs to the device that was current when it was created; that device must
+ *     be current in every call that launches work on it (SI_ERR_INVALID_ARG otherwise).
  *   - Active lists hold SLOT indices (positions in the layer's store), distinct.
  *     The list order does not change the result: contributions are accumulated in a
  *     fixed order chosen by the library, so repeated calls are bit-identical.
@@ -82,8 +86,10 @@ enum {
                                     another and may be computed in any order and several at a time: the SMs then
                                     work in up to four groups that each take every fourth step.  Without the flag
                                     every SM works through the steps in their order. */
-    SI_FLAG_SIMPLE_KERNELS = 256u /* decode: one plain-load kernel pair per step instead of the
+    SI_FLAG_SIMPLE_KERNELS = 256u, /* decode: one plain-load kernel pair per step instead of the
                                      persistent bulk-copy kernel (kept for cross-checking) */
+    SI_FLAG_PRENORM = 512u       /* si_decode_chain_forward: the FFN sees its input scaled to unit root mean
+                                    square, as the FFN of a pre-norm transformer block does */
 };
 
 /* selection modes for si_select */
@@ -168,7 +174,8 @@ int si_select(const float *scores, int n, int mode, int k, float tau, unsigned f
  * runs a gathered tensor-core contraction in which token t still uses exactly its own
  * list (unless SI_FLAG_UNION_UNMASKED).  Up to 4 tokens with lists of their own are taken
  * through the decode kernel one after the other instead, which is faster there; the result
- * is the same function of the inputs, and SI_FLAG_UNION_PATH forces the union path.  An
+ * is the same function of the inputs, and SI_FLAG_UNION_PATH forces the union path (also for a
+ * single token; the workspace must then be sized for T_max = 2).  An
  * empty list gives y = 0 (or x with SI_FLAG_RESIDUAL).  Accumulation is fp32; h is rounded
  * to the store dtype before the down projection only on the union path. */
 int si_ffn_forward(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
@@ -202,6 +209,36 @@ int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t 
                             int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
                             size_t ws_bytes, int32_t *status_dev, void *stream);
 
+/* Batch-1 decode over a stack whose steps depend on one another: step s + 1 takes the output of step s
+ * as its input, the way the FFN of layer l + 1 sees what layer l produced ("applied to each FFN layer",
+ * Section 4; decoding with the neuron set chosen for the prompt, Section 5).  The steps come in chains
+ * of chain_len: step s with s mod chain_len == 0 starts a chain and reads row s / chain_len of x; every
+ * other step reads row s - 1 of y.  One token through all layers is a chain of n_layers steps.
+ *   x   : device [ceil(n_steps / chain_len), d_model], store dtype: the input of every chain
+ *   y   : device [n_steps, d_model], STORE dtype (a step's output is the next step's input, so it is
+ *         rounded once, to the type the FFN reads)
+ *   flags: SI_FLAG_RESIDUAL  y_s = in_s + FFN(...) with in_s the step's input row;
+ *          SI_FLAG_PRENORM   FFN(in_s) is replaced by FFN(n(in_s)), n(v) = v / sqrt(mean(v^2) + norm_eps)
+ *                            rounded to the store dtype: the (gain-free) RMS normalisation in front of
+ *                            the FFN of a pre-norm block.  Without it the scale of a chain drifts by the
+ *                            square per step (h is a product of two projections of the input), so chains
+ *                            longer than a few steps leave the range of 16-bit types; the paper's models
+ *                            normalise in front of every FFN.  The sum of squares is formed in fp32 in
+ *                            a fixed order, so the result is run-to-run bit-stable;
+ *          SI_FLAG_LIST_PER_LAYER, SI_FLAG_CHECK as for si_decode_stack_forward.
+ *   xn_out: optional device [n_steps, d_model], store dtype: with SI_FLAG_PRENORM, the normalised and
+ *         rounded row every step fed to its dot products (for inspection); NULL otherwise.
+ *   layers, idx, idx_offsets, k_fixed, workspace (si_workspace_bytes with max_steps >= n_steps),
+ *   status_dev, stream: as for si_decode_stack_forward.
+ * No arithmetic of step s + 1 starts before row s of y is complete on every SM; what runs ahead is the
+ * weight stream: the lists are inputs of the call (the set is fixed per prompt), so the first records of
+ * step s + 1 are already in shared memory when its input arrives.  All steps run in one persistent
+ * launch; hidden sizes the persistent kernel does not cover return SI_ERR_UNSUPPORTED. */
+int si_decode_chain_forward(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len,
+                            const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                            void *y, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                            size_t ws_bytes, int32_t *status_dev, void *stream);
+
 /* Batch-1 selective FFN for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of si_ffn_forward with T = 1.)
  *
@@ -216,7 +253,8 @@ int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t 
  *   flags: SI_FLAG_RESIDUAL only (others are ignored).
  * Limits: d_model <= 8192 and at most 152 SMs; beyond that the call returns SI_ERR_TOO_LARGE and
  * launches nothing.  The call never allocates or frees memory, directly or through a library.
- * The first call on each device looks up the array's device address (the device must be current);
+ * The store's device must be current (SI_ERR_INVALID_ARG otherwise).
+ * The first call on each device looks up the array's device address;
  * make that first call outside any stream capture.  All calls on a device share the one array:
  * it needs no clearing between calls (each call overwrites what it later reads), but two calls
  * whose kernels overlap on the GPU -- different streams without ordering -- race on it.  Results
@@ -270,32 +308,6 @@ int si_prefill_forward(const si_store_t *store, int layer, const void *x, int T,
                        int alpha, int beta, int n_static, int phi_count, unsigned flags, int32_t *idx_out,
                        int cap, int32_t *n_out, float *acts_out, void *workspace, size_t ws_bytes,
                        void *vote_workspace, size_t vote_ws_bytes, int32_t *status_dev, void *stream);
-
-/* Diagnostics: while dev_buf (device int64 [num_SMs][16]) is set, each persistent decode
- * launch stores per-SM cycle counts of its phases there.  Slots 0..5: first consumer set (wait
- * for x, wait for a record + copy to registers, record arithmetic, accumulator hand-over,
- * wait for the hand-over buffer, dot products + exchange); 6..7: second set (wait for the
- * hand-over buffer, wait for a record); 8..13: first reducer warp (idle, wait for a free
- * partial-ring slot, copy accumulators out, publish, wait for all SMs, reduce + write y).
- * Pass NULL to switch it off.  Costs a few clock reads per record. */
-int si_debug_decode_profile(void *dev_buf);
-
-/* Diagnostics, a bit field (0 = normal operation).  Bits 0..2: persistent decode launches leave out
- * part of the work (1: the arithmetic, 2: the loads of the cross-SM reduction, 4: the cross-SM
- * exchange altogether; y is then meaningless) -- timing such a launch gives the practical ceiling of
- * the record stream on the same lists.  Bits 8..11: ring stages per consumer set (0 = as many as
- * fit).  Bits 12..15: number of step groups the SMs are split into, whatever the call's flags say
- * (0 = the library's choice: one, or up to four with SI_FLAG_STEPS_ANY_ORDER; used by the tests to
- * cover 1, 2 and 4 groups).  Results stay correct for every value of
- * bits 8..15. */
-int si_debug_decode_stream_only(int on);
-
-/* Diagnostics: one launch that reads `bytes` bytes (a multiple of 16) at the 16-byte-aligned device
- * pointer `mem` once with plain 16-byte loads, all SMs busy, and stores a checksum of them in
- * *checksum_dev (device uint32).  Timing it on the neuron store gives the read bandwidth a kernel
- * with no other work reaches on this GPU, the practical ceiling quoted beside the decode kernel.  The
- * paper has no counterpart. */
-int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream);
 
 /* ---------------------------------------------------------------- offline: profiler and load set
  *

@@ -1,0 +1,79 @@
+/*
+ * selectinfer_debug.h -- diagnostics of libselectinfer: entry points for tests and measurements.
+ *
+ * Nothing here is part of the method (the paper has no counterpart to any of it) and nothing here
+ * keeps state between calls: every knob is an argument of the call it applies to.
+ */
+#ifndef SELECTINFER_DEBUG_H
+#define SELECTINFER_DEBUG_H
+
+#include "selectinfer.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Options of one persistent decode launch.  All zero = normal operation. */
+typedef struct si_debug_decode_opts {
+    int skip_mask;         /* bit 0: leave out the arithmetic; bit 1: the loads of the cross-SM sum; bit 2: the
+                              cross-SM exchange altogether.  y is then meaningless; timing such a launch gives
+                              the practical ceiling of the record stream on the same lists. */
+    int ring_stages;       /* ring stages per consumer set (0 = as many as fit); results stay correct */
+    int step_groups;       /* step groups the SMs are split into, whatever the flags say (0 = the library's
+                              choice: one, or up to four with SI_FLAG_STEPS_ANY_ORDER); results stay correct */
+    int withhold;          /* 1: the producer warp of the first CTA never issues the second item of its first
+                              ring, so that CTA's consumers wait for a record that does not come: with a short
+                              wait_cycles this exercises the time-out path (status SI_ERR_TIMEOUT, grid-wide
+                              abort, clean return).  Nothing faults and no wait is unbounded. */
+    long long wait_cycles; /* limit of every device-side wait in clock cycles (0 = the default, about 2 s) */
+    void *profile;         /* device int64 [num_SMs][16] or NULL: per-SM cycle counts of the phases.  Slots 0..5:
+                              first consumer set (wait for x, wait for a record + copy to registers, record
+                              arithmetic, accumulator hand-over, wait for the hand-over buffer, dot products +
+                              exchange); 6..7: second set (wait for the hand-over buffer, wait for a record);
+                              8..13: first reducer warp (idle, wait for a free partial-ring slot, copy
+                              accumulators out, publish, wait for all SMs, reduce + write y). */
+} si_debug_decode_opts_t;
+
+/* si_decode_stack_forward with the options above (opts == NULL: identical to it). */
+int si_debug_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
+                                  const void *x, const int32_t *idx, const int32_t *idx_offsets,
+                                  int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
+                                  size_t ws_bytes, int32_t *status_dev, void *stream,
+                                  const si_debug_decode_opts_t *opts);
+
+/* si_decode_chain_forward with the options above (step_groups is ignored: a chain has one). */
+int si_debug_decode_chain_forward(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len,
+                                  const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                                  void *y, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                                  size_t ws_bytes, int32_t *status_dev, void *stream,
+                                  const si_debug_decode_opts_t *opts);
+
+/* One launch that reads `bytes` bytes (a multiple of 16) at the 16-byte-aligned device pointer `mem`
+ * once with plain 16-byte loads, all SMs busy, and stores a checksum of them in *checksum_dev (device
+ * uint32).  Timing it on the neuron store gives the read bandwidth a kernel with no other work reaches
+ * on this GPU, the practical ceiling quoted beside the decode kernel. */
+int si_debug_read_bandwidth(const void *mem, size_t bytes, unsigned int *checksum_dev, void *stream);
+
+/* The first stage of a multi-token si_ffn_forward call run on its own, with everything it leaves for
+ * the contractions copied out: the ascending union (union_out device int32 [n_loaded], *n_union_out
+ * device int32) and the tokens' slot bitmaps, which decide which union entries a token uses --
+ * masks_out device uint32 [T][mask_words], bit (s & 31) of word s >> 5 of row t set iff slot s is in
+ * list t; mask_words = ceil(n_loaded / 128) * 4.  Same kernels, same choice between them as in
+ * si_ffn_forward.  workspace as for si_ffn_forward with the same T and k_fixed. */
+int si_debug_union_masks(const si_store_t *store, int layer, int T, const int32_t *idx,
+                         const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
+                         uint32_t *masks_out, void *workspace, size_t ws_bytes, void *stream);
+
+/* si_ffn_forward for T > 1 (union path) with a limit on the probes of every device-side wait of the two
+ * contraction kernels (0 = the default) and, with withhold = 1, one operand tile of the first CTA of the
+ * gate/up kernel never loaded: its tensor-core warp waits for a stage that is never filled, the wait
+ * runs out, the kernel records SI_ERR_TIMEOUT in *status_dev, releases its tensor memory and returns. */
+int si_debug_ffn_forward_waits(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
+                               const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype, unsigned flags,
+                               void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream,
+                               long long spin_limit, int withhold);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SELECTINFER_DEBUG_H */

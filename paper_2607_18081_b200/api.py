@@ -1,7 +1,7 @@
 """Thin ctypes binding over libselectinfer.so: argument marshalling only.
 
 Every function here has the name and argument order of its C entry point
-(include/selectinfer.h) and takes torch CUDA tensors where the C side takes device
+(include/selectinfer.h; the si_debug_* diagnostics: include/selectinfer_debug.h) and takes torch CUDA tensors where the C side takes device
 pointers.  torch is used for device memory and the current stream, nothing else: no
 step of the path runs in Python or on the CPU.  If the CUDA library cannot be loaded
 the import of this module fails -- there is no fallback.
@@ -28,14 +28,16 @@ SI_FLAG_UNION_PATH = 32
 SI_FLAG_LIST_PER_LAYER = 64
 SI_FLAG_STEPS_ANY_ORDER = 128
 SI_FLAG_SIMPLE_KERNELS = 256
+SI_FLAG_PRENORM = 512
 SI_SELECT_TOPK, SI_SELECT_THRESHOLD = 0, 1
 
 EXPORTS = [
     "si_strerror", "si_last_cuda_error", "si_build_info", "si_store_bytes", "si_store_create", "si_store_free",
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
-    "si_layer_forward", "si_decode_stack_forward", "si_ffn_forward_noalloc", "si_union", "si_debug_decode_profile",
-    "si_debug_decode_stream_only", "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
+    "si_layer_forward", "si_decode_stack_forward", "si_decode_chain_forward", "si_ffn_forward_noalloc", "si_union",
+    "si_debug_decode_stack_forward", "si_debug_decode_chain_forward", "si_debug_union_masks", "si_debug_ffn_forward_waits",
+    "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
     "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce",
 ]
 
@@ -73,8 +75,11 @@ def _load_library() -> ctypes.CDLL:
     lib.si_decode_stack_forward.argtypes = [vp, ci, vp, vp, vp, vp, ci, vp, ci, cu, vp, sz, vp, vp]
     lib.si_union.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
     lib.si_ffn_forward_noalloc.argtypes = [vp, ci, vp, vp, ci, vp, ci, cu, vp, vp]
-    lib.si_debug_decode_profile.argtypes = [vp]
-    lib.si_debug_decode_stream_only.argtypes = [ci]
+    lib.si_decode_chain_forward.argtypes = [vp, ci, vp, ci, vp, vp, vp, ci, vp, vp, ctypes.c_float, cu, vp, sz, vp, vp]
+    lib.si_debug_decode_stack_forward.argtypes = lib.si_decode_stack_forward.argtypes + [vp]
+    lib.si_debug_decode_chain_forward.argtypes = lib.si_decode_chain_forward.argtypes + [vp]
+    lib.si_debug_union_masks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, sz, vp]
+    lib.si_debug_ffn_forward_waits.argtypes = lib.si_ffn_forward.argtypes + [ctypes.c_longlong, ci]
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
     lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
     lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
@@ -307,12 +312,61 @@ def si_debug_read_bandwidth(mem, nbytes: int, checksum, stream=None) -> None:
     _check(_lib.si_debug_read_bandwidth(_dp(mem), nbytes, _dp(checksum), _stream(stream)), "si_debug_read_bandwidth")
 
 
-def si_debug_decode_stream_only(on: bool) -> None:
-    _check(_lib.si_debug_decode_stream_only(1 if on else 0), "si_debug_decode_stream_only")
+class DecodeOpts(ctypes.Structure):
+    """si_debug_decode_opts_t: per-call diagnostics of a persistent decode launch (all zero = none)."""
+    _fields_ = [("skip_mask", ctypes.c_int), ("ring_stages", ctypes.c_int), ("step_groups", ctypes.c_int),
+                ("withhold", ctypes.c_int), ("wait_cycles", ctypes.c_longlong), ("profile", ctypes.c_void_p)]
 
 
-def si_debug_decode_profile(buf) -> None:
-    _check(_lib.si_debug_decode_profile(_dp(buf)), "si_debug_decode_profile")
+def _opts(skip_mask=0, ring_stages=0, step_groups=0, withhold=0, wait_cycles=0, profile=None) -> DecodeOpts:
+    return DecodeOpts(skip_mask, ring_stages, step_groups, withhold, wait_cycles,
+                      None if profile is None else profile.data_ptr())
+
+
+def si_debug_decode_stack_forward(handle, n_steps: int, layers, x, idx, idx_offsets, k_fixed: int, y, flags: int,
+                                  workspace, status=None, stream=None, **opts) -> None:
+    keep, p = _host_i32(layers)
+    o = _opts(**opts)
+    _check(_lib.si_debug_decode_stack_forward(handle, n_steps, p, _dp(x), _dp(idx), _dp(idx_offsets), k_fixed, _dp(y),
+                                              dtype_code(y.dtype), flags, _dp(workspace),
+                                              workspace.numel() * workspace.element_size(), _dp(status),
+                                              _stream(stream), ctypes.byref(o)), "si_debug_decode_stack_forward")
+
+
+def si_decode_chain_forward(handle, n_steps: int, layers, chain_len: int, x, idx, idx_offsets, k_fixed: int, y,
+                            xn_out, norm_eps: float, flags: int, workspace, status=None, stream=None) -> None:
+    keep, p = _host_i32(layers)
+    _check(_lib.si_decode_chain_forward(handle, n_steps, p, chain_len, _dp(x), _dp(idx), _dp(idx_offsets), k_fixed,
+                                        _dp(y), _dp(xn_out), norm_eps, flags, _dp(workspace),
+                                        workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)),
+           "si_decode_chain_forward")
+
+
+def si_debug_decode_chain_forward(handle, n_steps: int, layers, chain_len: int, x, idx, idx_offsets, k_fixed: int, y,
+                                  xn_out, norm_eps: float, flags: int, workspace, status=None, stream=None,
+                                  **opts) -> None:
+    keep, p = _host_i32(layers)
+    o = _opts(**opts)
+    _check(_lib.si_debug_decode_chain_forward(handle, n_steps, p, chain_len, _dp(x), _dp(idx), _dp(idx_offsets),
+                                              k_fixed, _dp(y), _dp(xn_out), norm_eps, flags, _dp(workspace),
+                                              workspace.numel() * workspace.element_size(), _dp(status),
+                                              _stream(stream), ctypes.byref(o)), "si_debug_decode_chain_forward")
+
+
+def si_debug_union_masks(handle, layer: int, T: int, idx, idx_offsets, k_fixed: int, union_out, n_union_out,
+                         masks_out, workspace, stream=None) -> None:
+    _check(_lib.si_debug_union_masks(handle, layer, T, _dp(idx), _dp(idx_offsets), k_fixed, _dp(union_out),
+                                     _dp(n_union_out), _dp(masks_out), _dp(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "si_debug_union_masks")
+
+
+def si_debug_ffn_forward_waits(handle, layer: int, x, T: int, idx, idx_offsets, k_fixed: int, y, flags: int,
+                               workspace, status, spin_limit: int, withhold: int, stream=None) -> None:
+    _check(_lib.si_debug_ffn_forward_waits(handle, layer, _dp(x), T, _dp(idx), _dp(idx_offsets), k_fixed, _dp(y),
+                                           dtype_code(y.dtype), flags, _dp(workspace),
+                                           workspace.numel() * workspace.element_size(), _dp(status),
+                                           _stream(stream), spin_limit, withhold), "si_debug_ffn_forward_waits")
 
 
 # ------------------------------------------------------------------------- owner object

@@ -2,6 +2,7 @@
 // si_layer_forward (selection + FFN), si_decode_stack_forward, si_union.
 #include "si_common.cuh"
 #include "si_decode_persistent.cuh"
+#include "selectinfer_debug.h"
 
 si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps) {
     si_ws_layout w;
@@ -42,7 +43,7 @@ static int check_common(const si_store *s, const void *x, const void *y, int y_d
     if (y_dtype != SI_F32 && y_dtype != s->dtype) return SI_ERR_INVALID_ARG;
     if (!si_aligned16(x) || !si_aligned16(y) || (((uintptr_t)workspace) & 255u)) return SI_ERR_ALIGNMENT;
     if (status_dev && (((uintptr_t)status_dev) & 3u)) return SI_ERR_ALIGNMENT;
-    return SI_OK;
+    return si_check_device(s);
 }
 
 extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
@@ -62,7 +63,7 @@ extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x,
                                         k_fixed, status_dev, stream);
         if (rc) return rc;
     }
-    if (T == 1) {
+    if (T == 1 && !(flags & SI_FLAG_UNION_PATH)) {
         int32_t l = layer;
         return si_decode_launch(store, 1, &l, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
                                 ws_bytes, status_dev, stream);
@@ -99,6 +100,7 @@ extern "C" int si_layer_forward(const si_store_t *store, int layer, const void *
     int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
     if (rc) return rc;
     if (layer < 0 || layer >= store->n_layers || T <= 0 || k < 0) return SI_ERR_INVALID_ARG;
+    if (!store->loaded[layer]) return SI_ERR_INVALID_ARG;      // before the selector is enqueued
     const int n = store->n_loaded[layer];
     if (k > n) return SI_ERR_OUT_OF_RANGE;
     if (!si_aligned16(scores)) return SI_ERR_ALIGNMENT;
@@ -115,10 +117,11 @@ extern "C" int si_layer_forward(const si_store_t *store, int layer, const void *
                           ws_bytes, status_dev, stream_);
 }
 
-extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
-                                       const void *x, const int32_t *idx, const int32_t *idx_offsets,
-                                       int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
-                                       size_t ws_bytes, int32_t *status_dev, void *stream_) {
+// si_decode_stack_forward and si_decode_chain_forward (ex->chain_len > 0) share their checks.
+static int decode_stack_impl(const si_store_t *store, int n_steps, const int32_t *layers, const void *x,
+                             const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype,
+                             unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream_,
+                             const si_decode_extra *ex) {
     int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
     if (rc) return rc;
     if (n_steps <= 0 || k_fixed < 0) return SI_ERR_INVALID_ARG;
@@ -128,10 +131,17 @@ extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, con
     for (int st = 0; st < n_steps; ++st) {
         int l = layers ? layers[st] : st % store->n_layers;
         if (l < 0 || l >= store->n_layers) return SI_ERR_INVALID_ARG;
+        if (!store->loaded[l]) return SI_ERR_INVALID_ARG;          // before anything is enqueued
         min_loaded = min_loaded < store->n_loaded[l] ? min_loaded : store->n_loaded[l];
     }
     if (!idx_offsets && k_fixed > min_loaded) return SI_ERR_OUT_OF_RANGE;
     if ((flags & SI_FLAG_LIST_PER_LAYER) && idx_offsets) return SI_ERR_INVALID_ARG;   // per-layer lists have one fixed length
+    if (ex && ex->chain_len > 0) {
+        if (y_dtype != store->dtype) return SI_ERR_INVALID_ARG;    // a step's output is the next step's input
+        if (!si_persistent_supported(store)) return SI_ERR_UNSUPPORTED;
+        if (ex->xn_out && !si_aligned16(ex->xn_out)) return SI_ERR_ALIGNMENT;
+        if (ex->prenorm && !(ex->norm_eps >= 0.f)) return SI_ERR_INVALID_ARG;
+    }
     cudaStream_t stream = (cudaStream_t)stream_;
     si_ws_layout ws = si_ws_carve(store, 1, k_fixed, n_steps);
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
@@ -153,7 +163,97 @@ extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, con
         }
     }
     return si_decode_launch(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
-                            ws_bytes, status_dev, stream);
+                            ws_bytes, status_dev, stream, ex);
+}
+
+static si_decode_extra extra_of(const si_debug_decode_opts_t *o) {
+    si_decode_extra ex;
+    if (o) {
+        ex.skip_mask = o->skip_mask; ex.ring_stages = o->ring_stages; ex.step_groups = o->step_groups;
+        ex.withhold = o->withhold; ex.wait_cycles = o->wait_cycles; ex.profile = (long long *)o->profile;
+    }
+    return ex;
+}
+
+extern "C" int si_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
+                                       const void *x, const int32_t *idx, const int32_t *idx_offsets,
+                                       int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
+                                       size_t ws_bytes, int32_t *status_dev, void *stream) {
+    return decode_stack_impl(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace, ws_bytes,
+                             status_dev, stream, nullptr);
+}
+
+extern "C" int si_debug_decode_stack_forward(const si_store_t *store, int n_steps, const int32_t *layers,
+                                             const void *x, const int32_t *idx, const int32_t *idx_offsets,
+                                             int k_fixed, void *y, int y_dtype, unsigned flags, void *workspace,
+                                             size_t ws_bytes, int32_t *status_dev, void *stream,
+                                             const si_debug_decode_opts_t *opts) {
+    if (opts && (opts->ring_stages < 0 || opts->step_groups < 0 || opts->wait_cycles < 0)) return SI_ERR_INVALID_ARG;
+    const si_decode_extra ex = extra_of(opts);
+    return decode_stack_impl(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace, ws_bytes,
+                             status_dev, stream, &ex);
+}
+
+static int chain_impl(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len, const void *x,
+                      const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y, void *xn_out,
+                      float norm_eps, unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
+                      void *stream, const si_debug_decode_opts_t *opts) {
+    if (chain_len < 1 || !si_store_ok(store)) return SI_ERR_INVALID_ARG;
+    if (flags & (SI_FLAG_STEPS_ANY_ORDER | SI_FLAG_SIMPLE_KERNELS)) return SI_ERR_INVALID_ARG;   // neither applies to a chain
+    if (opts && (opts->ring_stages < 0 || opts->wait_cycles < 0)) return SI_ERR_INVALID_ARG;
+    si_decode_extra ex = extra_of(opts);
+    ex.step_groups = 0;
+    ex.chain_len = chain_len;
+    ex.prenorm = (flags & SI_FLAG_PRENORM) != 0;
+    ex.norm_eps = norm_eps;
+    ex.xn_out = ex.prenorm ? xn_out : nullptr;
+    return decode_stack_impl(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, store->dtype, flags, workspace,
+                             ws_bytes, status_dev, stream, &ex);
+}
+
+extern "C" int si_decode_chain_forward(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len,
+                                       const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                                       void *y, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                                       size_t ws_bytes, int32_t *status_dev, void *stream) {
+    return chain_impl(store, n_steps, layers, chain_len, x, idx, idx_offsets, k_fixed, y, xn_out, norm_eps, flags, workspace,
+                      ws_bytes, status_dev, stream, nullptr);
+}
+
+extern "C" int si_debug_decode_chain_forward(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len,
+                                             const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                                             void *y, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                                             size_t ws_bytes, int32_t *status_dev, void *stream,
+                                             const si_debug_decode_opts_t *opts) {
+    return chain_impl(store, n_steps, layers, chain_len, x, idx, idx_offsets, k_fixed, y, xn_out, norm_eps, flags, workspace,
+                      ws_bytes, status_dev, stream, opts);
+}
+
+extern "C" int si_debug_ffn_forward_waits(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,
+                                          const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype, unsigned flags,
+                                          void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream,
+                                          long long spin_limit, int withhold) {
+    int rc = check_common(store, x, y, y_dtype, workspace, status_dev);
+    if (rc) return rc;
+    if (layer < 0 || layer >= store->n_layers || T <= 1 || k_fixed <= 0 || spin_limit < 0) return SI_ERR_INVALID_ARG;
+    if (!store->loaded[layer] || !idx) return SI_ERR_INVALID_ARG;
+    if (k_fixed > store->n_loaded[layer]) return SI_ERR_OUT_OF_RANGE;
+    if (!si_aligned16(idx)) return SI_ERR_ALIGNMENT;
+    if (ws_bytes < si_ws_carve(store, T, k_fixed, 1).total) return SI_ERR_NOMEM;
+    return si_multi_token_launch(store, layer, x, T, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace, ws_bytes,
+                                 status_dev, (cudaStream_t)stream, spin_limit, withhold);
+}
+
+extern "C" int si_debug_union_masks(const si_store_t *store, int layer, int T, const int32_t *idx,
+                                    const int32_t *idx_offsets, int k_fixed, int32_t *union_out, int32_t *n_union_out,
+                                    uint32_t *masks_out, void *workspace, size_t ws_bytes, void *stream) {
+    if (!si_store_ok(store) || layer < 0 || layer >= store->n_layers || T <= 0 || k_fixed < 0 || !union_out ||
+        !n_union_out || !masks_out || !workspace)
+        return SI_ERR_INVALID_ARG;
+    if (k_fixed > 0 && !idx) return SI_ERR_INVALID_ARG;
+    int rc = si_check_device(store);
+    if (rc) return rc;
+    return si_union_masks_launch(store, layer, T, idx, idx_offsets, k_fixed, union_out, n_union_out, masks_out, workspace,
+                                 ws_bytes, (cudaStream_t)stream);
 }
 
 extern "C" int si_union(const si_store_t *store, int layer, int T, const int32_t *idx,
@@ -163,6 +263,7 @@ extern "C" int si_union(const si_store_t *store, int layer, int T, const int32_t
         !n_union_out || !workspace)
         return SI_ERR_INVALID_ARG;
     if (k_fixed > 0 && !idx) return SI_ERR_INVALID_ARG;
+    if (int rc = si_check_device(store)) return rc;
     return si_union_launch(store, layer, T, idx, idx_offsets, k_fixed, union_out, n_union_out, workspace,
                            ws_bytes, (cudaStream_t)stream);
 }

@@ -1,4 +1,5 @@
-// Device-side validation of active lists (SI_FLAG_CHECK): every entry in [0, n_loaded) and
+// Device-side validation of active lists (SI_FLAG_CHECK): list offsets that start at or above 0,
+// never decrease and describe lists of at most k_fixed entries; every entry in [0, n_loaded) and
 // no entry twice.  One CTA per list marks a shared-memory bitmap; a bit seen twice is a
 // duplicate.  Only an error code is written; nothing else is touched.
 #include "si_common.cuh"
@@ -26,6 +27,10 @@ si_check_lists_kernel(const __grid_constant__ CheckParams P, const int32_t *__re
     __syncthreads();
     int base = offsets ? offsets[list] : list * k_fixed;
     int k = offsets ? offsets[list + 1] - base : k_fixed;
+    if (offsets && (base < 0 || k < 0 || k > k_fixed)) {     // a malformed offsets array: report, read no entry
+        if (threadIdx.x == 0) atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE);
+        return;
+    }
     for (int p = threadIdx.x; p < k; p += blockDim.x) {
         int s = idx[base + p];
         if (s < 0 || s >= n_loaded) { atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }

@@ -32,6 +32,13 @@ struct si_store {
 static inline size_t si_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline bool si_aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
 static inline bool si_store_ok(const si_store *s) { return s && s->magic == SI_MAGIC; }
+// A store's kernels, grid sizes and pointers belong to the device it was created on: that device has
+// to be current in every call that launches work on it.
+static inline int si_check_device(const si_store *s) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return SI_ERR_CUDA; }
+    return dev == s->device ? SI_OK : SI_ERR_INVALID_ARG;
+}
 
 // last CUDA runtime error seen by this library on the calling thread (si_last_cuda_error)
 int &si_last_cuda_error_code();
@@ -63,17 +70,32 @@ struct si_ws_layout {
 };
 si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps);
 
+// What a decode launch may carry beyond the arguments of si_decode_stack_forward: the chained mode of
+// si_decode_chain_forward and the per-call diagnostics of si_debug_decode_stack_forward.
+struct si_decode_extra {
+    int chain_len = 0;             // > 0: chained steps (persistent kernel only)
+    int prenorm = 0;
+    float norm_eps = 0.f;
+    void *xn_out = nullptr;
+    int skip_mask = 0, ring_stages = 0, step_groups = 0, withhold = 0;
+    long long wait_cycles = 0;     // 0: the default limit
+    long long *profile = nullptr;
+};
+
 // implemented in si_decode.cu
 int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host, const void *x,
                      const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y,
                      int y_dtype, unsigned flags, void *workspace, size_t ws_bytes,
-                     int32_t *status_dev, cudaStream_t stream);
+                     int32_t *status_dev, cudaStream_t stream, const si_decode_extra *ex = nullptr);
 
 // implemented in si_gemm.cu
 int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, const int32_t *idx,
                           const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype,
                           unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
-                          cudaStream_t stream);
+                          cudaStream_t stream, long long spin_limit = 0, int withhold = 0);
+int si_union_masks_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
+                          int k_fixed, int32_t *union_out, int32_t *n_union_out, uint32_t *masks_out,
+                          void *workspace, size_t ws_bytes, cudaStream_t stream);
 
 // implemented in si_select.cu
 size_t si_select_ws_bytes_impl(int n);

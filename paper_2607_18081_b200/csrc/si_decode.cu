@@ -8,28 +8,10 @@
 //   * "persistent" (si_decode_persistent.cuh): one launch for any number of steps, records
 //     streamed through a shared-memory ring by bulk async copies.
 // Both accumulate in a fixed order, so results are run-to-run bit-identical.
+#include <atomic>
+
 #include "si_common.cuh"
 #include "si_decode_persistent.cuh"
-
-long long *&si_decode_profile_buffer() {
-    static long long *buf = nullptr;
-    return buf;
-}
-
-int &si_decode_stream_only() {
-    static int v = 0;
-    return v;
-}
-
-extern "C" int si_debug_decode_stream_only(int on) {
-    si_decode_stream_only() = on;
-    return SI_OK;
-}
-
-extern "C" int si_debug_decode_profile(void *dev_buf) {
-    si_decode_profile_buffer() = (long long *)dev_buf;
-    return SI_OK;
-}
 
 namespace {
 
@@ -371,7 +353,7 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host, const void *x,
                      const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y,
                      int y_dtype, unsigned flags, void *workspace, size_t ws_bytes,
-                     int32_t *status_dev, cudaStream_t stream) {
+                     int32_t *status_dev, cudaStream_t stream, const si_decode_extra *ex) {
     si_ws_layout ws = si_ws_carve(s, 1, k_fixed, n_steps);
     if (ws_bytes < ws.total) return SI_ERR_NOMEM;
     if (n_steps <= 0) return SI_ERR_INVALID_ARG;
@@ -385,10 +367,12 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
     // kernel: a launch of it costs about 33 us beyond its steps, a plain step 12 us against 5.4 us
     // (replayed from a CUDA graph; launched one by one from the host three steps already favour the
     // persistent kernel, whose single launch costs the host less than six)
-    const bool use_simple = (flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps <= 2;
+    const bool chained = ex && ex->chain_len > 0;
+    if (chained && !si_persistent_supported(s)) return SI_ERR_UNSUPPORTED;    // chains live in the persistent kernel
+    const bool use_simple = !chained && ((flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps <= 2);
     if (!use_simple)
         return si_decode_persistent_launch(s, n_steps, layers_host, x, idx, idx_offsets, k_fixed, y, y_dtype, flags,
-                                           wsb, ws, status_dev, stream);
+                                           wsb, ws, status_dev, stream, ex);
     // simple path: one partial + one reduce launch per step.  With CSR lists the true length
     // is read on the device; k_fixed (an upper bound) only sizes the grid.
     const size_t esz = 2, ysz = (y_dtype == SI_F32) ? 4 : 2;
@@ -425,27 +409,25 @@ static __device__ __align__(256) float si_noalloc_scratch[(size_t)kNoAllocMaxCta
 // In host code the array's name above is only a handle; the device address has to be asked for,
 // once per device, with that device current.
 struct NoAllocDevices {
-    void *ptr[64];
-    bool ready[64];
+    std::atomic<void *> ptr[64];      // null until the device's address has been looked up
 };
 NoAllocDevices &noalloc_devices() {
-    static NoAllocDevices d = {};
+    static NoAllocDevices d;           // zero-initialised; constructed once (thread-safe in C++11)
     return d;
 }
 
-int noalloc_scratch_for_current_device(float **out) {
-    int dev = -1;
-    SI_CUDA_TRY(cudaGetDevice(&dev));
+// `dev` must be the current device.  Two host threads that make the first call on a device at the
+// same time both look the address up and both store the same value.
+int noalloc_scratch_for_device(int dev, float **out) {
     if (dev < 0 || dev >= 64) return SI_ERR_UNSUPPORTED;
     NoAllocDevices &d = noalloc_devices();
-    if (!d.ready[dev]) {
-        void *p = nullptr;
+    void *p = d.ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         SI_CUDA_TRY(cudaGetSymbolAddress(&p, si_noalloc_scratch));
         if (!p) return SI_ERR_CUDA;
-        d.ptr[dev] = p;
-        d.ready[dev] = true;
+        d.ptr[dev].store(p, std::memory_order_release);
     }
-    *out = (float *)d.ptr[dev];
+    *out = (float *)p;
     return SI_OK;
 }
 
@@ -463,8 +445,12 @@ extern "C" int si_ffn_forward_noalloc(const si_store_t *store, int layer, const 
     if (status_dev && (((uintptr_t)status_dev) & 3u)) return SI_ERR_ALIGNMENT;
     // the fixed scratch holds one fp32 row of d_model values per CTA of the partial kernel
     if (store->d_model > kNoAllocMaxDModel || 2 * store->num_sms > kNoAllocMaxCtas) return SI_ERR_TOO_LARGE;
+    // the scratch address and the grid size belong to one device: the store's, which must be current
+    int dev = -1;
+    SI_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != store->device) return SI_ERR_INVALID_ARG;
     float *scratch = nullptr;
-    int rc = noalloc_scratch_for_current_device(&scratch);
+    int rc = noalloc_scratch_for_device(dev, &scratch);
     if (rc != SI_OK) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     // every CTA of the partial kernel writes its whole row before the reduce kernel reads it, so

@@ -23,6 +23,15 @@
 //     fixed order (lane rows ascending, warp butterfly: deterministic split-K) and write y
 //     once.  The reduction trails the record stream and never stalls it.
 //
+// Chained mode (Params::chain_len > 0): step s takes the output row of step s - 1 as its input unless
+// s is the first step of a chain (s mod chain_len == 0), the way the FFN of layer l + 1 sees what layer
+// l produced.  Nothing of a step's arithmetic can then start before the step before it is complete: the
+// step's cross-SM sum runs at once (no lag), every CTA publishes "my columns of y are written", and the
+// producer issues the bulk copy of the next step's input only when every CTA has said so.  The record
+// rings are not held back: the lists are known up front (the set is fixed per prompt), so the first
+// records of the next step are in shared memory before its input is.  With Params::prenorm the input
+// row is normalised to unit root mean square (and rounded to the store type) before the dot products.
+//
 // Every wait is bounded: on expiry the kernel records SI_ERR_TIMEOUT, raises a grid-wide
 // abort flag, lets its outstanding copies land and returns.
 #pragma once
@@ -48,7 +57,8 @@ constexpr int kPartialDepth = 10;                 // D: partial-y buffers in fli
 constexpr int kFewSteps = 16;                     // launches this short carry their layer ids as kernel arguments
 constexpr int kProfSlots = 16;                    // int64 cycle counters per SM in the optional phase profile
 constexpr int kLag = 4;                           // a step's cross-SM reduction starts this many steps later
-constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
+constexpr long long kWaitCycles = 4000000000ll;   // default limit of every wait: ~2 s at 1.9 GHz
+constexpr long long kDrainCycles = 40000000ll;    // least time a leaving producer gives its copies in flight to land
 
 struct Params {
     const char *store_base;
@@ -73,7 +83,16 @@ struct Params {
                                   // reading the step's partials
     int32_t *status;
     long long *prof;              // optional phase profile: int64 [G][kProfSlots] cycle counters, or nullptr
-    int stream_only;              // diagnostics bit mask (see si_debug_decode_stream_only)
+    int stream_only;              // diagnostics bit mask (si_debug_decode_opts_t::skip_mask)
+    long long wait_cycles;        // limit of every wait, in clock cycles
+    int withhold;                 // diagnostics: the producer of CTA 0 never issues the second item of its first set
+    // chained mode
+    int chain_len;                // 0: every step's x is an input of the call; > 0: x holds one row per chain
+                                  // ([ceil(n_steps / chain_len)][d_model]) and step s with s mod chain_len != 0
+                                  // reads row s - 1 of y (store dtype) as its input
+    int prenorm;                  // the input row is scaled to unit root mean square before the FFN
+    float norm_eps;
+    uint16_t *xn_out;             // optional [n_steps][d_model]: the normalised, rounded input every step used
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -110,14 +129,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait; also gives up when the CTA-local abort flag is raised.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, volatile int *cta_abort) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, volatile int *cta_abort, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*cta_abort) return false;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 // Strong (gpu-scope) vector store and vector add-reduction at L2; one thread issues both to the same
@@ -142,16 +161,16 @@ __device__ __forceinline__ unsigned ld_relaxed_gpu(const unsigned *p) {
 }
 // Bounded wait until *ctr >= target; gives up on the grid-wide or CTA-local abort flag.
 __device__ __forceinline__ bool counter_wait_bounded(const unsigned *ctr, unsigned target, const unsigned *grid_abort,
-                                                     volatile int *cta_abort) {
+                                                     volatile int *cta_abort, long long limit, unsigned sleep_ns = 64) {
     if (ld_acquire_gpu(ctr) >= target) return true;
     long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 16; ++i) {
             if (ld_acquire_gpu(ctr) >= target) return true;
-            __nanosleep(64);
+            if (sleep_ns) __nanosleep(sleep_ns);
         }
         if (*cta_abort || ld_relaxed_gpu(grid_abort)) return false;
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
@@ -257,6 +276,7 @@ struct Smem {
     int meta[kMaxStages];
     uint4 desc[kSets][kDescRing];      // {src lo, src hi, bytes (0: nothing to copy), meta}
     float2 setpart[kSets][2][2 * kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products (16 warps in the one wide set)
+    float normpart[kSets][2][2 * kSetWarps];   // [set][step parity][warp] = sum of squares of the warp's share of the input row (prenorm)
     volatile int cta_abort;
 };
 
@@ -296,6 +316,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     const int nv = P.n_steps > grp ? (P.n_steps - grp + NG - 1) / NG : 0;   // steps of this group
     const int Gv = G * kSets;                  // consumer sets act as virtual CTAs 2b, 2b+1 of 2G
     const int d = P.d_model, chunks = P.chunks;
+    const long long wait_limit = P.wait_cycles;
+    const bool chained = P.chain_len > 0;      // (one step group then: the launch code sees to it)
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
@@ -349,8 +371,13 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     const int rs = step * NG + grp;               // step of the launch
                     const int layer = P.step_layers ? __ldg(P.step_layers + rs) : (P.n_few ? (int)P.few_layers[rs] : rs % P.n_layers);
                     if (t == 0) {
-                        pf_src = (unsigned long long)(P.x + (size_t)rs * d);
-                        pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
+                        // chained: the first step of a chain reads the caller's row, every other step the
+                        // output row of the step before it, which the issue lane may only fetch once every
+                        // CTA has written its columns of it (bit 31 of the byte count marks such an item)
+                        const bool from_y = chained && rs % P.chain_len != 0;
+                        pf_src = from_y ? (unsigned long long)(reinterpret_cast<const uint16_t *>(P.y) + (size_t)(rs - 1) * d)
+                                        : (unsigned long long)(P.x + (size_t)(chained ? rs / P.chain_len : rs) * d);
+                        pf_bytes = (uint32_t)d * 2 | (from_y ? 0x80000000u : 0u); pf_meta = g.cnt;
                     } else {
                         const int lbase = P.per_layer_lists ? layer * P.k_fixed : g.base;
                         const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - 1) * Gv);
@@ -403,10 +430,22 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             commit_window(do_commit);
             prefetch_window(do_commit && desc_ready < total);
             bool progressed = false;
-            if (have && n < i_ready) {
+            if (have && n < i_ready && !(P.withhold && blockIdx.x == 0 && iq == 0 && n == 1)) {
                 const int st = iq * S + is;
-                if (mbar_test_wait(&empty[st], iph ^ 1)) {
-                    const uint4 dsc = sm->desc[iq][n % kDescRing];
+                bool go = mbar_test_wait(&empty[st], iph ^ 1);
+                uint4 dsc = make_uint4(0, 0, 0, 0);
+                if (go) {
+                    dsc = sm->desc[iq][n % kDescRing];
+                    if (dsc.z & 0x80000000u) {
+                        // input row = output row of the step before: has every CTA written its columns?
+                        const unsigned long long src = ((unsigned long long)dsc.y << 32) | dsc.x;
+                        const int prev = (int)((src - (unsigned long long)P.y) / ((unsigned long long)d * 2));
+                        go = ld_acquire_gpu(P.counters + (size_t)prev * kCounterStride + 32) >= (unsigned)gridDim.x;
+                        if (go) asm volatile("fence.proxy.async;" ::: "memory");   // the bulk copy reads what generic stores wrote
+                        dsc.z &= 0x7FFFFFFFu;
+                    }
+                }
+                if (go) {
                     meta[st] = (int)dsc.w;
                     if (dsc.z != 0) {
                         mbar_arrive_expect_tx(&full[st], dsc.z);
@@ -424,8 +463,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             if (__any_sync(FULL, progressed)) {
                 t_last = clock64();
             } else {
-                if (*cta_abort || clock64() - t_last > kWaitCycles) { ok = false; break; }
-                __nanosleep(100);       // nothing to issue: do not burn issue slots and power
+                if (*cta_abort || clock64() - t_last > wait_limit) { ok = false; break; }
+                if (!chained) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -434,7 +473,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             const uint32_t last = n - S;           // set-ring index of this lane's last issued item
             const uint32_t ph = (last / S) & 1;
             long long t0 = clock64();
-            while (!mbar_try_wait(&full[iq * S + is], ph) && clock64() - t0 < kWaitCycles) {}
+            const long long drain = wait_limit > kDrainCycles ? wait_limit : kDrainCycles;
+            while (!mbar_try_wait(&full[iq * S + is], ph) && clock64() - t0 < drain) {}
         }
         return;
     }
@@ -475,7 +515,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             {
                 int cnt;
                 {   // x item
-                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
+                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
                     cnt = fail ? 0 : smeta[st];
                     const uint4 *xs = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
 #pragma unroll
@@ -487,12 +527,50 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     if (lane == 0) mbar_arrive(&sempty[st]);
                     if (++st == S) { st = 0; ph ^= 1; }
                 }
+                if (P.prenorm) {
+                    // sum of squares of the row: thread slice, warp butterfly, then (after the barrier
+                    // below) the set's warps in warp order -- the same order in every set of every CTA
+                    float ss = 0.f;
+#pragma unroll
+                    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float lo, hi;
+                            unpack2(xr[i][e], lo, hi);
+                            ss = fmaf(lo, lo, ss); ss = fmaf(hi, hi, ss);
+                        }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+                    if (lane == 0) sm->normpart[q][step & 1][sw] = ss;
+                }
                 // the record count steers the set's barriers: agree on it (and on failure) first
                 fail = set_barrier_or<kSetThreads>(q, fail);
                 if (fail) break;
+                if (P.prenorm) {
+                    float ss = 0.f;
+#pragma unroll
+                    for (int w = 0; w < kSetWarps; ++w) ss += sm->normpart[q][step & 1][w];
+                    const float scale = rsqrtf(ss / (float)d + P.norm_eps);
+                    const int rs = step * NG + grp;
+                    const bool emit = P.xn_out != nullptr && b == 0 && q == 0;
+#pragma unroll
+                    for (int i = 0; i < NCH; ++i) {
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float lo, hi;
+                            unpack2(xr[i][e], lo, hi);
+                            w4[e] = (uint32_t)si_cvt<DT>::from_float(lo * scale) | ((uint32_t)si_cvt<DT>::from_float(hi * scale) << 16);
+                            xr[i][e] = pair_of<DT>(w4[e]);        // the dot products see the rounded values
+                        }
+                        const int c = t + kSetThreads * i;
+                        if (emit && (kFull || c < chunks))
+                            reinterpret_cast<uint4 *>(P.xn_out + (size_t)rs * d)[c] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    }
+                }
                 SI_PROF(0);                               // wait for x
                 for (int i = 0; i < cnt; ++i) {
-                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort);
+                    fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
                     const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0 and no accumulate
                     // ---- copy this thread's chunks of the record into registers, free the stage
                     const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
@@ -570,7 +648,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             {
                 if (step > 0) {      // the buffer was last handed over at step - 1
                     const int ps = step - 1;
-                    fail |= !mbar_wait_bounded(&sm->accempty[q][ps % kReducerWarps], (uint32_t)((ps / kReducerWarps) & 1), cta_abort);
+                    fail |= !mbar_wait_bounded(&sm->accempty[q][ps % kReducerWarps], (uint32_t)((ps / kReducerWarps) & 1), cta_abort, wait_limit);
                 }
                 if (fail) break;
                 SI_PROF(4);                               // wait for the hand-over buffer
@@ -625,7 +703,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         float *const gpartial = P.partial + (size_t)grp * kPartialDepth * G * d;   // this group's ring of partial rows
         auto ctr_of = [&](int v) { return P.counters + ((size_t)v * NG + grp) * kCounterStride; };   // counters of the group's step v
         constexpr int kRowBatch = 13;                          // partial rows in flight per lane
-        for (int step = r; step < nv + kLag; step += kReducerWarps) {
+        const int lag = chained ? 0 : kLag;                    // chained: a step's sum is needed at once
+        for (int step = r; step < nv + lag; step += kReducerWarps) {
             int ok = 1;
             if (step < nv) {
                 // ---- phase A: take each set's accumulators as soon as that set hands them over.  The
@@ -649,14 +728,14 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                             if (!(taken & 1) && mbar_test_wait(&sm->accfull[0][r], par)) q = 0;
                             else if (kSets > 1 && !(taken & 2) && mbar_test_wait(&sm->accfull[kSets - 1][r], par)) q = 1;
                             else {
-                                if (*cta_abort || clock64() - t0 > kWaitCycles) break;
-                                __nanosleep(200);
+                                if (*cta_abort || clock64() - t0 > wait_limit) break;
+                                if (!chained) __nanosleep(200);
                             }
                         }
                         ok = q >= 0;
                         SI_RPROF(0);                      // idle: waiting for a set's hand-over
                         if (ok && sub == 0 && freed < (unsigned)G)
-                            ok = counter_wait_bounded(ctr_of(step - kPartialDepth) + 32, (unsigned)G, P.ctrl + 1, cta_abort);
+                            ok = counter_wait_bounded(ctr_of(step - kPartialDepth) + 32, (unsigned)G, P.ctrl + 1, cta_abort, wait_limit);
                     }
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     q = __shfl_sync(0xFFFFFFFFu, q, 0);
@@ -685,13 +764,18 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     SI_RPROF(2);                          // copy the accumulators out
                 }
             }
-            const int sr = step - kLag;
+            const int sr = step - lag;
+            if (chained && ok && !nosync) {
+                // the step's own sum follows at once: publish this CTA's partial row first
+                __syncwarp();
+                if (lane == 0) { __threadfence(); atomicAdd(ctr_of(step), 1u); }
+            }
             if (ok && sr >= 0 && !nosync) {
                 // ---- phase B: lane (group bg, row class brc) sums rows brc, brc + 4, ... of its column
                 // group in ascending order, kRowBatch loads in flight; two butterfly steps combine the
                 // four row classes (fixed order: deterministic split-K)
                 if (lane == 0)
-                    ok = counter_wait_bounded(ctr_of(sr), (unsigned)G, P.ctrl + 1, cta_abort);
+                    ok = counter_wait_bounded(ctr_of(sr), (unsigned)G, P.ctrl + 1, cta_abort, wait_limit, chained ? 0u : 64u);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 SI_RPROF(4);                              // every SM has published the step
                 if (ok) {
@@ -717,9 +801,17 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, o); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, o);
                     }
                     if (brc == 0 && bg < g_valid) {
-                        const size_t col = ((size_t)sr * NG + grp) * d + (size_t)(b * gpc + bg) * 4;
+                        const int rs = sr * NG + grp;                      // step of the launch
+                        const size_t cin = (size_t)(b * gpc + bg) * 4;     // first of the lane's four columns
+                        const size_t col = (size_t)rs * d + cin;
                         if (P.residual) {
-                            uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
+                            // the step's input row: the caller's, or in a chain the output row of the step before
+                            // (complete and visible: this step's records were only multiplied with it once every
+                            // CTA had published its columns; read at L2, where those stores went)
+                            const uint16_t *xin = !chained ? P.x + col
+                                                  : (rs % P.chain_len != 0 ? reinterpret_cast<const uint16_t *>(P.y) + (col - d)
+                                                                           : P.x + (size_t)(rs / P.chain_len) * d + cin);
+                            uint2 xw = chained ? __ldcg(reinterpret_cast<const uint2 *>(xin)) : __ldg(reinterpret_cast<const uint2 *>(xin));
                             v.x += si_cvt<DT>::lo(xw.x); v.y += si_cvt<DT>::hi(xw.x);
                             v.z += si_cvt<DT>::lo(xw.y); v.w += si_cvt<DT>::hi(xw.y);
                         }
@@ -744,8 +836,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             __syncwarp();
             if (lane == 0 && !nosync) {
                 __threadfence();
-                if (step < nv) atomicAdd(ctr_of(step), 1u);
-                if (sr >= 0 && sr + kPartialDepth < nv) atomicAdd(ctr_of(sr) + 32, 1u);
+                if (step < nv && !chained) atomicAdd(ctr_of(step), 1u);
+                // chained: the producers of every CTA wait for this count before they fetch the next step's input
+                if (sr >= 0 && (chained || sr + kPartialDepth < nv)) atomicAdd(ctr_of(sr) + 32, 1u);
             }
             SI_RPROF(3);                                  // publish (fence + atomics)
         }
@@ -779,13 +872,6 @@ inline bool wide_rows(int d_model) {
 
 }  // namespace si_persist
 
-// Diagnostics: when set, every persistent launch writes per-CTA cycle counts of the consumer
-// phases of set 0 (wait x, wait + copy records, arithmetic, reduction sums, partial store,
-// reduction issue, set merge).
-long long *&si_decode_profile_buffer();
-// Diagnostics bit mask: 1 = no arithmetic, 2 = no reduction loads, 4 = no cross-CTA exchange.
-int &si_decode_stream_only();
-
 inline bool si_persistent_supported(const si_store *s) {
     // thread t of a 256-thread set owns chunks t, t + 256 (, t + 512) of a row (d_model <= 6144); the
     // rings need at least two stages per consumer set beside the two hand-over buffers; a reducer warp's
@@ -807,13 +893,9 @@ template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8>
 inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
     auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP, SETW>;
     size_t smem = si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW);
-    static size_t smem_set[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // per device: the limit already raised for this instance
-    int dev = 0;
-    SI_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 8 || smem_set[dev] < smem) {
-        SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        if (dev >= 0 && dev < 8) smem_set[dev] = smem;
-    }
+    // the limit is raised to the most any instance needs (setting it is cheap, a host-side call, and
+    // keeps no state here that threads or devices could disagree about)
+    SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&P};
     SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G), dim3(si_persist::kThreads), args, smem, stream));
     return SI_OK;
@@ -822,7 +904,10 @@ inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cud
 inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int32_t *layers_host,
                                        const void *x, const int32_t *idx, const int32_t *idx_offsets,
                                        int k_fixed, void *y, int y_dtype, unsigned flags, char *wsb,
-                                       const si_ws_layout &ws, int32_t *status_dev, cudaStream_t stream) {
+                                       const si_ws_layout &ws, int32_t *status_dev, cudaStream_t stream,
+                                       const si_decode_extra *ex) {
+    static const si_decode_extra no_extra;
+    if (!ex) ex = &no_extra;
     si_persist::Params P;
     P.store_base = s->mem;
     for (int l = 0; l < s->n_layers; ++l) { P.rec_off[l] = s->rec_off[l]; P.n_loaded[l] = s->n_loaded[l]; }
@@ -846,9 +931,12 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.per_layer_lists = (flags & SI_FLAG_LIST_PER_LAYER) != 0 && !idx_offsets;
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
-    P.prof = si_decode_profile_buffer();
-    P.stream_only = si_decode_stream_only() & 0xFF;
-    if (((si_decode_stream_only() >> 8) & 0xF) && !wide) P.nstage = 2 * ((si_decode_stream_only() >> 8) & 0xF);   // diagnostics: shallower rings
+    P.prof = ex->profile;
+    P.stream_only = ex->skip_mask & 7;
+    if (ex->ring_stages > 0 && !wide && 2 * ex->ring_stages <= P.nstage) P.nstage = 2 * ex->ring_stages;   // diagnostics: shallower rings
+    P.wait_cycles = ex->wait_cycles > 0 ? ex->wait_cycles : si_persist::kWaitCycles;
+    P.withhold = ex->withhold;
+    P.chain_len = ex->chain_len; P.prenorm = ex->prenorm; P.norm_eps = ex->norm_eps; P.xn_out = (uint16_t *)ex->xn_out;
     int G = s->num_sms;
     if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
     // every CTA reduces at most kMaxGroups float4 column groups
@@ -858,8 +946,8 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // into groups that each take every n-th step on their own (launches of at least two steps per group;
     // a launch that uses fewer CTAs than SMs keeps one group).
     int ng = 1;
-    if (G == s->num_sms) {
-        const int forced = (si_decode_stream_only() >> 12) & 0xF;   // diagnostics: force a group count
+    if (G == s->num_sms && ex->chain_len == 0) {
+        const int forced = ex->step_groups;   // diagnostics: force a group count
         ng = forced ? forced : ((flags & SI_FLAG_STEPS_ANY_ORDER) ? si_persist::pick_groups(s->num_sms) : 1);
         while (ng > 1 && (s->num_sms % ng != 0 || n_steps < 2 * ng ||
                           (s->d_model / 4 + s->num_sms / ng - 1) / (s->num_sms / ng) > si_persist::kMaxGroups))

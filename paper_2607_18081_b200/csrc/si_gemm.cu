@@ -30,7 +30,7 @@ constexpr int kLoaderWarps = kLoaderThreads / 32;
 constexpr int kGemmThreads = kLoaderThreads + 32; // warp 8: MMA issue + tensor-memory allocation
 constexpr int kMaxStages = 6;
 constexpr int kChunkK = 64;                      // K elements per pipeline stage (128 bytes per row)
-constexpr long long kSpinLimit = 1ll << 24;      // bounded waits (mbarrier probes)
+constexpr long long kSpinLimit = 1ll << 24;      // default limit of every wait, in mbarrier probes
 constexpr size_t kPartialCap = (size_t)64 << 20; // bytes of fp32 partial tiles per contraction
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -46,9 +46,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false after kSpinLimit unsuccessful probes.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (long long i = 0; i < kSpinLimit; ++i)
+// Bounded wait: false after `limit` unsuccessful probes.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit) {
+    for (long long i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -295,6 +295,8 @@ struct GemmParams {
     uint16_t *h_out;               // gate/up: H [t_pad_total][nu_pad]
     void *y;                       // down: output [T][d_model]
     int y_f32, residual;
+    long long spin_limit;          // probes after which a wait gives up (SI_ERR_TIMEOUT)
+    int withhold;                  // diagnostics: the first gate/up CTA never loads the X tile of its first chunk
 };
 
 // Gate/up contraction.  One CTA per (union tile of 128, K split of d_model, token tile), flat grid.
@@ -368,9 +370,10 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         // gather: its gate and up tiles are two TMA copies out of the record matrix
         const int slot_first = P.union_slots[mt * 128];
         const bool run = P.union_slots[mt * 128 + 127] - slot_first == 127;
+        int armed = 0;                       // (thread 0) chunks whose tensor copies it has started
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
-            if (!mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
+            if (!mbar_wait(&empty[st], ph ^ 1, P.spin_limit)) { *failed = 1; break; }
             uint8_t *sg = tiles + (size_t)st * stage_bytes + off0, *su = sg + 128 * 128;
             if (!run) {
 #pragma unroll
@@ -380,7 +383,8 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                     grow[j] += 128;
                 }
             }
-            if (tid == 0) {      // the dense X tile comes as one TMA copy (token rows past T read as zero)
+            if (tid == 0) armed = c + 1;
+            if (tid == 0 && !(P.withhold && blockIdx.x == 0 && c == 0)) {      // the dense X tile comes as one TMA copy (token rows past T read as zero)
                 uint8_t *stage = tiles + (size_t)st * stage_bytes;
                 mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u + (run ? 2u * 128u * 128u : 0u));
                 if (run) {
@@ -393,7 +397,10 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         }
         cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
         // ---------------------------------------------------------------- epilogue
-        bool ok = !*failed && mbar_wait(accbar, 0);
+        bool ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
+        if (!ok && tid == 0)                 // a wait ran out: the tensor copies already started must still land before the CTA goes
+            for (int c = armed > P.nstage ? armed - P.nstage : 0; c < armed; ++c)
+                if (!(P.withhold && blockIdx.x == 0 && c == 0)) mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
         // a warp reads tensor-memory lanes 32*(warp % 4) ..: warps w and w + 4 share the rows and take
         // alternate 16-column blocks.  Thread row r = union row mt*128 + r: N gate values, N up values
@@ -444,7 +451,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
                 const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
-                ok = mbar_wait(&full[st], ph) && !*failed;
+                ok = mbar_wait(&full[st], ph, P.spin_limit) && !*failed;
                 if (!ok) break;
                 fence_async_proxy();               // the gathered rows were written by cp.async (generic proxy)
                 tc_fence_after();
@@ -595,6 +602,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         // the down rows of the first chunks (one per stage: the ring is empty) are fetched while the
         // gate/up kernel finishes
         const int pre = n_chunks < P.nstage ? n_chunks : P.nstage;
+        int armed_to = 0; bool h_primed = false;     // (thread 0) H tiles started: the primed ones, then up to chunk armed_to
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             int slots[4];
@@ -605,18 +613,20 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
             }
             if (c == pre) {      // (n_chunks > nstage) the ring is primed: now H is needed
                 pdl_wait();
+                h_primed = true;
                 if (tid == 0)
                     for (int q = 0; q < pre; ++q) {
                         mbar_arrive_expect_tx(&full[q], (uint32_t)N * 128u);
                         tma_load_tile(tiles + (size_t)q * stage_bytes + 64 * 256, &h_map, (c0 + q) * kChunkK, tok0, &full[q]);
                     }
             }
-            if (c >= pre && !mbar_wait(&empty[st], ph ^ 1)) { *failed = 1; break; }
+            if (c >= pre && !mbar_wait(&empty[st], ph ^ 1, P.spin_limit)) { *failed = 1; break; }
             uint8_t *sa = tiles + (size_t)st * stage_bytes;
 #pragma unroll
             for (int j = 0; j < 4; ++j)                                      // padded entries carry a valid slot
                 cp_async16(sa + j * 4096 + dst0, dsrc0 + (size_t)slots[j] * P.rec_bytes);
             if (c >= pre && tid == 0) {      // the dense H tile comes as one TMA copy
+                armed_to = c + 1;
                 mbar_arrive_expect_tx(&full[st], (uint32_t)N * 128u);
                 tma_load_tile(sa + 64 * 256, &h_map, (c0 + c) * kChunkK, tok0, &full[st]);
             }
@@ -624,6 +634,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         }
         if (n_chunks <= pre) {   // short K range: everything was primed above
             pdl_wait();
+            h_primed = true;
             if (tid == 0)
                 for (int q = 0; q < pre; ++q) {
                     mbar_arrive_expect_tx(&full[q], (uint32_t)N * 128u);
@@ -631,7 +642,12 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 }
         }
         cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
-        bool ok = !*failed && mbar_wait(accbar, 0);
+        bool ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
+        if (!ok && tid == 0) {               // a wait ran out: the tensor copies already started must still land before the CTA goes
+            const int armed = armed_to > pre ? armed_to : (h_primed ? pre : 0);
+            for (int c = armed > P.nstage ? armed - P.nstage : 0; c < armed; ++c)
+                mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
+        }
         tc_fence_after();
         // thread holds output column mt*128 + r for the tokens; warps w and w + 4 share the rows and
         // take alternate 16-token blocks
@@ -674,7 +690,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
                 const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
-                ok = mbar_wait(&full[st], ph) && !*failed;
+                ok = mbar_wait(&full[st], ph, P.spin_limit) && !*failed;
                 if (!ok) break;
                 fence_async_proxy();               // the gathered rows were written by cp.async (generic proxy)
                 tc_fence_after();
@@ -867,9 +883,65 @@ int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, con
     return SI_OK;
 }
 
+// The union stage of a multi-token call: the ascending union of the lists (padded to nu_pad entries), its
+// size, and -- when the tokens have lists of their own -- one slot bitmap per token; the counters the
+// contractions expect to be zero are cleared on the way.  One block when the lists are short and few,
+// several blocks with global atomics otherwise.
+static int union_stage_launch(const si_store *s, int n_loaded, int n_lists, bool own_lists, const int32_t *idx,
+                              const int32_t *idx_offsets, int k_fixed, const UnionScratch &us, int32_t *uni,
+                              int32_t *n_union, int nu_pad, int32_t *status_dev, cudaStream_t stream) {
+    const int words = (n_loaded + 31) / 32;
+    // token bitmaps are only read (and so only cleared) when the tokens have lists of their own
+    char *z0 = own_lists ? (char *)us.tokbits : (char *)us.bitmap;
+    const size_t zero_bytes = us.zero_bytes - (size_t)(z0 - (char *)us.tokbits);
+    const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
+    const size_t small_smem = ((size_t)2 * words + 2 + (own_lists ? (size_t)n_lists * us.mask_words : 0)) * 4;
+    if (entries <= kUnionSmallEntries && small_smem <= kUnionSmallSmem) {
+        // few entries, few lists: one block does everything in shared memory, the clearing of the
+        // counters included
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_union_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUnionSmallSmem));
+        uint32_t *zc = (uint32_t *)us.ticket;                          // ticket words and the arrival counters
+        const size_t zc_bytes = us.zero_bytes - (size_t)((char *)us.ticket - (char *)us.tokbits);
+        si_union_small_kernel<<<1, 1024, small_smem, stream>>>(
+            idx, idx_offsets, k_fixed, n_lists, n_loaded, zc, (int)(zc_bytes / 4),
+            own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
+    } else {
+        SI_CUDA_TRY(cudaMemsetAsync(z0, 0, zero_bytes, stream));
+        si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
+            idx, idx_offsets, k_fixed, n_lists, n_loaded, us.bitmap, own_lists ? us.tokbits : nullptr, us.mask_words,
+            us.ticket, uni, n_union, nu_pad, status_dev);
+    }
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}
+
+int si_union_masks_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
+                          int k_fixed, int32_t *union_out, int32_t *n_union_out, uint32_t *masks_out,
+                          void *workspace, size_t ws_bytes, cudaStream_t stream) {
+    si_ws_layout ws = si_ws_carve(s, T < 2 ? 2 : T, k_fixed, 1);
+    if (ws_bytes < ws.total) return SI_ERR_NOMEM;
+    char *wsb = (char *)workspace;
+    const int n_loaded = s->n_loaded[layer];
+    const size_t nl_pad = si_align_up((size_t)n_loaded, 128);
+    int32_t *uni = (int32_t *)(wsb + ws.union_off);
+    int32_t *n_union = uni + nl_pad;
+    long long cap = idx_offsets ? (long long)n_loaded : (long long)T * k_fixed;
+    if (cap > n_loaded) cap = n_loaded;
+    const int nu_pad = (int)si_align_up((size_t)cap, 128);
+    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, 0);
+    if (us.zero_bytes > ws.mask_bytes) return SI_ERR_NOMEM;
+    int rc = union_stage_launch(s, n_loaded, T, true, idx, idx_offsets, k_fixed, us, uni, n_union, nu_pad, nullptr, stream);
+    if (rc) return rc;
+    SI_CUDA_TRY(cudaMemcpyAsync(union_out, uni, (size_t)n_loaded * 4, cudaMemcpyDeviceToDevice, stream));
+    SI_CUDA_TRY(cudaMemcpyAsync(n_union_out, n_union, 4, cudaMemcpyDeviceToDevice, stream));
+    SI_CUDA_TRY(cudaMemcpyAsync(masks_out, us.tokbits, (size_t)T * us.mask_words * 4, cudaMemcpyDeviceToDevice, stream));
+    return SI_OK;
+}
+
 int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, const int32_t *idx,
                           const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype, unsigned flags,
-                          void *workspace, size_t ws_bytes, int32_t *status_dev, cudaStream_t stream) {
+                          void *workspace, size_t ws_bytes, int32_t *status_dev, cudaStream_t stream,
+                          long long spin_limit, int withhold) {
     const int d = s->d_model;
     if (d % 128 != 0) return SI_ERR_UNSUPPORTED;
     si_ws_layout ws = si_ws_carve(s, T < 2 ? 2 : T, k_fixed, 1);       // the multi-token regions exist from T_max = 2 on
@@ -908,32 +980,9 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn);
     if (us.zero_bytes > ws.mask_bytes) return SI_ERR_NOMEM;
     {
-        const int words = (n_loaded + 31) / 32;
-        // token bitmaps are only read (and so only cleared) when the tokens have lists of their own
-        char *z0 = own_lists ? (char *)us.tokbits : (char *)us.bitmap;
-        const size_t zero_bytes = us.zero_bytes - (size_t)(z0 - (char *)us.tokbits);
-        const int n_lists = shared ? 1 : T;
-        const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
-        const size_t small_smem = ((size_t)2 * words + 2 + (own_lists ? (size_t)n_lists * us.mask_words : 0)) * 4;
-        if (entries <= kUnionSmallEntries && small_smem <= kUnionSmallSmem) {
-            // few entries, few lists: one block does everything in shared memory, the clearing of the
-            // counters included
-            static bool attr_set = false;
-            if (!attr_set) {
-                SI_CUDA_TRY(cudaFuncSetAttribute(si_union_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUnionSmallSmem));
-                attr_set = true;
-            }
-            uint32_t *zc = (uint32_t *)us.ticket;                          // ticket words and the arrival counters
-            const size_t zc_bytes = us.zero_bytes - (size_t)((char *)us.ticket - (char *)us.tokbits);
-            si_union_small_kernel<<<1, 1024, small_smem, stream>>>(
-                idx, idx_offsets, k_fixed, n_lists, n_loaded, zc, (int)(zc_bytes / 4),
-                own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
-        } else {
-            SI_CUDA_TRY(cudaMemsetAsync(z0, 0, zero_bytes, stream));
-            si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
-                idx, idx_offsets, k_fixed, n_lists, n_loaded, us.bitmap, own_lists ? us.tokbits : nullptr, us.mask_words,
-                us.ticket, uni, n_union, nu_pad, status_dev);
-        }
+        int rc = union_stage_launch(s, n_loaded, shared ? 1 : T, own_lists, idx, idx_offsets, k_fixed, us, uni, n_union,
+                                    nu_pad, status_dev, stream);
+        if (rc) return rc;
     }
     // ---- tiling
     const int n_tok = tok_tiles > 1 ? tile_n : t_pad_total;
@@ -950,6 +999,7 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.tokbits = own_lists ? us.tokbits : nullptr; P.mask_words = us.mask_words;
     P.h_out = (uint16_t *)(wsb + ws.h_off);
     P.y = y; P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
+    P.spin_limit = spin_limit > 0 ? spin_limit : kSpinLimit; P.withhold = withhold;
     // gate/up: K = d_model may be split up to s1 ways (what the partial buffer holds); the kernel
     // picks the split from the real union size so that one wave of CTAs covers the SM slots (two CTAs
     // per SM with few tokens: the gathers are latency-bound)

@@ -169,6 +169,7 @@ extern "C" int si_load_neurons(si_store_t *store, int layer, const void *w_gate,
     if (n_loaded != store->n_loaded[layer] || n_base < 0 || n_base > n_loaded) return SI_ERR_INVALID_ARG;
     if (n_loaded > 0 && !neuron_ids) return SI_ERR_INVALID_ARG;
     if (!si_aligned16(w_gate) || !si_aligned16(w_up) || !si_aligned16(w_down)) return SI_ERR_ALIGNMENT;
+    if (int rc = si_check_device(store)) return rc;
     const int d = store->d_model, F = store->d_ff;
     {   // host-side validation of the neuron file: in range, distinct
         std::vector<char> seen((size_t)F, 0);

@@ -1,5 +1,5 @@
 """CPU-only checks of the C-ABI boundary: the library builds for sm_100a, loads, and exports
-every function declared in include/selectinfer.h.  No compute call is made."""
+every function declared in include/selectinfer.h and include/selectinfer_debug.h.  No compute call is made."""
 import ctypes
 import os
 import re
@@ -8,9 +8,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "selectinfer.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(si_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    for header in ("selectinfer.h", "selectinfer_debug.h"):
+        text = open(os.path.join(ROOT, "include", header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(si_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_builds_loads_and_exports_every_declared_symbol():

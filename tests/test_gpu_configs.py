@@ -6,7 +6,7 @@ import torch
 
 from oracle import selectinfer_oracle as so
 from paper_2607_18081_b200 import workloads as wl
-from tests.gpu_utils import LoadedModel, assert_close, from_dev, to_dev
+from tests.gpu_utils import LoadedModel, assert_close, assert_close_f32, from_dev, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -52,35 +52,72 @@ def test_c2_full_stack_one_launch_sampled(api):
     assert torch.equal(y, y2)
 
 
-@pytest.mark.parametrize("loaded_pct,active_pct", [(30, 5), (50, 20), (100, 50)])
-def test_c5_cells_decode_and_selector(api, loaded_pct, active_pct):
-    """Config 5 (Llama-3-8B FFN shape) cells: Zipf lists through the decode kernel, and N(0,1)
-    scores through si_layer_forward (selector + FFN) with bit-exact selection."""
-    cfg = wl.CONFIGS["c5"].with_(loaded_pct=loaded_pct, active_pct=active_pct, n_layers=1)
-    m = LoadedModel(cfg)
-    k, d, n = cfg.k_active, cfg.d_model, cfg.n_loaded
+@pytest.mark.parametrize("loaded_pct", wl.C5_LOADED)
+def test_c5_all_cells_decode_and_selector(api, loaded_pct):
+    """Config 5 (Llama-3-8B FFN shape), all sixteen cells (four active fractions per loaded fraction, one
+    layer): Zipf lists through the decode kernel in the stack call bench.py times, and N(0,1) scores through
+    si_layer_forward (selector + FFN) with bit-exact selection."""
+    base = wl.CONFIGS["c5"].with_(loaded_pct=loaded_pct, n_layers=1)
+    m = LoadedModel(base)
+    d, n = base.d_model, base.n_loaded
     tokens = 2
-    lists = wl.zipf_lists(cfg, 0, tokens)
-    x = wl.x_tokens(cfg, 0, tokens)
-    ws = m.store.workspace(1, k, tokens)
-    st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    y = torch.empty(tokens, d, dtype=torch.float32, device="cuda")
-    api.si_decode_stack_forward(m.store.handle, tokens, [0] * tokens, to_dev(x, cfg.dtype),
-                                torch.from_numpy(lists).cuda(), None, k, y, 0, ws, st)
-    torch.cuda.synchronize()
-    assert st.item() == 0
-    for t in range(tokens):
-        assert_close(from_dev(y[t]), m.oracle_y(0, x[t], lists[t]), f"cell {loaded_pct}/{active_pct} token {t}")
-    # runtime selector on the cell's scores, then the FFN on the selected list
-    sc = wl.scores(cfg, 0, 1)[0]
-    sel_out = torch.empty(k, dtype=torch.int32, device="cuda")
-    cnt = torch.zeros(4, dtype=torch.int32, device="cuda")
+    x = wl.x_tokens(base, 0, tokens)
+    sc = wl.scores(base, 0, 1)[0]
+    scd = torch.from_numpy(sc).cuda()
     sws = torch.zeros(max(api.si_select_workspace_bytes(n), 256), dtype=torch.uint8, device="cuda")
-    api.si_select(torch.from_numpy(sc).cuda(), api.SI_SELECT_TOPK, k, 0.0, 0, sel_out, cnt, sws)
-    ysel = torch.empty(d, dtype=torch.float32, device="cuda")
-    api.si_layer_forward(m.store.handle, 0, to_dev(x[0], cfg.dtype), 1, torch.from_numpy(sc).cuda(), k, None, None,
-                         ysel, 0, ws, st)
-    torch.cuda.synchronize()
-    want = np.sort(np.argsort(-sc.astype(np.float64), kind="stable")[:k]).astype(np.int32)
-    assert int(cnt[0].item()) == k and np.array_equal(sel_out.cpu().numpy(), want)
-    assert_close(from_dev(ysel), m.oracle_y(0, x[0], want), "selected list")
+    for active_pct in wl.C5_ACTIVE:
+        cfg = base.with_(active_pct=active_pct)
+        k = cfg.k_active
+        lists = wl.zipf_lists(cfg, 0, tokens)
+        ws = m.store.workspace(1, k, tokens)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        y = torch.empty(tokens, d, dtype=torch.float32, device="cuda")
+        api.si_decode_stack_forward(m.store.handle, tokens, [0] * tokens, to_dev(x, cfg.dtype),
+                                    torch.from_numpy(lists).cuda(), None, k, y, 0, ws, st)
+        # the persistent kernel as well (a stack call of two steps uses the per-step kernels)
+        y8 = torch.empty(8, d, dtype=torch.float32, device="cuda")
+        x8 = to_dev(np.tile(x, (4, 1)), cfg.dtype)
+        l8 = torch.from_numpy(np.tile(lists, (4, 1))).cuda()
+        ws8 = m.store.workspace(1, k, 8)
+        api.si_decode_stack_forward(m.store.handle, 8, [0] * 8, x8, l8, None, k, y8, 0, ws8, st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        for t in range(tokens):
+            ref = m.oracle_y(0, x[t], lists[t])
+            assert_close_f32(from_dev(y[t]), ref, f"cell {loaded_pct}/{active_pct} token {t}")
+            assert_close_f32(from_dev(y8[6 + t]), ref, f"cell {loaded_pct}/{active_pct} token {t}, persistent kernel")
+        # runtime selector on the cell's scores, then the FFN on the selected list
+        sel_out = torch.empty(k, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(4, dtype=torch.int32, device="cuda")
+        api.si_select(scd, api.SI_SELECT_TOPK, k, 0.0, 0, sel_out, cnt, sws)
+        ysel = torch.empty(d, dtype=torch.float32, device="cuda")
+        api.si_layer_forward(m.store.handle, 0, to_dev(x[0], cfg.dtype), 1, scd, k, None, None, ysel, 0, ws, st)
+        torch.cuda.synchronize()
+        want = np.sort(np.argsort(-sc.astype(np.float64), kind="stable")[:k]).astype(np.int32)
+        assert int(cnt[0].item()) == k and np.array_equal(sel_out.cpu().numpy(), want)
+        assert np.array_equal(want, so.select_topk(sc, k))
+        assert_close_f32(from_dev(ysel), m.oracle_y(0, x[0], want), f"cell {loaded_pct}/{active_pct} selected list")
+
+
+def test_c4_prefill_own_model_all_tokens_two_layers(api):
+    """Config 4 on a model built from config 4's own seeds: all 512 tokens of two layers, one shared list =
+    the first 40 % of the loaded slots, every token against the oracle."""
+    cfg = wl.CONFIGS["c4"]
+    m = LoadedModel(cfg, n_layers=2)
+    T, k, d = cfg.tokens, cfg.k_active, cfg.d_model
+    assert (T, k) == (512, 3082)
+    shared = np.arange(k, dtype=np.int32)
+    idx = torch.from_numpy(shared).cuda()
+    ws = m.store.workspace(T, k, 1)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for layer in range(2):
+        x = wl.x_tokens(cfg, layer, T)
+        y = torch.empty(T, d, dtype=torch.bfloat16, device="cuda")
+        api.si_ffn_forward(m.store.handle, layer, to_dev(x, cfg.dtype), T, idx, None, k, y, api.SI_FLAG_SHARED_LIST, ws, st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        wg, wu, wd = m.host[layer]
+        ref = so.ffn_tokens(wg, wu, wd, x, [m.ids[layer][shared]] * T, dtype=cfg.dtype, threads=so.host_threads())
+        yh = from_dev(y)
+        for t in range(T):
+            assert_close(yh[t], ref[t], f"layer {layer} token {t}")

@@ -5,7 +5,7 @@ import torch
 
 from oracle import selectinfer_oracle as so
 from paper_2607_18081_b200 import workloads as wl
-from tests.gpu_utils import LoadedModel, assert_close, from_dev, to_dev
+from tests.gpu_utils import LoadedModel, assert_close, assert_close_f32, from_dev, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -256,33 +256,30 @@ def test_7b_shaped_step_groups(api):
          max(lens), api.SI_FLAG_RESIDUAL, lambda s: ragged[s]),
         ("per layer", torch.from_numpy(per_layer).cuda(), None, k, api.SI_FLAG_LIST_PER_LAYER, lambda s: per_layer[s % L]),
     ]
-    try:
-        for name, idx, offsets, kk, flags, list_of in cases:
-            refs = None
-            for ng in (1, 2, 4, 0):       # 0: the library's own choice under SI_FLAG_STEPS_ANY_ORDER
-                api.lib().si_debug_decode_stream_only(ng << 12)
-                runs = []
-                for _ in range(2):
-                    y = torch.full((steps, cfg.d_model), 9.0, dtype=torch.float32, device="cuda")
-                    st = _status()
-                    # (the debug knob fixes the group count; the flag is what a caller would pass for more than one)
-                    api.si_decode_stack_forward(m.store.handle, steps, None, xd, idx, offsets, kk, y,
-                                                flags | (api.SI_FLAG_STEPS_ANY_ORDER if ng != 1 else 0), ws, st)
-                    torch.cuda.synchronize()
-                    assert st.item() == 0, (name, ng, api.strerror(int(st.item())))
-                    runs.append(y.cpu())
-                assert torch.equal(runs[0], runs[1]), f"{name}: {ng} groups not run-to-run bit-stable"
-                if refs is None:
-                    refs = []
-                    for s in range(steps):
-                        ref = m.oracle_y(s % L, x[s], list_of(s))
-                        if flags & api.SI_FLAG_RESIDUAL:
-                            ref = ref + wl.bits_to_float64(x[s], cfg.dtype)
-                        refs.append(ref)
+    for name, idx, offsets, kk, flags, list_of in cases:
+        refs = None
+        for ng in (1, 2, 4, 0):       # 0: the library's own choice under SI_FLAG_STEPS_ANY_ORDER
+            runs = []
+            for _ in range(2):
+                y = torch.full((steps, cfg.d_model), 9.0, dtype=torch.float32, device="cuda")
+                st = _status()
+                # (the per-call option fixes the group count; the flag is what a caller would pass for more than one)
+                api.si_debug_decode_stack_forward(m.store.handle, steps, None, xd, idx, offsets, kk, y,
+                                                  flags | (api.SI_FLAG_STEPS_ANY_ORDER if ng != 1 else 0), ws, st,
+                                                  step_groups=ng)
+                torch.cuda.synchronize()
+                assert st.item() == 0, (name, ng, api.strerror(int(st.item())))
+                runs.append(y.cpu())
+            assert torch.equal(runs[0], runs[1]), f"{name}: {ng} groups not run-to-run bit-stable"
+            if refs is None:
+                refs = []
                 for s in range(steps):
-                    assert_close(runs[0][s].double().numpy(), refs[s], f"{name}, {ng} groups, step {s}")
-    finally:
-        api.lib().si_debug_decode_stream_only(0)
+                    ref = m.oracle_y(s % L, x[s], list_of(s))
+                    if flags & api.SI_FLAG_RESIDUAL:
+                        ref = ref + wl.bits_to_float64(x[s], cfg.dtype)
+                    refs.append(ref)
+            for s in range(steps):
+                assert_close_f32(runs[0][s].double().numpy(), refs[s], f"{name}, {ng} groups, step {s}")
 
 
 def test_check_flag_reports_bad_lists_without_faulting(api):
