@@ -31,7 +31,11 @@ typedef struct si_debug_decode_opts {
                               arithmetic, accumulator hand-over, wait for the hand-over buffer, dot products +
                               exchange); 6..7: second set (wait for the hand-over buffer, wait for a record);
                               8..13: first reducer warp (idle, wait for a free partial-ring slot, copy
-                              accumulators out, publish, wait for all SMs, reduce + write y). */
+                              accumulators out, publish, wait for all SMs, reduce + write y).
+                              Chained launches: slots 0..7 first consumer set, 8..15 second set (wait for
+                              the input row, normalisation + records, wait for the second set / park the
+                              accumulators, store the CTA's row, wait for every CTA's row, gather the rows,
+                              wait for the class sums, column sums + y + next input row). */
 } si_debug_decode_opts_t;
 
 /* si_decode_stack_forward with the options above (opts == NULL: identical to it). */

@@ -23,14 +23,18 @@
 //     fixed order (lane rows ascending, warp butterfly: deterministic split-K) and write y
 //     once.  The reduction trails the record stream and never stalls it.
 //
-// Chained mode (Params::chain_len > 0): step s takes the output row of step s - 1 as its input unless
-// s is the first step of a chain (s mod chain_len == 0), the way the FFN of layer l + 1 sees what layer
-// l produced.  Nothing of a step's arithmetic can then start before the step before it is complete: the
-// step's cross-SM sum runs at once (no lag), every CTA publishes "my columns of y are written", and the
-// producer issues the bulk copy of the next step's input only when every CTA has said so.  The record
-// rings are not held back: the lists are known up front (the set is fixed per prompt), so the first
-// records of the next step are in shared memory before its input is.  With Params::prenorm the input
-// row is normalised to unit root mean square (and rounded to the store type) before the dot products.
+// Chained mode (template parameter CH; Params::chain_len > 0): step s takes the output row of step s - 1
+// as its input unless s is the first step of a chain (s mod chain_len == 0), the way the FFN of layer
+// l + 1 sees what layer l produced.  Nothing of a step's arithmetic can start before the step before it is
+// complete, so the time between the last record of a step and the first dot product of the next is pure
+// latency and the kernel is built to make it short: the reducer warps stay out of it; the consumers
+// themselves store the CTA's partial row as 8-byte words {value, tag}, gather their CTA's columns of every
+// row by polling those words (no fence, no flag, no second round trip), add them in a fixed order, write y
+// and publish the next input row the same way, and every consumer polls the words of the row it needs.
+// The record rings are not held back: the lists are known up front (the set is fixed per prompt), so a
+// step's first records are in shared memory, and the ones behind them on their way into L2, before its
+// input exists.  With Params::prenorm the input row is normalised to unit root mean square (and rounded
+// to the store type) before the dot products.
 //
 // Every wait is bounded: on expiry the kernel records SI_ERR_TIMEOUT, raises a grid-wide
 // abort flag, lets its outstanding copies land and returns.
@@ -49,6 +53,7 @@ constexpr int kConsumers = kSets * kSetThreads;
 constexpr int kConsumerWarps = kConsumers / 32;
 constexpr int kReducerWarps = 3;
 constexpr int kThreads = 32 + kConsumers + 32 * kReducerWarps;        // producer, consumers, reducers
+constexpr int kThreadsChained = 32 + kConsumers;                      // chained mode has no reducer warps
 constexpr int kMaxGroups = 32;                    // most float4 column groups one CTA reduces (d_model / 4 / CTAs per step group, rounded up)
 constexpr int kCounterStride = 64;                // uint32 per step: written at +0, reduced at +32 (own 128-byte lines)
 constexpr int kMaxStages = 16;
@@ -59,6 +64,9 @@ constexpr int kProfSlots = 16;                    // int64 cycle counters per SM
 constexpr int kLag = 4;                           // a step's cross-SM reduction starts this many steps later
 constexpr long long kWaitCycles = 4000000000ll;   // default limit of every wait: ~2 s at 1.9 GHz
 constexpr long long kDrainCycles = 40000000ll;    // least time a leaving producer gives its copies in flight to land
+constexpr int kLLRows = 8;                        // chained mode: most partial rows one consumer thread gathers per step
+constexpr int kChainCmb = 0, kChainXch = 1, kChainOwn = 2;   // chained mode: which hand-over barrier serves what ([0][..])
+constexpr int kChainRows = 0, kChainInput = 1;               // ... and [1][..]: "every CTA's row is written", "the input row is written"
 
 struct Params {
     const char *store_base;
@@ -93,6 +101,12 @@ struct Params {
     int prenorm;                  // the input row is scaled to unit root mean square before the FFN
     float norm_eps;
     uint16_t *xn_out;             // optional [n_steps][d_model]: the normalised, rounded input every step used
+    // chained mode: the two exchanges between the SMs go through words that carry their own "ready" mark --
+    // 8 bytes = {payload, tag}, written and read as a whole, tag = 1 + step -- so a reader polls the data
+    // itself and no fence, flag or second round trip stands between a store and its use
+    uint2 *ll_partial;            // [G][d_model] {fp32 partial sum of the CTA's records, tag}, zero at launch
+    uint2 *ll_x;                  // [2][d_model / 2] {two 16-bit values of the next input row, tag}, zero at launch
+    unsigned csum_off;            // chained mode: byte offset of the [columns][classes] class sums in shared memory
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -149,6 +163,18 @@ __device__ __forceinline__ void red_add_gpu_f4(float4 *p, float4 v) {
     asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
                  : "memory");
 }
+// 16 bytes = two {payload, tag} words; each 8-byte word is written by one store and read whole
+__device__ __forceinline__ uint4 ld_relaxed_gpu_v4(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_gpu_v4(uint4 *p, uint4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_gpu_v2(uint2 *p, uint2 v) {
+    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -161,17 +187,38 @@ __device__ __forceinline__ unsigned ld_relaxed_gpu(const unsigned *p) {
 }
 // Bounded wait until *ctr >= target; gives up on the grid-wide or CTA-local abort flag.
 __device__ __forceinline__ bool counter_wait_bounded(const unsigned *ctr, unsigned target, const unsigned *grid_abort,
-                                                     volatile int *cta_abort, long long limit, unsigned sleep_ns = 64) {
+                                                     volatile int *cta_abort, long long limit) {
     if (ld_acquire_gpu(ctr) >= target) return true;
     long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 16; ++i) {
             if (ld_acquire_gpu(ctr) >= target) return true;
-            if (sleep_ns) __nanosleep(sleep_ns);
+            __nanosleep(64);
         }
         if (*cta_abort || ld_relaxed_gpu(grid_abort)) return false;
         if (clock64() - t0 > limit) return false;
     }
+}
+// Chained mode: lane 0 of a warp polls an arrival counter that is only a hint ("the words you are about to
+// read have probably all been written") -- the words carry their own tags, so nothing depends on the counter
+// being ordered with them.  Returns false when the wait ran out or an abort flag is up.
+// One thread of the CTA polls (thousands of lanes polling one word would queue up in front of the very
+// increments they wait for) and passes the news on through a shared-memory barrier with one expected arrival.
+__device__ __forceinline__ bool hint_wait_cta(const unsigned *ctr, unsigned target, const unsigned *grid_abort,
+                                              volatile int *cta_abort, long long limit, bool poller, uint64_t *bar, uint32_t parity) {
+    if (poller) {
+        const long long t0 = clock64();
+        unsigned spins = 0;
+        while (ld_relaxed_gpu(ctr) < target) {
+            if ((++spins & 31u) == 0 && (*cta_abort || ld_relaxed_gpu(grid_abort) || clock64() - t0 > limit)) return false;
+        }
+        mbar_arrive(bar);
+        return true;
+    }
+    return mbar_wait_bounded(bar, parity, cta_abort, limit);
+}
+__device__ __forceinline__ void red_add_relaxed_gpu(unsigned *p, unsigned v) {
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t pol;
@@ -276,9 +323,9 @@ struct Smem {
     int meta[kMaxStages];
     uint4 desc[kSets][kDescRing];      // {src lo, src hi, bytes (0: nothing to copy), meta}
     float2 setpart[kSets][2][2 * kSetWarps];   // [set][buf][warp] = (gate, up) partial dot products (16 warps in the one wide set)
-    float normpart[kSets][2][2 * kSetWarps];   // [set][step parity][warp] = sum of squares of the warp's share of the input row (prenorm)
     volatile int cta_abort;
 };
+static_assert(sizeof(Smem) <= 3008, "the eight ring stages of d_model = 4096 leave 3008 bytes for this struct");
 
 __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code) {
     if (!sm->cta_abort) {
@@ -288,12 +335,362 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Chained mode, consumer side.  A step is two functions that are deliberately not inlined: the record
+// loop runs at the register limit, and the values one half keeps alive must not be in the other half's way
+// (a spill inside the record loop goes to L2 here, the shared memory carve-out leaves next to no L1).
+// What crosses from one to the other is a handful of integers; the sums cross through memory.
+
+// First half: fetch the step's input row (the caller's, or the {values, tag} words the SMs wrote at the
+// end of the step before), normalise it if asked to, run the set's records, and deliver the CTA's partial
+// row: the second set parks its accumulators in shared memory, the first adds them to its own and stores
+// the row as {partial sum, tag} words, then counts the row as written (a hint for the pollers).
+// ring: stage | phase parity << 8 | exchange-buffer parity << 9 of the set's next ring item.
+// optional phase profile of the chained steps: thread 0 of each set adds the cycles since its last stamp to a slot
+#define SI_CPROF(slot) do { if (cprof) { const long long now_ = clock64(); atomicAdd((unsigned long long *)(P.prof + (size_t)blockIdx.x * kProfSlots + (slot) + 8 * q_), (unsigned long long)(now_ - pt_)); pt_ = now_; } } while (0)
+
+template <int DT, int NCH, bool kFull>
+__device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, int step, unsigned &ring) {
+    constexpr int kSets = 2, kSetWarps = 8, kSetThreads = 256;
+    const int d = P.d_model, chunks = P.chunks, rec_bytes = d * 6, S = P.nstage / kSets;
+    const int G = gridDim.x, b = blockIdx.x;
+    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)P.nstage * rec_bytes + (size_t)kSets * d * 4);
+    float *comb = reinterpret_cast<float *>(smem + (size_t)P.nstage * rec_bytes);      // [d_model] second set's accumulators
+    volatile int *cta_abort = &sm->cta_abort;
+    const long long wait_limit = P.wait_cycles;
+    const int ct = threadIdx.x - 32, lane = ct & 31;
+    const int q = ct / kSetThreads, t = ct & (kSetThreads - 1), sw = t >> 5;
+    uint64_t *sfull = sm->full + q * S, *sempty = sm->empty + q * S;
+    const int *smeta = sm->meta + q * S;
+    const uint8_t *sring = smem + (size_t)q * S * rec_bytes;
+    int st = (int)(ring & 0xFFu); uint32_t ph = (ring >> 8) & 1u, recs = (ring >> 9) & 1u;
+    bool fail = false;
+    const uint32_t tag = (uint32_t)step + 1u;
+    const bool cprof = P.prof != nullptr && t == 0;
+    const int q_ = q;
+    long long pt_ = cprof ? clock64() : 0;
+
+    unsigned long long xr[NCH][4], acc[NCH][4];   // packed fp32 pairs
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { acc[i][e] = 0ull; xr[i][e] = 0ull; }
+    const int cnt = step_geom(P, step, G * kSets, kSets * b + q).cnt;
+    // ---- the input row
+    if (step % P.chain_len == 0) {
+        const uint4 *xs = reinterpret_cast<const uint4 *>(P.x + (size_t)(step / P.chain_len) * d);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int c = t + kSetThreads * i;
+            if (kFull || c < chunks) unpack8p<DT>(__ldg(xs + c), xr[i]);
+        }
+        if (ct == 0) mbar_arrive(&sm->accfull[1][kChainInput]);      // (nothing to wait for: keeps the barrier's phase in step)
+    } else {
+        // 8-byte words {two 16-bit values, tag = this step}; the count of CTAs that have written their
+        // columns is only a hint that spares the memory system 75 000 threads polling the words while the
+        // last CTAs are still at work: what counts is the tag in every word
+        const uint4 *lx = reinterpret_cast<const uint4 *>(P.ll_x + (size_t)(step & 1) * (d / 2));
+        fail |= !hint_wait_cta(P.counters + (size_t)(step - 1) * kCounterStride + 32, (unsigned)G, P.ctrl + 1, cta_abort,
+                               wait_limit, ct == 0, &sm->accfull[1][kChainInput], (uint32_t)(step & 1));
+        const long long t0 = clock64();
+        uint32_t spins = 0;
+        while (!fail) {
+            bool good = true;
+            uint4 w[NCH][2];
+#pragma unroll
+            for (int i = 0; i < NCH; ++i)
+                if (kFull || t + kSetThreads * i < chunks) {
+                    w[i][0] = ld_relaxed_gpu_v4(lx + (size_t)(t + kSetThreads * i) * 2);
+                    w[i][1] = ld_relaxed_gpu_v4(lx + (size_t)(t + kSetThreads * i) * 2 + 1);
+                }
+#pragma unroll
+            for (int i = 0; i < NCH; ++i)
+                if (kFull || t + kSetThreads * i < chunks) {
+                    good &= w[i][0].y == (uint32_t)step && w[i][0].w == (uint32_t)step && w[i][1].y == (uint32_t)step && w[i][1].w == (uint32_t)step;
+                    xr[i][0] = pair_of<DT>(w[i][0].x); xr[i][1] = pair_of<DT>(w[i][0].z);
+                    xr[i][2] = pair_of<DT>(w[i][1].x); xr[i][3] = pair_of<DT>(w[i][1].z);
+                }
+            if (good) break;
+            if ((++spins & 63u) == 0 && (*cta_abort || ld_relaxed_gpu(P.ctrl + 1) || clock64() - t0 > wait_limit)) fail = true;
+        }
+    }
+    if (P.prenorm) {
+        // sum of squares of the row: thread slice, warp butterfly, then (after the barrier below) the set's
+        // warps in warp order -- the same order in every set of every CTA.  The warp sums use the exchange
+        // buffer the next record would use; the record after it uses the other one.
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float lo, hi;
+                unpack2(xr[i][e], lo, hi);
+                ss = fmaf(lo, lo, ss); ss = fmaf(hi, hi, ss);
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if (lane == 0) sm->setpart[q][recs & 1][sw].x = ss;
+    }
+    SI_CPROF(0);                                          // the input row has arrived
+    fail = set_barrier_or<kSetThreads>(q, fail);          // one verdict for the set (and the warp sums are in place)
+    if (fail) return true;
+    if (P.prenorm) {
+        float ss = 0.f;
+#pragma unroll
+        for (int w = 0; w < kSetWarps; ++w) ss += sm->setpart[q][recs & 1][w].x;
+        recs ^= 1u;
+        const float scale = rsqrtf(ss / (float)d + P.norm_eps);
+        const bool emit = P.xn_out != nullptr && b == 0 && q == 0;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            uint32_t w4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float lo, hi;
+                unpack2(xr[i][e], lo, hi);
+                w4[e] = (uint32_t)si_cvt<DT>::from_float(lo * scale) | ((uint32_t)si_cvt<DT>::from_float(hi * scale) << 16);
+                xr[i][e] = pair_of<DT>(w4[e]);        // the dot products see the rounded values
+            }
+            const int c = t + kSetThreads * i;
+            if (emit && (kFull || c < chunks))
+                reinterpret_cast<uint4 *>(P.xn_out + (size_t)step * d)[c] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+    }
+    // ---- the set's records (the loop of the unchained kernel)
+    const bool noarith = (P.stream_only & 1) != 0;
+    for (int i = 0; i < cnt; ++i) {
+        fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
+        const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0 and no accumulate
+        const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * rec_bytes);
+        uint4 ga[NCH], up[NCH], dn[NCH];
+#pragma unroll
+        for (int k2 = 0; k2 < NCH; ++k2) {
+            const int c = t + kSetThreads * k2;
+            if (kFull) {
+                ga[k2] = rr[c]; up[k2] = rr[chunks + c]; dn[k2] = rr[2 * chunks + c];
+            } else {
+                const bool in = c < chunks;
+                ga[k2] = in ? rr[c] : make_uint4(0, 0, 0, 0);
+                up[k2] = in ? rr[chunks + c] : make_uint4(0, 0, 0, 0);
+                dn[k2] = in ? rr[2 * chunks + c] : make_uint4(0, 0, 0, 0);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sempty[st]);
+        if (++st == S) { st = 0; ph ^= 1; }
+        float g, u;
+        {
+            unsigned long long g2 = 0ull, u2 = 0ull;
+#pragma unroll
+            for (int k2 = 0; k2 < NCH; ++k2) { g2 = dot8p<DT>(ga[k2], xr[k2], g2); u2 = dot8p<DT>(up[k2], xr[k2], u2); }
+            float lo, hi;
+            unpack2(g2, lo, hi); g = lo + hi;
+            unpack2(u2, lo, hi); u = lo + hi;
+        }
+        {
+            const bool hi16 = (lane & 16) != 0;
+            float keep = (hi16 ? u : g) + __shfl_xor_sync(0xFFFFFFFFu, hi16 ? g : u, 16);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 8);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 4);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 2);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 1);
+            g = keep;
+        }
+        const uint32_t buf = recs & 1;
+        if ((lane & 15) == 0) reinterpret_cast<float *>(&sm->setpart[q][buf][sw])[lane >> 4] = g;
+        fail = set_barrier_or<kSetThreads>(q, fail);       // also orders the partials for the whole set
+        recs ^= 1u;
+        if (fail) return true;
+        float gs = 0.f, us = 0.f;
+        {
+            const float4 *pp = reinterpret_cast<const float4 *>(sm->setpart[q][buf]);
+#pragma unroll
+            for (int w = 0; w < kSetWarps / 2; ++w) {
+                const float4 v4 = pp[w];
+                gs += v4.x; us += v4.y; gs += v4.z; us += v4.w;
+            }
+        }
+        if (okr) {
+            const float h = si_silu_mul(gs, us);
+            const unsigned long long hh = pack2(h, h);
+#pragma unroll
+            for (int k2 = 0; k2 < NCH; ++k2) {
+                unsigned long long f[4];
+                unpack8p<DT>(dn[k2], f);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[k2][e] = fma2(hh, f[e], acc[k2][e]);
+            }
+        }
+    }
+    ring = (unsigned)st | (ph << 8) | ((recs & 1u) << 9);
+    SI_CPROF(1);                                          // normalisation + the set's records
+    // ---- the CTA's partial row
+    if (q == 1) {
+#pragma unroll
+        for (int k2 = 0; k2 < NCH; ++k2) {
+            const int c = t + kSetThreads * k2;
+            if (kFull || c < chunks) {
+                ulonglong2 *o = reinterpret_cast<ulonglong2 *>(comb + (size_t)c * 8);   // pairs are consecutive columns
+                o[0] = make_ulonglong2(acc[k2][0], acc[k2][1]);
+                o[1] = make_ulonglong2(acc[k2][2], acc[k2][3]);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm->accfull[0][kChainCmb]);
+        SI_CPROF(2);                                      // accumulators parked
+        return false;
+    }
+    fail |= !mbar_wait_bounded(&sm->accfull[0][kChainCmb], (uint32_t)(step & 1), cta_abort, wait_limit);
+    fail = set_barrier_or<kSetThreads>(q, fail);       // all of the row or none of it
+    if (fail) return true;
+    SI_CPROF(2);                                          // waited for the second set
+    // the sums of the two sets meet in shared memory, in column order ...
+#pragma unroll
+    for (int k2 = 0; k2 < NCH; ++k2) {
+        const int c = t + kSetThreads * k2;
+        if (kFull || c < chunks) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) unpack2(acc[k2][e], v[2 * e], v[2 * e + 1]);
+            float4 *pc = reinterpret_cast<float4 *>(comb + (size_t)c * 8);
+            const float4 o0 = pc[0], o1 = pc[1];
+            pc[0] = make_float4(v[0] + o0.x, v[1] + o0.y, v[2] + o0.z, v[3] + o0.w);
+            pc[1] = make_float4(v[4] + o1.x, v[5] + o1.y, v[6] + o1.z, v[7] + o1.w);
+        }
+    }
+    set_barrier_or<kSetThreads>(q, false);
+    // ... and leave as {sum, tag} words, each warp instruction writing 512 consecutive bytes (a thread storing
+    // the eight words of its own chunk would touch 32 lines with every instruction)
+    uint4 *row = reinterpret_cast<uint4 *>(P.ll_partial + (size_t)b * d);
+    for (int u = t; u < d / 2; u += kSetThreads) {
+        const float2 f = reinterpret_cast<const float2 *>(comb)[u];
+        st_relaxed_gpu_v4(row + u, make_uint4(__float_as_uint(f.x), tag, __float_as_uint(f.y), tag));
+    }
+    SI_CPROF(3);                                          // row words issued
+    // every thread of the set has issued its stores: count this CTA's row as written (a hint)
+    set_barrier_or<kSetThreads>(q, false);
+    if (t == 0) red_add_relaxed_gpu(P.counters + (size_t)step * kCounterStride, 1u);
+    SI_CPROF(7);                                          // (set 0, shares the last slot) barrier + count
+    return false;
+}
+
+// Second half: all 512 consumer threads gather this CTA's columns of every CTA's row (thread = two
+// columns x a class of rows, all of its rows in one round of loads, summed in row order), the class sums
+// meet in shared memory and are added in a fixed order -- deterministic, whatever arrives first -- and the
+// column owners add the residual, round once, write y and the {values, tag} words of the next input row.
+template <int DT, int LLR>
+__device__ __noinline__ bool chain_step_exchange(const Params &P, uint8_t *smem, int step) {
+    const int d = P.d_model, G = gridDim.x, b = blockIdx.x;
+    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)P.nstage * d * 6 + (size_t)2 * d * 4);
+    float *csum = reinterpret_cast<float *>(smem + P.csum_off);          // [columns][classes] class sums
+    volatile int *cta_abort = &sm->cta_abort;
+    const long long wait_limit = P.wait_cycles;
+    const int ct = threadIdx.x - 32, lane = ct & 31;
+    const uint32_t tag = (uint32_t)step + 1u, par = (uint32_t)(step & 1);
+    const int gpc = (d / 4 + G - 1) / G, pieces = gpc * 2, classes = kConsumers / pieces;
+    bool fail = false;
+    const bool cprof = P.prof != nullptr && (ct & 255) == 0;
+    const int q_ = ct >> 8;
+    long long pt_ = cprof ? clock64() : 0;
+    {
+        const int piece = ct % pieces, rc = ct / pieces;
+        const int col0 = b * gpc * 4 + piece * 2;
+        const int n_mine = (rc < classes && col0 < d) ? (G - rc + classes - 1) / classes : 0;     // rows rc, rc + classes, ...
+        const uint4 *src = reinterpret_cast<const uint4 *>(P.ll_partial + (size_t)rc * d + col0);
+        const size_t stride = (size_t)classes * d / 2;             // uint4 units between this thread's rows
+        fail |= !hint_wait_cta(P.counters + (size_t)step * kCounterStride, (unsigned)G, P.ctrl + 1, cta_abort, wait_limit,
+                               ct == 0, &sm->accfull[1][kChainRows], par);
+        SI_CPROF(4);                                      // every CTA's row counted as written
+        float sx = 0.f, sy = 0.f;
+        const long long t0 = clock64();
+        uint32_t spins = 0;
+        while (!fail) {
+            // the sum counts only if every word carried this step's tag (after the hint that is the rule)
+            float ax = 0.f, ay = 0.f;
+            bool good = true;
+            uint4 w[LLR];
+#pragma unroll
+            for (int i = 0; i < LLR; ++i)
+                if (i < n_mine) w[i] = ld_relaxed_gpu_v4(src + stride * i);
+#pragma unroll
+            for (int i = 0; i < LLR; ++i)
+                if (i < n_mine) {
+                    good &= w[i].y == tag && w[i].w == tag;
+                    ax += __uint_as_float(w[i].x); ay += __uint_as_float(w[i].z);
+                }
+            if (good) { sx = ax; sy = ay; break; }
+            if ((++spins & 63u) == 0 && (*cta_abort || ld_relaxed_gpu(P.ctrl + 1) || clock64() - t0 > wait_limit)) fail = true;
+        }
+        if (rc < classes) {
+            csum[(piece * 2) * classes + rc] = sx;
+            csum[(piece * 2 + 1) * classes + rc] = sy;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm->accfull[0][kChainXch]);
+        SI_CPROF(5);                                      // rows gathered
+    }
+    fail |= !mbar_wait_bounded(&sm->accfull[0][kChainXch], par, cta_abort, wait_limit);
+    SI_CPROF(6);                                          // all class sums in place
+    const int col = ct >> 2, p4 = ct & 3, per = (classes + 3) / 4;
+    const int gcol = b * gpc * 4 + col;
+    const bool owner = col < pieces * 2 && gcol < d;
+    float v = 0.f;
+    if (owner && !fail)
+        for (int c2 = p4 * per; c2 < (p4 + 1) * per && c2 < classes; ++c2) v += csum[col * classes + c2];
+    v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+    v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+    uint32_t o16 = 0;
+    if (owner && p4 == 0) {
+        uint32_t *prev = reinterpret_cast<uint32_t *>(csum + 1024) + col;      // this thread's output of the step before
+        if (P.residual) {
+            const uint32_t xin = step % P.chain_len != 0 ? *prev : (uint32_t)P.x[(size_t)(step / P.chain_len) * d + gcol];
+            v += si_cvt<DT>::lo(xin);
+        }
+        o16 = si_cvt<DT>::from_float(v);
+        *prev = o16;
+        if (!fail) reinterpret_cast<uint16_t *>(P.y)[(size_t)step * d + gcol] = (uint16_t)o16;
+    }
+    const uint32_t odd = __shfl_down_sync(0xFFFFFFFFu, o16, 4);      // the neighbouring column's value
+    const bool feeds = step + 1 < P.n_steps && (step + 1) % P.chain_len != 0;       // the next step reads this row
+    if (feeds && owner && p4 == 0 && (col & 1) == 0 && !fail)
+        st_relaxed_gpu_v2(P.ll_x + (size_t)((step + 1) & 1) * (d / 2) + gcol / 2, make_uint2(o16 | (odd << 16), tag));
+    // the warps that hold column owners meet (every step, so the barrier's phase follows the step), then one
+    // thread counts this CTA's columns as written (a hint)
+    if (ct < ((pieces * 8 + 31) & ~31)) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm->accfull[0][kChainOwn]);
+        if (ct == 0) {
+            if (!mbar_wait_bounded(&sm->accfull[0][kChainOwn], par, cta_abort, wait_limit)) fail = true;
+            else if (feeds) red_add_relaxed_gpu(P.counters + (size_t)step * kCounterStride + 32, 1u);
+        }
+    }
+    SI_CPROF(7);                                          // column sums, y, next input row
+    return fail;
+}
+
+#undef SI_CPROF
+
+template <int DT, int NCH, bool kFull, int LLR>
+__device__ __forceinline__ void chained_consumers(const Params &P, uint8_t *smem, Smem *sm) {
+    unsigned ring = 0;
+    bool fail = false;
+    for (int step = 0; step < P.n_steps && !fail; ++step) {
+        fail = chain_step_records<DT, NCH, kFull>(P, smem, step, ring);
+        if (!fail) fail = chain_step_exchange<DT, LLR>(P, smem, step);
+    }
+    if (fail && (threadIdx.x & 31) == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
+}
+
 // kProf: phase profile compiled in; kFull: every thread of a set owns NCH chunks of every row (chunks == NCH * 256);
 // GRP: float4 column groups a reducer warp covers at once (its 32 lanes = GRP groups x 32/GRP row classes);
 // SETW: warps per consumer set -- 8: two sets of 256 threads; 16: one set of 512 threads (rows too long for
 // two rings and two hand-over buffers: thread t then owns chunks t, t + 512)
-template <int DT, int NCH, bool kFull, bool kProf, int GRP, int SETW = 8>
-__global__ void __launch_bounds__(kThreads, 1)   // 19 warps: at most 96 registers per thread
+// CH: chained mode (every step reads the output of the step before it; the consumers themselves run the
+// exchanges between the SMs and the reducer warps have nothing to do)
+// LLR (chained): partial rows one consumer thread gathers per step (all in flight at once)
+template <int DT, int NCH, bool kFull, bool kProf, int GRP, int SETW = 8, bool CH = false, int LLR = 5>
+__global__ void __launch_bounds__(CH ? kThreadsChained : kThreads, 1)   // 20 warps: at most 96 registers per thread (chained: 17 warps, 120)
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int kSets = 16 / SETW, kSetWarps = SETW, kSetThreads = SETW * 32;   // shadow the two-set defaults
@@ -317,12 +714,20 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     const int Gv = G * kSets;                  // consumer sets act as virtual CTAs 2b, 2b+1 of 2G
     const int d = P.d_model, chunks = P.chunks;
     const long long wait_limit = P.wait_cycles;
-    const bool chained = P.chain_len > 0;      // (one step group then: the launch code sees to it)
+    constexpr bool chained = CH;               // (one step group then: the launch code sees to it)
+    constexpr int xi = CH ? 0 : 1;             // ring items per step that carry the input row (chained: none, the consumers fetch it)
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
         for (int q = 0; q < kSets; ++q)
             for (int w = 0; w < kReducerWarps; ++w) { mbar_init(&sm->accfull[q][w], kSetWarps); mbar_init(&sm->accempty[q][w], 1); }
+        if (CH) {     // chained mode has no hand-over to reducers: three of those barriers serve its consumers
+            const int gpc0 = (P.d_model / 4 + (int)gridDim.x - 1) / (int)gridDim.x;
+            mbar_init(&sm->accfull[0][kChainCmb], kSetWarps);               // second set's accumulators parked
+            mbar_init(&sm->accfull[0][kChainXch], kConsumerWarps);          // every warp's class sums written
+            mbar_init(&sm->accfull[0][kChainOwn], (gpc0 * 16 + 31) / 32);   // every column owner's stores issued
+            mbar_init(&sm->accfull[1][kChainRows], 1); mbar_init(&sm->accfull[1][kChainInput], 1);   // news from the polling thread
+        }
         sm->cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -361,8 +766,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 StepGeom g;
                 in = step < nvw;
                 if (in) g = step_geom(P, step * NG + grp, Gv, vb);
-                while (in && t > g.cnt) {
-                    t -= g.cnt + 1; ++step;
+                while (in && t >= g.cnt + xi) {
+                    t -= g.cnt + xi; ++step;
                     in = step < nvw;
                     if (in) g = step_geom(P, step * NG + grp, Gv, vb);
                 }
@@ -370,17 +775,12 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 if (in) {
                     const int rs = step * NG + grp;               // step of the launch
                     const int layer = P.step_layers ? __ldg(P.step_layers + rs) : (P.n_few ? (int)P.few_layers[rs] : rs % P.n_layers);
-                    if (t == 0) {
-                        // chained: the first step of a chain reads the caller's row, every other step the
-                        // output row of the step before it, which the issue lane may only fetch once every
-                        // CTA has written its columns of it (bit 31 of the byte count marks such an item)
-                        const bool from_y = chained && rs % P.chain_len != 0;
-                        pf_src = from_y ? (unsigned long long)(reinterpret_cast<const uint16_t *>(P.y) + (size_t)(rs - 1) * d)
-                                        : (unsigned long long)(P.x + (size_t)(chained ? rs / P.chain_len : rs) * d);
-                        pf_bytes = (uint32_t)d * 2 | (from_y ? 0x80000000u : 0u); pf_meta = g.cnt;
+                    if (t < xi) {
+                        pf_src = (unsigned long long)(P.x + (size_t)rs * d);
+                        pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
                     } else {
                         const int lbase = P.per_layer_lists ? layer * P.k_fixed : g.base;
-                        const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - 1) * Gv);
+                        const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - xi) * Gv);
                         const bool valid = slot >= 0 && slot < P.n_loaded[layer];
                         pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
                         pf_bytes = valid ? (uint32_t)rec_bytes : 0u; pf_meta = valid ? 1 : 0;
@@ -432,20 +832,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             bool progressed = false;
             if (have && n < i_ready && !(P.withhold && blockIdx.x == 0 && iq == 0 && n == 1)) {
                 const int st = iq * S + is;
-                bool go = mbar_test_wait(&empty[st], iph ^ 1);
-                uint4 dsc = make_uint4(0, 0, 0, 0);
-                if (go) {
-                    dsc = sm->desc[iq][n % kDescRing];
-                    if (dsc.z & 0x80000000u) {
-                        // input row = output row of the step before: has every CTA written its columns?
-                        const unsigned long long src = ((unsigned long long)dsc.y << 32) | dsc.x;
-                        const int prev = (int)((src - (unsigned long long)P.y) / ((unsigned long long)d * 2));
-                        go = ld_acquire_gpu(P.counters + (size_t)prev * kCounterStride + 32) >= (unsigned)gridDim.x;
-                        if (go) asm volatile("fence.proxy.async;" ::: "memory");   // the bulk copy reads what generic stores wrote
-                        dsc.z &= 0x7FFFFFFFu;
-                    }
-                }
-                if (go) {
+                if (mbar_test_wait(&empty[st], iph ^ 1)) {
+                    const uint4 dsc = sm->desc[iq][n % kDescRing];
                     meta[st] = (int)dsc.w;
                     if (dsc.z != 0) {
                         mbar_arrive_expect_tx(&full[st], dsc.z);
@@ -458,13 +846,21 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     ++issued;
                     n += S; iph ^= 1;
                     progressed = true;
+                    if (CH && n < i_ready && !(P.stream_only & 8)) {
+                        // chained: between two steps the ring stands still while the SMs exchange their sums;
+                        // the record that will follow this one through the stage is asked into L2 meanwhile
+                        const uint4 nx = sm->desc[iq][n % kDescRing];
+                        if (nx.z != 0)
+                            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;"
+                                         ::"l"(((unsigned long long)nx.y << 32) | nx.x), "r"(nx.z) : "memory");
+                    }
                 }
             }
             if (__any_sync(FULL, progressed)) {
                 t_last = clock64();
             } else {
                 if (*cta_abort || clock64() - t_last > wait_limit) { ok = false; break; }
-                if (!chained) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
+                if (!chained || (P.stream_only & 16)) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -482,14 +878,18 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     // Warp w runs on scheduler partition w mod 4.  The service warps (producer 0, reducers 4, 8, 12)
     // share partition 0 with one consumer warp, so that their rarely executed code does not compete
     // with four consumer warps for the partition's instruction cache and issue slots.
-    const bool is_reducer = (warp & 3) == 0 && warp >= 4 && warp <= 4 * kReducerWarps;
+    const bool is_reducer = !CH && (warp & 3) == 0 && warp >= 4 && warp <= 4 * kReducerWarps;
+    if constexpr (CH) {
+        chained_consumers<DT, NCH, kFull, LLR>(P, smem, sm);
+        return;
+    }
     if (!is_reducer) {
         // ------------------------------------------------------------------ consumers
         // Two independent sets of 8 warps; set q consumes ring q.  A landed record is copied
         // into registers (3*NCH 16-byte chunks per thread) and its stage handed back at once;
         // the arithmetic then runs out of registers, so the ring is refilled while the set
         // computes.  Thread t of a set owns chunks t, t+256 of every row.
-        const int cw = warp < 16 ? warp - (warp / 4 + 1) : warp - 4;   // consumer warp index 0..15
+        const int cw = CH ? warp - 1 : (warp < 16 ? warp - (warp / 4 + 1) : warp - 4);   // consumer warp index 0..15
         const int ct = cw * 32 + lane;           // 0..511
         const int q = ct / kSetThreads;          // consumer set
         const int t = ct & (kSetThreads - 1);    // thread within the set
@@ -527,47 +927,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     if (lane == 0) mbar_arrive(&sempty[st]);
                     if (++st == S) { st = 0; ph ^= 1; }
                 }
-                if (P.prenorm) {
-                    // sum of squares of the row: thread slice, warp butterfly, then (after the barrier
-                    // below) the set's warps in warp order -- the same order in every set of every CTA
-                    float ss = 0.f;
-#pragma unroll
-                    for (int i = 0; i < NCH; ++i)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float lo, hi;
-                            unpack2(xr[i][e], lo, hi);
-                            ss = fmaf(lo, lo, ss); ss = fmaf(hi, hi, ss);
-                        }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-                    if (lane == 0) sm->normpart[q][step & 1][sw] = ss;
-                }
                 // the record count steers the set's barriers: agree on it (and on failure) first
                 fail = set_barrier_or<kSetThreads>(q, fail);
                 if (fail) break;
-                if (P.prenorm) {
-                    float ss = 0.f;
-#pragma unroll
-                    for (int w = 0; w < kSetWarps; ++w) ss += sm->normpart[q][step & 1][w];
-                    const float scale = rsqrtf(ss / (float)d + P.norm_eps);
-                    const int rs = step * NG + grp;
-                    const bool emit = P.xn_out != nullptr && b == 0 && q == 0;
-#pragma unroll
-                    for (int i = 0; i < NCH; ++i) {
-                        uint32_t w4[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float lo, hi;
-                            unpack2(xr[i][e], lo, hi);
-                            w4[e] = (uint32_t)si_cvt<DT>::from_float(lo * scale) | ((uint32_t)si_cvt<DT>::from_float(hi * scale) << 16);
-                            xr[i][e] = pair_of<DT>(w4[e]);        // the dot products see the rounded values
-                        }
-                        const int c = t + kSetThreads * i;
-                        if (emit && (kFull || c < chunks))
-                            reinterpret_cast<uint4 *>(P.xn_out + (size_t)rs * d)[c] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-                    }
-                }
                 SI_PROF(0);                               // wait for x
                 for (int i = 0; i < cnt; ++i) {
                     fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
@@ -703,8 +1065,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         float *const gpartial = P.partial + (size_t)grp * kPartialDepth * G * d;   // this group's ring of partial rows
         auto ctr_of = [&](int v) { return P.counters + ((size_t)v * NG + grp) * kCounterStride; };   // counters of the group's step v
         constexpr int kRowBatch = 13;                          // partial rows in flight per lane
-        const int lag = chained ? 0 : kLag;                    // chained: a step's sum is needed at once
-        for (int step = r; step < nv + lag; step += kReducerWarps) {
+        for (int step = r; step < nv + kLag; step += kReducerWarps) {
             int ok = 1;
             if (step < nv) {
                 // ---- phase A: take each set's accumulators as soon as that set hands them over.  The
@@ -729,7 +1090,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                             else if (kSets > 1 && !(taken & 2) && mbar_test_wait(&sm->accfull[kSets - 1][r], par)) q = 1;
                             else {
                                 if (*cta_abort || clock64() - t0 > wait_limit) break;
-                                if (!chained) __nanosleep(200);
+                                __nanosleep(200);
                             }
                         }
                         ok = q >= 0;
@@ -764,18 +1125,13 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     SI_RPROF(2);                          // copy the accumulators out
                 }
             }
-            const int sr = step - lag;
-            if (chained && ok && !nosync) {
-                // the step's own sum follows at once: publish this CTA's partial row first
-                __syncwarp();
-                if (lane == 0) { __threadfence(); atomicAdd(ctr_of(step), 1u); }
-            }
+            const int sr = step - kLag;
             if (ok && sr >= 0 && !nosync) {
                 // ---- phase B: lane (group bg, row class brc) sums rows brc, brc + 4, ... of its column
                 // group in ascending order, kRowBatch loads in flight; two butterfly steps combine the
                 // four row classes (fixed order: deterministic split-K)
                 if (lane == 0)
-                    ok = counter_wait_bounded(ctr_of(sr), (unsigned)G, P.ctrl + 1, cta_abort, wait_limit, chained ? 0u : 64u);
+                    ok = counter_wait_bounded(ctr_of(sr), (unsigned)G, P.ctrl + 1, cta_abort, wait_limit);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 SI_RPROF(4);                              // every SM has published the step
                 if (ok) {
@@ -801,17 +1157,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, o); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, o);
                     }
                     if (brc == 0 && bg < g_valid) {
-                        const int rs = sr * NG + grp;                      // step of the launch
-                        const size_t cin = (size_t)(b * gpc + bg) * 4;     // first of the lane's four columns
-                        const size_t col = (size_t)rs * d + cin;
+                        const size_t col = ((size_t)sr * NG + grp) * d + (size_t)(b * gpc + bg) * 4;
                         if (P.residual) {
-                            // the step's input row: the caller's, or in a chain the output row of the step before
-                            // (complete and visible: this step's records were only multiplied with it once every
-                            // CTA had published its columns; read at L2, where those stores went)
-                            const uint16_t *xin = !chained ? P.x + col
-                                                  : (rs % P.chain_len != 0 ? reinterpret_cast<const uint16_t *>(P.y) + (col - d)
-                                                                           : P.x + (size_t)(rs / P.chain_len) * d + cin);
-                            uint2 xw = chained ? __ldcg(reinterpret_cast<const uint2 *>(xin)) : __ldg(reinterpret_cast<const uint2 *>(xin));
+                            uint2 xw = __ldg(reinterpret_cast<const uint2 *>(P.x + col));
                             v.x += si_cvt<DT>::lo(xw.x); v.y += si_cvt<DT>::hi(xw.x);
                             v.z += si_cvt<DT>::lo(xw.y); v.w += si_cvt<DT>::hi(xw.y);
                         }
@@ -836,9 +1184,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
             __syncwarp();
             if (lane == 0 && !nosync) {
                 __threadfence();
-                if (step < nv && !chained) atomicAdd(ctr_of(step), 1u);
-                // chained: the producers of every CTA wait for this count before they fetch the next step's input
-                if (sr >= 0 && (chained || sr + kPartialDepth < nv)) atomicAdd(ctr_of(sr) + 32, 1u);
+                if (step < nv) atomicAdd(ctr_of(step), 1u);
+                if (sr >= 0 && sr + kPartialDepth < nv) atomicAdd(ctr_of(sr) + 32, 1u);
             }
             SI_RPROF(3);                                  // publish (fence + atomics)
         }
@@ -872,6 +1219,7 @@ inline bool wide_rows(int d_model) {
 
 }  // namespace si_persist
 
+#ifndef SI_PERSIST_KERNEL_ONLY      // (a build of single kernel instantiations, to read their register use, leaves the host side out)
 inline bool si_persistent_supported(const si_store *s) {
     // thread t of a 256-thread set owns chunks t, t + 256 (, t + 512) of a row (d_model <= 6144); the
     // rings need at least two stages per consumer set beside the two hand-over buffers; a reducer warp's
@@ -889,15 +1237,16 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8>
-inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream) {
-    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP, SETW>;
-    size_t smem = si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW);
+template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8, bool CH = false, int LLR = 5>
+inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream, size_t extra_smem = 0) {
+    auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP, SETW, CH, LLR>;
+    size_t smem = si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW) + extra_smem;
     // the limit is raised to the most any instance needs (setting it is cheap, a host-side call, and
     // keeps no state here that threads or devices could disagree about)
     SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&P};
-    SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G), dim3(si_persist::kThreads), args, smem, stream));
+    SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G), dim3(CH ? si_persist::kThreadsChained : si_persist::kThreads),
+                                            args, smem, stream));
     return SI_OK;
 }
 
@@ -932,7 +1281,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
     P.prof = ex->profile;
-    P.stream_only = ex->skip_mask & 7;
+    P.stream_only = ex->skip_mask & 31;
     if (ex->ring_stages > 0 && !wide && 2 * ex->ring_stages <= P.nstage) P.nstage = 2 * ex->ring_stages;   // diagnostics: shallower rings
     P.wait_cycles = ex->wait_cycles > 0 ? ex->wait_cycles : si_persist::kWaitCycles;
     P.withhold = ex->withhold;
@@ -956,6 +1305,37 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.n_groups = ng;
     const int gpc = (s->d_model / 4 + G / ng - 1) / (G / ng);       // column groups per CTA -> lanes of a reducer warp
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
+    P.ll_partial = nullptr; P.ll_x = nullptr; P.csum_off = 0;
+    if (ex->chain_len > 0) {
+        // chained: two consumer sets only; the tagged exchange words live in the partial-row area and start at zero
+        if (wide) return SI_ERR_UNSUPPORTED;
+        const int pieces = gpc * 2, classes = si_persist::kConsumers / pieces;
+        const int rpt = classes < 1 ? si_persist::kLLRows + 1 : (G + classes - 1) / classes;   // partial rows a consumer thread gathers
+        if (rpt > si_persist::kLLRows) return SI_ERR_UNSUPPORTED;
+        const size_t ll_bytes = (size_t)G * s->d_model * 8 + (size_t)s->d_model * 8;
+        if (ll_bytes > ws.partial_bytes) return SI_ERR_NOMEM;
+        P.ll_partial = (uint2 *)(wsb + ws.partial_off);
+        P.ll_x = P.ll_partial + (size_t)G * s->d_model;
+        SI_CUDA_TRY(cudaMemsetAsync(P.ll_partial, 0, ll_bytes, stream));
+        // class sums (at most 4 KB) and the column owners' last outputs (512 B): in the second hand-over buffer where that
+        // is large enough, else behind everything
+        const size_t base = (size_t)P.nstage * s->d_model * 6;
+        size_t extra = 0;
+        if ((size_t)s->d_model * 4 >= 4096 + 512) P.csum_off = (unsigned)(base + (size_t)s->d_model * 4);
+        else { P.csum_off = (unsigned)si_align_up(si_persist::smem_bytes(s->d_model, P.nstage), 16); extra = 4096 + 512 + 16; }
+        const int set_threads_c = si_persist::kSetThreads;
+        const int nch_c = (P.chunks + set_threads_c - 1) / set_threads_c;
+        const bool full_c = P.chunks == nch_c * set_threads_c;
+#define SI_PLC(DT, N, F) (rpt <= 2 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, 2>(P, G, stream, extra)   \
+                          : rpt <= 5 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, 5>(P, G, stream, extra) \
+                                     : si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, si_persist::kLLRows>(P, G, stream, extra))
+#define SI_PLC2(DT) (nch_c <= 1 ? (full_c ? SI_PLC(DT, 1, true) : SI_PLC(DT, 1, false))   \
+                     : nch_c <= 2 ? (full_c ? SI_PLC(DT, 2, true) : SI_PLC(DT, 2, false)) \
+                                  : (full_c ? SI_PLC(DT, 3, true) : SI_PLC(DT, 3, false)))
+        return s->dtype == SI_BF16 ? SI_PLC2(SI_BF16) : SI_PLC2(SI_F16);
+#undef SI_PLC2
+#undef SI_PLC
+    }
     // NCH: 16-byte chunks per thread and row (256 threads per consumer set)
     const int set_threads = wide ? 2 * si_persist::kSetThreads : si_persist::kSetThreads;
     const int nch = (P.chunks + set_threads - 1) / set_threads;
@@ -983,3 +1363,4 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
 #undef SI_PL_W
 #undef SI_PL
 }
+#endif  // SI_PERSIST_KERNEL_ONLY
