@@ -8,9 +8,16 @@ tokens of the workload through all FFN layers, each layer running the selective 
 token's active list (one persistent launch through the C ABI).  The store is built once by
 the loader before timing.  Metric: selective-FFN decode tokens/s at batch 1.
 
-Prints ONE JSON line (rank 0).  With N > 1 (torchrun) each rank is an independent replica
-decoding its own tokens against its own copy of the store: no data-path collective, weak
-scaling, time = max over ranks.
+Prints ONE JSON line (rank 0).  The headline is configuration 2 with the (token, layer) steps
+independent of one another (every step's input given up front) and worked through in order.
+Beside it, in the same line: `chained` -- the same launch size with every layer reading the
+output of the layer before it, as inside a decoder; `steps_any_order`; and `configs` -- the other
+four configurations (c1 latency, c3 batch sizes, c4 prefill, the sixteen c5 cells), each measured
+on a stated reduced number of layers whose weights still exceed L2.
+
+With N > 1 each rank is an independent replica decoding its own tokens against its own copy of
+the store: no data-path collective, weak scaling, time = max over ranks.  Started without a
+launcher, `--gpus N` starts its own N ranks.
 """
 from __future__ import annotations
 
@@ -33,9 +40,9 @@ from paper_2607_18081_b200 import replicas, workloads as wl  # noqa: E402
 METRIC = "selective_ffn_decode_tokens_per_s_batch1"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of si_decode_persistent_kernel per (token, layer) step
-# of the config-2 shape, from the capture summarised in
-# profiles/decode_persistent_c2_8layers_32tokens_full.md: (9.6461e9 + 0.2290e9) / 256 steps
+# dram__bytes_read.sum + dram__bytes_write.sum of si_decode_persistent_kernel per (token, layer) step of
+# the config-2 shape: an ncu capture of an 8-layer x 32-token launch (256 steps) read 9.6454e9 and wrote
+# 0.2272e9 bytes; traffic grows in proportion to the steps (every step reads its own records once)
 NCU_DRAM_BYTES_PER_C2_STEP = (9.6454e9 + 0.2272e9) / 256
 FALLBACK_HBM_GBS = 6650.0
 
@@ -161,6 +168,222 @@ def run_reference(args):
         "e2e": {"value": tok_s, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
+
+
+# ----------------------------------------------------------------------------- measuring helpers
+
+def device_ms(torch, fn, reps, warm=3):
+    """Mean CUDA-event time of fn() over reps calls on the current stream, after warm-up."""
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def graphed(torch, fn):
+    """fn() captured once into a CUDA graph (host launch overhead out of the picture); returns a
+    callable that replays it, or fn itself if the capture is not possible."""
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g.replay, True
+    except Exception:                                   # pragma: no cover
+        torch.cuda.synchronize()
+        return fn, False
+
+
+def load_store(api, torch, cfg, n_layers, device):
+    tdt = api.torch_dtype(cfg.dtype)
+    store = api.NeuronStore(n_layers, cfg.d_model, cfg.d_ff, [cfg.n_loaded] * n_layers, cfg.dtype, device=device)
+    for l in range(n_layers):
+        wg, wu, wd = wl.layer_weights(cfg, l)
+        ids, _ = wl.loaded_ids(cfg, l)
+        to_dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(tdt)
+        store.load(l, to_dev(wg), to_dev(wu), to_dev(wd), ids, cfg.n_base)
+        del wg, wu, wd
+    torch.cuda.synchronize()
+    return store
+
+
+CHAIN_EPS = 1e-5
+
+
+def measure_chained(api, torch, store, cfg, heads_dev, idx_dev, ws, status, peaks, reps):
+    """The same launch size as the headline with every layer reading the output of the layer before it
+    (one chain per token, pre-norm + residual): microseconds per (token, layer) step and the rate the
+    selected bytes stream at."""
+    L, d, k, tokens = cfg.n_layers, cfg.d_model, cfg.k_active, cfg.tokens
+    n_steps = tokens * L
+    y = torch.empty(n_steps, d, dtype=api.torch_dtype(cfg.dtype), device="cuda")
+    flags = api.SI_FLAG_PRENORM | api.SI_FLAG_RESIDUAL
+
+    def launch():
+        api.si_decode_chain_forward(store.handle, n_steps, None, L, heads_dev, idx_dev, None, k, y, None, CHAIN_EPS,
+                                    flags, ws, status)
+
+    ms = device_ms(torch, launch, reps)
+    us_step = ms * 1e3 / n_steps
+    gbs = k * cfg.record_bytes / us_step / 1e3
+    return {"value": tokens / (ms * 1e-3), "unit": UNIT, "us_per_step": us_step, "achieved_gbs": gbs,
+            "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "launch_ms": ms,
+            "note": "si_decode_chain_forward: one chain per token through all layers, each layer's input = the rounded "
+                    "output of the layer before it (pre-norm + residual); no arithmetic of a step starts before the "
+                    "step before it is complete on every SM, only the weight stream runs ahead"}, y
+
+
+def extra_configs(api, torch, args, device, peaks, peak_kind):
+    """The four configurations beside the headline, each on a reduced number of layers whose weights
+    still exceed L2 (stated per entry), timed with CUDA events; per-layer calls replayed from CUDA graphs."""
+    out = {}
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hbm = peaks["hbm_gbs"]
+
+    # ---- c1: one small fp16 layer, 16 decode tokens; the whole store (2.1 MB) is L2-resident
+    try:
+        cfg = wl.CONFIGS["c1"]
+        store = load_store(api, torch, cfg, 1, device)
+        _, sor = wl.loaded_ids(cfg, 0)
+        tdt = api.torch_dtype(cfg.dtype)
+        x = torch.from_numpy(wl.x_tokens(cfg, 0, cfg.tokens).view(np.int16)).cuda().view(tdt)
+        idx = torch.from_numpy(wl.zipf_lists(cfg, 0, cfg.tokens, slot_of_rank=sor)).cuda()
+        y = torch.empty(cfg.tokens, cfg.d_model, dtype=tdt, device="cuda")
+        ws = store.workspace(1, cfg.k_active, cfg.tokens)
+        one, g1 = graphed(torch, lambda: api.si_ffn_forward(store.handle, 0, x[0], 1, idx[0], None, cfg.k_active, y[0], 0, ws, status))
+        allt, g2 = graphed(torch, lambda: api.si_decode_stack_forward(store.handle, cfg.tokens, [0] * cfg.tokens, x, idx, None,
+                                                                      cfg.k_active, y, 0, ws, status))
+        ms_one, ms_all = device_ms(torch, one, 200), device_ms(torch, allt, 100)
+        out["c1"] = {"workload": "c1: 1 layer d_model=512 d_ff=1376 f16, 688 loaded, 172 active, batch 1, 16 decode tokens",
+                     "us_per_token_single_call": ms_one * 1e3, "us_per_token_in_one_16_token_launch": ms_all * 1e3 / cfg.tokens,
+                     "tokens_per_s": cfg.tokens / (ms_all * 1e-3), "selected_bytes_per_token": cfg.k_active * cfg.record_bytes,
+                     "replayed_from_cuda_graph": bool(g1 and g2),
+                     "note": "the whole store (2.1 MB) is L2-resident: launch- and latency-bound, an HBM roofline does not apply"}
+        store.close(); del store, ws
+    except Exception as e:                              # pragma: no cover
+        out["c1"] = {"error": repr(e)}
+
+    # ---- c3 (batched decode over the union) and c4 (prefill, one shared list): per-layer calls, 4 layers
+    def multitoken(cfg, T, n_layers, groups, shared):
+        tdt = api.torch_dtype(cfg.dtype)
+        d, k = cfg.d_model, cfg.k_active
+        store = load_store(api, torch, cfg, n_layers, device)
+        x = torch.empty(groups, n_layers, T, d, dtype=torch.int16)
+        for l in range(n_layers):
+            x[:, l] = torch.from_numpy(wl.x_tokens(cfg, l, groups * T).view(np.int16)).view(groups, T, d)
+        x = x.cuda().view(tdt)
+        if shared:
+            idx, flags, usz = torch.arange(k, dtype=torch.int32, device="cuda"), api.SI_FLAG_SHARED_LIST, [k]
+        else:
+            blk = (T * k + 3) // 4 * 4                          # every (group, layer) block of lists starts 16-byte aligned
+            lists = np.zeros((groups, n_layers, blk), dtype=np.int32)
+            for l in range(n_layers):
+                lists[:, l, :T * k] = wl.zipf_lists(cfg, l, groups * T).reshape(groups, T * k)
+            usz = [len(np.unique(lists[g, l, :T * k])) for g in range(groups) for l in range(n_layers)]
+            idx, flags = torch.from_numpy(lists).cuda(), 0
+        y = torch.empty(groups, n_layers, T, d, dtype=tdt, device="cuda")
+        ws = store.workspace(max(T, 2), k, max(T, 1))
+
+        def run():
+            for g in range(groups):
+                for l in range(n_layers):
+                    api.si_ffn_forward(store.handle, l, x[g, l], T, idx if shared else idx[g, l, :T * k], None, k, y[g, l], flags, ws, status)
+
+        fn, was_graph = graphed(torch, run)
+        ms = device_ms(torch, fn, 10)
+        us_call = ms * 1e3 / (groups * n_layers)
+        store.close()
+        return us_call, float(np.mean(usz)), was_graph
+
+    try:
+        cfg3 = wl.CONFIGS["c3"]
+        cells = []
+        for B in wl.C3_BATCHES:
+            us_call, u, was_graph = multitoken(cfg3.with_(batch=B), B, 4, max(1, 8 // B) if B < 8 else 1, False)
+            tok_s = B / (us_call * 1e-6 * cfg3.n_layers)
+            ubytes = u * cfg3.record_bytes
+            cells.append({"batch": B, "tokens_per_s": tok_s, "us_per_layer_call": us_call, "mean_union": u,
+                          "union_overlap": 1.0 - u / (B * cfg3.k_active), "union_coverage_of_loaded": u / cfg3.n_loaded,
+                          "union_gbs": ubytes / us_call / 1e3, "frac": ubytes / us_call / 1e3 / hbm,
+                          "route": "decode kernel, token by token" if B <= 4 else "union + tensor-core contractions",
+                          "replayed_from_cuda_graph": was_graph})
+        out["c3"] = {"workload": "c3: 7B-shaped stack (d_model=4096, d_ff=11008, bf16, 7705 loaded), own 1541-slot Zipf list per "
+                                 "token, batch sizes 1..32; measured on 4 layers (757 MB of records), tokens/s scaled to 32 layers",
+                     "bound": "hbm", "peak": hbm, "peak_kind": f"of {peak_kind}", "cells": cells}
+    except Exception as e:                              # pragma: no cover
+        out["c3"] = {"error": repr(e)}
+    try:
+        cfg4 = wl.CONFIGS["c4"]
+        us_call, u, was_graph = multitoken(cfg4, cfg4.tokens, 4, 1, True)
+        tflops = 6.0 * cfg4.d_model * cfg4.k_active * cfg4.tokens / us_call / 1e6
+        out["c4"] = {"workload": "c4: 7B-shaped stack, 512 prefill tokens, one shared list of 3082 slots per layer; measured on 4 "
+                                 "layers, tokens/s scaled to 32 layers",
+                     "tokens_per_s": cfg4.tokens / (us_call * 1e-6 * cfg4.n_layers), "us_per_layer_call": us_call,
+                     "bound": "tensor", "achieved_tflops": tflops, "peak": peaks["bf16_tflops_sustained"],
+                     "frac": tflops / peaks["bf16_tflops_sustained"], "peak_kind": f"of {peak_kind} (sustained)",
+                     "replayed_from_cuda_graph": was_graph}
+    except Exception as e:                              # pragma: no cover
+        out["c4"] = {"error": repr(e)}
+
+    # ---- c5: 16 cells (loaded x active), 4 layers x 64 tokens per launch.  The loaded set of a cell is the
+    # first n_loaded ids of the layer's ranking, slot = rank, so one store holding every neuron serves all cells.
+    try:
+        n_layers = 4
+        base = wl.CONFIGS["c5"].with_(n_layers=n_layers, loaded_pct=100)
+        store = load_store(api, torch, base, n_layers, device)
+        tdt = api.torch_dtype(base.dtype)
+        d, tokens = base.d_model, base.tokens
+        n_steps = tokens * n_layers
+        x = torch.empty(tokens, n_layers, d, dtype=torch.int16)
+        for l in range(n_layers):
+            x[:, l] = torch.from_numpy(wl.x_tokens(base, l, tokens).view(np.int16))
+        x = x.cuda().view(tdt).view(n_steps, d)
+        heads = x.view(tokens, n_layers, d)[:, 0].contiguous()
+        y = torch.empty(n_steps, d, dtype=tdt, device="cuda")
+        cells = []
+        for lp in wl.C5_LOADED:
+            for ap in wl.C5_ACTIVE:
+                cfg = base.with_(loaded_pct=lp, active_pct=ap)
+                k = cfg.k_active
+                lists = np.empty((tokens, n_layers, k), dtype=np.int32)
+                for l in range(n_layers):
+                    lists[:, l] = wl.zipf_lists(cfg, l, tokens)
+                idx = torch.from_numpy(lists.reshape(n_steps, k)).cuda()
+                ws = store.workspace(1, k, n_steps)
+                ms = device_ms(torch, lambda: api.si_decode_stack_forward(store.handle, n_steps, None, x, idx, None, k, y, 0, ws, status), 5)
+                ms_any = device_ms(torch, lambda: api.si_decode_stack_forward(store.handle, n_steps, None, x, idx, None, k, y,
+                                                                              api.SI_FLAG_STEPS_ANY_ORDER, ws, status), 5)
+                ms_ch = device_ms(torch, lambda: api.si_decode_chain_forward(store.handle, n_steps, None, n_layers, heads, idx, None, k, y,
+                                                                             None, CHAIN_EPS, api.SI_FLAG_PRENORM | api.SI_FLAG_RESIDUAL,
+                                                                             ws, status), 3)
+                bytes_step = k * cfg.record_bytes
+                cell = {"loaded_pct": lp, "active_pct": ap, "k": k}
+                for name, m in (("in_order", ms), ("any_order", ms_any), ("chained", ms_ch)):
+                    us = m * 1e3 / n_steps
+                    cell[name] = {"us_per_step": us, "gbs": bytes_step / us / 1e3, "frac_of_nominal_8TBs": bytes_step / us / 1e3 / NOMINAL_HBM_GBS,
+                                  "tokens_per_s_32_layers": 1e6 / (us * 32)}
+                cells.append(cell)
+                del ws, idx
+        out["c5"] = {"workload": "c5: 8B-shaped FFN (d_model=4096, d_ff=14336, bf16), loaded {30,50,70,100}% x active {5,10,20,50}% of "
+                                 "loaded, Zipf lists, batch 1, 64 tokens; measured on 4 layers per launch (256 steps), tokens/s scaled "
+                                 "to 32 layers", "bound": "hbm", "cells": cells}
+        store.close()
+    except Exception as e:                              # pragma: no cover
+        out["c5"] = {"error": repr(e)}
+    if int(status.item()) != 0:
+        out["device_status"] = int(status.item())
+    return out
 
 # ----------------------------------------------------------------------------- our arm
 
@@ -324,10 +547,43 @@ def run_ours(args):
         time.sleep(0.3)
     total_ms, per_step_ms, (t0, t1) = timed(step_device, args.steps, max(args.warmup, 3))
     clocks = sampler.stop(t0, t1) if sampler else None
-    any_ms, any_per, _ = timed(step_device_any_order, args.steps, max(args.warmup, 3))
+    side_steps = max(3, min(args.steps, 20))               # the figures beside the headline need no long region
+    any_ms, any_per, _ = timed(step_device_any_order, side_steps, 3)
     e2e_ms, _, _ = timed(step_e2e, args.steps, max(args.warmup, 3))
     if int(status.item()) != 0:
         raise SystemExit(f"device status {status.item()}: {api.strerror(int(status.item()))}")
+    chained = None
+    if rank == 0 and not args.simple and not args.no_chained:
+        peaks_c, _ = measured_peaks()
+        heads_dev = x_dev.view(tokens, L, d)[:, 0].contiguous()         # a token's chain starts from its layer-0 input
+        chained, y_chain = measure_chained(api, torch, store, cfg, heads_dev, idx_dev, ws, status, peaks_c, side_steps)
+        if int(status.item()) != 0:
+            raise SystemExit(f"device status {status.item()} in the chained launch: {api.strerror(int(status.item()))}")
+        if cpu_tokens:
+            # parity of the chained launch: sampled steps against the oracle fed with the very input the device read
+            xn = torch.empty(n_steps, d, dtype=tdt, device="cuda")
+            api.si_decode_chain_forward(store.handle, n_steps, None, L, heads_dev, idx_dev, None, k, y_chain, xn, CHAIN_EPS,
+                                        api.SI_FLAG_PRENORM | api.SI_FLAG_RESIDUAL, ws, status)
+            torch.cuda.synchronize()
+            bits = lambda t_: t_.view(torch.int16).cpu().numpy().view(np.uint16)
+            t_s = cpu_tokens - 1
+            errs = []
+            for l in (0, L - 1):
+                s_ = t_s * L + l
+                wg, wu, wd = wl.layer_weights(cfg, l)
+                ids, sor = wl.loaded_ids(cfg, l)
+                x_in = bits(heads_dev[t_s]) if l == 0 else bits(y_chain[s_ - 1])
+                xin64 = oracle.widen_bits(x_in, cfg.dtype)
+                xn_ref = oracle.rmsnorm(xin64, CHAIN_EPS)
+                xn_dev = oracle.widen_bits(bits(xn[s_]), cfg.dtype)
+                lst = idx_host.view(n_steps, k)[s_].numpy()
+                ref = oracle.ffn(wg, wu, wd, bits(xn[s_]), ids[lst], dtype=cfg.dtype, threads=host_threads) + xin64
+                e = oracle.error_metrics(oracle.widen_bits(bits(y_chain[s_]), cfg.dtype), ref)
+                errs.append({"step": [t_s, l], "max_rel": e[0], "mean_rel": e[1],
+                             "norm_max_rel_dev": float(np.max(np.abs(xn_dev - xn_ref) / np.maximum(np.abs(xn_ref), 1e-30)))})
+                del wg, wu, wd
+            chained["parity_samples"] = errs
+            del xn
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
@@ -364,7 +620,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": y_host.numel() * y_host.element_size(),
                     "launches_per_step": n_chunk if not args.simple else 2 * n_steps,
                     "pipeline": f"chunks of {sizes} tokens: copies of one chunk overlap the launch of another"},
-            "gpu_launches": args.steps * (1 if not args.simple else 2 * n_steps),
+            "gpu_launches": args.steps * (1 if not args.simple else 2 * n_steps),     # (headline region; the side figures launch more)
             "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
@@ -379,9 +635,14 @@ def run_ours(args):
                                       if (cfg.name == "c2" and not args.simple) else None))},
             "load_seconds": load_s,
         }
+        out["config"]["steps"] = "independent: every (token, layer) step's input is given up front; worked through in order"
+        if clocks and clocks.get("sm_mhz"):
+            out["ms_per_step_x_sm_mhz"] = total_ms / args.steps * clocks["sm_mhz"]       # comparable across GPUs that clock differently
+        if chained is not None:
+            out["chained"] = chained
         any_launch_ms = statistics.mean(any_per)
         out["steps_any_order"] = {
-            "value": replicas.aggregate_throughput(tokens * args.steps, world, any_ms), "unit": UNIT,
+            "value": replicas.aggregate_throughput(tokens * side_steps, world, any_ms), "unit": UNIT,
             "achieved_gbs": alg_bytes / (any_launch_ms * 1e-3) / 1e9,
             "frac": alg_bytes / (any_launch_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "frac_of_read_only_kernel": alg_bytes / (any_launch_ms * 1e-3) / 1e9 / read_ceiling,
@@ -400,6 +661,11 @@ def run_ours(args):
                           f"{host_threads} OpenMP threads",
                 "single_thread": {"value": (cpu_layers_1t / L) / cpu_time_1t if cpu_time_1t > 0 else None, "unit": UNIT,
                                   "sample": f"1 token x {cpu_layers_1t} layers with one thread, scaled to {L} layers"}}
+        if world == 1 and not args.no_extra_configs and cfg.name == "c2":
+            store.close()
+            del store
+            torch.cuda.empty_cache()
+            out["configs"] = extra_configs(api, torch, args, f"cuda:{local_rank}", peaks, peak_kind)
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -500,7 +766,7 @@ def run_multitoken(args, cfg, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=80, help="timed steps (launches) of the headline: 80 x 25 ms = 2 s")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
@@ -511,12 +777,18 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="c3: tokens processed together per step")
     ap.add_argument("--cpu-tokens", type=int, default=8, help="tokens of the oracle cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chained", action="store_true", help="skip the chained launch beside the headline")
+    ap.add_argument("--no-extra-configs", action="store_true", help="skip the configs object (c1, c3, c4, c5)")
     ap.add_argument("--e2e-sizes", default="", help="tokens per chunk of the end-to-end pipeline, comma separated (default: derived)")
     ap.add_argument("--simple", action="store_true", help="time the per-step plain-load kernels instead")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch from an ncu capture (default: the committed capture of the "
                          "persistent kernel, scaled by the number of steps)")
     args = ap.parse_args()
+    # started without a launcher: start the N ranks ourselves (each re-enters here with WORLD_SIZE set)
+    rc = replicas.ensure_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:])
+    if rc is not None:
+        raise SystemExit(rc)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -65,8 +65,7 @@ constexpr int kLag = 4;                           // a step's cross-SM reduction
 constexpr long long kWaitCycles = 4000000000ll;   // default limit of every wait: ~2 s at 1.9 GHz
 constexpr long long kDrainCycles = 40000000ll;    // least time a leaving producer gives its copies in flight to land
 constexpr int kLLRows = 8;                        // chained mode: most partial rows one consumer thread gathers per step
-constexpr int kChainCmb = 0, kChainXch = 1, kChainOwn = 2;   // chained mode: which hand-over barrier serves what ([0][..])
-constexpr int kChainRows = 0, kChainInput = 1;               // ... and [1][..]: "every CTA's row is written", "the input row is written"
+constexpr int kChainCmb = 0, kChainXch = 1, kChainRows = 2;   // chained mode: which hand-over barrier serves what
 
 struct Params {
     const char *store_base;
@@ -385,14 +384,11 @@ __device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, 
             const int c = t + kSetThreads * i;
             if (kFull || c < chunks) unpack8p<DT>(__ldg(xs + c), xr[i]);
         }
-        if (ct == 0) mbar_arrive(&sm->accfull[1][kChainInput]);      // (nothing to wait for: keeps the barrier's phase in step)
     } else {
-        // 8-byte words {two 16-bit values, tag = this step}; the count of CTAs that have written their
-        // columns is only a hint that spares the memory system 75 000 threads polling the words while the
-        // last CTAs are still at work: what counts is the tag in every word
+        // 8-byte words {two 16-bit values, tag = this step}, polled until every word this thread needs carries
+        // the tag (the row is 16 KB for all of them together: polling it costs the memory system little, and
+        // measured a little less time than waiting for a count of the CTAs that have written their columns)
         const uint4 *lx = reinterpret_cast<const uint4 *>(P.ll_x + (size_t)(step & 1) * (d / 2));
-        fail |= !hint_wait_cta(P.counters + (size_t)(step - 1) * kCounterStride + 32, (unsigned)G, P.ctrl + 1, cta_abort,
-                               wait_limit, ct == 0, &sm->accfull[1][kChainInput], (uint32_t)(step & 1));
         const long long t0 = clock64();
         uint32_t spins = 0;
         while (!fail) {
@@ -600,7 +596,7 @@ __device__ __noinline__ bool chain_step_exchange(const Params &P, uint8_t *smem,
         const uint4 *src = reinterpret_cast<const uint4 *>(P.ll_partial + (size_t)rc * d + col0);
         const size_t stride = (size_t)classes * d / 2;             // uint4 units between this thread's rows
         fail |= !hint_wait_cta(P.counters + (size_t)step * kCounterStride, (unsigned)G, P.ctrl + 1, cta_abort, wait_limit,
-                               ct == 0, &sm->accfull[1][kChainRows], par);
+                               ct == 0, &sm->accfull[0][kChainRows], par);
         SI_CPROF(4);                                      // every CTA's row counted as written
         float sx = 0.f, sy = 0.f;
         const long long t0 = clock64();
@@ -655,16 +651,6 @@ __device__ __noinline__ bool chain_step_exchange(const Params &P, uint8_t *smem,
     const bool feeds = step + 1 < P.n_steps && (step + 1) % P.chain_len != 0;       // the next step reads this row
     if (feeds && owner && p4 == 0 && (col & 1) == 0 && !fail)
         st_relaxed_gpu_v2(P.ll_x + (size_t)((step + 1) & 1) * (d / 2) + gcol / 2, make_uint2(o16 | (odd << 16), tag));
-    // the warps that hold column owners meet (every step, so the barrier's phase follows the step), then one
-    // thread counts this CTA's columns as written (a hint)
-    if (ct < ((pieces * 8 + 31) & ~31)) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm->accfull[0][kChainOwn]);
-        if (ct == 0) {
-            if (!mbar_wait_bounded(&sm->accfull[0][kChainOwn], par, cta_abort, wait_limit)) fail = true;
-            else if (feeds) red_add_relaxed_gpu(P.counters + (size_t)step * kCounterStride + 32, 1u);
-        }
-    }
     SI_CPROF(7);                                          // column sums, y, next input row
     return fail;
 }
@@ -722,11 +708,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         for (int q = 0; q < kSets; ++q)
             for (int w = 0; w < kReducerWarps; ++w) { mbar_init(&sm->accfull[q][w], kSetWarps); mbar_init(&sm->accempty[q][w], 1); }
         if (CH) {     // chained mode has no hand-over to reducers: three of those barriers serve its consumers
-            const int gpc0 = (P.d_model / 4 + (int)gridDim.x - 1) / (int)gridDim.x;
             mbar_init(&sm->accfull[0][kChainCmb], kSetWarps);               // second set's accumulators parked
             mbar_init(&sm->accfull[0][kChainXch], kConsumerWarps);          // every warp's class sums written
-            mbar_init(&sm->accfull[0][kChainOwn], (gpc0 * 16 + 31) / 32);   // every column owner's stores issued
-            mbar_init(&sm->accfull[1][kChainRows], 1); mbar_init(&sm->accfull[1][kChainInput], 1);   // news from the polling thread
+            mbar_init(&sm->accfull[0][kChainRows], 1);                      // the polling thread's news: every CTA's row is written
         }
         sm->cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -846,7 +830,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     ++issued;
                     n += S; iph ^= 1;
                     progressed = true;
-                    if (CH && n < i_ready && !(P.stream_only & 8)) {
+                    if (CH && n < i_ready) {
                         // chained: between two steps the ring stands still while the SMs exchange their sums;
                         // the record that will follow this one through the stage is asked into L2 meanwhile
                         const uint4 nx = sm->desc[iq][n % kDescRing];
@@ -860,7 +844,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 t_last = clock64();
             } else {
                 if (*cta_abort || clock64() - t_last > wait_limit) { ok = false; break; }
-                if (!chained || (P.stream_only & 16)) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
+                if (!chained) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -1281,7 +1265,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
     P.prof = ex->profile;
-    P.stream_only = ex->skip_mask & 31;
+    P.stream_only = ex->skip_mask & 7;
     if (ex->ring_stages > 0 && !wide && 2 * ex->ring_stages <= P.nstage) P.nstage = 2 * ex->ring_stages;   // diagnostics: shallower rings
     P.wait_cycles = ex->wait_cycles > 0 ? ex->wait_cycles : si_persist::kWaitCycles;
     P.withhold = ex->withhold;

@@ -44,3 +44,32 @@ def barrier():
     import torch.distributed as dist
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.barrier()
+
+
+def launch_command(n_ranks: int, script: str, argv, port: int | None = None):
+    """Command line that starts `script argv...` as n_ranks processes of one node, one per GPU, the way
+    the benchmark contract launches a multi-GPU run (torch.distributed.run, rendezvous on 127.0.0.1)."""
+    import socket
+    import sys
+    if n_ranks < 1:
+        raise ValueError("n_ranks must be positive")
+    if port is None:
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), script, *[str(a) for a in argv]]
+
+
+def ensure_ranks(n_ranks: int, script: str, argv, env=None):
+    """If n_ranks > 1 and this process was not started by a launcher (no WORLD_SIZE in the environment),
+    start the ranks and return their exit code; otherwise return None and the caller carries on as the
+    rank it is.  NCCL's communicator set-up lines are left on for the ranks (stderr) unless the caller's
+    environment says otherwise, so a scaling run shows what transport it ran on."""
+    import subprocess
+    if n_ranks <= 1 or "WORLD_SIZE" in os.environ:
+        return None
+    child_env = dict(os.environ if env is None else env)
+    child_env.setdefault("NCCL_DEBUG", "INFO")
+    child_env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    return subprocess.call(launch_command(n_ranks, script, argv), env=child_env)

@@ -47,3 +47,31 @@ def test_two_replicas_over_gloo():
 def test_single_process_defaults():
     assert replicas.max_over_ranks(3.5) == 3.5
     assert replicas.token_range(0, 1, 128) == (0, 128)
+
+
+def test_ensure_ranks_starts_the_ranks_itself(tmp_path):
+    """`bench.py --gpus N` without a launcher: the process starts its own N ranks (here 2 gloo ranks on
+    CPU running a small child script) and hands their exit code back; inside a rank nothing is started."""
+    import json
+    import subprocess
+    import sys
+    cmd = replicas.launch_command(3, "x.py", ["--gpus", 3], port=1234)
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nproc-per-node=3" in cmd and cmd[-3:] == ["x.py", "--gpus", "3"] and "127.0.0.1" in cmd and "1234" in cmd
+    out = tmp_path / "ranks.json"
+    child = os.path.join(os.path.dirname(os.path.abspath(__file__)), "replica_child.py")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    env["PYTHONPATH"] = root + os.pathsep + env.get("PYTHONPATH", "")
+    saved = {k: os.environ.pop(k) for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK") if k in os.environ}
+    try:
+        assert replicas.ensure_ranks(1, child, [str(out)], env=env) is None          # one rank: nothing to start
+        rc = replicas.ensure_ranks(2, child, [str(out), "--flag"], env=env)
+        assert rc == 0
+        got = json.loads(out.read_text())
+        assert got == {"world": 2, "sum": 3.0, "max_ms": 11.0, "argv": ["--flag"]}
+        os.environ["WORLD_SIZE"] = "2"                                                # already a rank: nothing is started
+        assert replicas.ensure_ranks(2, child, [str(out)], env=env) is None
+    finally:
+        os.environ.pop("WORLD_SIZE", None)
+        os.environ.update(saved)
