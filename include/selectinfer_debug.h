@@ -25,6 +25,9 @@ typedef struct si_debug_decode_opts {
                               ring, so that CTA's consumers wait for a record that does not come: with a short
                               wait_cycles this exercises the time-out path (status SI_ERR_TIMEOUT, grid-wide
                               abort, clean return).  Nothing faults and no wait is unbounded. */
+    int chain_form;        /* si_debug_decode_chain_forward: 0 = the library's choice; 1 = the SMs exchange partial
+                              output rows; 2 = the split form that exchanges the activations (SI_ERR_UNSUPPORTED where
+                              it does not apply); results agree up to fp32 summation order */
     long long wait_cycles; /* limit of every device-side wait in clock cycles (0 = the default, about 2 s) */
     void *profile;         /* device int64 [num_SMs][16] or NULL: per-SM cycle counts of the phases.  Slots 0..5:
                               first consumer set (wait for x, wait for a record + copy to registers, record
@@ -32,10 +35,12 @@ typedef struct si_debug_decode_opts {
                               exchange); 6..7: second set (wait for the hand-over buffer, wait for a record);
                               8..13: first reducer warp (idle, wait for a free partial-ring slot, copy
                               accumulators out, publish, wait for all SMs, reduce + write y).
-                              Chained launches: slots 0..7 first consumer set, 8..15 second set (wait for
-                              the input row, normalisation + records, wait for the second set / park the
-                              accumulators, store the CTA's row, wait for every CTA's row, gather the rows,
-                              wait for the class sums, column sums + y + next input row). */
+                              Chained launches: slots 0..7 first consumer set, 8..15 second set.  Form 1:
+                              wait for the input row, normalisation + records, wait for the second set / park
+                              the accumulators, store the CTA's row, wait for every CTA's row, gather the rows,
+                              wait for the class sums, column sums + y + next input row.  Form 2 (split): 0 input
+                              row, 1 records, 4 gather h, 5 wait for all h and the slices, 6 partial sums,
+                              7 final sums + y + next input row. */
 } si_debug_decode_opts_t;
 
 /* si_decode_stack_forward with the options above (opts == NULL: identical to it). */

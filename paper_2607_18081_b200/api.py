@@ -315,11 +315,12 @@ def si_debug_read_bandwidth(mem, nbytes: int, checksum, stream=None) -> None:
 class DecodeOpts(ctypes.Structure):
     """si_debug_decode_opts_t: per-call diagnostics of a persistent decode launch (all zero = none)."""
     _fields_ = [("skip_mask", ctypes.c_int), ("ring_stages", ctypes.c_int), ("step_groups", ctypes.c_int),
-                ("withhold", ctypes.c_int), ("wait_cycles", ctypes.c_longlong), ("profile", ctypes.c_void_p)]
+                ("withhold", ctypes.c_int), ("chain_form", ctypes.c_int), ("wait_cycles", ctypes.c_longlong),
+                ("profile", ctypes.c_void_p)]
 
 
-def _opts(skip_mask=0, ring_stages=0, step_groups=0, withhold=0, wait_cycles=0, profile=None) -> DecodeOpts:
-    return DecodeOpts(skip_mask, ring_stages, step_groups, withhold, wait_cycles,
+def _opts(skip_mask=0, ring_stages=0, step_groups=0, withhold=0, chain_form=0, wait_cycles=0, profile=None) -> DecodeOpts:
+    return DecodeOpts(skip_mask, ring_stages, step_groups, withhold, chain_form, wait_cycles,
                       None if profile is None else profile.data_ptr())
 
 

@@ -171,6 +171,7 @@ static si_decode_extra extra_of(const si_debug_decode_opts_t *o) {
     if (o) {
         ex.skip_mask = o->skip_mask; ex.ring_stages = o->ring_stages; ex.step_groups = o->step_groups;
         ex.withhold = o->withhold; ex.wait_cycles = o->wait_cycles; ex.profile = (long long *)o->profile;
+        ex.chain_form = o->chain_form;
     }
     return ex;
 }

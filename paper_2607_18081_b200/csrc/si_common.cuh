@@ -74,6 +74,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
 // si_decode_chain_forward and the per-call diagnostics of si_debug_decode_stack_forward.
 struct si_decode_extra {
     int chain_len = 0;             // > 0: chained steps (persistent kernel only)
+    int chain_form = 0;            // 0: the library's choice; 1: the SMs exchange partial output rows; 2: split form (activations)
     int prenorm = 0;
     float norm_eps = 0.f;
     void *xn_out = nullptr;

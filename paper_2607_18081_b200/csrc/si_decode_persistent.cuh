@@ -66,6 +66,10 @@ constexpr long long kWaitCycles = 4000000000ll;   // default limit of every wait
 constexpr long long kDrainCycles = 40000000ll;    // least time a leaving producer gives its copies in flight to land
 constexpr int kLLRows = 8;                        // chained mode: most partial rows one consumer thread gathers per step
 constexpr int kChainCmb = 0, kChainXch = 1, kChainRows = 2;   // chained mode: which hand-over barrier serves what
+constexpr int kSplitSlicesFull = 0, kSplitSlicesFree = 1, kSplitH = 2, kSplitRed = 3, kSplitHint = 4, kSplitInput = 5;   // split form: accfull[q][w] taken as [q * 3 + w]
+constexpr int kSplitLoaderWarps = 2;                          // split form: warps that copy the down slices
+constexpr int kThreadsSplit = 32 + kConsumers + 32 * kSplitLoaderWarps;
+constexpr int kSplitKCapMax = 1856;                           // split form: list entries whose slices fit beside six ring stages at d_model 4096
 
 struct Params {
     const char *store_base;
@@ -106,6 +110,18 @@ struct Params {
     uint2 *ll_partial;            // [G][d_model] {fp32 partial sum of the CTA's records, tag}, zero at launch
     uint2 *ll_x;                  // [2][d_model / 2] {two 16-bit values of the next input row, tag}, zero at launch
     unsigned csum_off;            // chained mode: byte offset of the [columns][classes] class sums in shared memory
+    // chained mode, split form (template parameter CH == 2): a step is cut at the activations instead of
+    // at the output.  Every set computes h for its records from the gate and up rows alone and publishes it
+    // as one {h, tag} word; every CTA gathers all h of the step (a few KB) and forms the output columns it owns
+    // from 16-byte slices of ALL the step's down rows, which a loader warp pair has copied into shared memory
+    // long before (their addresses depend on the list alone).  What crosses between the SMs per step is then
+    // k + d_model words instead of the SMs x d_model partial sums of the other form.
+    unsigned stage_bytes;         // bytes of a ring stage (a whole record, or its gate and up rows)
+    unsigned copy_bytes;          // bytes the producer copies per record
+    unsigned sm_off;              // byte offset of the Smem struct
+    unsigned sbuf_off, hbuf_off, red_off, prev_off;   // split form: down slices [k_cap][64 B], h [k_cap], partial sums, last outputs
+    int k_cap;                    // split form: most list entries per step (what the slice buffer holds)
+    uint2 *ll_h;                  // split form: [2][k_cap] {h, tag}, zero at launch
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -148,6 +164,19 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     while (true) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
+        if (*cta_abort) return false;
+        if (clock64() - t0 > limit) return false;
+    }
+}
+// The same wait as a spin on the non-blocking probe: a thread suspended inside try_wait is not woken the
+// moment the phase completes, which costs the chained steps (whose every wait is on the critical path)
+// far more than the issue slots of a spin.
+__device__ __forceinline__ bool mbar_spin_bounded(uint64_t *bar, uint32_t parity, volatile int *cta_abort, long long limit) {
+    if (mbar_test_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    while (true) {
+        for (int i = 0; i < 32; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
         if (*cta_abort) return false;
         if (clock64() - t0 > limit) return false;
     }
@@ -346,37 +375,20 @@ __device__ __forceinline__ void raise_abort(const Params &P, Smem *sm, int code)
 // row: the second set parks its accumulators in shared memory, the first adds them to its own and stores
 // the row as {partial sum, tag} words, then counts the row as written (a hint for the pollers).
 // ring: stage | phase parity << 8 | exchange-buffer parity << 9 of the set's next ring item.
-// optional phase profile of the chained steps: thread 0 of each set adds the cycles since its last stamp to a slot
-#define SI_CPROF(slot) do { if (cprof) { const long long now_ = clock64(); atomicAdd((unsigned long long *)(P.prof + (size_t)blockIdx.x * kProfSlots + (slot) + 8 * q_), (unsigned long long)(now_ - pt_)); pt_ = now_; } } while (0)
 
+// Chained mode, both forms: the step's input row into packed fp32 pairs.  Either the caller's row (first
+// step of a chain) or the {two 16-bit values, tag} words the CTAs wrote at the end of the step before,
+// polled until every word this thread needs carries this step's tag (the row is 16 KB for all of them
+// together: polling it costs the memory system little, and measured a little less time than waiting for a
+// count of the CTAs that have written their columns).  With Params::prenorm the row is scaled to unit root
+// mean square and rounded to the store type.  Contains a barrier over the set that also ORs `fail`.
 template <int DT, int NCH, bool kFull>
-__device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, int step, unsigned &ring) {
-    constexpr int kSets = 2, kSetWarps = 8, kSetThreads = 256;
-    const int d = P.d_model, chunks = P.chunks, rec_bytes = d * 6, S = P.nstage / kSets;
-    const int G = gridDim.x, b = blockIdx.x;
-    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)P.nstage * rec_bytes + (size_t)kSets * d * 4);
-    float *comb = reinterpret_cast<float *>(smem + (size_t)P.nstage * rec_bytes);      // [d_model] second set's accumulators
+__device__ __forceinline__ bool chain_input(const Params &P, Smem *sm, int step, int q, int t, unsigned long long (&xr)[NCH][4],
+                                            uint32_t &recs, bool fail, uint64_t *hint_bar = nullptr, unsigned hint_target = 0) {
+    constexpr int kSetWarps = 8, kSetThreads = 256;
+    const int d = P.d_model, chunks = P.chunks, b = blockIdx.x, lane = t & 31, sw = t >> 5;
     volatile int *cta_abort = &sm->cta_abort;
     const long long wait_limit = P.wait_cycles;
-    const int ct = threadIdx.x - 32, lane = ct & 31;
-    const int q = ct / kSetThreads, t = ct & (kSetThreads - 1), sw = t >> 5;
-    uint64_t *sfull = sm->full + q * S, *sempty = sm->empty + q * S;
-    const int *smeta = sm->meta + q * S;
-    const uint8_t *sring = smem + (size_t)q * S * rec_bytes;
-    int st = (int)(ring & 0xFFu); uint32_t ph = (ring >> 8) & 1u, recs = (ring >> 9) & 1u;
-    bool fail = false;
-    const uint32_t tag = (uint32_t)step + 1u;
-    const bool cprof = P.prof != nullptr && t == 0;
-    const int q_ = q;
-    long long pt_ = cprof ? clock64() : 0;
-
-    unsigned long long xr[NCH][4], acc[NCH][4];   // packed fp32 pairs
-#pragma unroll
-    for (int i = 0; i < NCH; ++i)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { acc[i][e] = 0ull; xr[i][e] = 0ull; }
-    const int cnt = step_geom(P, step, G * kSets, kSets * b + q).cnt;
-    // ---- the input row
     if (step % P.chain_len == 0) {
         const uint4 *xs = reinterpret_cast<const uint4 *>(P.x + (size_t)(step / P.chain_len) * d);
 #pragma unroll
@@ -384,11 +396,17 @@ __device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, 
             const int c = t + kSetThreads * i;
             if (kFull || c < chunks) unpack8p<DT>(__ldg(xs + c), xr[i]);
         }
+        if (hint_bar && q == 0 && t == 0) mbar_arrive(hint_bar);      // (nothing to wait for: keeps the barrier's phase in step)
     } else {
         // 8-byte words {two 16-bit values, tag = this step}, polled until every word this thread needs carries
         // the tag (the row is 16 KB for all of them together: polling it costs the memory system little, and
         // measured a little less time than waiting for a count of the CTAs that have written their columns)
         const uint4 *lx = reinterpret_cast<const uint4 *>(P.ll_x + (size_t)(step & 1) * (d / 2));
+        // split form: one thread of the CTA waits for the count of CTAs that have written their columns (a hint),
+        // so that the row's few lines are read once instead of being polled by every thread of the GPU
+        if (hint_bar)
+            fail |= !hint_wait_cta(P.counters + (size_t)(step - 1) * kCounterStride + 32, hint_target, P.ctrl + 1, cta_abort, wait_limit,
+                                   q == 0 && t == 0, hint_bar, (uint32_t)(step & 1));
         const long long t0 = clock64();
         uint32_t spins = 0;
         while (!fail) {
@@ -428,7 +446,6 @@ __device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, 
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
         if (lane == 0) sm->setpart[q][recs & 1][sw].x = ss;
     }
-    SI_CPROF(0);                                          // the input row has arrived
     fail = set_barrier_or<kSetThreads>(q, fail);          // one verdict for the set (and the warp sums are in place)
     if (fail) return true;
     if (P.prenorm) {
@@ -453,6 +470,43 @@ __device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, 
                 reinterpret_cast<uint4 *>(P.xn_out + (size_t)step * d)[c] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
     }
+    return false;
+}
+
+// optional phase profile of the chained steps: thread 0 of each set adds the cycles since its last stamp to a slot
+#define SI_CPROF(slot) do { if (cprof) { const long long now_ = clock64(); atomicAdd((unsigned long long *)(P.prof + (size_t)blockIdx.x * kProfSlots + (slot) + 8 * q_), (unsigned long long)(now_ - pt_)); pt_ = now_; } } while (0)
+
+template <int DT, int NCH, bool kFull>
+__device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, int step, unsigned &ring) {
+    constexpr int kSets = 2, kSetWarps = 8, kSetThreads = 256;
+    const int d = P.d_model, chunks = P.chunks, rec_bytes = d * 6, S = P.nstage / kSets;
+    const int G = gridDim.x, b = blockIdx.x;
+    Smem *sm = reinterpret_cast<Smem *>(smem + P.sm_off);
+    float *comb = reinterpret_cast<float *>(smem + (size_t)P.nstage * rec_bytes);      // [d_model] second set's accumulators
+    volatile int *cta_abort = &sm->cta_abort;
+    const long long wait_limit = P.wait_cycles;
+    const int ct = threadIdx.x - 32, lane = ct & 31;
+    const int q = ct / kSetThreads, t = ct & (kSetThreads - 1), sw = t >> 5;
+    uint64_t *sfull = sm->full + q * S, *sempty = sm->empty + q * S;
+    const int *smeta = sm->meta + q * S;
+    const uint8_t *sring = smem + (size_t)q * S * rec_bytes;
+    int st = (int)(ring & 0xFFu); uint32_t ph = (ring >> 8) & 1u, recs = (ring >> 9) & 1u;
+    bool fail = false;
+    const uint32_t tag = (uint32_t)step + 1u;
+    const bool cprof = P.prof != nullptr && t == 0;
+    const int q_ = q;
+    long long pt_ = cprof ? clock64() : 0;
+
+    unsigned long long xr[NCH][4], acc[NCH][4];   // packed fp32 pairs
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { acc[i][e] = 0ull; xr[i][e] = 0ull; }
+    const int cnt = step_geom(P, step, G * kSets, kSets * b + q).cnt;
+    // ---- the input row
+    fail = chain_input<DT, NCH, kFull>(P, sm, step, q, t, xr, recs, fail);
+    SI_CPROF(0);                                          // the input row has arrived (and is normalised)
+    if (fail) return true;
     // ---- the set's records (the loop of the unchained kernel)
     const bool noarith = (P.stream_only & 1) != 0;
     for (int i = 0; i < cnt; ++i) {
@@ -578,7 +632,7 @@ __device__ __noinline__ bool chain_step_records(const Params &P, uint8_t *smem, 
 template <int DT, int LLR>
 __device__ __noinline__ bool chain_step_exchange(const Params &P, uint8_t *smem, int step) {
     const int d = P.d_model, G = gridDim.x, b = blockIdx.x;
-    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)P.nstage * d * 6 + (size_t)2 * d * 4);
+    Smem *sm = reinterpret_cast<Smem *>(smem + P.sm_off);
     float *csum = reinterpret_cast<float *>(smem + P.csum_off);          // [columns][classes] class sums
     volatile int *cta_abort = &sm->cta_abort;
     const long long wait_limit = P.wait_cycles;
@@ -655,6 +709,322 @@ __device__ __noinline__ bool chain_step_exchange(const Params &P, uint8_t *smem,
     return fail;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Chained mode, split form (CH == 2): the step is cut at the activations.
+//   first half   every set: h of its records from their gate and up rows (the ring carries only those),
+//                each h published as one {h, tag} word;
+//   second half  every CTA: all h of the step gathered (k words), then the output columns this CTA owns,
+//                sum over the step's records of h x (16-byte slices of their down rows), the slices copied
+//                into shared memory by two loader warps while the first half and the exchanges ran; residual,
+//                rounding, y, and the {values, tag} words of the next input row.
+// Column ownership: the d_model / 8 groups of eight columns (16 bytes of a down row) are dealt to the CTAs
+// in order, the first (groups mod CTAs) of them getting one more; a CTA owns at most four groups.
+struct SplitCols { int g0, ng; };
+__device__ __forceinline__ SplitCols split_cols(int d, int G, int b) {
+    const int ngrp = d / 8, base = ngrp / G, rem = ngrp % G;
+    SplitCols c;
+    c.ng = base + (b < rem ? 1 : 0);
+    c.g0 = b * base + (b < rem ? b : rem);
+    return c;
+}
+__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+// arrival that happens by itself once every cp.async this thread has issued so far has landed (counts as
+// one of the barrier's expected arrivals)
+__device__ __forceinline__ void cp_async_arrive_when_landed(uint64_t *bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ uint64_t *split_bar(Smem *sm, int which) { return &sm->accfull[0][0] + which; }
+
+struct SplitList { int base, k, layer; };
+__device__ __forceinline__ SplitList split_list(const Params &P, int step) {
+    SplitList l;
+    l.layer = P.step_layers ? __ldg(P.step_layers + step) : (P.n_few ? (int)P.few_layers[step] : step % P.n_layers);
+    if (P.idx_offsets) {
+        const int o0 = __ldg(P.idx_offsets + step), o1 = __ldg(P.idx_offsets + step + 1);
+        l.base = o0; l.k = o1 - o0 < 0 ? 0 : o1 - o0;
+    } else {
+        l.base = P.per_layer_lists ? l.layer * P.k_fixed : step * P.k_fixed; l.k = P.k_fixed;
+    }
+    if (l.k > P.k_cap) l.k = P.k_cap;       // (a longer list is reported by the first half; nothing is read beyond the buffers)
+    return l;
+}
+
+// The loader warps: for every step, once the second half of the step before has read the slice buffer, copy
+// this CTA's 16-byte column groups of every listed record's down row into it (slice p at p * 64 bytes).
+__device__ __forceinline__ void split_slice_loader(const Params &P, uint8_t *smem, Smem *sm, int lw, int lane) {
+    const int d = P.d_model, G = gridDim.x;
+    const SplitCols cols = split_cols(d, G, blockIdx.x);
+    uint8_t *sbuf = smem + P.sbuf_off;
+    bool ok = true;
+    for (int step = 0; step < P.n_steps && ok; ++step) {
+        if (step > 0) ok = mbar_wait_bounded(split_bar(sm, kSplitSlicesFree), (uint32_t)((step - 1) & 1), &sm->cta_abort, P.wait_cycles);
+        if (!ok) break;
+        const SplitList l = split_list(P, step);
+        if (cols.ng > 0) {
+            const char *rec = P.store_base + P.rec_off[l.layer] + (size_t)d * 4 + (size_t)cols.g0 * 16;   // down row, this CTA's columns
+            const int n_loaded = P.n_loaded[l.layer];
+            // all of this lane's list entries in one round of loads (a load per copy would put a trip to L2
+            // in front of every copy), then the copies
+            constexpr int kPer = kSplitKCapMax / (32 * kSplitLoaderWarps);
+            int slot[kPer];
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const int p = lw * 32 + lane + j * 32 * kSplitLoaderWarps;
+                slot[j] = p < l.k ? __ldg(P.idx + l.base + p) : -1;
+            }
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const int p = lw * 32 + lane + j * 32 * kSplitLoaderWarps;
+                if (p < l.k) {
+                    const char *src = rec + (size_t)((slot[j] >= 0 && slot[j] < n_loaded) ? slot[j] : 0) * ((size_t)d * 6);   // (a bad slot's h is zero)
+                    uint8_t *dst = sbuf + (size_t)p * 64;
+                    for (int g = 0; g < cols.ng; ++g) cp_async16(dst + g * 16, src + g * 16);
+                }
+            }
+        }
+        cp_async_arrive_when_landed(split_bar(sm, kSplitSlicesFull));
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");      // nothing of this thread may be in flight when the CTA ends
+    if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
+}
+
+// First half of a step (not inlined, like the halves of the other form): input row, then for each of the
+// set's records the two dot products, SiLU(g) * u, and the {h, tag} word of the record's list position.
+template <int DT, int NCH, bool kFull>
+__device__ __noinline__ bool split_step_gateup(const Params &P, uint8_t *smem, int step, unsigned &ring) {
+    constexpr int kSets = 2, kSetWarps = 8, kSetThreads = 256;
+    const int chunks = P.chunks, S = P.nstage / kSets;
+    const int G = gridDim.x, b = blockIdx.x;
+    Smem *sm = reinterpret_cast<Smem *>(smem + P.sm_off);
+    volatile int *cta_abort = &sm->cta_abort;
+    const long long wait_limit = P.wait_cycles;
+    const int ct = threadIdx.x - 32, lane = ct & 31;
+    const int q = ct / kSetThreads, t = ct & (kSetThreads - 1), sw = t >> 5;
+    uint64_t *sfull = sm->full + q * S, *sempty = sm->empty + q * S;
+    const int *smeta = sm->meta + q * S;
+    const uint8_t *sring = smem + (size_t)q * S * P.stage_bytes;
+    int st = (int)(ring & 0xFFu); uint32_t ph = (ring >> 8) & 1u, recs = (ring >> 9) & 1u;
+    bool fail = false;
+    const uint32_t tag = (uint32_t)step + 1u;
+    const bool cprof = P.prof != nullptr && t == 0;
+    const int q_ = q;
+    long long pt_ = cprof ? clock64() : 0;
+
+    unsigned long long xr[NCH][4];   // packed fp32 pairs
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) xr[i][e] = 0ull;
+    const StepGeom geo = step_geom(P, step, G * kSets, kSets * b + q);
+    if (geo.k > P.k_cap && t == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_OUT_OF_RANGE);   // a list longer than the call was sized for
+    fail = chain_input<DT, NCH, kFull>(P, sm, step, q, t, xr, recs, fail, split_bar(sm, kSplitInput), (unsigned)G);
+    SI_CPROF(0);                                          // the input row has arrived (and is normalised)
+    if (fail) return true;
+    uint2 *hrow = P.ll_h + (size_t)(step & 1) * P.k_cap;
+    const bool noarith = (P.stream_only & 1) != 0;
+    for (int i = 0; i < geo.cnt; ++i) {
+        fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
+        const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0
+        const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * P.stage_bytes);
+        uint4 ga[NCH], up[NCH];
+#pragma unroll
+        for (int k2 = 0; k2 < NCH; ++k2) {
+            const int c = t + kSetThreads * k2;
+            const bool in = kFull || c < chunks;
+            ga[k2] = in ? rr[c] : make_uint4(0, 0, 0, 0);
+            up[k2] = in ? rr[chunks + c] : make_uint4(0, 0, 0, 0);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sempty[st]);
+        if (++st == S) { st = 0; ph ^= 1; }
+        float g, u;
+        {
+            unsigned long long g2 = 0ull, u2 = 0ull;
+#pragma unroll
+            for (int k2 = 0; k2 < NCH; ++k2) { g2 = dot8p<DT>(ga[k2], xr[k2], g2); u2 = dot8p<DT>(up[k2], xr[k2], u2); }
+            float lo, hi;
+            unpack2(g2, lo, hi); g = lo + hi;
+            unpack2(u2, lo, hi); u = lo + hi;
+        }
+        {
+            const bool hi16 = (lane & 16) != 0;
+            float keep = (hi16 ? u : g) + __shfl_xor_sync(0xFFFFFFFFu, hi16 ? g : u, 16);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 8);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 4);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 2);
+            keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 1);
+            g = keep;
+        }
+        const uint32_t buf = recs & 1;
+        if ((lane & 15) == 0) reinterpret_cast<float *>(&sm->setpart[q][buf][sw])[lane >> 4] = g;
+        fail = set_barrier_or<kSetThreads>(q, fail);       // also orders the partials for the whole set
+        recs ^= 1u;
+        if (fail) return true;
+        if (t == 0) {
+            float gs = 0.f, us = 0.f;
+            const float4 *pp = reinterpret_cast<const float4 *>(sm->setpart[q][buf]);
+#pragma unroll
+            for (int w = 0; w < kSetWarps / 2; ++w) {
+                const float4 v4 = pp[w];
+                gs += v4.x; us += v4.y; gs += v4.z; us += v4.w;
+            }
+            const float h = okr ? si_silu_mul(gs, us) : 0.f;
+            const int p = geo.first + i * (G * kSets);
+            if (p < P.k_cap) st_relaxed_gpu_v2(hrow + p, make_uint2(__float_as_uint(h), tag));
+        }
+    }
+    ring = (unsigned)st | (ph << 8) | ((recs & 1u) << 9);
+    // this set's h words are on their way: count the set (a hint for the one polling thread of every CTA)
+    if (t == 0) red_add_relaxed_gpu(P.counters + (size_t)step * kCounterStride, 1u);
+    SI_CPROF(1);                                          // the set's records
+    return false;
+}
+
+// Second half: gather every h of the step, form this CTA's output columns from the slices, finish the step.
+template <int DT>
+__device__ __noinline__ bool split_step_down(const Params &P, uint8_t *smem, int step) {
+    const int d = P.d_model, G = gridDim.x, b = blockIdx.x;
+    Smem *sm = reinterpret_cast<Smem *>(smem + P.sm_off);
+    volatile int *cta_abort = &sm->cta_abort;
+    const long long wait_limit = P.wait_cycles;
+    const int ct = threadIdx.x - 32, lane = ct & 31;
+    const uint32_t tag = (uint32_t)step + 1u, par = (uint32_t)(step & 1);
+    float *hbuf = reinterpret_cast<float *>(smem + P.hbuf_off);
+    const uint8_t *sbuf = smem + P.sbuf_off;
+    float2 *red = reinterpret_cast<float2 *>(smem + P.red_off);           // [32 record classes][16 column pairs]
+    const SplitList l = split_list(P, step);
+    const SplitCols cols = split_cols(d, G, b);
+    bool fail = false;
+    const bool cprof = P.prof != nullptr && (ct & 255) == 0;
+    const int q_ = ct >> 8;
+    long long pt_ = cprof ? clock64() : 0;
+    // the buffers of the step before are free once every warp (the last: the one that finishes the step) has said so
+    if (step > 0) fail |= !mbar_spin_bounded(split_bar(sm, kSplitSlicesFree), (uint32_t)((step - 1) & 1), cta_abort, wait_limit);
+    {
+        // ---- all h of the step: two {h, tag} words per 16-byte load, polled until tagged
+        const uint4 *src = reinterpret_cast<const uint4 *>(P.ll_h + (size_t)(step & 1) * P.k_cap);
+        const int units = (l.k + 1) / 2;
+        // (thousands of threads polling the few lines of the h row would queue up in front of the stores they
+        // wait for: one thread waits for the count of sets, then every word is read once, tags checked)
+        fail |= !hint_wait_cta(P.counters + (size_t)step * kCounterStride, (unsigned)(2 * G), P.ctrl + 1, cta_abort, wait_limit,
+                               ct == 0, split_bar(sm, kSplitHint), par);
+        const long long t0 = clock64();
+        uint32_t spins = 0;
+        while (!fail) {
+            bool good = true;
+            uint4 w[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int u = ct + kConsumers * i;
+                if (u < units) w[i] = ld_relaxed_gpu_v4(src + u);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int u = ct + kConsumers * i;
+                if (u < units) {
+                    good &= w[i].y == tag && (2 * u + 1 >= l.k || w[i].w == tag);
+                    hbuf[2 * u] = __uint_as_float(w[i].x);
+                    if (2 * u + 1 < l.k) hbuf[2 * u + 1] = __uint_as_float(w[i].z);
+                }
+            }
+            if (good) break;
+            if ((++spins & 63u) == 0 && (*cta_abort || ld_relaxed_gpu(P.ctrl + 1) || clock64() - t0 > wait_limit)) fail = true;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(split_bar(sm, kSplitH));
+    }
+    SI_CPROF(4);                                          // this thread's share of h gathered
+    fail |= !mbar_spin_bounded(split_bar(sm, kSplitH), par, cta_abort, wait_limit);
+    fail |= !mbar_spin_bounded(split_bar(sm, kSplitSlicesFull), par, cta_abort, wait_limit);
+    SI_CPROF(5);                                          // all h and all slices in shared memory
+    {
+        // ---- lane (column group cg of eight, record class nc of 128): records nc, nc + 128, ... in ascending order,
+        // one 16-byte load per record; then the eight classes of the warp by a butterfly, and one row of 32 column
+        // sums per warp for the first warp to add up (all in a fixed order)
+        // (four neighbouring lanes read the 64 bytes of one slice, the next four the next slice: no bank conflicts)
+        const int cg = lane & 3, nc = (ct >> 5) * 8 + (lane >> 2);
+        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (cg < cols.ng && !fail) {
+            const uint8_t *sp = sbuf + cg * 16;
+            for (int p = nc; p < l.k; p += 128) {
+                const float h = hbuf[p];
+                const uint4 w = *reinterpret_cast<const uint4 *>(sp + (size_t)p * 64);
+                a[0] = fmaf(h, si_cvt<DT>::lo(w.x), a[0]); a[1] = fmaf(h, si_cvt<DT>::hi(w.x), a[1]);
+                a[2] = fmaf(h, si_cvt<DT>::lo(w.y), a[2]); a[3] = fmaf(h, si_cvt<DT>::hi(w.y), a[3]);
+                a[4] = fmaf(h, si_cvt<DT>::lo(w.z), a[4]); a[5] = fmaf(h, si_cvt<DT>::hi(w.z), a[5]);
+                a[6] = fmaf(h, si_cvt<DT>::lo(w.w), a[6]); a[7] = fmaf(h, si_cvt<DT>::hi(w.w), a[7]);
+            }
+        }
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a[e] += __shfl_xor_sync(0xFFFFFFFFu, a[e], o);
+        if (lane < 4) {
+            float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float *>(red) + (ct >> 5) * 32 + cg * 8);
+            dst[0] = make_float4(a[0], a[1], a[2], a[3]);
+            dst[1] = make_float4(a[4], a[5], a[6], a[7]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(split_bar(sm, kSplitRed));
+    }
+    SI_CPROF(6);                                          // partial sums
+    if (ct >= 32) {                                       // fifteen warps are done with the step's buffers
+        if (lane == 0) mbar_arrive(split_bar(sm, kSplitSlicesFree));
+        return fail;
+    }
+    // ---- the first warp finishes the step: the 32 record classes in ascending order, residual, rounding
+    fail |= !mbar_spin_bounded(split_bar(sm, kSplitRed), par, cta_abort, wait_limit);
+    // lane = column (32 of them): the sixteen warps' sums in warp order, all loads at once; even lanes then take
+    // their neighbour's value and finish a pair of columns
+    float vx = 0.f, vy;
+    {
+        const float *rf = reinterpret_cast<const float *>(red);
+        float r[kConsumerWarps];
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) r[w] = rf[w * 32 + lane];
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) vx += r[w];
+        vy = __shfl_down_sync(0xFFFFFFFFu, vx, 1);
+    }
+    const int pair = lane >> 1;
+    if ((lane & 1) == 0 && pair < 4 * cols.ng && !fail) {
+        const int gcol = cols.g0 * 8 + pair * 2;
+        uint32_t *prev = reinterpret_cast<uint32_t *>(smem + P.prev_off) + pair;     // this thread's output of the step before
+        if (P.residual) {
+            const uint32_t xin = step % P.chain_len != 0 ? *prev
+                                                         : *reinterpret_cast<const uint32_t *>(P.x + (size_t)(step / P.chain_len) * d + gcol);
+            vx += si_cvt<DT>::lo(xin); vy += si_cvt<DT>::hi(xin);
+        }
+        const uint32_t o = (uint32_t)si_cvt<DT>::from_float(vx) | ((uint32_t)si_cvt<DT>::from_float(vy) << 16);
+        *prev = o;
+        *reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(P.y) + (size_t)step * d + gcol) = o;
+        if (step + 1 < P.n_steps && (step + 1) % P.chain_len != 0)       // the next step reads this row
+            st_relaxed_gpu_v2(P.ll_x + (size_t)((step + 1) & 1) * (d / 2) + gcol / 2, make_uint2(o, tag));
+    }
+    __syncwarp();
+    if (lane == 0) {
+        // this CTA's words of the next input row are on their way: count the CTA (a hint), free the step's buffers
+        if (step + 1 < P.n_steps && (step + 1) % P.chain_len != 0) red_add_relaxed_gpu(P.counters + (size_t)step * kCounterStride + 32, 1u);
+        mbar_arrive(split_bar(sm, kSplitSlicesFree));
+    }
+    SI_CPROF(7);                                          // column sums, y, next input row
+    return fail;
+}
+
+template <int DT, int NCH, bool kFull>
+__device__ __forceinline__ void split_consumers(const Params &P, uint8_t *smem, Smem *sm) {
+    unsigned ring = 0;
+    bool fail = false;
+    for (int step = 0; step < P.n_steps && !fail; ++step) {
+        fail = split_step_gateup<DT, NCH, kFull>(P, smem, step, ring);
+        if (!fail) fail = split_step_down<DT>(P, smem, step);
+    }
+    if (fail && (threadIdx.x & 31) == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
+}
+
 #undef SI_CPROF
 
 template <int DT, int NCH, bool kFull, int LLR>
@@ -672,11 +1042,12 @@ __device__ __forceinline__ void chained_consumers(const Params &P, uint8_t *smem
 // GRP: float4 column groups a reducer warp covers at once (its 32 lanes = GRP groups x 32/GRP row classes);
 // SETW: warps per consumer set -- 8: two sets of 256 threads; 16: one set of 512 threads (rows too long for
 // two rings and two hand-over buffers: thread t then owns chunks t, t + 512)
-// CH: chained mode (every step reads the output of the step before it; the consumers themselves run the
-// exchanges between the SMs and the reducer warps have nothing to do)
-// LLR (chained): partial rows one consumer thread gathers per step (all in flight at once)
-template <int DT, int NCH, bool kFull, bool kProf, int GRP, int SETW = 8, bool CH = false, int LLR = 5>
-__global__ void __launch_bounds__(CH ? kThreadsChained : kThreads, 1)   // 20 warps: at most 96 registers per thread (chained: 17 warps, 120)
+// CH: 0 = every step's input is given; 1, 2 = chained mode (every step reads the output of the step before it;
+// the consumers themselves run the exchanges between the SMs and there are no reducer warps): 1 = the SMs
+// exchange partial output rows, 2 = the split form that exchanges the activations (two more warps load slices)
+// LLR (CH == 1): partial rows one consumer thread gathers per step (all in flight at once)
+template <int DT, int NCH, bool kFull, bool kProf, int GRP, int SETW = 8, int CH = 0, int LLR = 5>
+__global__ void __launch_bounds__(CH == 0 ? kThreads : (CH == 1 ? kThreadsChained : kThreadsSplit), 1)   // at most 20 warps: 96 registers per thread
 si_decode_persistent_kernel(const __grid_constant__ Params P) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int kSets = 16 / SETW, kSetWarps = SETW, kSetThreads = SETW * 32;   // shadow the two-set defaults
@@ -685,7 +1056,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     const int S = nstage / kSets;              // ring stages per consumer set
     uint8_t *ring = smem;
     float *accbuf = reinterpret_cast<float *>(smem + (size_t)nstage * rec_bytes);   // [set][d_model] hand-over to the reducers
-    Smem *sm = reinterpret_cast<Smem *>(smem + (size_t)nstage * rec_bytes + (size_t)kSets * P.d_model * 4);
+    Smem *sm = reinterpret_cast<Smem *>(smem + P.sm_off);
     uint64_t *full = sm->full, *empty = sm->empty;
     int *meta = sm->meta;
     volatile int *cta_abort = &sm->cta_abort;
@@ -700,17 +1071,25 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     const int Gv = G * kSets;                  // consumer sets act as virtual CTAs 2b, 2b+1 of 2G
     const int d = P.d_model, chunks = P.chunks;
     const long long wait_limit = P.wait_cycles;
-    constexpr bool chained = CH;               // (one step group then: the launch code sees to it)
+    constexpr bool chained = CH != 0;          // (one step group then: the launch code sees to it)
     constexpr int xi = CH ? 0 : 1;             // ring items per step that carry the input row (chained: none, the consumers fetch it)
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSetWarps); }
         for (int q = 0; q < kSets; ++q)
             for (int w = 0; w < kReducerWarps; ++w) { mbar_init(&sm->accfull[q][w], kSetWarps); mbar_init(&sm->accempty[q][w], 1); }
-        if (CH) {     // chained mode has no hand-over to reducers: three of those barriers serve its consumers
+        if (CH == 1) {     // chained mode has no hand-over to reducers: three of those barriers serve its consumers
             mbar_init(&sm->accfull[0][kChainCmb], kSetWarps);               // second set's accumulators parked
             mbar_init(&sm->accfull[0][kChainXch], kConsumerWarps);          // every warp's class sums written
             mbar_init(&sm->accfull[0][kChainRows], 1);                      // the polling thread's news: every CTA's row is written
+        }
+        if (CH == 2) {
+            mbar_init(split_bar(sm, kSplitSlicesFull), 32 * kSplitLoaderWarps);   // every loader lane's copies of the step landed
+            mbar_init(split_bar(sm, kSplitSlicesFree), kConsumerWarps);           // every consumer warp done with the step's buffers
+            mbar_init(split_bar(sm, kSplitH), kConsumerWarps);                    // every warp's share of h in shared memory
+            mbar_init(split_bar(sm, kSplitRed), kConsumerWarps);                  // every warp's partial sums in shared memory
+            mbar_init(split_bar(sm, kSplitHint), 1);                              // the polling thread's news: every set's h is written
+            mbar_init(split_bar(sm, kSplitInput), 1);                             // the same for the next input row
         }
         sm->cta_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -767,7 +1146,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - xi) * Gv);
                         const bool valid = slot >= 0 && slot < P.n_loaded[layer];
                         pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
-                        pf_bytes = valid ? (uint32_t)rec_bytes : 0u; pf_meta = valid ? 1 : 0;
+                        pf_bytes = valid ? P.copy_bytes : 0u; pf_meta = valid ? 1 : 0;
                     }
                 }
             }
@@ -821,7 +1200,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                     meta[st] = (int)dsc.w;
                     if (dsc.z != 0) {
                         mbar_arrive_expect_tx(&full[st], dsc.z);
-                        bulk_g2s(ring + (size_t)st * rec_bytes,
+                        bulk_g2s(ring + (size_t)st * P.stage_bytes,
                                  (const void *)(((unsigned long long)dsc.y << 32) | dsc.x), dsc.z, &full[st], policy);
                     } else {
                         if (P.status) atomicCAS(P.status, 0, SI_ERR_OUT_OF_RANGE);
@@ -844,7 +1223,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 t_last = clock64();
             } else {
                 if (*cta_abort || clock64() - t_last > wait_limit) { ok = false; break; }
-                if (!chained) __nanosleep(100);       // nothing to issue: do not burn issue slots and power
+                __nanosleep(100);       // nothing to issue: do not burn issue slots and power
             }
         }
         if (!ok && lane == 0) raise_abort(P, sm, SI_ERR_TIMEOUT);
@@ -862,9 +1241,14 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
     // Warp w runs on scheduler partition w mod 4.  The service warps (producer 0, reducers 4, 8, 12)
     // share partition 0 with one consumer warp, so that their rarely executed code does not compete
     // with four consumer warps for the partition's instruction cache and issue slots.
-    const bool is_reducer = !CH && (warp & 3) == 0 && warp >= 4 && warp <= 4 * kReducerWarps;
-    if constexpr (CH) {
+    const bool is_reducer = (warp & 3) == 0 && warp >= 4 && warp <= 4 * kReducerWarps;
+    if constexpr (CH == 1) {
         chained_consumers<DT, NCH, kFull, LLR>(P, smem, sm);
+        return;
+    }
+    if constexpr (CH == 2) {
+        if (warp > kConsumerWarps) split_slice_loader(P, smem, sm, warp - kConsumerWarps - 1, lane);
+        else split_consumers<DT, NCH, kFull>(P, smem, sm);
         return;
     }
     if (!is_reducer) {
@@ -873,7 +1257,7 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
         // into registers (3*NCH 16-byte chunks per thread) and its stage handed back at once;
         // the arithmetic then runs out of registers, so the ring is refilled while the set
         // computes.  Thread t of a set owns chunks t, t+256 of every row.
-        const int cw = CH ? warp - 1 : (warp < 16 ? warp - (warp / 4 + 1) : warp - 4);   // consumer warp index 0..15
+        const int cw = warp < 16 ? warp - (warp / 4 + 1) : warp - 4;   // consumer warp index 0..15
         const int ct = cw * 32 + lane;           // 0..511
         const int q = ct / kSetThreads;          // consumer set
         const int t = ct & (kSetThreads - 1);    // thread within the set
@@ -1221,15 +1605,18 @@ inline size_t si_persistent_partial_bytes(const si_store *s) {
     return (size_t)si_persist::kPartialDepth * s->num_sms * s->d_model * 4;
 }
 
-template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8, bool CH = false, int LLR = 5>
-inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream, size_t extra_smem = 0) {
+// total_smem: dynamic shared memory of the launch when it is not the unchained layout's (0: that layout's)
+template <int DT, int NCH, bool FULL, bool PROF, int GRP, int SETW = 8, int CH = 0, int LLR = 5>
+inline int si_decode_persistent_launch_t(const si_persist::Params &P, int G, cudaStream_t stream, size_t extra_smem = 0,
+                                         size_t total_smem = 0) {
     auto kern = si_persist::si_decode_persistent_kernel<DT, NCH, FULL, PROF, GRP, SETW, CH, LLR>;
-    size_t smem = si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW) + extra_smem;
+    size_t smem = total_smem ? total_smem : si_persist::smem_bytes(P.d_model, P.nstage, 16 / SETW) + extra_smem;
     // the limit is raised to the most any instance needs (setting it is cheap, a host-side call, and
     // keeps no state here that threads or devices could disagree about)
     SI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     void *args[] = {(void *)&P};
-    SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G), dim3(CH ? si_persist::kThreadsChained : si_persist::kThreads),
+    SI_CUDA_TRY(cudaLaunchCooperativeKernel((void *)kern, dim3(G),
+                                            dim3(CH == 0 ? si_persist::kThreads : (CH == 1 ? si_persist::kThreadsChained : si_persist::kThreadsSplit)),
                                             args, smem, stream));
     return SI_OK;
 }
@@ -1247,6 +1634,8 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.n_layers = s->n_layers; P.n_steps = n_steps; P.k_fixed = k_fixed; P.d_model = s->d_model;
     const bool wide = si_persist::wide_rows(s->d_model);
     P.chunks = s->d_model / 8; P.nstage = si_persist::pick_stages(s->d_model, wide ? 1 : 2);
+    P.stage_bytes = P.copy_bytes = (unsigned)s->d_model * 6;
+    P.sbuf_off = P.hbuf_off = P.red_off = P.prev_off = 0; P.k_cap = 0; P.ll_h = nullptr;
     P.step_layers = nullptr; P.n_few = 0;
     // steps region: [n_steps] layer ids | control words (256 bytes) | [n_steps][64] counters
     int32_t *steps = (int32_t *)(wsb + ws.steps_off);
@@ -1289,7 +1678,40 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.n_groups = ng;
     const int gpc = (s->d_model / 4 + G / ng - 1) / (G / ng);       // column groups per CTA -> lanes of a reducer warp
     SI_CUDA_TRY(cudaMemsetAsync(P.ctrl, 0, 256 + (size_t)n_steps * si_persist::kCounterStride * 4, stream));   // control words + counters
+    P.sm_off = (unsigned)((size_t)P.nstage * s->d_model * 6 + (size_t)(wide ? 1 : 2) * s->d_model * 4);
     P.ll_partial = nullptr; P.ll_x = nullptr; P.csum_off = 0;
+    // chained, split form: fixed-size slices need a CTA to own at most four groups of eight columns, every SM
+    // must take part (a CTA without records still owns columns), and the step's slices must fit shared memory
+    if (ex->chain_len > 0 && ex->chain_form != 1 && !wide && P.chunks <= 2 * si_persist::kSetThreads &&
+        s->d_model / 8 <= 4 * s->num_sms && k_fixed >= 1) {
+        const int Gs = s->num_sms;
+        const int k_cap = (int)si_align_up((size_t)k_fixed, 64);
+        const size_t tail = (size_t)k_cap * 64 + si_align_up((size_t)k_cap * 4, 16) + 4096 + 64 + sizeof(si_persist::Smem) + 64;
+        const size_t budget = 227 * 1024;
+        int nst = tail < budget ? (int)((budget - tail) / ((size_t)s->d_model * 4)) : 0;
+        nst = (nst > si_persist::kMaxStages ? si_persist::kMaxStages : nst) & ~1;
+        if (ex->ring_stages > 0 && 2 * ex->ring_stages <= nst) nst = 2 * ex->ring_stages;
+        const size_t ll_bytes = (size_t)s->d_model * 8 + (size_t)2 * k_cap * 8;       // input-row words, then the h words
+        if (nst >= 4 && k_cap <= si_persist::kSplitKCapMax && ll_bytes <= ws.partial_bytes) {
+            P.nstage = nst; P.stage_bytes = P.copy_bytes = (unsigned)s->d_model * 4; P.k_cap = k_cap;
+            size_t off = (size_t)nst * P.stage_bytes;
+            P.sbuf_off = (unsigned)off; off += (size_t)k_cap * 64;
+            P.hbuf_off = (unsigned)off; off += si_align_up((size_t)k_cap * 4, 16);
+            P.red_off = (unsigned)off; off += 4096;
+            P.prev_off = (unsigned)off; off += 64;
+            P.sm_off = (unsigned)off; off += sizeof(si_persist::Smem) + 64;
+            P.ll_x = (uint2 *)(wsb + ws.partial_off);
+            P.ll_h = P.ll_x + s->d_model;
+            SI_CUDA_TRY(cudaMemsetAsync(P.ll_x, 0, ll_bytes, stream));
+            const bool full_s = P.chunks == ((P.chunks + 255) / 256) * 256;
+#define SI_PLS(DT, N, F) si_decode_persistent_launch_t<DT, N, F, false, 8, 8, 2>(P, Gs, stream, 0, off)
+#define SI_PLS2(DT) (P.chunks <= 256 ? (full_s ? SI_PLS(DT, 1, true) : SI_PLS(DT, 1, false)) : (full_s ? SI_PLS(DT, 2, true) : SI_PLS(DT, 2, false)))
+            return s->dtype == SI_BF16 ? SI_PLS2(SI_BF16) : SI_PLS2(SI_F16);
+#undef SI_PLS2
+#undef SI_PLS
+        }
+        if (ex->chain_form == 2) return SI_ERR_UNSUPPORTED;       // the split form was asked for and does not fit
+    }
     if (ex->chain_len > 0) {
         // chained: two consumer sets only; the tagged exchange words live in the partial-row area and start at zero
         if (wide) return SI_ERR_UNSUPPORTED;
@@ -1310,9 +1732,9 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
         const int set_threads_c = si_persist::kSetThreads;
         const int nch_c = (P.chunks + set_threads_c - 1) / set_threads_c;
         const bool full_c = P.chunks == nch_c * set_threads_c;
-#define SI_PLC(DT, N, F) (rpt <= 2 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, 2>(P, G, stream, extra)   \
-                          : rpt <= 5 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, 5>(P, G, stream, extra) \
-                                     : si_decode_persistent_launch_t<DT, N, F, false, 8, 8, true, si_persist::kLLRows>(P, G, stream, extra))
+#define SI_PLC(DT, N, F) (rpt <= 2 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, 1, 2>(P, G, stream, extra)   \
+                          : rpt <= 5 ? si_decode_persistent_launch_t<DT, N, F, false, 8, 8, 1, 5>(P, G, stream, extra) \
+                                     : si_decode_persistent_launch_t<DT, N, F, false, 8, 8, 1, si_persist::kLLRows>(P, G, stream, extra))
 #define SI_PLC2(DT) (nch_c <= 1 ? (full_c ? SI_PLC(DT, 1, true) : SI_PLC(DT, 1, false))   \
                      : nch_c <= 2 ? (full_c ? SI_PLC(DT, 2, true) : SI_PLC(DT, 2, false)) \
                                   : (full_c ? SI_PLC(DT, 3, true) : SI_PLC(DT, 3, false)))

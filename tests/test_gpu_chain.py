@@ -66,10 +66,12 @@ def _check_steps_fed_with_device_inputs(api, m, y, xn, heads_bits, lists, chain_
         assert_close(so.widen_bits(yb[s], cfg.dtype), ref, f"step {s}")
 
 
+@pytest.mark.parametrize("form", [1, 2])
 @pytest.mark.parametrize("flags_name", ["plain", "residual", "prenorm", "prenorm+residual"])
-def test_c1_chains_match_the_oracle(api, flags_name):
+def test_c1_chains_match_the_oracle(api, flags_name, form):
     """Config-1 model (fp16, one layer used over and over): 6 chains of 3 steps plus a ragged tail of 2, every
-    step checked; and the whole chain against the oracle's own chain (its own rounding between steps)."""
+    step checked; and the whole chain against the oracle's own chain (its own rounding between steps).  Both
+    forms of the chained kernel: the SMs exchange partial output rows (1) or the activations (2)."""
     cfg = wl.CONFIGS["c1"]
     m = LoadedModel(cfg)
     flags = {"plain": 0, "residual": api.SI_FLAG_RESIDUAL, "prenorm": api.SI_FLAG_PRENORM,
@@ -84,7 +86,7 @@ def test_c1_chains_match_the_oracle(api, flags_name):
         heads = so.round_bits(so.widen_bits(heads, cfg.dtype) * 8.0, cfg.dtype)
     lists = wl.zipf_lists(cfg, 0, n_steps, slot_of_rank=m.slot_of_rank[0], first_token=40)
     y, xn, st = _run_chain(api, m, n_steps, chain_len, to_dev(heads, cfg.dtype), torch.from_numpy(lists).cuda(), None, k,
-                           flags, want_xn=True, layers=[0] * n_steps)
+                           flags, want_xn=True, layers=[0] * n_steps, chain_form=form)
     assert st == 0, api.strerror(st)
     _check_steps_fed_with_device_inputs(api, m, y, xn if flags & api.SI_FLAG_PRENORM else None, heads, lists, chain_len,
                                         flags, range(n_steps), lambda s: 0)
@@ -99,11 +101,12 @@ def test_c1_chains_match_the_oracle(api, flags_name):
             assert_close(from_dev(y[s]), so.widen_bits(out[s - s0], cfg.dtype), f"chain {c} step {s} (oracle's own chain)")
     # run-to-run bit stability
     y2, _, st = _run_chain(api, m, n_steps, chain_len, to_dev(heads, cfg.dtype), torch.from_numpy(lists).cuda(), None, k,
-                           flags, layers=[0] * n_steps)
+                           flags, layers=[0] * n_steps, chain_form=form)
     assert st == 0 and torch.equal(y, y2)
 
 
-def test_7b_two_layers_eight_tokens_chained(api):
+@pytest.mark.parametrize("form", [1, 2])
+def test_7b_two_layers_eight_tokens_chained(api, form):
     """Config-2 shape: 8 tokens, each a chain through 2 layers; fixed lists, ragged lists with offsets (one
     of them empty) and one list per layer; plain, residual and pre-norm chains."""
     cfg = wl.CONFIGS["c2"]
@@ -113,7 +116,7 @@ def test_7b_two_layers_eight_tokens_chained(api):
     heads = wl.x_tokens(cfg, 0, tokens, first_token=900)
     fixed = np.stack([wl.zipf_lists(cfg, s % L, 1, first_token=900 + s // L)[0] for s in range(n_steps)])
     g = np.random.default_rng(31)
-    lens = [int(v) for v in g.integers(1, 2 * k, size=n_steps)]
+    lens = [int(v) for v in g.integers(1, (2 * k if form == 1 else 1800), size=n_steps)]
     lens[5] = 0
     ragged = [np.sort(g.permutation(n)[:c]).astype(np.int32) for c in lens]
     off = np.zeros(n_steps + 1, dtype=np.int32)
@@ -130,12 +133,12 @@ def test_7b_two_layers_eight_tokens_chained(api):
          [per_layer[s % L] for s in range(n_steps)]),
     ]
     for name, idx, offsets, kk, flags, lists in cases:
-        y, xn, st = _run_chain(api, m, n_steps, L, hd, idx, offsets, kk, flags, want_xn=True)
+        y, xn, st = _run_chain(api, m, n_steps, L, hd, idx, offsets, kk, flags, want_xn=True, chain_form=form)
         assert st == 0, (name, api.strerror(st))
         _check_steps_fed_with_device_inputs(api, m, y, xn if flags & N else None, heads, lists, L, flags,
                                             range(n_steps), lambda s: s % L)
         # shallower rings change the timing of everything, not the result
-        y2, _, st = _run_chain(api, m, n_steps, L, hd, idx, offsets, kk, flags, ring_stages=2)
+        y2, _, st = _run_chain(api, m, n_steps, L, hd, idx, offsets, kk, flags, ring_stages=2, chain_form=form)
         assert st == 0 and torch.equal(y, y2), name
 
 
