@@ -241,6 +241,24 @@ int si_decode_chain_forward(const si_store_t *store, int n_steps, const int32_t 
                             void *y, void *xn_out, float norm_eps, unsigned flags, void *workspace,
                             size_t ws_bytes, int32_t *status_dev, void *stream);
 
+/* Decode with a static prefix.  Section 5: the static neurons are always computed and the dynamic ones are
+ * chosen per prompt; the static neurons are the base neurons, which come first in the store (slots
+ * 0 .. n_static-1 of every layer).  Every step computes its layer's slots 0 .. n_static-1 and the listed
+ * slots, which must all be >= n_static (a smaller one repeats a static neuron: SI_ERR_DUPLICATE under
+ * SI_FLAG_CHECK); the lists hold the dynamic neurons only, and the static part of a step is streamed
+ * straight from the store's first n_static records without a list entry being read.
+ *   chain_len == 0 : the steps are independent, x is [n_steps, d_model], as si_decode_stack_forward
+ *                    (y_dtype SI_F32 or the store dtype; xn_out and norm_eps unused);
+ *   chain_len  > 0 : chained steps as si_decode_chain_forward (x holds one row per chain, y has the
+ *                    store dtype, SI_FLAG_PRENORM / xn_out / norm_eps apply).
+ * The other arguments are those of the two calls; k_fixed bounds the listed (dynamic) entries of a step
+ * and n_static + k_fixed may not exceed a layer's loaded neurons.  Persistent kernel only
+ * (SI_ERR_UNSUPPORTED for hidden sizes it does not cover). */
+int si_decode_prefix_forward(const si_store_t *store, int n_steps, const int32_t *layers, int n_static, int chain_len,
+                             const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                             void *y, int y_dtype, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                             size_t ws_bytes, int32_t *status_dev, void *stream);
+
 /* Batch-1 selective FFN for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of si_ffn_forward with T = 1.)
  *

@@ -35,7 +35,7 @@ EXPORTS = [
     "si_strerror", "si_last_cuda_error", "si_build_info", "si_store_bytes", "si_store_create", "si_store_free",
     "si_load_neurons", "si_store_slot_to_global", "si_store_global_to_slot", "si_store_records",
     "si_workspace_bytes", "si_select_workspace_bytes", "si_select", "si_ffn_forward",
-    "si_layer_forward", "si_decode_stack_forward", "si_decode_chain_forward", "si_ffn_forward_noalloc", "si_union",
+    "si_layer_forward", "si_decode_stack_forward", "si_decode_chain_forward", "si_decode_prefix_forward", "si_ffn_forward_noalloc", "si_union",
     "si_debug_decode_stack_forward", "si_debug_decode_chain_forward", "si_debug_union_masks", "si_debug_ffn_forward_waits",
     "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
     "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce",
@@ -76,6 +76,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_union.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, sz, vp]
     lib.si_ffn_forward_noalloc.argtypes = [vp, ci, vp, vp, ci, vp, ci, cu, vp, vp]
     lib.si_decode_chain_forward.argtypes = [vp, ci, vp, ci, vp, vp, vp, ci, vp, vp, ctypes.c_float, cu, vp, sz, vp, vp]
+    lib.si_decode_prefix_forward.argtypes = [vp, ci, vp, ci, ci, vp, vp, vp, ci, vp, ci, vp, ctypes.c_float, cu, vp, sz, vp, vp]
     lib.si_debug_decode_stack_forward.argtypes = lib.si_decode_stack_forward.argtypes + [vp]
     lib.si_debug_decode_chain_forward.argtypes = lib.si_decode_chain_forward.argtypes + [vp]
     lib.si_debug_union_masks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, sz, vp]
@@ -341,6 +342,15 @@ def si_decode_chain_forward(handle, n_steps: int, layers, chain_len: int, x, idx
                                         _dp(y), _dp(xn_out), norm_eps, flags, _dp(workspace),
                                         workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)),
            "si_decode_chain_forward")
+
+
+def si_decode_prefix_forward(handle, n_steps: int, layers, n_static: int, chain_len: int, x, idx, idx_offsets, k_fixed: int, y,
+                             xn_out, norm_eps: float, flags: int, workspace, status=None, stream=None) -> None:
+    keep, p = _host_i32(layers)
+    _check(_lib.si_decode_prefix_forward(handle, n_steps, p, n_static, chain_len, _dp(x), _dp(idx), _dp(idx_offsets), k_fixed,
+                                         _dp(y), dtype_code(y.dtype), _dp(xn_out), norm_eps, flags, _dp(workspace),
+                                         workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)),
+           "si_decode_prefix_forward")
 
 
 def si_debug_decode_chain_forward(handle, n_steps: int, layers, chain_len: int, x, idx, idx_offsets, k_fixed: int, y,

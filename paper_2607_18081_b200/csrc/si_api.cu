@@ -134,8 +134,11 @@ static int decode_stack_impl(const si_store_t *store, int n_steps, const int32_t
         if (!store->loaded[l]) return SI_ERR_INVALID_ARG;          // before anything is enqueued
         min_loaded = min_loaded < store->n_loaded[l] ? min_loaded : store->n_loaded[l];
     }
-    if (!idx_offsets && k_fixed > min_loaded) return SI_ERR_OUT_OF_RANGE;
+    const int n_static = ex ? ex->n_static : 0;
+    if (n_static < 0 || n_static > min_loaded) return SI_ERR_OUT_OF_RANGE;
+    if (!idx_offsets && k_fixed > min_loaded - n_static) return SI_ERR_OUT_OF_RANGE;
     if ((flags & SI_FLAG_LIST_PER_LAYER) && idx_offsets) return SI_ERR_INVALID_ARG;   // per-layer lists have one fixed length
+    if (n_static > 0 && !si_persistent_supported(store)) return SI_ERR_UNSUPPORTED;
     if (ex && ex->chain_len > 0) {
         if (y_dtype != store->dtype) return SI_ERR_INVALID_ARG;    // a step's output is the next step's input
         if (!si_persistent_supported(store)) return SI_ERR_UNSUPPORTED;
@@ -154,11 +157,11 @@ static int decode_stack_impl(const si_store_t *store, int n_steps, const int32_t
         }
         if ((flags & SI_FLAG_LIST_PER_LAYER) && !idx_offsets) {     // one list per layer: check list l against layer l
             for (int l = 0; l < store->n_layers; ++l) {
-                rc = si_check_lists_launch_impl(store, 1, l, nullptr, idx + (size_t)l * k_fixed, nullptr, k_fixed, status_dev, stream);
+                rc = si_check_lists_launch_impl(store, 1, l, nullptr, idx + (size_t)l * k_fixed, nullptr, k_fixed, status_dev, stream, n_static);
                 if (rc) return rc;
             }
         } else {
-            rc = si_check_lists_launch_impl(store, n_steps, -1, layers_dev, idx, idx_offsets, k_fixed, status_dev, stream);
+            rc = si_check_lists_launch_impl(store, n_steps, -1, layers_dev, idx, idx_offsets, k_fixed, status_dev, stream, n_static);
             if (rc) return rc;
         }
     }
@@ -198,12 +201,13 @@ extern "C" int si_debug_decode_stack_forward(const si_store_t *store, int n_step
 static int chain_impl(const si_store_t *store, int n_steps, const int32_t *layers, int chain_len, const void *x,
                       const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y, void *xn_out,
                       float norm_eps, unsigned flags, void *workspace, size_t ws_bytes, int32_t *status_dev,
-                      void *stream, const si_debug_decode_opts_t *opts) {
+                      void *stream, const si_debug_decode_opts_t *opts, int n_static = 0) {
     if (chain_len < 1 || !si_store_ok(store)) return SI_ERR_INVALID_ARG;
     if (flags & (SI_FLAG_STEPS_ANY_ORDER | SI_FLAG_SIMPLE_KERNELS)) return SI_ERR_INVALID_ARG;   // neither applies to a chain
     if (opts && (opts->ring_stages < 0 || opts->wait_cycles < 0)) return SI_ERR_INVALID_ARG;
     si_decode_extra ex = extra_of(opts);
     ex.step_groups = 0;
+    ex.n_static = n_static;
     ex.chain_len = chain_len;
     ex.prenorm = (flags & SI_FLAG_PRENORM) != 0;
     ex.norm_eps = norm_eps;
@@ -227,6 +231,23 @@ extern "C" int si_debug_decode_chain_forward(const si_store_t *store, int n_step
                                              const si_debug_decode_opts_t *opts) {
     return chain_impl(store, n_steps, layers, chain_len, x, idx, idx_offsets, k_fixed, y, xn_out, norm_eps, flags, workspace,
                       ws_bytes, status_dev, stream, opts);
+}
+
+extern "C" int si_decode_prefix_forward(const si_store_t *store, int n_steps, const int32_t *layers, int n_static, int chain_len,
+                                        const void *x, const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
+                                        void *y, int y_dtype, void *xn_out, float norm_eps, unsigned flags, void *workspace,
+                                        size_t ws_bytes, int32_t *status_dev, void *stream) {
+    if (n_static < 0 || chain_len < 0) return SI_ERR_INVALID_ARG;
+    if (chain_len > 0) {
+        if (si_store_ok(store) && y_dtype != store->dtype) return SI_ERR_INVALID_ARG;
+        return chain_impl(store, n_steps, layers, chain_len, x, idx, idx_offsets, k_fixed, y, xn_out, norm_eps, flags, workspace,
+                          ws_bytes, status_dev, stream, nullptr, n_static);
+    }
+    if (flags & (SI_FLAG_PRENORM | SI_FLAG_SIMPLE_KERNELS)) return SI_ERR_INVALID_ARG;     // the norm belongs to chains; prefixes to the persistent kernel
+    si_decode_extra ex;
+    ex.n_static = n_static;
+    return decode_stack_impl(store, n_steps, layers, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace, ws_bytes,
+                             status_dev, stream, &ex);
 }
 
 extern "C" int si_debug_ffn_forward_waits(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,

@@ -15,7 +15,7 @@ struct CheckParams {
 
 __global__ void __launch_bounds__(256)
 si_check_lists_kernel(const __grid_constant__ CheckParams P, const int32_t *__restrict__ idx,
-                      const int32_t *__restrict__ offsets, int k_fixed, int32_t *status) {
+                      const int32_t *__restrict__ offsets, int k_fixed, int32_t *status, int min_slot) {
     extern __shared__ unsigned int bitmap[];
     const int list = blockIdx.x;
     int layer = P.layer_fixed >= 0 ? P.layer_fixed
@@ -34,6 +34,7 @@ si_check_lists_kernel(const __grid_constant__ CheckParams P, const int32_t *__re
     for (int p = threadIdx.x; p < k; p += blockDim.x) {
         int s = idx[base + p];
         if (s < 0 || s >= n_loaded) { atomicCAS(status, 0, SI_ERR_OUT_OF_RANGE); continue; }
+        if (s < min_slot) { atomicCAS(status, 0, SI_ERR_DUPLICATE); continue; }     // a slot of the static prefix, which the step computes anyway
         unsigned int bit = 1u << (s & 31);
         unsigned int old = atomicOr(&bitmap[s >> 5], bit);
         if (old & bit) atomicCAS(status, 0, SI_ERR_DUPLICATE);
@@ -44,7 +45,7 @@ si_check_lists_kernel(const __grid_constant__ CheckParams P, const int32_t *__re
 
 int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed, const int32_t *step_layers_dev,
                                const int32_t *idx, const int32_t *idx_offsets, int k_fixed,
-                               int32_t *status_dev, cudaStream_t stream) {
+                               int32_t *status_dev, cudaStream_t stream, int min_slot) {
     if (!status_dev || n_lists <= 0) return SI_OK;
     if (s->n_layers > 128) return SI_ERR_UNSUPPORTED;
     CheckParams P;
@@ -53,7 +54,7 @@ int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed, 
     P.n_layers = s->n_layers; P.layer_fixed = layer_fixed; P.step_layers = step_layers_dev;
     size_t smem = (size_t)((max_loaded + 31) / 32 + 1) * 4;
     if (smem > 48 * 1024) return SI_ERR_UNSUPPORTED;
-    si_check_lists_kernel<<<n_lists, 256, smem, stream>>>(P, idx, idx_offsets, k_fixed, status_dev);
+    si_check_lists_kernel<<<n_lists, 256, smem, stream>>>(P, idx, idx_offsets, k_fixed, status_dev, min_slot);
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;
 }

@@ -73,6 +73,7 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
 // What a decode launch may carry beyond the arguments of si_decode_stack_forward: the chained mode of
 // si_decode_chain_forward and the per-call diagnostics of si_debug_decode_stack_forward.
 struct si_decode_extra {
+    int n_static = 0;              // static prefix (persistent kernel only)
     int chain_len = 0;             // > 0: chained steps (persistent kernel only)
     int chain_form = 0;            // 0: the library's choice; 1: the SMs exchange partial output rows; 2: split form (activations)
     int prenorm = 0;
@@ -121,7 +122,7 @@ int si_prefill_vote_launch(const void *acts, int acts_dtype, int T, int n, int r
 int si_check_lists_launch_impl(const si_store *s, int n_lists, int layer_fixed,
                                const int32_t *step_layers_dev, const int32_t *idx,
                                const int32_t *idx_offsets, int k_fixed, int32_t *status_dev,
-                               cudaStream_t stream);
+                               cudaStream_t stream, int min_slot = 0);
 
 // implemented in si_gemm.cu
 size_t si_gemm_partial_bytes(const si_store *s, int T_max);

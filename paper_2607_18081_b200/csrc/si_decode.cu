@@ -367,8 +367,8 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
     // kernel: a launch of it costs about 33 us beyond its steps, a plain step 12 us against 5.4 us
     // (replayed from a CUDA graph; launched one by one from the host three steps already favour the
     // persistent kernel, whose single launch costs the host less than six)
-    const bool chained = ex && ex->chain_len > 0;
-    if (chained && !si_persistent_supported(s)) return SI_ERR_UNSUPPORTED;    // chains live in the persistent kernel
+    const bool chained = ex && (ex->chain_len > 0 || ex->n_static > 0);
+    if (chained && !si_persistent_supported(s)) return SI_ERR_UNSUPPORTED;    // chains and static prefixes live in the persistent kernel
     const bool use_simple = !chained && ((flags & SI_FLAG_SIMPLE_KERNELS) != 0 || !si_persistent_supported(s) || n_steps <= 2);
     if (!use_simple)
         return si_decode_persistent_launch(s, n_steps, layers_host, x, idx, idx_offsets, k_fixed, y, y_dtype, flags,

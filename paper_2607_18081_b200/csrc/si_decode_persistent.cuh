@@ -85,6 +85,9 @@ struct Params {
     void *y;
     int y_f32, residual;
     int per_layer_lists;          // fixed-length lists only: idx is [n_layers][k_fixed], a step uses the list of its layer
+    int n_static;                 // every step also computes slots 0 .. n_static-1 of its layer (the static neurons, which come
+                                  // first in the store) ahead of its listed entries: positions 0 .. n_static-1 of the step need
+                                  // no list load at all
     int n_groups;                 // step groups: CTA c belongs to group c mod n_groups and, with the other CTAs of its
                                   // group, runs the steps s = group (mod n_groups); 1 = every CTA works on every step
     float *partial;               // [n_groups][D][G][d_model], G = CTAs per group
@@ -326,6 +329,7 @@ __device__ __forceinline__ unsigned long long dot8p(const uint4 &v, const unsign
 }
 
 // Per-step list geometry: which entries of the step's list belong to virtual CTA b of G.
+// (k counts the static prefix and the listed entries; base is where the listed entries start in idx)
 struct StepGeom { int base, k, first, cnt; };
 __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, int b) {
     StepGeom g;
@@ -336,6 +340,7 @@ __device__ __forceinline__ StepGeom step_geom(const Params &P, int step, int G, 
     } else {
         g.base = step * P.k_fixed; g.k = P.k_fixed; before = (long long)step * P.k_fixed;
     }
+    g.k += P.n_static; before += (long long)step * P.n_static;     // the static prefix comes first in every step
     int rot = (int)(before % G);
     g.first = (b - rot + G) % G;
     g.cnt = g.k > g.first ? (g.k - g.first + G - 1) / G : 0;
@@ -748,6 +753,7 @@ __device__ __forceinline__ SplitList split_list(const Params &P, int step) {
     } else {
         l.base = P.per_layer_lists ? l.layer * P.k_fixed : step * P.k_fixed; l.k = P.k_fixed;
     }
+    l.k += P.n_static;
     if (l.k > P.k_cap) l.k = P.k_cap;       // (a longer list is reported by the first half; nothing is read beyond the buffers)
     return l;
 }
@@ -773,7 +779,7 @@ __device__ __forceinline__ void split_slice_loader(const Params &P, uint8_t *sme
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
                 const int p = lw * 32 + lane + j * 32 * kSplitLoaderWarps;
-                slot[j] = p < l.k ? __ldg(P.idx + l.base + p) : -1;
+                slot[j] = p < l.k ? (p < P.n_static ? p : __ldg(P.idx + l.base + (p - P.n_static))) : -1;
             }
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
@@ -1143,7 +1149,8 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                         pf_bytes = (uint32_t)d * 2; pf_meta = g.cnt;
                     } else {
                         const int lbase = P.per_layer_lists ? layer * P.k_fixed : g.base;
-                        const int slot = __ldg(P.idx + lbase + g.first + (long long)(t - xi) * Gv);
+                        const long long pos = g.first + (long long)(t - xi) * Gv;       // position in the step: static prefix, then the list
+                        const int slot = pos < P.n_static ? (int)pos : __ldg(P.idx + lbase + (pos - P.n_static));
                         const bool valid = slot >= 0 && slot < P.n_loaded[layer];
                         pf_src = (unsigned long long)(P.store_base + P.rec_off[layer] + (size_t)(valid ? slot : 0) * rec_bytes);
                         pf_bytes = valid ? P.copy_bytes : 0u; pf_meta = valid ? 1 : 0;
@@ -1651,6 +1658,8 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.x = (const uint16_t *)x; P.idx = idx; P.idx_offsets = idx_offsets; P.y = y;
     P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
     P.per_layer_lists = (flags & SI_FLAG_LIST_PER_LAYER) != 0 && !idx_offsets;
+    P.n_static = ex->n_static;
+    const int k_total = k_fixed + ex->n_static;       // most positions of a step
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
     P.prof = ex->profile;
@@ -1660,7 +1669,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.withhold = ex->withhold;
     P.chain_len = ex->chain_len; P.prenorm = ex->prenorm; P.norm_eps = ex->norm_eps; P.xn_out = (uint16_t *)ex->xn_out;
     int G = s->num_sms;
-    if (!idx_offsets && k_fixed < G) G = k_fixed < 1 ? 1 : k_fixed;
+    if (!idx_offsets && k_total < G) G = k_total < 1 ? 1 : k_total;
     // every CTA reduces at most kMaxGroups float4 column groups
     const int g_min = (s->d_model / 4 + si_persist::kMaxGroups - 1) / si_persist::kMaxGroups;
     if (G < g_min) G = g_min;
@@ -1676,7 +1685,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     int ng = 1;
     if (G == s->num_sms && ex->chain_len == 0) {
         const int forced = ex->step_groups;   // diagnostics: force a group count
-        const int by_length = k_fixed <= 600 ? 4 : (k_fixed <= 1100 ? 2 : 1);
+        const int by_length = k_total <= 600 ? 4 : (k_total <= 1100 ? 2 : 1);
         ng = forced ? forced : ((flags & SI_FLAG_STEPS_ANY_ORDER) ? si_persist::pick_groups(s->num_sms) : by_length);
         while (ng > 1 && (s->num_sms % ng != 0 || n_steps < 2 * ng ||
                           (s->d_model / 4 + s->num_sms / ng - 1) / (s->num_sms / ng) > si_persist::kMaxGroups))
@@ -1690,9 +1699,9 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // chained, split form: fixed-size slices need a CTA to own at most four groups of eight columns, every SM
     // must take part (a CTA without records still owns columns), and the step's slices must fit shared memory
     if (ex->chain_len > 0 && ex->chain_form != 1 && !wide && P.chunks <= 2 * si_persist::kSetThreads &&
-        s->d_model / 8 <= 4 * s->num_sms && k_fixed >= 1) {
+        s->d_model / 8 <= 4 * s->num_sms && k_total >= 1) {
         const int Gs = s->num_sms;
-        const int k_cap = (int)si_align_up((size_t)k_fixed, 64);
+        const int k_cap = (int)si_align_up((size_t)k_total, 64);
         const size_t tail = (size_t)k_cap * 64 + si_align_up((size_t)k_cap * 4, 16) + 4096 + 64 + sizeof(si_persist::Smem) + 64;
         const size_t budget = 227 * 1024;
         int nst = tail < budget ? (int)((budget - tail) / ((size_t)s->d_model * 4)) : 0;
