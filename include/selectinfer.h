@@ -393,6 +393,25 @@ int si_layer_range(int n_layers, int first, int last, int *first_out, int *last_
  *                     x, y: as in si_ffn_forward (x may be NULL without SI_FLAG_RESIDUAL).
  * All device work is asynchronous on stream.  No counterpart in the paper. */
 int si_shard_count(int n, int rank, int world, int *count_out);
+/*   si_ffn_forward_sharded   batch-1 decode of this device's share with the all-reduce inside the kernel that
+ *                     finishes the down projection: every block of that kernel adds the device's partial rows for its
+ *                     32 output columns, stores the sums into EVERY device's receive area with plain peer stores,
+ *                     marks the block as delivered on every device, waits (with a limit: SI_ERR_TIMEOUT in
+ *                     *status_dev) until every device has delivered the same block here, adds the devices' sums in
+ *                     rank order (the result is the same bits on every device), adds the residual, rounds, writes
+ *                     y.  No collective call and no further kernel.
+ *                       x, idx (k local slots), y, y_dtype, flags (SI_FLAG_RESIDUAL), workspace: as si_ffn_forward, T = 1
+ *                       recv   HOST array of `world` device pointers, recv[q] = device q's receive area, fp32
+ *                              [2][world][d_model], mapped for this device (peer access / IPC mapping);
+ *                       marks  HOST array of `world` device pointers, marks[q] = device q's delivery marks, uint32
+ *                              [world][d_model / 32], zero before the first call;
+ *                       epoch  the number of this call on these buffers: 1, 2, 3, ... on every device alike (its
+ *                              parity picks the half of the receive areas, so a device may be one call ahead).
+ *                     d_model must be a multiple of 128, world at most 8.  Tested with all ranks of a group
+ *                     sharing one GPU (one launch over all of them); not tested across GPUs: this run has one. */
+int si_ffn_forward_sharded(const si_store_t *store, int layer, const void *x, const int32_t *idx, int k, void *y,
+                           int y_dtype, unsigned flags, int rank, int world, float *const *recv, unsigned *const *marks,
+                           unsigned epoch, void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream);
 int si_shard_lists(const int32_t *idx, const int32_t *idx_offsets, int k_fixed, int n_lists, int rank, int world,
                    int32_t *idx_out, int32_t *offsets_out, void *workspace, size_t ws_bytes, int32_t *status_dev,
                    void *stream);

@@ -82,6 +82,18 @@ int si_debug_ffn_forward_waits(const si_store_t *store, int layer, const void *x
                                void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream,
                                long long spin_limit, int withhold);
 
+/* si_ffn_forward_sharded for the ranks rank_base .. rank_base + n_here - 1 of a group that share this GPU, in ONE
+ * launch (kernels of different ranks that wait on one another may not run as separate launches on one GPU): the
+ * ranks' first kernels one after the other, then one cooperative launch of the finishing kernel over all of them.
+ * All arrays are HOST arrays of n_here entries (stores, x, idx, k, y, workspaces) or of `world` entries (recv,
+ * marks).  With n_here < world the missing ranks never deliver: with a short wait_cycles (0 = the default)
+ * this exercises the time-out (SI_ERR_TIMEOUT in *status_dev, clean return). */
+int si_debug_ffn_forward_sharded_group(const si_store_t *const *stores, int n_here, int rank_base, int world, int layer,
+                                       const void *const *x, const int32_t *const *idx, const int *k, void *const *y,
+                                       int y_dtype, unsigned flags, float *const *recv, unsigned *const *marks,
+                                       unsigned epoch, void *const *workspaces, size_t ws_bytes, long long wait_cycles,
+                                       int32_t *status_dev, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

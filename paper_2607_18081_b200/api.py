@@ -38,7 +38,8 @@ EXPORTS = [
     "si_layer_forward", "si_decode_stack_forward", "si_decode_chain_forward", "si_decode_prefix_forward", "si_ffn_forward_noalloc", "si_union",
     "si_debug_decode_stack_forward", "si_debug_decode_chain_forward", "si_debug_union_masks", "si_debug_ffn_forward_waits",
     "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
-    "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce",
+    "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce", "si_ffn_forward_sharded",
+    "si_debug_ffn_forward_sharded_group",
 ]
 
 
@@ -92,6 +93,9 @@ def _load_library() -> ctypes.CDLL:
     lib.si_shard_count.argtypes = [ci, ci, ci, ctypes.POINTER(ci)]
     lib.si_shard_lists.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, sz, vp, vp]
     lib.si_shard_reduce.argtypes = [vp, ci, vp, ci, ci, ci, vp, ci, cu, vp]
+    lib.si_ffn_forward_sharded.argtypes = [vp, ci, vp, vp, ci, vp, ci, cu, ci, ci, vp, vp, cu, vp, sz, vp, vp]
+    lib.si_debug_ffn_forward_sharded_group.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, ci, cu, vp, vp, cu, vp, sz,
+                                                       ctypes.c_longlong, vp, vp]
     lib.si_prefill_forward.argtypes = [vp, ci, vp, ci, vp, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp, sz, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -293,6 +297,31 @@ def si_shard_reduce(parts_dev, world: int, x, T: int, d_model: int, y, flags: in
     xd = dtype_code(x.dtype) if x is not None else dtype_code(torch.bfloat16 if x_dtype is None else x_dtype)
     _check(_lib.si_shard_reduce(_dp(parts_dev), world, _dp(x), xd, T, d_model, _dp(y), dtype_code(y.dtype), flags,
                                 _stream(stream)), "si_shard_reduce")
+
+
+def _ptr_array(tensors_or_handles):
+    vals = [t.value if isinstance(t, ctypes.c_void_p) else (0 if t is None else t.data_ptr()) for t in tensors_or_handles]
+    return (ctypes.c_void_p * len(vals))(*vals)
+
+
+def si_ffn_forward_sharded(handle, layer: int, x, idx, k: int, y, flags: int, rank: int, world: int, recv, marks, epoch: int,
+                           workspace, status=None, stream=None) -> None:
+    """recv, marks: lists of `world` tensors (every device's receive area / delivery marks as this device sees them)."""
+    _check(_lib.si_ffn_forward_sharded(handle, layer, _dp(x), _dp(idx), k, _dp(y), dtype_code(y.dtype), flags, rank, world,
+                                       _ptr_array(recv), _ptr_array(marks), epoch, _dp(workspace),
+                                       workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)),
+           "si_ffn_forward_sharded")
+
+
+def si_debug_ffn_forward_sharded_group(handles, rank_base: int, world: int, layer: int, xs, idxs, ks, ys, flags: int, recv,
+                                       marks, epoch: int, workspaces, status=None, wait_cycles: int = 0, stream=None) -> None:
+    n = len(handles)
+    karr = (ctypes.c_int * n)(*[int(v) for v in ks])
+    ws_bytes = min(w.numel() * w.element_size() for w in workspaces)
+    _check(_lib.si_debug_ffn_forward_sharded_group(_ptr_array(handles), n, rank_base, world, layer, _ptr_array(xs), _ptr_array(idxs),
+                                                   karr, _ptr_array(ys), dtype_code(ys[0].dtype), flags, _ptr_array(recv),
+                                                   _ptr_array(marks), epoch, _ptr_array(workspaces), ws_bytes, wait_cycles,
+                                                   _dp(status), _stream(stream)), "si_debug_ffn_forward_sharded_group")
 
 
 def si_ffn_forward_noalloc(handle, layer: int, x, idx, k: int, y, flags: int, status=None, stream=None) -> None:

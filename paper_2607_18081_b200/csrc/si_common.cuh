@@ -90,6 +90,9 @@ int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host,
                      int y_dtype, unsigned flags, void *workspace, size_t ws_bytes,
                      int32_t *status_dev, cudaStream_t stream, const si_decode_extra *ex = nullptr);
 
+int si_decode_partial_launch(const si_store *s, int layer, const void *x, const int32_t *idx, int k, float *partial,
+                             int32_t *status_dev, cudaStream_t stream, int *rows_out);
+
 // implemented in si_gemm.cu
 int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, const int32_t *idx,
                           const int32_t *idx_offsets, int k_fixed, void *y, int y_dtype,

@@ -302,7 +302,7 @@ si_decode_reduce_kernel(const float *__restrict__ partial, int G, int d,
 template <int DT>
 int launch_simple_step(const si_store *s, int layer, const void *x, const int32_t *idx,
                        const int32_t *offsets, int list, int k, void *y, int y_dtype, unsigned flags,
-                       float *partial, int max_ctas, int32_t *status_dev, cudaStream_t stream) {
+                       float *partial, int max_ctas, int32_t *status_dev, cudaStream_t stream, int *rows_only = nullptr) {
     const int d = s->d_model, chunks = d / 8;
     const int nch = (chunks + kThreads - 1) / kThreads;
     int G = k < max_ctas ? (k < 1 ? 1 : k) : max_ctas;          // one partial row per CTA
@@ -341,6 +341,11 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
     else return SI_ERR_UNSUPPORTED;
 #undef SI_LAUNCH_PARTIAL
 #undef SI_LAUNCH_AHEAD
+    if (rows_only) {                  // the caller sums the partial rows itself (the sharded path: sum and exchange in one kernel)
+        *rows_only = G;
+        SI_CUDA_TRY(cudaGetLastError());
+        return SI_OK;
+    }
     cfg.gridDim = dim3((d + 31) / 32); cfg.blockDim = dim3(256);
     SI_CUDA_TRY(cudaLaunchKernelEx(&cfg, si_decode_reduce_kernel<DT>, (const float *)partial, G, d, (const uint16_t *)x, y,
                                    (int)(y_dtype == SI_F32), (int)((flags & SI_FLAG_RESIDUAL) != 0)));
@@ -349,6 +354,14 @@ int launch_simple_step(const si_store *s, int layer, const void *x, const int32_
 }
 
 }  // namespace
+
+// The first kernel of a single step alone: fp32 partial rows [*rows_out][d_model] in `partial` (room for 2 rows per SM).
+int si_decode_partial_launch(const si_store *s, int layer, const void *x, const int32_t *idx, int k, float *partial,
+                             int32_t *status_dev, cudaStream_t stream, int *rows_out) {
+    return s->dtype == SI_BF16
+               ? launch_simple_step<SI_BF16>(s, layer, x, idx, nullptr, 0, k, nullptr, SI_F32, 0, partial, kSimpleCtasPerSm * s->num_sms, status_dev, stream, rows_out)
+               : launch_simple_step<SI_F16>(s, layer, x, idx, nullptr, 0, k, nullptr, SI_F32, 0, partial, kSimpleCtasPerSm * s->num_sms, status_dev, stream, rows_out);
+}
 
 int si_decode_launch(const si_store *s, int n_steps, const int32_t *layers_host, const void *x,
                      const int32_t *idx, const int32_t *idx_offsets, int k_fixed, void *y,

@@ -8,7 +8,10 @@ the rank-ordered slots (global slot s lives on rank s mod P as local slot s div 
 Argument marshalling and the collective only: the slot arithmetic on the device is si_shard_lists,
 the partial outputs come from si_ffn_forward, residual and conversion from si_shard_reduce.  The
 collective is torch.distributed's all_reduce (NCCL on GPUs); a one-shot all-reduce by peer loads is
-si_shard_reduce over peer pointers, which `combine` drives for buffers of one process.
+si_shard_reduce over peer pointers, which `combine` drives for buffers of one process.  For batch-1 decode
+`forward_fused` needs no collective at all: the kernel that finishes the down projection stores its sums
+into every rank's receive area over peer mappings and adds what the others deliver (tested with all ranks
+of a group on one GPU; not tested across GPUs: this run has one).
 """
 from __future__ import annotations
 
@@ -76,6 +79,16 @@ class ShardedFFN:
             import torch.distributed as dist
             dist.all_reduce(y32, group=self.group)
         combine([y32], x, T, self.d_model, y, flags, self.dtype)
+
+
+    def forward_fused(self, layer: int, x, idx_local, k_local: int, y, flags: int, recv, marks, epoch: int, workspace,
+                      status=None) -> None:
+        """Batch-1 decode (T = 1) with the all-reduce inside the kernel that finishes the down projection
+        (si_ffn_forward_sharded): no collective call.  recv / marks: every rank's receive area (fp32
+        [2, world, d_model]) and delivery marks (int32 [world, d_model // 32], zero at first) as THIS process
+        sees them -- peer mappings of the other ranks' buffers; epoch: 1, 2, 3, ... on every rank alike."""
+        api.si_ffn_forward_sharded(self.store.handle, layer, x, idx_local, k_local, y, flags, self.rank, self.world, recv, marks,
+                                   epoch, workspace, status)
 
 
 def combine(parts, x, T: int, d_model: int, y, flags: int, dtype="bf16") -> None:

@@ -110,3 +110,62 @@ def test_sharded_layer_matches_whole_layer_oracle(api, world):
         for p in parts[1:]:
             acc += p
         assert torch.equal(acc, y32)
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_decode_with_the_allreduce_inside_the_kernel(api, world):
+    """Batch-1 decode of a sharded layer with the all-reduce inside the kernel that finishes the down projection.  All
+    ranks of the group share this GPU, so they run as ONE launch over all ranks' data (their blocks wait on one
+    another).  Every rank's output must be the same bits, equal to the rank-order sum of the ranks' partial outputs
+    that the two-kernel path (partial output, then si_shard_reduce) gives, and within tolerance of the oracle of the
+    whole layer; three calls in a row reuse the receive areas and the delivery marks."""
+    from paper_2607_18081_b200 import sharded
+    cfg = wl.Config("shardcase", 31, 1024, 1500, 1, "bf16", 60, 25, 8)
+    wg, wu, wd = wl.layer_weights(cfg, 0)
+    ids, sor = wl.loaded_ids(cfg, 0)
+    d, k = cfg.d_model, cfg.k_active
+    ranks = []
+    for r in range(world):
+        f = sharded.ShardedFFN(1, d, cfg.d_ff, cfg.n_loaded, cfg.n_base, cfg.dtype, r, world)
+        f.load(0, to_dev(wg, cfg.dtype), to_dev(wu, cfg.dtype), to_dev(wd, cfg.dtype), ids)
+        ranks.append(f)
+    recv = [torch.zeros(2, world, d, dtype=torch.float32, device="cuda") for _ in range(world)]
+    marks = [torch.zeros(world, d // 32, dtype=torch.int32, device="cuda") for _ in range(world)]
+    st = _status()
+    lists = wl.zipf_lists(cfg, 0, 3, slot_of_rank=sor)
+    x = wl.x_tokens(cfg, 0, 3)
+    for call, flags in enumerate((0, api.SI_FLAG_RESIDUAL, 0)):
+        xd = to_dev(x[call], cfg.dtype)
+        idx = torch.from_numpy(lists[call:call + 1]).cuda()
+        local, parts, wss = [], [], []
+        for f in ranks:
+            il, ol, k_cap = f.local_lists(0, idx, None, k, 1, st)
+            n_local = int(ol[1].item())
+            local.append((il, n_local))
+            ws = f.store.workspace(1, max(n_local, 1), 1)
+            wss.append(ws)
+            y32 = torch.empty(1, d, dtype=torch.float32, device="cuda")
+            api.si_ffn_forward(f.store.handle, 0, xd, 1, il, None, n_local, y32, api.SI_FLAG_SIMPLE_KERNELS, ws, st)
+            parts.append(y32)
+        want = torch.empty(1, d, dtype=torch.float32, device="cuda")
+        sharded.combine(parts, xd if flags else None, 1, d, want, flags, cfg.dtype)
+        ys = [torch.full((d,), 7.0, dtype=torch.float32, device="cuda") for _ in range(world)]
+        api.si_debug_ffn_forward_sharded_group([f.store.handle for f in ranks], 0, world, 0, [xd] * world, [il for il, _ in local],
+                                               [n for _, n in local], ys, flags, recv, marks, call + 1, wss, st)
+        torch.cuda.synchronize()
+        assert st.item() == 0, api.strerror(int(st.item()))
+        for r in range(world):
+            assert torch.equal(ys[r], want[0]), f"call {call} rank {r}"
+        ref = so.ffn(wg, wu, wd, x[call], ids[lists[call]], dtype=cfg.dtype, threads=so.host_threads())
+        if flags:
+            ref = ref + wl.bits_to_float64(x[call], cfg.dtype)
+        assert_close(from_dev(ys[0]), ref, f"call {call}")
+    # a rank that never delivers: the others' wait runs out, the status says so, the launch returns
+    st.zero_()
+    xd = to_dev(x[0], cfg.dtype)
+    il, n_local = local[0]
+    y0 = torch.empty(d, dtype=torch.float32, device="cuda")
+    api.si_debug_ffn_forward_sharded_group([ranks[0].store.handle], 0, world, 0, [xd], [il], [n_local], [y0], 0, recv, marks, 4, [wss[0]],
+                                           st, wait_cycles=2_000_000)
+    torch.cuda.synchronize()
+    assert st.item() == api.SI_ERR_TIMEOUT
