@@ -21,8 +21,12 @@ si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps)
     size_t gpart = si_gemm_partial_bytes(s, T_max);
     take(w.partial_off, w.partial_bytes, part > gpart ? part : gpart);
     take(w.sel_off, w.sel_bytes, (size_t)T_max * (size_t)(k_max + 1) * 4);
-    take(w.union_off, w.union_bytes, T_max > 1 ? nl_pad * 4 + 256 : 0);   // union, count
-    take(w.mask_off, w.mask_bytes, T_max > 1 ? (t_pad + 1) * (nl_pad / 32) * 4 + si_gemm_counter_bytes(s, nl_pad, t_pad) : 0);   // token slot bitmaps, union bitmap, counters
+    // the union stage's outputs exist twice (w.half_* bytes each): the union of a call is built while the contractions
+    // of the call before it still read theirs
+    w.union_half = T_max > 1 ? si_align_up(nl_pad * 4 + 256, 256) : 0;
+    w.mask_half = T_max > 1 ? si_align_up((t_pad + 1) * (nl_pad / 32) * 4 + si_gemm_counter_bytes(s, nl_pad, t_pad), 256) : 0;
+    take(w.union_off, w.union_bytes, 2 * w.union_half);   // union, count
+    take(w.mask_off, w.mask_bytes, 2 * w.mask_half);      // token slot bitmaps, union bitmap, counters
     take(w.h_off, w.h_bytes, T_max > 1 ? t_pad * nl_pad * 2 : 0);
     take(w.selws_off, w.selws_bytes, (size_t)T_max * si_select_ws_bytes_impl(nl_max));
     take(w.steps_off, w.steps_bytes, si_align_up((size_t)max_steps * 4, 256) + 256 + (size_t)max_steps * 256);   // layer ids, control words, 2 counter lines per step

@@ -6,6 +6,7 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <atomic>
 #include <vector>
 
 #include "selectinfer.h"
@@ -23,6 +24,8 @@ struct si_store {
     std::vector<int> n_loaded, n_base;
     std::vector<char> loaded;              // layer packed at least once
     std::vector<size_t> rec_off, s2g_off, g2s_off;
+    // multi-token calls alternate between the two copies of the union stage's outputs (see si_ws_carve)
+    mutable std::atomic<unsigned> mt_calls{0};
     size_t record_bytes() const { return (size_t)3 * d_model * 2; }
     const uint16_t *records(int l) const { return (const uint16_t *)(mem + rec_off[l]); }
     int32_t *s2g(int l) const { return (int32_t *)(mem + s2g_off[l]); }
@@ -61,8 +64,9 @@ struct si_ws_layout {
     size_t ctrl_off, ctrl_bytes;
     size_t partial_off, partial_bytes;
     size_t sel_off, sel_bytes;         // int32 [T_max][k_max] selected lists + [T_max] counts
-    size_t union_off, union_bytes;     // int32 [n_loaded_max] union + count
-    size_t mask_off, mask_bytes;       // uint32 [T_max + 1][ceil(n_loaded_max / 32)] slot bitmaps, then counters
+    size_t union_off, union_bytes;     // 2 x (int32 [n_loaded_max] union + count)
+    size_t mask_off, mask_bytes;       // 2 x (uint32 [T_max + 1][ceil(n_loaded_max / 32)] slot bitmaps, then counters)
+    size_t union_half, mask_half;      // bytes of one of the two copies
     size_t h_off, h_bytes;             // 16-bit H [T_pad][n_loaded_max padded]
     size_t selws_off, selws_bytes;     // selector scratch
     size_t steps_off, steps_bytes;     // per-step descriptors for stack calls

@@ -226,16 +226,18 @@ si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     // thread t takes the consecutive entries [t * per, (t + 1) * per): a list is ascending, so its entries
     // fall into the same bitmap word several in a row, and the thread collects their bits in a register
     // and updates shared memory once per (list, word) run
-    const int per = (total + 1023) / 1024;                         // <= kUnionSmallBatch (launch condition)
-    const int e_lo = tid * per;
-    int sl[kUnionSmallBatch];
-#pragma unroll
-    for (int j = 0; j < kUnionSmallBatch; ++j) { const int e = e_lo + j; sl[j] = (j < per && e < total) ? idx[e] : -1; }
+    // (longer inputs take several rounds of kUnionSmallBatch entries per thread)
+    const int rounds = (total + 1024 * kUnionSmallBatch - 1) / (1024 * kUnionSmallBatch);
+    const int per = rounds > 1 ? kUnionSmallBatch : (total + 1023) / 1024;
     for (int w = tid; w < zero_words; w += 1024) zero_g[w] = 0u;
     for (int w = tid; w < words; w += 1024) sh[w] = 0u;
     for (int w = tid; w < tok_words; w += 1024) tok_s[w] = 0u;
     __syncthreads();
-    {
+    for (int round = 0; round < (rounds > 0 ? rounds : 1); ++round) {
+        const int e_lo = round * 1024 * kUnionSmallBatch + tid * per;
+        int sl[kUnionSmallBatch];
+#pragma unroll
+        for (int j = 0; j < kUnionSmallBatch; ++j) { const int e = e_lo + j; sl[j] = (j < per && e < total) ? idx[e] : -1; }
         int t = 0, t_end = 0;                                      // list of the current entry, first entry past it
         if (e_lo < total) {
             if (offsets) {            // largest t with offsets[t] <= e_lo
@@ -269,6 +271,11 @@ si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     __syncthreads();
     for (int w = tid; w < tok_words; w += 1024) tokbits[w] = tok_s[w];
     union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
+    // This kernel reads the caller's lists and writes a copy of the union stage's outputs that nothing else is
+    // using, so it may run while the kernel before it in the stream (the down contraction of the call before)
+    // still works.  It ends only after that kernel has: whoever waits for this kernel's results then also sees
+    // everything that kernel wrote (the next gate/up contraction may read, as its x, the y of the call before).
+    pdl_wait();
 }
 
 // ------------------------------------------------------------------------------- contractions
@@ -580,6 +587,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
 
     // The gate/up kernel lets this kernel start only after the union kernel has completed, so the union
     // and the down rows it names can be read at once; only H has to wait for the gate/up kernel.
+    pdl_launch();                               // the union stage of the next call may be scheduled (it writes other buffers)
     const int n_u = *P.n_union;
     const int total_chunks = (n_u + kChunkK - 1) / kChunkK;        // 64 union entries per chunk
     const int k_per = (total_chunks + P.n_split - 1) / P.n_split;
@@ -769,6 +777,18 @@ __global__ void si_gemm_reduce_kernel(const float *__restrict__ partial, int n_s
     else reinterpret_cast<uint16_t *>(y)[(size_t)t * d + j] = si_cvt<DT>::from_float(a);
 }
 
+// Any kernel as a programmatic dependent of its predecessor in the stream.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // Launch a contraction kernel so that it may be scheduled while the previous kernel of the stream is
 // still finishing (the kernel itself waits for that kernel's results with pdl_wait()).
 cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap), dim3 grid, size_t smem, cudaStream_t stream,
@@ -827,11 +847,11 @@ int pick_stages_gemm(size_t stage_bytes, int n_tok) {
 // Zero-on-entry scratch of a multi-token call, carved from the workspace's mask region:
 // [T][mask_words] token slot bitmaps | [mask_words] union bitmap | counters (ticket, tile counters)
 struct UnionScratch { uint32_t *tokbits, *bitmap; unsigned *ticket, *ctr; size_t zero_bytes; int mask_words; };
-UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws, int T, int n_loaded, int n_ctr) {
+UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws, int T, int n_loaded, int n_ctr, int half = 0) {
     (void)s;
     UnionScratch u;
     u.mask_words = (int)(si_align_up((size_t)n_loaded, 128) / 32);
-    u.tokbits = (uint32_t *)(wsb + ws.mask_off);
+    u.tokbits = (uint32_t *)(wsb + ws.mask_off + (size_t)half * ws.mask_half);
     u.bitmap = u.tokbits + (size_t)T * u.mask_words;
     u.ticket = (unsigned *)(u.bitmap + u.mask_words);
     u.ctr = u.ticket + 64;
@@ -839,6 +859,9 @@ UnionScratch union_scratch(const si_store *s, char *wsb, const si_ws_layout &ws,
     return u;
 }
 constexpr long long kUnionSmallEntries = 16 * 1024;     // up to here one block builds the union faster than several
+constexpr long long kUnionOverlapEntries = 64 * 1024;   // up to here one block builds it while the call before still runs: its
+                                                        // time is hidden, and the several-block kernel (whose bitmaps a memset
+                                                        // must clear first, in stream order) cannot run early
 constexpr size_t kUnionSmallSmem = 160 * 1024;          // shared memory the one-block union may use
 int union_blocks(const si_store *s, long long entries) {
     // one entry per thread while the blocks fit the machine at once: an entry is a chain of dependent
@@ -889,22 +912,27 @@ int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, con
 // several blocks with global atomics otherwise.
 static int union_stage_launch(const si_store *s, int n_loaded, int n_lists, bool own_lists, const int32_t *idx,
                               const int32_t *idx_offsets, int k_fixed, const UnionScratch &us, int32_t *uni,
-                              int32_t *n_union, int nu_pad, int32_t *status_dev, cudaStream_t stream) {
+                              int32_t *n_union, int nu_pad, int32_t *status_dev, cudaStream_t stream, bool may_overlap = false) {
     const int words = (n_loaded + 31) / 32;
     // token bitmaps are only read (and so only cleared) when the tokens have lists of their own
     char *z0 = own_lists ? (char *)us.tokbits : (char *)us.bitmap;
     const size_t zero_bytes = us.zero_bytes - (size_t)(z0 - (char *)us.tokbits);
     const long long entries = idx_offsets ? (long long)n_lists * n_loaded : (long long)n_lists * k_fixed;
     const size_t small_smem = ((size_t)2 * words + 2 + (own_lists ? (size_t)n_lists * us.mask_words : 0)) * 4;
-    if (entries <= kUnionSmallEntries && small_smem <= kUnionSmallSmem) {
+    if (entries <= (may_overlap ? kUnionOverlapEntries : kUnionSmallEntries) && small_smem <= kUnionSmallSmem) {
         // few entries, few lists: one block does everything in shared memory, the clearing of the
         // counters included
         SI_CUDA_TRY(cudaFuncSetAttribute(si_union_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUnionSmallSmem));
         uint32_t *zc = (uint32_t *)us.ticket;                          // ticket words and the arrival counters
         const size_t zc_bytes = us.zero_bytes - (size_t)((char *)us.ticket - (char *)us.tokbits);
-        si_union_small_kernel<<<1, 1024, small_smem, stream>>>(
-            idx, idx_offsets, k_fixed, n_lists, n_loaded, zc, (int)(zc_bytes / 4),
-            own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
+        if (may_overlap)      // as a programmatic dependent: it may start while the contraction before it still runs
+            SI_CUDA_TRY(launch_pdl(si_union_small_kernel, dim3(1), dim3(1024), small_smem, stream, idx, idx_offsets, k_fixed, n_lists,
+                                   n_loaded, zc, (int)(zc_bytes / 4), own_lists ? us.tokbits : (uint32_t *)nullptr, us.mask_words, uni,
+                                   n_union, nu_pad, status_dev));
+        else
+            si_union_small_kernel<<<1, 1024, small_smem, stream>>>(
+                idx, idx_offsets, k_fixed, n_lists, n_loaded, zc, (int)(zc_bytes / 4),
+                own_lists ? us.tokbits : nullptr, us.mask_words, uni, n_union, nu_pad, status_dev);
     } else {
         SI_CUDA_TRY(cudaMemsetAsync(z0, 0, zero_bytes, stream));
         si_union_build_kernel<<<union_blocks(s, entries), 1024, (size_t)(2 * words + 2) * 4, stream>>>(
@@ -929,7 +957,7 @@ int si_union_masks_launch(const si_store *s, int layer, int T, const int32_t *id
     if (cap > n_loaded) cap = n_loaded;
     const int nu_pad = (int)si_align_up((size_t)cap, 128);
     UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, 0);
-    if (us.zero_bytes > ws.mask_bytes) return SI_ERR_NOMEM;
+    if (us.zero_bytes > ws.mask_half) return SI_ERR_NOMEM;
     int rc = union_stage_launch(s, n_loaded, T, true, idx, idx_offsets, k_fixed, us, uni, n_union, nu_pad, nullptr, stream);
     if (rc) return rc;
     SI_CUDA_TRY(cudaMemcpyAsync(union_out, uni, (size_t)n_loaded * 4, cudaMemcpyDeviceToDevice, stream));
@@ -960,9 +988,10 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
         SI_CUDA_TRY(cudaGetLastError());
         return SI_OK;
     }
-    // ---- union
+    // ---- union (this call's copy of the union stage's outputs: the other copy may still be read by the call before)
+    const int half = (int)(s->mt_calls.fetch_add(1u, std::memory_order_relaxed) & 1u);
     const size_t nl_pad = si_align_up((size_t)n_loaded, 128);
-    int32_t *uni = (int32_t *)(wsb + ws.union_off);
+    int32_t *uni = (int32_t *)(wsb + ws.union_off + (size_t)half * ws.union_half);
     int32_t *n_union = uni + nl_pad;                       // one int32 (64 reserved)
     // host-known upper bound of the union size sizes the grids
     long long cap = shared ? (long long)k_fixed : (idx_offsets ? (long long)n_loaded : (long long)T * k_fixed);
@@ -977,11 +1006,11 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     const int tok_tiles = (t_pad_total + tile_n - 1) / tile_n;
     const bool own_lists = !shared && !(flags & SI_FLAG_UNION_UNMASKED);   // membership differs per token
     const int n_ctr_gu = m_tiles * tok_tiles, n_ctr_dn = (d / 128) * tok_tiles;
-    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn);
-    if (us.zero_bytes > ws.mask_bytes) return SI_ERR_NOMEM;
+    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn, half);
+    if (us.zero_bytes > ws.mask_half) return SI_ERR_NOMEM;
     {
         int rc = union_stage_launch(s, n_loaded, shared ? 1 : T, own_lists, idx, idx_offsets, k_fixed, us, uni, n_union,
-                                    nu_pad, status_dev, stream);
+                                    nu_pad, status_dev, stream, true);
         if (rc) return rc;
     }
     // ---- tiling
