@@ -327,3 +327,33 @@ def test_host_side_argument_errors(api, c1):
     assert status_of(lambda: api.si_ffn_forward(h, 0, xd[1:], 1, idx, None, 4, y[1:], 0, ws)) == api.SI_ERR_ALIGNMENT
     yh = torch.empty(cfg.d_model, dtype=torch.bfloat16, device="cuda")     # store is fp16
     assert status_of(lambda: api.si_ffn_forward(h, 0, xd, 1, idx, None, 4, yh, 0, ws)) == api.SI_ERR_INVALID_ARG
+
+
+def test_unloaded_layer_is_refused_before_anything_runs(api):
+    """A layer that was never loaded is refused on the host before anything is enqueued (single call, selector
+    call, stack call)."""
+    cfg = _tiny_cfg()
+    store = api.NeuronStore(2, cfg.d_model, cfg.d_ff, [cfg.n_loaded] * 2, cfg.dtype)
+    wg, wu, wd = wl.layer_weights(cfg, 0)
+    ids, _ = wl.loaded_ids(cfg, 0)
+    store.load(0, to_dev(wg, cfg.dtype), to_dev(wu, cfg.dtype), to_dev(wd, cfg.dtype), ids, cfg.n_base)   # layer 1 stays unloaded
+    n = cfg.n_loaded
+    xd = to_dev(wl.x_tokens(cfg, 0, 4), cfg.dtype)
+    y = torch.full((4, cfg.d_model), 5.0, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(16, dtype=torch.int32, device="cuda")
+    scores = torch.zeros(n, dtype=torch.float32, device="cuda")
+    ws = store.workspace(1, n, 4)
+    st = _status()
+
+    def status_of(fn):
+        with pytest.raises(api.SelectInferError) as e:
+            fn()
+        return e.value.status
+
+    assert status_of(lambda: api.si_ffn_forward(store.handle, 1, xd[0], 1, idx, None, 4, y[0], 0, ws, st)) == api.SI_ERR_INVALID_ARG
+    assert status_of(lambda: api.si_layer_forward(store.handle, 1, xd[0], 1, scores, 4, None, None, y[0], 0, ws, st)) == api.SI_ERR_INVALID_ARG
+    assert status_of(lambda: api.si_decode_stack_forward(store.handle, 4, [0, 0, 1, 0], xd, idx, None, 4, y, api.SI_FLAG_CHECK, ws, st)) \
+        == api.SI_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert st.item() == 0 and bool((y == 5.0).all())                  # nothing ran
+    store.close()
