@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libselectinfer.so")
-SOURCES = ["si_store.cu", "si_decode.cu", "si_select.cu", "si_check.cu", "si_gemm.cu", "si_vote.cu", "si_profile.cu", "si_shard.cu", "si_api.cu"]
+SOURCES = ["si_store.cu", "si_decode.cu", "si_select.cu", "si_check.cu", "si_gemm.cu", "si_gemm_pair.cu", "si_vote.cu", "si_profile.cu", "si_shard.cu", "si_api.cu"]
 
 
 def _nvcc() -> str:

@@ -19,104 +19,16 @@
 // machine.  The finishing passes (combine, split reduction) have no kernels of their own: an
 // unsplit tile is finished in the contraction's epilogue, a split tile by the CTA that delivers
 // its last fp32 partial, which sums the partials in split order -- so results are deterministic.
-#include <cuda.h>       // CUtensorMap and the encode function's signature only; the function is looked up at run time
+#include "si_tc.cuh"
 
-#include "si_common.cuh"
+using namespace si_tc;
 
 namespace {
 
-constexpr int kLoaderThreads = 256;              // warps 0..7: gather loads, later the epilogue
-constexpr int kLoaderWarps = kLoaderThreads / 32;
-constexpr int kGemmThreads = kLoaderThreads + 32; // warp 8: MMA issue + tensor-memory allocation
-constexpr int kMaxStages = 6;
-constexpr int kChunkK = 64;                      // K elements per pipeline stage (128 bytes per row)
-constexpr long long kSpinLimit = 1ll << 24;      // default limit of every wait, in mbarrier probes
-constexpr size_t kPartialCap = (size_t)64 << 20; // bytes of fp32 partial tiles per contraction
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false after `limit` unsuccessful probes.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit) {
-    for (long long i = 0; i < limit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
-}
-// Arrival that fires by itself once all cp.async copies this thread has issued so far have landed: the
-// loader never blocks on its own copies, so every stage can be in flight and the producer side is
-// decoupled from the consumer (counts as one of the barrier's expected arrivals).
-__device__ __forceinline__ void cp_async_arrive_when_landed(uint64_t *bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
-// while its predecessor in the stream still runs; pdl_wait() returns once the predecessor has
-// finished and its writes are visible, pdl_launch() lets the successor start being scheduled.  Both
-// are no-ops in launches without the attribute.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// TMA: one 2-D tile of a dense 16-bit matrix (box = 64 columns x box rows, 128-byte swizzle) into shared
-// memory; x = first column (a multiple of 64, i.e. of 128 bytes), y = first row; rows past the matrix
-// read as zero.  Completion is counted in bytes on the mbarrier.
-__device__ __forceinline__ void tma_load_tile(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(smem_u32(dst_smem)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte
-// offsets in 16-byte units, descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint32_t lo = ((smem_addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
-    uint32_t hi = ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
-    return ((uint64_t)hi << 32) | lo;
-}
-// Instruction descriptor for kind::f16: fp32 accumulate, A/B format (0 f16, 1 bf16), majors.
-__device__ __forceinline__ uint32_t make_idesc(int fmt, int a_mn_major, int b_mn_major, int M, int N) {
-    return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | ((uint32_t)a_mn_major << 15) |
-           ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 // ------------------------------------------------------------------------------- union
 // sh[0 .. words) holds the bitmap; sh[words .. 2*words + 2) is scratch.  Writes the ascending union, its
-// size, and pads the list up to union_cap with its first entry (padded positions contribute nothing).
-__device__ __forceinline__ void union_scan_emit(uint32_t *sh, uint32_t *warp_tot, int words, int32_t *__restrict__ union_out,
+// size, and pads the list up to union_cap with valid slots.
+__device__ __forceinline__ void union_scan_emit(uint32_t *sh, uint32_t *warp_tot, int words, int n_loaded, int32_t *__restrict__ union_out,
                                                 int32_t *__restrict__ n_union_out, int union_cap) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t *bitmap = sh;                         // [words]
@@ -152,9 +64,16 @@ __device__ __forceinline__ void union_scan_emit(uint32_t *sh, uint32_t *warp_tot
         }
     }
     {
-        int first = 0;
+        // Padding.  The slots that follow the last entry, as long as they exist: a union that is a run of consecutive
+        // slots (a static prefix, a whole layer) stays one over its padding, and tiles of consecutive slots are fetched
+        // by tensor copies.  Past the last loaded slot: the first entry.  (Padded positions contribute nothing.)
+        int first = 0, last = 0;
         for (int w = 0; w < words; ++w) if (bitmap[w]) { first = w * 32 + __ffs(bitmap[w]) - 1; break; }
-        for (int p = n_u + tid; p < union_cap; p += 1024) union_out[p] = first;
+        for (int w = words - 1; w >= 0; --w) if (bitmap[w]) { last = w * 32 + 31 - __clz(bitmap[w]); break; }
+        for (int p = n_u + tid; p < union_cap; p += 1024) {
+            const int v = last + 1 + (p - n_u);
+            union_out[p] = v < n_loaded ? v : first;
+        }
     }
 }
 
@@ -201,7 +120,7 @@ si_union_build_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     const int words = (n_loaded + 31) / 32;
     for (int w = tid; w < words; w += 1024) sh[w] = __ldcg(bitmap_g + w);
     __syncthreads();
-    union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
+    union_scan_emit(sh, warp_tot, words, n_loaded, union_out, n_union_out, union_cap);
 }
 
 // The same result from one block, for calls with few list entries and few lists: the union's bitmap and
@@ -270,7 +189,7 @@ si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
     }
     __syncthreads();
     for (int w = tid; w < tok_words; w += 1024) tokbits[w] = tok_s[w];
-    union_scan_emit(sh, warp_tot, words, union_out, n_union_out, union_cap);
+    union_scan_emit(sh, warp_tot, words, n_loaded, union_out, n_union_out, union_cap);
     // This kernel reads the caller's lists and writes a copy of the union stage's outputs that nothing else is
     // using, so it may run while the kernel before it in the stream (the down contraction of the call before)
     // still works.  It ends only after that kernel has: whoever waits for this kernel's results then also sees
@@ -279,33 +198,6 @@ si_union_small_kernel(const int32_t *__restrict__ idx, const int32_t *__restrict
 }
 
 // ------------------------------------------------------------------------------- contractions
-struct GemmParams {
-    const char *rec_base;          // records of the layer
-    int rec_bytes, d_model, chunks;
-    const int32_t *union_slots;    // padded union (device)
-    const int32_t *n_union;        // device
-    int nu_pad;                    // padded union size the grids were sized for
-    const uint16_t *x;             // [T, d_model]
-    int T, n_tok;                  // tokens, N of the MMA (multiple of 16, <= 256)
-    const uint16_t *h;             // [t_pad_total][nu_pad] (down)
-    int t_pad_total;
-    float *partial;                // gate/up: [S][2][nu_pad][t_pad_total]; down: [S][t_pad_total][d_model]
-    int n_split;                   // K splits
-    int fmt;                       // 0 f16, 1 bf16
-    int nstage;
-    int32_t *status;
-    // fused finishing passes: the CTA that completes a tile's last K split sums the splits
-    int tok_tiles, target_ctas;    // gate/up: token tiles; CTAs that can be resident at once
-    unsigned *tile_ctr;            // per (tile, token tile) arrival counters, zero on entry
-    const uint32_t *tokbits;       // [T][mask_words] slot bitmaps of the tokens' own lists, or nullptr: all tokens
-    int mask_words;                //   use the whole union
-    uint16_t *h_out;               // gate/up: H [t_pad_total][nu_pad]
-    void *y;                       // down: output [T][d_model]
-    int y_f32, residual;
-    long long spin_limit;          // probes after which a wait gives up (SI_ERR_TIMEOUT)
-    int withhold;                  // diagnostics: the first gate/up CTA never loads the X tile of its first chunk
-};
-
 // Gate/up contraction.  One CTA per (union tile of 128, K split of d_model, token tile), flat grid.
 // D_gate[128 neurons x N tokens] (+)= Wg[U tile, k] . X[tokens, k]^T, same for up, accumulated in
 // tensor memory (columns [0,N) gate, [N,2N) up).
@@ -813,30 +705,6 @@ cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap, CUten
     return cudaLaunchKernelEx(&cfg, kern, P, m0, m1);
 }
 
-// Tensor map of a dense row-major 16-bit matrix [rows][cols] for tiles of box_rows x 64 columns with the
-// 128-byte swizzle the MMA descriptors expect.  base must be 16-byte aligned, row_bytes a multiple of 16.
-int make_tile_map(CUtensorMap *map, const void *base, size_t cols, size_t rows, size_t row_bytes, int box_rows) {
-    typedef CUresult (*encode_fn_t)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-    static encode_fn_t encode = nullptr;
-    if (!encode) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        SI_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-        if (!fn || q != cudaDriverEntryPointSuccess) return SI_ERR_CUDA;
-        encode = (encode_fn_t)fn;
-    }
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)kChunkK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? SI_OK : SI_ERR_CUDA;
-}
-
 int pick_stages_gemm(size_t stage_bytes, int n_tok) {
     // few tokens: the kernels are latency-bound gathers, two CTAs per SM hide more of it
     size_t budget = n_tok <= 16 ? 112 * 1024 : 200 * 1024;
@@ -1029,6 +897,9 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.h_out = (uint16_t *)(wsb + ws.h_off);
     P.y = y; P.y_f32 = y_dtype == SI_F32; P.residual = (flags & SI_FLAG_RESIDUAL) != 0;
     P.spin_limit = spin_limit > 0 ? spin_limit : kSpinLimit; P.withhold = withhold;
+    P.pair_n = 0;
+    if (si_pair_path_applies(s, T))
+        return si_pair_contractions_launch(s, P, n_loaded, wsb + ws.h_off, ws.h_bytes, stream);
     // gate/up: K = d_model may be split up to s1 ways (what the partial buffer holds); the kernel
     // picks the split from the real union size so that one wave of CTAs covers the SM slots (two CTAs
     // per SM with few tokens: the gathers are latency-bound)

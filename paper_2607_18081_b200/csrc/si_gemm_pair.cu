@@ -1,0 +1,512 @@
+// Prefill contractions on pairs of SMs (more than 128 tokens in a call).
+//
+// With hundreds of tokens the two contractions of a multi-token call are bound by how fast an SM can fill
+// its shared memory, not by HBM: a 128 x 128 tile needs 48 KB of operands for 512 tensor-pipe cycles.  Here a
+// thread-block cluster of two CTAs works on one tile with tcgen05.mma.cta_group::2 (M = 256: the tokens, 128
+// per CTA; N = 256 or 128 store columns, each CTA holding half of them in its shared memory), so every CTA
+// loads its own 128 tokens and only HALF of the weight tile the pair multiplies them with:
+//
+//   gate/up   D[256 tokens x (128 gate | 128 up)] = X[tokens, k] . W[U tile, k]^T     (K = d_model)
+//             CTA 0 of the pair loads the tile's gate rows, CTA 1 its up rows; a thread of the epilogue owns
+//             one token and finds gate and up of a neuron in its own registers: H = member . SiLU(g) . u
+//   down      D[256 tokens x N columns] = H[tokens, U_k] . Wd[U_k, columns]           (K = |U|)
+//             CTA r loads columns r * N/2 .. of the 64 down rows of a chunk (MN-major operand)
+//
+// No K split and no partial tiles: H and y are written straight from tensor memory.  Each CTA tracks the
+// stages of its own shared memory with local mbarriers, exactly as the one-CTA kernels do; the pair is coupled
+// by two signals only: the second CTA's MMA warp relays "my half of stage s has landed" to a barrier of the
+// first (the one that issues the MMAs), and the commit that frees a stage (or declares the accumulators
+// complete) arrives on the barriers of both.  All waits are bounded; both CTAs stay until a last cluster
+// barrier, so neither is signalled after it has gone.
+#include "si_tc.cuh"
+
+using namespace si_tc;
+
+namespace {
+
+constexpr int kPairMaxStages = 8;
+constexpr int kPairTokens = 256;                 // tokens of a pair's tile (M of the MMA), 128 per CTA
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// wait on a barrier that a thread of the other CTA arrives on (cluster-scope acquire); bounded like mbar_wait
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, long long limit) {
+    for (long long i = 0; i < limit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// D[256 x N] (+)= A . B over the pair: A rows and B rows of either CTA are read from its own shared memory at
+// the descriptors' offsets; issued by one thread of the pair's first CTA
+__device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the barrier at this offset in BOTH CTAs once the MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+
+// One pipeline stage of the pair's MMA thread as a single instruction sequence: probe the NEXT stage's barrier,
+// issue this stage's four MMAs (K = 16 each), commit them to this stage's "empty" barriers of both CTAs, and only
+// then read the probe's answer.  A probe takes a couple of hundred cycles to answer; issued first, it is answered
+// while the MMAs are being issued instead of ahead of them.  Returns whether the next stage had already landed.
+__device__ __forceinline__ bool pair_issue_stage(uint32_t d_tmem, const uint64_t (&a)[4], const uint64_t (&b)[4], uint32_t idesc,
+                                                 uint32_t accumulate_first, uint64_t *empty_bar, uint64_t *next_full, uint32_t next_parity) {
+    uint32_t landed;
+    asm volatile(
+        "{\n\t.reg .pred q, p, t;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 q, [%12], %13;\n\t"
+        "setp.ne.b32 p, %10, 0;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %6, %11, p;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %3, %7, %11, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %4, %8, %11, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %5, %9, %11, t;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%14], %15;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(landed)
+        : "r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(accumulate_first),
+          "r"(idesc), "r"(smem_u32(next_full)), "r"(next_parity), "r"(smem_u32(empty_bar)), "h"((uint16_t)3)
+        : "memory");
+    return landed != 0;
+}
+
+struct PairBars {
+    // stage landed.  In the pair's first CTA one arrival more is expected: the second CTA's word that ITS half has landed
+    uint64_t full_t[kPairMaxStages];     // ... tensor copies only (one arrival: the thread that starts them)
+    uint64_t full_g[kPairMaxStages];     // ... gathered rows + the dense tile (all loader threads + 1)
+    uint64_t empty[kPairMaxStages];      // the MMAs have read the stage (both CTAs are told)
+    uint64_t accbar;                     // accumulators complete (both CTAs are told)
+    uint32_t tmem_slot;
+    int failed;
+};
+
+// set-up common to both kernels: barriers, tensor memory of the pair, cluster barrier.  Returns the tensor-memory base.
+__device__ __forceinline__ uint32_t pair_setup(PairBars *B, int nstage, uint32_t ncols, uint32_t rank) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        const uint32_t from_peer = rank == 0 ? 1u : 0u;
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(&B->full_t[s], 1 + from_peer); mbar_init(&B->full_g[s], kLoaderThreads + 1 + from_peer);
+            mbar_init(&B->empty[s], 1);
+        }
+        mbar_init(&B->accbar, 1);
+        B->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kLoaderWarps) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_slot)), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                  // the other CTA's barriers exist before anything is signalled across
+    tc_fence_after();
+    return *reinterpret_cast<volatile uint32_t *>(&B->tmem_slot);
+}
+
+__device__ __forceinline__ void pair_teardown(uint32_t tmem, uint32_t ncols) {
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                  // nobody reads this CTA's shared or tensor memory any more, nobody signals it
+    if ((threadIdx.x >> 5) == kLoaderWarps)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
+}
+
+// The MMA warp's loop.  First CTA: wait until both halves of a stage have landed (its own copies and the second
+// CTA's word arrive on the same barrier), issue, free the stage in both CTAs.  Second CTA: pass the completion of
+// its own stage barrier on to the first CTA's.  `gathered`: the stage holds rows written by cp.async (generic
+// proxy), which need a proxy fence before the MMAs read them.  descs(c, st, a, b) fills in the operand
+// descriptors of the stage's four MMAs.
+template <typename DescFn>
+__device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool gathered, int n_chunks, int nstage, long long limit,
+                                              uint32_t rank, uint32_t tmem, uint32_t idesc, DescFn descs) {
+    volatile int *failed = &B->failed;
+    bool ok = true;
+    if (rank == 0) {
+        bool landed = false;                   // the probe for this chunk's stage was already answered "yes"
+        int st = 0; uint32_t ph = 0;
+        for (int c = 0; c < n_chunks; ++c) {
+            if (!landed) ok = mbar_wait_cluster(&full[st], ph, limit);
+            if (!ok) break;
+            if (gathered) fence_async_proxy();
+            tc_fence_after();
+            uint64_t a[4], b[4];
+            descs(c, st, a, b);
+            int st1 = st + 1; uint32_t ph1 = ph;
+            if (st1 == nstage) { st1 = 0; ph1 ^= 1u; }
+            // (after the last chunk the probe looks at a stage that nothing refills: it answers "no" and is not used)
+            landed = pair_issue_stage(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[st1], ph1);
+            st = st1; ph = ph1;
+        }
+        if (!ok) *failed = 1;
+        umma_commit_pair(&B->accbar);          // accumulators complete (or nothing was issued): told to both CTAs
+    } else {
+        const uint32_t remote0 = map_to_cta(smem_u32(&full[0]), 0);
+        for (int c = 0; c < n_chunks; ++c) {
+            const int st = c % nstage; const uint32_t ph = (c / nstage) & 1;
+            ok = mbar_wait(&full[st], ph, limit);
+            if (!ok) break;
+            if (gathered) fence_async_proxy();   // this CTA's gathered rows are visible to the MMAs before the first CTA is told
+            mbar_arrive_remote(remote0 + (uint32_t)st * 8u);
+        }
+        if (!ok) *failed = 1;
+    }
+}
+
+// Gate/up contraction: one pair per (union tile of 128 neurons, 256 tokens).
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map,
+                      const __grid_constant__ CUtensorMap rec_map) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    constexpr int stage_bytes = 2 * 128 * 128;                    // this CTA's X tile, this CTA's 128 weight rows
+    uint8_t *tiles = smem;
+    PairBars *B = reinterpret_cast<PairBars *>(smem + (size_t)P.nstage * stage_bytes);
+    volatile int *failed = &B->failed;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    constexpr uint32_t ncols = 256;                               // 128 gate + 128 up accumulator columns
+    const uint32_t tmem = pair_setup(B, P.nstage, ncols, rank);
+
+    pdl_wait();                                 // the union kernel's results
+    pdl_launch();
+    const int pair = blockIdx.x >> 1;
+    const int n_tiles = P.nu_pad / 128;
+    const int nt = pair % n_tiles, tp = pair / n_tiles;
+    const int n_u = *P.n_union;
+    const bool active = nt * 128 < n_u;          // tiles past the real union have nothing to do
+    const int n_chunks = active ? P.d_model / kChunkK : 0;
+    const int tok0 = tp * kPairTokens + (int)rank * 128;          // this CTA's tokens
+    // a tile of 128 consecutive slots needs no gather: its rows are one tensor copy out of the record matrix
+    const int slot_first = P.union_slots[nt * 128];
+    const bool run = P.union_slots[nt * 128 + 127] - slot_first == 127;
+    uint64_t *full = run ? B->full_t : B->full_g;
+    const bool withhold = P.withhold && blockIdx.x == 0;
+
+    if (warp < kLoaderWarps) {
+        int armed = 0;                       // (a thread that starts tensor copies) 1 + the last chunk whose copies it has started
+        if (run) {
+            // two threads (of different warps) start the copies of alternate chunks: one thread's round of probe,
+            // expect and two tensor copies takes longer than the MMAs of a chunk
+            if (lane == 0 && warp < 2) {
+                for (int c = warp; c < n_chunks; c += 2) {
+                    const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
+                    if (!mbar_wait(&B->empty[st], ph ^ 1, P.spin_limit)) { *failed = 1; break; }
+                    if (withhold && c == 0) continue;
+                    uint8_t *stage = tiles + (size_t)st * stage_bytes;
+                    armed = c + 1;
+                    mbar_arrive_expect_tx(&full[st], (uint32_t)stage_bytes);
+                    tma_load_tile(stage, &x_map, c * kChunkK, tok0, &full[st]);
+                    tma_load_tile(stage + 128 * 128, &rec_map, (int)rank * P.d_model + c * kChunkK, slot_first, &full[st]);
+                }
+            }
+        } else {
+            // copy j of a thread covers 16-byte piece (tid & 7) of tile row 32*j + (tid >> 3): a warp instruction
+            // reads four whole 128-byte row segments
+            const int q8 = tid & 7, r32 = tid >> 3;
+            const char *wrow[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                wrow[j] = P.rec_base + (size_t)P.union_slots[nt * 128 + 32 * j + r32] * P.rec_bytes + (size_t)rank * P.d_model * 2 + q8 * 16;
+            const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);
+            for (int c = 0; c < n_chunks; ++c) {
+                const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
+                if (!mbar_wait_relaxed(&B->empty[st], ph ^ 1, P.spin_limit, 32)) { *failed = 1; break; }
+                uint8_t *stage = tiles + (size_t)st * stage_bytes;
+                uint8_t *sw = stage + 128 * 128 + off0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { cp_async16(sw + j * 4096, wrow[j]); wrow[j] += 128; }
+                if (tid == 0 && !(withhold && c == 0)) {
+                    armed = c + 1;
+                    mbar_arrive_expect_tx(&full[st], 128u * 128u);
+                    tma_load_tile(stage, &x_map, c * kChunkK, tok0, &full[st]);
+                }
+                cp_async_arrive_when_landed(&full[st]);
+            }
+            cp_async_wait_all();             // nothing of this thread may still be in flight when the CTA ends
+        }
+        // ---------------------------------------------------------------- epilogue
+        bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
+        if (!ok && armed > 0)                // a wait ran out: the tensor copies this thread started must still land before the CTA goes
+            for (int c = armed - 1; c >= 0 && c > armed - 1 - P.nstage; c -= run ? 2 : 1)
+                mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
+        tc_fence_after();
+        if (ok && active) {
+            // thread = token (tensor-memory lane); warps w and w + 4 share the lanes and take 64 neurons each
+            const int q = warp & 3, half = warp >> 2;
+            const int t = tok0 + q * 32 + lane;
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+            uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + (size_t)nt * 128 + 64 * half;
+            const uint32_t *tb = P.tokbits && t < P.T ? P.tokbits + (size_t)t * P.mask_words : nullptr;
+            for (int n0 = 0; n0 < 64; n0 += 16) {
+                uint32_t g[16], u[16];
+                tmem_ld16(trow + (uint32_t)(64 * half + n0), g);
+                tmem_ld16(trow + (uint32_t)(128 + 64 * half + n0), u);
+                uint32_t w[8];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int i = nt * 128 + 64 * half + n0 + j;
+                    bool keep = t < P.T && i < n_u;
+                    if (keep && tb) { const int slot = P.union_slots[i]; keep = (tb[slot >> 5] >> (slot & 31)) & 1u; }
+                    const float out = keep ? si_silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j])) : 0.f;
+                    const uint32_t b = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
+                    if (j & 1) w[j >> 1] |= b << 16; else w[j >> 1] = b;
+                }
+                *reinterpret_cast<uint4 *>(hrow + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(hrow + n0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+        }
+        if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
+    } else if (lane == 0) {
+        const uint32_t idesc = make_idesc(P.fmt, 0, 0, 256, 256);
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, [&](int, int st, uint64_t (&a)[4], uint64_t (&b)[4]) {
+            const uint32_t sx = smem_u32(tiles + (size_t)st * stage_bytes), sw = sx + 128 * 128;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) { a[k4] = make_desc(sx + k4 * 32, 16, 1024); b[k4] = make_desc(sw + k4 * 32, 16, 1024); }
+        });
+    }
+    pair_teardown(tmem, ncols);
+}
+
+// y for this CTA's 128 tokens x N columns, straight from tensor memory (residual added, rounded to the output type).
+template <int N>
+__device__ __forceinline__ void down_epilogue(const GemmParams &P, bool ok, int n_chunks, uint32_t tmem, int warp, int lane, int tok0, int ct) {
+    constexpr int kHalfCols = N / 2;
+    if (!ok) return;
+    // thread = token; warps w and w + 4 share the lanes and take half of the tile's columns each
+    const int q = warp & 3, half = warp >> 2;
+    const int t = tok0 + q * 32 + lane;
+    const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+    const size_t o0 = (size_t)t * P.d_model + (size_t)ct * N + half * kHalfCols;
+    for (int n0 = 0; n0 < kHalfCols; n0 += 16) {
+        uint32_t v[16];
+        if (n_chunks > 0) tmem_ld16(trow + (uint32_t)(half * kHalfCols + n0), v);
+        if (t >= P.T) continue;
+        float a[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) a[j] = n_chunks > 0 ? __uint_as_float(v[j]) : 0.f;
+        if (P.residual) {
+            const uint4 x0 = *reinterpret_cast<const uint4 *>(P.x + o0 + n0), x1 = *reinterpret_cast<const uint4 *>(P.x + o0 + n0 + 8);
+            const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                a[2 * j] += P.fmt ? si_cvt<SI_BF16>::lo(xw[j]) : si_cvt<SI_F16>::lo(xw[j]);
+                a[2 * j + 1] += P.fmt ? si_cvt<SI_BF16>::hi(xw[j]) : si_cvt<SI_F16>::hi(xw[j]);
+            }
+        }
+        if (P.y_f32) {
+            float4 *yo = reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + o0 + n0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) yo[j] = make_float4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+        } else {
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                w[j] = P.fmt ? ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j + 1]) << 16))
+                             : ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j + 1]) << 16));
+            uint4 *yo = reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(P.y) + o0 + n0);
+            yo[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            yo[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+    }
+}
+
+// Down contraction: one pair per (N output columns, 256 tokens); N = P.pair_n (128 or 256), half of them per CTA.
+template <int N>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap h_map,
+                    const __grid_constant__ CUtensorMap rec_map) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    constexpr int kHalfCols = N / 2;                              // output columns whose down rows this CTA loads
+    constexpr int kWBytes = 64 * kHalfCols * 2;                   // 64 union entries x kHalfCols columns
+    constexpr int stage_bytes = 128 * 128 + kWBytes;              // this CTA's H tile, its half of the down rows
+    constexpr int kCopies = kWBytes / 16 / kLoaderThreads;        // 16-byte copies per loader thread and chunk (2 or 4)
+    uint8_t *tiles = smem;
+    PairBars *B = reinterpret_cast<PairBars *>(smem + (size_t)P.nstage * stage_bytes);
+    volatile int *failed = &B->failed;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    constexpr uint32_t ncols = N;
+    const uint32_t tmem = pair_setup(B, P.nstage, ncols, rank);
+
+    pdl_wait();                                 // H (and, through the gate/up kernel's own wait, the union)
+    pdl_launch();
+    const int pair = blockIdx.x >> 1;
+    const int col_tiles = P.d_model / N;
+    const int ct = pair % col_tiles, tp = pair / col_tiles;
+    const int n_u = *P.n_union;
+    const int n_chunks = (n_u + kChunkK - 1) / kChunkK;           // 64 union entries per chunk
+    const int tok0 = tp * kPairTokens + (int)rank * 128;
+    // a union that is one run of consecutive slots (a static prefix, a whole layer) needs no gather: the down rows of
+    // a chunk are tensor copies out of the record matrix (64 slots x 64 columns each)
+    const int slot_first = P.union_slots[0];
+    const bool run = n_chunks > 0 && P.union_slots[n_chunks * kChunkK - 1] - slot_first == n_chunks * kChunkK - 1;
+    uint64_t *full = run ? B->full_t : B->full_g;
+
+    if (warp < kLoaderWarps && run) {
+        int armed = 0;
+        if (lane == 0 && warp < 2) {         // two threads start the copies of alternate chunks
+            const int col0 = 2 * P.d_model + ct * N + (int)rank * kHalfCols;
+            for (int c = warp; c < n_chunks; c += 2) {
+                const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
+                if (!mbar_wait(&B->empty[st], ph ^ 1, P.spin_limit)) { *failed = 1; break; }
+                uint8_t *stage = tiles + (size_t)st * stage_bytes;
+                armed = c + 1;
+                mbar_arrive_expect_tx(&full[st], (uint32_t)stage_bytes);
+                tma_load_tile(stage, &h_map, c * kChunkK, tok0, &full[st]);
+#pragma unroll
+                for (int hh = 0; hh < kHalfCols / 64; ++hh)
+                    tma_load_tile(stage + 128 * 128 + hh * 8192, &rec_map, col0 + hh * 64, slot_first + c * kChunkK, &full[st]);
+            }
+        }
+        bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
+        if (!ok && armed > 0)                // a wait ran out: the tensor copies this thread started must still land before the CTA goes
+            for (int c = armed - 1; c >= 0 && c > armed - 1 - P.nstage; c -= 2)
+                mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
+        tc_fence_after();
+        down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
+        if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
+    } else if (warp < kLoaderWarps) {
+        // Copy j of a thread covers 16-byte piece `pc` of the down-row segment of chunk entry kk = kEntStep*j + e.
+        // Entry kk, 64-column half hh, piece p land at hh*8192 + (kk >> 3)*1024 + (kk & 7)*128 + ((p ^ (kk & 7)) << 4):
+        // the MN-major layout with 128-byte swizzle (8 entries x 64 columns per 1024-byte atom).
+        constexpr int kPieces = kHalfCols * 2 / 16;               // 16-byte pieces per entry segment (8 or 16)
+        constexpr int kEntStep = kLoaderThreads / kPieces;        // entries covered by one copy of all threads (32 or 16)
+        const int pc = tid % kPieces, e = tid / kPieces;
+        const int k8 = e & 7;
+        const int dst0 = (pc >> 3) * 8192 + (e >> 3) * 1024 + k8 * 128 + (((pc & 7) ^ k8) << 4);
+        const char *src0 = P.rec_base + (size_t)P.d_model * 4 + ((size_t)ct * N + (size_t)rank * kHalfCols) * 2 + pc * 16;
+        int armed = 0;
+        int slots_next[kCopies];                                   // union slots of the next chunk (fetched one chunk ahead)
+#pragma unroll
+        for (int j = 0; j < kCopies; ++j) slots_next[j] = n_chunks > 0 ? P.union_slots[kEntStep * j + e] : 0;
+        for (int c = 0; c < n_chunks; ++c) {
+            const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
+            int slots[kCopies];
+#pragma unroll
+            for (int j = 0; j < kCopies; ++j) {                     // padded entries carry a valid slot
+                slots[j] = slots_next[j];
+                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c + 1) * kChunkK + kEntStep * j + e];
+            }
+            if (!mbar_wait_relaxed(&B->empty[st], ph ^ 1, P.spin_limit, 32)) { *failed = 1; break; }
+            uint8_t *stage = tiles + (size_t)st * stage_bytes;
+#pragma unroll
+            for (int j = 0; j < kCopies; ++j)
+                cp_async16(stage + 128 * 128 + dst0 + j * (kEntStep / 8) * 1024, src0 + (size_t)slots[j] * P.rec_bytes);
+            if (tid == 0) {
+                armed = c + 1;
+                mbar_arrive_expect_tx(&full[st], 128u * 128u);
+                tma_load_tile(stage, &h_map, c * kChunkK, tok0, &full[st]);
+            }
+            cp_async_arrive_when_landed(&full[st]);
+        }
+        cp_async_wait_all();
+        bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
+        if (!ok && armed > 0)                // a wait ran out: the tensor copies already started must still land before the CTA goes
+            for (int c = armed - 1; c >= 0 && c > armed - 1 - P.nstage; --c)
+                mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
+        tc_fence_after();
+        down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
+        if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
+    } else if (lane == 0) {
+        const uint32_t idesc = make_idesc(P.fmt, 0, 1, 256, N);
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, [&](int, int st, uint64_t (&a)[4], uint64_t (&b)[4]) {
+            const uint32_t sh = smem_u32(tiles + (size_t)st * stage_bytes), sw = sh + 128 * 128;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {   // 16 union entries per MMA = two 8-entry groups of 1024 bytes
+                a[k4] = make_desc(sh + k4 * 32, 16, 1024); b[k4] = make_desc(sw + k4 * 2048, 8192, 1024);
+            }
+        });
+    }
+    pair_teardown(tmem, ncols);
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pair(void (*kern)(KArgs...), int pairs, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+int stages_for(size_t stage_bytes) {
+    int n = (int)(((size_t)227 * 1024 - sizeof(PairBars) - 1024) / stage_bytes);
+    return n > kPairMaxStages ? kPairMaxStages : n;
+}
+
+}  // namespace
+
+bool si_pair_path_applies(const si_store *s, int T) {
+    return T > 128 && s->d_model % 256 == 0;
+}
+
+// Both contractions of a call with more than 128 tokens, after the union stage (P holds the call's parameters;
+// h_buf has room for t_pad_alloc x nu_pad 16-bit values).
+int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, void *h_buf, size_t h_bytes, cudaStream_t stream) {
+    const int d = P.d_model;
+    const int tok_pairs = (P.T + kPairTokens - 1) / kPairTokens;
+    const int t_pad_alloc = tok_pairs * kPairTokens;
+    if ((size_t)t_pad_alloc * P.nu_pad * 2 > h_bytes) return SI_ERR_NOMEM;
+    P.t_pad_total = t_pad_alloc; P.n_tok = kPairTokens; P.n_split = 1;
+    P.h = (const uint16_t *)h_buf; P.h_out = (uint16_t *)h_buf;
+    {
+        const size_t stage = 2 * 128 * 128;
+        P.nstage = stages_for(stage);
+        const size_t smem = (size_t)P.nstage * stage + sizeof(PairBars);
+        SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CUtensorMap x_map, rec_map;
+        int rc = make_tile_map(&x_map, P.x, (size_t)d, (size_t)P.T, (size_t)d * 2, 128);
+        if (rc) return rc;
+        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 128);
+        if (rc) return rc;
+        SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel, (P.nu_pad / 128) * tok_pairs, smem, stream, P, x_map, rec_map));
+    }
+    {
+        // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs: take 256 only when that
+        // still puts a pair on most SM pairs
+        const int n = (d / 256) * tok_pairs * 2 >= s->num_sms * 3 / 4 ? 256 : 128;
+        P.pair_n = n;
+        const size_t stage = 128 * 128 + (size_t)64 * n;
+        P.nstage = stages_for(stage);
+        const size_t smem = (size_t)P.nstage * stage + sizeof(PairBars);
+        CUtensorMap h_map, rec_map;
+        int rc = make_tile_map(&h_map, h_buf, (size_t)P.nu_pad, (size_t)t_pad_alloc, (size_t)P.nu_pad * 2, 128);
+        if (rc) return rc;
+        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 64);
+        if (rc) return rc;
+        if (n == 256) {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256>, (d / 256) * tok_pairs, smem, stream, P, h_map, rec_map));
+        } else {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<128>, (d / 128) * tok_pairs, smem, stream, P, h_map, rec_map));
+        }
+    }
+    SI_CUDA_TRY(cudaGetLastError());
+    return SI_OK;
+}

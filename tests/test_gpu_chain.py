@@ -229,26 +229,35 @@ def test_decode_wait_runs_out_and_the_next_call_is_correct(api, chained):
         assert_close(from_dev(y32[t]), m.oracle_y(0, x[t], lists[t]), f"after the time-out, step {t}")
 
 
-def test_contraction_wait_runs_out_and_the_next_call_is_correct(api):
+@pytest.mark.parametrize("T,prefix", [(8, False), (200, False), (200, True)])
+def test_contraction_wait_runs_out_and_the_next_call_is_correct(api, T, prefix):
     """The same for the tensor-core path: one operand tile of the first gate/up CTA is never loaded, its
     MMA-issuing thread gives up after a few thousand probes, the kernels record SI_ERR_TIMEOUT, give their
-    tensor memory back and return; the next call on the same workspace is correct."""
+    tensor memory back and return; the next call on the same workspace is correct.  8 tokens: the one-CTA
+    kernels; 200 tokens: the CTA-pair kernels, with gathered weight rows (own lists) and with weight tiles
+    fetched by tensor copies (a shared prefix list) -- there the CTA that issues the pair's MMAs gives up,
+    tells both CTAs so, and the pair leaves together."""
     cfg = wl.CONFIGS["c1"]
     m = LoadedModel(cfg)
-    T, k = 8, cfg.k_active
-    lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=m.slot_of_rank[0])
+    k = cfg.k_active
+    if prefix:
+        lists = np.tile(np.arange(k, dtype=np.int32), (T, 1))
+        flat, flags = lists[0].copy(), api.SI_FLAG_SHARED_LIST
+    else:
+        lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=m.slot_of_rank[0])
+        flat, flags = lists, api.SI_FLAG_UNION_PATH
     x = wl.x_tokens(cfg, 0, T)
-    xd, idx = to_dev(x, cfg.dtype), torch.from_numpy(lists).cuda()
+    xd, idx = to_dev(x, cfg.dtype), torch.from_numpy(np.ascontiguousarray(flat)).cuda()
     ws = m.store.workspace(T, k, 1)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     y = torch.empty(T, cfg.d_model, dtype=torch.float32, device="cuda")
-    api.si_debug_ffn_forward_waits(m.store.handle, 0, xd, T, idx, None, k, y, api.SI_FLAG_UNION_PATH, ws, st,
+    api.si_debug_ffn_forward_waits(m.store.handle, 0, xd, T, idx, None, k, y, flags, ws, st,
                                    spin_limit=20_000, withhold=1)
     torch.cuda.synchronize()
     assert st.item() == api.SI_ERR_TIMEOUT
     st.zero_()
-    api.si_ffn_forward(m.store.handle, 0, xd, T, idx, None, k, y, api.SI_FLAG_UNION_PATH, ws, st)
+    api.si_ffn_forward(m.store.handle, 0, xd, T, idx, None, k, y, flags, ws, st)
     torch.cuda.synchronize()
     assert st.item() == 0
-    for t in range(T):
+    for t in sorted({0, 1, T // 2, T - 1}):
         assert_close(from_dev(y[t]), m.oracle_y(0, x[t], lists[t]), f"after the time-out, token {t}")

@@ -164,8 +164,9 @@ def test_7b_prefill_shared_list(api, m7b):
 
 
 def test_7b_many_tokens_own_lists_residual(api, m7b):
-    """300 tokens with lists of their own: two 256-wide token tiles, the union covers nearly the whole
-    loaded set, the down contraction is split along K and finished by the last-arriving CTA."""
+    """300 tokens with lists of their own (more than 128 tokens: the contractions run on CTA pairs, 256 tokens
+    per pair): the union covers nearly the whole loaded set, every token keeps to its own list through its
+    slot bitmap, the second token tile is ragged."""
     cfg = m7b.cfg
     T, k = 300, cfg.k_active
     lists = wl.zipf_lists(cfg, 0, T)
@@ -178,7 +179,8 @@ def test_7b_many_tokens_own_lists_residual(api, m7b):
 
 @pytest.mark.parametrize("T", [130, 200])
 def test_c1_many_tokens_narrow_token_tiles(api, c1, T):
-    """More than 128 tokens over a small layer: 128-wide token tiles, ragged lists, padded last tile."""
+    """More than 128 tokens over a small layer (CTA pairs, one ragged tile of 256 tokens): ragged lists with an
+    empty one, then a shared list of scattered slots (gathered weight rows), fp16 output."""
     cfg = c1.cfg
     n = cfg.n_loaded
     g = np.random.default_rng(100 + T)
@@ -195,3 +197,32 @@ def test_c1_many_tokens_narrow_token_tiles(api, c1, T):
     y = _run(api, c1, 0, x, shared, None, len(shared), T, flags=api.SI_FLAG_SHARED_LIST, y_dtype=torch.float16)
     for t in (0, 127, 128, T - 1):
         assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], shared), f"shared list, T={T} token {t}")
+
+
+def test_many_tokens_degenerate_unions(api, c1, m7b):
+    """Calls with more than 128 tokens whose union is tiny, empty, or a prefix that ends inside a tile."""
+    cfg = c1.cfg
+    n = cfg.n_loaded
+    T = 256
+    x = wl.x_tokens(cfg, 0, T, first_token=3)
+    # five scattered slots shared by all tokens: one active weight tile, one K chunk of the down contraction
+    shared = np.array([1, 17, 18, 400, n - 1], np.int32)
+    y = _run(api, c1, 0, x, shared, None, len(shared), T, flags=api.SI_FLAG_SHARED_LIST)
+    for t in (0, 100, 128, 255):
+        assert_close(from_dev(y[t]), c1.oracle_y(0, x[t], shared), f"five shared slots, token {t}")
+    # every list empty: y = x exactly (residual), y = 0 without it
+    T = 200
+    off = np.zeros(T + 1, np.int32)
+    y = _run(api, c1, 0, x[:T], np.zeros(4, np.int32), off, n, T, flags=api.SI_FLAG_RESIDUAL)
+    assert np.array_equal(from_dev(y), wl.bits_to_float64(x[:T], cfg.dtype))
+    y = _run(api, c1, 0, x[:T], np.zeros(4, np.int32), off, n, T)
+    assert not from_dev(y).any()
+    # 129 tokens (the second CTA of the pair holds one token) over a prefix of 1000 slots of a 7B-shaped layer:
+    # seven whole tiles fetched by tensor copies and a last tile of 104 real entries
+    cfg7 = m7b.cfg
+    T, k = 129, 1000
+    x7 = wl.x_tokens(cfg7, 0, T, first_token=900)
+    prefix = np.arange(k, dtype=np.int32)
+    y = _run(api, m7b, 0, x7, prefix, None, k, T, flags=api.SI_FLAG_SHARED_LIST, y_dtype=torch.bfloat16)
+    for t in (0, 127, 128):
+        assert_close(from_dev(y[t]), m7b.oracle_y(0, x7[t], prefix), f"129 tokens, token {t}")
