@@ -25,6 +25,7 @@ using namespace si_tc;
 namespace {
 
 constexpr int kPairMaxStages = 8;
+constexpr int kPrefetchAhead = 16;               // chunks between a weight tile's L2 prefetch and its copy into shared memory
 constexpr int kPairTokens = 256;                 // tokens of a pair's tile (M of the MMA), 128 per CTA
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -93,6 +94,41 @@ __device__ __forceinline__ bool pair_issue_stage(uint32_t d_tmem, const uint64_t
     return landed != 0;
 }
 
+// Two stages in one sequence: the probes of the two stages after them come first and are read last, so that they
+// have the time of eight MMAs to be answered (under load a probe takes several hundred cycles -- more than the four
+// MMAs of one stage when these are narrow).  bit 0 / 1 of the result: stage c + 2 / c + 3 had already landed.
+__device__ __forceinline__ uint32_t pair_issue_two_stages(uint32_t d_tmem, const uint64_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc,
+                                                          uint32_t accumulate_first, uint64_t *empty0, uint64_t *empty1,
+                                                          uint64_t *next_full0, uint32_t next_parity0, uint64_t *next_full1, uint32_t next_parity1) {
+    uint32_t landed;
+    asm volatile(
+        "{\n\t.reg .pred q0, q1, p, t;\n\t.reg .b32 r0, r1;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 q0, [%20], %21;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 q1, [%22], %23;\n\t"
+        "setp.ne.b32 p, %18, 0;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %10, %19, p;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %3, %11, %19, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %4, %12, %19, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %5, %13, %19, t;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%24], %26;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %6, %14, %19, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %7, %15, %19, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %8, %16, %19, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %9, %17, %19, t;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%25], %26;\n\t"
+        "selp.u32 r0, 1, 0, q0;\n\t"
+        "selp.u32 r1, 2, 0, q1;\n\t"
+        "or.b32 %0, r0, r1;\n\t}"
+        : "=r"(landed)
+        : "r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
+          "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7]),
+          "r"(accumulate_first), "r"(idesc), "r"(smem_u32(next_full0)), "r"(next_parity0), "r"(smem_u32(next_full1)), "r"(next_parity1),
+          "r"(smem_u32(empty0)), "r"(smem_u32(empty1)), "h"((uint16_t)3)
+        : "memory");
+    return landed;
+}
+
 struct PairBars {
     // stage landed.  In the pair's first CTA one arrival more is expected: the second CTA's word that ITS half has landed
     uint64_t full_t[kPairMaxStages];     // ... tensor copies only (one arrival: the thread that starts them)
@@ -138,28 +174,47 @@ __device__ __forceinline__ void pair_teardown(uint32_t tmem, uint32_t ncols) {
 // The MMA warp's loop.  First CTA: wait until both halves of a stage have landed (its own copies and the second
 // CTA's word arrive on the same barrier), issue, free the stage in both CTAs.  Second CTA: pass the completion of
 // its own stage barrier on to the first CTA's.  `gathered`: the stage holds rows written by cp.async (generic
-// proxy), which need a proxy fence before the MMAs read them.  descs(c, st, a, b) fills in the operand
-// descriptors of the stage's four MMAs.
-template <typename DescFn>
+// proxy), which need a proxy fence before the MMAs read them.  a0 / b0: the operand descriptors of the four MMAs
+// of stage 0; those of stage s follow by adding s * stage_bytes to the address field.  The MMAs of a stage are
+// issued back to back with as little as possible in between: an MMA instruction is not handed over before the
+// one ahead of it is nearly done, so whatever the thread does between two stages the tensor pipe waits for.
 __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool gathered, int n_chunks, int nstage, long long limit,
-                                              uint32_t rank, uint32_t tmem, uint32_t idesc, DescFn descs) {
+                                              uint32_t rank, uint32_t tmem, uint32_t idesc, const uint64_t (&a0)[4], const uint64_t (&b0)[4],
+                                              uint32_t stage_bytes) {
     volatile int *failed = &B->failed;
     bool ok = true;
     if (rank == 0) {
-        bool landed = false;                   // the probe for this chunk's stage was already answered "yes"
+        // stages are issued two at a time; `landed` bit 0 / 1: the probe of the first / second of the two was answered "yes"
+        uint32_t landed = 0;
         int st = 0; uint32_t ph = 0;
-        for (int c = 0; c < n_chunks; ++c) {
-            if (!landed) ok = mbar_wait_cluster(&full[st], ph, limit);
+        const uint64_t step = (uint64_t)(stage_bytes >> 4);     // (the address field holds bytes / 16 and never overflows: shared memory is < 256 KB)
+        auto next = [&](int &s_, uint32_t &p_) { if (++s_ == nstage) { s_ = 0; p_ ^= 1u; } };
+        int c = 0;
+        for (; c + 1 < n_chunks; c += 2) {
+            int s1 = st; uint32_t p1 = ph; next(s1, p1);
+            if (!(landed & 1u)) ok = mbar_wait_cluster(&full[st], ph, limit);
+            if (ok && !(landed & 2u)) ok = mbar_wait_cluster(&full[s1], p1, limit);
             if (!ok) break;
-            if (gathered) fence_async_proxy();
-            tc_fence_after();
-            uint64_t a[4], b[4];
-            descs(c, st, a, b);
-            int st1 = st + 1; uint32_t ph1 = ph;
-            if (st1 == nstage) { st1 = 0; ph1 ^= 1u; }
-            // (after the last chunk the probe looks at a stage that nothing refills: it answers "no" and is not used)
-            landed = pair_issue_stage(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[st1], ph1);
-            st = st1; ph = ph1;
+            if (gathered) { fence_async_proxy(); tc_fence_after(); }
+            const uint64_t o0 = step * (uint64_t)st, o1 = step * (uint64_t)s1;
+            const uint64_t a[8] = {a0[0] + o0, a0[1] + o0, a0[2] + o0, a0[3] + o0, a0[0] + o1, a0[1] + o1, a0[2] + o1, a0[3] + o1};
+            const uint64_t b[8] = {b0[0] + o0, b0[1] + o0, b0[2] + o0, b0[3] + o0, b0[0] + o1, b0[1] + o1, b0[2] + o1, b0[3] + o1};
+            int s2 = s1; uint32_t p2 = p1; next(s2, p2);
+            int s3 = s2; uint32_t p3 = p2; next(s3, p3);
+            // (probes past the last chunk look at stages that nothing refills: they answer "no" and are not used)
+            landed = pair_issue_two_stages(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &B->empty[s1], &full[s2], p2, &full[s3], p3);
+            st = s2; ph = p2;
+        }
+        if (ok && c < n_chunks) {              // an odd chunk is left
+            if (!(landed & 1u)) ok = mbar_wait_cluster(&full[st], ph, limit);
+            if (ok) {
+                if (gathered) { fence_async_proxy(); tc_fence_after(); }
+                const uint64_t o0 = step * (uint64_t)st;
+                const uint64_t a[4] = {a0[0] + o0, a0[1] + o0, a0[2] + o0, a0[3] + o0};
+                const uint64_t b[4] = {b0[0] + o0, b0[1] + o0, b0[2] + o0, b0[3] + o0};
+                int s1 = st; uint32_t p1 = ph; next(s1, p1);
+                pair_issue_stage(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[s1], p1);
+            }
         }
         if (!ok) *failed = 1;
         umma_commit_pair(&B->accbar);          // accumulators complete (or nothing was issued): told to both CTAs
@@ -173,6 +228,44 @@ __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool 
             mbar_arrive_remote(remote0 + (uint32_t)st * 8u);
         }
         if (!ok) *failed = 1;
+    }
+}
+
+// H for this CTA's 128 tokens x the tile's 128 neurons, straight from tensor memory: thread = token (lane of the
+// tensor memory), gate in columns [0, 128), up in [128, 256); warps w and w + 4 share the lanes and take 64 neurons
+// each.  Written without a branch per element: SiLU(g) * u is formed for every element and kept or zeroed by a select.
+template <int DT>
+__device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tmem, int warp, int lane, int tok0, int nt, int n_u) {
+    const int q = warp & 3, half = warp >> 2;
+    const int t = tok0 + q * 32 + lane;
+    const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+    const int i0 = nt * 128 + 64 * half;                          // union position of this thread's first neuron
+    uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + i0;
+    const int lim = t < P.T ? n_u - i0 : 0;                       // positions below lim are real entries of a real token
+    const bool own = P.tokbits != nullptr;                        // (uniform) every token keeps to its own list
+    const uint32_t *tb = own ? P.tokbits + (size_t)(t < P.T ? t : 0) * P.mask_words : nullptr;
+    for (int n0 = 0; n0 < 64; n0 += 16) {
+        uint32_t g[16], u[16];
+        tmem_ld16(trow + (uint32_t)(64 * half + n0), g);
+        tmem_ld16(trow + (uint32_t)(128 + 64 * half + n0), u);
+        uint32_t member = 0xFFFFu;                                // bit j: the token selected neuron n0 + j
+        if (own) {
+            member = 0;
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+                const int slot = P.union_slots[i0 + n0 + jj];     // the same address in every lane
+                member |= ((tb[slot >> 5] >> (slot & 31)) & 1u) << jj;
+            }
+        }
+        uint32_t w[8];
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+            const uint32_t bits = si_cvt<DT>::from_float(si_silu_mul(__uint_as_float(g[jj]), __uint_as_float(u[jj])));
+            const uint32_t b = (n0 + jj < lim && ((member >> jj) & 1u)) ? bits : 0u;
+            if (jj & 1) w[jj >> 1] |= b << 16; else w[jj >> 1] = b;
+        }
+        *reinterpret_cast<uint4 *>(hrow + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4 *>(hrow + n0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
     }
 }
 
@@ -220,6 +313,10 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                     mbar_arrive_expect_tx(&full[st], (uint32_t)stage_bytes);
                     tma_load_tile(stage, &x_map, c * kChunkK, tok0, &full[st]);
                     tma_load_tile(stage + 128 * 128, &rec_map, (int)rank * P.d_model + c * kChunkK, slot_first, &full[st]);
+                    // the weights come from HBM: ask for the tile of a later chunk now, so that its copy finds it in L2
+                    // (the ring alone holds too few bytes for that latency); one of the token tiles asks for all
+                    if (tp == 0 && c + kPrefetchAhead < n_chunks)
+                        tma_prefetch_tile(&rec_map, (int)rank * P.d_model + (c + kPrefetchAhead) * kChunkK, slot_first);
                 }
             }
         } else {
@@ -254,38 +351,17 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
         if (ok && active) {
-            // thread = token (tensor-memory lane); warps w and w + 4 share the lanes and take 64 neurons each
-            const int q = warp & 3, half = warp >> 2;
-            const int t = tok0 + q * 32 + lane;
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
-            uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + (size_t)nt * 128 + 64 * half;
-            const uint32_t *tb = P.tokbits && t < P.T ? P.tokbits + (size_t)t * P.mask_words : nullptr;
-            for (int n0 = 0; n0 < 64; n0 += 16) {
-                uint32_t g[16], u[16];
-                tmem_ld16(trow + (uint32_t)(64 * half + n0), g);
-                tmem_ld16(trow + (uint32_t)(128 + 64 * half + n0), u);
-                uint32_t w[8];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int i = nt * 128 + 64 * half + n0 + j;
-                    bool keep = t < P.T && i < n_u;
-                    if (keep && tb) { const int slot = P.union_slots[i]; keep = (tb[slot >> 5] >> (slot & 31)) & 1u; }
-                    const float out = keep ? si_silu_mul(__uint_as_float(g[j]), __uint_as_float(u[j])) : 0.f;
-                    const uint32_t b = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
-                    if (j & 1) w[j >> 1] |= b << 16; else w[j >> 1] = b;
-                }
-                *reinterpret_cast<uint4 *>(hrow + n0) = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4 *>(hrow + n0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
-            }
+            if (P.fmt) gateup_epilogue<SI_BF16>(P, tmem, warp, lane, tok0, nt, n_u);
+            else gateup_epilogue<SI_F16>(P, tmem, warp, lane, tok0, nt, n_u);
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (lane == 0) {
         const uint32_t idesc = make_idesc(P.fmt, 0, 0, 256, 256);
-        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, [&](int, int st, uint64_t (&a)[4], uint64_t (&b)[4]) {
-            const uint32_t sx = smem_u32(tiles + (size_t)st * stage_bytes), sw = sx + 128 * 128;
+        const uint32_t sx = smem_u32(tiles), sw = sx + 128 * 128;
+        uint64_t a0[4], b0[4];
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) { a[k4] = make_desc(sx + k4 * 32, 16, 1024); b[k4] = make_desc(sw + k4 * 32, 16, 1024); }
-        });
+        for (int k4 = 0; k4 < 4; ++k4) { a0[k4] = make_desc(sx + k4 * 32, 16, 1024); b0[k4] = make_desc(sw + k4 * 32, 16, 1024); }
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes);
     }
     pair_teardown(tmem, ncols);
 }
@@ -379,6 +455,10 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
 #pragma unroll
                 for (int hh = 0; hh < kHalfCols / 64; ++hh)
                     tma_load_tile(stage + 128 * 128 + hh * 8192, &rec_map, col0 + hh * 64, slot_first + c * kChunkK, &full[st]);
+                if (tp == 0 && c + kPrefetchAhead < n_chunks)
+#pragma unroll
+                    for (int hh = 0; hh < kHalfCols / 64; ++hh)
+                        tma_prefetch_tile(&rec_map, col0 + hh * 64, slot_first + (c + kPrefetchAhead) * kChunkK);
             }
         }
         bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
@@ -432,13 +512,13 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (lane == 0) {
         const uint32_t idesc = make_idesc(P.fmt, 0, 1, 256, N);
-        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, [&](int, int st, uint64_t (&a)[4], uint64_t (&b)[4]) {
-            const uint32_t sh = smem_u32(tiles + (size_t)st * stage_bytes), sw = sh + 128 * 128;
+        const uint32_t sh = smem_u32(tiles), sw = sh + 128 * 128;
+        uint64_t a0[4], b0[4];
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {   // 16 union entries per MMA = two 8-entry groups of 1024 bytes
-                a[k4] = make_desc(sh + k4 * 32, 16, 1024); b[k4] = make_desc(sw + k4 * 2048, 8192, 1024);
-            }
-        });
+        for (int k4 = 0; k4 < 4; ++k4) {       // 16 union entries per MMA = two 8-entry groups of 1024 bytes
+            a0[k4] = make_desc(sh + k4 * 32, 16, 1024); b0[k4] = make_desc(sw + k4 * 2048, 8192, 1024);
+        }
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes);
     }
     pair_teardown(tmem, ncols);
 }
