@@ -317,13 +317,21 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 uint32_t g[16], u[16];
                 tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, g);
                 tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(N + n0), u);
+                // (no branch per element: SiLU(g) * u is formed for every element and kept or zeroed by a select)
+                uint32_t member = 0;                               // bit q: token n0 + q uses this row's neuron
+                if (n_chunks > 0 && i < n_u) {
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        const int t = tok0 + n0 + q;
+                        const uint32_t bit = P.tokbits ? (P.tokbits[(size_t)(t < P.T ? t : 0) * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u : 1u;
+                        member |= (t < P.T ? bit : 0u) << q;
+                    }
+                }
 #pragma unroll
                 for (int q = 0; q < 16; ++q) {
-                    const int t = tok0 + n0 + q;
-                    bool keep = n_chunks > 0 && t < P.T && i < n_u;
-                    if (keep && P.tokbits) keep = (P.tokbits[(size_t)t * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u;
-                    const float out = keep ? si_silu_mul(__uint_as_float(g[q]), __uint_as_float(u[q])) : 0.f;
-                    hs[(n0 + q) * kRowPitch + r] = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
+                    const float v = si_silu_mul(__uint_as_float(g[q]), __uint_as_float(u[q]));
+                    const uint16_t hb = P.fmt ? si_cvt<SI_BF16>::from_float(v) : si_cvt<SI_F16>::from_float(v);
+                    hs[(n0 + q) * kRowPitch + r] = (member >> q) & 1u ? hb : (uint16_t)0;
                 }
             }
         } else if (ok && n_chunks > 0) {
@@ -428,9 +436,10 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 }
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float out = (member >> k) & 1u ? si_silu_mul(gg[k], uu[k]) : 0.f;
-                hs[(n + k) * kRowPitch + r] = P.fmt ? si_cvt<SI_BF16>::from_float(out) : si_cvt<SI_F16>::from_float(out);
+            for (int k = 0; k < 4; ++k) {      // (a select, not a branch per element)
+                const float v = si_silu_mul(gg[k], uu[k]);
+                const uint16_t hb = P.fmt ? si_cvt<SI_BF16>::from_float(v) : si_cvt<SI_F16>::from_float(v);
+                hs[(n + k) * kRowPitch + r] = (member >> k) & 1u ? hb : (uint16_t)0;
             }
         }
         __syncthreads();
