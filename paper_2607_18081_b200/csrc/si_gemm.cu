@@ -10,15 +10,15 @@
 // Token t therefore uses exactly its own list (Section 5 applied per token), whatever the
 // other tokens selected; with SI_FLAG_UNION_UNMASKED every token uses the whole union.
 //
-// Tiling.  Both contractions put the weight side on the MMA M dimension (128 rows of the
-// store per CTA tile) and the tokens on N (T padded to 16; tiles of 128 or 256 tokens beyond
-// that), so with one token tile the weights -- the dominant bytes -- are read exactly once.
-// Weight rows are gathered straight out of the neuron records with 16-byte cp.async copies into
-// the 128-byte-swizzled shared memory layouts the MMA descriptors expect (gate/up rows are
-// K-major, down rows MN-major).  K is split across CTAs so that small unions still fill the
-// machine.  The finishing passes (combine, split reduction) have no kernels of their own: an
-// unsplit tile is finished in the contraction's epilogue, a split tile by the CTA that delivers
-// its last fp32 partial, which sums the partials in split order -- so results are deterministic.
+// Tiling (this file: up to 128 tokens -- batched decode; calls with more tokens run on CTA pairs, si_gemm_pair.cu).
+// Both contractions put the weight side on the MMA M dimension (128 rows of the store per tile) and the tokens
+// on N (T padded to 16), so the weights -- the dominant bytes -- are read exactly once.  Weight rows are gathered
+// straight out of the neuron records with 16-byte cp.async copies into the 128-byte-swizzled shared memory
+// layouts the MMA descriptors expect (gate/up rows are K-major, down rows MN-major).  K is split among the CTAs
+// of a thread-block cluster (1, 2, 4 or 8 per tile) so that small unions still fill the machine; the CTAs of a
+// cluster sum their partial accumulators through distributed shared memory, in rank order -- so results do not
+// depend on timing --, and the finishing passes (combine, residual, rounding) run on the summed tile: there are
+// no partial tiles in global memory, no counters and no kernels for the finishing passes.
 #include "si_tc.cuh"
 
 using namespace si_tc;
@@ -233,21 +233,21 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // Flat grid sized on the host for the largest possible union.  The real union is known here: its
-    // tiles are split along K just far enough to give every SM slot one unit (P.n_split is the most
-    // the partial buffer holds), and the surplus CTAs leave at once.
+    // Flat grid sized on the host for the largest possible union: one thread-block cluster per union tile of 128,
+    // whose CTAs split K = d_model among themselves (cluster size = P.n_split, chosen on the host).  The real union
+    // is known here; the clusters of tiles past it leave at once.
     pdl_wait();                                 // the union kernel's results
     pdl_launch();
     const int n_u = *P.n_union;
     const int n_real = n_u > 128 ? (n_u + 127) / 128 : 1;
-    int ns = P.target_ctas / (n_real * P.tok_tiles);
-    ns = ns < 1 ? 1 : (ns > P.n_split ? P.n_split : ns);
-    if ((int)blockIdx.x >= n_real * P.tok_tiles * ns) {
+    const int ns = P.n_split;
+    const int ks = ns > 1 ? (int)cluster_ctarank() : 0, mt = blockIdx.x / ns, tt = 0;
+    if (mt >= n_real) {
         if (warp == kLoaderWarps)
             asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
         return;
     }
-    const int ks = blockIdx.x % ns, mt = (blockIdx.x / ns) % n_real, tt = blockIdx.x / (ns * n_real);
+    bool ok = true;                             // (loader / epilogue threads) no wait of this thread ran out
     const int total_k = P.d_model / kChunkK;                       // chunks; split ks takes an even share of them
     const int c0 = (int)((long long)ks * total_k / ns), c1 = (int)((long long)(ks + 1) * total_k / ns);
     const int n_chunks = c1 > c0 ? c1 - c0 : 0;
@@ -296,7 +296,7 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         }
         cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
         // ---------------------------------------------------------------- epilogue
-        bool ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
+        ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
         if (!ok && tid == 0)                 // a wait ran out: the tensor copies already started must still land before the CTA goes
             for (int c = armed > P.nstage ? armed - P.nstage : 0; c < armed; ++c)
                 if (!(P.withhold && blockIdx.x == 0 && c == 0)) mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
@@ -304,8 +304,6 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         // a warp reads tensor-memory lanes 32*(warp % 4) ..: warps w and w + 4 share the rows and take
         // alternate 16-column blocks.  Thread row r = union row mt*128 + r: N gate values, N up values
         const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
-        float *pg = P.partial + (((size_t)ks * 2 + 0) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
-        float *pu = P.partial + (((size_t)ks * 2 + 1) * P.nu_pad + (size_t)mt * 128 + r) * P.t_pad_total + tok0;
         if (ok && ns == 1) {
             // whole K in this CTA: form H straight from the accumulators (no partial tiles); the tile is
             // staged in shared memory -- every MMA has finished reading the stages -- and written out below
@@ -334,21 +332,6 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                     hs[(n0 + q) * kRowPitch + r] = (member >> q) & 1u ? hb : (uint16_t)0;
                 }
             }
-        } else if (ok && n_chunks > 0) {
-            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
-                uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4 *>(pg + n0 + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(N + n0), v);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4 *>(pu + n0 + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-            }
-        } else if (ok) {
-            for (int n0 = 16 * cb; n0 < N; n0 += 32)
-                for (int n = n0; n < n0 + 16; ++n) { pg[n] = 0.f; pu[n] = 0.f; }
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else {
@@ -375,74 +358,61 @@ si_gemm_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
             umma_commit(accbar);                  // accumulators complete (or nothing was issued)
         }
     }
-    __threadfence();                       // this CTA's partial tile is visible device-wide ...
     tc_fence_before();
     __syncthreads();
+    if (ns > 1) {
+        // ---- K split across the cluster: the partial accumulators are summed through distributed shared memory.
+        // CTA j of the cluster owns the tile's rows [j * 128 / ns, (j + 1) * 128 / ns): every CTA writes its partial
+        // values of those rows into slot (its rank) of CTA j's staging area (the pipeline stages, free once every
+        // CTA's MMAs are complete: first cluster barrier), and after the second barrier CTA j sums the slots in rank
+        // order -- so H does not depend on timing -- and forms H for its rows.
+        const int rows_per = 128 / ns, pitch = 2 * N + 4;            // floats per staged row: N gate, N up, padding
+        float *stg = reinterpret_cast<float *>(smem);                // [ns][rows_per][pitch]
+        cluster_sync_all();
+        if (warp < kLoaderWarps && ok) {
+            tc_fence_after();
+            const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
+            const uint32_t dst = map_to_cta(smem_u32(stg + ((size_t)ks * rows_per + (r % rows_per)) * pitch), (uint32_t)(r / rows_per));
+            for (int n0 = 16 * cb; n0 < 2 * N; n0 += 32) {           // columns [0, N) gate, [N, 2N) up
+                uint32_t v[16];
+                if (n_chunks > 0) tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    st_cluster_v4(dst + (uint32_t)(n0 + 4 * q) * 4u, n_chunks > 0 ? v[4 * q] : 0u, n_chunks > 0 ? v[4 * q + 1] : 0u,
+                                  n_chunks > 0 ? v[4 * q + 2] : 0u, n_chunks > 0 ? v[4 * q + 3] : 0u);
+            }
+        }
+        tc_fence_before();
+        cluster_sync_all();
+        if (!*failed) {
+            // one item = (token n, row rr of this CTA's rows): consecutive threads take consecutive rows, so a
+            // token's H values are written side by side
+            for (int it = tid; it < rows_per * N; it += kGemmThreads) {
+                const int n = it / rows_per, rr = it - n * rows_per;
+                const int i = mt * 128 + ks * rows_per + rr, t = tok0 + n;
+                float g = 0.f, u = 0.f;
+                for (int sp = 0; sp < ns; ++sp) {
+                    const float *row = stg + ((size_t)sp * rows_per + rr) * pitch;
+                    g += row[n]; u += row[N + n];
+                }
+                bool member = i < n_u && t < P.T;
+                if (member && P.tokbits) {
+                    const int slot = P.union_slots[i];
+                    member = (P.tokbits[(size_t)t * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u;
+                }
+                const float v = si_silu_mul(g, u);
+                const uint16_t hb = P.fmt ? si_cvt<SI_BF16>::from_float(v) : si_cvt<SI_F16>::from_float(v);
+                P.h_out[(size_t)t * P.nu_pad + i] = member ? hb : (uint16_t)0;
+            }
+        }
+    }
     if (warp == kLoaderWarps) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
     }
-    // ---- combine: the CTA that delivers the tile's last K split forms H for the tile.  The splits are
-    // summed in split order whoever is last, so H does not depend on the arrival order.
-    int *last_flag = const_cast<int *>(failed) + 1;
-    if (ns > 1) {
-        if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * P.tok_tiles + tt], 1u) == (unsigned)ns - 1;   // ... before it is counted
-        __syncthreads();
-        if (!*last_flag || *failed) return;
-        __threadfence();
-    } else if (*failed) {
-        return;
-    }
-    {
-        // H[t][i] = member(t, U[i]) ? SiLU(sum_s G) * (sum_s U) : 0, rounded to the store dtype.  Reads
-        // run along tokens (the partial tiles are [position][token]), H is [token][position]: transpose
-        // through shared memory (the pipeline stages are free now)
+    if (ns == 1 && !*failed) {
+        // the tile staged by the epilogue: H is [token][position]
         constexpr int kRowPitch = 128 + 8;                           // uint16 per token row of the staging tile
-        uint16_t *hs = reinterpret_cast<uint16_t *>(smem);
-        const size_t plane = (size_t)P.nu_pad * P.t_pad_total;       // one gate or up plane of a split
-        // one item = (union row, four consecutive tokens); all of an item's loads are issued before any
-        // is used, four splits at a time
-        const int nq = N / 4;
-        for (int it = tid; it < (ns > 1 ? 128 * nq : 0); it += kGemmThreads) {
-            const int r = it / nq, n = (it - r * nq) * 4;
-            const int i = mt * 128 + r;
-            const float *prow = P.partial + (size_t)i * P.t_pad_total + tok0 + n;
-            float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-            for (int sp0 = 0; sp0 < ns; sp0 += 4) {
-                float4 gv[4], uv[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const bool in = sp0 + k < ns;
-                    gv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k)) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    uv[k] = in ? __ldcg(reinterpret_cast<const float4 *>(prow + (size_t)(2 * (sp0 + k) + 1) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    g.x += gv[k].x; g.y += gv[k].y; g.z += gv[k].z; g.w += gv[k].w;
-                    u.x += uv[k].x; u.y += uv[k].y; u.z += uv[k].z; u.w += uv[k].w;
-                }
-            }
-            const float gg[4] = {g.x, g.y, g.z, g.w}, uu[4] = {u.x, u.y, u.z, u.w};
-            uint32_t member = 0;
-            if (i < n_u) {
-                if (P.tokbits) {
-                    const int slot = P.union_slots[i];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (tok0 + n + k < P.T)
-                            member |= ((P.tokbits[(size_t)(tok0 + n + k) * P.mask_words + (slot >> 5)] >> (slot & 31)) & 1u) << k;
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) member |= (tok0 + n + k < P.T ? 1u : 0u) << k;
-                }
-            }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {      // (a select, not a branch per element)
-                const float v = si_silu_mul(gg[k], uu[k]);
-                const uint16_t hb = P.fmt ? si_cvt<SI_BF16>::from_float(v) : si_cvt<SI_F16>::from_float(v);
-                hs[(n + k) * kRowPitch + r] = (member >> k) & 1u ? hb : (uint16_t)0;
-            }
-        }
-        __syncthreads();
+        const uint16_t *hs = reinterpret_cast<const uint16_t *>(smem);
         for (int e = tid; e < N * 16; e += kGemmThreads) {
             const int n = e >> 4, piece = e & 15;
             *reinterpret_cast<uint4 *>(P.h_out + (size_t)(tok0 + n) * P.nu_pad + (size_t)mt * 128 + piece * 8) =
@@ -468,7 +438,9 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
     volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mt = blockIdx.x, ks = blockIdx.y, tt = blockIdx.z;
+    // grid = (column tiles, K splits): the CTAs of a column tile form a thread-block cluster along y
+    const int mt = blockIdx.x, ks = blockIdx.y, tt = 0;
+    bool ok = true;                             // (loader / epilogue threads) no wait of this thread ran out
     // ---- set-up that needs nothing from the gate/up kernel (runs while that kernel finishes)
     uint32_t ncols = 32; while (ncols < (uint32_t)N) ncols <<= 1;
     if (tid == 0) {
@@ -551,7 +523,7 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 }
         }
         cp_async_wait_all();                 // nothing of this thread may still be in flight when the CTA ends
-        bool ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
+        ok = mbar_wait(accbar, 0, P.spin_limit) && !*failed;
         if (!ok && tid == 0) {               // a wait ran out: the tensor copies already started must still land before the CTA goes
             const int armed = armed_to > pre ? armed_to : (h_primed ? pre : 0);
             for (int c = armed > P.nstage ? armed - P.nstage : 0; c < armed; ++c)
@@ -561,7 +533,6 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         // thread holds output column mt*128 + r for the tokens; warps w and w + 4 share the rows and
         // take alternate 16-token blocks
         const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
-        float *py = P.partial + ((size_t)ks * P.t_pad_total + tok0) * P.d_model + (size_t)mt * 128 + r;
         if (ok && P.n_split == 1) {
             // whole K in this CTA: write y straight from the accumulators (a warp writes 32 consecutive
             // columns of one token at a time)
@@ -580,16 +551,6 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                     else reinterpret_cast<uint16_t *>(P.y)[o] = P.fmt ? si_cvt<SI_BF16>::from_float(a) : si_cvt<SI_F16>::from_float(a);
                 }
             }
-        } else if (ok && n_chunks > 0) {
-            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
-                uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
-#pragma unroll
-                for (int q = 0; q < 16; ++q) py[(size_t)(n0 + q) * P.d_model] = __uint_as_float(v[q]);
-            }
-        } else if (ok) {
-            for (int n0 = 16 * cb; n0 < N; n0 += 32)
-                for (int n = n0; n < n0 + 16; ++n) py[(size_t)n * P.d_model] = 0.f;
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else {
@@ -614,54 +575,47 @@ si_gemm_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
             umma_commit(accbar);
         }
     }
-    __threadfence();                       // this CTA's partial tile is visible device-wide ...
     tc_fence_before();
     __syncthreads();
+    const int ns = P.n_split;
+    if (ns > 1) {
+        // ---- K split across the cluster, summed through distributed shared memory (as in the gate/up kernel): CTA j
+        // owns output columns [j * 128 / ns, (j + 1) * 128 / ns) of the tile, receives every CTA's partial values
+        // of those columns in slot (rank), sums the slots in rank order, adds the residual and writes y.
+        const int cols_per = 128 / ns, pitch = N + 4;               // floats per staged column: N tokens, padding
+        float *stg = reinterpret_cast<float *>(smem);                // [ns][cols_per][pitch]
+        cluster_sync_all();                                          // every CTA's MMAs are complete: the stages are free
+        if (warp < kLoaderWarps && ok) {
+            tc_fence_after();
+            const int r = (warp & 3) * 32 + lane, cb = warp >> 2;
+            const uint32_t dst = map_to_cta(smem_u32(stg + ((size_t)ks * cols_per + (r % cols_per)) * pitch), (uint32_t)(r / cols_per));
+            for (int n0 = 16 * cb; n0 < N; n0 += 32) {
+                uint32_t v[16];
+                if (n_chunks > 0) tmem_ld16(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)n0, v);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    st_cluster_v4(dst + (uint32_t)(n0 + 4 * q) * 4u, n_chunks > 0 ? v[4 * q] : 0u, n_chunks > 0 ? v[4 * q + 1] : 0u,
+                                  n_chunks > 0 ? v[4 * q + 2] : 0u, n_chunks > 0 ? v[4 * q + 3] : 0u);
+            }
+        }
+        tc_fence_before();
+        cluster_sync_all();
+        if (!*failed) {
+            // one item = (token n, column cc of this CTA's columns): consecutive threads write consecutive columns
+            for (int it = tid; it < cols_per * N; it += kGemmThreads) {
+                const int n = it / cols_per, cc = it - n * cols_per, t = tok0 + n;
+                if (t >= P.T) continue;
+                float a = 0.f;
+                for (int sp = 0; sp < ns; ++sp) a += stg[((size_t)sp * cols_per + cc) * pitch + n];
+                const size_t o = (size_t)t * P.d_model + (size_t)mt * 128 + ks * cols_per + cc;
+                if (P.residual) a += P.fmt ? si_cvt<SI_BF16>::lo((uint32_t)P.x[o]) : si_cvt<SI_F16>::lo((uint32_t)P.x[o]);
+                if (P.y_f32) reinterpret_cast<float *>(P.y)[o] = a;
+                else reinterpret_cast<uint16_t *>(P.y)[o] = P.fmt ? si_cvt<SI_BF16>::from_float(a) : si_cvt<SI_F16>::from_float(a);
+            }
+        }
+    }
     if (warp == kLoaderWarps) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
-    }
-    // ---- reduce: the CTA that delivers the column tile's last K split writes y for the tile:
-    // y[t][j] = (x[t][j] +) sum over the splits in split order (independent of the arrival order)
-    if (P.n_split == 1) return;
-    int *last_flag = const_cast<int *>(failed) + 1;
-    if (tid == 0) *last_flag = atomicAdd(&P.tile_ctr[mt * gridDim.z + tt], 1u) == (unsigned)P.n_split - 1;   // ... before it is counted
-    __syncthreads();
-    if (!*last_flag || *failed) return;
-    __threadfence();
-    // one item = (token, four consecutive columns); an item's loads are issued before any is used
-    for (int it = tid; it < N * 32; it += kGemmThreads) {
-        const int n = it >> 5, col = mt * 128 + (it & 31) * 4, t = tok0 + n;
-        if (t >= P.T) continue;
-        const float *pp = P.partial + (size_t)t * P.d_model + col;
-        const size_t plane = (size_t)P.t_pad_total * P.d_model;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp0 = 0; sp0 < P.n_split; sp0 += 8) {
-            float4 v[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                v[k] = sp0 + k < P.n_split ? __ldcg(reinterpret_cast<const float4 *>(pp + (size_t)(sp0 + k) * plane)) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) { a.x += v[k].x; a.y += v[k].y; a.z += v[k].z; a.w += v[k].w; }
-        }
-        const size_t o = (size_t)t * P.d_model + col;
-        if (P.residual) {
-            const uint2 xw = *reinterpret_cast<const uint2 *>(P.x + o);
-            if (P.fmt) { a.x += si_cvt<SI_BF16>::lo(xw.x); a.y += si_cvt<SI_BF16>::hi(xw.x); a.z += si_cvt<SI_BF16>::lo(xw.y); a.w += si_cvt<SI_BF16>::hi(xw.y); }
-            else { a.x += si_cvt<SI_F16>::lo(xw.x); a.y += si_cvt<SI_F16>::hi(xw.x); a.z += si_cvt<SI_F16>::lo(xw.y); a.w += si_cvt<SI_F16>::hi(xw.y); }
-        }
-        if (P.y_f32) {
-            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + o) = a;
-        } else {
-            uint2 w;
-            if (P.fmt) {
-                w.x = (uint32_t)si_cvt<SI_BF16>::from_float(a.x) | ((uint32_t)si_cvt<SI_BF16>::from_float(a.y) << 16);
-                w.y = (uint32_t)si_cvt<SI_BF16>::from_float(a.z) | ((uint32_t)si_cvt<SI_BF16>::from_float(a.w) << 16);
-            } else {
-                w.x = (uint32_t)si_cvt<SI_F16>::from_float(a.x) | ((uint32_t)si_cvt<SI_F16>::from_float(a.y) << 16);
-                w.y = (uint32_t)si_cvt<SI_F16>::from_float(a.z) | ((uint32_t)si_cvt<SI_F16>::from_float(a.w) << 16);
-            }
-            *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(P.y) + o) = w;
-        }
     }
 }
 
@@ -690,28 +644,19 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
-// Launch a contraction kernel so that it may be scheduled while the previous kernel of the stream is
-// still finishing (the kernel itself waits for that kernel's results with pdl_wait()).
-cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap), dim3 grid, size_t smem, cudaStream_t stream,
-                                     const GemmParams &P, const CUtensorMap &map) {
+// Launch a contraction kernel as thread-block clusters of `cluster` CTAs, so that it may be scheduled while the
+// previous kernel of the stream is still finishing (the kernel itself waits for that kernel's results with pdl_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after_predecessor(void (*kern)(KArgs...), dim3 grid, dim3 cluster, size_t smem, cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, P, map);
-}
-
-cudaError_t launch_after_predecessor(void (*kern)(GemmParams, CUtensorMap, CUtensorMap), dim3 grid, size_t smem,
-                                     cudaStream_t stream, const GemmParams &P, const CUtensorMap &m0, const CUtensorMap &m1) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, P, m0, m1);
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster.x; attr[1].val.clusterDim.y = cluster.y; attr[1].val.clusterDim.z = cluster.z;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
 int pick_stages_gemm(size_t stage_bytes, int n_tok) {
@@ -755,10 +700,10 @@ size_t si_gemm_partial_bytes(const si_store *s, int T_max) {
     return T_max > 1 ? kPartialCap : 0;
 }
 
-// Counters a call may need beyond the bitmaps: one per (tile, token tile) of either contraction.
+// Zero-on-entry words a call needs beyond the bitmaps.
 size_t si_gemm_counter_bytes(const si_store *s, size_t nl_pad, size_t t_pad) {
-    const size_t tok_tiles = (t_pad + 127) / 128;
-    return (64 + (nl_pad / 128 + (size_t)s->d_model / 128 + 2) * tok_tiles) * 4;
+    (void)s; (void)nl_pad; (void)t_pad;
+    return 64 * 4;                              // the union kernel's ticket words
 }
 
 int si_union_launch(const si_store *s, int layer, int T, const int32_t *idx, const int32_t *idx_offsets,
@@ -876,30 +821,21 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     const int nu_pad = (int)si_align_up((size_t)cap, 128);
     const int t_pad_total = (int)si_align_up((size_t)T, 16);
     const int m_tiles = nu_pad / 128;
-    // token tile width: 256 reads the weights least often, but with few weight tiles 128-wide token
-    // tiles put twice as many CTAs to work (and often make K splits unnecessary)
-    int tile_n = 256;
-    if (t_pad_total > 128 && m_tiles * ((t_pad_total + 255) / 256) * 10 < s->num_sms * 6) tile_n = 128;
-    const int tok_tiles = (t_pad_total + tile_n - 1) / tile_n;
     const bool own_lists = !shared && !(flags & SI_FLAG_UNION_UNMASKED);   // membership differs per token
-    const int n_ctr_gu = m_tiles * tok_tiles, n_ctr_dn = (d / 128) * tok_tiles;
-    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, n_ctr_gu + n_ctr_dn, half);
+    UnionScratch us = union_scratch(s, wsb, ws, T, n_loaded, 0, half);
     if (us.zero_bytes > ws.mask_half) return SI_ERR_NOMEM;
     {
         int rc = union_stage_launch(s, n_loaded, shared ? 1 : T, own_lists, idx, idx_offsets, k_fixed, us, uni, n_union,
                                     nu_pad, status_dev, stream, true);
         if (rc) return rc;
     }
-    // ---- tiling
-    const int n_tok = tok_tiles > 1 ? tile_n : t_pad_total;
-    // with several token tiles every tile must be full width: pad the token dimension
-    const int t_pad_alloc = tok_tiles * n_tok;
+    // ---- tiling (calls with more than 128 tokens leave for the CTA-pair kernels below: one token tile here)
+    const int n_tok = t_pad_total, t_pad_alloc = t_pad_total;
     GemmParams P;
     P.rec_base = (const char *)s->records(layer); P.rec_bytes = (int)s->record_bytes(); P.d_model = d; P.chunks = d / 8;
     P.union_slots = uni; P.n_union = n_union; P.nu_pad = nu_pad;
     P.x = (const uint16_t *)x; P.T = T; P.n_tok = n_tok;
     P.h = (const uint16_t *)(wsb + ws.h_off); P.t_pad_total = t_pad_alloc;
-    P.partial = (float *)(wsb + ws.partial_off);
     P.fmt = s->dtype == SI_BF16 ? 1 : 0;
     P.status = status_dev;
     P.tokbits = own_lists ? us.tokbits : nullptr; P.mask_words = us.mask_words;
@@ -909,52 +845,44 @@ int si_multi_token_launch(const si_store *s, int layer, const void *x, int T, co
     P.pair_n = 0;
     if (si_pair_path_applies(s, T))
         return si_pair_contractions_launch(s, P, n_loaded, wsb + ws.h_off, ws.h_bytes, stream);
-    // gate/up: K = d_model may be split up to s1 ways (what the partial buffer holds); the kernel
-    // picks the split from the real union size so that one wave of CTAs covers the SM slots (two CTAs
-    // per SM with few tokens: the gathers are latency-bound)
+    // (here T <= 128: one token tile.)  Both contractions split K among the CTAs of a thread-block cluster (1, 2, 4 or
+    // 8 CTAs per tile), which sum their partial accumulators through distributed shared memory.  The cluster sizes
+    // aim at one wave of CTAs over the SM slots (two CTAs per SM with few tokens: the gathers are latency-bound).
     const int target = (t_pad_alloc <= 16 ? 2 : 1) * s->num_sms;
     const int k_chunks = d / kChunkK;
-    int s1 = k_chunks < 8 ? k_chunks : 8;
-    const size_t part_cap = kPartialCap < ws.partial_bytes ? kPartialCap : ws.partial_bytes;
-    while (s1 > 1 && (size_t)s1 * 2 * nu_pad * t_pad_alloc * 4 > part_cap) --s1;
-    if ((size_t)2 * nu_pad * t_pad_alloc * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
     if ((size_t)t_pad_alloc * nu_pad * 2 > ws.h_bytes) return SI_ERR_NOMEM;
     {
+        // gate/up: the grid is sized for the largest possible union, whose tiles past the real union leave at once
+        int s1 = 1;
+        while (s1 < 8 && s1 * 2 <= k_chunks && m_tiles * s1 * 2 <= target) s1 *= 2;
         const size_t stage = 2 * 128 * 128 + (size_t)n_tok * 128;
         P.nstage = pick_stages_gemm(stage, n_tok); P.n_split = s1;
         if (P.nstage < 2) return SI_ERR_UNSUPPORTED;
+        if (s1 > 1 && (size_t)128 * (2 * n_tok + 4) * 4 > (size_t)P.nstage * stage) return SI_ERR_UNSUPPORTED;   // staging area of the cluster sum
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        const int units = m_tiles * tok_tiles;
-        dim3 grid(units > target ? units : target);
-        P.tok_tiles = tok_tiles; P.target_ctas = target;
-        P.tile_ctr = us.ctr;
         CUtensorMap x_map, rec_map;
         int rc = make_tile_map(&x_map, x, (size_t)d, (size_t)T, (size_t)d * 2, n_tok);
         if (rc) return rc;
         // the layer's records as a matrix [n_loaded][3 * d_model]: 128 consecutive slots x 64 columns per tile
         rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 128);
         if (rc) return rc;
-        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, grid, smem, stream, P, x_map, rec_map));
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_gateup_kernel, dim3(m_tiles * s1), dim3(s1), smem, stream, P, x_map, rec_map));
     }
-    // down: split K = union
-    int s2 = (t_pad_alloc <= 16 ? 2 * s->num_sms : s->num_sms) / ((d / 128) * tok_tiles);
-    if (s2 < 1) s2 = 1;
-    if (s2 > 8) s2 = 8;
-    if (s2 > nu_pad / kChunkK) s2 = nu_pad / kChunkK;
-    while (s2 > 1 && (size_t)s2 * t_pad_alloc * d * 4 > kPartialCap) --s2;
-    if ((size_t)s2 * t_pad_alloc * d * 4 > ws.partial_bytes) return SI_ERR_NOMEM;
     {
+        // down: K = the union
+        int s2 = 1;
+        while (s2 < 8 && s2 * 2 <= nu_pad / kChunkK && (d / 128) * s2 * 2 <= target) s2 *= 2;
         const size_t stage = 64 * 256 + (size_t)n_tok * 128;
         P.nstage = pick_stages_gemm(stage, n_tok); P.n_split = s2;
+        if (P.nstage < 2) return SI_ERR_UNSUPPORTED;
+        if (s2 > 1 && (size_t)128 * (n_tok + 4) * 4 > (size_t)P.nstage * stage) return SI_ERR_UNSUPPORTED;
         size_t smem = (size_t)P.nstage * stage + 256;
         SI_CUDA_TRY(cudaFuncSetAttribute(si_gemm_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        dim3 grid(d / 128, s2, tok_tiles);
-        P.tile_ctr = us.ctr + n_ctr_gu;
         CUtensorMap h_map;
         int rc = make_tile_map(&h_map, wsb + ws.h_off, (size_t)nu_pad, (size_t)t_pad_alloc, (size_t)nu_pad * 2, n_tok);
         if (rc) return rc;
-        SI_CUDA_TRY(launch_after_predecessor(si_gemm_down_kernel, grid, smem, stream, P, h_map));
+        SI_CUDA_TRY(launch_after_predecessor(si_gemm_down_kernel, dim3(d / 128, s2, 1), dim3(1, s2, 1), smem, stream, P, h_map));
     }
     SI_CUDA_TRY(cudaGetLastError());
     return SI_OK;

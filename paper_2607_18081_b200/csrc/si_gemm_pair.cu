@@ -28,16 +28,6 @@ constexpr int kPairMaxStages = 8;
 constexpr int kPrefetchAhead = 16;               // chunks between a weight tile's L2 prefetch and its copy into shared memory
 constexpr int kPairTokens = 256;                 // tokens of a pair's tile (M of the MMA), 128 per CTA
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
-    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank)); return r;
-}
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
@@ -542,7 +532,7 @@ int stages_for(size_t stage_bytes) {
 }  // namespace
 
 bool si_pair_path_applies(const si_store *s, int T) {
-    return T > 128 && s->d_model % 256 == 0;
+    return T > 128 && s->d_model % 128 == 0;
 }
 
 // Both contractions of a call with more than 128 tokens, after the union stage (P holds the call's parameters;
@@ -569,7 +559,7 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
     {
         // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs: take 256 only when that
         // still puts a pair on most SM pairs
-        const int n = (d / 256) * tok_pairs * 2 >= s->num_sms * 3 / 4 ? 256 : 128;
+        const int n = d % 256 == 0 && (d / 256) * tok_pairs * 2 >= s->num_sms * 3 / 4 ? 256 : 128;
         P.pair_n = n;
         const size_t stage = 128 * 128 + (size_t)64 * n;
         P.nstage = stages_for(stage);

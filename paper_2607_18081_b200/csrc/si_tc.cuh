@@ -110,6 +110,20 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank)); return r;
+}
+// 16 bytes into the shared memory of a CTA of the cluster (address from map_to_cta)
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 // ------------------------------------------------------------------------------- parameters
 struct GemmParams {
     const char *rec_base;          // records of the layer
@@ -121,14 +135,10 @@ struct GemmParams {
     int T, n_tok;                  // tokens, N of the MMA (multiple of 16, <= 256)
     const uint16_t *h;             // [t_pad_total][nu_pad] (down)
     int t_pad_total;
-    float *partial;                // gate/up: [S][2][nu_pad][t_pad_total]; down: [S][t_pad_total][d_model]
-    int n_split;                   // K splits
+    int n_split;                   // K splits = CTAs of the thread-block cluster that works on a tile
     int fmt;                       // 0 f16, 1 bf16
     int nstage;
     int32_t *status;
-    // fused finishing passes: the CTA that completes a tile's last K split sums the splits
-    int tok_tiles, target_ctas;    // gate/up: token tiles; CTAs that can be resident at once
-    unsigned *tile_ctr;            // per (tile, token tile) arrival counters, zero on entry
     const uint32_t *tokbits;       // [T][mask_words] slot bitmaps of the tokens' own lists, or nullptr: all tokens
     int mask_words;                //   use the whole union
     uint16_t *h_out;               // gate/up: H [t_pad_total][nu_pad]
