@@ -221,23 +221,24 @@ __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool 
     }
 }
 
-// H for this CTA's 128 tokens x the tile's 128 neurons, straight from tensor memory: thread = token (lane of the
-// tensor memory), gate in columns [0, 128), up in [128, 256); warps w and w + 4 share the lanes and take 64 neurons
+// H for this CTA's 128 tokens x the tile's W neurons, straight from tensor memory: thread = token (lane of the
+// tensor memory), gate in columns [0, W), up in [W, 2W); warps w and w + 4 share the lanes and take W / 2 neurons
 // each.  Written without a branch per element: SiLU(g) * u is formed for every element and kept or zeroed by a select.
-template <int DT>
+template <int DT, int W>
 __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tmem, int warp, int lane, int tok0, int nt, int n_u) {
     const int q = warp & 3, half = warp >> 2;
     const int t = tok0 + q * 32 + lane;
     const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
-    const int i0 = nt * 128 + 64 * half;                          // union position of this thread's first neuron
+    const int i0 = nt * W + (W / 2) * half;                       // union position of this thread's first neuron
     uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + i0;
     const int lim = t < P.T ? n_u - i0 : 0;                       // positions below lim are real entries of a real token
     const bool own = P.tokbits != nullptr;                        // (uniform) every token keeps to its own list
     const uint32_t *tb = own ? P.tokbits + (size_t)(t < P.T ? t : 0) * P.mask_words : nullptr;
-    for (int n0 = 0; n0 < 64; n0 += 16) {
+    for (int n0 = 0; n0 < W / 2; n0 += 16) {
+        if (i0 + n0 >= P.nu_pad) break;                           // (a last tile of 96 may reach past the padded union)
         uint32_t g[16], u[16];
-        tmem_ld16(trow + (uint32_t)(64 * half + n0), g);
-        tmem_ld16(trow + (uint32_t)(128 + 64 * half + n0), u);
+        tmem_ld16(trow + (uint32_t)((W / 2) * half + n0), g);
+        tmem_ld16(trow + (uint32_t)(W + (W / 2) * half + n0), u);
         uint32_t member = 0xFFFFu;                                // bit j: the token selected neuron n0 + j
         if (own) {
             member = 0;
@@ -259,32 +260,38 @@ __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tm
     }
 }
 
-// Gate/up contraction: one pair per (union tile of 128 neurons, 256 tokens).
+// Gate/up contraction: one pair per (union tile of W neurons, 256 tokens); W = 128, or 96 when that puts a tile on
+// more of the SM pairs (N of the MMA = 2 W: the tile's gate rows and up rows).
+template <int W>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map,
                       const __grid_constant__ CUtensorMap rec_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
-    constexpr int stage_bytes = 2 * 128 * 128;                    // this CTA's X tile, this CTA's 128 weight rows
+    constexpr int stage_bytes = 128 * 128 + W * 128;              // this CTA's X tile, this CTA's W weight rows
     uint8_t *tiles = smem;
     PairBars *B = reinterpret_cast<PairBars *>(smem + (size_t)P.nstage * stage_bytes);
     volatile int *failed = &B->failed;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();
-    constexpr uint32_t ncols = 256;                               // 128 gate + 128 up accumulator columns
+    constexpr uint32_t ncols = 256;                               // W gate + W up accumulator columns
     const uint32_t tmem = pair_setup(B, P.nstage, ncols, rank);
 
     pdl_wait();                                 // the union kernel's results
     pdl_launch();
     const int pair = blockIdx.x >> 1;
-    const int n_tiles = P.nu_pad / 128;
+    const int n_tiles = (P.nu_pad + W - 1) / W;
     const int nt = pair % n_tiles, tp = pair / n_tiles;
     const int n_u = *P.n_union;
-    const bool active = nt * 128 < n_u;          // tiles past the real union have nothing to do
+    // tiles past the real union have nothing to do (the down contraction reads H in chunks of 64 entries: up to there
+    // H must be written)
+    const bool active = nt * W < (n_u + kChunkK - 1) / kChunkK * kChunkK;
     const int n_chunks = active ? P.d_model / kChunkK : 0;
     const int tok0 = tp * kPairTokens + (int)rank * 128;          // this CTA's tokens
-    // a tile of 128 consecutive slots needs no gather: its rows are one tensor copy out of the record matrix
-    const int slot_first = P.union_slots[nt * 128];
-    const bool run = P.union_slots[nt * 128 + 127] - slot_first == 127;
+    // union entry of tile row r (a last tile of 96 may reach past the padded union: its surplus rows repeat the last entry)
+    auto entry = [&](int r) { const int e = nt * W + r; return e < P.nu_pad ? e : P.nu_pad - 1; };
+    // a tile of W consecutive slots needs no gather: its rows are one tensor copy out of the record matrix
+    const int slot_first = P.union_slots[entry(0)];
+    const bool run = nt * W + W <= P.nu_pad && P.union_slots[nt * W + W - 1] - slot_first == W - 1;
     uint64_t *full = run ? B->full_t : B->full_g;
     const bool withhold = P.withhold && blockIdx.x == 0;
 
@@ -313,10 +320,10 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
             // copy j of a thread covers 16-byte piece (tid & 7) of tile row 32*j + (tid >> 3): a warp instruction
             // reads four whole 128-byte row segments
             const int q8 = tid & 7, r32 = tid >> 3;
-            const char *wrow[4];
+            const char *wrow[W / 32];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                wrow[j] = P.rec_base + (size_t)P.union_slots[nt * 128 + 32 * j + r32] * P.rec_bytes + (size_t)rank * P.d_model * 2 + q8 * 16;
+            for (int j = 0; j < W / 32; ++j)
+                wrow[j] = P.rec_base + (size_t)P.union_slots[entry(32 * j + r32)] * P.rec_bytes + (size_t)rank * P.d_model * 2 + q8 * 16;
             const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);
             for (int c = 0; c < n_chunks; ++c) {
                 const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
@@ -324,7 +331,7 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 uint8_t *stage = tiles + (size_t)st * stage_bytes;
                 uint8_t *sw = stage + 128 * 128 + off0;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { cp_async16(sw + j * 4096, wrow[j]); wrow[j] += 128; }
+                for (int j = 0; j < W / 32; ++j) { cp_async16(sw + j * 4096, wrow[j]); wrow[j] += 128; }
                 if (tid == 0 && !(withhold && c == 0)) {
                     armed = c + 1;
                     mbar_arrive_expect_tx(&full[st], 128u * 128u);
@@ -341,12 +348,12 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
         if (ok && active) {
-            if (P.fmt) gateup_epilogue<SI_BF16>(P, tmem, warp, lane, tok0, nt, n_u);
-            else gateup_epilogue<SI_F16>(P, tmem, warp, lane, tok0, nt, n_u);
+            if (P.fmt) gateup_epilogue<SI_BF16, W>(P, tmem, warp, lane, tok0, nt, n_u);
+            else gateup_epilogue<SI_F16, W>(P, tmem, warp, lane, tok0, nt, n_u);
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (lane == 0) {
-        const uint32_t idesc = make_idesc(P.fmt, 0, 0, 256, 256);
+        const uint32_t idesc = make_idesc(P.fmt, 0, 0, 256, 2 * W);
         const uint32_t sx = smem_u32(tiles), sw = sx + 128 * 128;
         uint64_t a0[4], b0[4];
 #pragma unroll
@@ -545,16 +552,26 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
     P.t_pad_total = t_pad_alloc; P.n_tok = kPairTokens; P.n_split = 1;
     P.h = (const uint16_t *)h_buf; P.h_out = (uint16_t *)h_buf;
     {
-        const size_t stage = 2 * 128 * 128;
+        // tiles of 128 neurons, or of 96 when that costs less: cost = waves of pair tiles over the SM pairs x tile width
+        const int slots = s->num_sms / 2;
+        const int pairs128 = (P.nu_pad / 128) * tok_pairs, pairs96 = ((P.nu_pad + 95) / 96) * tok_pairs;
+        const int cost128 = ((pairs128 + slots - 1) / slots) * 128, cost96 = ((pairs96 + slots - 1) / slots) * 96;
+        const int w = cost96 < cost128 ? 96 : 128;
+        const size_t stage = 128 * 128 + (size_t)w * 128;
         P.nstage = stages_for(stage);
         const size_t smem = (size_t)P.nstage * stage + sizeof(PairBars);
-        SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         CUtensorMap x_map, rec_map;
         int rc = make_tile_map(&x_map, P.x, (size_t)d, (size_t)P.T, (size_t)d * 2, 128);
         if (rc) return rc;
-        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 128);
+        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, w);
         if (rc) return rc;
-        SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel, (P.nu_pad / 128) * tok_pairs, smem, stream, P, x_map, rec_map));
+        if (w == 96) {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<96>, pairs96, smem, stream, P, x_map, rec_map));
+        } else {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<128>, pairs128, smem, stream, P, x_map, rec_map));
+        }
     }
     {
         // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs: take 256 only when that
