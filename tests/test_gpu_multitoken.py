@@ -226,3 +226,20 @@ def test_many_tokens_degenerate_unions(api, c1, m7b):
     y = _run(api, m7b, 0, x7, prefix, None, k, T, flags=api.SI_FLAG_SHARED_LIST, y_dtype=torch.bfloat16)
     for t in (0, 127, 128):
         assert_close(from_dev(y[t]), m7b.oracle_y(0, x7[t], prefix), f"129 tokens, token {t}")
+
+
+@pytest.mark.parametrize("T", [48, 100, 128])
+def test_7b_up_to_128_tokens_cluster_split(api, m7b, T):
+    """The widest token tiles of the one-CTA kernels (48, 112 and 128 columns of tensor memory per accumulator): K is
+    split over a thread-block cluster and the partial accumulators are summed through distributed shared memory,
+    whose staging area grows with the token count.  Own lists, residual, 16-bit output; run twice: bit-stable."""
+    cfg = m7b.cfg
+    k = cfg.k_active
+    lists = wl.zipf_lists(cfg, 0, T, first_token=5)
+    x = wl.x_tokens(cfg, 0, T, first_token=40)
+    y = _run(api, m7b, 0, x, lists, None, k, T, flags=api.SI_FLAG_RESIDUAL, y_dtype=torch.bfloat16)
+    for t in sorted({0, 15, 16, T // 2, T - 1}):
+        ref = m7b.oracle_y(0, x[t], lists[t]) + wl.bits_to_float64(x[t], cfg.dtype)
+        assert_close(from_dev(y[t]), ref, f"T={T} token {t}")
+    y2 = _run(api, m7b, 0, x, lists, None, k, T, flags=api.SI_FLAG_RESIDUAL, y_dtype=torch.bfloat16)
+    assert torch.equal(y, y2)
