@@ -231,6 +231,8 @@ __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tm
     const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
     const int i0 = nt * W + (W / 2) * half;                       // union position of this thread's first neuron
     uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + i0;
+    const bool has_row = t < P.t_pad_total;                       // H has rows for the tokens padded to 16 only (no early
+                                                                  // return: the tensor-memory loads below are warp-wide)
     const int lim = t < P.T ? n_u - i0 : 0;                       // positions below lim are real entries of a real token
     const bool own = P.tokbits != nullptr;                        // (uniform) every token keeps to its own list
     const uint32_t *tb = own ? P.tokbits + (size_t)(t < P.T ? t : 0) * P.mask_words : nullptr;
@@ -255,8 +257,10 @@ __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tm
             const uint32_t b = (n0 + jj < lim && ((member >> jj) & 1u)) ? bits : 0u;
             if (jj & 1) w[jj >> 1] |= b << 16; else w[jj >> 1] = b;
         }
-        *reinterpret_cast<uint4 *>(hrow + n0) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4 *>(hrow + n0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+        if (has_row) {
+            *reinterpret_cast<uint4 *>(hrow + n0) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(hrow + n0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
     }
 }
 
@@ -547,7 +551,8 @@ bool si_pair_path_applies(const si_store *s, int T) {
 int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, void *h_buf, size_t h_bytes, cudaStream_t stream) {
     const int d = P.d_model;
     const int tok_pairs = (P.T + kPairTokens - 1) / kPairTokens;
-    const int t_pad_alloc = tok_pairs * kPairTokens;
+    // H holds the tokens padded to 16 rows; a tile's rows past them are not written, and read as zero through the tensor map
+    const int t_pad_alloc = (int)si_align_up((size_t)P.T, 16);
     if ((size_t)t_pad_alloc * P.nu_pad * 2 > h_bytes) return SI_ERR_NOMEM;
     P.t_pad_total = t_pad_alloc; P.n_tok = kPairTokens; P.n_split = 1;
     P.h = (const uint16_t *)h_buf; P.h_out = (uint16_t *)h_buf;
