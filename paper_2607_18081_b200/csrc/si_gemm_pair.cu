@@ -53,10 +53,11 @@ __device__ __forceinline__ void umma_pair(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// arrives on the barrier at this offset in BOTH CTAs once the MMAs issued so far have completed
-__device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
+// arrives on the barrier at this offset in BOTH CTAs of the pair (mask: their ranks in the cluster) once the MMAs issued
+// so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t mask) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+                 ::"r"(smem_u32(bar)), "h"(mask) : "memory");
 }
 
 // One pipeline stage of the pair's MMA thread as a single instruction sequence: probe the NEXT stage's barrier,
@@ -64,7 +65,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar) {
 // then read the probe's answer.  A probe takes a couple of hundred cycles to answer; issued first, it is answered
 // while the MMAs are being issued instead of ahead of them.  Returns whether the next stage had already landed.
 __device__ __forceinline__ bool pair_issue_stage(uint32_t d_tmem, const uint64_t (&a)[4], const uint64_t (&b)[4], uint32_t idesc,
-                                                 uint32_t accumulate_first, uint64_t *empty_bar, uint64_t *next_full, uint32_t next_parity) {
+                                                 uint32_t accumulate_first, uint64_t *empty_bar, uint64_t *next_full, uint32_t next_parity, uint16_t mask) {
     uint32_t landed;
     asm volatile(
         "{\n\t.reg .pred q, p, t;\n\t"
@@ -79,7 +80,7 @@ __device__ __forceinline__ bool pair_issue_stage(uint32_t d_tmem, const uint64_t
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(landed)
         : "r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(accumulate_first),
-          "r"(idesc), "r"(smem_u32(next_full)), "r"(next_parity), "r"(smem_u32(empty_bar)), "h"((uint16_t)3)
+          "r"(idesc), "r"(smem_u32(next_full)), "r"(next_parity), "r"(smem_u32(empty_bar)), "h"(mask)
         : "memory");
     return landed != 0;
 }
@@ -89,7 +90,8 @@ __device__ __forceinline__ bool pair_issue_stage(uint32_t d_tmem, const uint64_t
 // MMAs of one stage when these are narrow).  bit 0 / 1 of the result: stage c + 2 / c + 3 had already landed.
 __device__ __forceinline__ uint32_t pair_issue_two_stages(uint32_t d_tmem, const uint64_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc,
                                                           uint32_t accumulate_first, uint64_t *empty0, uint64_t *empty1,
-                                                          uint64_t *next_full0, uint32_t next_parity0, uint64_t *next_full1, uint32_t next_parity1) {
+                                                          uint64_t *next_full0, uint32_t next_parity0, uint64_t *next_full1, uint32_t next_parity1,
+                                                          uint16_t mask) {
     uint32_t landed;
     asm volatile(
         "{\n\t.reg .pred q0, q1, p, t;\n\t.reg .b32 r0, r1;\n\t"
@@ -114,7 +116,7 @@ __device__ __forceinline__ uint32_t pair_issue_two_stages(uint32_t d_tmem, const
         : "r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
           "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7]),
           "r"(accumulate_first), "r"(idesc), "r"(smem_u32(next_full0)), "r"(next_parity0), "r"(smem_u32(next_full1)), "r"(next_parity1),
-          "r"(smem_u32(empty0)), "r"(smem_u32(empty1)), "h"((uint16_t)3)
+          "r"(smem_u32(empty0)), "r"(smem_u32(empty1)), "h"(mask)
         : "memory");
     return landed;
 }
@@ -170,7 +172,9 @@ __device__ __forceinline__ void pair_teardown(uint32_t tmem, uint32_t ncols) {
 // one ahead of it is nearly done, so whatever the thread does between two stages the tensor pipe waits for.
 __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool gathered, int n_chunks, int nstage, long long limit,
                                               uint32_t rank, uint32_t tmem, uint32_t idesc, const uint64_t (&a0)[4], const uint64_t (&b0)[4],
-                                              uint32_t stage_bytes) {
+                                              uint32_t stage_bytes, uint32_t leader = 0) {
+    // rank: this CTA's place in its pair (0 issues the MMAs); leader: the cluster rank of the pair's first CTA
+    const uint16_t mask = (uint16_t)(3u << leader);
     volatile int *failed = &B->failed;
     bool ok = true;
     if (rank == 0) {
@@ -192,7 +196,7 @@ __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool 
             int s2 = s1; uint32_t p2 = p1; next(s2, p2);
             int s3 = s2; uint32_t p3 = p2; next(s3, p3);
             // (probes past the last chunk look at stages that nothing refills: they answer "no" and are not used)
-            landed = pair_issue_two_stages(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &B->empty[s1], &full[s2], p2, &full[s3], p3);
+            landed = pair_issue_two_stages(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &B->empty[s1], &full[s2], p2, &full[s3], p3, mask);
             st = s2; ph = p2;
         }
         if (ok && c < n_chunks) {              // an odd chunk is left
@@ -203,13 +207,13 @@ __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool 
                 const uint64_t a[4] = {a0[0] + o0, a0[1] + o0, a0[2] + o0, a0[3] + o0};
                 const uint64_t b[4] = {b0[0] + o0, b0[1] + o0, b0[2] + o0, b0[3] + o0};
                 int s1 = st; uint32_t p1 = ph; next(s1, p1);
-                pair_issue_stage(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[s1], p1);
+                pair_issue_stage(tmem, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[s1], p1, mask);
             }
         }
         if (!ok) *failed = 1;
-        umma_commit_pair(&B->accbar);          // accumulators complete (or nothing was issued): told to both CTAs
+        umma_commit_pair(&B->accbar, mask);    // accumulators complete (or nothing was issued): told to both CTAs
     } else {
-        const uint32_t remote0 = map_to_cta(smem_u32(&full[0]), 0);
+        const uint32_t remote0 = map_to_cta(smem_u32(&full[0]), leader);
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % nstage; const uint32_t ph = (c / nstage) & 1;
             ok = mbar_wait(&full[st], ph, limit);
@@ -367,7 +371,34 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
     pair_teardown(tmem, ncols);
 }
 
-// y for this CTA's 128 tokens x N columns, straight from tensor memory (residual added, rounded to the output type).
+// Sixteen consecutive output columns of one token: residual added, rounded to the output type, written.
+__device__ __forceinline__ void down_store16(const GemmParams &P, size_t o, float (&a)[16]) {
+    if (P.residual) {
+        const uint4 x0 = *reinterpret_cast<const uint4 *>(P.x + o), x1 = *reinterpret_cast<const uint4 *>(P.x + o + 8);
+        const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            a[2 * j] += P.fmt ? si_cvt<SI_BF16>::lo(xw[j]) : si_cvt<SI_F16>::lo(xw[j]);
+            a[2 * j + 1] += P.fmt ? si_cvt<SI_BF16>::hi(xw[j]) : si_cvt<SI_F16>::hi(xw[j]);
+        }
+    }
+    if (P.y_f32) {
+        float4 *yo = reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + o);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) yo[j] = make_float4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
+    } else {
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            w[j] = P.fmt ? ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j + 1]) << 16))
+                         : ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j + 1]) << 16));
+        uint4 *yo = reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(P.y) + o);
+        yo[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        yo[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+}
+
+// y for this CTA's 128 tokens x N columns, straight from tensor memory.
 template <int N>
 __device__ __forceinline__ void down_epilogue(const GemmParams &P, bool ok, int n_chunks, uint32_t tmem, int warp, int lane, int tok0, int ct) {
     constexpr int kHalfCols = N / 2;
@@ -384,35 +415,62 @@ __device__ __forceinline__ void down_epilogue(const GemmParams &P, bool ok, int 
         float a[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) a[j] = n_chunks > 0 ? __uint_as_float(v[j]) : 0.f;
-        if (P.residual) {
-            const uint4 x0 = *reinterpret_cast<const uint4 *>(P.x + o0 + n0), x1 = *reinterpret_cast<const uint4 *>(P.x + o0 + n0 + 8);
-            const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+        down_store16(P, o0 + n0, a);
+    }
+}
+
+// The same when two pairs of a cluster of four CTAs have each summed half of K into their own accumulators of the
+// same 256-column tile (pair kq: K half kq): CTA (kq, r) finishes columns [kq * 128, kq * 128 + 128) of its 128 tokens.
+// It sends the other 128 columns of its accumulators to CTA (1 - kq, r) -- which holds the other K half of the same
+// tokens -- through distributed shared memory, receives that CTA's values for its own columns, and adds them in
+// K order.  The staging area is the pipeline stages, free once every CTA's MMAs are complete (first cluster barrier).
+__device__ __forceinline__ void down_epilogue_split(const GemmParams &P, uint8_t *smem, bool ok, int n_chunks, uint32_t tmem, int warp,
+                                                    int lane, int tok0, int ct, uint32_t kq, uint32_t rank) {
+    constexpr int kPitch = 128 + 4;                               // floats per staged token row
+    float *stg = reinterpret_cast<float *>(smem);                 // [128 tokens][kPitch]
+    const int q = warp & 3, half = warp >> 2;
+    const int row = q * 32 + lane, t = tok0 + row;
+    const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp < kLoaderWarps) {
+        tc_fence_after();
+        const uint32_t dst = map_to_cta(smem_u32(stg + (size_t)row * kPitch + half * 64), ((1u - kq) << 1) | rank);
+        for (int n0 = 0; n0 < 64; n0 += 16) {
+            uint32_t v[16];
+            if (n_chunks > 0) tmem_ld16(trow + (uint32_t)((1 - (int)kq) * 128 + half * 64 + n0), v);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                a[2 * j] += P.fmt ? si_cvt<SI_BF16>::lo(xw[j]) : si_cvt<SI_F16>::lo(xw[j]);
-                a[2 * j + 1] += P.fmt ? si_cvt<SI_BF16>::hi(xw[j]) : si_cvt<SI_F16>::hi(xw[j]);
-            }
+            for (int i = 0; i < 4; ++i)
+                st_cluster_v4(dst + (uint32_t)(n0 + 4 * i) * 4u, n_chunks > 0 ? v[4 * i] : 0u, n_chunks > 0 ? v[4 * i + 1] : 0u,
+                              n_chunks > 0 ? v[4 * i + 2] : 0u, n_chunks > 0 ? v[4 * i + 3] : 0u);
         }
-        if (P.y_f32) {
-            float4 *yo = reinterpret_cast<float4 *>(reinterpret_cast<float *>(P.y) + o0 + n0);
+        tc_fence_before();
+    }
+    cluster_sync_all();
+    if (warp < kLoaderWarps && ok) {
+        tc_fence_after();
+        const size_t o0 = (size_t)t * P.d_model + (size_t)ct * 256 + kq * 128 + half * 64;
+        for (int n0 = 0; n0 < 64; n0 += 16) {
+            uint32_t v[16];
+            if (n_chunks > 0) tmem_ld16(trow + (uint32_t)(kq * 128 + half * 64 + n0), v);
+            if (t >= P.T) continue;
+            const float *rv = stg + (size_t)row * kPitch + half * 64 + n0;
+            float a[16];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) yo[j] = make_float4(a[4 * j], a[4 * j + 1], a[4 * j + 2], a[4 * j + 3]);
-        } else {
-            uint32_t w[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                w[j] = P.fmt ? ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_BF16>::from_float(a[2 * j + 1]) << 16))
-                             : ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j]) | ((uint32_t)si_cvt<SI_F16>::from_float(a[2 * j + 1]) << 16));
-            uint4 *yo = reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(P.y) + o0 + n0);
-            yo[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            yo[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            for (int j = 0; j < 16; ++j) {
+                const float own = n_chunks > 0 ? __uint_as_float(v[j]) : 0.f;
+                a[j] = kq == 0 ? own + rv[j] : rv[j] + own;       // K half 0 first, whoever adds
+            }
+            down_store16(P, o0 + n0, a);
         }
     }
 }
 
-// Down contraction: one pair per (N output columns, 256 tokens); N = P.pair_n (128 or 256), half of them per CTA.
-template <int N>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+// Down contraction: one pair per (N output columns, 256 tokens); N = 128 or 256, half of them per CTA.  KS = 2: a
+// cluster of four CTAs -- two pairs -- works on a tile, each pair on half of K (N = 256 only).
+template <int N, int KS>
+__global__ void __cluster_dims__(2 * KS, 1, 1) __launch_bounds__(kGemmThreads, 1)
 si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap h_map,
                     const __grid_constant__ CUtensorMap rec_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -424,22 +482,28 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
     PairBars *B = reinterpret_cast<PairBars *>(smem + (size_t)P.nstage * stage_bytes);
     volatile int *failed = &B->failed;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t rank = cluster_ctarank();
+    static_assert(KS == 1 || N == 256, "the K split finishes 128 columns per pair");
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t rank = crank & 1u, kq = crank >> 1, leader = crank & ~1u;   // place in the pair, K share of the pair, first CTA of the pair
     constexpr uint32_t ncols = N;
     const uint32_t tmem = pair_setup(B, P.nstage, ncols, rank);
+    bool ok = true;                             // (loader / epilogue threads) no wait of this thread ran out
 
     pdl_wait();                                 // H (and, through the gate/up kernel's own wait, the union)
     pdl_launch();
-    const int pair = blockIdx.x >> 1;
+    const int tile = blockIdx.x / (2 * KS);
     const int col_tiles = P.d_model / N;
-    const int ct = pair % col_tiles, tp = pair / col_tiles;
+    const int ct = tile % col_tiles, tp = tile / col_tiles;
     const int n_u = *P.n_union;
-    const int n_chunks = (n_u + kChunkK - 1) / kChunkK;           // 64 union entries per chunk
+    const int all_chunks = (n_u + kChunkK - 1) / kChunkK;         // 64 union entries per chunk
+    const int per = (all_chunks + KS - 1) / KS;
+    const int c_lo = (int)kq * per;                                // this pair's share of K
+    const int n_chunks = all_chunks - c_lo < per ? (all_chunks > c_lo ? all_chunks - c_lo : 0) : per;
     const int tok0 = tp * kPairTokens + (int)rank * 128;
     // a union that is one run of consecutive slots (a static prefix, a whole layer) needs no gather: the down rows of
     // a chunk are tensor copies out of the record matrix (64 slots x 64 columns each)
     const int slot_first = P.union_slots[0];
-    const bool run = n_chunks > 0 && P.union_slots[n_chunks * kChunkK - 1] - slot_first == n_chunks * kChunkK - 1;
+    const bool run = all_chunks > 0 && P.union_slots[all_chunks * kChunkK - 1] - slot_first == all_chunks * kChunkK - 1;
     uint64_t *full = run ? B->full_t : B->full_g;
 
     if (warp < kLoaderWarps && run) {
@@ -452,22 +516,22 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
                 uint8_t *stage = tiles + (size_t)st * stage_bytes;
                 armed = c + 1;
                 mbar_arrive_expect_tx(&full[st], (uint32_t)stage_bytes);
-                tma_load_tile(stage, &h_map, c * kChunkK, tok0, &full[st]);
+                tma_load_tile(stage, &h_map, (c_lo + c) * kChunkK, tok0, &full[st]);
 #pragma unroll
                 for (int hh = 0; hh < kHalfCols / 64; ++hh)
-                    tma_load_tile(stage + 128 * 128 + hh * 8192, &rec_map, col0 + hh * 64, slot_first + c * kChunkK, &full[st]);
+                    tma_load_tile(stage + 128 * 128 + hh * 8192, &rec_map, col0 + hh * 64, slot_first + (c_lo + c) * kChunkK, &full[st]);
                 if (tp == 0 && c + kPrefetchAhead < n_chunks)
 #pragma unroll
                     for (int hh = 0; hh < kHalfCols / 64; ++hh)
-                        tma_prefetch_tile(&rec_map, col0 + hh * 64, slot_first + (c + kPrefetchAhead) * kChunkK);
+                        tma_prefetch_tile(&rec_map, col0 + hh * 64, slot_first + (c_lo + c + kPrefetchAhead) * kChunkK);
             }
         }
-        bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
+        ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
         if (!ok && armed > 0)                // a wait ran out: the tensor copies this thread started must still land before the CTA goes
             for (int c = armed - 1; c >= 0 && c > armed - 1 - P.nstage; c -= 2)
                 mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
-        down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
+        if (KS == 1) down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (warp < kLoaderWarps) {
         // Copy j of a thread covers 16-byte piece `pc` of the down-row segment of chunk entry kk = kEntStep*j + e.
@@ -482,14 +546,14 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         int armed = 0;
         int slots_next[kCopies];                                   // union slots of the next chunk (fetched one chunk ahead)
 #pragma unroll
-        for (int j = 0; j < kCopies; ++j) slots_next[j] = n_chunks > 0 ? P.union_slots[kEntStep * j + e] : 0;
+        for (int j = 0; j < kCopies; ++j) slots_next[j] = n_chunks > 0 ? P.union_slots[c_lo * kChunkK + kEntStep * j + e] : 0;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % P.nstage; const uint32_t ph = (c / P.nstage) & 1;
             int slots[kCopies];
 #pragma unroll
             for (int j = 0; j < kCopies; ++j) {                     // padded entries carry a valid slot
                 slots[j] = slots_next[j];
-                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c + 1) * kChunkK + kEntStep * j + e];
+                if (c + 1 < n_chunks) slots_next[j] = P.union_slots[(c_lo + c + 1) * kChunkK + kEntStep * j + e];
             }
             if (!mbar_wait_relaxed(&B->empty[st], ph ^ 1, P.spin_limit, 32)) { *failed = 1; break; }
             uint8_t *stage = tiles + (size_t)st * stage_bytes;
@@ -499,17 +563,17 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
             if (tid == 0) {
                 armed = c + 1;
                 mbar_arrive_expect_tx(&full[st], 128u * 128u);
-                tma_load_tile(stage, &h_map, c * kChunkK, tok0, &full[st]);
+                tma_load_tile(stage, &h_map, (c_lo + c) * kChunkK, tok0, &full[st]);
             }
             cp_async_arrive_when_landed(&full[st]);
         }
         cp_async_wait_all();
-        bool ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
+        ok = mbar_wait_relaxed(&B->accbar, 0, P.spin_limit, 256) && !*failed;
         if (!ok && armed > 0)                // a wait ran out: the tensor copies already started must still land before the CTA goes
             for (int c = armed - 1; c >= 0 && c > armed - 1 - P.nstage; --c)
                 mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
-        down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
+        if (KS == 1) down_epilogue<N>(P, ok, n_chunks, tmem, warp, lane, tok0, ct);
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (lane == 0) {
         const uint32_t idesc = make_idesc(P.fmt, 0, 1, 256, N);
@@ -519,15 +583,16 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         for (int k4 = 0; k4 < 4; ++k4) {       // 16 union entries per MMA = two 8-entry groups of 1024 bytes
             a0[k4] = make_desc(sh + k4 * 32, 16, 1024); b0[k4] = make_desc(sw + k4 * 2048, 8192, 1024);
         }
-        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes);
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes, leader);
     }
+    if (KS == 2) down_epilogue_split(P, smem, ok, n_chunks, tmem, warp, lane, tok0, ct, kq, rank);
     pair_teardown(tmem, ncols);
 }
 
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pair(void (*kern)(KArgs...), int pairs, size_t smem, cudaStream_t stream, Args... args) {
+cudaError_t launch_pair(void (*kern)(KArgs...), int ctas, size_t smem, cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cfg.gridDim = dim3(ctas); cfg.blockDim = dim3(kGemmThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -572,16 +637,22 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
         if (rc) return rc;
         if (w == 96) {
             SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<96>, pairs96, smem, stream, P, x_map, rec_map));
+            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<96>, 2 * pairs96, smem, stream, P, x_map, rec_map));
         } else {
             SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<128>, pairs128, smem, stream, P, x_map, rec_map));
+            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<128>, 2 * pairs128, smem, stream, P, x_map, rec_map));
         }
     }
     {
-        // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs: take 256 only when that
-        // still puts a pair on most SM pairs
-        const int n = d % 256 == 0 && (d / 256) * tok_pairs * 2 >= s->num_sms * 3 / 4 ? 256 : 128;
+        // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs.  When tiles of 256 columns
+        // would leave most SM pairs without one, two pairs share a tile of 256, half of K each (a cluster of four CTAs
+        // that exchanges its partial accumulators through distributed shared memory) -- as long as that is one wave and
+        // K is long enough to pay for the exchange (measured at 512 tokens: level at 50 chunks of K, 6 % ahead at 72,
+        // 18 % at 121); tiles of 128 columns otherwise.
+        const int tiles256 = d % 256 == 0 ? (d / 256) * tok_pairs : 0;
+        const bool fills = tiles256 > 0 && tiles256 * 2 >= s->num_sms * 3 / 4;
+        const bool split = tiles256 > 0 && !fills && tiles256 * 4 <= s->num_sms && P.nu_pad / kChunkK >= 64;
+        const int n = fills || split ? 256 : 128;
         P.pair_n = n;
         const size_t stage = 128 * 128 + (size_t)64 * n;
         P.nstage = stages_for(stage);
@@ -591,12 +662,15 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
         if (rc) return rc;
         rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, 64);
         if (rc) return rc;
-        if (n == 256) {
-            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256>, (d / 256) * tok_pairs, smem, stream, P, h_map, rec_map));
+        if (split) {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 2>, 4 * tiles256, smem, stream, P, h_map, rec_map));
+        } else if (n == 256) {
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 1>, 2 * tiles256, smem, stream, P, h_map, rec_map));
         } else {
-            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<128>, (d / 128) * tok_pairs, smem, stream, P, h_map, rec_map));
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<128, 1>, 2 * (d / 128) * tok_pairs, smem, stream, P, h_map, rec_map));
         }
     }
     SI_CUDA_TRY(cudaGetLastError());
