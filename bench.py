@@ -316,7 +316,7 @@ def extra_configs(api, torch, args, device, peaks, peak_kind):
             cells.append({"batch": B, "tokens_per_s": tok_s, "us_per_layer_call": us_call, "mean_union": u,
                           "union_overlap": 1.0 - u / (B * cfg3.k_active), "union_coverage_of_loaded": u / cfg3.n_loaded,
                           "union_gbs": ubytes / us_call / 1e3, "frac": ubytes / us_call / 1e3 / hbm,
-                          "route": "decode kernel, token by token" if B <= 4 else "union + tensor-core contractions",
+                          "route": "decode kernel, token by token" if B <= 4 else "union + tensor-core contractions (K split over thread-block clusters)",
                           "replayed_from_cuda_graph": was_graph})
         out["c3"] = {"workload": "c3: 7B-shaped stack (d_model=4096, d_ff=11008, bf16, 7705 loaded), own 1541-slot Zipf list per "
                                  "token, batch sizes 1..32; measured on 4 layers (757 MB of records), tokens/s scaled to 32 layers",
@@ -332,7 +332,14 @@ def extra_configs(api, torch, args, device, peaks, peak_kind):
                      "tokens_per_s": cfg4.tokens / (us_call * 1e-6 * cfg4.n_layers), "us_per_layer_call": us_call,
                      "bound": "tensor", "achieved_tflops": tflops, "peak": peaks["bf16_tflops_sustained"],
                      "frac": tflops / peaks["bf16_tflops_sustained"], "peak_kind": f"of {peak_kind} (sustained)",
-                     "replayed_from_cuda_graph": was_graph}
+                     "replayed_from_cuda_graph": was_graph,
+                     "kernels": "CTA pairs (tcgen05.mma.cta_group::2): tokens on M, store columns on N, weight tiles by tensor copies"}
+        # the same call over ALL loaded neurons (what the prefill of a prompt runs before it votes: Section 5)
+        cfg4a = cfg4.with_(active_pct=100)
+        us_all, _, _ = multitoken(cfg4a, cfg4a.tokens, 4, 1, True)
+        tf_all = 6.0 * cfg4a.d_model * cfg4a.k_active * cfg4a.tokens / us_all / 1e6
+        out["c4"]["all_loaded"] = {"k": cfg4a.k_active, "us_per_layer_call": us_all, "achieved_tflops": tf_all,
+                                   "frac": tf_all / peaks["bf16_tflops_sustained"]}
     except Exception as e:                              # pragma: no cover
         out["c4"] = {"error": repr(e)}
 
