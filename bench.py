@@ -316,7 +316,7 @@ def extra_configs(api, torch, args, device, peaks, peak_kind):
             cells.append({"batch": B, "tokens_per_s": tok_s, "us_per_layer_call": us_call, "mean_union": u,
                           "union_overlap": 1.0 - u / (B * cfg3.k_active), "union_coverage_of_loaded": u / cfg3.n_loaded,
                           "union_gbs": ubytes / us_call / 1e3, "frac": ubytes / us_call / 1e3 / hbm,
-                          "route": "decode kernel, token by token" if B <= 4 else "union + tensor-core contractions (K split over thread-block clusters)",
+                          "route": "decode kernel" if B == 1 else "union + tensor-core contractions (K split over thread-block clusters)",
                           "replayed_from_cuda_graph": was_graph})
         out["c3"] = {"workload": "c3: 7B-shaped stack (d_model=4096, d_ff=11008, bf16, 7705 loaded), own 1541-slot Zipf list per "
                                  "token, batch sizes 1..32; measured on 4 layers (757 MB of records), tokens/s scaled to 32 layers",
@@ -715,7 +715,7 @@ def run_multitoken(args, cfg, rank, world, local_rank):
             lists[:, l] = ll.reshape(n_groups, T, k)
         union_sizes = [len(np.unique(lists[g, l])) for g in range(n_groups) for l in range(min(L, 4))]
         idx = torch.from_numpy(lists).cuda()
-        flags = api.SI_FLAG_UNION_PATH     # config 3 is about the union path (few tokens would otherwise take the decode route)
+        flags = api.SI_FLAG_UNION_PATH     # config 3 is about the union path (a single token would otherwise take the decode kernel)
     y = torch.empty(n_groups, L, T, d, dtype=tdt, device="cuda")
     ws = store.workspace(T, k, 1)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")

@@ -76,9 +76,8 @@ enum {
     SI_FLAG_UNION_UNMASKED = 4u, /* T > 1 only: every token uses the whole union (extension) */
     SI_FLAG_SCORE_ABS = 8u,      /* si_select: rank |score| instead of score */
     SI_FLAG_SHARED_LIST = 16u,   /* T > 1 only: idx is ONE list of k_fixed slots used by every token */
-    SI_FLAG_UNION_PATH = 32u,    /* T > 1 only: always form the union and run the tensor-core contractions
-                                    (by default up to 4 tokens with lists of their own go through the
-                                    batch-1 decode kernel one after the other, which is faster there) */
+    SI_FLAG_UNION_PATH = 32u,    /* si_ffn_forward: form the union and run the tensor-core contractions also for a
+                                    single token (calls with more than one token always do) */
     SI_FLAG_LIST_PER_LAYER = 64u, /* si_decode_stack_forward, fixed-length lists only: idx holds ONE list per layer
                                     ([n_layers, k_fixed]) and every step uses the list of its layer -- the paper's
                                     decode, where the set chosen during prefill stays fixed for the prompt */
@@ -171,10 +170,9 @@ int si_select(const float *scores, int n, int mode, int k, float tau, unsigned f
  *   y   : device [T, d_model] of y_dtype (SI_F32, or the store dtype)
  * T == 1 runs the memory-bound decode kernel; T > 1 forms the union of the lists and
  * runs a gathered tensor-core contraction in which token t still uses exactly its own
- * list (unless SI_FLAG_UNION_UNMASKED).  Up to 4 tokens with lists of their own are taken
- * through the decode kernel one after the other instead, which is faster there; the result
- * is the same function of the inputs, and SI_FLAG_UNION_PATH forces the union path (also for a
- * single token; the workspace must then be sized for T_max = 2).  An
+ * list (unless SI_FLAG_UNION_UNMASKED); this path needs d_model % 128 == 0
+ * (SI_ERR_UNSUPPORTED otherwise).  SI_FLAG_UNION_PATH forces the union path for a single
+ * token as well (the workspace must then be sized for T_max = 2).  An
  * empty list gives y = 0 (or x with SI_FLAG_RESIDUAL).  Accumulation is fp32; h is rounded
  * to the store dtype before the down projection only on the union path. */
 int si_ffn_forward(const si_store_t *store, int layer, const void *x, int T, const int32_t *idx,

@@ -72,24 +72,10 @@ extern "C" int si_ffn_forward(const si_store_t *store, int layer, const void *x,
         return si_decode_launch(store, 1, &l, x, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
                                 ws_bytes, status_dev, stream);
     }
-    // A few tokens with lists of their own: one persistent decode launch that takes the tokens one
-    // after the other streams T * k records at full speed and is faster than forming the union and
-    // running the two contractions, whose fixed parts weigh more than the records the union saves
-    // (measured: 40 us against 49 us at T = 4, 62 against 57 at T = 8 on a 7B-shaped layer).
-    constexpr int kDecodeRouteMaxT = 4;
-    if (T <= kDecodeRouteMaxT && !(flags & (SI_FLAG_SHARED_LIST | SI_FLAG_UNION_UNMASKED | SI_FLAG_UNION_PATH)) &&
-        si_persistent_supported(store)) {
-        // lists handed over inside the workspace (si_layer_forward) must lie outside the decode layout
-        const size_t decode_total = si_ws_carve(store, 1, k_fixed, T).total;
-        const char *w0 = (const char *)workspace, *ip = (const char *)idx;
-        if (!(ip >= w0 && ip < w0 + decode_total)) {
-            int32_t ls[kDecodeRouteMaxT];
-            for (int t = 0; t < T; ++t) ls[t] = layer;
-            // the tokens of a call are independent of one another by definition
-            return si_decode_launch(store, T, ls, x, idx, idx_offsets, k_fixed, y, y_dtype, flags | SI_FLAG_STEPS_ANY_ORDER,
-                                    workspace, ws_bytes, status_dev, stream);
-        }
-    }
+    // (Taking a few tokens through the decode kernel one after the other was faster than the union path while that
+    // path summed its K splits through global memory: 37.0 against 42.9 us at T = 4 on a 7B-shaped layer.  With the
+    // cluster sums it is the other way round -- 31.3 against 37.0 us at T = 4, 25.5 against 27.6 at T = 2 -- so every
+    // call with more than one token forms the union.)
     return si_multi_token_launch(store, layer, x, T, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace,
                                  ws_bytes, status_dev, stream);
 }

@@ -60,8 +60,8 @@ def test_union_is_bit_exact(api, c1):
 
 @pytest.mark.parametrize("T", [2, 4, 16])
 def test_c1_multitoken_matches_per_token_oracle(api, c1, T):
-    """Both routes for a few tokens: the default (decode kernel token by token up to 4 tokens) and
-    the union path forced by its flag."""
+    """A few tokens, with and without the flag that forces the union path (which every call with more than one token
+    takes anyway)."""
     cfg = c1.cfg
     lists = wl.zipf_lists(cfg, 0, T, slot_of_rank=c1.slot_of_rank[0])
     x = wl.x_tokens(cfg, 0, T)
