@@ -6,13 +6,14 @@
 // per CTA; N = 256 or 128 store columns, each CTA holding half of them in its shared memory), so every CTA
 // loads its own 128 tokens and only HALF of the weight tile the pair multiplies them with:
 //
-//   gate/up   D[256 tokens x (128 gate | 128 up)] = X[tokens, k] . W[U tile, k]^T     (K = d_model)
+//   gate/up   D[256 tokens x (W gate | W up)] = X[tokens, k] . W[U tile, k]^T         (K = d_model; W = 128 or 96)
 //             CTA 0 of the pair loads the tile's gate rows, CTA 1 its up rows; a thread of the epilogue owns
 //             one token and finds gate and up of a neuron in its own registers: H = member . SiLU(g) . u
 //   down      D[256 tokens x N columns] = H[tokens, U_k] . Wd[U_k, columns]           (K = |U|)
 //             CTA r loads columns r * N/2 .. of the 64 down rows of a chunk (MN-major operand)
 //
-// No K split and no partial tiles: H and y are written straight from tensor memory.  Each CTA tracks the
+// No partial tiles in global memory: H and y are written straight from tensor memory (with a long K, two pairs
+// share a down tile, half of K each, and exchange their accumulators through distributed shared memory).  Each CTA tracks the
 // stages of its own shared memory with local mbarriers, exactly as the one-CTA kernels do; the pair is coupled
 // by two signals only: the second CTA's MMA warp relays "my half of stage s has landed" to a barrier of the
 // first (the one that issues the MMAs), and the commit that frees a stage (or declares the accumulators
