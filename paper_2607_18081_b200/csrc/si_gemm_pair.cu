@@ -122,6 +122,36 @@ __device__ __forceinline__ uint32_t pair_issue_two_stages(uint32_t d_tmem, const
     return landed;
 }
 
+// One stage of a tile that is two sub-tiles wide (two accumulators, one A operand): the probe of the next stage, the
+// four MMAs of the first sub-tile, the four of the second (same A descriptors, B descriptors b[4..7], accumulator d1),
+// one commit, the probe's answer.
+__device__ __forceinline__ bool pair_issue_wide_stage(uint32_t d0, uint32_t d1, const uint64_t (&a)[4], const uint64_t (&b)[8], uint32_t idesc,
+                                                      uint32_t accumulate_first, uint64_t *empty_bar, uint64_t *next_full, uint32_t next_parity,
+                                                      uint16_t mask) {
+    uint32_t landed;
+    asm volatile(
+        "{\n\t.reg .pred q, p, t;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 q, [%17], %18;\n\t"
+        "setp.ne.b32 p, %15, 0;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %3, %7, %16, p;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%2], %3, %11, %16, p;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %4, %8, %16, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%2], %4, %12, %16, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %5, %9, %16, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%2], %5, %13, %16, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%1], %6, %10, %16, t;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%2], %6, %14, %16, t;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%19], %20;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(landed)
+        : "r"(d0), "r"(d1), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]),
+          "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7]), "r"(accumulate_first), "r"(idesc), "r"(smem_u32(next_full)), "r"(next_parity),
+          "r"(smem_u32(empty_bar)), "h"(mask)
+        : "memory");
+    return landed != 0;
+}
+
 struct PairBars {
     // stage landed.  In the pair's first CTA one arrival more is expected: the second CTA's word that ITS half has landed
     uint64_t full_t[kPairMaxStages];     // ... tensor copies only (one arrival: the thread that starts them)
@@ -173,12 +203,33 @@ __device__ __forceinline__ void pair_teardown(uint32_t tmem, uint32_t ncols) {
 // one ahead of it is nearly done, so whatever the thread does between two stages the tensor pipe waits for.
 __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool gathered, int n_chunks, int nstage, long long limit,
                                               uint32_t rank, uint32_t tmem, uint32_t idesc, const uint64_t (&a0)[4], const uint64_t (&b0)[4],
-                                              uint32_t stage_bytes, uint32_t leader = 0) {
-    // rank: this CTA's place in its pair (0 issues the MMAs); leader: the cluster rank of the pair's first CTA
+                                              uint32_t stage_bytes, uint32_t leader = 0, uint32_t wide_b_bytes = 0,
+                                              uint32_t wide_d_cols = 0) {
+    // rank: this CTA's place in its pair (0 issues the MMAs); leader: the cluster rank of the pair's first CTA;
+    // wide_b_bytes != 0: the tile is two sub-tiles wide -- the second sub-tile's B rows lie wide_b_bytes further on
+    // in a stage, its accumulator wide_d_cols columns further on in tensor memory
     const uint16_t mask = (uint16_t)(3u << leader);
     volatile int *failed = &B->failed;
     bool ok = true;
-    if (rank == 0) {
+    if (rank == 0 && wide_b_bytes) {
+        bool landed = false;
+        int st = 0; uint32_t ph = 0;
+        const uint64_t step = (uint64_t)(stage_bytes >> 4), sub = (uint64_t)(wide_b_bytes >> 4);
+        for (int c = 0; c < n_chunks; ++c) {
+            if (!landed) ok = mbar_wait_cluster(&full[st], ph, limit);
+            if (!ok) break;
+            if (gathered) { fence_async_proxy(); tc_fence_after(); }
+            const uint64_t o = step * (uint64_t)st;
+            const uint64_t a[4] = {a0[0] + o, a0[1] + o, a0[2] + o, a0[3] + o};
+            const uint64_t b[8] = {b0[0] + o, b0[1] + o, b0[2] + o, b0[3] + o, b0[0] + o + sub, b0[1] + o + sub, b0[2] + o + sub, b0[3] + o + sub};
+            int s1 = st; uint32_t p1 = ph;
+            if (++s1 == nstage) { s1 = 0; p1 ^= 1u; }
+            landed = pair_issue_wide_stage(tmem, tmem + wide_d_cols, a, b, idesc, c ? 1u : 0u, &B->empty[st], &full[s1], p1, mask);
+            st = s1; ph = p1;
+        }
+        if (!ok) *failed = 1;
+        umma_commit_pair(&B->accbar, mask);
+    } else if (rank == 0) {
         // stages are issued two at a time; `landed` bit 0 / 1: the probe of the first / second of the two was answered "yes"
         uint32_t landed = 0;
         int st = 0; uint32_t ph = 0;
@@ -226,26 +277,29 @@ __device__ __forceinline__ void pair_mma_loop(PairBars *B, uint64_t *full, bool 
     }
 }
 
-// H for this CTA's 128 tokens x the tile's W neurons, straight from tensor memory: thread = token (lane of the
-// tensor memory), gate in columns [0, W), up in [W, 2W); warps w and w + 4 share the lanes and take W / 2 neurons
+// H for this CTA's 128 tokens x the tile's S * W neurons, straight from tensor memory: thread = token (lane of the
+// tensor memory); sub-tile s has its gate values in columns [s * 2W, s * 2W + W) and its up values in the W columns
+// after them.  Warps w and w + 4 share the lanes: with one sub-tile they take W / 2 neurons each, with two a sub-tile
 // each.  Written without a branch per element: SiLU(g) * u is formed for every element and kept or zeroed by a select.
-template <int DT, int W>
+template <int DT, int W, int S>
 __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tmem, int warp, int lane, int tok0, int nt, int n_u) {
     const int q = warp & 3, half = warp >> 2;
     const int t = tok0 + q * 32 + lane;
-    const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
-    const int i0 = nt * W + (W / 2) * half;                       // union position of this thread's first neuron
+    constexpr int kCount = S == 1 ? W / 2 : W;                    // neurons of this thread
+    const int sub = S == 1 ? 0 : half, r0 = S == 1 ? (W / 2) * half : 0;
+    const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(sub * 2 * W + r0);
+    const int i0 = nt * S * W + sub * W + r0;                     // union position of this thread's first neuron
     uint16_t *hrow = P.h_out + (size_t)t * P.nu_pad + i0;
     const bool has_row = t < P.t_pad_total;                       // H has rows for the tokens padded to 16 only (no early
                                                                   // return: the tensor-memory loads below are warp-wide)
     const int lim = t < P.T ? n_u - i0 : 0;                       // positions below lim are real entries of a real token
     const bool own = P.tokbits != nullptr;                        // (uniform) every token keeps to its own list
     const uint32_t *tb = own ? P.tokbits + (size_t)(t < P.T ? t : 0) * P.mask_words : nullptr;
-    for (int n0 = 0; n0 < W / 2; n0 += 16) {
-        if (i0 + n0 >= P.nu_pad) break;                           // (a last tile of 96 may reach past the padded union)
+    for (int n0 = 0; n0 < kCount; n0 += 16) {
+        if (i0 + n0 >= P.nu_pad) break;                           // (a last tile may reach past the padded union)
         uint32_t g[16], u[16];
-        tmem_ld16(trow + (uint32_t)((W / 2) * half + n0), g);
-        tmem_ld16(trow + (uint32_t)(W + (W / 2) * half + n0), u);
+        tmem_ld16(trow + (uint32_t)n0, g);
+        tmem_ld16(trow + (uint32_t)(W + n0), u);
         uint32_t member = 0xFFFFu;                                // bit j: the token selected neuron n0 + j
         if (own) {
             member = 0;
@@ -269,38 +323,41 @@ __device__ __forceinline__ void gateup_epilogue(const GemmParams &P, uint32_t tm
     }
 }
 
-// Gate/up contraction: one pair per (union tile of W neurons, 256 tokens); W = 128, or 96 when that puts a tile on
-// more of the SM pairs (N of the MMA = 2 W: the tile's gate rows and up rows).
-template <int W>
+// Gate/up contraction: one pair per (union tile of S * W neurons, 256 tokens).  N of an MMA = 2 W: the gate rows and
+// the up rows of W neurons; S = 2: the tile is two such sub-tiles with an accumulator each, which share the X tile
+// (less operand traffic per MMA cycle, and half as many tiles: large unions in one wave instead of two).  The host
+// picks (W, S) by cost: waves of pair tiles over the SM pairs x the MMA time of a tile's chunk.
+template <int W, int S>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constant__ CUtensorMap x_map,
                       const __grid_constant__ CUtensorMap rec_map) {
     extern __shared__ __align__(1024) uint8_t smem[];
-    constexpr int stage_bytes = 128 * 128 + W * 128;              // this CTA's X tile, this CTA's W weight rows
+    constexpr int R = S * W;                                      // weight rows of a tile (per CTA: the gate rows, or the up rows)
+    constexpr int stage_bytes = 128 * 128 + R * 128;              // this CTA's X tile, this CTA's R weight rows
     uint8_t *tiles = smem;
     PairBars *B = reinterpret_cast<PairBars *>(smem + (size_t)P.nstage * stage_bytes);
     volatile int *failed = &B->failed;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();
-    constexpr uint32_t ncols = 256;                               // W gate + W up accumulator columns
+    constexpr uint32_t ncols = S == 1 ? 256 : 512;                // per sub-tile W gate + W up accumulator columns
     const uint32_t tmem = pair_setup(B, P.nstage, ncols, rank);
 
     pdl_wait();                                 // the union kernel's results
     pdl_launch();
     const int pair = blockIdx.x >> 1;
-    const int n_tiles = (P.nu_pad + W - 1) / W;
+    const int n_tiles = (P.nu_pad + R - 1) / R;
     const int nt = pair % n_tiles, tp = pair / n_tiles;
     const int n_u = *P.n_union;
     // tiles past the real union have nothing to do (the down contraction reads H in chunks of 64 entries: up to there
     // H must be written)
-    const bool active = nt * W < (n_u + kChunkK - 1) / kChunkK * kChunkK;
+    const bool active = nt * R < (n_u + kChunkK - 1) / kChunkK * kChunkK;
     const int n_chunks = active ? P.d_model / kChunkK : 0;
     const int tok0 = tp * kPairTokens + (int)rank * 128;          // this CTA's tokens
-    // union entry of tile row r (a last tile of 96 may reach past the padded union: its surplus rows repeat the last entry)
-    auto entry = [&](int r) { const int e = nt * W + r; return e < P.nu_pad ? e : P.nu_pad - 1; };
-    // a tile of W consecutive slots needs no gather: its rows are one tensor copy out of the record matrix
+    // union entry of tile row r (a last tile may reach past the padded union: its surplus rows repeat the last entry)
+    auto entry = [&](int r) { const int e = nt * R + r; return e < P.nu_pad ? e : P.nu_pad - 1; };
+    // a tile of R consecutive slots needs no gather: its rows are one tensor copy out of the record matrix
     const int slot_first = P.union_slots[entry(0)];
-    const bool run = nt * W + W <= P.nu_pad && P.union_slots[nt * W + W - 1] - slot_first == W - 1;
+    const bool run = nt * R + R <= P.nu_pad && P.union_slots[nt * R + R - 1] - slot_first == R - 1;
     uint64_t *full = run ? B->full_t : B->full_g;
     const bool withhold = P.withhold && blockIdx.x == 0;
 
@@ -329,9 +386,9 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
             // copy j of a thread covers 16-byte piece (tid & 7) of tile row 32*j + (tid >> 3): a warp instruction
             // reads four whole 128-byte row segments
             const int q8 = tid & 7, r32 = tid >> 3;
-            const char *wrow[W / 32];
+            const char *wrow[R / 32];
 #pragma unroll
-            for (int j = 0; j < W / 32; ++j)
+            for (int j = 0; j < R / 32; ++j)
                 wrow[j] = P.rec_base + (size_t)P.union_slots[entry(32 * j + r32)] * P.rec_bytes + (size_t)rank * P.d_model * 2 + q8 * 16;
             const int off0 = r32 * 128 + ((q8 ^ (r32 & 7)) << 4);
             for (int c = 0; c < n_chunks; ++c) {
@@ -340,7 +397,7 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 uint8_t *stage = tiles + (size_t)st * stage_bytes;
                 uint8_t *sw = stage + 128 * 128 + off0;
 #pragma unroll
-                for (int j = 0; j < W / 32; ++j) { cp_async16(sw + j * 4096, wrow[j]); wrow[j] += 128; }
+                for (int j = 0; j < R / 32; ++j) { cp_async16(sw + j * 4096, wrow[j]); wrow[j] += 128; }
                 if (tid == 0 && !(withhold && c == 0)) {
                     armed = c + 1;
                     mbar_arrive_expect_tx(&full[st], 128u * 128u);
@@ -357,8 +414,8 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
                 mbar_wait(&full[c % P.nstage], (c / P.nstage) & 1, P.spin_limit);
         tc_fence_after();
         if (ok && active) {
-            if (P.fmt) gateup_epilogue<SI_BF16, W>(P, tmem, warp, lane, tok0, nt, n_u);
-            else gateup_epilogue<SI_F16, W>(P, tmem, warp, lane, tok0, nt, n_u);
+            if (P.fmt) gateup_epilogue<SI_BF16, W, S>(P, tmem, warp, lane, tok0, nt, n_u);
+            else gateup_epilogue<SI_F16, W, S>(P, tmem, warp, lane, tok0, nt, n_u);
         }
         if (!ok && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
     } else if (lane == 0) {
@@ -367,7 +424,8 @@ si_pair_gateup_kernel(const __grid_constant__ GemmParams P, const __grid_constan
         uint64_t a0[4], b0[4];
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4) { a0[k4] = make_desc(sx + k4 * 32, 16, 1024); b0[k4] = make_desc(sw + k4 * 32, 16, 1024); }
-        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes);
+        pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes, 0u,
+                      S == 2 ? (uint32_t)(W * 128) : 0u, (uint32_t)(2 * W));
     }
     pair_teardown(tmem, ncols);
 }
@@ -623,26 +681,36 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
     P.t_pad_total = t_pad_alloc; P.n_tok = kPairTokens; P.n_split = 1;
     P.h = (const uint16_t *)h_buf; P.h_out = (uint16_t *)h_buf;
     {
-        // tiles of 128 neurons, or of 96 when that costs less: cost = waves of pair tiles over the SM pairs x tile width
+        // tiles of W = 128 or 96 neurons, or of two sub-tiles of 128 or 112: cost = waves of pair tiles over the SM pairs x
+        // the MMA time of a tile's chunk (4 MMAs of N = 2 W per sub-tile: 4 S W cycles, plus what a stage costs besides)
         const int slots = s->num_sms / 2;
-        const int pairs128 = (P.nu_pad / 128) * tok_pairs, pairs96 = ((P.nu_pad + 95) / 96) * tok_pairs;
-        const int cost128 = ((pairs128 + slots - 1) / slots) * 128, cost96 = ((pairs96 + slots - 1) / slots) * 96;
-        const int w = cost96 < cost128 ? 96 : 128;
-        const size_t stage = 128 * 128 + (size_t)w * 128;
+        struct Shape { int w, sub; } shapes[] = {{128, 1}, {96, 1}, {128, 2}, {112, 2}};
+        int best = 0; long best_cost = -1; int best_pairs = 0;
+        for (int i = 0; i < 4; ++i) {
+            const int r = shapes[i].w * shapes[i].sub;
+            const int pairs = ((P.nu_pad + r - 1) / r) * tok_pairs;
+            const long cost = (long)((pairs + slots - 1) / slots) * (4 * r + 78);
+            if (best_cost < 0 || cost < best_cost) { best = i; best_cost = cost; best_pairs = pairs; }
+        }
+        const int w = shapes[best].w, sub = shapes[best].sub;
+        const size_t stage = 128 * 128 + (size_t)w * sub * 128;
         P.nstage = stages_for(stage);
         const size_t smem = (size_t)P.nstage * stage + sizeof(PairBars);
         CUtensorMap x_map, rec_map;
         int rc = make_tile_map(&x_map, P.x, (size_t)d, (size_t)P.T, (size_t)d * 2, 128);
         if (rc) return rc;
-        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, w);
+        rc = make_tile_map(&rec_map, P.rec_base, (size_t)3 * d, (size_t)n_loaded, (size_t)P.rec_bytes, w * sub);
         if (rc) return rc;
-        if (w == 96) {
-            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<96>, 2 * pairs96, smem, stream, P, x_map, rec_map));
-        } else {
-            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<128>, 2 * pairs128, smem, stream, P, x_map, rec_map));
-        }
+#define SI_LAUNCH_GATEUP(WW, SS)                                                                                                    \
+        do {                                                                                                                        \
+            SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_gateup_kernel<WW, SS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+            SI_CUDA_TRY(launch_pair(si_pair_gateup_kernel<WW, SS>, 2 * best_pairs, smem, stream, P, x_map, rec_map));               \
+        } while (0)
+        if (w == 128 && sub == 1) SI_LAUNCH_GATEUP(128, 1);
+        else if (w == 96) SI_LAUNCH_GATEUP(96, 1);
+        else if (w == 128) SI_LAUNCH_GATEUP(128, 2);
+        else SI_LAUNCH_GATEUP(112, 2);
+#undef SI_LAUNCH_GATEUP
     }
     {
         // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs.  When tiles of 256 columns
