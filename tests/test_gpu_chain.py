@@ -261,3 +261,28 @@ def test_contraction_wait_runs_out_and_the_next_call_is_correct(api, T, prefix):
     assert st.item() == 0
     for t in sorted({0, 1, T // 2, T - 1}):
         assert_close(from_dev(y[t]), m.oracle_y(0, x[t], lists[t]), f"after the time-out, token {t}")
+
+
+def test_wide_pair_tiles_wait_runs_out_and_the_next_call_is_correct(api):
+    """300 tokens over all loaded neurons of a 7B-shaped layer: gate/up tiles of two sub-tiles (two accumulators per
+    CTA) and a down contraction whose K is split between two pairs of a cluster of four.  The first pair's first X
+    tile is withheld: SI_ERR_TIMEOUT, a clean return, and a correct call afterwards."""
+    cfg = wl.CONFIGS["c2"]
+    m = LoadedModel(cfg, n_layers=1)
+    T, k = 300, cfg.n_loaded
+    shared = np.arange(k, dtype=np.int32)
+    x = wl.x_tokens(cfg, 0, T)
+    xd, idx = to_dev(x, cfg.dtype), torch.from_numpy(shared).cuda()
+    ws = m.store.workspace(T, k, 1)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.empty(T, cfg.d_model, dtype=torch.float32, device="cuda")
+    api.si_debug_ffn_forward_waits(m.store.handle, 0, xd, T, idx, None, k, y, api.SI_FLAG_SHARED_LIST, ws, st,
+                                   spin_limit=20_000, withhold=1)
+    torch.cuda.synchronize()
+    assert st.item() == api.SI_ERR_TIMEOUT
+    st.zero_()
+    api.si_ffn_forward(m.store.handle, 0, xd, T, idx, None, k, y, api.SI_FLAG_SHARED_LIST, ws, st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    for t in (0, 255, 299):
+        assert_close(from_dev(y[t]), m.oracle_y(0, x[t], shared), f"after the time-out, token {t}")
