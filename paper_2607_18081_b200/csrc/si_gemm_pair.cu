@@ -152,12 +152,20 @@ __device__ __forceinline__ bool pair_issue_wide_stage(uint32_t d0, uint32_t d1, 
     return landed != 0;
 }
 
+// `bytes` (a multiple of 16) from this CTA's shared memory into the shared memory of another CTA of the cluster; completion
+// is counted in bytes on an mbarrier of that CTA (both addresses from map_to_cta)
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, const void *src_smem, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(smem_u32(src_smem)), "r"(bytes), "r"(bar_cluster) : "memory");
+}
+
 struct PairBars {
     // stage landed.  In the pair's first CTA one arrival more is expected: the second CTA's word that ITS half has landed
     uint64_t full_t[kPairMaxStages];     // ... tensor copies only (one arrival: the thread that starts them)
     uint64_t full_g[kPairMaxStages];     // ... gathered rows + the dense tile (all loader threads + 1)
     uint64_t empty[kPairMaxStages];      // the MMAs have read the stage (both CTAs are told)
     uint64_t accbar;                     // accumulators complete (both CTAs are told)
+    uint64_t xbar;                       // (K split) the other pair's partial accumulators have arrived
     uint32_t tmem_slot;
     int failed;
 };
@@ -172,6 +180,7 @@ __device__ __forceinline__ uint32_t pair_setup(PairBars *B, int nstage, uint32_t
             mbar_init(&B->empty[s], 1);
         }
         mbar_init(&B->accbar, 1);
+        mbar_init(&B->xbar, 1);
         B->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -480,48 +489,63 @@ __device__ __forceinline__ void down_epilogue(const GemmParams &P, bool ok, int 
 
 // The same when two pairs of a cluster of four CTAs have each summed half of K into their own accumulators of the
 // same 256-column tile (pair kq: K half kq): CTA (kq, r) finishes columns [kq * 128, kq * 128 + 128) of its 128 tokens.
-// It sends the other 128 columns of its accumulators to CTA (1 - kq, r) -- which holds the other K half of the same
-// tokens -- through distributed shared memory, receives that CTA's values for its own columns, and adds them in
-// K order.  The staging area is the pipeline stages, free once every CTA's MMAs are complete (first cluster barrier).
-__device__ __forceinline__ void down_epilogue_split(const GemmParams &P, uint8_t *smem, bool ok, int n_chunks, uint32_t tmem, int warp,
-                                                    int lane, int tok0, int ct, uint32_t kq, uint32_t rank) {
+// It stages the other 128 columns of its accumulators in its own shared memory and sends them to CTA (1 - kq, r) --
+// which holds the other K half of the same tokens -- as one bulk copy through distributed shared memory (remote
+// stores from every thread took five times as long), receives that CTA's values for its own columns the same way,
+// and adds them in K order.  The staging areas are the pipeline stages, free once every CTA's MMAs are complete (the
+// cluster barrier below); a CTA leaves only after the last cluster barrier, i.e. after its own block has been received.
+__device__ __forceinline__ void down_epilogue_split(const GemmParams &P, uint8_t *smem, PairBars *B, bool ok, int n_chunks, uint32_t tmem,
+                                                    int warp, int lane, int tok0, int ct, uint32_t kq, uint32_t rank) {
     constexpr int kPitch = 128 + 4;                               // floats per staged token row
-    float *stg = reinterpret_cast<float *>(smem);                 // [128 tokens][kPitch]
+    constexpr uint32_t kBlockBytes = 128 * kPitch * 4;            // 67584
+    float *snd = reinterpret_cast<float *>(smem);                 // [128 tokens][kPitch]: what this CTA sends
+    float *rcv = reinterpret_cast<float *>(smem + 68 * 1024);     // ... and what it receives
+    const int tid = threadIdx.x;
     const int q = warp & 3, half = warp >> 2;
     const int row = q * 32 + lane, t = tok0 + row;
     const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();
+    if (tid == 0) mbar_arrive_expect_tx(&B->xbar, kBlockBytes);
     if (warp < kLoaderWarps) {
         tc_fence_after();
-        const uint32_t dst = map_to_cta(smem_u32(stg + (size_t)row * kPitch + half * 64), ((1u - kq) << 1) | rank);
+        float *srow = snd + (size_t)row * kPitch + half * 64;
         for (int n0 = 0; n0 < 64; n0 += 16) {
             uint32_t v[16];
             if (n_chunks > 0) tmem_ld16(trow + (uint32_t)((1 - (int)kq) * 128 + half * 64 + n0), v);
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                st_cluster_v4(dst + (uint32_t)(n0 + 4 * i) * 4u, n_chunks > 0 ? v[4 * i] : 0u, n_chunks > 0 ? v[4 * i + 1] : 0u,
-                              n_chunks > 0 ? v[4 * i + 2] : 0u, n_chunks > 0 ? v[4 * i + 3] : 0u);
+                *reinterpret_cast<uint4 *>(srow + n0 + 4 * i) = n_chunks > 0 ? make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3])
+                                                                              : make_uint4(0u, 0u, 0u, 0u);
         }
         tc_fence_before();
     }
-    cluster_sync_all();
-    if (warp < kLoaderWarps && ok) {
-        tc_fence_after();
-        const size_t o0 = (size_t)t * P.d_model + (size_t)ct * 256 + kq * 128 + half * 64;
-        for (int n0 = 0; n0 < 64; n0 += 16) {
-            uint32_t v[16];
-            if (n_chunks > 0) tmem_ld16(trow + (uint32_t)(kq * 128 + half * 64 + n0), v);
-            if (t >= P.T) continue;
-            const float *rv = stg + (size_t)row * kPitch + half * 64 + n0;
-            float a[16];
+    fence_async_proxy();                     // the staged block was written with ordinary stores; the copy reads it through the async proxy
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t partner = ((1u - kq) << 1) | rank;
+        bulk_copy_to_cta(map_to_cta(smem_u32(rcv), partner), snd, kBlockBytes, map_to_cta(smem_u32(&B->xbar), partner));
+    }
+    if (warp < kLoaderWarps) {
+        const bool got = mbar_wait_cluster(&B->xbar, 0, P.spin_limit);
+        if (!got && tid == 0 && P.status) atomicCAS(P.status, 0, SI_ERR_TIMEOUT);
+        if (ok && got) {
+            tc_fence_after();
+            const size_t o0 = (size_t)t * P.d_model + (size_t)ct * 256 + kq * 128 + half * 64;
+            for (int n0 = 0; n0 < 64; n0 += 16) {
+                uint32_t v[16];
+                if (n_chunks > 0) tmem_ld16(trow + (uint32_t)(kq * 128 + half * 64 + n0), v);
+                if (t >= P.T) continue;
+                const float *rv = rcv + (size_t)row * kPitch + half * 64 + n0;
+                float a[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float own = n_chunks > 0 ? __uint_as_float(v[j]) : 0.f;
-                a[j] = kq == 0 ? own + rv[j] : rv[j] + own;       // K half 0 first, whoever adds
+                for (int j = 0; j < 16; ++j) {
+                    const float own = n_chunks > 0 ? __uint_as_float(v[j]) : 0.f;
+                    a[j] = kq == 0 ? own + rv[j] : rv[j] + own;   // K half 0 first, whoever adds
+                }
+                down_store16(P, o0 + n0, a);
             }
-            down_store16(P, o0 + n0, a);
         }
     }
 }
@@ -644,7 +668,7 @@ si_pair_down_kernel(const __grid_constant__ GemmParams P, const __grid_constant_
         }
         pair_mma_loop(B, full, !run, n_chunks, P.nstage, P.spin_limit, rank, tmem, idesc, a0, b0, (uint32_t)stage_bytes, leader);
     }
-    if (KS == 2) down_epilogue_split(P, smem, ok, n_chunks, tmem, warp, lane, tok0, ct, kq, rank);
+    if (KS == 2) down_epilogue_split(P, smem, B, ok, n_chunks, tmem, warp, lane, tok0, ct, kq, rank);
     pair_teardown(tmem, ncols);
 }
 
@@ -716,11 +740,11 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
         // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs.  When tiles of 256 columns
         // would leave most SM pairs without one, two pairs share a tile of 256, half of K each (a cluster of four CTAs
         // that exchanges its partial accumulators through distributed shared memory) -- as long as that is one wave and
-        // K is long enough to pay for the exchange (measured at 512 tokens: level at 50 chunks of K, 6 % ahead at 72,
-        // 18 % at 121); tiles of 128 columns otherwise.
+        // K is long enough to pay for the exchange (measured at 512 tokens: 3 % ahead of the 128-column tiles at 50
+        // chunks of K, 18 % at 121); tiles of 128 columns otherwise.
         const int tiles256 = d % 256 == 0 ? (d / 256) * tok_pairs : 0;
         const bool fills = tiles256 > 0 && tiles256 * 2 >= s->num_sms * 3 / 4;
-        const bool split = tiles256 > 0 && !fills && tiles256 * 4 <= s->num_sms && P.nu_pad / kChunkK >= 64;
+        const bool split = tiles256 > 0 && !fills && tiles256 * 4 <= s->num_sms && P.nu_pad / kChunkK >= 32;
         const int n = fills || split ? 256 : 128;
         P.pair_n = n;
         const size_t stage = 128 * 128 + (size_t)64 * n;
