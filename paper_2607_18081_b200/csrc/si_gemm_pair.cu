@@ -152,13 +152,6 @@ __device__ __forceinline__ bool pair_issue_wide_stage(uint32_t d0, uint32_t d1, 
     return landed != 0;
 }
 
-// `bytes` (a multiple of 16) from this CTA's shared memory into the shared memory of another CTA of the cluster; completion
-// is counted in bytes on an mbarrier of that CTA (both addresses from map_to_cta)
-__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, const void *src_smem, uint32_t bytes, uint32_t bar_cluster) {
-    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst_cluster), "r"(smem_u32(src_smem)), "r"(bytes), "r"(bar_cluster) : "memory");
-}
-
 struct PairBars {
     // stage landed.  In the pair's first CTA one arrival more is expected: the second CTA's word that ITS half has landed
     uint64_t full_t[kPairMaxStages];     // ... tensor copies only (one arrival: the thread that starts them)

@@ -124,6 +124,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+// `bytes` (a multiple of 16) from this CTA's shared memory into the shared memory of another CTA of the cluster; completion
+// is counted in bytes on an mbarrier of that CTA (both addresses from map_to_cta)
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, const void *src_smem, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(smem_u32(src_smem)), "r"(bytes), "r"(bar_cluster) : "memory");
+}
+
 // ------------------------------------------------------------------------------- parameters
 struct GemmParams {
     const char *rec_base;          // records of the layer
