@@ -82,6 +82,16 @@ int si_debug_ffn_forward_waits(const si_store_t *store, int layer, const void *x
                                void *workspace, size_t ws_bytes, int32_t *status_dev, void *stream,
                                long long spin_limit, int withhold);
 
+/* Host logic only (no device is touched): the kernel shapes si_ffn_forward picks for a call with T tokens (T > 128) whose
+ * union has room for union_cap entries (a multiple of 128), on a device of num_sms SMs.
+ *   out[0], out[1] : gate/up tiles: neurons per sub-tile (128, 112 or 96) and sub-tiles per tile (1 or 2)
+ *   out[2]         : CTA pairs of the gate/up launch
+ *   out[3], out[4] : down tiles: output columns per pair tile (128 or 256) and pairs that share a tile, each with a
+ *                    part of K (1 or 2)
+ *   out[5]         : CTAs of the down launch
+ * SI_ERR_INVALID_ARG for T <= 128, d_model not a multiple of 128, union_cap not a positive multiple of 128. */
+int si_debug_pair_plan(int d_model, int union_cap, int T, int num_sms, int out[6]);
+
 /* si_ffn_forward_sharded for the ranks rank_base .. rank_base + n_here - 1 of a group that share this GPU, in ONE
  * launch (kernels of different ranks that wait on one another may not run as separate launches on one GPU): the
  * ranks' first kernels one after the other, then one cooperative launch of the finishing kernel over all of them.

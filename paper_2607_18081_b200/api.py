@@ -39,7 +39,7 @@ EXPORTS = [
     "si_debug_decode_stack_forward", "si_debug_decode_chain_forward", "si_debug_union_masks", "si_debug_ffn_forward_waits",
     "si_debug_read_bandwidth", "si_prefill_vote_workspace_bytes", "si_prefill_vote", "si_prefill_forward", "si_layer_range", "si_profile_accumulate", "si_profile_merge", "si_profile_rank",
     "si_loadset", "si_shard_count", "si_shard_lists", "si_shard_reduce", "si_ffn_forward_sharded",
-    "si_debug_ffn_forward_sharded_group",
+    "si_debug_ffn_forward_sharded_group", "si_debug_pair_plan",
 ]
 
 
@@ -83,6 +83,7 @@ def _load_library() -> ctypes.CDLL:
     lib.si_debug_union_masks.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp, vp, sz, vp]
     lib.si_debug_ffn_forward_waits.argtypes = lib.si_ffn_forward.argtypes + [ctypes.c_longlong, ci]
     lib.si_debug_read_bandwidth.argtypes = [vp, ctypes.c_size_t, vp, vp]
+    lib.si_debug_pair_plan.argtypes = [ci, ci, ci, ci, ctypes.POINTER(ctypes.c_int)]
     lib.si_prefill_vote_workspace_bytes.argtypes = [ci, ci, ci, psz]
     lib.si_prefill_vote.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, cu, vp, ci, vp, vp, vp, sz, vp]
     lib.si_profile_accumulate.argtypes = [vp, ci, ci, ci, vp, vp]
@@ -399,6 +400,14 @@ def si_debug_union_masks(handle, layer: int, T: int, idx, idx_offsets, k_fixed: 
                                      _dp(n_union_out), _dp(masks_out), _dp(workspace),
                                      workspace.numel() * workspace.element_size(), _stream(stream)),
            "si_debug_union_masks")
+
+
+def si_debug_pair_plan(d_model: int, union_cap: int, T: int, num_sms: int) -> dict:
+    """Kernel shapes of a call with more than 128 tokens (host logic only, no device needed)."""
+    out = (ctypes.c_int * 6)()
+    _check(_lib.si_debug_pair_plan(d_model, union_cap, T, num_sms, out), "si_debug_pair_plan")
+    return {"gateup_w": out[0], "gateup_sub": out[1], "gateup_pairs": out[2], "down_n": out[3], "down_ksplit": out[4],
+            "down_ctas": out[5]}
 
 
 def si_debug_ffn_forward_waits(handle, layer: int, x, T: int, idx, idx_offsets, k_fixed: int, y, flags: int,

@@ -3,6 +3,7 @@
 #include "si_common.cuh"
 #include "si_decode_persistent.cuh"
 #include "selectinfer_debug.h"
+#include "si_tc.cuh"
 
 si_ws_layout si_ws_carve(const si_store *s, int T_max, int k_max, int max_steps) {
     si_ws_layout w;
@@ -253,6 +254,16 @@ extern "C" int si_debug_ffn_forward_waits(const si_store_t *store, int layer, co
     if (ws_bytes < si_ws_carve(store, T, k_fixed, 1).total) return SI_ERR_NOMEM;
     return si_multi_token_launch(store, layer, x, T, idx, idx_offsets, k_fixed, y, y_dtype, flags, workspace, ws_bytes,
                                  status_dev, (cudaStream_t)stream, spin_limit, withhold);
+}
+
+extern "C" int si_debug_pair_plan(int d_model, int union_cap, int T, int num_sms, int out[6]) {
+    if (!out || T <= 128 || d_model <= 0 || d_model % 128 != 0 || union_cap <= 0 || union_cap % 128 != 0 || num_sms < 2)
+        return SI_ERR_INVALID_ARG;
+    si_pair_plan_t plan;
+    si_pair_plan(d_model, union_cap, T, num_sms, &plan);
+    out[0] = plan.gateup_w; out[1] = plan.gateup_sub; out[2] = plan.gateup_pairs;
+    out[3] = plan.down_n; out[4] = plan.down_ksplit; out[5] = plan.down_ctas;
+    return SI_OK;
 }
 
 extern "C" int si_debug_union_masks(const si_store_t *store, int layer, int T, const int32_t *idx,

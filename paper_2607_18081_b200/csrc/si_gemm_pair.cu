@@ -683,6 +683,37 @@ int stages_for(size_t stage_bytes) {
 
 }  // namespace
 
+// The kernel shapes of a call with T tokens (T > 128) whose union has room for nu_pad entries, on a device of num_sms
+// SMs.  Host logic only.
+//   gate/up: tiles of W = 128 or 96 neurons, or of two sub-tiles of 128 or 112: cost = waves of pair tiles over the SM
+//            pairs x the MMA time of a tile's chunk (4 MMAs of N = 2 W per sub-tile: 4 S W cycles, plus what a stage
+//            costs besides)
+//   down:    256 columns per pair halve the H traffic of a column, 128 give twice the pairs.  When tiles of 256 columns
+//            would leave most SM pairs without one, two pairs share a tile of 256, half of K each (a cluster of four
+//            CTAs that exchanges its partial accumulators through distributed shared memory) -- as long as that is one
+//            wave and K is long enough to pay for the exchange (measured at 512 tokens: 3 % ahead of the 128-column
+//            tiles at 50 chunks of K, 18 % at 121); tiles of 128 columns otherwise.
+void si_pair_plan(int d_model, int nu_pad, int T, int num_sms, si_pair_plan_t *plan) {
+    const int tok_pairs = (T + kPairTokens - 1) / kPairTokens;
+    const int slots = num_sms / 2;
+    static const struct { int w, sub; } shapes[] = {{128, 1}, {96, 1}, {128, 2}, {112, 2}};
+    long best_cost = -1;
+    for (int i = 0; i < 4; ++i) {
+        const int r = shapes[i].w * shapes[i].sub;
+        const int pairs = ((nu_pad + r - 1) / r) * tok_pairs;
+        const long cost = (long)((pairs + slots - 1) / slots) * (4 * r + 78);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost; plan->gateup_w = shapes[i].w; plan->gateup_sub = shapes[i].sub; plan->gateup_pairs = pairs;
+        }
+    }
+    const int tiles256 = d_model % 256 == 0 ? (d_model / 256) * tok_pairs : 0;
+    const bool fills = tiles256 > 0 && tiles256 * 2 >= num_sms * 3 / 4;
+    const bool split = tiles256 > 0 && !fills && tiles256 * 4 <= num_sms && nu_pad / kChunkK >= 32;
+    plan->down_n = fills || split ? 256 : 128;
+    plan->down_ksplit = split ? 2 : 1;
+    plan->down_ctas = split ? 4 * tiles256 : (plan->down_n == 256 ? 2 * tiles256 : 2 * (d_model / 128) * tok_pairs);
+}
+
 bool si_pair_path_applies(const si_store *s, int T) {
     return T > 128 && s->d_model % 128 == 0;
 }
@@ -691,25 +722,15 @@ bool si_pair_path_applies(const si_store *s, int T) {
 // h_buf has room for t_pad_alloc x nu_pad 16-bit values).
 int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, void *h_buf, size_t h_bytes, cudaStream_t stream) {
     const int d = P.d_model;
-    const int tok_pairs = (P.T + kPairTokens - 1) / kPairTokens;
     // H holds the tokens padded to 16 rows; a tile's rows past them are not written, and read as zero through the tensor map
     const int t_pad_alloc = (int)si_align_up((size_t)P.T, 16);
     if ((size_t)t_pad_alloc * P.nu_pad * 2 > h_bytes) return SI_ERR_NOMEM;
     P.t_pad_total = t_pad_alloc; P.n_tok = kPairTokens; P.n_split = 1;
     P.h = (const uint16_t *)h_buf; P.h_out = (uint16_t *)h_buf;
+    si_pair_plan_t plan;
+    si_pair_plan(d, P.nu_pad, P.T, s->num_sms, &plan);
     {
-        // tiles of W = 128 or 96 neurons, or of two sub-tiles of 128 or 112: cost = waves of pair tiles over the SM pairs x
-        // the MMA time of a tile's chunk (4 MMAs of N = 2 W per sub-tile: 4 S W cycles, plus what a stage costs besides)
-        const int slots = s->num_sms / 2;
-        struct Shape { int w, sub; } shapes[] = {{128, 1}, {96, 1}, {128, 2}, {112, 2}};
-        int best = 0; long best_cost = -1; int best_pairs = 0;
-        for (int i = 0; i < 4; ++i) {
-            const int r = shapes[i].w * shapes[i].sub;
-            const int pairs = ((P.nu_pad + r - 1) / r) * tok_pairs;
-            const long cost = (long)((pairs + slots - 1) / slots) * (4 * r + 78);
-            if (best_cost < 0 || cost < best_cost) { best = i; best_cost = cost; best_pairs = pairs; }
-        }
-        const int w = shapes[best].w, sub = shapes[best].sub;
+        const int w = plan.gateup_w, sub = plan.gateup_sub, best_pairs = plan.gateup_pairs;
         const size_t stage = 128 * 128 + (size_t)w * sub * 128;
         P.nstage = stages_for(stage);
         const size_t smem = (size_t)P.nstage * stage + sizeof(PairBars);
@@ -730,15 +751,8 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
 #undef SI_LAUNCH_GATEUP
     }
     {
-        // 256 columns per pair halve the H traffic of a column, 128 give twice the pairs.  When tiles of 256 columns
-        // would leave most SM pairs without one, two pairs share a tile of 256, half of K each (a cluster of four CTAs
-        // that exchanges its partial accumulators through distributed shared memory) -- as long as that is one wave and
-        // K is long enough to pay for the exchange (measured at 512 tokens: 3 % ahead of the 128-column tiles at 50
-        // chunks of K, 18 % at 121); tiles of 128 columns otherwise.
-        const int tiles256 = d % 256 == 0 ? (d / 256) * tok_pairs : 0;
-        const bool fills = tiles256 > 0 && tiles256 * 2 >= s->num_sms * 3 / 4;
-        const bool split = tiles256 > 0 && !fills && tiles256 * 4 <= s->num_sms && P.nu_pad / kChunkK >= 32;
-        const int n = fills || split ? 256 : 128;
+        const int n = plan.down_n;
+        const bool split = plan.down_ksplit == 2;
         P.pair_n = n;
         const size_t stage = 128 * 128 + (size_t)64 * n;
         P.nstage = stages_for(stage);
@@ -750,13 +764,13 @@ int si_pair_contractions_launch(const si_store *s, GemmParams P, int n_loaded, v
         if (rc) return rc;
         if (split) {
             SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 2>, 4 * tiles256, smem, stream, P, h_map, rec_map));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 2>, plan.down_ctas, smem, stream, P, h_map, rec_map));
         } else if (n == 256) {
             SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 1>, 2 * tiles256, smem, stream, P, h_map, rec_map));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<256, 1>, plan.down_ctas, smem, stream, P, h_map, rec_map));
         } else {
             SI_CUDA_TRY(cudaFuncSetAttribute(si_pair_down_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<128, 1>, 2 * (d / 128) * tok_pairs, smem, stream, P, h_map, rec_map));
+            SI_CUDA_TRY(launch_pair(si_pair_down_kernel<128, 1>, plan.down_ctas, smem, stream, P, h_map, rec_map));
         }
     }
     SI_CUDA_TRY(cudaGetLastError());

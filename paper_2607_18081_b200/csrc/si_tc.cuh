@@ -182,6 +182,13 @@ inline int make_tile_map(CUtensorMap *map, const void *base, size_t cols, size_t
 
 }  // namespace si_tc
 
+// Kernel shapes of a call with more than 128 tokens (see si_pair_plan in si_gemm_pair.cu)
+struct si_pair_plan_t {
+    int gateup_w, gateup_sub, gateup_pairs;   // neurons per sub-tile, sub-tiles per tile, CTA pairs launched
+    int down_n, down_ksplit, down_ctas;       // output columns per pair tile, pairs sharing a tile (K split), CTAs launched
+};
+void si_pair_plan(int d_model, int nu_pad, int T, int num_sms, si_pair_plan_t *plan);
+
 // Contractions of calls with more than 128 tokens on pairs of SMs (si_gemm_pair.cu)
 bool si_pair_path_applies(const si_store *s, int T);
 int si_pair_contractions_launch(const si_store *s, si_tc::GemmParams P, int n_loaded, void *h_buf, size_t h_bytes, cudaStream_t stream);

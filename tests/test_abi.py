@@ -4,6 +4,8 @@ import ctypes
 import os
 import re
 
+import pytest
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -104,3 +106,36 @@ def test_shard_entry_points_host_side():
     assert lib.si_shard_reduce(buf, 2, null, api.SI_BF16, 1, 64, buf, api.SI_F32, api.SI_FLAG_RESIDUAL, null) == \
         api.SI_ERR_INVALID_ARG                                                              # residual without x
     assert lib.si_shard_reduce(buf, 2, null, api.SI_F32, 1, 64, buf, api.SI_F32, 0, null) == api.SI_ERR_INVALID_ARG
+
+
+def test_kernel_shapes_of_calls_with_many_tokens():
+    """Host logic: which tile shapes a call with more than 128 tokens gets (gate/up: neurons per sub-tile, sub-tiles per
+    tile; down: columns per pair tile, K split), on a device of 148 SMs = 74 SM pairs.  The choice minimises waves of
+    pair tiles x the time of a tile's chunk."""
+    from paper_2607_18081_b200 import api
+    # config 4: 512 tokens, union of 3082 slots (room for 3200), d_model 4096.  Tiles of 128 neurons would be 25 x 2 = 50
+    # pairs, tiles of 96 are 34 x 2 = 68: still one wave, a quarter less work per pair.  Down: 16 x 2 tiles of 256
+    # columns would use 64 SMs, so two pairs share a tile, half of K each: 32 x 4 = 128 CTAs.
+    p = api.si_debug_pair_plan(4096, 3200, 512, 148)
+    assert (p["gateup_w"], p["gateup_sub"], p["gateup_pairs"]) == (96, 1, 68)
+    assert (p["down_n"], p["down_ksplit"], p["down_ctas"]) == (256, 2, 128)
+    # all 7705 loaded neurons (room for 7808): 122 tiles of 128 would be two waves; 35 x 2 = 70 tiles of 2 x 112 are one
+    p = api.si_debug_pair_plan(4096, 7808, 512, 148)
+    assert (p["gateup_w"], p["gateup_sub"], p["gateup_pairs"]) == (112, 2, 70)
+    assert (p["down_n"], p["down_ksplit"]) == (256, 2)
+    # a union of 4608 slots is exactly 36 x 2 = 72 tiles of 128: one full wave, nothing to gain from narrower tiles
+    p = api.si_debug_pair_plan(4096, 4608, 512, 148)
+    assert (p["gateup_w"], p["gateup_sub"], p["gateup_pairs"]) == (128, 1, 72)
+    # 2048 tokens: 8 token tiles x 16 column tiles of 256 fill the machine without a K split
+    p = api.si_debug_pair_plan(4096, 3200, 2048, 148)
+    assert (p["down_n"], p["down_ksplit"], p["down_ctas"]) == (256, 1, 256)
+    # a short K (room for 1024 slots: 16 chunks) does not pay for the exchange of a K split: tiles of 128 columns
+    p = api.si_debug_pair_plan(4096, 1024, 512, 148)
+    assert (p["down_n"], p["down_ksplit"], p["down_ctas"]) == (128, 1, 128)
+    # a hidden size that is no multiple of 256 (640) has 128-column tiles only
+    p = api.si_debug_pair_plan(640, 768, 200, 148)
+    assert (p["down_n"], p["down_ksplit"], p["down_ctas"]) == (128, 1, 10)
+    for bad in ((4096, 3200, 128, 148), (4000, 3200, 512, 148), (4096, 3000, 512, 148), (4096, 0, 512, 148)):
+        with pytest.raises(api.SelectInferError) as e:
+            api.si_debug_pair_plan(*bad)
+        assert e.value.status == api.SI_ERR_INVALID_ARG
