@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of si_decode_persistent_kernel per (token, layer) step of
 # the config-2 shape: an ncu capture of an 8-layer x 32-token launch (256 steps) read 9.6434e9 and wrote
 # 0.2278e9 bytes; traffic grows in proportion to the steps (every step reads its own records once)
-NCU_DRAM_BYTES_PER_C2_STEP = (9.3513e9 + 0.0727e9) / 256
+NCU_DRAM_BYTES_PER_C2_STEP = (9.6434e9 + 0.2278e9) / 256
 FALLBACK_HBM_GBS = 6650.0
 
 
