@@ -9,10 +9,9 @@ token's active list (one persistent launch through the C ABI).  The store is bui
 the loader before timing.  Metric: selective-FFN decode tokens/s at batch 1.
 
 Prints ONE JSON line (rank 0).  The headline is configuration 2 with the (token, layer) steps
-independent of one another (every step's input given up front): the library's default schedule, in
-which the SMs work in four groups that each take every fourth step.  Beside it, in the same line:
-`chained` -- the same launch size with every layer reading the output of the layer before it, as inside
-a decoder; `steps_one_group` -- every SM on every step, in order; and `configs` -- the other
+independent of one another (every step's input given up front) and worked through in order.
+Beside it, in the same line: `chained` -- the same launch size with every layer reading the
+output of the layer before it, as inside a decoder; `steps_any_order`; and `configs` -- the other
 four configurations (c1 latency, c3 batch sizes, c4 prefill, the sixteen c5 cells), each measured
 on a stated reduced number of layers whose weights still exceed L2.
 
@@ -370,14 +369,14 @@ def extra_configs(api, torch, args, device, peaks, peak_kind):
                 idx = torch.from_numpy(lists.reshape(n_steps, k)).cuda()
                 ws = store.workspace(1, k, n_steps)
                 ms = device_ms(torch, lambda: api.si_decode_stack_forward(store.handle, n_steps, None, x, idx, None, k, y, 0, ws, status), 5)
-                ms_one = device_ms(torch, lambda: api.si_debug_decode_stack_forward(store.handle, n_steps, None, x, idx, None, k, y, 0, ws,
-                                                                                    status, step_groups=1), 5)
+                ms_any = device_ms(torch, lambda: api.si_decode_stack_forward(store.handle, n_steps, None, x, idx, None, k, y,
+                                                                              api.SI_FLAG_STEPS_ANY_ORDER, ws, status), 5)
                 ms_ch = device_ms(torch, lambda: api.si_decode_chain_forward(store.handle, n_steps, None, n_layers, heads, idx, None, k, y,
                                                                              None, CHAIN_EPS, api.SI_FLAG_PRENORM | api.SI_FLAG_RESIDUAL,
                                                                              ws, status), 3)
                 bytes_step = k * cfg.record_bytes
                 cell = {"loaded_pct": lp, "active_pct": ap, "k": k}
-                for name, m in (("default", ms), ("one_group", ms_one), ("chained", ms_ch)):
+                for name, m in (("in_order", ms), ("any_order", ms_any), ("chained", ms_ch)):
                     us = m * 1e3 / n_steps
                     cell[name] = {"us_per_step": us, "gbs": bytes_step / us / 1e3, "frac_of_nominal_8TBs": bytes_step / us / 1e3 / NOMINAL_HBM_GBS,
                                   "tokens_per_s_32_layers": 1e6 / (us * 32)}
@@ -470,11 +469,11 @@ def run_ours(args):
     def step_device():
         api.si_decode_stack_forward(store.handle, n_steps, None, x_dev, idx_dev, None, k, y_dev, flags, ws, status)
 
-    # the same launch with every SM on every step, the steps in their order (the schedule for long lists before
-    # four step groups became the default at every length): reported beside the headline
-    def step_device_one_group():
-        api.si_debug_decode_stack_forward(store.handle, n_steps, None, x_dev, idx_dev, None, k, y_dev, flags, ws, status,
-                                          step_groups=1)
+    # the same launch with the caller's statement that the steps are independent (every step's x is an input),
+    # which lets the SMs work in step groups: reported beside the headline, which keeps the steps in order
+    def step_device_any_order():
+        api.si_decode_stack_forward(store.handle, n_steps, None, x_dev, idx_dev, None, k, y_dev,
+                                    flags | api.SI_FLAG_STEPS_ANY_ORDER, ws, status)
 
     # End to end: the step's x and lists start in pinned host memory and y ends there.  The tokens go
     # through in chunks so that the copies of one chunk run beside the decode launch of another
@@ -556,7 +555,7 @@ def run_ours(args):
     total_ms, per_step_ms, (t0, t1) = timed(step_device, args.steps, max(args.warmup, 3))
     clocks = sampler.stop(t0, t1) if sampler else None
     side_steps = max(3, min(args.steps, 20))               # the figures beside the headline need no long region
-    one_ms, one_per, _ = timed(step_device_one_group, side_steps, 3)
+    any_ms, any_per, _ = timed(step_device_any_order, side_steps, 3)
     e2e_ms, _, _ = timed(step_e2e, args.steps, max(args.warmup, 3))
     if int(status.item()) != 0:
         raise SystemExit(f"device status {status.item()}: {api.strerror(int(status.item()))}")
@@ -643,20 +642,19 @@ def run_ours(args):
                                       if (cfg.name == "c2" and not args.simple) else None))},
             "load_seconds": load_s,
         }
-        out["config"]["steps"] = ("independent: every (token, layer) step's input is given up front; the SMs work in four "
-                                  "groups that each take every fourth step (the library's default schedule)")
+        out["config"]["steps"] = "independent: every (token, layer) step's input is given up front; worked through in order"
         if clocks and clocks.get("sm_mhz"):
             out["ms_per_step_x_sm_mhz"] = total_ms / args.steps * clocks["sm_mhz"]       # comparable across GPUs that clock differently
         if chained is not None:
             out["chained"] = chained
-        one_launch_ms = statistics.mean(one_per)
-        out["steps_one_group"] = {
-            "value": replicas.aggregate_throughput(tokens * side_steps, world, one_ms), "unit": UNIT,
-            "achieved_gbs": alg_bytes / (one_launch_ms * 1e-3) / 1e9,
-            "frac": alg_bytes / (one_launch_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "frac_of_read_only_kernel": alg_bytes / (one_launch_ms * 1e-3) / 1e9 / read_ceiling,
-            "note": "same launch with every SM on every step, the steps in their order (si_debug_decode_stack_forward, "
-                    "step_groups = 1): a step's fixed work is then paid by all 148 SMs instead of 37"}
+        any_launch_ms = statistics.mean(any_per)
+        out["steps_any_order"] = {
+            "value": replicas.aggregate_throughput(tokens * side_steps, world, any_ms), "unit": UNIT,
+            "achieved_gbs": alg_bytes / (any_launch_ms * 1e-3) / 1e9,
+            "frac": alg_bytes / (any_launch_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "frac_of_read_only_kernel": alg_bytes / (any_launch_ms * 1e-3) / 1e9 / read_ceiling,
+            "note": "same launch with SI_FLAG_STEPS_ANY_ORDER: the SMs work in four groups that each take every "
+                    "fourth step; not the headline, which keeps every SM on the steps in their order"}
         if cpu_tokens:
             # parity spot check of the timed configuration against the oracle samples
             errs = []

@@ -81,9 +81,9 @@ enum {
     SI_FLAG_LIST_PER_LAYER = 64u, /* si_decode_stack_forward, fixed-length lists only: idx holds ONE list per layer
                                     ([n_layers, k_fixed]) and every step uses the list of its layer -- the paper's
                                     decode, where the set chosen during prefill stays fixed for the prompt */
-    SI_FLAG_STEPS_ANY_ORDER = 128u, /* si_decode_stack_forward: accepted and without effect -- the SMs work in up to four
-                                    groups that each take every fourth step at every list length by default (the flag
-                                    asked for that when only short lists were spread this way) */
+    SI_FLAG_STEPS_ANY_ORDER = 128u, /* si_decode_stack_forward: the SMs work in up to four groups that each take every
+                                    fourth step, whatever the lists' length (without the flag: one group for long
+                                    lists, two or four for short ones, see there) */
     SI_FLAG_SIMPLE_KERNELS = 256u, /* decode: one plain-load kernel pair per step instead of the
                                      persistent bulk-copy kernel (kept for cross-checking) */
     SI_FLAG_PRENORM = 512u       /* si_decode_chain_forward: the FFN sees its input scaled to unit root mean
@@ -192,13 +192,14 @@ int si_layer_forward(const si_store_t *store, int layer, const void *x, int T, c
  * persistent launch, step s using layer layers[s] (HOST int32 [n_steps], or NULL for
  * s mod n_layers).  x, y: device [n_steps, d_model]; idx: device [n_steps, k_fixed]
  * (or CSR over n_steps lists).  Every step's x is an input of the call, so the steps do not depend
- * on one another (si_decode_chain_forward is the call for steps that do).  The weight stream of
- * later steps is prefetched while earlier steps finish, and a step's sum over the SMs completes a few
- * steps behind the stream.  The schedule is the library's: the SMs
- * work in up to four groups that each take every fourth step -- within a group in the steps' order --,
- * which divides the fixed work of a step by the number of groups and is ahead of every SM working on
- * every step at every list length that was measured (215 to 7168 entries).  All of y is complete when
- * the call's work on the stream is.
+ * on one another (si_decode_chain_forward is the call for steps that do).  Every SM works through
+ * its steps in their order; the weight stream of later steps is prefetched while earlier steps
+ * finish, and a step's sum over the SMs completes a few steps behind the stream.  A step is spread
+ * over as many SMs as its list keeps busy: all of them for lists of more than 1100 entries (k_fixed),
+ * half of them up to 1100, a quarter up to 600 -- the SMs then work in two or four groups that each
+ * take every second or fourth step, which divides the fixed work of a step by the number of groups.
+ * SI_FLAG_STEPS_ANY_ORDER asks for four groups whatever the length.  All of y is complete when the
+ * call's work on the stream is.
  * Results equal n_steps si_ffn_forward(T = 1) calls up to fp32 summation order (the split of
  * a list over SMs depends on the step's position in the call); each is run-to-run bit-stable.
  * With SI_FLAG_LIST_PER_LAYER (fixed-length lists only) idx is [n_layers, k_fixed] and a step

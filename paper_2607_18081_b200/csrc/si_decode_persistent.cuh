@@ -1676,16 +1676,17 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     // Step groups: the SMs are split into groups that each take every n-th step on their own (launches of at
     // least two steps per group; a launch that uses fewer CTAs than SMs keeps one group).  The steps of a
     // stack call are independent of one another by its contract (every step's input is given), so how many
-    // SMs share a step is a question of throughput alone: a step's fixed work -- the input row into both
+    // SMs share a step is a question of what keeps them busy: a step's fixed work -- the input row into both
     // rings, two hand-overs, a partial row per CTA and its share of the cross-SM sum -- costs about 3.4 us on all
-    // SMs whatever the list's length, about 1.8 us on half and 1.0 us on a quarter of them.  Four groups are
-    // ahead at every list length that was measured (215 to 7168 entries: by 5 % at the long end, 15 % at 1541,
-    // three times at the short end), so four it is; within a group every SM works through the group's steps in
-    // their order.  (SI_FLAG_STEPS_ANY_ORDER asked for this when shorter lists only were spread by default.)
+    // SMs whatever the list's length, about 1.8 us on half and 1.0 us on a quarter of them.  Lists of up to 600
+    // entries (at most four records per SM otherwise) therefore go to a quarter of the SMs, lists of up to 1100
+    // to half, longer ones to all SMs, every SM working through its steps in their order; a caller who passes
+    // SI_FLAG_STEPS_ANY_ORDER gets four groups whatever the length.
     int ng = 1;
     if (G == s->num_sms && ex->chain_len == 0) {
         const int forced = ex->step_groups;   // diagnostics: force a group count
-        ng = forced ? forced : si_persist::pick_groups(s->num_sms);
+        const int by_length = k_total <= 600 ? 4 : (k_total <= 1100 ? 2 : 1);
+        ng = forced ? forced : ((flags & SI_FLAG_STEPS_ANY_ORDER) ? si_persist::pick_groups(s->num_sms) : by_length);
         while (ng > 1 && (s->num_sms % ng != 0 || n_steps < 2 * ng ||
                           (s->d_model / 4 + s->num_sms / ng - 1) / (s->num_sms / ng) > si_persist::kMaxGroups))
             ng >>= 1;
