@@ -246,7 +246,7 @@ __device__ __forceinline__ bool hint_wait_cta(const unsigned *ctr, unsigned targ
         mbar_arrive(bar);
         return true;
     }
-    return mbar_wait_bounded(bar, parity, cta_abort, limit);
+    return mbar_spin_bounded(bar, parity, cta_abort, limit);
 }
 __device__ __forceinline__ void red_add_relaxed_gpu(unsigned *p, unsigned v) {
     asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -772,22 +772,31 @@ __device__ __forceinline__ void split_slice_loader(const Params &P, uint8_t *sme
         if (cols.ng > 0) {
             const char *rec = P.store_base + P.rec_off[l.layer] + (size_t)d * 4 + (size_t)cols.g0 * 16;   // down row, this CTA's columns
             const int n_loaded = P.n_loaded[l.layer];
-            // all of this lane's list entries in one round of loads (a load per copy would put a trip to L2
-            // in front of every copy), then the copies
+            // A warp takes 32 list entries at a time: one coalesced load of their slots (all of a lane's loads in one
+            // round first: a load per copy would put a trip to L2 in front of every copy), then four copy
+            // instructions in which four neighbouring lanes fetch the (up to) 64 bytes of one record's slice, so
+            // that an instruction asks for eight whole pieces instead of 32 scattered 16-byte ones.
             constexpr int kPer = kSplitKCapMax / (32 * kSplitLoaderWarps);
             int slot[kPer];
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
-                const int p = lw * 32 + lane + j * 32 * kSplitLoaderWarps;
+                const int p = (j * kSplitLoaderWarps + lw) * 32 + lane;
                 slot[j] = p < l.k ? (p < P.n_static ? p : __ldg(P.idx + l.base + (p - P.n_static))) : -1;
             }
+            const int g = lane & 3, sub = lane >> 2;
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
-                const int p = lw * 32 + lane + j * 32 * kSplitLoaderWarps;
-                if (p < l.k) {
-                    const char *src = rec + (size_t)((slot[j] >= 0 && slot[j] < n_loaded) ? slot[j] : 0) * ((size_t)d * 6);   // (a bad slot's h is zero)
-                    uint8_t *dst = sbuf + (size_t)p * 64;
-                    for (int g = 0; g < cols.ng; ++g) cp_async16(dst + g * 16, src + g * 16);
+                const int p0 = (j * kSplitLoaderWarps + lw) * 32;
+                if (p0 < l.k) {                              // (uniform over the warp)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const int sl = __shfl_sync(0xFFFFFFFFu, slot[j], r * 8 + sub);
+                        const int p = p0 + r * 8 + sub;
+                        if (p < l.k && g < cols.ng && !(P.stream_only & 16)) {
+                            const char *src = rec + (size_t)((sl >= 0 && sl < n_loaded) ? sl : 0) * ((size_t)d * 6);   // (a bad slot's h is zero)
+                            cp_async16(sbuf + (size_t)p * 64 + g * 16, src + g * 16);
+                        }
+                    }
                 }
             }
         }
@@ -832,7 +841,7 @@ __device__ __noinline__ bool split_step_gateup(const Params &P, uint8_t *smem, i
     uint2 *hrow = P.ll_h + (size_t)(step & 1) * P.k_cap;
     const bool noarith = (P.stream_only & 1) != 0;
     for (int i = 0; i < geo.cnt; ++i) {
-        fail |= !mbar_wait_bounded(&sfull[st], ph, cta_abort, wait_limit);
+        fail |= !mbar_spin_bounded(&sfull[st], ph, cta_abort, wait_limit);
         const bool okr = !fail && smeta[st] != 0 && !noarith;   // else: h = 0
         const uint4 *rr = reinterpret_cast<const uint4 *>(sring + (size_t)st * P.stage_bytes);
         uint4 ga[NCH], up[NCH];
@@ -869,7 +878,7 @@ __device__ __noinline__ bool split_step_gateup(const Params &P, uint8_t *smem, i
         fail = set_barrier_or<kSetThreads>(q, fail);       // also orders the partials for the whole set
         recs ^= 1u;
         if (fail) return true;
-        if (t == 0) {
+        if (t == ((i & (kSetWarps - 1)) << 5)) {             // the set's warps take turns: the sums of a record are off the other records' path
             float gs = 0.f, us = 0.f;
             const float4 *pp = reinterpret_cast<const float4 *>(sm->setpart[q][buf]);
 #pragma unroll
@@ -1205,7 +1214,9 @@ si_decode_persistent_kernel(const __grid_constant__ Params P) {
                 if (mbar_test_wait(&empty[st], iph ^ 1)) {
                     const uint4 dsc = sm->desc[iq][n % kDescRing];
                     meta[st] = (int)dsc.w;
-                    if (dsc.z != 0) {
+                    if (dsc.z != 0 && (P.stream_only & 8)) {
+                        mbar_arrive(&full[st]);
+                    } else if (dsc.z != 0) {
                         mbar_arrive_expect_tx(&full[st], dsc.z);
                         bulk_g2s(ring + (size_t)st * P.stage_bytes,
                                  (const void *)(((unsigned long long)dsc.y << 32) | dsc.x), dsc.z, &full[st], policy);
@@ -1663,7 +1674,7 @@ inline int si_decode_persistent_launch(const si_store *s, int n_steps, const int
     P.partial = (float *)(wsb + ws.partial_off);
     P.status = status_dev;
     P.prof = ex->profile;
-    P.stream_only = ex->skip_mask & 7;
+    P.stream_only = ex->skip_mask & 31;
     if (ex->ring_stages > 0 && !wide && 2 * ex->ring_stages <= P.nstage) P.nstage = 2 * ex->ring_stages;   // diagnostics: shallower rings
     P.wait_cycles = ex->wait_cycles > 0 ? ex->wait_cycles : si_persist::kWaitCycles;
     P.withhold = ex->withhold;
