@@ -237,8 +237,20 @@ def measure_chained(api, torch, store, cfg, heads_dev, idx_dev, ws, status, peak
     ms = device_ms(torch, launch, reps)
     us_step = ms * 1e3 / n_steps
     gbs = k * cfg.record_bytes / us_step / 1e3
+
+    # the same launch through the diagnostics call with no weight copied at all (skip_mask bits 3 and 4: neither the
+    # records nor the down slices; its y is meaningless and goes to a buffer of its own): what the exchanges between
+    # the SMs and the arithmetic of the dependent steps cost by themselves
+    y_floor = torch.empty_like(y)
+
+    def launch_no_weights():
+        api.si_debug_decode_chain_forward(store.handle, n_steps, None, L, heads_dev, idx_dev, None, k, y_floor, None,
+                                          CHAIN_EPS, flags, ws, status, skip_mask=24)
+
+    ms_floor = device_ms(torch, launch_no_weights, max(2, reps // 2))
     return {"value": tokens / (ms * 1e-3), "unit": UNIT, "us_per_step": us_step, "achieved_gbs": gbs,
             "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "launch_ms": ms,
+            "us_per_step_without_weight_traffic": ms_floor * 1e3 / n_steps,
             "note": "si_decode_chain_forward: one chain per token through all layers, each layer's input = the rounded "
                     "output of the layer before it (pre-norm + residual); no arithmetic of a step starts before the "
                     "step before it is complete on every SM, only the weight stream runs ahead"}, y

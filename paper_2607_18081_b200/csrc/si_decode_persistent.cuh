@@ -451,7 +451,7 @@ __device__ __forceinline__ bool chain_input(const Params &P, Smem *sm, int step,
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
         if (lane == 0) sm->setpart[q][recs & 1][sw].x = ss;
     }
-    fail = set_barrier_or<kSetThreads>(q, fail);          // one verdict for the set (and the warp sums are in place)
+    fail = set_barrier_or<kSetThreads>(q, fail);          // one answer for the whole set (and the warp sums are in place)
     if (fail) return true;
     if (P.prenorm) {
         float ss = 0.f;

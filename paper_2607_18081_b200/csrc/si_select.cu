@@ -309,7 +309,7 @@ si_select_kernel(const float *__restrict__ scores, int n, int row_stride, int mo
         }
     };
     if (per <= 32) {
-        // the range's verdicts fit two 32-bit masks: classify once, then walk the set bits
+        // the range's answers fit two 32-bit masks: classify once, then walk the set bits
         uint32_t gm = 0, em = 0;
         for (int i = lo; i < hi; ++i) {
             bool gt, eq;
