@@ -170,6 +170,27 @@ def test_c2_full_size_chained_sampled(api):
     assert st == 0 and torch.equal(y, y2)
 
 
+def test_chained_launch_without_weight_copies_ends_cleanly_and_the_next_call_is_correct(api):
+    """The diagnostics launch that copies neither records nor down slices (skip_mask bits 3 and 4: the
+    bench times it for the cost of the exchanges alone): it must end with status 0 whatever garbage it
+    computes, and an ordinary launch on the same workspace right after it must be correct."""
+    cfg = wl.CONFIGS["c2"]
+    m = LoadedModel(cfg, n_layers=2)
+    L, tokens, k = 2, 4, cfg.k_active
+    n_steps = L * tokens
+    heads = wl.x_tokens(cfg, 0, tokens, first_token=300)
+    lists = np.stack([wl.zipf_lists(cfg, s % L, 1, first_token=300 + s // L)[0] for s in range(n_steps)])
+    hd, idx = to_dev(heads, cfg.dtype), torch.from_numpy(lists).cuda()
+    flags = api.SI_FLAG_RESIDUAL | api.SI_FLAG_PRENORM
+    for mask in (8, 16, 24):
+        _, _, st = _run_chain(api, m, n_steps, L, hd, idx, None, k, flags, skip_mask=mask, chain_form=2)
+        assert st == 0, (mask, api.strerror(st))
+    y, xn, st = _run_chain(api, m, n_steps, L, hd, idx, None, k, flags, want_xn=True)
+    assert st == 0, api.strerror(st)
+    _check_steps_fed_with_device_inputs(api, m, y, xn, heads, [lists[s] for s in range(n_steps)], L, flags,
+                                        range(n_steps), lambda s: s % L)
+
+
 def test_chain_argument_errors(api):
     cfg = wl.CONFIGS["c1"]
     m = LoadedModel(cfg)
