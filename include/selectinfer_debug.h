@@ -17,11 +17,11 @@ extern "C" {
 typedef struct si_debug_decode_opts {
     int skip_mask;         /* bit 0: leave out the arithmetic; bit 1: the loads of the cross-SM sum; bit 2: the
                               cross-SM exchange altogether.  y is then meaningless; timing such a launch gives
-                              the practical ceiling of the record stream on the same lists.  Chained calls in
-                              the split form also take bit 3: ring stages are handed to the consumers without
-                              their record being copied, and bit 4: the down slices are not copied -- with both
-                              set a launch reads no weights at all and its time is what the exchanges and the
-                              arithmetic of the dependent steps cost by themselves. */
+                              the practical ceiling of the record stream on the same lists.  Bit 3: ring stages
+                              are handed to the consumers without their record being copied; bit 4 (chained
+                              calls in the split form): the down slices are not copied -- with both set a
+                              chained launch reads no weights at all and its time is what the exchanges and
+                              the arithmetic of the dependent steps cost by themselves. */
     int ring_stages;       /* ring stages per consumer set (0 = as many as fit); results stay correct */
     int step_groups;       /* step groups the SMs are split into, whatever the flags say (0 = the library's
                               choice: one, or up to four with SI_FLAG_STEPS_ANY_ORDER); results stay correct */
